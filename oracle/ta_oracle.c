@@ -1,0 +1,240 @@
+/*
+ * Tensorized-attention CPU oracle (fp64).  TEST INFRASTRUCTURE ONLY.
+ *
+ * A plain, slow, step-by-step implementation of the paper's Algorithm 1
+ * ("Tensorized attention forward") for ONE attention head, plus the reverse-mode
+ * derivative of exactly that recurrence.  Nothing here is blocked, fused or
+ * reordered beyond what the algorithm states; the only parallelism is an OpenMP
+ * loop over the independent mode-i vectors ("segments") of one hop.
+ *
+ * This file shares no code with the CUDA path and is never called by it.
+ *
+ * Notation (Section 3.1 / 3.2 of the paper): the N tokens of a head are viewed,
+ * by row-major reshape, as a tensor n_1 x ... x n_m (dims[0] = n_1 is the
+ * slowest-varying coordinate).  Mode-i flattening (Eq. 4) batches the
+ * N / n_i vectors obtained by fixing every coordinate except the i-th; the
+ * tokens of one such vector are base + t * s_i, t = 0..n_i-1, with
+ * s_i = prod_{l>i} n_l.
+ *
+ * Forward (Algorithm 1):
+ *     O = V
+ *     for i = 0 .. m-1:                      (first dimension first)
+ *         A_i = softmax(Q_i K_i^T * scale  o  M_i)       (Eq. 4, row-wise softmax)
+ *         O_i = A_i O_i                                   (value update)
+ *     return vec(O)
+ * Q and K are the same un-updated projections in every hop; only O is carried.
+ * The mask M_i removes entries from the softmax (their weight is exactly 0);
+ * the causal M_i keeps key position u <= query position t along mode i.
+ */
+#include <math.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+/* Attention weights of one segment: P[t*n+u], rows sum to 1 (Eq. 1 / Eq. 4). */
+static void segment_weights(const double *Q, const double *K, long base, long stride,
+                            int n, int D, double scale, int causal, double *P)
+{
+    for (int t = 0; t < n; ++t) {
+        const double *qt = Q + (base + (long)t * stride) * D;
+        int nu = causal ? t + 1 : n;          /* visible keys of row t */
+        double mx = -INFINITY;
+        for (int u = 0; u < nu; ++u) {
+            const double *ku = K + (base + (long)u * stride) * D;
+            double s = 0.0;
+            for (int c = 0; c < D; ++c) s += qt[c] * ku[c];
+            s *= scale;
+            P[t * n + u] = s;
+            if (s > mx) mx = s;
+        }
+        double den = 0.0;
+        for (int u = 0; u < nu; ++u) {
+            double e = exp(P[t * n + u] - mx);
+            P[t * n + u] = e;
+            den += e;
+        }
+        for (int u = 0; u < nu; ++u) P[t * n + u] /= den;
+        for (int u = nu; u < n; ++u) P[t * n + u] = 0.0;   /* masked: weight exactly 0 */
+    }
+}
+
+/* stride s_i and the enumeration of segments of hop i:
+ * segment index g in [0, N/n_i) -> (outer, inner) -> base token outer*n_i*s_i + inner */
+static long hop_stride(const int *dims, int ndims, int i)
+{
+    long s = 1;
+    for (int l = i + 1; l < ndims; ++l) s *= dims[l];
+    return s;
+}
+
+/*
+ * One head, forward.  q,k,v: [N][D] fp64 (k,v are the head's KV head).
+ * out: [N][D].  xs (optional, may be NULL): [(ndims+1)][N][D], receives
+ * X_0 = V, X_1, ..., X_m = out (the value tensor after each hop), which the
+ * backward pass below needs.
+ * Returns 0, or -1 on bad arguments / allocation failure.
+ */
+int ta_oracle_forward_head(const double *q, const double *k, const double *v, double *out,
+                           long N, int D, const int *dims, int ndims, int causal,
+                           double scale, double *xs)
+{
+    if (!q || !k || !v || !out || !dims || ndims < 1 || N < 1 || D < 1) return -1;
+    long prod = 1;
+    for (int i = 0; i < ndims; ++i) { if (dims[i] < 1) return -1; prod *= dims[i]; }
+    if (prod != N) return -1;
+
+    size_t bytes = (size_t)N * D * sizeof(double);
+    double *cur = (double *)malloc(bytes), *nxt = (double *)malloc(bytes);
+    if (!cur || !nxt) { free(cur); free(nxt); return -1; }
+    memcpy(cur, v, bytes);                                  /* Initialize O = V */
+    if (xs) memcpy(xs, v, bytes);
+
+    int fail = 0;
+    for (int i = 0; i < ndims; ++i) {                       /* for i = 0 to m-1 */
+        const int n = dims[i];
+        const long s = hop_stride(dims, ndims, i);
+        const long nseg = N / n;
+        #pragma omp parallel
+        {
+            double *P = (double *)malloc((size_t)n * n * sizeof(double));
+            if (!P) {
+                #pragma omp atomic write
+                fail = 1;
+            }
+            #pragma omp for schedule(static)
+            for (long g = 0; g < nseg; ++g) {
+                if (!P) continue;
+                long outer = g / s, inner = g % s;
+                long base = outer * n * s + inner;
+                segment_weights(q, k, base, s, n, D, scale, causal, P);   /* A_i */
+                for (int t = 0; t < n; ++t) {               /* O_i = A_i O_i, folded back */
+                    double *o = nxt + (base + (long)t * s) * D;
+                    for (int c = 0; c < D; ++c) o[c] = 0.0;
+                    for (int u = 0; u < n; ++u) {
+                        double p = P[t * n + u];
+                        if (p == 0.0) continue;
+                        const double *x = cur + (base + (long)u * s) * D;
+                        for (int c = 0; c < D; ++c) o[c] += p * x[c];
+                    }
+                }
+            }
+            free(P);
+        }
+        if (fail) break;
+        double *tmp = cur; cur = nxt; nxt = tmp;
+        if (xs) memcpy(xs + (size_t)(i + 1) * N * D, cur, bytes);
+    }
+    if (!fail) memcpy(out, cur, bytes);
+    free(cur); free(nxt);
+    return fail ? -1 : 0;
+}
+
+/*
+ * One head, backward of the recurrence above (the paper gives no formula for it;
+ * this is the chain rule applied hop by hop, in reverse hop order).
+ * With X_0 = V, X_{i+1} = A_i X_i per segment, out = X_m and G_m = dout:
+ *     G_i  = A_i^T G_{i+1}                       gradient w.r.t. the hop's input
+ *     dP   = G_{i+1} X_i^T
+ *     dS   = A_i o (dP - rowsum(A_i o dP))       softmax derivative, masked entries 0
+ *     dQ  += scale * dS K        dK += scale * dS^T Q        (summed over hops)
+ *     dV   = G_0
+ * xs: [(ndims+1)][N][D] as written by ta_oracle_forward_head.
+ * dq, dk, dv: [N][D], overwritten (the caller sums dk, dv over a GQA group).
+ */
+int ta_oracle_backward_head(const double *q, const double *k, const double *xs,
+                            const double *dout, double *dq, double *dk, double *dv,
+                            long N, int D, const int *dims, int ndims, int causal,
+                            double scale)
+{
+    if (!q || !k || !xs || !dout || !dq || !dk || !dv || !dims || ndims < 1) return -1;
+    long prod = 1;
+    for (int i = 0; i < ndims; ++i) { if (dims[i] < 1) return -1; prod *= dims[i]; }
+    if (prod != N) return -1;
+
+    size_t bytes = (size_t)N * D * sizeof(double);
+    double *g = (double *)malloc(bytes), *gn = (double *)malloc(bytes);
+    if (!g || !gn) { free(g); free(gn); return -1; }
+    memcpy(g, dout, bytes);
+    memset(dq, 0, bytes);
+    memset(dk, 0, bytes);
+
+    int fail = 0;
+    for (int i = ndims - 1; i >= 0; --i) {
+        const int n = dims[i];
+        const long s = hop_stride(dims, ndims, i);
+        const long nseg = N / n;
+        const double *x = xs + (size_t)i * N * D;           /* X_i: the hop's input */
+        #pragma omp parallel
+        {
+            double *P = (double *)malloc((size_t)n * n * sizeof(double));
+            double *dS = (double *)malloc((size_t)n * n * sizeof(double));
+            if (!P || !dS) {
+                #pragma omp atomic write
+                fail = 1;
+            }
+            #pragma omp for schedule(static)
+            for (long sg = 0; sg < nseg; ++sg) {
+                if (!P || !dS) continue;
+                long outer = sg / s, inner = sg % s;
+                long base = outer * n * s + inner;
+                segment_weights(q, k, base, s, n, D, scale, causal, P);
+                /* dP[t][u] = <G_{i+1}[t], X_i[u]>, then dS */
+                for (int t = 0; t < n; ++t) {
+                    const double *gt = g + (base + (long)t * s) * D;
+                    double dot = 0.0;
+                    for (int u = 0; u < n; ++u) {
+                        const double *xu = x + (base + (long)u * s) * D;
+                        double a = 0.0;
+                        for (int c = 0; c < D; ++c) a += gt[c] * xu[c];
+                        dS[t * n + u] = a;
+                        dot += P[t * n + u] * a;
+                    }
+                    for (int u = 0; u < n; ++u)
+                        dS[t * n + u] = P[t * n + u] * (dS[t * n + u] - dot);
+                }
+                /* G_i = P^T G_{i+1};  dQ += scale dS K;  dK += scale dS^T Q
+                 * (segments are disjoint token sets, so no two threads touch the same row) */
+                for (int u = 0; u < n; ++u) {
+                    double *go = gn + (base + (long)u * s) * D;
+                    double *dku = dk + (base + (long)u * s) * D;
+                    for (int c = 0; c < D; ++c) go[c] = 0.0;
+                    for (int t = 0; t < n; ++t) {
+                        const double *gt = g + (base + (long)t * s) * D;
+                        const double *qt = q + (base + (long)t * s) * D;
+                        double p = P[t * n + u], ds = scale * dS[t * n + u];
+                        for (int c = 0; c < D; ++c) { go[c] += p * gt[c]; dku[c] += ds * qt[c]; }
+                    }
+                }
+                for (int t = 0; t < n; ++t) {
+                    double *dqt = dq + (base + (long)t * s) * D;
+                    for (int u = 0; u < n; ++u) {
+                        const double *ku = k + (base + (long)u * s) * D;
+                        double ds = scale * dS[t * n + u];
+                        for (int c = 0; c < D; ++c) dqt[c] += ds * ku[c];
+                    }
+                }
+            }
+            free(P); free(dS);
+        }
+        if (fail) break;
+        double *tmp = g; g = gn; gn = tmp;
+    }
+    if (!fail) memcpy(dv, g, bytes);
+    free(g); free(gn);
+    return fail ? -1 : 0;
+}
+
+int ta_oracle_num_threads(void)
+{
+    int n = 1;
+#ifdef _OPENMP
+    #pragma omp parallel
+    {
+        #pragma omp master
+        n = omp_get_num_threads();
+    }
+#endif
+    return n;
+}

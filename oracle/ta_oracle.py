@@ -1,0 +1,197 @@
+"""Tensorized-attention oracle: Python face of the fp64 C implementation of Algorithm 1,
+plus a brute-force dense (N x N) construction used to pin it.
+
+TEST INFRASTRUCTURE ONLY -- never imported by the CUDA package.
+
+Two independent routes to the same result live here:
+
+* ``forward`` / ``backward`` call ``ta_oracle.c`` (Algorithm 1, hop by hop, one head at a
+  time in fp64; backward = chain rule through that recurrence).
+* ``dense_hop_matrix`` / ``forward_dense`` write every hop as one N x N row-stochastic
+  matrix over all tokens (Eq. 3 unfolded: token j attends token k in hop i only if all their
+  tensor coordinates except the i-th agree) and multiply them out with numpy.  It is only
+  usable for tiny N and exists so that the C code is checked against something that does not
+  share its indexing.
+
+Parity pins (tests/test_oracle_pins.py): ndims=1 equals textbook attention (Eq. 1); size-1
+dimensions are no-ops; C route == dense route; separable (Kronecker) inputs give
+(U_1 (x) ... (x) U_m) V and, non-causal, ordinary full attention; constant V is a fixed point;
+Q=0 gives (prefix-)box means; causality probe; the row-major reshape pin of Section 4.4
+(one step on the first dimension of {32,32,32} is 1024 tokens); GQA equals explicit KV
+repetition; backward equals central finite differences and dV = A_eff^T dout.
+"""
+from __future__ import annotations
+
+import ctypes
+import math
+import os
+
+import numpy as np
+
+from . import build as _build
+
+_LIB = None
+
+
+def _lib():
+    global _LIB
+    if _LIB is None:
+        path = _build.build()
+        lib = ctypes.CDLL(path)
+        dp = ctypes.POINTER(ctypes.c_double)
+        ip = ctypes.POINTER(ctypes.c_int)
+        lib.ta_oracle_forward_head.restype = ctypes.c_int
+        lib.ta_oracle_forward_head.argtypes = [dp, dp, dp, dp, ctypes.c_long, ctypes.c_int, ip,
+                                               ctypes.c_int, ctypes.c_int, ctypes.c_double, dp]
+        lib.ta_oracle_backward_head.restype = ctypes.c_int
+        lib.ta_oracle_backward_head.argtypes = [dp, dp, dp, dp, dp, dp, dp, ctypes.c_long,
+                                                ctypes.c_int, ip, ctypes.c_int, ctypes.c_int,
+                                                ctypes.c_double]
+        lib.ta_oracle_num_threads.restype = ctypes.c_int
+        _LIB = lib
+    return _LIB
+
+
+def num_threads() -> int:
+    """Threads the OpenMP loops of the C oracle actually use."""
+    return int(_lib().ta_oracle_num_threads())
+
+
+def _dptr(a: np.ndarray):
+    return a.ctypes.data_as(ctypes.POINTER(ctypes.c_double))
+
+
+def _f64(a) -> np.ndarray:
+    return np.ascontiguousarray(np.asarray(a), dtype=np.float64)
+
+
+def _check(q, k, v, dims):
+    q = np.asarray(q)
+    k = np.asarray(k)
+    v = np.asarray(v)
+    if q.ndim != 4 or k.ndim != 4 or v.shape != k.shape:
+        raise ValueError("q:[B,H,N,D], k,v:[B,H_kv,N,D] expected")
+    B, H, N, D = q.shape
+    Hkv = k.shape[1]
+    if k.shape != (B, Hkv, N, D) or H % Hkv:
+        raise ValueError("inconsistent q/k/v shapes")
+    dims = [int(x) for x in dims]
+    if len(dims) < 1 or any(x < 1 for x in dims) or math.prod(dims) != N:
+        raise ValueError("prod(dims) must equal N")
+    return B, H, Hkv, N, D, dims
+
+
+def forward(q, k, v, dims, causal: bool, scale: float | None = None, heads=None,
+            return_xs: bool = False):
+    """Algorithm 1 for every (or the listed) head, fp64.
+
+    q: [B,H,N,D]; k, v: [B,H_kv,N,D] (any float dtype; converted head by head to fp64).
+    Query head h uses KV head h // (H/H_kv).  scale defaults to 1/sqrt(D) (Eq. 4).
+    heads: optional list of (b, h) pairs; then the result is [len(heads), N, D].
+    Returns out [B,H,N,D] fp64 (and, with return_xs, the list of per-head [m+1,N,D]
+    value tensors X_0=V ... X_m=out keyed like the output).
+    """
+    B, H, Hkv, N, D, dims = _check(q, k, v, dims)
+    g = H // Hkv
+    scale = 1.0 / math.sqrt(D) if scale is None else float(scale)
+    cdims = (ctypes.c_int * len(dims))(*dims)
+    pairs = [(b, h) for b in range(B) for h in range(H)] if heads is None else list(heads)
+    out = np.empty((len(pairs), N, D), dtype=np.float64)
+    xs_all = []
+    lib = _lib()
+    for idx, (b, h) in enumerate(pairs):
+        qh, kh, vh = _f64(q[b, h]), _f64(k[b, h // g]), _f64(v[b, h // g])
+        xs = np.empty((len(dims) + 1, N, D), dtype=np.float64) if return_xs else None
+        rc = lib.ta_oracle_forward_head(_dptr(qh), _dptr(kh), _dptr(vh), _dptr(out[idx]),
+                                        N, D, cdims, len(dims), int(bool(causal)), scale,
+                                        _dptr(xs) if return_xs else None)
+        if rc != 0:
+            raise RuntimeError("ta_oracle_forward_head failed")
+        if return_xs:
+            xs_all.append(xs)
+    if heads is None:
+        out = out.reshape(B, H, N, D)
+    return (out, xs_all) if return_xs else out
+
+
+def backward(dout, q, k, v, dims, causal: bool, scale: float | None = None):
+    """Gradients of sum(out * dout) w.r.t. q, k, v (fp64), GQA groups summed into dk, dv."""
+    B, H, Hkv, N, D, dims = _check(q, k, v, dims)
+    g = H // Hkv
+    scale = 1.0 / math.sqrt(D) if scale is None else float(scale)
+    cdims = (ctypes.c_int * len(dims))(*dims)
+    dq = np.zeros((B, H, N, D))
+    dk = np.zeros((B, Hkv, N, D))
+    dv = np.zeros((B, Hkv, N, D))
+    lib = _lib()
+    for b in range(B):
+        for h in range(H):
+            qh, kh, vh = _f64(q[b, h]), _f64(k[b, h // g]), _f64(v[b, h // g])
+            o = np.empty((N, D))
+            xs = np.empty((len(dims) + 1, N, D))
+            rc = lib.ta_oracle_forward_head(_dptr(qh), _dptr(kh), _dptr(vh), _dptr(o), N, D,
+                                            cdims, len(dims), int(bool(causal)), scale,
+                                            _dptr(xs))
+            if rc != 0:
+                raise RuntimeError("ta_oracle_forward_head failed")
+            dqh, dkh, dvh = np.empty((N, D)), np.empty((N, D)), np.empty((N, D))
+            rc = lib.ta_oracle_backward_head(_dptr(qh), _dptr(kh), _dptr(xs),
+                                             _dptr(_f64(dout[b, h])), _dptr(dqh), _dptr(dkh),
+                                             _dptr(dvh), N, D, cdims, len(dims),
+                                             int(bool(causal)), scale)
+            if rc != 0:
+                raise RuntimeError("ta_oracle_backward_head failed")
+            dq[b, h] = dqh
+            dk[b, h // g] += dkh
+            dv[b, h // g] += dvh
+    return dq, dk, dv
+
+
+# --------------------------------------------------------------------------------------
+# Brute force: every hop as a dense N x N matrix (tiny N only).  Independent of the C code.
+# --------------------------------------------------------------------------------------
+
+def dense_hop_matrix(qh, kh, dims, i: int, causal: bool, scale: float | None = None):
+    """The N x N matrix of hop i for one head (Eq. 3 written over flat token indices).
+
+    Entry [j, k] is the softmax weight of key token k for query token j; it is non-zero only
+    if j and k agree in every tensor coordinate except the i-th (and, causal, k_i <= j_i).
+    """
+    qh = np.asarray(qh, dtype=np.float64)
+    kh = np.asarray(kh, dtype=np.float64)
+    N, D = qh.shape
+    scale = 1.0 / math.sqrt(D) if scale is None else float(scale)
+    coords = np.stack(np.unravel_index(np.arange(N), tuple(dims)), axis=1)   # row-major
+    allowed = np.ones((N, N), dtype=bool)
+    for l in range(len(dims)):
+        cj, ck = coords[:, l][:, None], coords[:, l][None, :]
+        if l != i:
+            allowed &= cj == ck
+        elif causal:
+            allowed &= ck <= cj
+    s = (qh @ kh.T) * scale
+    s = np.where(allowed, s, -np.inf)
+    s = s - s.max(axis=1, keepdims=True)
+    e = np.exp(s)
+    return e / e.sum(axis=1, keepdims=True)
+
+
+def dense_effective_matrix(qh, kh, dims, causal: bool, scale: float | None = None):
+    """A_eff = A^_{m-1} ... A^_1 A^_0, the N x N map from V to the output of one head."""
+    N = np.asarray(qh).shape[0]
+    a = np.eye(N)
+    for i in range(len(dims)):
+        a = dense_hop_matrix(qh, kh, dims, i, causal, scale) @ a
+    return a
+
+
+def forward_dense(q, k, v, dims, causal: bool, scale: float | None = None):
+    """Brute-force forward for all heads via dense_effective_matrix (tiny N only)."""
+    B, H, Hkv, N, D, dims = _check(q, k, v, dims)
+    g = H // Hkv
+    out = np.empty((B, H, N, D))
+    for b in range(B):
+        for h in range(H):
+            a = dense_effective_matrix(q[b, h], k[b, h // g], dims, causal, scale)
+            out[b, h] = a @ np.asarray(v[b, h // g], dtype=np.float64)
+    return out
