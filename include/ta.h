@@ -1,0 +1,183 @@
+/*
+ * ta.h -- C ABI of the B200 tensorized-attention library (libta_b200.so).
+ *
+ * The library computes the forward (and backward) pass of Tensorized Attention
+ * (arxiv 2410.20926, Section 3.2, Algorithm 1) over already-projected q, k, v:
+ *
+ *     the N tokens of a head are viewed, by row-major reshape, as a tensor
+ *     n_1 x ... x n_m  (dims[0] = n_1 varies slowest; prod(dims) == N);
+ *     O = V;  for i = 0 .. m-1:  O <- A_i x_i O,  A_i = softmax(Q (x)_i K * scale o M_i)
+ *
+ * i.e. one "hop" per tensor dimension; hop i is a batch of N / n_i independent
+ * n_i x n_i softmax attentions over the tokens {base + t * s_i}, s_i = prod_{l>i} n_l
+ * (Eq. 3 / Eq. 4: mode-i flattening; done here by strided addressing, nothing is ever
+ * transposed in memory).  Q and K are the same in every hop; only O is carried.
+ * The causal mask M_i keeps key coordinate u <= query coordinate t along dimension i and
+ * removes the other entries from the softmax.  Query head h reads KV head h / (H / H_kv).
+ *
+ * Conventions common to every call
+ *   - Pointers named q/k/v/out/dout/dq/dk/dv/workspace are DEVICE pointers unless the
+ *     function name ends in _host.  `dims` is always a HOST pointer, read during the call.
+ *   - Layout: q, out, dout, dq: [B][H][N][D];  k, v, dk, dv: [B][H_kv][N][D];
+ *     contiguous, D innermost, token order = row-major order of the n_1 x ... x n_m tensor.
+ *     Base pointers must be 16-byte aligned.
+ *   - All buffers are owned by the caller.  `out` must not overlap q, k or v.
+ *   - Calls only enqueue work on `stream` (they do not synchronise) unless stated.
+ *   - Return value: TA_OK (0) or a negative TA_ERR_* code; nothing is thrown, printed or
+ *     aborted.  On an error return no kernel has been launched by that call.
+ *   - Hops with n_i == 1 are identities and are skipped.  ndims == 1 is ordinary attention.
+ *   - Kernels are built for sm_100a only; on another device the calls return TA_ERR_ARCH.
+ */
+#ifndef TA_B200_H
+#define TA_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Same type as the CUDA runtime's cudaStream_t. */
+typedef struct CUstream_st *ta_stream_t;
+
+enum {
+    TA_OK = 0,
+    TA_ERR_INVALID_ARG = -1, /* NULL pointer, non-positive size, ndims outside [1, TA_MAX_DIMS], dims[i] < 1 */
+    TA_ERR_SHAPE = -2,       /* prod(dims) != N, or H % H_kv != 0 */
+    TA_ERR_UNSUPPORTED = -3, /* D > TA_MAX_HEAD_DIM, unknown dtype or flag */
+    TA_ERR_ALIGNMENT = -4,   /* a base pointer is not 16-byte aligned */
+    TA_ERR_WORKSPACE = -5,   /* workspace missing or too small (see ta_workspace_bytes) */
+    TA_ERR_ARCH = -6,        /* current device is not compute capability 10.x */
+    TA_ERR_CUDA = -7,        /* a CUDA runtime / driver call failed (cudaGetLastError is preserved) */
+    TA_ERR_TIMEOUT = -8,     /* a bounded device-side wait gave up (seen by ta_device_status) */
+    TA_ERR_TOO_LARGE = -9    /* size beyond a documented fixed limit */
+};
+
+enum { TA_DTYPE_BF16 = 0, TA_DTYPE_F32 = 1 };
+
+enum {
+    TA_MAX_DIMS = 8,
+    TA_MAX_HEAD_DIM = 256
+};
+
+/* flags of ta_params.flags */
+enum {
+    TA_FLAG_NO_TENSOR_CORE = 1u << 0, /* run every hop on the generic CUDA-core kernel        */
+    TA_FLAG_NO_HOP_FUSION = 1u << 1,  /* one launch per hop, no cross-hop scheduling / fusion  */
+    TA_FLAG_SAVE_HOPS = 1u << 2       /* store hop inputs X_1..X_{m-1} in the workspace (for ta_backward) */
+};
+
+/* modes of ta_workspace_bytes */
+enum { TA_WS_FORWARD = 0, TA_WS_FORWARD_SAVE = 1, TA_WS_BACKWARD = 2 };
+
+/*
+ * Forward pass, bf16 storage (Algorithm 1; fp32 accumulation and fp32 softmax; the
+ * attention weights are rounded to bf16 before the value product, and the value tensor
+ * carried between hops is stored as bf16 in `out`).
+ *   q [B,H,N,D], k, v [B,H_kv,N,D]: device, bf16, read only.
+ *   out [B,H,N,D]: device, bf16, written (used as the in-place value tensor between hops).
+ *   dims: host array of ndims positive ints, prod == N.  causal: 0 or 1.
+ * Scale is 1/sqrt(D) in every hop (Eq. 4).
+ * Hops the tensor-core kernel covers (D in {64,128}, n_i <= 128) run in place in `out` and
+ * need no other memory.  Other hops (large n_i, other D) run on the generic kernel, which
+ * cannot update in place: for them the library uses an internal device scratch buffer of
+ * B*H*N*D elements that it allocates on first need and keeps (cudaMalloc: synchronous, so
+ * such a first call must not happen during stream capture).  ta_forward_ex takes a caller
+ * workspace instead.
+ */
+int ta_forward(const void *q, const void *k, const void *v, void *out,
+               int B, int H, int H_kv, int N, int D,
+               const int *dims, int ndims, int causal, ta_stream_t stream);
+
+/* Same, fp32 storage and fp32 arithmetic throughout (CUDA-core kernels; no tensor cores,
+ * because TF32 would not meet a 1e-4 tolerance). */
+int ta_forward_f32(const void *q, const void *k, const void *v, void *out,
+                   int B, int H, int H_kv, int N, int D,
+                   const int *dims, int ndims, int causal, ta_stream_t stream);
+
+/* Extended forward.  Zero-initialise the struct, set struct_bytes = sizeof(ta_params). */
+typedef struct ta_params {
+    size_t struct_bytes;   /* sizeof(ta_params) of the caller's header                       */
+    const void *q, *k, *v; /* device                                                         */
+    void *out;             /* device                                                         */
+    int B, H, H_kv, N, D;
+    const int *dims;       /* host                                                           */
+    int ndims;
+    int causal;
+    int dtype;             /* TA_DTYPE_*                                                     */
+    float softmax_scale;   /* 0 -> 1/sqrt(D)                                                 */
+    void *workspace;       /* device, 256-byte aligned, or NULL                              */
+    size_t workspace_bytes;
+    unsigned flags;        /* TA_FLAG_*                                                      */
+    int hop_begin;         /* run hops [hop_begin, hop_end) only; 0,0 -> all hops.  With      */
+    int hop_end;           /* hop_begin > 0 the value tensor is read from `out` (layout of q) */
+                           /* instead of v.                                                  */
+    ta_stream_t stream;
+} ta_params;
+
+/*
+ * ta_forward_ex: as ta_forward with every option explicit.  If `workspace` is non-NULL it
+ * is used for the generic kernel's second value buffer (and, with TA_FLAG_SAVE_HOPS, for
+ * the hop inputs X_1..X_{m-1}, [m-1][B][H][N][D] in the storage dtype, which ta_backward
+ * reads); it must hold ta_workspace_bytes(...) bytes or TA_ERR_WORKSPACE is returned.
+ */
+int ta_forward_ex(const ta_params *p);
+
+/*
+ * Backward pass of Algorithm 1 (the paper states no formula; this is the chain rule through
+ * the recurrence, hops in reverse order): given dout = d loss / d out it writes
+ *   dq [B,H,N,D], dk, dv [B,H_kv,N,D]   (storage dtype of the inputs; dk, dv summed over
+ *   the H/H_kv query heads of a group; dq, dk summed over hops).
+ * bf16 storage.  `workspace` (device) must hold ta_workspace_bytes(..., TA_WS_BACKWARD) bytes;
+ * the pass recomputes the attention weights and the hop inputs from q, k, v.
+ * `out` is not read (it may be NULL).
+ */
+int ta_backward(const void *dout, const void *q, const void *k, const void *v, const void *out,
+                void *dq, void *dk, void *dv,
+                int B, int H, int H_kv, int N, int D,
+                const int *dims, int ndims, int causal,
+                void *workspace, size_t workspace_bytes, ta_stream_t stream);
+
+/* Bytes of device workspace a call needs (0 if none); mode = TA_WS_*.  dtype = TA_DTYPE_*.
+ * Returns 0 for invalid shapes as well (the call itself reports the error). */
+size_t ta_workspace_bytes(int B, int H, int H_kv, int N, int D,
+                          const int *dims, int ndims, int dtype, int mode);
+
+/*
+ * Whole forward pass from HOST buffers (bf16 or fp32 by `dtype`): copies q, k, v to device
+ * staging memory owned by the library (allocated on first use, grown on demand, released by
+ * ta_release), runs ta_forward_ex there and copies `out` back, all on `stream`; the host
+ * buffers should be pinned for the copies to be asynchronous.  Returns after enqueueing; the
+ * caller synchronises `stream` before reading out_host.
+ */
+int ta_forward_host(const void *q_host, const void *k_host, const void *v_host, void *out_host,
+                    int B, int H, int H_kv, int N, int D,
+                    const int *dims, int ndims, int causal, int dtype, ta_stream_t stream);
+
+/*
+ * Text description of the launch plan the library would use for a problem (one line per hop:
+ * kernel path, segment length, stride, tile packing, source / destination buffer).  Pure
+ * host code: needs no GPU.  Writes at most `cap` bytes including the terminating NUL into
+ * `buf` (host) and returns TA_OK or the TA_ERR_* the forward call would return.
+ */
+int ta_plan_describe(int B, int H, int H_kv, int N, int D, const int *dims, int ndims,
+                     int causal, int dtype, unsigned flags, char *buf, size_t cap);
+
+/* Error word written by device code when a bounded wait expired (0 = none).  Synchronises
+ * the device; clears the word.  Returns TA_OK, TA_ERR_TIMEOUT or TA_ERR_CUDA. */
+int ta_device_status(void);
+
+/* Number of kernels this library has launched in the calling process (all streams). */
+unsigned long long ta_launch_count(void);
+
+/* Frees device memory the library holds (staging and scratch arenas).  Synchronises. */
+int ta_release(void);
+
+const char *ta_status_string(int status);
+int ta_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TA_B200_H */

@@ -1,0 +1,366 @@
+// C ABI of libta_b200.so: argument validation, the host-side hop planner and the launch loop
+// of Algorithm 1 (one hop per tensor dimension, first dimension first).
+#include <atomic>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <mutex>
+
+#include "ta_internal.h"
+
+namespace ta {
+
+static std::atomic<unsigned long long> g_launches{0};
+void count_launch(unsigned n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+int validate_shape(int B, int H, int H_kv, int N, int D, const int *dims, int ndims, int dtype) {
+    if (!dims || B <= 0 || H <= 0 || H_kv <= 0 || N <= 0 || D <= 0) return TA_ERR_INVALID_ARG;
+    if (ndims < 1 || ndims > TA_MAX_DIMS) return TA_ERR_INVALID_ARG;
+    long long prod = 1;
+    for (int i = 0; i < ndims; ++i) {
+        if (dims[i] < 1) return TA_ERR_INVALID_ARG;
+        prod *= dims[i];
+        if (prod > (1ll << 40)) return TA_ERR_SHAPE;
+    }
+    if (prod != N || H % H_kv != 0) return TA_ERR_SHAPE;
+    if (dtype != TA_DTYPE_BF16 && dtype != TA_DTYPE_F32) return TA_ERR_UNSUPPORTED;
+    if (D > TA_MAX_HEAD_DIM) return TA_ERR_UNSUPPORTED;
+    return TA_OK;
+}
+
+static bool tc_eligible(int D, int n, int dtype, unsigned flags) {
+    return dtype == TA_DTYPE_BF16 && (D == 64 || D == 128) && n <= 128 && !(flags & TA_FLAG_NO_TENSOR_CORE);
+}
+
+// Packs whole segments into a 128-row tile: ci consecutive `inner` positions, then co
+// consecutive `outer` positions (co only when the inner extent is exhausted, and only if it
+// divides the outer extent so that a tile never straddles two heads).
+static void tile_packing(HopDesc &h) {
+    const int cap = 128 / h.n;                       // segments per tile
+    h.ci = (int)(h.stride < cap ? h.stride : cap);
+    int co = cap / h.ci;
+    if (h.ci < h.stride) co = 1;
+    if (co > h.outer) co = (int)h.outer;
+    while (co > 1 && h.outer % co != 0) --co;
+    h.co = co;
+    h.rows = h.ci * h.co * h.n;
+    h.tiles_inner = (h.stride + h.ci - 1) / h.ci;
+    h.tiles_outer = (h.outer + h.co - 1) / h.co;
+}
+
+int build_plan(int B, int H, int H_kv, int N, int D, const int *dims, int ndims, int dtype,
+               unsigned flags, int hop_begin, int hop_end, Plan *plan) {
+    int rc = validate_shape(B, H, H_kv, N, D, dims, ndims, dtype);
+    if (rc != TA_OK) return rc;
+    if (flags & ~(unsigned)(TA_FLAG_NO_TENSOR_CORE | TA_FLAG_NO_HOP_FUSION | TA_FLAG_SAVE_HOPS))
+        return TA_ERR_UNSUPPORTED;
+    if (hop_begin == 0 && hop_end == 0) hop_end = ndims;
+    if (hop_begin < 0 || hop_end > ndims || hop_begin > hop_end) return TA_ERR_INVALID_ARG;
+    memset(plan, 0, sizeof(*plan));
+    for (int i = hop_begin; i < hop_end; ++i) {
+        if (dims[i] == 1) continue;  // softmax over one element: identity hop
+        HopDesc &h = plan->hops[plan->nhops++];
+        h.hop = i;
+        h.n = dims[i];
+        h.stride = 1;
+        for (int l = i + 1; l < ndims; ++l) h.stride *= dims[l];
+        h.outer = (long long)N / ((long long)h.n * h.stride);
+        h.path = tc_eligible(D, h.n, dtype, flags) ? PATH_TC : PATH_SIMT;
+        if (h.path == PATH_TC) tile_packing(h);
+    }
+    const size_t tensor_bytes = (size_t)B * H * N * D * elem_bytes(dtype);
+    const int nh = plan->nhops;
+    if (nh == 0) return TA_OK;
+    const int first_src = hop_begin > 0 ? BUF_OUT : BUF_V;
+    if (flags & TA_FLAG_SAVE_HOPS) {
+        // X_{j+1} of hop j goes to save slot j (buffer id 3 + j); the last hop writes `out`.
+        for (int j = 0; j < nh; ++j) {
+            plan->hops[j].src = j == 0 ? first_src : 3 + (j - 1);
+            plan->hops[j].dst = j == nh - 1 ? BUF_OUT : 3 + j;
+        }
+        plan->save_bytes = (size_t)(nh - 1) * tensor_bytes;
+        return TA_OK;
+    }
+    // The tensor-core kernel updates in place; the generic kernel needs src != dst.  Assign
+    // buffers from the last hop (which must land in `out`) backwards.
+    int dst = BUF_OUT;
+    for (int j = nh - 1; j >= 0; --j) {
+        HopDesc &h = plan->hops[j];
+        h.dst = dst;
+        if (j == 0) {
+            h.src = first_src;
+        } else {
+            h.src = h.path == PATH_TC ? dst : (dst == BUF_OUT ? BUF_SCRATCH : BUF_OUT);
+            dst = h.src;
+        }
+    }
+    if (plan->hops[0].path == PATH_SIMT && plan->hops[0].src == plan->hops[0].dst) {
+        // only reachable with hop_begin > 0: the caller's `out` is first copied to scratch
+        plan->hops[0].src = BUF_SCRATCH;
+    }
+    for (int j = 0; j < nh; ++j)
+        if (plan->hops[j].src == BUF_SCRATCH || plan->hops[j].dst == BUF_SCRATCH) plan->need_scratch = true;
+    if (plan->need_scratch) plan->scratch_bytes = tensor_bytes;
+    return TA_OK;
+}
+
+// ---------------------------------------------------------------------------------------
+// Device scratch / staging arenas owned by the library (grow-only, one per process).
+// ---------------------------------------------------------------------------------------
+struct Arena {
+    void *ptr = nullptr;
+    size_t bytes = 0;
+    int device = -1;
+    int reserve(size_t need) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess) return TA_ERR_CUDA;
+        if (ptr && dev == device && bytes >= need) return TA_OK;
+        if (ptr) {
+            cudaDeviceSynchronize();
+            cudaFree(ptr);
+            ptr = nullptr;
+            bytes = 0;
+        }
+        if (cudaMalloc(&ptr, need) != cudaSuccess) {
+            ptr = nullptr;
+            return TA_ERR_CUDA;
+        }
+        bytes = need;
+        device = dev;
+        return TA_OK;
+    }
+    void release() {
+        if (ptr) cudaFree(ptr);
+        ptr = nullptr;
+        bytes = 0;
+        device = -1;
+    }
+};
+static std::mutex g_arena_mutex;
+static Arena g_scratch, g_staging;
+
+static int check_arch() {
+    static std::atomic<int> cached{1};  // 1 = unknown
+    int c = cached.load();
+    if (c != 1) return c;
+    int dev = 0, major = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) {
+        cudaGetLastError();
+        return TA_ERR_CUDA;
+    }
+    c = major == 10 ? TA_OK : TA_ERR_ARCH;
+    cached.store(c);
+    return c;
+}
+
+static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static int forward_impl(const ta_params &p) {
+    if (!p.q || !p.k || !p.v || !p.out) return TA_ERR_INVALID_ARG;
+    Plan plan;
+    int rc = build_plan(p.B, p.H, p.H_kv, p.N, p.D, p.dims, p.ndims, p.dtype, p.flags, p.hop_begin,
+                        p.hop_end, &plan);
+    if (rc != TA_OK) return rc;
+    if (!aligned16(p.q) || !aligned16(p.k) || !aligned16(p.v) || !aligned16(p.out)) return TA_ERR_ALIGNMENT;
+    if (p.workspace && (reinterpret_cast<uintptr_t>(p.workspace) & 255u)) return TA_ERR_ALIGNMENT;
+    const size_t need = plan.scratch_bytes + plan.save_bytes;
+    if ((p.flags & TA_FLAG_SAVE_HOPS) && plan.save_bytes && !p.workspace) return TA_ERR_WORKSPACE;
+    if (p.workspace && p.workspace_bytes < need) return TA_ERR_WORKSPACE;
+    rc = check_arch();
+    if (rc != TA_OK) return rc;
+
+    Problem pb;
+    pb.q = p.q; pb.k = p.k; pb.v = p.v; pb.out = p.out;
+    pb.B = p.B; pb.H = p.H; pb.H_kv = p.H_kv; pb.N = p.N; pb.D = p.D;
+    for (int i = 0; i < p.ndims; ++i) pb.dims[i] = p.dims[i];
+    pb.ndims = p.ndims; pb.causal = p.causal ? 1 : 0; pb.dtype = p.dtype;
+    pb.scale = p.softmax_scale != 0.f ? p.softmax_scale : 1.0f / sqrtf((float)p.D);
+    pb.flags = p.flags; pb.hop_begin = p.hop_begin; pb.hop_end = p.hop_end;
+    pb.stream = (cudaStream_t)p.stream;
+
+    char *ws = (char *)p.workspace;
+    if (!ws && plan.need_scratch) {
+        std::lock_guard<std::mutex> lock(g_arena_mutex);
+        rc = g_scratch.reserve(plan.scratch_bytes);
+        if (rc != TA_OK) return rc;
+        ws = (char *)g_scratch.ptr;
+    }
+    const size_t tensor_bytes = (size_t)p.B * p.H * p.N * p.D * elem_bytes(p.dtype);
+    auto buffer = [&](int id) -> void * {
+        if (id == BUF_V) return const_cast<void *>(p.v);
+        if (id == BUF_OUT) return p.out;
+        if (id == BUF_SCRATCH) return ws;
+        return ws + plan.scratch_bytes + (size_t)(id - 3) * tensor_bytes;
+    };
+
+    if (plan.nhops == 0) {
+        if (p.hop_begin > 0) return TA_OK;  // value tensor already in `out`
+        return launch_broadcast_kv(pb);
+    }
+    if (p.hop_begin > 0 && plan.hops[0].src == BUF_SCRATCH) {
+        if (cudaMemcpyAsync(ws, p.out, tensor_bytes, cudaMemcpyDeviceToDevice, pb.stream) != cudaSuccess)
+            return TA_ERR_CUDA;
+    }
+    for (int j = 0; j < plan.nhops; ++j) {
+        const HopDesc &h = plan.hops[j];
+        const void *xin = buffer(h.src);
+        const int xin_heads = h.src == BUF_V ? p.H_kv : p.H;
+        void *xout = buffer(h.dst);
+        rc = h.path == PATH_TC ? launch_hop_tc(pb, h, xin, xin_heads, xout)
+                               : launch_hop_simt(pb, h, xin, xin_heads, xout);
+        if (rc != TA_OK) return rc;
+    }
+    return TA_OK;
+}
+
+}  // namespace ta
+
+using namespace ta;
+
+extern "C" {
+
+int ta_forward_ex(const ta_params *p) {
+    if (!p || p->struct_bytes != sizeof(ta_params)) return TA_ERR_INVALID_ARG;
+    return forward_impl(*p);
+}
+
+static int forward_simple(const void *q, const void *k, const void *v, void *out, int B, int H, int H_kv,
+                          int N, int D, const int *dims, int ndims, int causal, int dtype,
+                          ta_stream_t stream) {
+    ta_params p;
+    memset(&p, 0, sizeof(p));
+    p.struct_bytes = sizeof(p);
+    p.q = q; p.k = k; p.v = v; p.out = out;
+    p.B = B; p.H = H; p.H_kv = H_kv; p.N = N; p.D = D;
+    p.dims = dims; p.ndims = ndims; p.causal = causal; p.dtype = dtype;
+    p.stream = stream;
+    return forward_impl(p);
+}
+
+int ta_forward(const void *q, const void *k, const void *v, void *out, int B, int H, int H_kv, int N, int D,
+               const int *dims, int ndims, int causal, ta_stream_t stream) {
+    return forward_simple(q, k, v, out, B, H, H_kv, N, D, dims, ndims, causal, TA_DTYPE_BF16, stream);
+}
+
+int ta_forward_f32(const void *q, const void *k, const void *v, void *out, int B, int H, int H_kv, int N,
+                   int D, const int *dims, int ndims, int causal, ta_stream_t stream) {
+    return forward_simple(q, k, v, out, B, H, H_kv, N, D, dims, ndims, causal, TA_DTYPE_F32, stream);
+}
+
+size_t ta_workspace_bytes(int B, int H, int H_kv, int N, int D, const int *dims, int ndims, int dtype,
+                          int mode) {
+    Plan plan;
+    unsigned flags = mode == TA_WS_FORWARD_SAVE ? TA_FLAG_SAVE_HOPS : 0u;
+    if (build_plan(B, H, H_kv, N, D, dims, ndims, dtype, flags, 0, 0, &plan) != TA_OK) return 0;
+    if (mode == TA_WS_BACKWARD) return 0;
+    return plan.scratch_bytes + plan.save_bytes;
+}
+
+int ta_forward_host(const void *qh, const void *kh, const void *vh, void *outh, int B, int H, int H_kv, int N,
+                    int D, const int *dims, int ndims, int causal, int dtype, ta_stream_t stream) {
+    if (!qh || !kh || !vh || !outh) return TA_ERR_INVALID_ARG;
+    int rc = validate_shape(B, H, H_kv, N, D, dims, ndims, dtype);
+    if (rc != TA_OK) return rc;
+    rc = check_arch();
+    if (rc != TA_OK) return rc;
+    const size_t e = elem_bytes(dtype);
+    const size_t qb = (size_t)B * H * N * D * e, kb = (size_t)B * H_kv * N * D * e;
+    auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
+    char *base;
+    {
+        std::lock_guard<std::mutex> lock(g_arena_mutex);
+        rc = g_staging.reserve(2 * up(qb) + 2 * up(kb));
+        if (rc != TA_OK) return rc;
+        base = (char *)g_staging.ptr;
+    }
+    char *dq = base, *dk = dq + up(qb), *dv = dk + up(kb), *dout = dv + up(kb);
+    cudaStream_t s = (cudaStream_t)stream;
+    if (cudaMemcpyAsync(dq, qh, qb, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+        cudaMemcpyAsync(dk, kh, kb, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+        cudaMemcpyAsync(dv, vh, kb, cudaMemcpyHostToDevice, s) != cudaSuccess)
+        return TA_ERR_CUDA;
+    rc = forward_simple(dq, dk, dv, dout, B, H, H_kv, N, D, dims, ndims, causal, dtype, stream);
+    if (rc != TA_OK) return rc;
+    if (cudaMemcpyAsync(outh, dout, qb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return TA_ERR_CUDA;
+    return TA_OK;
+}
+
+int ta_backward(const void *dout, const void *q, const void *k, const void *v, const void *out, void *dq,
+                void *dk, void *dv, int B, int H, int H_kv, int N, int D, const int *dims, int ndims,
+                int causal, void *workspace, size_t workspace_bytes, ta_stream_t stream) {
+    (void)out; (void)causal; (void)workspace; (void)workspace_bytes; (void)stream;
+    if (!dout || !q || !k || !v || !dq || !dk || !dv) return TA_ERR_INVALID_ARG;
+    int rc = validate_shape(B, H, H_kv, N, D, dims, ndims, TA_DTYPE_BF16);
+    if (rc != TA_OK) return rc;
+    return TA_ERR_UNSUPPORTED;
+}
+
+static const char *buf_name(int id) {
+    switch (id) {
+        case BUF_V: return "v";
+        case BUF_OUT: return "out";
+        case BUF_SCRATCH: return "scratch";
+        default: return "save";
+    }
+}
+
+int ta_plan_describe(int B, int H, int H_kv, int N, int D, const int *dims, int ndims, int causal, int dtype,
+                     unsigned flags, char *buf, size_t cap) {
+    if (!buf || cap == 0) return TA_ERR_INVALID_ARG;
+    buf[0] = 0;
+    Plan plan;
+    int rc = build_plan(B, H, H_kv, N, D, dims, ndims, dtype, flags, 0, 0, &plan);
+    if (rc != TA_OK) return rc;
+    size_t off = 0;
+    auto emit = [&](const char *fmt, auto... a) {
+        if (off >= cap) return;
+        int w = snprintf(buf + off, cap - off, fmt, a...);
+        if (w > 0) off += (size_t)w;
+    };
+    emit("hops=%d causal=%d dtype=%s scratch_bytes=%zu save_bytes=%zu\n", plan.nhops, causal ? 1 : 0,
+         dtype == TA_DTYPE_F32 ? "f32" : "bf16", plan.scratch_bytes, plan.save_bytes);
+    for (int j = 0; j < plan.nhops; ++j) {
+        const HopDesc &h = plan.hops[j];
+        if (h.path == PATH_TC)
+            emit("hop=%d path=tc n=%d stride=%lld outer=%lld ci=%d co=%d rows=%d tiles_per_head=%lld src=%s dst=%s\n",
+                 h.hop, h.n, h.stride, h.outer, h.ci, h.co, h.rows, h.tiles_inner * h.tiles_outer,
+                 buf_name(h.src), buf_name(h.dst));
+        else
+            emit("hop=%d path=simt n=%d stride=%lld outer=%lld src=%s dst=%s\n", h.hop, h.n, h.stride, h.outer,
+                 buf_name(h.src), buf_name(h.dst));
+    }
+    return TA_OK;
+}
+
+int ta_device_status(void) { return read_device_status(); }
+
+unsigned long long ta_launch_count(void) { return g_launches.load(); }
+
+int ta_release(void) {
+    std::lock_guard<std::mutex> lock(g_arena_mutex);
+    if (g_scratch.ptr || g_staging.ptr) cudaDeviceSynchronize();
+    g_scratch.release();
+    g_staging.release();
+    return TA_OK;
+}
+
+const char *ta_status_string(int status) {
+    switch (status) {
+        case TA_OK: return "ok";
+        case TA_ERR_INVALID_ARG: return "invalid argument";
+        case TA_ERR_SHAPE: return "shape mismatch: prod(dims) != N or H % H_kv != 0";
+        case TA_ERR_UNSUPPORTED: return "unsupported configuration";
+        case TA_ERR_ALIGNMENT: return "pointer or row size not 16-byte aligned";
+        case TA_ERR_WORKSPACE: return "workspace missing or too small";
+        case TA_ERR_ARCH: return "device is not compute capability 10.x";
+        case TA_ERR_CUDA: return "CUDA call failed";
+        case TA_ERR_TIMEOUT: return "device-side wait timed out";
+        case TA_ERR_TOO_LARGE: return "size beyond a fixed limit";
+        default: return "unknown status";
+    }
+}
+
+int ta_version(void) { return 100; }
+
+}  // extern "C"

@@ -1,0 +1,79 @@
+// Internal declarations shared by the translation units of libta_b200.so.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "ta.h"
+
+namespace ta {
+
+// Buffers a hop may read its value tensor from / write it to.
+enum BufferId { BUF_V = 0, BUF_OUT = 1, BUF_SCRATCH = 2 };
+
+enum HopPath {
+    PATH_SIMT = 0,  // generic CUDA-core kernel, any n_i / D, fp32 or bf16 storage
+    PATH_TC = 1     // tcgen05 tensor-core kernel: bf16, D in {64,128}, n_i <= 128
+};
+
+// One hop of Algorithm 1 as a strided view X[outer][t][inner][D] of a head:
+//   token(outer, t, inner) = outer * n * stride + t * stride + inner.
+struct HopDesc {
+    int hop;          // index i in dims
+    int n;            // n_i, segment length
+    long long stride; // s_i = prod_{l>i} n_l  (= number of `inner` positions)
+    long long outer;  // N / (n * stride), per head
+    int path;         // HopPath
+    int src, dst;     // BufferId of the value tensor read / written
+    // Tensor-core tiling: a tile packs ci (along inner) x co (along outer) whole segments,
+    // rows = ci * co * n <= 128, row r of the tile = (co_l * ci + ci_l) * n + t.
+    int ci, co, rows;
+    long long tiles_inner, tiles_outer;  // per head
+};
+
+struct Plan {
+    int nhops;  // hops with n_i > 1
+    HopDesc hops[TA_MAX_DIMS];
+    bool need_scratch;      // some hop writes to / reads from BUF_SCRATCH
+    size_t scratch_bytes;   // B*H*N*D*elem when need_scratch
+    size_t save_bytes;      // (nhops-1)*B*H*N*D*elem, hop inputs X_1.. for backward
+};
+
+struct Problem {
+    const void *q, *k, *v;
+    void *out;
+    int B, H, H_kv, N, D;
+    int dims[TA_MAX_DIMS];
+    int ndims;
+    int causal;
+    int dtype;
+    float scale;  // already resolved (1/sqrt(D) default)
+    unsigned flags;
+    int hop_begin, hop_end;
+    cudaStream_t stream;
+};
+
+static inline size_t elem_bytes(int dtype) { return dtype == TA_DTYPE_F32 ? 4 : 2; }
+
+// Host-only: validates sizes (not pointers) and builds the plan.  Returns TA_OK / TA_ERR_*.
+int validate_shape(int B, int H, int H_kv, int N, int D, const int *dims, int ndims, int dtype);
+int build_plan(int B, int H, int H_kv, int N, int D, const int *dims, int ndims, int dtype,
+               unsigned flags, int hop_begin, int hop_end, Plan *plan);
+
+// Kernel launchers (each returns TA_OK or TA_ERR_CUDA).  xin has `xin_heads` heads per batch
+// (H_kv when reading v, H otherwise); xout always has H heads.
+int launch_hop_simt(const Problem &pb, const HopDesc &hd, const void *xin, int xin_heads,
+                    void *xout);
+int launch_hop_tc(const Problem &pb, const HopDesc &hd, const void *xin, int xin_heads,
+                  void *xout);
+// out[b,h] = v[b, h / (H/H_kv)] (all dims equal to 1).
+int launch_broadcast_kv(const Problem &pb);
+
+void count_launch(unsigned n = 1);
+
+// Device error word (bounded waits that expired).
+int read_device_status();
+
+}  // namespace ta

@@ -1,0 +1,218 @@
+// Generic CUDA-core kernel for one hop of tensorized attention (Algorithm 1, loop body;
+// Eq. 4): any segment length n_i, any head dim <= 256, fp32 or bf16 storage, fp32 arithmetic.
+//
+// One CTA handles BQ consecutive query positions of one segment and walks the segment's keys
+// in blocks of 32 with a running (online) softmax, so n_i is unbounded (ndims == 1 is ordinary
+// attention).  Because several CTAs read the same value rows, the hop cannot update the value
+// tensor in place: xin and xout are different buffers.
+//
+// This is the path of the fp32 configuration (TF32 tensor cores cannot meet its 1e-4
+// tolerance) and of hops the tcgen05 kernel does not cover.
+#include <cuda_bf16.h>
+
+#include "ta_internal.h"
+
+namespace ta {
+namespace {
+
+constexpr int kThreads = 128;
+constexpr int kWarps = kThreads / 32;
+constexpr int kRowsPerWarp = 4;
+constexpr int BQ = kWarps * kRowsPerWarp;  // 16 query rows per CTA
+constexpr int BK = 32;                     // keys per block: one per lane
+
+struct SimtArgs {
+    int N, D, n, H, H_kv, xin_heads, causal;
+    long long stride, outer;      // s_i, outer count per head
+    long long segs_per_head;      // outer * stride
+    int qblocks;                  // ceil(n / BQ)
+    long long items;              // B*H*segs_per_head*qblocks
+    float scale;
+};
+
+template <typename T> __device__ __forceinline__ float to_f32(T x);
+template <> __device__ __forceinline__ float to_f32<float>(float x) { return x; }
+template <> __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 x) { return __bfloat162float(x); }
+template <typename T> __device__ __forceinline__ T from_f32(float x);
+template <> __device__ __forceinline__ float from_f32<float>(float x) { return x; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float x) { return __float2bfloat16_rn(x); }
+
+__device__ __forceinline__ float warp_max(float x) {
+#pragma unroll
+    for (int o = 16; o; o >>= 1) x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, o));
+    return x;
+}
+__device__ __forceinline__ float warp_sum(float x) {
+#pragma unroll
+    for (int o = 16; o; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+    return x;
+}
+
+template <typename T, int DPL>  // DPL = columns per lane, D <= 32 * DPL
+__global__ void __launch_bounds__(kThreads)
+hop_simt_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__restrict__ xin,
+                T *__restrict__ xout, SimtArgs a) {
+    extern __shared__ float smem[];
+    const int D = a.D, ldk = D + 1;
+    float *sQ = smem;                 // [BQ][D]
+    float *sK = sQ + BQ * D;          // [BK][D+1]
+    float *sV = sK + BK * ldk;        // [BK][D+1]
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = a.H / a.H_kv;
+
+    for (long long item = blockIdx.x; item < a.items; item += gridDim.x) {
+        const int qb = (int)(item % a.qblocks);
+        long long rest = item / a.qblocks;
+        const long long seg = rest % a.segs_per_head;
+        const long long bh = rest / a.segs_per_head;
+        const int b = (int)(bh / a.H), h = (int)(bh % a.H);
+        const long long kvh = (long long)b * a.H_kv + h / g;
+        const long long xh = (a.xin_heads == a.H) ? bh : kvh;
+        const long long outer = seg / a.stride, inner = seg % a.stride;
+        const long long base = outer * a.n * a.stride + inner;   // first token of the segment
+        const T *qh = q + bh * (long long)a.N * D;
+        const T *kh = k + kvh * (long long)a.N * D;
+        const T *xh_p = xin + xh * (long long)a.N * D;
+        T *oh = xout + bh * (long long)a.N * D;
+        const int t0 = qb * BQ;
+
+        __syncthreads();   // previous item's smem no longer in use
+        for (int idx = threadIdx.x; idx < BQ * D; idx += kThreads) {
+            int r = idx / D, c = idx % D, t = t0 + r;
+            sQ[idx] = (t < a.n) ? to_f32<T>(qh[(base + (long long)t * a.stride) * D + c]) : 0.f;
+        }
+
+        float m[kRowsPerWarp], l[kRowsPerWarp], o[kRowsPerWarp][DPL];
+#pragma unroll
+        for (int r = 0; r < kRowsPerWarp; ++r) {
+            m[r] = -INFINITY;
+            l[r] = 0.f;
+#pragma unroll
+            for (int j = 0; j < DPL; ++j) o[r][j] = 0.f;
+        }
+
+        const int t_last = min(a.n, t0 + BQ) - 1;
+        const int key_end = a.causal ? t_last + 1 : a.n;
+        for (int k0 = 0; k0 < key_end; k0 += BK) {
+            __syncthreads();
+            for (int idx = threadIdx.x; idx < BK * D; idx += kThreads) {
+                int u = idx / D, c = idx % D, key = k0 + u;
+                float kvv = 0.f, xv = 0.f;
+                if (key < a.n) {
+                    long long off = (base + (long long)key * a.stride) * D + c;
+                    kvv = to_f32<T>(kh[off]);
+                    xv = to_f32<T>(xh_p[off]);
+                }
+                sK[u * ldk + c] = kvv;
+                sV[u * ldk + c] = xv;
+            }
+            __syncthreads();
+            const int key = k0 + lane;
+#pragma unroll
+            for (int r = 0; r < kRowsPerWarp; ++r) {
+                const int row = warp * kRowsPerWarp + r, t = t0 + row;
+                if (t >= a.n) continue;                        // warp-uniform
+                const float *qr = sQ + row * D, *kr = sK + lane * ldk;
+                float s = 0.f;
+                for (int c = 0; c < D; ++c) s = fmaf(qr[c], kr[c], s);
+                s *= a.scale;
+                const bool valid = key < a.n && (!a.causal || key <= t);
+                s = valid ? s : -INFINITY;
+                const float m_new = fmaxf(m[r], warp_max(s));  // finite: key 0 is always visible
+                const float p = valid ? expf(s - m_new) : 0.f;
+                const float alpha = expf(m[r] - m_new);
+                l[r] = l[r] * alpha + warp_sum(p);
+                m[r] = m_new;
+#pragma unroll
+                for (int j = 0; j < DPL; ++j) o[r][j] *= alpha;
+                for (int u = 0; u < BK; ++u) {
+                    const float pu = __shfl_sync(0xffffffffu, p, u);
+#pragma unroll
+                    for (int j = 0; j < DPL; ++j) {
+                        const int c = lane + 32 * j;
+                        if (c < D) o[r][j] = fmaf(pu, sV[u * ldk + c], o[r][j]);
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int r = 0; r < kRowsPerWarp; ++r) {
+            const int t = t0 + warp * kRowsPerWarp + r;
+            if (t >= a.n) continue;
+            const float inv = 1.f / l[r];
+#pragma unroll
+            for (int j = 0; j < DPL; ++j) {
+                const int c = lane + 32 * j;
+                if (c < D) oh[(base + (long long)t * a.stride) * D + c] = from_f32<T>(o[r][j] * inv);
+            }
+        }
+    }
+}
+
+template <typename T>
+__global__ void broadcast_kv_kernel(const T *__restrict__ v, T *__restrict__ out, long long per_head,
+                                    int H, int H_kv, long long total) {
+    const int g = H / H_kv;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
+         i += (long long)gridDim.x * blockDim.x) {
+        long long bh = i / per_head, r = i % per_head;
+        long long b = bh / H, h = bh % H;
+        out[i] = v[(b * H_kv + h / g) * per_head + r];
+    }
+}
+
+template <typename T, int DPL>
+int launch_t(const Problem &pb, const HopDesc &hd, const void *xin, int xin_heads, void *xout) {
+    SimtArgs a;
+    a.N = pb.N; a.D = pb.D; a.n = hd.n; a.H = pb.H; a.H_kv = pb.H_kv; a.xin_heads = xin_heads;
+    a.causal = pb.causal; a.stride = hd.stride; a.outer = hd.outer;
+    a.segs_per_head = hd.outer * hd.stride;
+    a.qblocks = (hd.n + BQ - 1) / BQ;
+    a.items = (long long)pb.B * pb.H * a.segs_per_head * a.qblocks;
+    a.scale = pb.scale;
+    size_t smem = sizeof(float) * ((size_t)BQ * pb.D + 2 * (size_t)BK * (pb.D + 1));
+    auto kern = hop_simt_kernel<T, DPL>;
+    if (smem > 48 * 1024) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+            return TA_ERR_CUDA;
+    }
+    long long grid = a.items < (1ll << 20) ? a.items : (1ll << 20);
+    kern<<<(unsigned)grid, kThreads, smem, pb.stream>>>((const T *)pb.q, (const T *)pb.k, (const T *)xin,
+                                                       (T *)xout, a);
+    count_launch();
+    return cudaPeekAtLastError() == cudaSuccess ? TA_OK : TA_ERR_CUDA;
+}
+
+template <typename T>
+int launch_d(const Problem &pb, const HopDesc &hd, const void *xin, int xin_heads, void *xout) {
+    const int dpl = (pb.D + 31) / 32;
+    switch (dpl) {
+        case 1: return launch_t<T, 1>(pb, hd, xin, xin_heads, xout);
+        case 2: return launch_t<T, 2>(pb, hd, xin, xin_heads, xout);
+        case 3: case 4: return launch_t<T, 4>(pb, hd, xin, xin_heads, xout);
+        default: return launch_t<T, 8>(pb, hd, xin, xin_heads, xout);
+    }
+}
+
+}  // namespace
+
+int launch_hop_simt(const Problem &pb, const HopDesc &hd, const void *xin, int xin_heads, void *xout) {
+    if (pb.dtype == TA_DTYPE_F32) return launch_d<float>(pb, hd, xin, xin_heads, xout);
+    return launch_d<__nv_bfloat16>(pb, hd, xin, xin_heads, xout);
+}
+
+int launch_broadcast_kv(const Problem &pb) {
+    const long long per_head = (long long)pb.N * pb.D;
+    const long long total = per_head * pb.B * pb.H;
+    const unsigned grid = (unsigned)((total + 255) / 256 < 148 * 16 ? (total + 255) / 256 : 148 * 16);
+    if (pb.dtype == TA_DTYPE_F32)
+        broadcast_kv_kernel<float><<<grid, 256, 0, pb.stream>>>((const float *)pb.v, (float *)pb.out, per_head,
+                                                                pb.H, pb.H_kv, total);
+    else
+        broadcast_kv_kernel<__nv_bfloat16><<<grid, 256, 0, pb.stream>>>(
+            (const __nv_bfloat16 *)pb.v, (__nv_bfloat16 *)pb.out, per_head, pb.H, pb.H_kv, total);
+    count_launch();
+    return cudaPeekAtLastError() == cudaSuccess ? TA_OK : TA_ERR_CUDA;
+}
+
+}  // namespace ta

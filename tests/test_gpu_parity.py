@@ -1,0 +1,133 @@
+"""GPU parity: the CUDA library (through its C ABI) against the fp64 oracle, element by element
+on the same seeded inputs.  Tolerances: bf16 storage max abs <= 2e-2 and mean abs <= 2e-3;
+fp32 path max abs <= 1e-4."""
+import math
+
+import numpy as np
+import pytest
+
+import oracle
+import paper_2410_20926_b200 as ta
+from paper_2410_20926_b200 import inputs as ta_inputs
+
+from helpers import assert_close, check_case, gpu_forward
+
+pytestmark = pytest.mark.gpu
+
+
+# ---------------------------------------------------------------- fp32 / generic kernel
+def test_config1_f32():
+    c = ta_inputs.CONFIGS[1]
+    inp = ta_inputs.make_config_inputs(c)
+    got = gpu_forward(inp, c.B, c.H, c.H_kv, c.N, c.D, c.dims, c.causal, "f32")
+    ref = oracle.forward(inp["q"], inp["k"], inp["v"], c.dims, c.causal)
+    assert_close(got, ref, "f32")
+
+
+@pytest.mark.parametrize("dims,D,causal", [
+    ([3, 5, 7], 40, True), ([3, 5, 7], 40, False), ([200], 64, True), ([70], 96, False),
+    ([2, 33], 32, True), ([17, 1, 3], 8, True), ([1, 1], 16, False), ([4, 4, 4, 4], 72, True),
+])
+def test_generic_f32_ragged(dims, D, causal):
+    check_case(2, 4, 2, math.prod(dims), D, dims, causal, "f32", seed=101)
+
+
+@pytest.mark.parametrize("dims,D,causal", [([6, 20], 64, True), ([150], 128, False), ([3, 5, 7], 48, True)])
+def test_generic_bf16(dims, D, causal):
+    check_case(1, 4, 2, math.prod(dims), D, dims, causal, "bf16", seed=102,
+               flags=ta.TA_FLAG_NO_TENSOR_CORE)
+
+
+# ---------------------------------------------------------------- tensor-core kernel
+@pytest.mark.parametrize("dims,D,causal", [
+    ([4, 64], 128, True),          # strided hop with 32 segments/tile + contiguous hop, 2 segments/tile
+    ([64, 64], 128, False),
+    ([32, 8, 32], 128, True),      # three hops, 4 segments per tile
+    ([16, 16], 64, True),          # D = 64, 8 segments per tile
+    ([128, 3], 128, True),         # one segment per tile, ragged inner extent (3 < ci)
+    ([2, 4, 12], 64, True),        # n does not divide 128: partly filled tiles
+    ([5, 24, 7], 128, False),      # odd everything: clipped boxes on the inner dimension
+    ([3, 100], 128, True),         # n = 100: single partly filled segment per tile
+    ([2, 2, 2, 2, 2, 2, 2], 64, True),
+])
+def test_tensor_core_small(dims, D, causal):
+    check_case(1, 4, 2, math.prod(dims), D, dims, causal, "bf16", seed=103)
+
+
+def test_tensor_core_batch_and_gqa_indexing():
+    check_case(3, 8, 2, 512, 128, [8, 64], True, "bf16", seed=104)
+    check_case(2, 6, 6, 256, 64, [16, 16], False, "bf16", seed=105)
+
+
+def test_mixed_paths_use_scratch():
+    # hop 0 on tensor cores, hop 1 (n = 160 > 128) on the generic kernel
+    check_case(1, 2, 1, 4 * 160, 64, [4, 160], True, "bf16", seed=106)
+
+
+def test_unit_dims_and_broadcast():
+    check_case(1, 4, 2, 64, 64, [1, 64, 1], True, "bf16", seed=107)
+    inp = ta_inputs.make_inputs(2, 4, 2, 1, 64, "bf16", 108)
+    got = gpu_forward(inp, 2, 4, 2, 1, 64, [1], True, "bf16")
+    np.testing.assert_array_equal(got, np.repeat(inp["v"], 2, axis=1))
+
+
+def test_hop_range_matches_oracle_intermediates():
+    B, H, Hkv, D, dims = 1, 2, 1, 128, [8, 16, 32]
+    N = math.prod(dims)
+    inp = ta_inputs.make_inputs(B, H, Hkv, N, D, "bf16", 109)
+    _, xs = oracle.forward(inp["q"], inp["k"], inp["v"], dims, True, return_xs=True)
+    got = gpu_forward(inp, B, H, Hkv, N, D, dims, True, "bf16", hop_begin=0, hop_end=1)
+    assert_close(got, np.stack([x[1] for x in xs])[None], "bf16")
+
+
+def test_save_hops_workspace():
+    import torch
+    B, H, Hkv, D, dims = 1, 2, 1, 64, [4, 8, 16]
+    N = math.prod(dims)
+    inp = ta_inputs.make_inputs(B, H, Hkv, N, D, "bf16", 110)
+    nbytes = ta.ta_workspace_bytes(B, H, Hkv, N, D, dims, ta.TA_DTYPE_BF16, ta.TA_WS_FORWARD_SAVE)
+    assert nbytes == 2 * B * H * N * D * 2
+    ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    got = gpu_forward(inp, B, H, Hkv, N, D, dims, True, "bf16", flags=ta.TA_FLAG_SAVE_HOPS,
+                      workspace=ws, workspace_bytes=nbytes)
+    ref, xs = oracle.forward(inp["q"], inp["k"], inp["v"], dims, True, return_xs=True)
+    assert_close(got, ref, "bf16")
+    saved = ws.view(torch.bfloat16).view(2, B, H, N, D).float().cpu().numpy()
+    for j in range(2):
+        assert_close(saved[j], np.stack([x[j + 1] for x in xs])[None], "bf16")
+
+
+def test_deterministic_and_in_place_safe():
+    c = ta_inputs.CONFIGS[2]
+    inp = ta_inputs.make_inputs(1, 4, 2, c.N, c.D, "bf16", 111)
+    a = gpu_forward(inp, 1, 4, 2, c.N, c.D, c.dims, True, "bf16")
+    b = gpu_forward(inp, 1, 4, 2, c.N, c.D, c.dims, True, "bf16")
+    np.testing.assert_array_equal(a, b)
+
+
+# ---------------------------------------------------------------- the benchmark configurations
+def test_config2_bf16():
+    c = ta_inputs.CONFIGS[2]
+    inp = ta_inputs.make_config_inputs(c)
+    got = gpu_forward(inp, c.B, c.H, c.H_kv, c.N, c.D, c.dims, c.causal, "bf16")
+    ref = oracle.forward(inp["q"], inp["k"], inp["v"], c.dims, c.causal)
+    assert_close(got, ref, "bf16")
+
+
+@pytest.mark.parametrize("idx,heads", [(3, [(0, 0), (0, 6), (0, 31)]), (4, [(0, 3), (0, 28)]),
+                                       (5, [(0, 9), (1, 22)])])
+def test_full_size_configs_sampled_heads(idx, heads):
+    """Full-size runs in the launch configuration the benchmark times; whole heads are compared
+    (the oracle computes one head at a time)."""
+    c = ta_inputs.CONFIGS[idx]
+    inp = ta_inputs.make_config_inputs(c)
+    got = gpu_forward(inp, c.B, c.H, c.H_kv, c.N, c.D, c.dims, c.causal, "bf16")
+    ref = oracle.forward(inp["q"], inp["k"], inp["v"], c.dims, c.causal, heads=heads)
+    sel = np.stack([got[b, h] for b, h in heads])
+    assert_close(sel, ref, "bf16")
+    # properties that hold at any size: finite, inside the range of V per column
+    assert np.isfinite(got).all()
+    g = c.H // c.H_kv
+    vmax = np.repeat(inp["v"].max(axis=2), g, axis=1)[:, :, None, :]
+    vmin = np.repeat(inp["v"].min(axis=2), g, axis=1)[:, :, None, :]
+    assert (got <= vmax + 0.05).all() and (got >= vmin - 0.05).all()
