@@ -156,6 +156,34 @@ int ta_forward_host(const void *q_host, const void *k_host, const void *v_host, 
                     const int *dims, int ndims, int causal, int dtype, ta_stream_t stream);
 
 /*
+ * ta_forward_static: forward pass that allocates nothing.  (The paper has no counterpart;
+ * this entry point exists for deployment reasons only.)
+ *
+ * For callers that cannot call cudaMalloc where they need the result: code inside a
+ * latency-critical serving loop (cudaMalloc synchronises the device), processes whose device
+ * memory is entirely managed by a pool the library cannot reach, and plug-ins that are only
+ * permitted to launch kernels.  Same arguments and result as ta_forward_ex with default
+ * options (dtype = TA_DTYPE_*), but the second value buffer that hops on the generic kernel
+ * need (fp32 storage, n_i > 128, head dims other than 64 / 128) comes from a fixed array of
+ * TA_STATIC_SCRATCH_BYTES that is part of the loaded module -- every GPU that loads the
+ * library holds those bytes until the process exits.  The call makes no cudaMalloc / cudaFree
+ * and calls no allocating routine.
+ *   - Problems whose value tensor (B*H*N*D elements) exceeds the array are rejected with
+ *     TA_ERR_TOO_LARGE before anything is launched.  Problems that need no second buffer
+ *     (every hop on the tensor-core kernel) have no size limit here.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current); make that first call before any stream capture begins.
+ *   - All calls on a device share the one array and it keeps the previous call's contents.
+ *     Nothing has to be cleared (each call overwrites every row it later reads), but calls
+ *     whose kernels can overlap on the GPU -- different streams or host threads -- race:
+ *     issue them on a single stream.
+ */
+#define TA_STATIC_SCRATCH_BYTES (16u << 20)
+int ta_forward_static(const void *q, const void *k, const void *v, void *out,
+                      int B, int H, int H_kv, int N, int D,
+                      const int *dims, int ndims, int causal, int dtype, ta_stream_t stream);
+
+/*
  * Text description of the launch plan the library would use for a problem (one line per hop:
  * kernel path, segment length, stride, tile packing, source / destination buffer).  Pure
  * host code: needs no GPU.  Writes at most `cap` bytes including the terminating NUL into

@@ -23,7 +23,8 @@ TA_WS_FORWARD, TA_WS_FORWARD_SAVE, TA_WS_BACKWARD = 0, 1, 2
 
 EXPORTS = ("ta_forward", "ta_forward_f32", "ta_forward_ex", "ta_backward", "ta_workspace_bytes",
            "ta_forward_host", "ta_plan_describe", "ta_device_status", "ta_launch_count",
-           "ta_release", "ta_status_string", "ta_version")
+           "ta_release", "ta_status_string", "ta_version", "ta_forward_static")
+TA_STATIC_SCRATCH_BYTES = 16 << 20
 
 
 class TaError(RuntimeError):
@@ -69,6 +70,7 @@ def load():
     lib.ta_workspace_bytes.argtypes = [ci, ci, ci, ci, ci, ip, ci, ci, ci]
     lib.ta_workspace_bytes.restype = ctypes.c_size_t
     lib.ta_forward_host.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, ci, ip, ci, ci, ci, vp]
+    lib.ta_forward_static.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, ci, ip, ci, ci, ci, vp]
     lib.ta_plan_describe.argtypes = [ci, ci, ci, ci, ci, ip, ci, ci, ci, ctypes.c_uint,
                                      ctypes.c_char_p, ctypes.c_size_t]
     lib.ta_device_status.argtypes = []
@@ -185,6 +187,16 @@ def ta_forward_host(q_host, k_host, v_host, out_host, B, H, H_kv, N, D, dims, ca
     return _done(load().ta_forward_host(_ptr(q_host), _ptr(k_host), _ptr(v_host), _ptr(out_host),
                                         B, H, H_kv, N, D, d, nd, int(bool(causal)), dtype,
                                         _stream(stream)), "ta_forward_host", check)
+
+
+def ta_forward_static(q, k, v, out, B, H, H_kv, N, D, dims, causal, dtype=TA_DTYPE_BF16,
+                      stream=None, check=True) -> int:
+    """Forward pass that allocates no device memory (scratch is a fixed array inside the
+    library, TA_STATIC_SCRATCH_BYTES); see include/ta.h for who needs this and its limits."""
+    d, nd = _dims(dims)
+    return _done(load().ta_forward_static(_ptr(q), _ptr(k), _ptr(v), _ptr(out), B, H, H_kv, N, D,
+                                          d, nd, int(bool(causal)), dtype, _stream(stream)),
+                 "ta_forward_static", check)
 
 
 def ta_plan_describe(B, H, H_kv, N, D, dims, causal, dtype=TA_DTYPE_BF16, flags=0,
