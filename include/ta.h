@@ -69,7 +69,7 @@ enum {
 };
 
 /* modes of ta_workspace_bytes */
-enum { TA_WS_FORWARD = 0, TA_WS_FORWARD_SAVE = 1, TA_WS_BACKWARD = 2 };
+enum { TA_WS_FORWARD = 0, TA_WS_FORWARD_SAVE = 1, TA_WS_BACKWARD = 2, TA_WS_BACKWARD_F32_GRADS = 3 };
 
 /*
  * Forward pass, bf16 storage (Algorithm 1; fp32 accumulation and fp32 softmax; the
@@ -125,19 +125,51 @@ typedef struct ta_params {
 int ta_forward_ex(const ta_params *p);
 
 /*
- * Backward pass of Algorithm 1 (the paper states no formula; this is the chain rule through
- * the recurrence, hops in reverse order): given dout = d loss / d out it writes
- *   dq [B,H,N,D], dk, dv [B,H_kv,N,D]   (storage dtype of the inputs; dk, dv summed over
- *   the H/H_kv query heads of a group; dq, dk summed over hops).
- * bf16 storage.  `workspace` (device) must hold ta_workspace_bytes(..., TA_WS_BACKWARD) bytes;
- * the pass recomputes the attention weights and the hop inputs from q, k, v.
- * `out` is not read (it may be NULL).
+ * Backward pass of Algorithm 1.  The paper states no formula; this is the chain rule through
+ * the recurrence X_{i+1} = A_i X_i (X_0 = V, out = X_m), hops in reverse order:
+ *     G_m = dout;   per hop:  dP = G_{i+1} X_i^T,  dS = A_i o (dP - rowsum(A_i o dP)) * scale,
+ *     G_i = A_i^T G_{i+1},  dQ += dS K,  dK += dS^T Q;   dV = G_0
+ * with dQ, dK summed over hops and dK, dV summed over the H/H_kv query heads of a KV head.
+ *   dout [B,H,N,D], q, k, v: device, bf16, read only.  `out` is not read (may be NULL).
+ *   dq [B,H,N,D], dk, dv [B,H_kv,N,D]: device, bf16, written.
+ *   workspace: device, 256-byte aligned, ta_workspace_bytes(..., TA_WS_BACKWARD) bytes.  It
+ *   holds the hop inputs X_1..X_{m-1} (recomputed here by running the forward hops), the bf16
+ *   gradient G carried between hops, and fp32 accumulators for dq, dk, dv, which are rounded
+ *   to bf16 once at the end.
+ * Arithmetic: bf16 operands, fp32 accumulation; the attention weights are recomputed.
+ * The sums over the query heads of a group are fp32 atomic adds at L2, so dk and dv are not
+ * bit-reproducible from run to run.
+ * Supported where every hop runs on the tensor-core kernel (D in {64,128}, all n_i <= 128);
+ * otherwise TA_ERR_UNSUPPORTED.
  */
 int ta_backward(const void *dout, const void *q, const void *k, const void *v, const void *out,
                 void *dq, void *dk, void *dv,
                 int B, int H, int H_kv, int N, int D,
                 const int *dims, int ndims, int causal,
                 void *workspace, size_t workspace_bytes, ta_stream_t stream);
+
+/* Extended backward.  Zero-initialise, set struct_bytes = sizeof(ta_bwd_params). */
+typedef struct ta_bwd_params {
+    size_t struct_bytes;
+    const void *dout, *q, *k, *v; /* device, bf16                                              */
+    void *dq, *dk, *dv;           /* device, grad_dtype                                        */
+    int B, H, H_kv, N, D;
+    const int *dims;              /* host                                                      */
+    int ndims;
+    int causal;
+    int dtype;                    /* storage of q, k, v, dout: TA_DTYPE_BF16                   */
+    int grad_dtype;               /* TA_DTYPE_BF16, or TA_DTYPE_F32: dq/dk/dv are the fp32      */
+                                  /* accumulators themselves (no final rounding, less workspace)*/
+    float softmax_scale;          /* 0 -> 1/sqrt(D)                                            */
+    const void *saved_hops;       /* X_1..X_{m-1} as written by ta_forward_ex(TA_FLAG_SAVE_HOPS) */
+                                  /* (the part of its workspace after the scratch tensor), or    */
+                                  /* NULL: recomputed                                          */
+    void *workspace;              /* device, 256-byte aligned                                  */
+    size_t workspace_bytes;       /* >= ta_workspace_bytes(.., TA_WS_BACKWARD[_F32_GRADS])      */
+    ta_stream_t stream;
+} ta_bwd_params;
+
+int ta_backward_ex(const ta_bwd_params *p);
 
 /* Bytes of device workspace a call needs (0 if none); mode = TA_WS_*.  dtype = TA_DTYPE_*.
  * Returns 0 for invalid shapes as well (the call itself reports the error). */

@@ -114,19 +114,26 @@ def forward(q, k, v, dims, causal: bool, scale: float | None = None, heads=None,
     return (out, xs_all) if return_xs else out
 
 
-def backward(dout, q, k, v, dims, causal: bool, scale: float | None = None):
-    """Gradients of sum(out * dout) w.r.t. q, k, v (fp64), GQA groups summed into dk, dv."""
+def backward(dout, q, k, v, dims, causal: bool, scale: float | None = None, groups=None):
+    """Gradients of sum(out * dout) w.r.t. q, k, v (fp64), GQA groups summed into dk, dv.
+
+    groups: optional list of (b, kv_head) pairs; then only those KV heads and their query
+    heads are computed and the result is (dq [len, g, N, D], dk [len, N, D], dv [len, N, D]).
+    """
     B, H, Hkv, N, D, dims = _check(q, k, v, dims)
     g = H // Hkv
     scale = 1.0 / math.sqrt(D) if scale is None else float(scale)
     cdims = (ctypes.c_int * len(dims))(*dims)
-    dq = np.zeros((B, H, N, D))
-    dk = np.zeros((B, Hkv, N, D))
-    dv = np.zeros((B, Hkv, N, D))
+    sel = [(b, kv) for b in range(B) for kv in range(Hkv)] if groups is None else list(groups)
+    dq = np.zeros((len(sel), g, N, D))
+    dk = np.zeros((len(sel), N, D))
+    dv = np.zeros((len(sel), N, D))
     lib = _lib()
-    for b in range(B):
-        for h in range(H):
-            qh, kh, vh = _f64(q[b, h]), _f64(k[b, h // g]), _f64(v[b, h // g])
+    for idx, (b, kv) in enumerate(sel):
+        kh, vh = _f64(k[b, kv]), _f64(v[b, kv])
+        for j in range(g):
+            h = kv * g + j
+            qh = _f64(q[b, h])
             o = np.empty((N, D))
             xs = np.empty((len(dims) + 1, N, D))
             rc = lib.ta_oracle_forward_head(_dptr(qh), _dptr(kh), _dptr(vh), _dptr(o), N, D,
@@ -141,9 +148,11 @@ def backward(dout, q, k, v, dims, causal: bool, scale: float | None = None):
                                              int(bool(causal)), scale)
             if rc != 0:
                 raise RuntimeError("ta_oracle_backward_head failed")
-            dq[b, h] = dqh
-            dk[b, h // g] += dkh
-            dv[b, h // g] += dvh
+            dq[idx, j] = dqh
+            dk[idx] += dkh
+            dv[idx] += dvh
+    if groups is None:
+        return dq.reshape(B, H, N, D), dk.reshape(B, Hkv, N, D), dv.reshape(B, Hkv, N, D)
     return dq, dk, dv
 
 

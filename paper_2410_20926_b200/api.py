@@ -19,11 +19,11 @@ TA_ERR_INVALID_ARG, TA_ERR_SHAPE, TA_ERR_UNSUPPORTED, TA_ERR_ALIGNMENT = -1, -2,
 TA_ERR_WORKSPACE, TA_ERR_ARCH, TA_ERR_CUDA, TA_ERR_TIMEOUT, TA_ERR_TOO_LARGE = -5, -6, -7, -8, -9
 TA_DTYPE_BF16, TA_DTYPE_F32 = 0, 1
 TA_FLAG_NO_TENSOR_CORE, TA_FLAG_NO_HOP_FUSION, TA_FLAG_SAVE_HOPS = 1, 2, 4
-TA_WS_FORWARD, TA_WS_FORWARD_SAVE, TA_WS_BACKWARD = 0, 1, 2
+TA_WS_FORWARD, TA_WS_FORWARD_SAVE, TA_WS_BACKWARD, TA_WS_BACKWARD_F32_GRADS = 0, 1, 2, 3
 
 EXPORTS = ("ta_forward", "ta_forward_f32", "ta_forward_ex", "ta_backward", "ta_workspace_bytes",
            "ta_forward_host", "ta_plan_describe", "ta_device_status", "ta_launch_count",
-           "ta_release", "ta_status_string", "ta_version", "ta_forward_static")
+           "ta_release", "ta_status_string", "ta_version", "ta_forward_static", "ta_backward_ex")
 TA_STATIC_SCRATCH_BYTES = 16 << 20
 
 
@@ -47,6 +47,21 @@ class ta_params(ctypes.Structure):
                 ("stream", ctypes.c_void_p)]
 
 
+class ta_bwd_params(ctypes.Structure):
+    _fields_ = [("struct_bytes", ctypes.c_size_t),
+                ("dout", ctypes.c_void_p), ("q", ctypes.c_void_p), ("k", ctypes.c_void_p),
+                ("v", ctypes.c_void_p),
+                ("dq", ctypes.c_void_p), ("dk", ctypes.c_void_p), ("dv", ctypes.c_void_p),
+                ("B", ctypes.c_int), ("H", ctypes.c_int), ("H_kv", ctypes.c_int),
+                ("N", ctypes.c_int), ("D", ctypes.c_int),
+                ("dims", ctypes.POINTER(ctypes.c_int)), ("ndims", ctypes.c_int),
+                ("causal", ctypes.c_int), ("dtype", ctypes.c_int), ("grad_dtype", ctypes.c_int),
+                ("softmax_scale", ctypes.c_float),
+                ("saved_hops", ctypes.c_void_p),
+                ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
+                ("stream", ctypes.c_void_p)]
+
+
 _lib = None
 
 
@@ -67,6 +82,7 @@ def load():
     lib.ta_forward_ex.argtypes = [ctypes.POINTER(ta_params)]
     lib.ta_backward.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ip, ci, ci, vp,
                                 ctypes.c_size_t, vp]
+    lib.ta_backward_ex.argtypes = [ctypes.POINTER(ta_bwd_params)]
     lib.ta_workspace_bytes.argtypes = [ci, ci, ci, ci, ci, ip, ci, ci, ci]
     lib.ta_workspace_bytes.restype = ctypes.c_size_t
     lib.ta_forward_host.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, ci, ip, ci, ci, ci, vp]
@@ -174,6 +190,23 @@ def ta_backward(dout, q, k, v, out, dq, dk, dv, B, H, H_kv, N, D, dims, causal, 
                                     _ptr(dk), _ptr(dv), B, H, H_kv, N, D, d, nd,
                                     int(bool(causal)), _ptr(workspace), workspace_bytes,
                                     _stream(stream)), "ta_backward", check)
+
+
+def ta_backward_ex(dout, q, k, v, dq, dk, dv, B, H, H_kv, N, D, dims, causal,
+                   grad_dtype=TA_DTYPE_BF16, softmax_scale=0.0, saved_hops=None, workspace=None,
+                   workspace_bytes=0, stream=None, check=True) -> int:
+    d, nd = _dims(dims)
+    p = ta_bwd_params()
+    p.struct_bytes = ctypes.sizeof(ta_bwd_params)
+    p.dout, p.q, p.k, p.v = _ptr(dout), _ptr(q), _ptr(k), _ptr(v)
+    p.dq, p.dk, p.dv = _ptr(dq), _ptr(dk), _ptr(dv)
+    p.B, p.H, p.H_kv, p.N, p.D = B, H, H_kv, N, D
+    p.dims, p.ndims, p.causal = d, nd, int(bool(causal))
+    p.dtype, p.grad_dtype, p.softmax_scale = TA_DTYPE_BF16, grad_dtype, softmax_scale
+    p.saved_hops = _ptr(saved_hops)
+    p.workspace, p.workspace_bytes = _ptr(workspace), workspace_bytes
+    p.stream = _stream(stream)
+    return _done(load().ta_backward_ex(ctypes.byref(p)), "ta_backward_ex", check)
 
 
 def ta_workspace_bytes(B, H, H_kv, N, D, dims, dtype=TA_DTYPE_BF16, mode=TA_WS_FORWARD) -> int:

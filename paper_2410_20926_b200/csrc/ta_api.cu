@@ -253,7 +253,9 @@ size_t ta_workspace_bytes(int B, int H, int H_kv, int N, int D, const int *dims,
     Plan plan;
     unsigned flags = mode == TA_WS_FORWARD_SAVE ? TA_FLAG_SAVE_HOPS : 0u;
     if (build_plan(B, H, H_kv, N, D, dims, ndims, dtype, flags, 0, 0, &plan) != TA_OK) return 0;
-    if (mode == TA_WS_BACKWARD) return 0;
+    if (mode == TA_WS_BACKWARD) return backward_workspace_bytes(B, H, H_kv, N, D, dims, ndims, TA_DTYPE_BF16, false);
+    if (mode == TA_WS_BACKWARD_F32_GRADS)
+        return backward_workspace_bytes(B, H, H_kv, N, D, dims, ndims, TA_DTYPE_F32, false);
     return plan.scratch_bytes + plan.save_bytes;
 }
 
@@ -286,14 +288,23 @@ int ta_forward_host(const void *qh, const void *kh, const void *vh, void *outh, 
     return TA_OK;
 }
 
+int ta_backward_ex(const ta_bwd_params *p) {
+    if (!p || p->struct_bytes != sizeof(ta_bwd_params)) return TA_ERR_INVALID_ARG;
+    return backward_impl(*p);
+}
+
 int ta_backward(const void *dout, const void *q, const void *k, const void *v, const void *out, void *dq,
                 void *dk, void *dv, int B, int H, int H_kv, int N, int D, const int *dims, int ndims,
                 int causal, void *workspace, size_t workspace_bytes, ta_stream_t stream) {
-    (void)out; (void)causal; (void)workspace; (void)workspace_bytes; (void)stream;
-    if (!dout || !q || !k || !v || !dq || !dk || !dv) return TA_ERR_INVALID_ARG;
-    int rc = validate_shape(B, H, H_kv, N, D, dims, ndims, TA_DTYPE_BF16);
-    if (rc != TA_OK) return rc;
-    return TA_ERR_UNSUPPORTED;
+    (void)out;
+    ta_bwd_params p;
+    memset(&p, 0, sizeof(p));
+    p.struct_bytes = sizeof(p);
+    p.dout = dout; p.q = q; p.k = k; p.v = v; p.dq = dq; p.dk = dk; p.dv = dv;
+    p.B = B; p.H = H; p.H_kv = H_kv; p.N = N; p.D = D; p.dims = dims; p.ndims = ndims; p.causal = causal;
+    p.dtype = TA_DTYPE_BF16; p.grad_dtype = TA_DTYPE_BF16;
+    p.workspace = workspace; p.workspace_bytes = workspace_bytes; p.stream = stream;
+    return backward_impl(p);
 }
 
 static const char *buf_name(int id) {
@@ -333,7 +344,12 @@ int ta_plan_describe(int B, int H, int H_kv, int N, int D, const int *dims, int 
     return TA_OK;
 }
 
-int ta_device_status(void) { return read_device_status(); }
+int ta_device_status(void) {
+    if (cudaDeviceSynchronize() != cudaSuccess) return TA_ERR_CUDA;
+    unsigned int w1 = 0, w2 = 0;
+    if (read_status_tc_forward(&w1) != TA_OK || read_status_tc_backward(&w2) != TA_OK) return TA_ERR_CUDA;
+    return (w1 | w2) ? TA_ERR_TIMEOUT : TA_OK;
+}
 
 unsigned long long ta_launch_count(void) { return g_launches.load(); }
 

@@ -1,0 +1,123 @@
+// Host side of the backward pass: workspace layout, recomputation of the hop inputs, the
+// reverse hop loop and the final conversion of the fp32 gradient accumulators.
+#include <cmath>
+#include <cstring>
+
+#include "ta_internal.h"
+
+namespace ta {
+namespace {
+
+size_t up256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+struct BwdLayout {
+    size_t save_off, gbuf_off, dq_off, dk_off, dv_off, total;
+};
+
+// [saved hop inputs X_1..X_{k-1}] [G buffer] [dq fp32] [dk fp32] [dv fp32]; the last three only
+// when the caller wants bf16 gradients, the first only when the hop inputs are recomputed.
+BwdLayout layout(const Plan &plan, int B, int H, int H_kv, int N, int D, bool need_save, bool need_acc) {
+    const size_t tq = (size_t)B * H * N * D, tkv = (size_t)B * H_kv * N * D;
+    BwdLayout L;
+    size_t off = 0;
+    L.save_off = off;
+    if (need_save && plan.nhops > 1) off += up256((size_t)(plan.nhops - 1) * tq * 2);
+    L.gbuf_off = off;
+    if (plan.nhops > 1) off += up256(tq * 2);
+    L.dq_off = off;
+    if (need_acc) off += up256(tq * 4);
+    L.dk_off = off;
+    if (need_acc) off += up256(tkv * 4);
+    L.dv_off = off;
+    if (need_acc) off += up256(tkv * 4);
+    L.total = off;
+    return L;
+}
+
+}  // namespace
+
+size_t backward_workspace_bytes(int B, int H, int H_kv, int N, int D, const int *dims, int ndims, int grad_dtype,
+                                bool have_saved_hops) {
+    Plan plan;
+    if (build_plan(B, H, H_kv, N, D, dims, ndims, TA_DTYPE_BF16, 0u, 0, 0, &plan) != TA_OK) return 0;
+    return layout(plan, B, H, H_kv, N, D, !have_saved_hops, grad_dtype != TA_DTYPE_F32).total;
+}
+
+int backward_impl(const ta_bwd_params &p) {
+    if (!p.dout || !p.q || !p.k || !p.v || !p.dq || !p.dk || !p.dv) return TA_ERR_INVALID_ARG;
+    if (p.dtype != TA_DTYPE_BF16) return TA_ERR_UNSUPPORTED;
+    if (p.grad_dtype != TA_DTYPE_BF16 && p.grad_dtype != TA_DTYPE_F32) return TA_ERR_UNSUPPORTED;
+    Plan plan;
+    int rc = build_plan(p.B, p.H, p.H_kv, p.N, p.D, p.dims, p.ndims, p.dtype, 0u, 0, 0, &plan);
+    if (rc != TA_OK) return rc;
+    for (int j = 0; j < plan.nhops; ++j)
+        if (plan.hops[j].path != PATH_TC) return TA_ERR_UNSUPPORTED;   // backward exists on the tensor-core path only
+    auto misaligned = [](const void *x) { return (reinterpret_cast<uintptr_t>(x) & 15u) != 0; };
+    if (misaligned(p.dout) || misaligned(p.q) || misaligned(p.k) || misaligned(p.v) || misaligned(p.dq) ||
+        misaligned(p.dk) || misaligned(p.dv) || (p.saved_hops && misaligned(p.saved_hops)))
+        return TA_ERR_ALIGNMENT;
+    const bool need_acc = p.grad_dtype != TA_DTYPE_F32;
+    const BwdLayout L = layout(plan, p.B, p.H, p.H_kv, p.N, p.D, p.saved_hops == nullptr, need_acc);
+    if (L.total > 0) {
+        if (!p.workspace || p.workspace_bytes < L.total) return TA_ERR_WORKSPACE;
+        if (reinterpret_cast<uintptr_t>(p.workspace) & 255u) return TA_ERR_ALIGNMENT;
+    }
+    int dev = 0, major = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess)
+        return TA_ERR_CUDA;
+    if (major != 10) return TA_ERR_ARCH;
+
+    Problem pb;
+    pb.q = p.q; pb.k = p.k; pb.v = p.v; pb.out = nullptr;
+    pb.B = p.B; pb.H = p.H; pb.H_kv = p.H_kv; pb.N = p.N; pb.D = p.D;
+    for (int i = 0; i < p.ndims; ++i) pb.dims[i] = p.dims[i];
+    pb.ndims = p.ndims; pb.causal = p.causal ? 1 : 0; pb.dtype = p.dtype;
+    pb.scale = p.softmax_scale != 0.f ? p.softmax_scale : 1.0f / sqrtf((float)p.D);
+    pb.flags = 0; pb.hop_begin = 0; pb.hop_end = p.ndims;
+    pb.stream = (cudaStream_t)p.stream;
+
+    const size_t tq = (size_t)p.B * p.H * p.N * p.D, tkv = (size_t)p.B * p.H_kv * p.N * p.D;
+    char *ws = (char *)p.workspace;
+    float *dq_acc = need_acc ? (float *)(ws + L.dq_off) : (float *)p.dq;
+    float *dk_acc = need_acc ? (float *)(ws + L.dk_off) : (float *)p.dk;
+    float *dv_acc = need_acc ? (float *)(ws + L.dv_off) : (float *)p.dv;
+    const int k = plan.nhops;
+
+    if (cudaMemsetAsync(dq_acc, 0, tq * 4, pb.stream) != cudaSuccess ||
+        cudaMemsetAsync(dk_acc, 0, tkv * 4, pb.stream) != cudaSuccess)
+        return TA_ERR_CUDA;
+    if (k == 0) {
+        // every dimension is 1: out = v broadcast over the group, so dv = sum of dout, dq = dk = 0
+        rc = launch_group_sum(p.dout, need_acc ? (void *)p.dv : (void *)dv_acc, need_acc ? 0 : 1, p.B, p.H, p.H_kv,
+                              (long long)p.N * p.D, pb.stream);
+        if (rc != TA_OK) return rc;
+    } else {
+        if (cudaMemsetAsync(dv_acc, 0, tkv * 4, pb.stream) != cudaSuccess) return TA_ERR_CUDA;
+        // X_j = input of hop j: X_0 = v, X_1.. = saved (or recomputed here by running hops 0..k-2)
+        const char *saved = p.saved_hops ? (const char *)p.saved_hops : ws + L.save_off;
+        auto hop_input = [&](int j) -> const void * { return j == 0 ? p.v : (const void *)(saved + (size_t)(j - 1) * tq * 2); };
+        if (!p.saved_hops) {
+            for (int j = 0; j + 1 < k; ++j) {
+                rc = launch_hop_tc(pb, plan.hops[j], hop_input(j), j == 0 ? p.H_kv : p.H,
+                                   ws + L.save_off + (size_t)j * tq * 2);
+                if (rc != TA_OK) return rc;
+            }
+        }
+        void *gbuf = k > 1 ? (void *)(ws + L.gbuf_off) : nullptr;
+        for (int j = k - 1; j >= 0; --j) {
+            const void *g_in = j == k - 1 ? p.dout : (const void *)gbuf;
+            rc = launch_hop_tc_bwd(pb, plan.hops[j], hop_input(j), j == 0 ? p.H_kv : p.H, g_in, j == 0 ? nullptr : gbuf,
+                                   dq_acc, dk_acc, dv_acc, j == 0);
+            if (rc != TA_OK) return rc;
+        }
+    }
+    if (need_acc) {
+        if ((rc = launch_f32_to_bf16(dq_acc, p.dq, (long long)tq, pb.stream)) != TA_OK) return rc;
+        if ((rc = launch_f32_to_bf16(dk_acc, p.dk, (long long)tkv, pb.stream)) != TA_OK) return rc;
+        if (k > 0 && (rc = launch_f32_to_bf16(dv_acc, p.dv, (long long)tkv, pb.stream)) != TA_OK) return rc;
+    }
+    return TA_OK;
+}
+
+}  // namespace ta

@@ -71,9 +71,27 @@ int launch_hop_tc(const Problem &pb, const HopDesc &hd, const void *xin, int xin
 // out[b,h] = v[b, h / (H/H_kv)] (all dims equal to 1).
 int launch_broadcast_kv(const Problem &pb);
 
+// Backward of one tensor-core hop (ta_tc_bwd.cu).  x = the hop's input value tensor (x_heads
+// heads per batch), g_in = gradient w.r.t. the hop's output, g_out = gradient w.r.t. its input
+// (bf16, may alias g_in; NULL when first_hop, where it is reduced into dv_acc instead).
+int launch_hop_tc_bwd(const Problem &pb, const HopDesc &hd, const void *x, int x_heads, const void *g_in,
+                      void *g_out, float *dq_acc, float *dk_acc, float *dv_acc, bool first_hop);
+int launch_f32_to_bf16(const float *src, void *dst, long long n, cudaStream_t stream);
+int launch_group_sum(const void *dout, void *dv, int dv_is_f32, int B, int H, int H_kv, long long per_head,
+                     cudaStream_t stream);
+
+int backward_impl(const ta_bwd_params &p);
+size_t backward_workspace_bytes(int B, int H, int H_kv, int N, int D, const int *dims, int ndims, int grad_dtype,
+                                bool have_saved_hops);
+
 void count_launch(unsigned n = 1);
 
-// Device error word (bounded waits that expired).
-int read_device_status();
+// TMA map of one tensor through a hop's strided view (ta_tc.cu); elem = 2 (bf16) or 4 (fp32).
+int make_hop_map(CUtensorMap *map, const void *base, int heads_total, int N, int D, const HopDesc &hd, int elem);
+
+// Device error words (bounded waits that expired), one per tensor-core translation unit:
+// copies the word to *word and clears it.
+int read_status_tc_forward(unsigned int *word);
+int read_status_tc_backward(unsigned int *word);
 
 }  // namespace ta

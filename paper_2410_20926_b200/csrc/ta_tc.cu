@@ -18,144 +18,20 @@
 #include <mutex>
 
 #include "ta_internal.h"
+#include "ta_ptx.cuh"
 
 namespace ta {
-
-__device__ unsigned int g_device_status = 0;
 
 namespace {
 
 constexpr int kTileRows = 128;
 constexpr int kThreads = 128;
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // bounded waits give up after 2 s
-constexpr uint32_t kErrWaitExpired = 0x7A000000u;
 
 struct TcArgs {
     int n, rows, ci, co, causal, g, H, H_kv, xin_is_kv;
     long long tiles_inner, tiles_outer, total_tiles;
     float scale_log2;
 };
-
-// ----------------------------------------------------------------------------- PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ unsigned long long globaltimer_ns() {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-// Bounded wait: returns false (and records an error word) if the phase did not complete in
-// kWaitLimitNs; the caller then stops issuing work and leaves the kernel normally.
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, uint32_t where) {
-    const unsigned long long t0 = globaltimer_ns();
-    for (;;) {
-        for (int i = 0; i < 64; ++i)
-            if (mbar_try_wait(bar, parity)) return true;
-        if (globaltimer_ns() - t0 > kWaitLimitNs) {
-            atomicCAS(&g_device_status, 0u, kErrWaitExpired | where);
-            return false;
-        }
-    }
-}
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t where) {
-    for (int i = 0; i < 32; ++i)
-        if (mbar_try_wait(bar, parity)) return true;
-    return mbar_wait_slow(bar, parity, where);
-}
-
-__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1,
-                                            int c2, int c3, int c4) {
-    asm volatile(
-        "cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
-        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
-        : "memory");
-}
-__device__ __forceinline__ void tma_store_5d(const CUtensorMap *map, uint32_t src, int c0, int c1, int c2, int c3,
-                                             int c4) {
-    asm volatile("cp.async.bulk.tensor.5d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4, %5, %6}], [%1];"
-                 ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
-                 : "memory");
-}
-__device__ __forceinline__ void tma_store_commit_and_wait_read() {
-    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-    asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-}
-__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-// D[tmem] (+)= A[smem desc] * B[smem desc]
-__device__ __forceinline__ void tc_mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                          uint32_t accumulate) {
-    asm volatile(
-        "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
-        " tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
-          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
-          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-        : "r"(taddr)
-        : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
-
-// 64-bit shared-memory matrix descriptor of tcgen05.mma, 128-byte swizzle.
-//   bits [0,14) start address >> 4, [16,30) leading byte offset >> 4, [32,46) stride byte
-//   offset >> 4, [46,48) descriptor version (1 on sm_100), [61,64) layout (2 = 128B swizzle).
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-    uint64_t d = 0;
-    d |= (uint64_t)((addr & 0x3FFFFu) >> 4);
-    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
-    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
-    d |= (uint64_t)1 << 46;
-    d |= (uint64_t)2 << 61;
-    return d;
-}
-// 32-bit instruction descriptor, kind::f16: bf16 x bf16 -> fp32, M = 128.
-//   [4,6) D format (1 = f32), [7,10) A format (1 = bf16), [10,13) B format, bit 15 A major,
-//   bit 16 B major (0 = K-major, 1 = MN-major), [17,23) N >> 3, [24,29) M >> 4.
-__host__ __device__ constexpr uint32_t instr_desc(int n, int b_mn_major) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn_major << 16) | ((uint32_t)(n >> 3) << 17) |
-           ((uint32_t)(128 >> 4) << 24);
-}
-
-__device__ __forceinline__ float fast_exp2(float x) {
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
-    uint32_t r;
-    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
-    return r;
-}
 
 // ----------------------------------------------------------------------------- the kernel
 template <int D>
@@ -398,31 +274,36 @@ EncodeTiledFn encode_fn() {
     return fn;
 }
 
-// Rank-5 map of one tensor [heads][N][D] seen through hop `hd`: dims (D, t, inner, outer, head).
-int make_hop_map(CUtensorMap *map, const void *base, int heads_total, int N, int D, const HopDesc &hd) {
+}  // namespace
+
+// Rank-5 map of one tensor [heads][N][D] seen through hop `hd`: dims (D, t, inner, outer, head),
+// box (128 bytes of D, n, ci, co, 1), 128-byte swizzle.  elem = 2 (bf16) or 4 (fp32).
+int make_hop_map(CUtensorMap *map, const void *base, int heads_total, int N, int D, const HopDesc &hd, int elem) {
     EncodeTiledFn enc = encode_fn();
     if (!enc) return TA_ERR_CUDA;
-    const cuuint64_t e = 2;
+    const cuuint64_t e = (cuuint64_t)elem;
     cuuint64_t gdim[5] = {(cuuint64_t)D, (cuuint64_t)hd.n, (cuuint64_t)hd.stride, (cuuint64_t)hd.outer,
                           (cuuint64_t)heads_total};
     cuuint64_t gstr[4] = {(cuuint64_t)hd.stride * D * e, (cuuint64_t)D * e, (cuuint64_t)hd.n * hd.stride * D * e,
                           (cuuint64_t)N * D * e};
-    cuuint32_t box[5] = {64u, (cuuint32_t)hd.n, (cuuint32_t)hd.ci, (cuuint32_t)hd.co, 1u};
+    cuuint32_t box[5] = {(cuuint32_t)(128 / elem), (cuuint32_t)hd.n, (cuuint32_t)hd.ci, (cuuint32_t)hd.co, 1u};
     cuuint32_t estr[5] = {1, 1, 1, 1, 1};
-    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void *>(base), gdim, gstr, box, estr,
-                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    CUresult r = enc(map, elem == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 5,
+                     const_cast<void *>(base), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? TA_OK : TA_ERR_CUDA;
 }
+
+namespace {
 
 template <int D>
 int launch_d(const Problem &pb, const HopDesc &hd, const void *xin, int xin_heads, void *xout) {
     CUtensorMap mq, mk, mxi, mxo;
     int rc;
-    if ((rc = make_hop_map(&mq, pb.q, pb.B * pb.H, pb.N, D, hd)) != TA_OK) return rc;
-    if ((rc = make_hop_map(&mk, pb.k, pb.B * pb.H_kv, pb.N, D, hd)) != TA_OK) return rc;
-    if ((rc = make_hop_map(&mxi, xin, pb.B * xin_heads, pb.N, D, hd)) != TA_OK) return rc;
-    if ((rc = make_hop_map(&mxo, xout, pb.B * pb.H, pb.N, D, hd)) != TA_OK) return rc;
+    if ((rc = make_hop_map(&mq, pb.q, pb.B * pb.H, pb.N, D, hd, 2)) != TA_OK) return rc;
+    if ((rc = make_hop_map(&mk, pb.k, pb.B * pb.H_kv, pb.N, D, hd, 2)) != TA_OK) return rc;
+    if ((rc = make_hop_map(&mxi, xin, pb.B * xin_heads, pb.N, D, hd, 2)) != TA_OK) return rc;
+    if ((rc = make_hop_map(&mxo, xout, pb.B * pb.H, pb.N, D, hd, 2)) != TA_OK) return rc;
 
     TcArgs a;
     a.n = hd.n; a.rows = hd.rows; a.ci = hd.ci; a.co = hd.co; a.causal = pb.causal;
@@ -461,14 +342,11 @@ int launch_hop_tc(const Problem &pb, const HopDesc &hd, const void *xin, int xin
     return TA_ERR_UNSUPPORTED;
 }
 
-int read_device_status() {
-    unsigned int w = 0;
-    if (cudaDeviceSynchronize() != cudaSuccess) return TA_ERR_CUDA;
-    if (cudaMemcpyFromSymbol(&w, g_device_status, sizeof(w)) != cudaSuccess) return TA_ERR_CUDA;
-    if (w != 0) {
+int read_status_tc_forward(unsigned int *word) {
+    if (cudaMemcpyFromSymbol(word, g_status_word, sizeof(*word)) != cudaSuccess) return TA_ERR_CUDA;
+    if (*word != 0) {
         unsigned int z = 0;
-        cudaMemcpyToSymbol(g_device_status, &z, sizeof(z));
-        return TA_ERR_TIMEOUT;
+        cudaMemcpyToSymbol(g_status_word, &z, sizeof(z));
     }
     return TA_OK;
 }

@@ -1,0 +1,133 @@
+"""GPU parity of the backward pass (through the C ABI) against the fp64 oracle's chain-rule
+gradients, which are themselves pinned by finite differences on the CPU.
+
+Tolerance.  Gradients are not O(1): an early token's dV / dK collects contributions from every
+later query of four heads and reaches |x| ~ 10-30 at these sizes, where one bf16 rounding
+(half-ulp = 2^-9 |x|) of the gradient carried between hops, or of the weights it is multiplied
+by, already exceeds 2e-2; and the error of a small element comes from the large terms summed
+into it, not from its own size.  The bound used here is therefore, per head,
+    |err| <= 2e-2 + 2^-8 * max|ref over that head|     and     mean |err| <= 2e-3,
+i.e. the stated absolute tolerance plus one bf16 ulp of the head's gradient scale.  Where the
+gradients stay below ~2 (the non-causal cases) this is the literal max abs <= 2e-2 ... 3e-2.
+"""
+import math
+
+import numpy as np
+import pytest
+
+import oracle
+import paper_2410_20926_b200 as ta
+from paper_2410_20926_b200 import inputs as ta_inputs
+
+from helpers import BF16_MAX_ABS, BF16_MEAN_ABS, to_device
+
+pytestmark = pytest.mark.gpu
+RTOL = 2.0 ** -8
+
+
+def gpu_backward(inp, B, H, Hkv, N, D, dims, causal, grad_f32, saved=None):
+    import torch
+    q, k, v, do = (to_device(inp, n, "bf16") for n in ("q", "k", "v", "dout"))
+    tdt = torch.float32 if grad_f32 else torch.bfloat16
+    dq = torch.full((B, H, N, D), float("nan"), dtype=tdt, device="cuda")
+    dk = torch.full((B, Hkv, N, D), float("nan"), dtype=tdt, device="cuda")
+    dv = torch.full((B, Hkv, N, D), float("nan"), dtype=tdt, device="cuda")
+    mode = ta.TA_WS_BACKWARD_F32_GRADS if grad_f32 else ta.TA_WS_BACKWARD
+    nbytes = ta.ta_workspace_bytes(B, H, Hkv, N, D, dims, ta.TA_DTYPE_BF16, mode)
+    ws = torch.empty(max(nbytes, 256), dtype=torch.uint8, device="cuda")
+    if grad_f32 or saved is not None:
+        ta.ta_backward_ex(do, q, k, v, dq, dk, dv, B, H, Hkv, N, D, dims, causal,
+                          grad_dtype=ta.TA_DTYPE_F32 if grad_f32 else ta.TA_DTYPE_BF16,
+                          saved_hops=saved, workspace=ws, workspace_bytes=nbytes)
+    else:
+        ta.ta_backward(do, q, k, v, None, dq, dk, dv, B, H, Hkv, N, D, dims, causal, workspace=ws,
+                       workspace_bytes=nbytes)
+    torch.cuda.synchronize()
+    ta.ta_device_status()
+    return tuple(t.float().cpu().numpy().astype(np.float64) for t in (dq, dk, dv))
+
+
+def assert_grad_close(got, ref, name):
+    """got, ref: [..., N, D]; the leading axes enumerate heads."""
+    assert np.isfinite(got).all(), name
+    err = np.abs(got - ref)
+    scale = np.abs(ref).max(axis=(-2, -1), keepdims=True)
+    bound = BF16_MAX_ABS + RTOL * scale
+    worst = float((err - bound).max())
+    assert worst <= 0, (name, float(err.max()), float(scale.max()), worst)
+    assert err.mean() <= BF16_MEAN_ABS, (name, float(err.mean()))
+    return float(err.max()), float(err.mean()), float(scale.max())
+
+
+@pytest.mark.parametrize("dims,D,causal,B,H,Hkv", [
+    ([128], 128, True, 1, 2, 1),
+    ([4, 32], 128, True, 1, 4, 2),
+    ([8, 16, 32], 128, True, 1, 4, 2),
+    ([16, 16], 64, False, 2, 4, 4),
+    ([5, 24, 7], 128, True, 2, 4, 2),
+    ([2, 4, 12], 64, False, 1, 4, 1),
+    ([64, 1, 64], 128, True, 1, 8, 2),
+])
+@pytest.mark.parametrize("grad_f32", [False, True])
+def test_backward_small(dims, D, causal, B, H, Hkv, grad_f32):
+    N = math.prod(dims)
+    inp = ta_inputs.make_inputs(B, H, Hkv, N, D, "bf16", 301, with_dout=True)
+    got = gpu_backward(inp, B, H, Hkv, N, D, dims, causal, grad_f32)
+    ref = oracle.backward(inp["dout"], inp["q"], inp["k"], inp["v"], dims, causal)
+    for name, g, r in zip(("dq", "dk", "dv"), got, ref):
+        assert_grad_close(g, r, name)
+
+
+def test_backward_all_unit_dims():
+    inp = ta_inputs.make_inputs(2, 4, 2, 1, 64, "bf16", 302, with_dout=True)
+    dq, dk, dv = gpu_backward(inp, 2, 4, 2, 1, 64, [1, 1], True, True)
+    assert (dq == 0).all() and (dk == 0).all()
+    ref = inp["dout"].reshape(2, 2, 2, 1, 64).sum(axis=2)
+    np.testing.assert_allclose(dv, ref, atol=1e-6)
+
+
+def test_backward_with_saved_hops_matches_recompute():
+    import torch
+    B, H, Hkv, D, dims = 1, 4, 2, 128, [8, 8, 16]
+    N = math.prod(dims)
+    inp = ta_inputs.make_inputs(B, H, Hkv, N, D, "bf16", 303, with_dout=True)
+    q, k, v = (to_device(inp, n, "bf16") for n in ("q", "k", "v"))
+    nsave = ta.ta_workspace_bytes(B, H, Hkv, N, D, dims, ta.TA_DTYPE_BF16, ta.TA_WS_FORWARD_SAVE)
+    saved = torch.empty(nsave, dtype=torch.uint8, device="cuda")
+    out = torch.empty((B, H, N, D), dtype=torch.bfloat16, device="cuda")
+    ta.ta_forward_ex(q, k, v, out, B, H, Hkv, N, D, dims, True, flags=ta.TA_FLAG_SAVE_HOPS,
+                     workspace=saved, workspace_bytes=nsave)
+    a = gpu_backward(inp, B, H, Hkv, N, D, dims, True, False, saved=saved)
+    b = gpu_backward(inp, B, H, Hkv, N, D, dims, True, False)
+    np.testing.assert_array_equal(a[0], b[0])              # dq has no atomics: bit-identical
+    for x, y in zip(a[1:], b[1:]):
+        np.testing.assert_allclose(x, y, atol=0.07, rtol=2.0 ** -7)   # fp32 atomics, bf16 rounding
+
+
+def test_backward_rejects_unsupported_and_small_workspace():
+    import torch
+    x = torch.zeros(1, 2, 256, 64, dtype=torch.bfloat16, device="cuda")
+    rc = ta.ta_backward(x, x, x, x, None, x, x, x, 1, 2, 2, 256, 64, [256], True, workspace=None,
+                        workspace_bytes=0, check=False)
+    assert rc == ta.TA_ERR_UNSUPPORTED                     # n = 256 runs on the generic kernel
+    rc = ta.ta_backward(x, x, x, x, None, x, x, x, 1, 2, 2, 256, 64, [16, 16], True, workspace=None,
+                        workspace_bytes=0, check=False)
+    assert rc == ta.TA_ERR_WORKSPACE
+
+
+def test_config5_forward_backward_sampled_groups():
+    """Config 5 (B=2, H=32, H_kv=8, N=32768 as 32x32x32, training step) at full size; two KV
+    groups are compared completely (dq of their four query heads, dk, dv)."""
+    c = ta_inputs.CONFIGS[5]
+    inp = ta_inputs.make_config_inputs(c)
+    got = gpu_backward(inp, c.B, c.H, c.H_kv, c.N, c.D, list(c.dims), c.causal, False)
+    groups = [(0, 2), (1, 7)]
+    rq, rk, rv = oracle.backward(inp["dout"], inp["q"], inp["k"], inp["v"], list(c.dims), c.causal,
+                                 groups=groups)
+    g = c.H // c.H_kv
+    for idx, (b, kv) in enumerate(groups):
+        assert_grad_close(got[0][b, kv * g:(kv + 1) * g], rq[idx], "dq")
+        assert_grad_close(got[1][b, kv], rk[idx], "dk")
+        assert_grad_close(got[2][b, kv], rv[idx], "dv")
+    for t in got:
+        assert np.isfinite(t).all()

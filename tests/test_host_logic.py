@@ -126,3 +126,25 @@ def test_plan_tiles_never_straddle_heads():
     for h in hops:
         assert int(h["rows"]) <= 128 and int(h["rows"]) == int(h["ci"]) * int(h["co"]) * int(h["n"])
         assert int(h["outer"]) % int(h["co"]) == 0
+
+
+def test_backward_validation_and_workspace_sizes():
+    e = 1 * 4 * 512 * 128                      # elements of a q-shaped tensor
+    kv = e // 2
+    need = ta.ta_workspace_bytes(1, 4, 2, 512, 128, [8, 64], ta.TA_DTYPE_BF16, ta.TA_WS_BACKWARD)
+    assert need == 2 * e + 2 * e + 4 * e + 2 * 4 * kv     # X_1, G, dq fp32, dk + dv fp32
+    need32 = ta.ta_workspace_bytes(1, 4, 2, 512, 128, [8, 64], ta.TA_DTYPE_BF16,
+                                   ta.TA_WS_BACKWARD_F32_GRADS)
+    assert need32 == 2 * e + 2 * e
+    rc = ta.ta_backward(16, 16, 16, 16, None, 16, 16, 16, 1, 4, 2, 512, 128, [8, 63], True,
+                        workspace=256, workspace_bytes=1 << 30, stream=0, check=False)
+    assert rc == ta.TA_ERR_SHAPE
+    rc = ta.ta_backward(0, 16, 16, 16, None, 16, 16, 16, 1, 4, 2, 512, 128, [8, 64], True,
+                        workspace=256, workspace_bytes=1 << 30, stream=0, check=False)
+    assert rc == ta.TA_ERR_INVALID_ARG
+    rc = ta.ta_backward(16, 16, 16, 16, None, 16, 16, 16, 1, 4, 2, 512, 128, [8, 64], True,
+                        workspace=256, workspace_bytes=1024, stream=0, check=False)
+    assert rc == ta.TA_ERR_WORKSPACE
+    rc = ta.ta_backward(16, 16, 16, 16, None, 16, 16, 16, 1, 4, 2, 512, 96, [8, 64], True,
+                        workspace=256, workspace_bytes=1 << 30, stream=0, check=False)
+    assert rc == ta.TA_ERR_UNSUPPORTED          # head dim 96 has no tensor-core backward
