@@ -56,6 +56,33 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_
     return mbar_wait_slow(bar, parity, where);
 }
 
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// Bounded wait that also gives up as soon as another role of the CTA has raised `*abort_flag`
+// (a shared-memory word): a pipeline whose stages wait on one another drains in one time-out
+// instead of one per stage.  On expiry the flag is raised and the error word recorded.
+__device__ __noinline__ bool mbar_wait_abortable_slow(uint32_t bar, uint32_t parity, uint32_t where,
+                                                      volatile uint32_t *abort_flag) {
+    const unsigned long long t0 = globaltimer_ns();
+    for (;;) {
+        for (int i = 0; i < 64; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (globaltimer_ns() - t0 > kWaitLimitNs) {
+            atomicCAS(&g_status_word, 0u, kErrWaitExpired | where);
+            *abort_flag = 1u;
+            return false;
+        }
+    }
+}
+__device__ __forceinline__ bool mbar_wait_abortable(uint32_t bar, uint32_t parity, uint32_t where,
+                                                    volatile uint32_t *abort_flag) {
+    for (int i = 0; i < 16; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_abortable_slow(bar, parity, where, abort_flag);
+}
+
 __device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1,
                                             int c2, int c3, int c4) {
     asm volatile(

@@ -9,10 +9,21 @@
 // layout of tcgen05.mma for Q and K, and the MN-major one for the value tile.
 //
 // Per tile:  S = Q K^T (tcgen05.mma, fp32 in TMEM)  ->  block-diagonal + causal mask, row softmax
-// in fp32 registers (tcgen05.ld), un-normalised weights rounded to bf16 into shared memory
-// (over the Q/K tiles, which are dead by then)  ->  O = P X (tcgen05.mma, fp32 in TMEM)  ->
-// O / rowsum -> bf16 -> shared memory (over the X tile)  ->  TMA store to the same strided rows.
-// Because a tile owns whole segments, the value tensor is updated in place.
+// in fp32 registers (tcgen05.ld), un-normalised weights rounded to bf16 into shared memory  ->
+// O = P X (tcgen05.mma, fp32 in TMEM)  ->  O / rowsum -> bf16 -> shared memory (over the X tile)
+// ->  TMA store to the same strided rows.  Because a tile owns whole segments, the value tensor
+// is updated in place.
+//
+// The kernel is persistent (one CTA per SM) and warp-specialised, so that the HBM traffic of
+// the next tiles overlaps the arithmetic of the current one:
+//   warp 0      TMA producer: K tile of a work item (shared by the query heads of a GQA group
+//               that the item covers), then Q and X tiles per head, into rings of shared memory
+//   warp 1      MMA issuer: S(t) as soon as Q(t), K are in; O(t-1) once P(t-1), X(t-1) are
+//   warps 4-7   softmax + epilogue of the even tiles   } each warp owns 32 TMEM lanes (rows);
+//   warps 8-11  softmax + epilogue of the odd tiles    } S and O are double-buffered in TMEM
+//   warp 2      TMA store of finished tiles; hands the X slot back to the producer
+// Every wait is an mbarrier wait with a time limit; when one expires the CTA raises a flag that
+// ends all its roles, waits for its copies in flight, frees its TMEM and returns.
 #include <cuda_bf16.h>
 
 #include <mutex>
@@ -25,54 +36,107 @@ namespace ta {
 namespace {
 
 constexpr int kTileRows = 128;
-constexpr int kThreads = 128;
+constexpr int kThreads = 384;
+constexpr int kNK = 2;   // K ring (one slot per work item)
+constexpr int kNQ = 2;   // Q ring (one slot per tile)
+
+template <int D>
+struct PipeCfg {
+    static constexpr int kHalves = D / 64;                     // 64-column (128-byte) slabs per row
+    static constexpr uint32_t kSlabBytes = kTileRows * 128;    // one [128 rows][64 cols] bf16 slab
+    static constexpr uint32_t kTileBytes = kHalves * kSlabBytes;
+    static constexpr uint32_t kPBytes = 2 * kSlabBytes;        // P: 128 x 128 bf16
+    static constexpr int kNX = D == 128 ? 2 : 4;               // X ring (value tile in, output tile out)
+    static constexpr uint32_t kOffK = 0;
+    static constexpr uint32_t kOffQ = kOffK + kNK * kTileBytes;
+    static constexpr uint32_t kOffP = kOffQ + kNQ * kTileBytes;
+    static constexpr uint32_t kOffX = kOffP + kPBytes;
+    static constexpr uint32_t kOffBar = kOffX + kNX * kTileBytes;
+    static constexpr int kNumBars = 2 * kNK + 2 * kNQ + 3 * kNX + 2 + 2 + 2;
+    static constexpr uint32_t kSmemBytes = kOffBar + kNumBars * 8 + 16 + 1024 /*alignment slack*/;
+    static constexpr uint32_t kTmemCols = 512;                 // S: 2 x 128 columns, O: 2 x 128
+    static constexpr uint32_t kColS = 0, kColO = 256;
+};
 
 struct TcArgs {
     int n, rows, ci, co, causal, g, H, H_kv, xin_is_kv;
-    long long tiles_inner, tiles_outer, total_tiles;
+    int gi, hsplit;            // query heads per work item, items per GQA group (gi * hsplit == g)
+    long long tiles_inner, tiles_outer, total_items;
     float scale_log2;
 };
 
+struct ItemCoord {
+    int c_inner, c_outer, kv_head, q_head0;
+};
+// item -> (head chunk of the group, inner tile, outer tile, kv head, batch); the head chunks of
+// a GQA group are adjacent so that their common K (and V) tile is hot in L2.
+__device__ __forceinline__ ItemCoord decode_item(const TcArgs &a, long long item) {
+    ItemCoord c;
+    long long rest = item;
+    const int hs = (int)(rest % a.hsplit); rest /= a.hsplit;
+    c.c_inner = (int)(rest % a.tiles_inner) * a.ci; rest /= a.tiles_inner;
+    c.c_outer = (int)(rest % a.tiles_outer) * a.co; rest /= a.tiles_outer;
+    c.kv_head = (int)rest;                                      // b * H_kv + kvh
+    c.q_head0 = (c.kv_head / a.H_kv) * a.H + (c.kv_head % a.H_kv) * a.g + hs * a.gi;
+    return c;
+}
+
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+
 // ----------------------------------------------------------------------------- the kernel
 template <int D>
-__global__ void __launch_bounds__(kThreads)
-hop_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-              const __grid_constant__ CUtensorMap map_xin, const __grid_constant__ CUtensorMap map_xout,
-              const TcArgs a) {
-    constexpr int kHalves = D / 64;                 // 64-column (128-byte) slabs per row
-    constexpr uint32_t kSlabBytes = kTileRows * 128;  // one [128 rows][64 cols] bf16 slab
-    constexpr uint32_t kTileBytes = kHalves * kSlabBytes;
-    constexpr uint32_t kTmemCols = 256;             // S: 128 columns, O: D columns
-    constexpr uint32_t kOCol = 128;
+__global__ void __launch_bounds__(kThreads, 1)
+hop_pipe_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                const __grid_constant__ CUtensorMap map_xin, const __grid_constant__ CUtensorMap map_xout,
+                const TcArgs a) {
+    using C = PipeCfg<D>;
+    constexpr int kHalves = C::kHalves;
+    constexpr uint32_t kSlabBytes = C::kSlabBytes, kTileBytes = C::kTileBytes;
+    constexpr int kNX = C::kNX;
 
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    const uint32_t sQ = smem_u32(smem);
-    const uint32_t sK = sQ + kTileBytes;
-    const uint32_t sX = sK + kTileBytes;
-    const uint32_t sP = sQ;                         // P (128 x 128 bf16, 32 KB) reuses the Q/K space
-    uint64_t *bars = (uint64_t *)(smem + 3 * kTileBytes);
-    const uint32_t bar_qk = smem_u32(bars + 0), bar_x = smem_u32(bars + 1), bar_s = smem_u32(bars + 2),
-                   bar_o = smem_u32(bars + 3);
-    uint32_t *tmem_slot = (uint32_t *)(bars + 4);
+    const uint32_t s0 = smem_u32(smem);
+    const uint32_t sK = s0 + C::kOffK, sQ = s0 + C::kOffQ, sP = s0 + C::kOffP, sX = s0 + C::kOffX;
+    const uint32_t bar0 = s0 + C::kOffBar;
+    // barrier indices
+    auto k_full = [&](int i) { return bar0 + 8u * (uint32_t)i; };
+    auto k_free = [&](int i) { return bar0 + 8u * (uint32_t)(kNK + i); };
+    auto q_full = [&](int i) { return bar0 + 8u * (uint32_t)(2 * kNK + i); };
+    auto q_free = [&](int i) { return bar0 + 8u * (uint32_t)(2 * kNK + kNQ + i); };
+    constexpr int kB0 = 2 * kNK + 2 * kNQ;
+    auto x_full = [&](int i) { return bar0 + 8u * (uint32_t)(kB0 + i); };
+    auto x_free = [&](int i) { return bar0 + 8u * (uint32_t)(kB0 + kNX + i); };
+    auto out_full = [&](int i) { return bar0 + 8u * (uint32_t)(kB0 + 2 * kNX + i); };
+    constexpr int kB1 = kB0 + 3 * kNX;
+    auto s_full = [&](int i) { return bar0 + 8u * (uint32_t)(kB1 + i); };
+    auto o_full = [&](int i) { return bar0 + 8u * (uint32_t)(kB1 + 2 + i); };
+    const uint32_t p_full = bar0 + 8u * (uint32_t)(kB1 + 4), p_free = bar0 + 8u * (uint32_t)(kB1 + 5);
+    uint32_t *tmem_slot = (uint32_t *)(smem + C::kOffBar + C::kNumBars * 8);
+    volatile uint32_t *abort_flag = tmem_slot + 1;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
     // ---- one-time setup
-    for (uint32_t i = tid; i < 3 * kTileBytes / 16; i += kThreads)
+    for (uint32_t i = tid; i < C::kOffBar / 16; i += kThreads)
         ((uint4 *)smem)[i] = make_uint4(0, 0, 0, 0);   // rows a box never fills must stay finite
     if (tid == 0) {
-        mbar_init(bar_qk, 1);
-        mbar_init(bar_x, 1);
-        mbar_init(bar_s, 1);
-        mbar_init(bar_o, 1);
+        for (int i = 0; i < kNK; ++i) { mbar_init(k_full(i), 1); mbar_init(k_free(i), 1); }
+        for (int i = 0; i < kNQ; ++i) { mbar_init(q_full(i), 1); mbar_init(q_free(i), 1); }
+        for (int i = 0; i < kNX; ++i) { mbar_init(x_full(i), 1); mbar_init(x_free(i), 1); mbar_init(out_full(i), 4); }
+        for (int i = 0; i < 2; ++i) { mbar_init(s_full(i), 1); mbar_init(o_full(i), 1); }
+        mbar_init(p_full, 4);
+        mbar_init(p_free, 1);
+        *abort_flag = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     fence_proxy_async_smem();
-    if (warp == 0) {
+    if (warp == 3) {
         __syncwarp();
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
-                     "r"(kTmemCols)
+                     "r"(C::kTmemCols)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
@@ -80,179 +144,262 @@ hop_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    const uint32_t tmem_lane = tmem_base + ((uint32_t)(warp * 32) << 16);
 
-    constexpr uint32_t idesc_s = instr_desc(128, 0);
-    constexpr uint32_t idesc_o = instr_desc(D, 1);
+    // tiles this CTA processes: its work items (round robin over the grid) x gi heads each
+    const long long my_items = (a.total_items - blockIdx.x + gridDim.x - 1) / gridDim.x;
+    const uint32_t T = (uint32_t)(my_items * a.gi);
+    const uint32_t slab_tx = (uint32_t)a.rows * 128u;
 
-    const int r = warp * 32 + lane;                 // this thread's tile row = TMEM lane
-    const int seg = r / a.n;
-    const bool row_valid = r < a.rows;
-    const int c_lo = seg * a.n;
-    const int c_hi = a.causal ? r + 1 : c_lo + a.n; // visible key columns [c_lo, c_hi)
-    // columns any row of this warp needs (warp-uniform)
-    const int w_lo = ((warp * 32) / a.n) * a.n;
-    int w_hi = min(a.rows, ((warp * 32 + 31) / a.n + 1) * a.n);
-    if (a.causal) w_hi = min(w_hi, warp * 32 + 32);
-    const bool warp_valid = warp * 32 < a.rows;
-
-    bool ok = true;
-    uint32_t it = 0;
-    for (long long tile = blockIdx.x; tile < a.total_tiles; tile += gridDim.x, ++it) {
-        const uint32_t parity = it & 1u;
-        // tile -> (query head of the group, inner tile, outer tile, kv head, batch); the heads
-        // of a GQA group are adjacent so that their common K (and V) tile is hot in L2.
-        long long rest = tile;
-        const int hg = (int)(rest % a.g); rest /= a.g;
-        const int c_inner = (int)(rest % a.tiles_inner) * a.ci; rest /= a.tiles_inner;
-        const int c_outer = (int)(rest % a.tiles_outer) * a.co; rest /= a.tiles_outer;
-        const int kv_head = (int)rest;                              // b * H_kv + kvh
-        const int q_head = (kv_head / a.H_kv) * a.H + (kv_head % a.H_kv) * a.g + hg;
-        const int x_head = a.xin_is_kv ? kv_head : q_head;
-
-        if (tid == 0) {
-            const uint32_t slab_tx = (uint32_t)a.rows * 128u;
-            mbar_expect_tx(bar_qk, 2 * kHalves * slab_tx);
+    if (warp == 0) {
+        // =============================================================== TMA producer
+        if (lane == 0) {
+            uint32_t t = 0, it = 0;
+            // slots armed so far and the parity of the last phase armed on each (k 0-1, q 2-3, x 4-7)
+            uint32_t armed = 0, last_par = 0;
+            auto arm = [&](uint32_t bit, uint32_t parity) {
+                armed |= bit;
+                last_par = parity ? (last_par | bit) : (last_par & ~bit);
+            };
+            bool ok = true;
+            for (long long item = blockIdx.x; ok && item < a.total_items; item += gridDim.x, ++it) {
+                const ItemCoord c = decode_item(a, item);
+                const int ks = it & 1;
+                const uint32_t kpar = (it >> 1) & 1;
+                ok = mbar_wait_abortable(k_free(ks), kpar ^ 1, 0x10, abort_flag);
+                if (!ok) break;
+                mbar_expect_tx(k_full(ks), kHalves * slab_tx);
+                arm(1u << ks, kpar);
 #pragma unroll
-            for (int h = 0; h < kHalves; ++h) tma_load_5d(sQ + h * kSlabBytes, &map_q, bar_qk, 64 * h, 0, c_inner, c_outer, q_head);
+                for (int h = 0; h < kHalves; ++h)
+                    tma_load_5d(sK + ks * kTileBytes + h * kSlabBytes, &map_k, k_full(ks), 64 * h, 0, c.c_inner, c.c_outer, c.kv_head);
+                for (int j = 0; j < a.gi; ++j, ++t) {
+                    const int q_head = c.q_head0 + j;
+                    const int x_head = a.xin_is_kv ? c.kv_head : q_head;
+                    const int qs = t & 1;
+                    const uint32_t qpar = (t >> 1) & 1;
+                    ok = mbar_wait_abortable(q_free(qs), qpar ^ 1, 0x11, abort_flag);
+                    if (!ok) break;
+                    mbar_expect_tx(q_full(qs), kHalves * slab_tx);
+                    arm(4u << qs, qpar);
 #pragma unroll
-            for (int h = 0; h < kHalves; ++h) tma_load_5d(sK + h * kSlabBytes, &map_k, bar_qk, 64 * h, 0, c_inner, c_outer, kv_head);
-            mbar_expect_tx(bar_x, kHalves * slab_tx);
+                    for (int h = 0; h < kHalves; ++h)
+                        tma_load_5d(sQ + qs * kTileBytes + h * kSlabBytes, &map_q, q_full(qs), 64 * h, 0, c.c_inner, c.c_outer, q_head);
+                    const int xs = t % kNX;
+                    const uint32_t xpar = (t / kNX) & 1;
+                    ok = mbar_wait_abortable(x_free(xs), xpar ^ 1, 0x12, abort_flag);
+                    if (!ok) break;
+                    mbar_expect_tx(x_full(xs), kHalves * slab_tx);
+                    arm(16u << xs, xpar);
 #pragma unroll
-            for (int h = 0; h < kHalves; ++h) tma_load_5d(sX + h * kSlabBytes, &map_xin, bar_x, 64 * h, 0, c_inner, c_outer, x_head);
-
-            ok = mbar_wait(bar_qk, parity, 1);
-            if (ok) {
+                    for (int h = 0; h < kHalves; ++h)
+                        tma_load_5d(sX + xs * kTileBytes + h * kSlabBytes, &map_xin, x_full(xs), 64 * h, 0, c.c_inner, c.c_outer, x_head);
+                }
+            }
+            if (!ok) {
+                // leaving early: let the copies already issued land (bounded) before the CTA's
+                // shared memory is released
+                const unsigned long long t0 = globaltimer_ns();
+                for (int slot = 0; slot < 4 + kNX; ++slot) {
+                    if (!(armed & (1u << slot))) continue;
+                    const uint32_t bar = slot < 2 ? k_full(slot) : (slot < 4 ? q_full(slot - 2) : x_full(slot - 4));
+                    while (!mbar_try_wait(bar, (last_par >> slot) & 1u) && globaltimer_ns() - t0 < 10000000ull) {
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // =============================================================== MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc_s = instr_desc(128, 0);
+            constexpr uint32_t idesc_o = instr_desc(D, 1);
+            const int kblocks = (a.rows + 15) >> 4;
+            bool ok = true;
+            auto issue_o = [&](uint32_t u) -> bool {
+                // O(u)[128 x D] = P[128 x rows] X[rows x D]; X rows are keys (MN-major B operand)
+                const int xs = u % kNX;
+                if (!mbar_wait_abortable(p_full, u & 1, 0x21, abort_flag)) return false;
+                if (!mbar_wait_abortable(x_full(xs), (u / kNX) & 1, 0x22, abort_flag)) return false;
                 tc_fence_after();
-                // S[128 x 128] = Q[128 x D] K^T : D/16 instructions of K = 16
+                const uint32_t d_tmem = tmem_base + C::kColO + (u & 1) * 128;
+                const uint32_t x_base = sX + xs * kTileBytes;
+                for (int kb = 0; kb < kblocks; ++kb) {
+                    const uint32_t a_off = (kb >> 2) * kSlabBytes + (kb & 3) * 32;
+                    tc_mma_ss(d_tmem, smem_desc_sw128(sP + a_off, 16, 1024),
+                              smem_desc_sw128(x_base + kb * 2048, kSlabBytes, 1024), idesc_o, kb > 0);
+                }
+                tc_commit(o_full(u & 1));
+                tc_commit(p_free);
+                return true;
+            };
+            uint32_t it = 0, j = 0;
+            for (uint32_t t = 0; ok && t < T; ++t) {
+                const int ks = it & 1, qs = t & 1;
+                if (j == 0) ok = mbar_wait_abortable(k_full(ks), (it >> 1) & 1, 0x23, abort_flag);
+                if (ok) ok = mbar_wait_abortable(q_full(qs), (t >> 1) & 1, 0x24, abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+                // S(t)[128 x 128] = Q[128 x D] K^T : D/16 instructions of K = 16.  The S buffer is
+                // free: O(t-2) was issued after the softmax of tile t-2 had signalled p_full.
+                const uint32_t q_base = sQ + qs * kTileBytes, k_base = sK + ks * kTileBytes;
 #pragma unroll
                 for (int kb = 0; kb < D / 16; ++kb) {
                     const uint32_t off = (kb >> 2) * kSlabBytes + (kb & 3) * 32;
-                    tc_mma_ss(tmem_base, smem_desc_sw128(sQ + off, 16, 1024), smem_desc_sw128(sK + off, 16, 1024),
-                              idesc_s, kb > 0);
+                    tc_mma_ss(tmem_base + C::kColS + (t & 1) * 128, smem_desc_sw128(q_base + off, 16, 1024),
+                              smem_desc_sw128(k_base + off, 16, 1024), idesc_s, kb > 0);
                 }
-                tc_commit(bar_s);
+                tc_commit(s_full(t & 1));
+                tc_commit(q_free(qs));
+                if (++j == (uint32_t)a.gi) {
+                    tc_commit(k_free(ks));
+                    j = 0;
+                    ++it;
+                }
+                if (t > 0) ok = issue_o(t - 1);
             }
+            if (ok && T > 0) issue_o(T - 1);
         }
-        __syncwarp();
-        if (ok) ok = mbar_wait(bar_s, parity, 2);
-        ok = __all_sync(0xffffffffu, ok);          // keep every warp converged for the aligned TMEM ops
-        tc_fence_after();
+    } else if (warp == 2) {
+        // =============================================================== TMA store
+        if (lane == 0) {
+            uint32_t t = 0;
+            bool ok = true;
+            for (long long item = blockIdx.x; ok && item < a.total_items; item += gridDim.x) {
+                const ItemCoord c = decode_item(a, item);
+                for (int j = 0; j < a.gi; ++j, ++t) {
+                    const int xs = t % kNX;
+                    ok = mbar_wait_abortable(out_full(xs), (t / kNX) & 1, 0x30, abort_flag);
+                    if (!ok) break;
+#pragma unroll
+                    for (int h = 0; h < kHalves; ++h)
+                        tma_store_5d(&map_xout, sX + xs * kTileBytes + h * kSlabBytes, 64 * h, 0, c.c_inner, c.c_outer, c.q_head0 + j);
+                    tma_store_commit_and_wait_read();
+                    mbar_arrive(x_free(xs));
+                }
+            }
+            tma_store_wait_all();
+        }
+    } else if (warp >= 4) {
+        // =============================================================== softmax + epilogue
+        const int b = (warp - 4) >> 2;                  // tile parity this warpgroup serves
+        const int wq = warp & 3;                        // TMEM lane quarter of this warp
+        const uint32_t tmem_lane = tmem_base + ((uint32_t)(wq * 32) << 16);
+        const int r = wq * 32 + lane;                   // this thread's tile row = TMEM lane
+        const int seg = r / a.n;
+        const bool row_valid = r < a.rows;
+        const int c_lo = seg * a.n;
+        const int c_hi = a.causal ? r + 1 : c_lo + a.n; // visible key columns [c_lo, c_hi)
+        // columns any row of this warp needs (warp-uniform)
+        const int w_lo = ((wq * 32) / a.n) * a.n;
+        int w_hi = min(a.rows, ((wq * 32 + 31) / a.n + 1) * a.n);
+        if (a.causal) w_hi = min(w_hi, wq * 32 + 32);
+        const bool warp_valid = wq * 32 < a.rows;
+        const int nchunks = (a.rows + 31) >> 5;         // 32-column chunks of P the MMA reads
+        const uint32_t s_col = tmem_lane + C::kColS + b * 128, o_col = tmem_lane + C::kColO + b * 128;
 
-        // ---- softmax over the row's visible columns; P (un-normalised, bf16) -> sP
-        float row_sum = 1.f;
-        if (ok) {
+        bool ok = true;
+        for (uint32_t t = b; t < T; t += 2) {
+            const uint32_t par = (t >> 1) & 1;
+            ok = mbar_wait_abortable(s_full(b), par, 0x40, abort_flag);
+            ok = __all_sync(0xffffffffu, ok);           // keep the warp converged for the aligned TMEM ops
+            if (!ok) break;
+            tc_fence_after();
+
+            // ---- softmax over the row's visible columns; P (un-normalised, bf16) -> sP
             float m = -INFINITY;
             uint32_t v[32];
 #pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
+            for (int c = 0; c < nchunks; ++c) {
                 if (!(warp_valid && 32 * c < w_hi && 32 * c + 32 > w_lo)) continue;   // warp-uniform
-                tmem_ld32(tmem_lane + 32 * c, v);
+                tmem_ld32(s_col + 32 * c, v);
 #pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    const int col = 32 * c + j;
-                    const float s = __uint_as_float(v[j]);
+                for (int jj = 0; jj < 32; ++jj) {
+                    const int col = 32 * c + jj;
+                    const float s = __uint_as_float(v[jj]);
                     if (col >= c_lo && col < c_hi) m = fmaxf(m, s);
                 }
             }
             const float m_scaled = row_valid ? m * a.scale_log2 : 0.f;
             float sum = 0.f;
             const uint32_t row_base = sP + (uint32_t)r * 128u;
+            bool p_free_ok = false;
 #pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
+            for (int c = 0; c < nchunks; ++c) {
                 uint32_t pk[16];
                 if (warp_valid && 32 * c < w_hi && 32 * c + 32 > w_lo) {
-                    tmem_ld32(tmem_lane + 32 * c, v);
+                    tmem_ld32(s_col + 32 * c, v);
 #pragma unroll
-                    for (int j = 0; j < 32; j += 2) {
-                        const int col = 32 * c + j;
-                        float p0 = fast_exp2(__uint_as_float(v[j]) * a.scale_log2 - m_scaled);
-                        float p1 = fast_exp2(__uint_as_float(v[j + 1]) * a.scale_log2 - m_scaled);
+                    for (int jj = 0; jj < 32; jj += 2) {
+                        const int col = 32 * c + jj;
+                        float p0 = fast_exp2(__uint_as_float(v[jj]) * a.scale_log2 - m_scaled);
+                        float p1 = fast_exp2(__uint_as_float(v[jj + 1]) * a.scale_log2 - m_scaled);
                         p0 = (row_valid && col >= c_lo && col < c_hi) ? p0 : 0.f;
                         p1 = (row_valid && col + 1 >= c_lo && col + 1 < c_hi) ? p1 : 0.f;
                         const uint32_t w = pack_bf16x2(p0, p1);
-                        pk[j >> 1] = w;
+                        pk[jj >> 1] = w;
                         sum += __uint_as_float(w << 16) + __uint_as_float(w & 0xFFFF0000u);
                     }
                 } else {
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) pk[j] = 0u;
+                    for (int jj = 0; jj < 16; ++jj) pk[jj] = 0u;
+                }
+                if (!p_free_ok) {
+                    // the P buffer is shared by both warpgroups: wait until O(t-1) has consumed it
+                    ok = mbar_wait_abortable(p_free, (t & 1) ^ 1, 0x41, abort_flag);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    p_free_ok = true;
                 }
                 const uint32_t slab = row_base + (uint32_t)(c >> 1) * kSlabBytes;
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     const uint32_t chunk = (uint32_t)(((c & 1) * 4 + i) ^ (r & 7));
-                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(slab + chunk * 16), "r"(pk[4 * i]),
-                                 "r"(pk[4 * i + 1]), "r"(pk[4 * i + 2]), "r"(pk[4 * i + 3])
-                                 : "memory");
+                    st_shared_v4(slab + chunk * 16, pk[4 * i], pk[4 * i + 1], pk[4 * i + 2], pk[4 * i + 3]);
                 }
             }
-            row_sum = row_valid ? sum : 1.f;
-        }
-        fence_proxy_async_smem();
-        tc_fence_before();
-        __syncthreads();
+            if (!ok) break;
+            const float inv = row_valid ? 1.f / sum : 1.f;
+            fence_proxy_async_smem();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(p_full);
 
-        if (tid == 0 && ok) {
+            // ---- epilogue: O / rowsum -> bf16 -> X slot (same swizzled box layout) -> store warp
+            const int xs = t % kNX;
+            ok = mbar_wait_abortable(o_full(b), par, 0x42, abort_flag);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
             tc_fence_after();
-            ok = mbar_wait(bar_x, parity, 3);
-            if (ok) {
-                // O[128 x D] = P[128 x rows] X[rows x D]; X rows are keys (MN-major B operand)
-                const int kblocks = (a.rows + 15) >> 4;
-                for (int kb = 0; kb < kblocks; ++kb) {
-                    const uint32_t a_off = (kb >> 2) * kSlabBytes + (kb & 3) * 32;
-                    tc_mma_ss(tmem_base + kOCol, smem_desc_sw128(sP + a_off, 16, 1024),
-                              smem_desc_sw128(sX + kb * 2048, kSlabBytes, 1024), idesc_o, kb > 0);
-                }
-                tc_commit(bar_o);
-            }
-        }
-        __syncwarp();
-        if (ok) ok = mbar_wait(bar_o, parity, 4);
-        ok = __all_sync(0xffffffffu, ok);
-        tc_fence_after();
-
-        // ---- epilogue: O / rowsum -> bf16 -> sX (same swizzled box layout) -> TMA store
-        if (ok && warp_valid) {
-            const float inv = 1.f / row_sum;
-            uint32_t v[32];
+            if (warp_valid) {
+                const uint32_t x_row = sX + xs * kTileBytes + (uint32_t)r * 128u;
 #pragma unroll 1
-            for (int c = 0; c < D / 32; ++c) {
-                tmem_ld32(tmem_lane + kOCol + 32 * c, v);   // whole warp, rows beyond `rows` discard it
-                uint32_t pk[16];
+                for (int c = 0; c < D / 32; ++c) {
+                    tmem_ld32(o_col + 32 * c, v);       // whole warp; rows beyond `rows` discard it
+                    uint32_t pk[16];
 #pragma unroll
-                for (int j = 0; j < 32; j += 2)
-                    pk[j >> 1] = pack_bf16x2(__uint_as_float(v[j]) * inv, __uint_as_float(v[j + 1]) * inv);
-                const uint32_t slab = sX + (uint32_t)(c >> 1) * kSlabBytes + (uint32_t)r * 128u;
-                if (row_valid) {
+                    for (int jj = 0; jj < 32; jj += 2)
+                        pk[jj >> 1] = pack_bf16x2(__uint_as_float(v[jj]) * inv, __uint_as_float(v[jj + 1]) * inv);
+                    const uint32_t slab = x_row + (uint32_t)(c >> 1) * kSlabBytes;
+                    if (row_valid) {
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const uint32_t chunk = (uint32_t)(((c & 1) * 4 + i) ^ (r & 7));
-                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(slab + chunk * 16),
-                                     "r"(pk[4 * i]), "r"(pk[4 * i + 1]), "r"(pk[4 * i + 2]), "r"(pk[4 * i + 3])
-                                     : "memory");
+                        for (int i = 0; i < 4; ++i) {
+                            const uint32_t chunk = (uint32_t)(((c & 1) * 4 + i) ^ (r & 7));
+                            st_shared_v4(slab + chunk * 16, pk[4 * i], pk[4 * i + 1], pk[4 * i + 2], pk[4 * i + 3]);
+                        }
                     }
                 }
             }
+            fence_proxy_async_smem();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(out_full(xs));
         }
-        fence_proxy_async_smem();
-        tc_fence_before();
-        const int all_ok = __syncthreads_and(ok ? 1 : 0);
-        if (tid == 0 && all_ok) {
-#pragma unroll
-            for (int h = 0; h < kHalves; ++h) tma_store_5d(&map_xout, sX + h * kSlabBytes, 64 * h, 0, c_inner, c_outer, q_head);
-            tma_store_commit_and_wait_read();
-        }
-        __syncthreads();
-        if (!all_ok) break;
     }
 
-    if (tid == 0) tma_store_wait_all();
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) {
+    if (warp == 3) {
         __syncwarp();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(C::kTmemCols) : "memory");
     }
 }
 
@@ -305,13 +452,6 @@ int launch_d(const Problem &pb, const HopDesc &hd, const void *xin, int xin_head
     if ((rc = make_hop_map(&mxi, xin, pb.B * xin_heads, pb.N, D, hd, 2)) != TA_OK) return rc;
     if ((rc = make_hop_map(&mxo, xout, pb.B * pb.H, pb.N, D, hd, 2)) != TA_OK) return rc;
 
-    TcArgs a;
-    a.n = hd.n; a.rows = hd.rows; a.ci = hd.ci; a.co = hd.co; a.causal = pb.causal;
-    a.g = pb.H / pb.H_kv; a.H = pb.H; a.H_kv = pb.H_kv; a.xin_is_kv = xin_heads != pb.H ? 1 : 0;
-    a.tiles_inner = hd.tiles_inner; a.tiles_outer = hd.tiles_outer;
-    a.total_tiles = (long long)pb.B * pb.H * hd.tiles_inner * hd.tiles_outer;
-    a.scale_log2 = pb.scale * 1.4426950408889634f;
-
     static int num_sms = 0;
     if (num_sms == 0) {
         int dev = 0;
@@ -319,16 +459,29 @@ int launch_d(const Problem &pb, const HopDesc &hd, const void *xin, int xin_head
         if (cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || num_sms <= 0)
             num_sms = 148;
     }
-    constexpr size_t smem = 3 * (size_t)(D / 64) * kTileRows * 128 + 1024 /*alignment slack*/ + 64 /*barriers*/;
-    auto kern = hop_tc_kernel<D>;
+    TcArgs a;
+    a.n = hd.n; a.rows = hd.rows; a.ci = hd.ci; a.co = hd.co; a.causal = pb.causal;
+    a.g = pb.H / pb.H_kv; a.H = pb.H; a.H_kv = pb.H_kv; a.xin_is_kv = xin_heads != pb.H ? 1 : 0;
+    a.tiles_inner = hd.tiles_inner; a.tiles_outer = hd.tiles_outer;
+    // A work item covers gi query heads of one GQA group on one tile position (they share the
+    // K tile); groups are split across items only when there are too few items to fill the GPU.
+    const long long positions = (long long)pb.B * pb.H_kv * hd.tiles_inner * hd.tiles_outer;
+    a.hsplit = 1;
+    for (int d = 2; d <= a.g && positions * a.hsplit < 2ll * num_sms; ++d)
+        if (a.g % d == 0) a.hsplit = d;
+    a.gi = a.g / a.hsplit;
+    a.total_items = positions * a.hsplit;
+    a.scale_log2 = pb.scale * 1.4426950408889634f;
+
+    constexpr size_t smem = PipeCfg<D>::kSmemBytes;
+    auto kern = hop_pipe_kernel<D>;
     static bool configured = false;
     if (!configured) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
             return TA_ERR_CUDA;
         configured = true;
     }
-    const long long max_ctas = 2ll * num_sms;
-    const unsigned grid = (unsigned)(a.total_tiles < max_ctas ? a.total_tiles : max_ctas);
+    const unsigned grid = (unsigned)(a.total_items < num_sms ? a.total_items : num_sms);
     kern<<<grid, kThreads, smem, pb.stream>>>(mq, mk, mxi, mxo, a);
     count_launch();
     return cudaPeekAtLastError() == cudaSuccess ? TA_OK : TA_ERR_CUDA;
