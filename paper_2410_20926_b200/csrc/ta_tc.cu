@@ -9,10 +9,11 @@
 // layout of tcgen05.mma for Q and K, and the MN-major one for the value tile.
 //
 // Per tile:  S = Q K^T (tcgen05.mma, fp32 in TMEM)  ->  block-diagonal + causal mask, row softmax
-// in fp32 registers (tcgen05.ld), un-normalised weights rounded to bf16 into shared memory  ->
-// O = P X (tcgen05.mma, fp32 in TMEM)  ->  O / rowsum -> bf16 -> shared memory (over the X tile)
-// ->  TMA store to the same strided rows.  Because a tile owns whole segments, the value tensor
-// is updated in place.
+// in fp32 registers (tcgen05.ld), un-normalised weights rounded to bf16 and written back to
+// tensor memory over S (tcgen05.st)  ->  O = P X (tcgen05.mma with the A operand in TMEM, fp32
+// accumulator in TMEM)  ->  O / rowsum -> bf16 -> shared memory (over the X tile)  ->  TMA store
+// to the same strided rows.  Because a tile owns whole segments, the value tensor is updated
+// in place.  Shared memory holds only operand tiles: K x 2, Q x 2, X x 3 (D = 128).
 //
 // The kernel is persistent (one CTA per SM) and warp-specialised, so that the HBM traffic of
 // the next tiles overlaps the arithmetic of the current one:
@@ -45,16 +46,15 @@ struct PipeCfg {
     static constexpr int kHalves = D / 64;                     // 64-column (128-byte) slabs per row
     static constexpr uint32_t kSlabBytes = kTileRows * 128;    // one [128 rows][64 cols] bf16 slab
     static constexpr uint32_t kTileBytes = kHalves * kSlabBytes;
-    static constexpr uint32_t kPBytes = 2 * kSlabBytes;        // P: 128 x 128 bf16
-    static constexpr int kNX = D == 128 ? 2 : 4;               // X ring (value tile in, output tile out)
+    static constexpr int kNX = D == 128 ? 3 : 6;               // X ring (value tile in, output tile out)
     static constexpr uint32_t kOffK = 0;
     static constexpr uint32_t kOffQ = kOffK + kNK * kTileBytes;
-    static constexpr uint32_t kOffP = kOffQ + kNQ * kTileBytes;
-    static constexpr uint32_t kOffX = kOffP + kPBytes;
+    static constexpr uint32_t kOffX = kOffQ + kNQ * kTileBytes;
     static constexpr uint32_t kOffBar = kOffX + kNX * kTileBytes;
     static constexpr int kNumBars = 2 * kNK + 2 * kNQ + 3 * kNX + 2 + 2 + 2;
     static constexpr uint32_t kSmemBytes = kOffBar + kNumBars * 8 + 16 + 1024 /*alignment slack*/;
-    static constexpr uint32_t kTmemCols = 512;                 // S: 2 x 128 columns, O: 2 x 128
+    // S: 2 x 128 fp32 columns (P, bf16, is written over the first 64 columns of its S), O: 2 x 128
+    static constexpr uint32_t kTmemCols = 512;
     static constexpr uint32_t kColS = 0, kColO = 256;
 };
 
@@ -99,7 +99,7 @@ hop_pipe_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const uint32_t s0 = smem_u32(smem);
-    const uint32_t sK = s0 + C::kOffK, sQ = s0 + C::kOffQ, sP = s0 + C::kOffP, sX = s0 + C::kOffX;
+    const uint32_t sK = s0 + C::kOffK, sQ = s0 + C::kOffQ, sX = s0 + C::kOffX;
     const uint32_t bar0 = s0 + C::kOffBar;
     // barrier indices
     auto k_full = [&](int i) { return bar0 + 8u * (uint32_t)i; };
@@ -113,7 +113,7 @@ hop_pipe_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     constexpr int kB1 = kB0 + 3 * kNX;
     auto s_full = [&](int i) { return bar0 + 8u * (uint32_t)(kB1 + i); };
     auto o_full = [&](int i) { return bar0 + 8u * (uint32_t)(kB1 + 2 + i); };
-    const uint32_t p_full = bar0 + 8u * (uint32_t)(kB1 + 4), p_free = bar0 + 8u * (uint32_t)(kB1 + 5);
+    auto p_full = [&](int i) { return bar0 + 8u * (uint32_t)(kB1 + 4 + i); };
     uint32_t *tmem_slot = (uint32_t *)(smem + C::kOffBar + C::kNumBars * 8);
     volatile uint32_t *abort_flag = tmem_slot + 1;
 
@@ -126,9 +126,7 @@ hop_pipe_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         for (int i = 0; i < kNK; ++i) { mbar_init(k_full(i), 1); mbar_init(k_free(i), 1); }
         for (int i = 0; i < kNQ; ++i) { mbar_init(q_full(i), 1); mbar_init(q_free(i), 1); }
         for (int i = 0; i < kNX; ++i) { mbar_init(x_full(i), 1); mbar_init(x_free(i), 1); mbar_init(out_full(i), 4); }
-        for (int i = 0; i < 2; ++i) { mbar_init(s_full(i), 1); mbar_init(o_full(i), 1); }
-        mbar_init(p_full, 4);
-        mbar_init(p_free, 1);
+        for (int i = 0; i < 2; ++i) { mbar_init(s_full(i), 1); mbar_init(o_full(i), 1); mbar_init(p_full(i), 4); }
         *abort_flag = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -215,20 +213,19 @@ hop_pipe_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             const int kblocks = (a.rows + 15) >> 4;
             bool ok = true;
             auto issue_o = [&](uint32_t u) -> bool {
-                // O(u)[128 x D] = P[128 x rows] X[rows x D]; X rows are keys (MN-major B operand)
+                // O(u)[128 x D] = P[128 x rows] X[rows x D]; P from tensor memory (16 keys = 8
+                // columns per instruction), X rows are keys (MN-major B operand)
                 const int xs = u % kNX;
-                if (!mbar_wait_abortable(p_full, u & 1, 0x21, abort_flag)) return false;
+                if (!mbar_wait_abortable(p_full(u & 1), (u >> 1) & 1, 0x21, abort_flag)) return false;
                 if (!mbar_wait_abortable(x_full(xs), (u / kNX) & 1, 0x22, abort_flag)) return false;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + C::kColO + (u & 1) * 128;
+                const uint32_t p_tmem = tmem_base + C::kColS + (u & 1) * 128;
                 const uint32_t x_base = sX + xs * kTileBytes;
-                for (int kb = 0; kb < kblocks; ++kb) {
-                    const uint32_t a_off = (kb >> 2) * kSlabBytes + (kb & 3) * 32;
-                    tc_mma_ss(d_tmem, smem_desc_sw128(sP + a_off, 16, 1024),
-                              smem_desc_sw128(x_base + kb * 2048, kSlabBytes, 1024), idesc_o, kb > 0);
-                }
+                for (int kb = 0; kb < kblocks; ++kb)
+                    tc_mma_ts(d_tmem, p_tmem + kb * 8, smem_desc_sw128(x_base + kb * 2048, kSlabBytes, 1024), idesc_o,
+                              kb > 0);
                 tc_commit(o_full(u & 1));
-                tc_commit(p_free);
                 return true;
             };
             uint32_t it = 0, j = 0;
@@ -238,8 +235,8 @@ hop_pipe_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 if (ok) ok = mbar_wait_abortable(q_full(qs), (t >> 1) & 1, 0x24, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
-                // S(t)[128 x 128] = Q[128 x D] K^T : D/16 instructions of K = 16.  The S buffer is
-                // free: O(t-2) was issued after the softmax of tile t-2 had signalled p_full.
+                // S(t)[128 x 128] = Q[128 x D] K^T : D/16 instructions of K = 16.  Its buffer last
+                // held P(t-2), the operand of O(t-2), which was issued earlier and executes first.
                 const uint32_t q_base = sQ + qs * kTileBytes, k_base = sK + ks * kTileBytes;
 #pragma unroll
                 for (int kb = 0; kb < D / 16; ++kb) {
@@ -304,7 +301,8 @@ hop_pipe_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             if (!ok) break;
             tc_fence_after();
 
-            // ---- softmax over the row's visible columns; P (un-normalised, bf16) -> sP
+            // ---- softmax over the row's visible columns; P (un-normalised, bf16) -> tensor memory,
+            // two keys per 32-bit column, over the S columns already consumed
             float m = -INFINITY;
             uint32_t v[32];
 #pragma unroll 1
@@ -320,8 +318,6 @@ hop_pipe_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             }
             const float m_scaled = row_valid ? m * a.scale_log2 : 0.f;
             float sum = 0.f;
-            const uint32_t row_base = sP + (uint32_t)r * 128u;
-            bool p_free_ok = false;
 #pragma unroll 1
             for (int c = 0; c < nchunks; ++c) {
                 uint32_t pk[16];
@@ -342,26 +338,13 @@ hop_pipe_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 #pragma unroll
                     for (int jj = 0; jj < 16; ++jj) pk[jj] = 0u;
                 }
-                if (!p_free_ok) {
-                    // the P buffer is shared by both warpgroups: wait until O(t-1) has consumed it
-                    ok = mbar_wait_abortable(p_free, (t & 1) ^ 1, 0x41, abort_flag);
-                    ok = __all_sync(0xffffffffu, ok);
-                    if (!ok) break;
-                    p_free_ok = true;
-                }
-                const uint32_t slab = row_base + (uint32_t)(c >> 1) * kSlabBytes;
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const uint32_t chunk = (uint32_t)(((c & 1) * 4 + i) ^ (r & 7));
-                    st_shared_v4(slab + chunk * 16, pk[4 * i], pk[4 * i + 1], pk[4 * i + 2], pk[4 * i + 3]);
-                }
+                tmem_st16(s_col + 16 * c, pk);
             }
-            if (!ok) break;
+            tmem_st_wait();
             const float inv = row_valid ? 1.f / sum : 1.f;
-            fence_proxy_async_smem();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(p_full);
+            if (lane == 0) mbar_arrive(p_full(b));
 
             // ---- epilogue: O / rowsum -> bf16 -> X slot (same swizzled box layout) -> store warp
             const int xs = t % kNX;
