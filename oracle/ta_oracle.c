@@ -25,6 +25,17 @@
  * Q and K are the same un-updated projections in every hop; only O is carried.
  * The mask M_i removes entries from the softmax (their weight is exactly 0);
  * the causal M_i keeps key position u <= query position t along mode i.
+ *
+ * Tensorized positional encoding (Section 3.2, "Tensorized Positional Encoding"): the
+ * position of a token is the vector of its coordinates (j_1..j_m) and, following Llama,
+ * RoPE encodes it.  The paper gives no formula (its appendix on this is not in the text);
+ * the reading implemented here, when rope_base > 0: in hop i the queries and keys are
+ * rotated by the token's coordinate j_i along the dimension the hop attends over, with
+ * the Llama pairing of feature c with c + D/2 and angle j_i * rope_base^(-2c/D),
+ *     x'_c       = x_c cos a - x_{c+D/2} sin a
+ *     x'_{c+D/2} = x_{c+D/2} cos a + x_c sin a ,       c = 0 .. D/2-1,
+ * so that a hop's scores depend on the relative position t - u along that dimension.
+ * The value tensor is never rotated.
  */
 #include <math.h>
 #include <stdlib.h>
@@ -69,6 +80,25 @@ static long hop_stride(const int *dims, int ndims, int i)
     return s;
 }
 
+/* y[j] = R(p_j) x[j] with p_j = (j / stride) mod n, the coordinate of token j along the hop's
+ * dimension; sign = +1 rotates, -1 applies the transpose (inverse) rotation. */
+static void rope_rotate(const double *x, double *y, long N, int D, long stride, int n,
+                        double base, int sign)
+{
+    const int half = D / 2;
+    for (long j = 0; j < N; ++j) {
+        const double p = (double)((j / stride) % n);
+        for (int c = 0; c < half; ++c) {
+            const double a = sign * p * pow(base, -2.0 * c / D);
+            const double cs = cos(a), sn = sin(a);
+            const double x1 = x[j * D + c], x2 = x[j * D + c + half];
+            y[j * D + c] = x1 * cs - x2 * sn;
+            y[j * D + c + half] = x2 * cs + x1 * sn;
+        }
+        if (D & 1) y[j * D + D - 1] = x[j * D + D - 1];
+    }
+}
+
 /*
  * One head, forward.  q,k,v: [N][D] fp64 (k,v are the head's KV head).
  * out: [N][D].  xs (optional, may be NULL): [(ndims+1)][N][D], receives
@@ -76,9 +106,9 @@ static long hop_stride(const int *dims, int ndims, int i)
  * backward pass below needs.
  * Returns 0, or -1 on bad arguments / allocation failure.
  */
-int ta_oracle_forward_head(const double *q, const double *k, const double *v, double *out,
-                           long N, int D, const int *dims, int ndims, int causal,
-                           double scale, double *xs)
+static int forward_head_impl(const double *q, const double *k, const double *v, double *out,
+                             long N, int D, const int *dims, int ndims, int causal,
+                             double scale, double rope_base, double *xs)
 {
     if (!q || !k || !v || !out || !dims || ndims < 1 || N < 1 || D < 1) return -1;
     long prod = 1;
@@ -87,15 +117,26 @@ int ta_oracle_forward_head(const double *q, const double *k, const double *v, do
 
     size_t bytes = (size_t)N * D * sizeof(double);
     double *cur = (double *)malloc(bytes), *nxt = (double *)malloc(bytes);
-    if (!cur || !nxt) { free(cur); free(nxt); return -1; }
+    double *qr = NULL, *kr = NULL;                          /* rotated q, k of the current hop */
+    if (rope_base > 0.0) { qr = (double *)malloc(bytes); kr = (double *)malloc(bytes); }
+    if (!cur || !nxt || (rope_base > 0.0 && (!qr || !kr))) {
+        free(cur); free(nxt); free(qr); free(kr);
+        return -1;
+    }
     memcpy(cur, v, bytes);                                  /* Initialize O = V */
     if (xs) memcpy(xs, v, bytes);
 
     int fail = 0;
+    const double *q_in = q, *k_in = k;
     for (int i = 0; i < ndims; ++i) {                       /* for i = 0 to m-1 */
         const int n = dims[i];
         const long s = hop_stride(dims, ndims, i);
         const long nseg = N / n;
+        if (rope_base > 0.0) {                              /* positions along dimension i */
+            rope_rotate(q_in, qr, N, D, s, n, rope_base, +1);
+            rope_rotate(k_in, kr, N, D, s, n, rope_base, +1);
+            q = qr; k = kr;
+        }
         #pragma omp parallel
         {
             double *P = (double *)malloc((size_t)n * n * sizeof(double));
@@ -127,8 +168,24 @@ int ta_oracle_forward_head(const double *q, const double *k, const double *v, do
         if (xs) memcpy(xs + (size_t)(i + 1) * N * D, cur, bytes);
     }
     if (!fail) memcpy(out, cur, bytes);
-    free(cur); free(nxt);
+    free(cur); free(nxt); free(qr); free(kr);
     return fail ? -1 : 0;
+}
+
+int ta_oracle_forward_head(const double *q, const double *k, const double *v, double *out,
+                           long N, int D, const int *dims, int ndims, int causal,
+                           double scale, double *xs)
+{
+    return forward_head_impl(q, k, v, out, N, D, dims, ndims, causal, scale, 0.0, xs);
+}
+
+/* As above with the tensorized positional encoding (rope_base > 0, e.g. 10000). */
+int ta_oracle_forward_head_rope(const double *q, const double *k, const double *v, double *out,
+                                long N, int D, const int *dims, int ndims, int causal,
+                                double scale, double rope_base, double *xs)
+{
+    if (!(rope_base > 0.0)) return -1;
+    return forward_head_impl(q, k, v, out, N, D, dims, ndims, causal, scale, rope_base, xs);
 }
 
 /*
@@ -142,11 +199,13 @@ int ta_oracle_forward_head(const double *q, const double *k, const double *v, do
  *     dV   = G_0
  * xs: [(ndims+1)][N][D] as written by ta_oracle_forward_head.
  * dq, dk, dv: [N][D], overwritten (the caller sums dk, dv over a GQA group).
+ * With rope_base > 0 each hop works on its rotated queries and keys q' = R q, k' = R k and
+ * the gradients it finds for them are rotated back (dq += R^T dq') before they are summed.
  */
-int ta_oracle_backward_head(const double *q, const double *k, const double *xs,
-                            const double *dout, double *dq, double *dk, double *dv,
-                            long N, int D, const int *dims, int ndims, int causal,
-                            double scale)
+static int backward_head_impl(const double *q, const double *k, const double *xs,
+                              const double *dout, double *dq, double *dk, double *dv,
+                              long N, int D, const int *dims, int ndims, int causal,
+                              double scale, double rope_base)
 {
     if (!q || !k || !xs || !dout || !dq || !dk || !dv || !dims || ndims < 1) return -1;
     long prod = 1;
@@ -155,17 +214,36 @@ int ta_oracle_backward_head(const double *q, const double *k, const double *xs,
 
     size_t bytes = (size_t)N * D * sizeof(double);
     double *g = (double *)malloc(bytes), *gn = (double *)malloc(bytes);
-    if (!g || !gn) { free(g); free(gn); return -1; }
+    double *qr = NULL, *kr = NULL, *dqr = NULL, *dkr = NULL, *tmp_rot = NULL;
+    const int rope = rope_base > 0.0;
+    if (rope) {
+        qr = (double *)malloc(bytes); kr = (double *)malloc(bytes);
+        dqr = (double *)malloc(bytes); dkr = (double *)malloc(bytes);
+        tmp_rot = (double *)malloc(bytes);
+    }
+    if (!g || !gn || (rope && (!qr || !kr || !dqr || !dkr || !tmp_rot))) {
+        free(g); free(gn); free(qr); free(kr); free(dqr); free(dkr); free(tmp_rot);
+        return -1;
+    }
     memcpy(g, dout, bytes);
     memset(dq, 0, bytes);
     memset(dk, 0, bytes);
 
     int fail = 0;
+    const double *q_in = q, *k_in = k;
+    double *dq_out = dq, *dk_out = dk;
     for (int i = ndims - 1; i >= 0; --i) {
         const int n = dims[i];
         const long s = hop_stride(dims, ndims, i);
         const long nseg = N / n;
         const double *x = xs + (size_t)i * N * D;           /* X_i: the hop's input */
+        if (rope) {
+            rope_rotate(q_in, qr, N, D, s, n, rope_base, +1);
+            rope_rotate(k_in, kr, N, D, s, n, rope_base, +1);
+            q = qr; k = kr;
+            memset(dqr, 0, bytes); memset(dkr, 0, bytes);
+            dq = dqr; dk = dkr;                             /* this hop's dq', dk' */
+        }
         #pragma omp parallel
         {
             double *P = (double *)malloc((size_t)n * n * sizeof(double));
@@ -219,11 +297,35 @@ int ta_oracle_backward_head(const double *q, const double *k, const double *xs,
             free(P); free(dS);
         }
         if (fail) break;
+        if (rope) {                                         /* dq += R^T dq', dk += R^T dk' */
+            rope_rotate(dqr, tmp_rot, N, D, s, n, rope_base, -1);
+            for (long e = 0; e < N * D; ++e) dq_out[e] += tmp_rot[e];
+            rope_rotate(dkr, tmp_rot, N, D, s, n, rope_base, -1);
+            for (long e = 0; e < N * D; ++e) dk_out[e] += tmp_rot[e];
+        }
         double *tmp = g; g = gn; gn = tmp;
     }
     if (!fail) memcpy(dv, g, bytes);
-    free(g); free(gn);
+    free(g); free(gn); free(qr); free(kr); free(dqr); free(dkr); free(tmp_rot);
     return fail ? -1 : 0;
+}
+
+int ta_oracle_backward_head(const double *q, const double *k, const double *xs,
+                            const double *dout, double *dq, double *dk, double *dv,
+                            long N, int D, const int *dims, int ndims, int causal,
+                            double scale)
+{
+    return backward_head_impl(q, k, xs, dout, dq, dk, dv, N, D, dims, ndims, causal, scale, 0.0);
+}
+
+int ta_oracle_backward_head_rope(const double *q, const double *k, const double *xs,
+                                 const double *dout, double *dq, double *dk, double *dv,
+                                 long N, int D, const int *dims, int ndims, int causal,
+                                 double scale, double rope_base)
+{
+    if (!(rope_base > 0.0)) return -1;
+    return backward_head_impl(q, k, xs, dout, dq, dk, dv, N, D, dims, ndims, causal, scale,
+                              rope_base);
 }
 
 int ta_oracle_num_threads(void)

@@ -19,6 +19,14 @@ dimensions are no-ops; C route == dense route; separable (Kronecker) inputs give
 Q=0 gives (prefix-)box means; causality probe; the row-major reshape pin of Section 4.4
 (one step on the first dimension of {32,32,32} is 1024 tokens); GQA equals explicit KV
 repetition; backward equals central finite differences and dV = A_eff^T dout.
+
+Tensorized positional encoding (``rope_base``): in hop i queries and keys are rotated (RoPE,
+Llama pairing c <-> c + D/2) by the token's coordinate along dimension i.  The C route
+rotates the vectors; the dense route never rotates anything -- it writes the score in the
+relative form Re sum_c zq_c conj(zk_c) exp(i (p_j - p_k) theta_c) with complex features
+z_c = x_c + i x_{c+D/2} -- so the two share neither code nor formula.  Extra pins: a third,
+matrix-form implementation for one dimension; closed-form scores sin / cos of the relative
+position for unit-vector inputs (fixes pairing, sign and the frequency ladder).
 """
 from __future__ import annotations
 
@@ -47,6 +55,14 @@ def _lib():
         lib.ta_oracle_backward_head.argtypes = [dp, dp, dp, dp, dp, dp, dp, ctypes.c_long,
                                                 ctypes.c_int, ip, ctypes.c_int, ctypes.c_int,
                                                 ctypes.c_double]
+        lib.ta_oracle_forward_head_rope.restype = ctypes.c_int
+        lib.ta_oracle_forward_head_rope.argtypes = [dp, dp, dp, dp, ctypes.c_long, ctypes.c_int, ip,
+                                                    ctypes.c_int, ctypes.c_int, ctypes.c_double,
+                                                    ctypes.c_double, dp]
+        lib.ta_oracle_backward_head_rope.restype = ctypes.c_int
+        lib.ta_oracle_backward_head_rope.argtypes = [dp, dp, dp, dp, dp, dp, dp, ctypes.c_long,
+                                                     ctypes.c_int, ip, ctypes.c_int, ctypes.c_int,
+                                                     ctypes.c_double, ctypes.c_double]
         lib.ta_oracle_num_threads.restype = ctypes.c_int
         _LIB = lib
     return _LIB
@@ -81,13 +97,24 @@ def _check(q, k, v, dims):
     return B, H, Hkv, N, D, dims
 
 
+def _fwd_head(lib, qh, kh, vh, out, N, D, cdims, m, causal, scale, rope_base, xs):
+    if rope_base:
+        return lib.ta_oracle_forward_head_rope(_dptr(qh), _dptr(kh), _dptr(vh), _dptr(out), N, D,
+                                               cdims, m, int(bool(causal)), scale,
+                                               float(rope_base), _dptr(xs) if xs is not None else None)
+    return lib.ta_oracle_forward_head(_dptr(qh), _dptr(kh), _dptr(vh), _dptr(out), N, D, cdims, m,
+                                      int(bool(causal)), scale, _dptr(xs) if xs is not None else None)
+
+
 def forward(q, k, v, dims, causal: bool, scale: float | None = None, heads=None,
-            return_xs: bool = False):
+            return_xs: bool = False, rope_base: float | None = None):
     """Algorithm 1 for every (or the listed) head, fp64.
 
     q: [B,H,N,D]; k, v: [B,H_kv,N,D] (any float dtype; converted head by head to fp64).
     Query head h uses KV head h // (H/H_kv).  scale defaults to 1/sqrt(D) (Eq. 4).
     heads: optional list of (b, h) pairs; then the result is [len(heads), N, D].
+    rope_base: None / 0 for no positional encoding, else the RoPE base (Llama: 10000) of the
+    tensorized positional encoding (hop i rotates q, k by the coordinate along dimension i).
     Returns out [B,H,N,D] fp64 (and, with return_xs, the list of per-head [m+1,N,D]
     value tensors X_0=V ... X_m=out keyed like the output).
     """
@@ -102,9 +129,8 @@ def forward(q, k, v, dims, causal: bool, scale: float | None = None, heads=None,
     for idx, (b, h) in enumerate(pairs):
         qh, kh, vh = _f64(q[b, h]), _f64(k[b, h // g]), _f64(v[b, h // g])
         xs = np.empty((len(dims) + 1, N, D), dtype=np.float64) if return_xs else None
-        rc = lib.ta_oracle_forward_head(_dptr(qh), _dptr(kh), _dptr(vh), _dptr(out[idx]),
-                                        N, D, cdims, len(dims), int(bool(causal)), scale,
-                                        _dptr(xs) if return_xs else None)
+        rc = _fwd_head(lib, qh, kh, vh, out[idx], N, D, cdims, len(dims), causal, scale,
+                       rope_base, xs)
         if rc != 0:
             raise RuntimeError("ta_oracle_forward_head failed")
         if return_xs:
@@ -114,7 +140,8 @@ def forward(q, k, v, dims, causal: bool, scale: float | None = None, heads=None,
     return (out, xs_all) if return_xs else out
 
 
-def backward(dout, q, k, v, dims, causal: bool, scale: float | None = None, groups=None):
+def backward(dout, q, k, v, dims, causal: bool, scale: float | None = None, groups=None,
+             rope_base: float | None = None):
     """Gradients of sum(out * dout) w.r.t. q, k, v (fp64), GQA groups summed into dk, dv.
 
     groups: optional list of (b, kv_head) pairs; then only those KV heads and their query
@@ -136,16 +163,21 @@ def backward(dout, q, k, v, dims, causal: bool, scale: float | None = None, grou
             qh = _f64(q[b, h])
             o = np.empty((N, D))
             xs = np.empty((len(dims) + 1, N, D))
-            rc = lib.ta_oracle_forward_head(_dptr(qh), _dptr(kh), _dptr(vh), _dptr(o), N, D,
-                                            cdims, len(dims), int(bool(causal)), scale,
-                                            _dptr(xs))
+            rc = _fwd_head(lib, qh, kh, vh, o, N, D, cdims, len(dims), causal, scale, rope_base, xs)
             if rc != 0:
                 raise RuntimeError("ta_oracle_forward_head failed")
             dqh, dkh, dvh = np.empty((N, D)), np.empty((N, D)), np.empty((N, D))
-            rc = lib.ta_oracle_backward_head(_dptr(qh), _dptr(kh), _dptr(xs),
-                                             _dptr(_f64(dout[b, h])), _dptr(dqh), _dptr(dkh),
-                                             _dptr(dvh), N, D, cdims, len(dims),
-                                             int(bool(causal)), scale)
+            if rope_base:
+                rc = lib.ta_oracle_backward_head_rope(_dptr(qh), _dptr(kh), _dptr(xs),
+                                                      _dptr(_f64(dout[b, h])), _dptr(dqh),
+                                                      _dptr(dkh), _dptr(dvh), N, D, cdims,
+                                                      len(dims), int(bool(causal)), scale,
+                                                      float(rope_base))
+            else:
+                rc = lib.ta_oracle_backward_head(_dptr(qh), _dptr(kh), _dptr(xs),
+                                                 _dptr(_f64(dout[b, h])), _dptr(dqh), _dptr(dkh),
+                                                 _dptr(dvh), N, D, cdims, len(dims),
+                                                 int(bool(causal)), scale)
             if rc != 0:
                 raise RuntimeError("ta_oracle_backward_head failed")
             dq[idx, j] = dqh
@@ -160,7 +192,8 @@ def backward(dout, q, k, v, dims, causal: bool, scale: float | None = None, grou
 # Brute force: every hop as a dense N x N matrix (tiny N only).  Independent of the C code.
 # --------------------------------------------------------------------------------------
 
-def dense_hop_matrix(qh, kh, dims, i: int, causal: bool, scale: float | None = None):
+def dense_hop_matrix(qh, kh, dims, i: int, causal: bool, scale: float | None = None,
+                     rope_base: float | None = None):
     """The N x N matrix of hop i for one head (Eq. 3 written over flat token indices).
 
     Entry [j, k] is the softmax weight of key token k for query token j; it is non-zero only
@@ -178,29 +211,45 @@ def dense_hop_matrix(qh, kh, dims, i: int, causal: bool, scale: float | None = N
             allowed &= cj == ck
         elif causal:
             allowed &= ck <= cj
-    s = (qh @ kh.T) * scale
+    if rope_base:
+        # relative form of the rotary score: features c and c + D/2 form one complex number
+        half = D // 2
+        zq = qh[:, :half] + 1j * qh[:, half:2 * half]
+        zk = kh[:, :half] + 1j * kh[:, half:2 * half]
+        theta = float(rope_base) ** (-2.0 * np.arange(half) / D)
+        rel = (coords[:, i][:, None] - coords[:, i][None, :]).astype(np.float64)   # p_j - p_k
+        s = np.zeros((N, N))
+        for c in range(half):
+            s += np.real(np.outer(zq[:, c], np.conj(zk[:, c])) * np.exp(1j * rel * theta[c]))
+        if D % 2:
+            s += np.outer(qh[:, -1], kh[:, -1])
+        s = s * scale
+    else:
+        s = (qh @ kh.T) * scale
     s = np.where(allowed, s, -np.inf)
     s = s - s.max(axis=1, keepdims=True)
     e = np.exp(s)
     return e / e.sum(axis=1, keepdims=True)
 
 
-def dense_effective_matrix(qh, kh, dims, causal: bool, scale: float | None = None):
+def dense_effective_matrix(qh, kh, dims, causal: bool, scale: float | None = None,
+                           rope_base: float | None = None):
     """A_eff = A^_{m-1} ... A^_1 A^_0, the N x N map from V to the output of one head."""
     N = np.asarray(qh).shape[0]
     a = np.eye(N)
     for i in range(len(dims)):
-        a = dense_hop_matrix(qh, kh, dims, i, causal, scale) @ a
+        a = dense_hop_matrix(qh, kh, dims, i, causal, scale, rope_base) @ a
     return a
 
 
-def forward_dense(q, k, v, dims, causal: bool, scale: float | None = None):
+def forward_dense(q, k, v, dims, causal: bool, scale: float | None = None,
+                  rope_base: float | None = None):
     """Brute-force forward for all heads via dense_effective_matrix (tiny N only)."""
     B, H, Hkv, N, D, dims = _check(q, k, v, dims)
     g = H // Hkv
     out = np.empty((B, H, N, D))
     for b in range(B):
         for h in range(H):
-            a = dense_effective_matrix(q[b, h], k[b, h // g], dims, causal, scale)
+            a = dense_effective_matrix(q[b, h], k[b, h // g], dims, causal, scale, rope_base)
             out[b, h] = a @ np.asarray(v[b, h // g], dtype=np.float64)
     return out
