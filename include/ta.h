@@ -113,6 +113,8 @@ typedef struct ta_params {
     int hop_begin;         /* run hops [hop_begin, hop_end) only; 0,0 -> all hops.  With      */
     int hop_end;           /* hop_begin > 0 the value tensor is read from `out` (layout of q) */
                            /* instead of v.                                                  */
+    float rope_base;       /* 0: none.  > 0 (Llama: 10000): tensorized positional encoding    */
+                           /* (Section 3.2), applied inside the kernels -- see ta_forward_ex  */
     ta_stream_t stream;
 } ta_params;
 
@@ -121,6 +123,17 @@ typedef struct ta_params {
  * is used for the generic kernel's second value buffer (and, with TA_FLAG_SAVE_HOPS, for
  * the hop inputs X_1..X_{m-1}, [m-1][B][H][N][D] in the storage dtype, which ta_backward
  * reads); it must hold ta_workspace_bytes(...) bytes or TA_ERR_WORKSPACE is returned.
+ *
+ * Tensorized positional encoding (Section 3.2, "Tensorized Positional Encoding": a token's
+ * position is the vector of its coordinates j_1..j_m, encoded with RoPE as in Llama).  With
+ * rope_base > 0 the un-rotated q and k are passed as usual and, in hop i, every query and
+ * key is rotated by its coordinate j_i along the dimension the hop attends over: feature c is
+ * paired with c + D/2 and turned by the angle j_i * rope_base^(-2c/D), so the hop's scores
+ * depend on relative positions along that dimension.  The rotation happens on the operand
+ * tiles in shared memory, between the TMA load and the MMA -- no rotated copy of q or k ever
+ * exists in global memory.  D must be even (else TA_ERR_UNSUPPORTED); a negative or NaN base
+ * is TA_ERR_INVALID_ARG.  The value tensor is never rotated.
+ * ta_backward does not take the positional encoding.
  */
 int ta_forward_ex(const ta_params *p);
 

@@ -44,6 +44,7 @@ class ta_params(ctypes.Structure):
                 ("softmax_scale", ctypes.c_float),
                 ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
                 ("flags", ctypes.c_uint), ("hop_begin", ctypes.c_int), ("hop_end", ctypes.c_int),
+                ("rope_base", ctypes.c_float),
                 ("stream", ctypes.c_void_p)]
 
 
@@ -169,7 +170,7 @@ def ta_forward_f32(q, k, v, out, B, H, H_kv, N, D, dims, causal, stream=None, ch
 
 def ta_forward_ex(q, k, v, out, B, H, H_kv, N, D, dims, causal, dtype=TA_DTYPE_BF16,
                   softmax_scale=0.0, workspace=None, workspace_bytes=0, flags=0, hop_begin=0,
-                  hop_end=0, stream=None, check=True) -> int:
+                  hop_end=0, rope_base=0.0, stream=None, check=True) -> int:
     d, nd = _dims(dims)
     p = ta_params()
     p.struct_bytes = ctypes.sizeof(ta_params)
@@ -179,6 +180,7 @@ def ta_forward_ex(q, k, v, out, B, H, H_kv, N, D, dims, causal, dtype=TA_DTYPE_B
     p.causal, p.dtype, p.softmax_scale = int(bool(causal)), dtype, softmax_scale
     p.workspace, p.workspace_bytes = _ptr(workspace), workspace_bytes
     p.flags, p.hop_begin, p.hop_end = flags, hop_begin, hop_end
+    p.rope_base = rope_base
     p.stream = _stream(stream)
     return _done(load().ta_forward_ex(ctypes.byref(p)), "ta_forward_ex", check)
 

@@ -158,6 +158,8 @@ static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 
 
 static int forward_impl(const ta_params &p) {
     if (!p.q || !p.k || !p.v || !p.out) return TA_ERR_INVALID_ARG;
+    if (p.rope_base < 0.f || !(p.rope_base == p.rope_base)) return TA_ERR_INVALID_ARG;
+    if (p.rope_base > 0.f && (p.D & 1)) return TA_ERR_UNSUPPORTED;
     Plan plan;
     int rc = build_plan(p.B, p.H, p.H_kv, p.N, p.D, p.dims, p.ndims, p.dtype, p.flags, p.hop_begin,
                         p.hop_end, &plan);
@@ -176,6 +178,7 @@ static int forward_impl(const ta_params &p) {
     for (int i = 0; i < p.ndims; ++i) pb.dims[i] = p.dims[i];
     pb.ndims = p.ndims; pb.causal = p.causal ? 1 : 0; pb.dtype = p.dtype;
     pb.scale = p.softmax_scale != 0.f ? p.softmax_scale : 1.0f / sqrtf((float)p.D);
+    pb.rope_base = p.rope_base;
     pb.flags = p.flags; pb.hop_begin = p.hop_begin; pb.hop_end = p.hop_end;
     pb.stream = (cudaStream_t)p.stream;
 

@@ -74,6 +74,7 @@ int backward_impl(const ta_bwd_params &p) {
     for (int i = 0; i < p.ndims; ++i) pb.dims[i] = p.dims[i];
     pb.ndims = p.ndims; pb.causal = p.causal ? 1 : 0; pb.dtype = p.dtype;
     pb.scale = p.softmax_scale != 0.f ? p.softmax_scale : 1.0f / sqrtf((float)p.D);
+    pb.rope_base = 0.f;
     pb.flags = 0; pb.hop_begin = 0; pb.hop_end = p.ndims;
     pb.stream = (cudaStream_t)p.stream;
 

@@ -50,6 +50,7 @@ struct Problem {
     int causal;
     int dtype;
     float scale;  // already resolved (1/sqrt(D) default)
+    float rope_base;  // 0 = no positional encoding
     unsigned flags;
     int hop_begin, hop_end;
     cudaStream_t stream;

@@ -28,7 +28,24 @@ struct SimtArgs {
     int qblocks;                  // ceil(n / BQ)
     long long items;              // B*H*segs_per_head*qblocks
     float scale;
+    float rope_log2_base;         // 0: no positional encoding; else log2 of the RoPE base
 };
+
+// Tensorized positional encoding (Section 3.2): rows of `x` ([rows][ld] fp32 in shared memory)
+// sit at positions pos0, pos0 + 1, .. of a segment; feature c is paired with c + D/2 and
+// turned by the angle position * base^(-2c/D).
+__device__ __forceinline__ void rope_rows(float *x, int rows, int ld, int D, int pos0, float log2_base) {
+    const int half = D >> 1;
+    for (int idx = threadIdx.x; idx < rows * half; idx += blockDim.x) {
+        const int r = idx / half, c = idx % half;
+        const float theta = exp2f(-2.f * (float)c / (float)D * log2_base);
+        float sn, cs;
+        sincosf((float)(pos0 + r) * theta, &sn, &cs);
+        const float x1 = x[r * ld + c], x2 = x[r * ld + c + half];
+        x[r * ld + c] = x1 * cs - x2 * sn;
+        x[r * ld + c + half] = x2 * cs + x1 * sn;
+    }
+}
 
 template <typename T> __device__ __forceinline__ float to_f32(T x);
 template <> __device__ __forceinline__ float to_f32<float>(float x) { return x; }
@@ -81,6 +98,10 @@ hop_simt_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__res
             int r = idx / D, c = idx % D, t = t0 + r;
             sQ[idx] = (t < a.n) ? to_f32<T>(qh[(base + (long long)t * a.stride) * D + c]) : 0.f;
         }
+        if (a.rope_log2_base != 0.f) {
+            __syncthreads();
+            rope_rows(sQ, BQ, D, D, t0, a.rope_log2_base);
+        }
 
         float m[kRowsPerWarp], l[kRowsPerWarp], o[kRowsPerWarp][DPL];
 #pragma unroll
@@ -107,6 +128,10 @@ hop_simt_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__res
                 sV[u * ldk + c] = xv;
             }
             __syncthreads();
+            if (a.rope_log2_base != 0.f) {
+                rope_rows(sK, BK, ldk, D, k0, a.rope_log2_base);
+                __syncthreads();
+            }
             const int key = k0 + lane;
 #pragma unroll
             for (int r = 0; r < kRowsPerWarp; ++r) {
@@ -170,6 +195,7 @@ int launch_t(const Problem &pb, const HopDesc &hd, const void *xin, int xin_head
     a.qblocks = (hd.n + BQ - 1) / BQ;
     a.items = (long long)pb.B * pb.H * a.segs_per_head * a.qblocks;
     a.scale = pb.scale;
+    a.rope_log2_base = pb.rope_base > 0.f ? log2f(pb.rope_base) : 0.f;
     size_t smem = sizeof(float) * ((size_t)BQ * pb.D + 2 * (size_t)BK * (pb.D + 1));
     auto kern = hop_simt_kernel<T, DPL>;
     if (smem > 48 * 1024) {

@@ -23,9 +23,13 @@
 //   warps 4-7   softmax + epilogue of the even tiles   } each warp owns 32 TMEM lanes (rows);
 //   warps 8-11  softmax + epilogue of the odd tiles    } S and O are double-buffered in TMEM
 //   warp 2      TMA store of finished tiles; hands the X slot back to the producer
+//   warps 12-19 (only with the tensorized positional encoding, Section 3.2) rotate the K and Q
+//               tiles in place in shared memory by the rows' coordinate along the hop's
+//               dimension (RoPE, feature c paired with c + D/2) before the MMA issuer sees them
 // Every wait is an mbarrier wait with a time limit; when one expires the CTA raises a flag that
 // ends all its roles, waits for its copies in flight, frees its TMEM and returns.
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 
 #include <mutex>
 
@@ -37,7 +41,8 @@ namespace ta {
 namespace {
 
 constexpr int kTileRows = 128;
-constexpr int kThreads = 384;
+constexpr int kThreads = 384;        // without the positional encoding
+constexpr int kThreadsRope = 640;    // + two warpgroups that rotate Q and K tiles
 constexpr int kNK = 2;   // K ring (one slot per work item)
 constexpr int kNQ = 2;   // Q ring (one slot per tile)
 
@@ -51,7 +56,7 @@ struct PipeCfg {
     static constexpr uint32_t kOffQ = kOffK + kNK * kTileBytes;
     static constexpr uint32_t kOffX = kOffQ + kNQ * kTileBytes;
     static constexpr uint32_t kOffBar = kOffX + kNX * kTileBytes;
-    static constexpr int kNumBars = 2 * kNK + 2 * kNQ + 3 * kNX + 2 + 2 + 2;
+    static constexpr int kNumBars = 2 * kNK + 2 * kNQ + 3 * kNX + 2 + 2 + 2 + kNK + kNQ;
     static constexpr uint32_t kSmemBytes = kOffBar + kNumBars * 8 + 16 + 1024 /*alignment slack*/;
     // S: 2 x 128 fp32 columns (P, bf16, is written over the first 64 columns of its S), O: 2 x 128
     static constexpr uint32_t kTmemCols = 512;
@@ -63,6 +68,7 @@ struct TcArgs {
     int gi, hsplit;            // query heads per work item, items per GQA group (gi * hsplit == g)
     long long tiles_inner, tiles_outer, total_items;
     float scale_log2;
+    float rope_log2_base;      // log2 of the RoPE base (rotating variant only)
 };
 
 struct ItemCoord {
@@ -86,8 +92,8 @@ __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t
 }
 
 // ----------------------------------------------------------------------------- the kernel
-template <int D>
-__global__ void __launch_bounds__(kThreads, 1)
+template <int D, bool kRope>
+__global__ void __launch_bounds__(kRope ? kThreadsRope : kThreads, 1)
 hop_pipe_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                 const __grid_constant__ CUtensorMap map_xin, const __grid_constant__ CUtensorMap map_xout,
                 const TcArgs a) {
@@ -114,19 +120,23 @@ hop_pipe_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     auto s_full = [&](int i) { return bar0 + 8u * (uint32_t)(kB1 + i); };
     auto o_full = [&](int i) { return bar0 + 8u * (uint32_t)(kB1 + 2 + i); };
     auto p_full = [&](int i) { return bar0 + 8u * (uint32_t)(kB1 + 4 + i); };
+    auto k_rot = [&](int i) { return bar0 + 8u * (uint32_t)(kB1 + 6 + i); };          // rotated K ready
+    auto q_rot = [&](int i) { return bar0 + 8u * (uint32_t)(kB1 + 6 + kNK + i); };    // rotated Q ready
     uint32_t *tmem_slot = (uint32_t *)(smem + C::kOffBar + C::kNumBars * 8);
     volatile uint32_t *abort_flag = tmem_slot + 1;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
     // ---- one-time setup
-    for (uint32_t i = tid; i < C::kOffBar / 16; i += kThreads)
+    for (uint32_t i = tid; i < C::kOffBar / 16; i += blockDim.x)
         ((uint4 *)smem)[i] = make_uint4(0, 0, 0, 0);   // rows a box never fills must stay finite
     if (tid == 0) {
         for (int i = 0; i < kNK; ++i) { mbar_init(k_full(i), 1); mbar_init(k_free(i), 1); }
         for (int i = 0; i < kNQ; ++i) { mbar_init(q_full(i), 1); mbar_init(q_free(i), 1); }
         for (int i = 0; i < kNX; ++i) { mbar_init(x_full(i), 1); mbar_init(x_free(i), 1); mbar_init(out_full(i), 4); }
         for (int i = 0; i < 2; ++i) { mbar_init(s_full(i), 1); mbar_init(o_full(i), 1); mbar_init(p_full(i), 4); }
+        for (int i = 0; i < kNK; ++i) mbar_init(k_rot(i), 8);
+        for (int i = 0; i < kNQ; ++i) mbar_init(q_rot(i), 8);
         *abort_flag = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -231,8 +241,8 @@ hop_pipe_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             uint32_t it = 0, j = 0;
             for (uint32_t t = 0; ok && t < T; ++t) {
                 const int ks = it & 1, qs = t & 1;
-                if (j == 0) ok = mbar_wait_abortable(k_full(ks), (it >> 1) & 1, 0x23, abort_flag);
-                if (ok) ok = mbar_wait_abortable(q_full(qs), (t >> 1) & 1, 0x24, abort_flag);
+                if (j == 0) ok = mbar_wait_abortable(kRope ? k_rot(ks) : k_full(ks), (it >> 1) & 1, 0x23, abort_flag);
+                if (ok) ok = mbar_wait_abortable(kRope ? q_rot(qs) : q_full(qs), (t >> 1) & 1, 0x24, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
                 // S(t)[128 x 128] = Q[128 x D] K^T : D/16 instructions of K = 16.  Its buffer last
@@ -274,6 +284,82 @@ hop_pipe_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 }
             }
             tma_store_wait_all();
+        }
+    } else if (kRope && warp >= 12) {
+        // =============================================================== RoPE on the K and Q tiles
+        // Row r of a tile sits at position t = r mod n of its segment, the same in every tile.
+        // A thread owns one 16-byte chunk of features (8 adjacent c < D/2, and their partners
+        // c + D/2) at the positions t = tsub, tsub + kTStep, .. (< n) of EVERY segment of the
+        // tile, so the cos / sin it needs never change: they sit in registers as fp16 pairs
+        // (absolute error 2^-12, far below bf16), computed once per launch, and a tile costs one
+        // 16-byte load and store per 8 features plus the multiply-adds.
+        constexpr int kChunks = D / 16;                   // 16-byte chunks of the first half of a row
+        const int rt = tid - 12 * 32;                     // 0 .. 255
+        const int chunk = rt % kChunks;
+        const int tsub = rt / kChunks;                    // 0 .. 31 (D = 128) or 0 .. 63 (D = 64)
+        constexpr int kTStep = 256 / kChunks;             // positions covered by one sweep of the threads
+        constexpr int kMaxPos = 128 / kTStep;             // sweeps to reach n = 128
+        const int segs = a.rows / a.n;
+        __half2 cs[kMaxPos][8];
+#pragma unroll
+        for (int pi = 0; pi < kMaxPos; ++pi)
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const float ang = (float)(tsub + kTStep * pi) *
+                                  exp2f(-2.f * (float)(8 * chunk + e) / (float)D * a.rope_log2_base);
+                cs[pi][e] = __floats2half2_rn(__cosf(ang), __sinf(ang));
+            }
+
+        auto rotate_tile = [&](uint32_t tile) {
+#pragma unroll
+            for (int pi = 0; pi < kMaxPos; ++pi) {
+                const int t = tsub + kTStep * pi;
+                if (t >= a.n) break;
+#pragma unroll 2
+                for (int sg = 0; sg < segs; ++sg) {
+                    const int r = sg * a.n + t;
+                    const uint32_t row = tile + (uint32_t)r * 128u;
+                    const uint32_t addr_a = row + (((uint32_t)chunk ^ (uint32_t)(r & 7)) << 4);
+                    const uint32_t addr_b = D == 128 ? addr_a + kSlabBytes                   // partner: second slab
+                                                     : row + (((uint32_t)(chunk + 4) ^ (uint32_t)(r & 7)) << 4);
+                    uint32_t ua[4], ub[4];
+                    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                                 : "=r"(ua[0]), "=r"(ua[1]), "=r"(ua[2]), "=r"(ua[3]) : "r"(addr_a) : "memory");
+                    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                                 : "=r"(ub[0]), "=r"(ub[1]), "=r"(ub[2]), "=r"(ub[3]) : "r"(addr_b) : "memory");
+#pragma unroll
+                    for (int e2 = 0; e2 < 4; ++e2) {
+                        const float a0 = __uint_as_float(ua[e2] << 16), a1 = __uint_as_float(ua[e2] & 0xFFFF0000u);
+                        const float b0 = __uint_as_float(ub[e2] << 16), b1 = __uint_as_float(ub[e2] & 0xFFFF0000u);
+                        const float2 f0 = __half22float2(cs[pi][2 * e2]), f1 = __half22float2(cs[pi][2 * e2 + 1]);
+                        ua[e2] = pack_bf16x2(a0 * f0.x - b0 * f0.y, a1 * f1.x - b1 * f1.y);
+                        ub[e2] = pack_bf16x2(b0 * f0.x + a0 * f0.y, b1 * f1.x + a1 * f1.y);
+                    }
+                    st_shared_v4(addr_a, ua[0], ua[1], ua[2], ua[3]);
+                    st_shared_v4(addr_b, ub[0], ub[1], ub[2], ub[3]);
+                }
+            }
+            fence_proxy_async_smem();
+            __syncwarp();
+        };
+
+        bool ok = true;
+        uint32_t t = 0, it = 0;
+        for (long long item = blockIdx.x; ok && item < a.total_items; item += gridDim.x, ++it) {
+            const int ks = it & 1;
+            ok = mbar_wait_abortable(k_full(ks), (it >> 1) & 1, 0x50, abort_flag);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            rotate_tile(sK + ks * kTileBytes);
+            if (lane == 0) mbar_arrive(k_rot(ks));
+            for (int j = 0; j < a.gi; ++j, ++t) {
+                const int qs = t & 1;
+                ok = mbar_wait_abortable(q_full(qs), (t >> 1) & 1, 0x51, abort_flag);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                rotate_tile(sQ + qs * kTileBytes);
+                if (lane == 0) mbar_arrive(q_rot(qs));
+            }
         }
     } else if (warp >= 4) {
         // =============================================================== softmax + epilogue
@@ -455,17 +541,23 @@ int launch_d(const Problem &pb, const HopDesc &hd, const void *xin, int xin_head
     a.gi = a.g / a.hsplit;
     a.total_items = positions * a.hsplit;
     a.scale_log2 = pb.scale * 1.4426950408889634f;
+    a.rope_log2_base = pb.rope_base > 0.f ? log2f(pb.rope_base) : 0.f;
 
     constexpr size_t smem = PipeCfg<D>::kSmemBytes;
-    auto kern = hop_pipe_kernel<D>;
+    const unsigned grid = (unsigned)(a.total_items < num_sms ? a.total_items : num_sms);
     static bool configured = false;
     if (!configured) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        if (cudaFuncSetAttribute(hop_pipe_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+                cudaSuccess ||
+            cudaFuncSetAttribute(hop_pipe_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+                cudaSuccess)
             return TA_ERR_CUDA;
         configured = true;
     }
-    const unsigned grid = (unsigned)(a.total_items < num_sms ? a.total_items : num_sms);
-    kern<<<grid, kThreads, smem, pb.stream>>>(mq, mk, mxi, mxo, a);
+    if (pb.rope_base > 0.f)
+        hop_pipe_kernel<D, true><<<grid, kThreadsRope, smem, pb.stream>>>(mq, mk, mxi, mxo, a);
+    else
+        hop_pipe_kernel<D, false><<<grid, kThreads, smem, pb.stream>>>(mq, mk, mxi, mxo, a);
     count_launch();
     return cudaPeekAtLastError() == cudaSuccess ? TA_OK : TA_ERR_CUDA;
 }
