@@ -237,7 +237,11 @@ def run_ours(args, cfg):
     stream = torch.cuda.current_stream()
 
     def step():
-        ta.ta_forward(q, k, v, out, cfg.B, cfg.H, cfg.H_kv, cfg.N, cfg.D, dims, cfg.causal, stream=stream)
+        if args.rope_base > 0:
+            ta.ta_forward_ex(q, k, v, out, cfg.B, cfg.H, cfg.H_kv, cfg.N, cfg.D, dims, cfg.causal,
+                             rope_base=args.rope_base, stream=stream)
+        else:
+            ta.ta_forward(q, k, v, out, cfg.B, cfg.H, cfg.H_kv, cfg.N, cfg.D, dims, cfg.causal, stream=stream)
 
     for _ in range(max(args.warmup, 3)):
         step()
@@ -287,8 +291,9 @@ def run_ours(args, cfg):
     e2e_value = aggregate(cfg.B * cfg.N, world, e2e_ms, e2e_steps)
     h2d = sum(host[n].numel() * 2 for n in ("q", "k", "v"))
     d2h = host["out"].numel() * 2
-    # the e2e result must be the same bits as the device-resident run
-    same = bool(torch.equal(host["out"], out.cpu()))
+    # the e2e result must be the same bits as the device-resident run (the host entry point
+    # takes no positional encoding, so there is nothing to compare with --rope-base)
+    same = bool(torch.equal(host["out"], out.cpu())) if args.rope_base == 0 else None
 
     if rank != 0:
         return
@@ -306,10 +311,14 @@ def run_ours(args, cfg):
                 "useful_tflops": step_flops(cfg) / (ms / args.steps * 1e-3) / 1e12}
     cpu, _ = oracle_sample(cfg, inp, min_seconds=args.cpu_seconds)
 
+    cfg_desc = workload_config(cfg, world)
+    if args.rope_base > 0:
+        cfg_desc["workload"] += f", tensorized positional encoding fused (RoPE base {args.rope_base:g})"
+        cfg_desc["rope_base"] = args.rope_base
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": workload_config(cfg, world), "clocks": clocks,
+            "config": cfg_desc, "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "ms_per_step": e2e_ms / e2e_steps, "steps": e2e_steps, "matches_device_run": same},
             "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu}
@@ -324,6 +333,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=4, help="workload: index into the five configurations")
     ap.add_argument("--cpu-seconds", type=float, default=10.0, help="CPU time budget of the oracle sample")
+    ap.add_argument("--rope-base", type=float, default=0.0,
+                    help="> 0: time the forward with the fused tensorized positional encoding (not the "
+                         "headline workload; device-timed value only)")
     args = ap.parse_args()
     cfg = ta_inputs.CONFIGS[args.config]
     if args.impl == "reference":
