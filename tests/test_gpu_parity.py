@@ -54,6 +54,13 @@ def test_tensor_core_small(dims, D, causal):
     check_case(1, 4, 2, math.prod(dims), D, dims, causal, "bf16", seed=103)
 
 
+# Shapes of the paper's bidirectional workloads (Section 3.3: 512 tokens as {32,16} and {8,8,8};
+# Appendix D: 1024 patches as 2 to 4 levels), RoBERTa-like heads (H = 12, D = 64), non-causal.
+@pytest.mark.parametrize("dims", [[32, 16], [8, 8, 8], [32, 32], [16, 16, 4], [16, 4, 4, 4], [8, 128], [128, 8]])
+def test_encoder_shapes_noncausal(dims):
+    check_case(2, 12, 12, math.prod(dims), 64, dims, False, "bf16", seed=112)
+
+
 def test_tensor_core_batch_and_gqa_indexing():
     check_case(3, 8, 2, 512, 128, [8, 64], True, "bf16", seed=104)
     check_case(2, 6, 6, 256, 64, [16, 16], False, "bf16", seed=105)
