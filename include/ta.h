@@ -150,8 +150,8 @@ int ta_forward_ex(const ta_params *p);
  *   gradient G carried between hops, and fp32 accumulators for dq, dk, dv, which are rounded
  *   to bf16 once at the end.
  * Arithmetic: bf16 operands, fp32 accumulation; the attention weights are recomputed.
- * The sums over the query heads of a group are fp32 atomic adds at L2, so dk and dv are not
- * bit-reproducible from run to run.
+ * The sums over the query heads of a group are taken in tensor memory inside one CTA and the
+ * sums over hops in launch order, so the result is bit-reproducible from run to run.
  * Supported where every hop runs on the tensor-core kernel (D in {64,128}, all n_i <= 128);
  * otherwise TA_ERR_UNSUPPORTED.
  */

@@ -85,16 +85,17 @@ int backward_impl(const ta_bwd_params &p) {
     float *dv_acc = need_acc ? (float *)(ws + L.dv_off) : (float *)p.dv;
     const int k = plan.nhops;
 
-    if (cudaMemsetAsync(dq_acc, 0, tq * 4, pb.stream) != cudaSuccess ||
-        cudaMemsetAsync(dk_acc, 0, tkv * 4, pb.stream) != cudaSuccess)
-        return TA_ERR_CUDA;
     if (k == 0) {
+        if (cudaMemsetAsync(dq_acc, 0, tq * 4, pb.stream) != cudaSuccess ||
+            cudaMemsetAsync(dk_acc, 0, tkv * 4, pb.stream) != cudaSuccess)
+            return TA_ERR_CUDA;
         // every dimension is 1: out = v broadcast over the group, so dv = sum of dout, dq = dk = 0
         rc = launch_group_sum(p.dout, need_acc ? (void *)p.dv : (void *)dv_acc, need_acc ? 0 : 1, p.B, p.H, p.H_kv,
                               (long long)p.N * p.D, pb.stream);
         if (rc != TA_OK) return rc;
     } else {
-        if (cudaMemsetAsync(dv_acc, 0, tkv * 4, pb.stream) != cudaSuccess) return TA_ERR_CUDA;
+        // No clearing: the first hop processed (the last hop) stores dq / dk, later ones add to
+        // them, and hop 0 stores dv; every row of every head is covered by exactly one tile.
         // X_j = input of hop j: X_0 = v, X_1.. = saved (or recomputed here by running hops 0..k-2)
         const char *saved = p.saved_hops ? (const char *)p.saved_hops : ws + L.save_off;
         auto hop_input = [&](int j) -> const void * { return j == 0 ? p.v : (const void *)(saved + (size_t)(j - 1) * tq * 2); };
@@ -109,7 +110,7 @@ int backward_impl(const ta_bwd_params &p) {
         for (int j = k - 1; j >= 0; --j) {
             const void *g_in = j == k - 1 ? p.dout : (const void *)gbuf;
             rc = launch_hop_tc_bwd(pb, plan.hops[j], hop_input(j), j == 0 ? p.H_kv : p.H, g_in, j == 0 ? nullptr : gbuf,
-                                   dq_acc, dk_acc, dv_acc, j == 0);
+                                   dq_acc, dk_acc, dv_acc, j == 0, j != k - 1);
             if (rc != TA_OK) return rc;
         }
     }

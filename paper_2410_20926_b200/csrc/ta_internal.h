@@ -74,9 +74,11 @@ int launch_broadcast_kv(const Problem &pb);
 
 // Backward of one tensor-core hop (ta_tc_bwd.cu).  x = the hop's input value tensor (x_heads
 // heads per batch), g_in = gradient w.r.t. the hop's output, g_out = gradient w.r.t. its input
-// (bf16, may alias g_in; NULL when first_hop, where it is reduced into dv_acc instead).
+// (bf16, may alias g_in; NULL when first_hop, where it is summed over the group into dv_acc
+// instead).  accumulate = false: dq_acc / dk_acc are overwritten (the first hop processed),
+// true: added to.  dv_acc is always overwritten (only the first hop writes it).
 int launch_hop_tc_bwd(const Problem &pb, const HopDesc &hd, const void *x, int x_heads, const void *g_in,
-                      void *g_out, float *dq_acc, float *dk_acc, float *dv_acc, bool first_hop);
+                      void *g_out, float *dq_acc, float *dk_acc, float *dv_acc, bool first_hop, bool accumulate);
 int launch_f32_to_bf16(const float *src, void *dst, long long n, cudaStream_t stream);
 int launch_group_sum(const void *dout, void *dv, int dv_is_f32, int B, int H, int H_kv, long long per_head,
                      cudaStream_t stream);

@@ -8,11 +8,21 @@
 //     G_i = P^T G_{i+1}          dQ += dS K          dK += dS^T Q
 //
 // Tiles, strided TMA maps and the block-diagonal packing of short segments are those of the
-// forward kernel.  Per tile: two MMAs into TMEM (S = Q K^T, dP = G X^T), the softmax and its
-// derivative in registers, P and dS (bf16) to shared memory, then three MMAs: G_i (A = P as an
-// MN-major operand, i.e. P^T), dQ (A = dS K-major) and dK (A = dS MN-major).  dQ / dK / dV are
-// accumulated in fp32 global buffers by TMA reduce-add (they sum over hops and, for dK / dV,
-// over the query heads of a GQA group); G_i is carried to the next hop as bf16, in place.
+// forward kernel.  A work item is one tile position of one KV head; the H/H_kv query heads of
+// the group are processed in turn against the same K tile, and their dK (and, in the first
+// hop, dV = G_0) contributions are summed in tensor memory and leave the SM once per item.
+// Per head: two MMAs into TMEM (S = Q K^T, dP = G X^T), the softmax and its derivative in
+// registers, P (over the X tile, dead by then) and dS (bf16) to shared memory, then three
+// MMAs: G_i (A = P as an MN-major operand, i.e. P^T; over the S columns), dQ (A = dS K-major;
+// over the dP columns) and dK (A = dS MN-major).  dQ and dK go to fp32 buffers in global
+// memory -- plain TMA stores in the first hop processed, TMA reduce-add afterwards (they sum
+// over hops) -- and G_i is carried to the next hop as bf16, in place.
+//
+// Persistent, one CTA per SM.  Warps 0-3 compute (thread 0 issues the MMAs and the stores);
+// warp 4 issues the TMA loads: Q and G of the next head land in a second stage while the
+// current head computes, X and K as soon as the MMAs that read their slots have completed, so
+// that loads overlap the epilogue.  Every wait is bounded; when one expires the CTA raises a
+// flag that ends both roles, lets its copies land, frees its TMEM and returns.
 #include <cuda_bf16.h>
 
 #include "ta_internal.h"
@@ -22,61 +32,101 @@ namespace ta {
 namespace {
 
 constexpr int kTileRows = 128;
-constexpr int kThreads = 128;
+constexpr int kThreads = 160;          // + the producer warp
 
 struct BwdArgs {
     int n, rows, ci, co, causal, g, H, H_kv, x_is_kv, first_hop;
-    long long tiles_inner, tiles_outer, total_tiles;
+    int accumulate;                    // 0: dQ / dK are stored (first hop processed), 1: reduce-added
+    long long tiles_inner, tiles_outer, total_items;
     float scale_log2, scale;
 };
+
+template <int D>
+struct BwdCfg {
+    static constexpr int kHalves = D / 64;
+    static constexpr uint32_t kSlabBytes = kTileRows * 128;          // [128 rows][128 bytes]
+    static constexpr uint32_t kTileBytes = kHalves * kSlabBytes;     // one bf16 operand tile
+    static constexpr uint32_t kPBytes = 2 * kSlabBytes;              // 128 x 128 bf16
+    static constexpr uint32_t kStageBytes = 2 * kTileBytes;          // {Q, G} of one head = one fp32 output tile
+    static constexpr uint32_t kOffK = 0;
+    static constexpr uint32_t kOffStage = kOffK + kTileBytes;        // 2 stages
+    static constexpr uint32_t kOffXP = kOffStage + 2 * kStageBytes;  // X, then P
+    static constexpr uint32_t kOffDS = kOffXP + kPBytes;             // dS, then the bf16 G_i staging
+    static constexpr uint32_t kOffBar = kOffDS + kPBytes;
+    static constexpr int kNumBars = 10;
+    static constexpr uint32_t kSmemBytes = kOffBar + kNumBars * 8 + 16 + 1024;
+    static constexpr uint32_t kTmemCols = 512;
+    // S then G_i | dP then dQ | dK summed over the group | dV summed over the group (first hop)
+    static constexpr uint32_t kColS = 0, kColDP = 128, kColDK = 256, kColDV = 384;
+};
+
+struct BwdItem {
+    int c_inner, c_outer, kv_head, q_head0;
+};
+__device__ __forceinline__ BwdItem decode_bwd_item(const BwdArgs &a, long long item) {
+    BwdItem c;
+    long long rest = item;
+    c.c_inner = (int)(rest % a.tiles_inner) * a.ci; rest /= a.tiles_inner;
+    c.c_outer = (int)(rest % a.tiles_outer) * a.co; rest /= a.tiles_outer;
+    c.kv_head = (int)rest;
+    c.q_head0 = (c.kv_head / a.H_kv) * a.H + (c.kv_head % a.H_kv) * a.g;
+    return c;
+}
 
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 
+// barrier + AND over the 128 compute threads (named barrier 1)
+__device__ __forceinline__ bool wg_all(bool pred) {
+    uint32_t r;
+    asm volatile(
+        "{\n .reg .pred p, q;\n setp.ne.b32 q, %1, 0;\n bar.red.and.pred p, 1, 128, q;\n selp.u32 %0, 1, 0, p;\n}"
+        : "=r"(r)
+        : "r"((uint32_t)pred)
+        : "memory");
+    return r != 0;
+}
+__device__ __forceinline__ void wg_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
 template <int D>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 1)
 hop_tc_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                   const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_gin,
                   const __grid_constant__ CUtensorMap map_gout, const __grid_constant__ CUtensorMap map_dq,
                   const __grid_constant__ CUtensorMap map_dk, const __grid_constant__ CUtensorMap map_dv,
                   const BwdArgs a) {
-    constexpr int kHalves = D / 64;
-    constexpr uint32_t kSlabBytes = kTileRows * 128;          // [128 rows][128 bytes]
-    constexpr uint32_t kTileBytes = kHalves * kSlabBytes;     // one bf16 input tile
-    constexpr uint32_t kPBytes = 2 * kSlabBytes;              // 128 x 128 bf16
-    constexpr uint32_t kStageBytes = 2 * kTileBytes;          // one fp32 output tile
-    constexpr uint32_t kTmemCols = 512;
-    constexpr uint32_t kColS = 0, kColDP = 128, kColG = 256, kColDQ = 384, kColDK = 0;
+    using C = BwdCfg<D>;
+    constexpr int kHalves = C::kHalves;
+    constexpr uint32_t kSlabBytes = C::kSlabBytes, kTileBytes = C::kTileBytes, kStageBytes = C::kStageBytes;
 
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const uint32_t s0 = smem_u32(smem);
-    const uint32_t sQ = s0, sK = sQ + kTileBytes, sX = sK + kTileBytes, sG = sX + kTileBytes;
-    const uint32_t sP = sG + kTileBytes, sdS = sP + kPBytes;
-    constexpr uint32_t kDataBytes = 4 * kTileBytes + 2 * kPBytes;
-    // output staging after all MMAs have completed (every input is dead by then)
-    const uint32_t stDQ = s0, stDK = s0 + kStageBytes, stG = s0 + 2 * kStageBytes;
-    uint64_t *bars = (uint64_t *)(smem + kDataBytes);
-    const uint32_t bar_qk = smem_u32(bars + 0), bar_gx = smem_u32(bars + 1), bar_s = smem_u32(bars + 2),
-                   bar_o = smem_u32(bars + 3);
-    uint32_t *tmem_slot = (uint32_t *)(bars + 4);
+    const uint32_t sK = s0 + C::kOffK, sXP = s0 + C::kOffXP, sdS = s0 + C::kOffDS;
+    auto sQ = [&](int s) { return s0 + C::kOffStage + (uint32_t)s * kStageBytes; };
+    auto sG = [&](int s) { return s0 + C::kOffStage + (uint32_t)s * kStageBytes + kTileBytes; };
+    const uint32_t bar0 = s0 + C::kOffBar;
+    const uint32_t k_full = bar0, k_free = bar0 + 8, x_full = bar0 + 48, xp_free = bar0 + 56, s_done = bar0 + 64,
+                   o_done = bar0 + 72;
+    auto qg_full = [&](int s) { return bar0 + 16u + 8u * (uint32_t)s; };
+    auto qg_free = [&](int s) { return bar0 + 32u + 8u * (uint32_t)s; };
+    uint32_t *tmem_slot = (uint32_t *)(smem + C::kOffBar + C::kNumBars * 8);
+    volatile uint32_t *abort_flag = tmem_slot + 1;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
-    for (uint32_t i = tid; i < kDataBytes / 16; i += kThreads) ((uint4 *)smem)[i] = make_uint4(0, 0, 0, 0);
+    for (uint32_t i = tid; i < C::kOffBar / 16; i += kThreads) ((uint4 *)smem)[i] = make_uint4(0, 0, 0, 0);
     if (tid == 0) {
-        mbar_init(bar_qk, 1);
-        mbar_init(bar_gx, 1);
-        mbar_init(bar_s, 1);
-        mbar_init(bar_o, 1);
+        for (int i = 0; i < C::kNumBars; ++i) mbar_init(bar0 + 8u * (uint32_t)i, 1);
+        *abort_flag = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     fence_proxy_async_smem();
     if (warp == 0) {
         __syncwarp();
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
-                     "r"(kTmemCols)
+                     "r"(C::kTmemCols)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
@@ -84,230 +134,323 @@ hop_tc_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    const uint32_t tmem_lane = tmem_base + ((uint32_t)(warp * 32) << 16);
+    const uint32_t slab_tx = (uint32_t)a.rows * 128u;
 
-    constexpr uint32_t idesc_s = instr_desc(128, 0, 0);        // A, B K-major, N = 128
-    constexpr uint32_t idesc_g = instr_desc(D, 1, 1);          // A = P^T / dS^T (MN-major), B MN-major
-    constexpr uint32_t idesc_dq = instr_desc(D, 1, 0);         // A = dS K-major, B MN-major
-
-    const int r = warp * 32 + lane;
-    const int seg = r / a.n;
-    const bool row_valid = r < a.rows;
-    const int c_lo = seg * a.n;
-    const int c_hi = a.causal ? r + 1 : c_lo + a.n;
-    const int w_lo = ((warp * 32) / a.n) * a.n;
-    int w_hi = min(a.rows, ((warp * 32 + 31) / a.n + 1) * a.n);
-    if (a.causal) w_hi = min(w_hi, warp * 32 + 32);
-    const bool warp_valid = warp * 32 < a.rows;
-
-    bool ok = true;
-    uint32_t it = 0;
-    for (long long tile = blockIdx.x; tile < a.total_tiles; tile += gridDim.x, ++it) {
-        const uint32_t parity = it & 1u;
-        long long rest = tile;
-        const int hg = (int)(rest % a.g); rest /= a.g;
-        const int c_inner = (int)(rest % a.tiles_inner) * a.ci; rest /= a.tiles_inner;
-        const int c_outer = (int)(rest % a.tiles_outer) * a.co; rest /= a.tiles_outer;
-        const int kv_head = (int)rest;
-        const int q_head = (kv_head / a.H_kv) * a.H + (kv_head % a.H_kv) * a.g + hg;
-        const int x_head = a.x_is_kv ? kv_head : q_head;
-
-        if (tid == 0) {
-            const uint32_t slab_tx = (uint32_t)a.rows * 128u;
-            mbar_expect_tx(bar_qk, 2 * kHalves * slab_tx);
+    if (warp == 4) {
+        // =============================================================== TMA producer
+        if (lane == 0) {
+            uint32_t t = 0, it = 0;
+            bool ok = true;
+            // phases armed last on each barrier, for the drain on an early exit
+            uint32_t armed = 0, last_par = 0;        // bits: 0 k, 1-2 qg, 3 x
+            auto arm = [&](uint32_t bit, uint32_t parity) {
+                armed |= bit;
+                last_par = parity ? (last_par | bit) : (last_par & ~bit);
+            };
+            for (long long item = blockIdx.x; ok && item < a.total_items; item += gridDim.x, ++it) {
+                const BwdItem c = decode_bwd_item(a, item);
+                for (int j = 0; j < a.g; ++j, ++t) {
+                    const int q_head = c.q_head0 + j;
+                    const int x_head = a.x_is_kv ? c.kv_head : q_head;
+                    const int s = t & 1;
+                    const uint32_t par = (t >> 1) & 1;
+                    ok = mbar_wait_abortable(qg_free(s), par ^ 1, 0x60, abort_flag);
+                    if (!ok) break;
+                    mbar_expect_tx(qg_full(s), 2 * kHalves * slab_tx);
+                    arm(2u << s, par);
 #pragma unroll
-            for (int h = 0; h < kHalves; ++h) tma_load_5d(sQ + h * kSlabBytes, &map_q, bar_qk, 64 * h, 0, c_inner, c_outer, q_head);
+                    for (int h = 0; h < kHalves; ++h)
+                        tma_load_5d(sQ(s) + h * kSlabBytes, &map_q, qg_full(s), 64 * h, 0, c.c_inner, c.c_outer, q_head);
 #pragma unroll
-            for (int h = 0; h < kHalves; ++h) tma_load_5d(sK + h * kSlabBytes, &map_k, bar_qk, 64 * h, 0, c_inner, c_outer, kv_head);
-            mbar_expect_tx(bar_gx, 2 * kHalves * slab_tx);
+                    for (int h = 0; h < kHalves; ++h)
+                        tma_load_5d(sG(s) + h * kSlabBytes, &map_gin, qg_full(s), 64 * h, 0, c.c_inner, c.c_outer, q_head);
+                    if (j == 0) {
+                        ok = mbar_wait_abortable(k_free, (it & 1) ^ 1, 0x61, abort_flag);
+                        if (!ok) break;
+                        mbar_expect_tx(k_full, kHalves * slab_tx);
+                        arm(1u, it & 1);
 #pragma unroll
-            for (int h = 0; h < kHalves; ++h) tma_load_5d(sG + h * kSlabBytes, &map_gin, bar_gx, 64 * h, 0, c_inner, c_outer, q_head);
-#pragma unroll
-            for (int h = 0; h < kHalves; ++h) tma_load_5d(sX + h * kSlabBytes, &map_x, bar_gx, 64 * h, 0, c_inner, c_outer, x_head);
-
-            ok = mbar_wait(bar_qk, parity, 0x11);
-            if (ok) {
-                tc_fence_after();
-#pragma unroll
-                for (int kb = 0; kb < D / 16; ++kb) {
-                    const uint32_t off = (kb >> 2) * kSlabBytes + (kb & 3) * 32;
-                    tc_mma_ss(tmem_base + kColS, smem_desc_sw128(sQ + off, 16, 1024),
-                              smem_desc_sw128(sK + off, 16, 1024), idesc_s, kb > 0);
-                }
-                ok = mbar_wait(bar_gx, parity, 0x12);
-            }
-            if (ok) {
-#pragma unroll
-                for (int kb = 0; kb < D / 16; ++kb) {
-                    const uint32_t off = (kb >> 2) * kSlabBytes + (kb & 3) * 32;
-                    tc_mma_ss(tmem_base + kColDP, smem_desc_sw128(sG + off, 16, 1024),
-                              smem_desc_sw128(sX + off, 16, 1024), idesc_s, kb > 0);
-                }
-                tc_commit(bar_s);
-            }
-        }
-        __syncwarp();
-        if (ok) ok = mbar_wait(bar_s, parity, 0x13);
-        ok = __all_sync(0xffffffffu, ok);
-        tc_fence_after();
-
-        // ---- softmax and its derivative for this thread's row
-        if (ok) {
-            uint32_t vs[32], vd[32];
-            float m = -INFINITY;
-#pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
-                if (!(warp_valid && 32 * c < w_hi && 32 * c + 32 > w_lo)) continue;
-                tmem_ld32(tmem_lane + kColS + 32 * c, vs);
-#pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    const int col = 32 * c + j;
-                    if (col >= c_lo && col < c_hi) m = fmaxf(m, __uint_as_float(vs[j]));
-                }
-            }
-            const float m_s = row_valid ? m * a.scale_log2 : 0.f;
-            float l = 0.f, dot = 0.f;
-#pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
-                if (!(warp_valid && 32 * c < w_hi && 32 * c + 32 > w_lo)) continue;
-                tmem_ld32(tmem_lane + kColS + 32 * c, vs);
-                tmem_ld32(tmem_lane + kColDP + 32 * c, vd);
-#pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    const int col = 32 * c + j;
-                    float p = fast_exp2(__uint_as_float(vs[j]) * a.scale_log2 - m_s);
-                    const bool vis = row_valid && col >= c_lo && col < c_hi;
-                    p = vis ? p : 0.f;
-                    l += p;
-                    dot += vis ? p * __uint_as_float(vd[j]) : 0.f;
-                }
-            }
-            const float inv_l = row_valid ? 1.f / l : 0.f;
-            const float delta = dot * inv_l;
-            const uint32_t rowP = sP + (uint32_t)r * 128u, rowS = sdS + (uint32_t)r * 128u;
-#pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
-                uint32_t pp[16], ps[16];
-                if (warp_valid && 32 * c < w_hi && 32 * c + 32 > w_lo) {
-                    tmem_ld32(tmem_lane + kColS + 32 * c, vs);
-                    tmem_ld32(tmem_lane + kColDP + 32 * c, vd);
-#pragma unroll
-                    for (int j = 0; j < 32; j += 2) {
-                        float pv[2], dv[2];
-#pragma unroll
-                        for (int e = 0; e < 2; ++e) {
-                            const int col = 32 * c + j + e;
-                            const bool vis = row_valid && col >= c_lo && col < c_hi;
-                            float p = fast_exp2(__uint_as_float(vs[j + e]) * a.scale_log2 - m_s) * inv_l;
-                            p = vis ? p : 0.f;
-                            pv[e] = p;
-                            dv[e] = vis ? p * (__uint_as_float(vd[j + e]) - delta) * a.scale : 0.f;
-                        }
-                        pp[j >> 1] = pack_bf16x2(pv[0], pv[1]);
-                        ps[j >> 1] = pack_bf16x2(dv[0], dv[1]);
+                        for (int h = 0; h < kHalves; ++h)
+                            tma_load_5d(sK + h * kSlabBytes, &map_k, k_full, 64 * h, 0, c.c_inner, c.c_outer, c.kv_head);
                     }
-                } else {
+                    ok = mbar_wait_abortable(xp_free, (t & 1) ^ 1, 0x62, abort_flag);
+                    if (!ok) break;
+                    mbar_expect_tx(x_full, kHalves * slab_tx);
+                    arm(8u, t & 1);
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) { pp[j] = 0u; ps[j] = 0u; }
+                    for (int h = 0; h < kHalves; ++h)
+                        tma_load_5d(sXP + h * kSlabBytes, &map_x, x_full, 64 * h, 0, c.c_inner, c.c_outer, x_head);
                 }
-                const uint32_t slab = (uint32_t)(c >> 1) * kSlabBytes;
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const uint32_t chunk = (uint32_t)(((c & 1) * 4 + i) ^ (r & 7)) * 16;
-                    st_shared_v4(rowP + slab + chunk, pp[4 * i], pp[4 * i + 1], pp[4 * i + 2], pp[4 * i + 3]);
-                    st_shared_v4(rowS + slab + chunk, ps[4 * i], ps[4 * i + 1], ps[4 * i + 2], ps[4 * i + 3]);
+            }
+            if (!ok) {
+                const unsigned long long t0 = globaltimer_ns();
+                for (int b = 0; b < 4; ++b) {
+                    if (!(armed & (1u << b))) continue;
+                    const uint32_t bar = b == 0 ? k_full : (b == 3 ? x_full : qg_full(b - 1));
+                    while (!mbar_try_wait(bar, (last_par >> b) & 1u) && globaltimer_ns() - t0 < 10000000ull) {
+                    }
                 }
             }
         }
-        fence_proxy_async_smem();
-        tc_fence_before();
-        __syncthreads();
+    } else {
+        // =============================================================== compute warps
+        const uint32_t tmem_lane = tmem_base + ((uint32_t)(warp * 32) << 16);
+        constexpr uint32_t idesc_s = instr_desc(128, 0, 0);        // A, B K-major, N = 128
+        constexpr uint32_t idesc_g = instr_desc(D, 1, 1);          // A = P^T / dS^T (MN-major), B MN-major
+        constexpr uint32_t idesc_dq = instr_desc(D, 1, 0);         // A = dS K-major, B MN-major
 
-        if (tid == 0 && ok) {
-            tc_fence_after();
-            const int kblocks = (a.rows + 15) >> 4;
-            for (int kb = 0; kb < kblocks; ++kb) {
-                const uint32_t k_off = kb * 2048;                                  // 16 rows of 128 bytes
-                const uint32_t a_off = (kb >> 2) * kSlabBytes + (kb & 3) * 32;     // 16 columns of a K-major tile
-                // G_i[key, d] = sum_q P[q, key] G[q, d]
-                tc_mma_ss(tmem_base + kColG, smem_desc_sw128(sP + k_off, kSlabBytes, 1024),
-                          smem_desc_sw128(sG + k_off, kSlabBytes, 1024), idesc_g, kb > 0);
-                // dQ[q, d] = sum_key dS[q, key] K[key, d]
-                tc_mma_ss(tmem_base + kColDQ, smem_desc_sw128(sdS + a_off, 16, 1024),
-                          smem_desc_sw128(sK + k_off, kSlabBytes, 1024), idesc_dq, kb > 0);
-                // dK[key, d] = sum_q dS[q, key] Q[q, d]
-                tc_mma_ss(tmem_base + kColDK, smem_desc_sw128(sdS + k_off, kSlabBytes, 1024),
-                          smem_desc_sw128(sQ + k_off, kSlabBytes, 1024), idesc_g, kb > 0);
-            }
-            tc_commit(bar_o);
-        }
-        __syncwarp();
-        if (ok) ok = mbar_wait(bar_o, parity, 0x14);
-        ok = __all_sync(0xffffffffu, ok);
-        tc_fence_after();
+        const int r = warp * 32 + lane;
+        const int seg = r / a.n;
+        const bool row_valid = r < a.rows;
+        const int c_lo = seg * a.n;
+        const int c_hi = a.causal ? r + 1 : c_lo + a.n;
+        const int w_lo = ((warp * 32) / a.n) * a.n;
+        int w_hi = min(a.rows, ((warp * 32 + 31) / a.n + 1) * a.n);
+        if (a.causal) w_hi = min(w_hi, warp * 32 + 32);
+        const bool warp_valid = warp * 32 < a.rows;
+        const int kblocks = (a.rows + 15) >> 4;
 
-        // ---- epilogue: TMEM -> shared staging (box layouts) -> TMA reduce-add / store
-        if (ok && warp_valid) {
+        // fp32 accumulator columns -> shared staging in the layout of the fp32 maps (32-column slabs)
+        auto stage_f32 = [&](uint32_t col0, uint32_t stage) {
+            if (!warp_valid) return;
             uint32_t v[32];
 #pragma unroll 1
-            for (int which = 0; which < 3; ++which) {
-                const uint32_t col0 = which == 0 ? kColDQ : (which == 1 ? kColDK : kColG);
-                const uint32_t stage = which == 0 ? stDQ : (which == 1 ? stDK : stG);
-                const bool as_bf16 = which == 2 && !a.first_hop;
+            for (int c = 0; c < D / 32; ++c) {
+                tmem_ld32(tmem_lane + col0 + 32 * c, v);
+                if (!row_valid) continue;
+                const uint32_t row = stage + (uint32_t)c * kSlabBytes + (uint32_t)r * 128u;
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    st_shared_v4(row + (uint32_t)((i ^ (r & 7)) * 16), v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+            }
+        };
+
+        uint32_t t = 0, it = 0;
+        bool ok = true;
+        for (long long item = blockIdx.x; ok && item < a.total_items; item += gridDim.x, ++it) {
+            const BwdItem c = decode_bwd_item(a, item);
+            for (int j = 0; j < a.g; ++j, ++t) {
+                const int s = t & 1;
+                const uint32_t par = t & 1;
+                const int q_head = c.q_head0 + j;
+                const bool last_head = j == a.g - 1;
+                const uint32_t q_base = sQ(s), g_base = sG(s);
+
+                // ---- S = Q K^T and dP = G X^T
+                if (tid == 0) {
+                    bool k0 = true;
+                    if (j == 0) k0 = mbar_wait_abortable(k_full, it & 1, 0x71, abort_flag);
+                    if (k0) k0 = mbar_wait_abortable(qg_full(s), (t >> 1) & 1, 0x72, abort_flag);
+                    if (k0) {
+                        tc_fence_after();
+#pragma unroll
+                        for (int kb = 0; kb < D / 16; ++kb) {
+                            const uint32_t off = (kb >> 2) * kSlabBytes + (kb & 3) * 32;
+                            tc_mma_ss(tmem_base + C::kColS, smem_desc_sw128(q_base + off, 16, 1024),
+                                      smem_desc_sw128(sK + off, 16, 1024), idesc_s, kb > 0);
+                        }
+                        k0 = mbar_wait_abortable(x_full, par, 0x73, abort_flag);
+                    }
+                    if (k0) {
+                        tc_fence_after();
+#pragma unroll
+                        for (int kb = 0; kb < D / 16; ++kb) {
+                            const uint32_t off = (kb >> 2) * kSlabBytes + (kb & 3) * 32;
+                            tc_mma_ss(tmem_base + C::kColDP, smem_desc_sw128(g_base + off, 16, 1024),
+                                      smem_desc_sw128(sXP + off, 16, 1024), idesc_s, kb > 0);
+                        }
+                        tc_commit(s_done);
+                    }
+                    ok = k0;
+                }
+                __syncwarp();
+                if (ok) ok = mbar_wait_abortable(s_done, par, 0x74, abort_flag);
+                ok = wg_all(ok);
+                if (!ok) break;
+                tc_fence_after();
+
+                // ---- softmax and its derivative for this thread's row; P -> X slot, dS -> its slot
+                {
+                    uint32_t vs[32], vd[32];
+                    float m = -INFINITY;
 #pragma unroll 1
-                for (int c = 0; c < D / 32; ++c) {
-                    tmem_ld32(tmem_lane + col0 + 32 * c, v);
-                    if (!row_valid) continue;
-                    if (as_bf16) {
-                        uint32_t pk[16];
+                    for (int cc = 0; cc < 4; ++cc) {
+                        if (!(warp_valid && 32 * cc < w_hi && 32 * cc + 32 > w_lo)) continue;
+                        tmem_ld32(tmem_lane + C::kColS + 32 * cc, vs);
 #pragma unroll
-                        for (int j = 0; j < 32; j += 2)
-                            pk[j >> 1] = pack_bf16x2(__uint_as_float(v[j]), __uint_as_float(v[j + 1]));
-                        const uint32_t row = stage + (uint32_t)(c >> 1) * kSlabBytes + (uint32_t)r * 128u;
+                        for (int jj = 0; jj < 32; ++jj) {
+                            const int col = 32 * cc + jj;
+                            if (col >= c_lo && col < c_hi) m = fmaxf(m, __uint_as_float(vs[jj]));
+                        }
+                    }
+                    const float m_s = row_valid ? m * a.scale_log2 : 0.f;
+                    float l = 0.f, dot = 0.f;
+#pragma unroll 1
+                    for (int cc = 0; cc < 4; ++cc) {
+                        if (!(warp_valid && 32 * cc < w_hi && 32 * cc + 32 > w_lo)) continue;
+                        tmem_ld32(tmem_lane + C::kColS + 32 * cc, vs);
+                        tmem_ld32(tmem_lane + C::kColDP + 32 * cc, vd);
 #pragma unroll
-                        for (int i = 0; i < 4; ++i)
-                            st_shared_v4(row + (uint32_t)((((c & 1) * 4 + i) ^ (r & 7)) * 16), pk[4 * i], pk[4 * i + 1],
-                                         pk[4 * i + 2], pk[4 * i + 3]);
-                    } else {
-                        const uint32_t row = stage + (uint32_t)c * kSlabBytes + (uint32_t)r * 128u;   // 32 floats
+                        for (int jj = 0; jj < 32; ++jj) {
+                            const int col = 32 * cc + jj;
+                            float p = fast_exp2(__uint_as_float(vs[jj]) * a.scale_log2 - m_s);
+                            const bool vis = row_valid && col >= c_lo && col < c_hi;
+                            p = vis ? p : 0.f;
+                            l += p;
+                            dot += vis ? p * __uint_as_float(vd[jj]) : 0.f;
+                        }
+                    }
+                    const float inv_l = row_valid ? 1.f / l : 0.f;
+                    const float delta = dot * inv_l;
+                    const uint32_t rowP = sXP + (uint32_t)r * 128u, rowS = sdS + (uint32_t)r * 128u;
+#pragma unroll 1
+                    for (int cc = 0; cc < 4; ++cc) {
+                        uint32_t pp[16], ps[16];
+                        if (warp_valid && 32 * cc < w_hi && 32 * cc + 32 > w_lo) {
+                            tmem_ld32(tmem_lane + C::kColS + 32 * cc, vs);
+                            tmem_ld32(tmem_lane + C::kColDP + 32 * cc, vd);
 #pragma unroll
-                        for (int i = 0; i < 8; ++i)
-                            st_shared_v4(row + (uint32_t)((i ^ (r & 7)) * 16), v[4 * i], v[4 * i + 1], v[4 * i + 2],
-                                         v[4 * i + 3]);
+                            for (int jj = 0; jj < 32; jj += 2) {
+                                float pv[2], dv[2];
+#pragma unroll
+                                for (int e = 0; e < 2; ++e) {
+                                    const int col = 32 * cc + jj + e;
+                                    const bool vis = row_valid && col >= c_lo && col < c_hi;
+                                    float p = fast_exp2(__uint_as_float(vs[jj + e]) * a.scale_log2 - m_s) * inv_l;
+                                    p = vis ? p : 0.f;
+                                    pv[e] = p;
+                                    dv[e] = vis ? p * (__uint_as_float(vd[jj + e]) - delta) * a.scale : 0.f;
+                                }
+                                pp[jj >> 1] = pack_bf16x2(pv[0], pv[1]);
+                                ps[jj >> 1] = pack_bf16x2(dv[0], dv[1]);
+                            }
+                        } else {
+#pragma unroll
+                            for (int jj = 0; jj < 16; ++jj) { pp[jj] = 0u; ps[jj] = 0u; }
+                        }
+                        const uint32_t slab = (uint32_t)(cc >> 1) * kSlabBytes;
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const uint32_t chunk = (uint32_t)(((cc & 1) * 4 + i) ^ (r & 7)) * 16;
+                            st_shared_v4(rowP + slab + chunk, pp[4 * i], pp[4 * i + 1], pp[4 * i + 2], pp[4 * i + 3]);
+                            st_shared_v4(rowS + slab + chunk, ps[4 * i], ps[4 * i + 1], ps[4 * i + 2], ps[4 * i + 3]);
+                        }
                     }
                 }
+                fence_proxy_async_smem();
+                tc_fence_before();
+                wg_sync();
+
+                // ---- G_i = P^T G (first hop: dV += P^T G), dQ = dS K, dK += dS^T Q
+                if (tid == 0) {
+                    tc_fence_after();
+                    const uint32_t g_acc = tmem_base + (a.first_hop ? C::kColDV : C::kColS);
+                    for (int kb = 0; kb < kblocks; ++kb) {
+                        const uint32_t k_off = kb * 2048;                                  // 16 rows of 128 bytes
+                        const uint32_t a_off = (kb >> 2) * kSlabBytes + (kb & 3) * 32;     // 16 columns of a K-major tile
+                        // G_i[key, d] = sum_q P[q, key] G[q, d]
+                        tc_mma_ss(g_acc, smem_desc_sw128(sXP + k_off, kSlabBytes, 1024),
+                                  smem_desc_sw128(g_base + k_off, kSlabBytes, 1024), idesc_g,
+                                  (kb > 0 || (a.first_hop && j > 0)) ? 1u : 0u);
+                        // dQ[q, d] = sum_key dS[q, key] K[key, d]
+                        tc_mma_ss(tmem_base + C::kColDP, smem_desc_sw128(sdS + a_off, 16, 1024),
+                                  smem_desc_sw128(sK + k_off, kSlabBytes, 1024), idesc_dq, kb > 0);
+                        // dK[key, d] += sum_q dS[q, key] Q[q, d]   (summed over the heads of the item)
+                        tc_mma_ss(tmem_base + C::kColDK, smem_desc_sw128(sdS + k_off, kSlabBytes, 1024),
+                                  smem_desc_sw128(q_base + k_off, kSlabBytes, 1024), idesc_g,
+                                  (kb > 0 || j > 0) ? 1u : 0u);
+                    }
+                    tc_commit(o_done);
+                    tc_commit(xp_free);                // the X / P slot may take the next head's X
+                    if (last_head) tc_commit(k_free);
+                }
+                __syncwarp();
+                ok = mbar_wait_abortable(o_done, par, 0x75, abort_flag);
+                ok = wg_all(ok);
+                if (!ok) break;
+                tc_fence_after();
+
+                // ---- epilogue: dQ (fp32, over this head's Q and G tiles) and G_i (bf16, over dS)
+                stage_f32(C::kColDP, q_base);
+                if (!a.first_hop && warp_valid) {
+                    uint32_t v[32];
+#pragma unroll 1
+                    for (int cc = 0; cc < D / 32; ++cc) {
+                        tmem_ld32(tmem_lane + C::kColS + 32 * cc, v);
+                        if (!row_valid) continue;
+                        uint32_t pk[16];
+#pragma unroll
+                        for (int jj = 0; jj < 32; jj += 2)
+                            pk[jj >> 1] = pack_bf16x2(__uint_as_float(v[jj]), __uint_as_float(v[jj + 1]));
+                        const uint32_t row = sdS + (uint32_t)(cc >> 1) * kSlabBytes + (uint32_t)r * 128u;
+#pragma unroll
+                        for (int i = 0; i < 4; ++i)
+                            st_shared_v4(row + (uint32_t)((((cc & 1) * 4 + i) ^ (r & 7)) * 16), pk[4 * i], pk[4 * i + 1],
+                                         pk[4 * i + 2], pk[4 * i + 3]);
+                    }
+                }
+                fence_proxy_async_smem();
+                tc_fence_before();
+                wg_sync();
+                if (tid == 0) {
+#pragma unroll
+                    for (int sl = 0; sl < D / 32; ++sl) {
+                        if (a.accumulate)
+                            tma_reduce_add_5d(&map_dq, q_base + sl * kSlabBytes, 32 * sl, 0, c.c_inner, c.c_outer, q_head);
+                        else
+                            tma_store_5d(&map_dq, q_base + sl * kSlabBytes, 32 * sl, 0, c.c_inner, c.c_outer, q_head);
+                    }
+                    if (!a.first_hop) {
+#pragma unroll
+                        for (int h = 0; h < kHalves; ++h)
+                            tma_store_5d(&map_gout, sdS + h * kSlabBytes, 64 * h, 0, c.c_inner, c.c_outer, q_head);
+                    }
+                    tma_store_commit_and_wait_read();
+                }
+                if (last_head) {
+                    // ---- once per item: dK (and, in the first hop, dV) of the whole group
+                    wg_sync();                         // the staging space has been read out
+                    tc_fence_after();
+                    stage_f32(C::kColDK, q_base);
+                    fence_proxy_async_smem();
+                    tc_fence_before();
+                    wg_sync();
+                    if (tid == 0) {
+#pragma unroll
+                        for (int sl = 0; sl < D / 32; ++sl) {
+                            if (a.accumulate)
+                                tma_reduce_add_5d(&map_dk, q_base + sl * kSlabBytes, 32 * sl, 0, c.c_inner, c.c_outer, c.kv_head);
+                            else
+                                tma_store_5d(&map_dk, q_base + sl * kSlabBytes, 32 * sl, 0, c.c_inner, c.c_outer, c.kv_head);
+                        }
+                        tma_store_commit_and_wait_read();
+                    }
+                    if (a.first_hop) {
+                        wg_sync();
+                        tc_fence_after();
+                        stage_f32(C::kColDV, q_base);
+                        fence_proxy_async_smem();
+                        tc_fence_before();
+                        wg_sync();
+                        if (tid == 0) {
+#pragma unroll
+                            for (int sl = 0; sl < D / 32; ++sl)
+                                tma_store_5d(&map_dv, q_base + sl * kSlabBytes, 32 * sl, 0, c.c_inner, c.c_outer, c.kv_head);
+                            tma_store_commit_and_wait_read();
+                        }
+                    }
+                }
+                if (tid == 0) mbar_arrive(qg_free(s));   // this stage may take the head after next
             }
         }
-        fence_proxy_async_smem();
-        tc_fence_before();
-        const int all_ok = __syncthreads_and(ok ? 1 : 0);
-        if (tid == 0 && all_ok) {
-#pragma unroll
-            for (int s = 0; s < D / 32; ++s) {
-                tma_reduce_add_5d(&map_dq, stDQ + s * kSlabBytes, 32 * s, 0, c_inner, c_outer, q_head);
-                tma_reduce_add_5d(&map_dk, stDK + s * kSlabBytes, 32 * s, 0, c_inner, c_outer, kv_head);
-            }
-            if (a.first_hop) {
-#pragma unroll
-                for (int s = 0; s < D / 32; ++s)
-                    tma_reduce_add_5d(&map_dv, stG + s * kSlabBytes, 32 * s, 0, c_inner, c_outer, kv_head);
-            } else {
-#pragma unroll
-                for (int h = 0; h < kHalves; ++h)
-                    tma_store_5d(&map_gout, stG + h * kSlabBytes, 64 * h, 0, c_inner, c_outer, q_head);
-            }
-            tma_store_commit_and_wait_read();
-        }
-        __syncthreads();
-        if (!all_ok) break;
+        if (tid == 0) tma_store_wait_all();
     }
 
-    if (tid == 0) tma_store_wait_all();
     tc_fence_before();
     __syncthreads();
     if (warp == 0) {
         __syncwarp();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(C::kTmemCols) : "memory");
     }
 }
 
@@ -345,7 +488,7 @@ __global__ void group_sum_kernel(const __nv_bfloat16 *__restrict__ dout, TO *__r
 
 template <int D>
 int launch_bwd_d(const Problem &pb, const HopDesc &hd, const void *x, int x_heads, const void *g_in, void *g_out,
-                 float *dq_acc, float *dk_acc, float *dv_acc, bool first_hop) {
+                 float *dq_acc, float *dk_acc, float *dv_acc, bool first_hop, bool accumulate) {
     CUtensorMap mq, mk, mx, mgi, mgo, mdq, mdk, mdv;
     int rc;
     if ((rc = make_hop_map(&mq, pb.q, pb.B * pb.H, pb.N, D, hd, 2)) != TA_OK) return rc;
@@ -361,8 +504,9 @@ int launch_bwd_d(const Problem &pb, const HopDesc &hd, const void *x, int x_head
     a.n = hd.n; a.rows = hd.rows; a.ci = hd.ci; a.co = hd.co; a.causal = pb.causal;
     a.g = pb.H / pb.H_kv; a.H = pb.H; a.H_kv = pb.H_kv; a.x_is_kv = x_heads != pb.H ? 1 : 0;
     a.first_hop = first_hop ? 1 : 0;
+    a.accumulate = accumulate ? 1 : 0;
     a.tiles_inner = hd.tiles_inner; a.tiles_outer = hd.tiles_outer;
-    a.total_tiles = (long long)pb.B * pb.H * hd.tiles_inner * hd.tiles_outer;
+    a.total_items = (long long)pb.B * pb.H_kv * hd.tiles_inner * hd.tiles_outer;
     a.scale = pb.scale;
     a.scale_log2 = pb.scale * 1.4426950408889634f;
 
@@ -373,7 +517,7 @@ int launch_bwd_d(const Problem &pb, const HopDesc &hd, const void *x, int x_head
         if (cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || num_sms <= 0)
             num_sms = 148;
     }
-    constexpr size_t smem = 4 * (size_t)(D / 64) * kTileRows * 128 + 2 * 2 * kTileRows * 128 + 1024 + 64;
+    constexpr size_t smem = BwdCfg<D>::kSmemBytes;
     auto kern = hop_tc_bwd_kernel<D>;
     static bool configured = false;
     if (!configured) {
@@ -381,7 +525,7 @@ int launch_bwd_d(const Problem &pb, const HopDesc &hd, const void *x, int x_head
             return TA_ERR_CUDA;
         configured = true;
     }
-    const unsigned grid = (unsigned)(a.total_tiles < num_sms ? a.total_tiles : num_sms);
+    const unsigned grid = (unsigned)(a.total_items < num_sms ? a.total_items : num_sms);
     kern<<<grid, kThreads, smem, pb.stream>>>(mq, mk, mx, mgi, mgo, mdq, mdk, mdv, a);
     count_launch();
     return cudaPeekAtLastError() == cudaSuccess ? TA_OK : TA_ERR_CUDA;
@@ -390,9 +534,11 @@ int launch_bwd_d(const Problem &pb, const HopDesc &hd, const void *x, int x_head
 }  // namespace
 
 int launch_hop_tc_bwd(const Problem &pb, const HopDesc &hd, const void *x, int x_heads, const void *g_in,
-                      void *g_out, float *dq_acc, float *dk_acc, float *dv_acc, bool first_hop) {
-    if (pb.D == 128) return launch_bwd_d<128>(pb, hd, x, x_heads, g_in, g_out, dq_acc, dk_acc, dv_acc, first_hop);
-    if (pb.D == 64) return launch_bwd_d<64>(pb, hd, x, x_heads, g_in, g_out, dq_acc, dk_acc, dv_acc, first_hop);
+                      void *g_out, float *dq_acc, float *dk_acc, float *dv_acc, bool first_hop, bool accumulate) {
+    if (pb.D == 128)
+        return launch_bwd_d<128>(pb, hd, x, x_heads, g_in, g_out, dq_acc, dk_acc, dv_acc, first_hop, accumulate);
+    if (pb.D == 64)
+        return launch_bwd_d<64>(pb, hd, x, x_heads, g_in, g_out, dq_acc, dk_acc, dv_acc, first_hop, accumulate);
     return TA_ERR_UNSUPPORTED;
 }
 
