@@ -68,6 +68,34 @@ int build_plan(int B, int H, int H_kv, int N, int D, const int *dims, int ndims,
         h.path = tc_eligible(D, h.n, dtype, flags) ? PATH_TC : PATH_SIMT;
         if (h.path == PATH_TC) tile_packing(h);
     }
+    // Hop fusion: the longest run of trailing dimensions i0..ndims-1 whose product is at most one
+    // 128-row tile (all of them in the requested hop range and on the tensor-core path) becomes one
+    // pass over contiguous blocks -- Q, K and the value tensor are read once for all those hops.
+    if (!(flags & (TA_FLAG_NO_HOP_FUSION | TA_FLAG_SAVE_HOPS)) && hop_end == ndims && plan->nhops >= 2) {
+        long long block = 1;
+        int first = plan->nhops;                     // index in plan->hops of the first fused hop
+        for (int j = plan->nhops - 1; j >= 0; --j) {
+            const HopDesc &h = plan->hops[j];
+            if (h.path != PATH_TC || (long long)h.n * h.stride > 128) break;
+            block = (long long)h.n * h.stride;       // = prod(dims[h.hop ..])
+            first = j;
+        }
+        const int nf = plan->nhops - first;
+        if (nf >= 2) {
+            HopDesc f = plan->hops[first];
+            f.nf = nf;
+            for (int j = 0; j < nf; ++j) {
+                f.sub_n[j] = plan->hops[first + j].n;
+                f.sub_stride[j] = (int)plan->hops[first + j].stride;
+            }
+            f.n = (int)block;
+            f.stride = 1;
+            f.outer = (long long)N / block;
+            tile_packing(f);
+            plan->hops[first] = f;
+            plan->nhops = first + 1;
+        }
+    }
     const size_t tensor_bytes = (size_t)B * H * N * D * elem_bytes(dtype);
     const int nh = plan->nhops;
     if (nh == 0) return TA_OK;
@@ -161,7 +189,9 @@ static int forward_impl(const ta_params &p) {
     if (p.rope_base < 0.f || !(p.rope_base == p.rope_base)) return TA_ERR_INVALID_ARG;
     if (p.rope_base > 0.f && (p.D & 1)) return TA_ERR_UNSUPPORTED;
     Plan plan;
-    int rc = build_plan(p.B, p.H, p.H_kv, p.N, p.D, p.dims, p.ndims, p.dtype, p.flags, p.hop_begin,
+    // the positional encoding gives every hop its own rotated Q and K: nothing to share, no fusion
+    const unsigned plan_flags = p.flags | (p.rope_base > 0.f ? (unsigned)TA_FLAG_NO_HOP_FUSION : 0u);
+    int rc = build_plan(p.B, p.H, p.H_kv, p.N, p.D, p.dims, p.ndims, p.dtype, plan_flags, p.hop_begin,
                         p.hop_end, &plan);
     if (rc != TA_OK) return rc;
     if (!aligned16(p.q) || !aligned16(p.k) || !aligned16(p.v) || !aligned16(p.out)) return TA_ERR_ALIGNMENT;
@@ -336,7 +366,12 @@ int ta_plan_describe(int B, int H, int H_kv, int N, int D, const int *dims, int 
          dtype == TA_DTYPE_F32 ? "f32" : "bf16", plan.scratch_bytes, plan.save_bytes);
     for (int j = 0; j < plan.nhops; ++j) {
         const HopDesc &h = plan.hops[j];
-        if (h.path == PATH_TC)
+        if (h.path == PATH_TC && h.nf > 1) {
+            emit("hop=%d path=tc-fused hops=%d block=%d blocks_per_tile=%d rows=%d tiles_per_head=%lld src=%s dst=%s sub=",
+                 h.hop, h.nf, h.n, h.co, h.rows, h.tiles_inner * h.tiles_outer, buf_name(h.src), buf_name(h.dst));
+            for (int f = 0; f < h.nf; ++f) emit("%s%dx%d", f ? "," : "", h.sub_n[f], h.sub_stride[f]);
+            emit("%s", "\n");
+        } else if (h.path == PATH_TC)
             emit("hop=%d path=tc n=%d stride=%lld outer=%lld ci=%d co=%d rows=%d tiles_per_head=%lld src=%s dst=%s\n",
                  h.hop, h.n, h.stride, h.outer, h.ci, h.co, h.rows, h.tiles_inner * h.tiles_outer,
                  buf_name(h.src), buf_name(h.dst));
@@ -349,9 +384,11 @@ int ta_plan_describe(int B, int H, int H_kv, int N, int D, const int *dims, int 
 
 int ta_device_status(void) {
     if (cudaDeviceSynchronize() != cudaSuccess) return TA_ERR_CUDA;
-    unsigned int w1 = 0, w2 = 0;
-    if (read_status_tc_forward(&w1) != TA_OK || read_status_tc_backward(&w2) != TA_OK) return TA_ERR_CUDA;
-    return (w1 | w2) ? TA_ERR_TIMEOUT : TA_OK;
+    unsigned int w1 = 0, w2 = 0, w3 = 0;
+    if (read_status_tc_forward(&w1) != TA_OK || read_status_tc_backward(&w2) != TA_OK ||
+        read_status_tc_fused(&w3) != TA_OK)
+        return TA_ERR_CUDA;
+    return (w1 | w2 | w3) ? TA_ERR_TIMEOUT : TA_OK;
 }
 
 unsigned long long ta_launch_count(void) { return g_launches.load(); }

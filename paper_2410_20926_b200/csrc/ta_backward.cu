@@ -39,7 +39,7 @@ BwdLayout layout(const Plan &plan, int B, int H, int H_kv, int N, int D, bool ne
 size_t backward_workspace_bytes(int B, int H, int H_kv, int N, int D, const int *dims, int ndims, int grad_dtype,
                                 bool have_saved_hops) {
     Plan plan;
-    if (build_plan(B, H, H_kv, N, D, dims, ndims, TA_DTYPE_BF16, 0u, 0, 0, &plan) != TA_OK) return 0;
+    if (build_plan(B, H, H_kv, N, D, dims, ndims, TA_DTYPE_BF16, TA_FLAG_NO_HOP_FUSION, 0, 0, &plan) != TA_OK) return 0;
     return layout(plan, B, H, H_kv, N, D, !have_saved_hops, grad_dtype != TA_DTYPE_F32).total;
 }
 
@@ -48,7 +48,8 @@ int backward_impl(const ta_bwd_params &p) {
     if (p.dtype != TA_DTYPE_BF16) return TA_ERR_UNSUPPORTED;
     if (p.grad_dtype != TA_DTYPE_BF16 && p.grad_dtype != TA_DTYPE_F32) return TA_ERR_UNSUPPORTED;
     Plan plan;
-    int rc = build_plan(p.B, p.H, p.H_kv, p.N, p.D, p.dims, p.ndims, p.dtype, 0u, 0, 0, &plan);
+    // hop by hop: the backward needs every hop's input
+    int rc = build_plan(p.B, p.H, p.H_kv, p.N, p.D, p.dims, p.ndims, p.dtype, TA_FLAG_NO_HOP_FUSION, 0, 0, &plan);
     if (rc != TA_OK) return rc;
     for (int j = 0; j < plan.nhops; ++j)
         if (plan.hops[j].path != PATH_TC) return TA_ERR_UNSUPPORTED;   // backward exists on the tensor-core path only

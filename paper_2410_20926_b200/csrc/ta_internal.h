@@ -31,6 +31,12 @@ struct HopDesc {
     // rows = ci * co * n <= 128, row r of the tile = (co_l * ci + ci_l) * n + t.
     int ci, co, rows;
     long long tiles_inner, tiles_outer;  // per head
+    // Hop fusion: when the trailing dimensions i0..m-1 together span at most 128 tokens, their
+    // hops run as ONE tensor-core pass over contiguous blocks of n = prod(dims[i0..]) rows (stride
+    // 1): nf > 1 sub-hops, sub-hop f attends along a dimension of extent sub_n[f] whose
+    // coordinate has stride sub_stride[f] tokens inside the block.  nf <= 1: an ordinary hop.
+    int nf;
+    int sub_n[TA_MAX_DIMS], sub_stride[TA_MAX_DIMS];
 };
 
 struct Plan {
@@ -69,6 +75,8 @@ int launch_hop_simt(const Problem &pb, const HopDesc &hd, const void *xin, int x
                     void *xout);
 int launch_hop_tc(const Problem &pb, const HopDesc &hd, const void *xin, int xin_heads,
                   void *xout);
+// Fused trailing hops (hd.nf > 1), ta_tc_fused.cu; called through launch_hop_tc.
+int launch_hop_tc_fused(const Problem &pb, const HopDesc &hd, const void *xin, int xin_heads, void *xout);
 // out[b,h] = v[b, h / (H/H_kv)] (all dims equal to 1).
 int launch_broadcast_kv(const Problem &pb);
 
@@ -96,5 +104,6 @@ int make_hop_map(CUtensorMap *map, const void *base, int heads_total, int N, int
 // copies the word to *word and clears it.
 int read_status_tc_forward(unsigned int *word);
 int read_status_tc_backward(unsigned int *word);
+int read_status_tc_fused(unsigned int *word);
 
 }  // namespace ta

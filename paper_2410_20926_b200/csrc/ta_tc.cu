@@ -565,6 +565,7 @@ int launch_d(const Problem &pb, const HopDesc &hd, const void *xin, int xin_head
 }  // namespace
 
 int launch_hop_tc(const Problem &pb, const HopDesc &hd, const void *xin, int xin_heads, void *xout) {
+    if (hd.nf > 1) return launch_hop_tc_fused(pb, hd, xin, xin_heads, xout);
     if (pb.D == 128) return launch_d<128>(pb, hd, xin, xin_heads, xout);
     if (pb.D == 64) return launch_d<64>(pb, hd, xin, xin_heads, xout);
     return TA_ERR_UNSUPPORTED;

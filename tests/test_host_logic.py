@@ -120,7 +120,8 @@ def test_plan_skips_unit_dims_and_routes_generic_hops():
 
 def test_plan_tiles_never_straddle_heads():
     # n = 12: 10 segments would fit a 128-row tile, but outer = 8 is not a multiple of 10
-    _, hops = parse_plan(ta.ta_plan_describe(1, 2, 2, 96, 64, [2, 4, 12], False))
+    _, hops = parse_plan(ta.ta_plan_describe(1, 2, 2, 96, 64, [2, 4, 12], False,
+                                             flags=ta.TA_FLAG_NO_HOP_FUSION))
     last = hops[-1]
     assert int(last["co"]) == 8 and int(last["rows"]) == 96
     for h in hops:
@@ -148,3 +149,18 @@ def test_backward_validation_and_workspace_sizes():
     rc = ta.ta_backward(16, 16, 16, 16, None, 16, 16, 16, 1, 4, 2, 512, 96, [8, 64], True,
                         workspace=256, workspace_bytes=1 << 30, stream=0, check=False)
     assert rc == ta.TA_ERR_UNSUPPORTED          # head dim 96 has no tensor-core backward
+
+
+def test_plan_fuses_trailing_dimensions_that_fit_a_tile():
+    text = ta.ta_plan_describe(1, 12, 12, 512, 64, [8, 8, 8], False, ta.TA_DTYPE_BF16, 0)
+    assert "hops=2" in text.splitlines()[0]
+    assert "path=tc-fused hops=2 block=64 blocks_per_tile=2" in text and "sub=8x8,8x1" in text
+    text = ta.ta_plan_describe(1, 12, 12, 1024, 64, [16, 4, 4, 4], False, ta.TA_DTYPE_BF16, 0)
+    assert "path=tc-fused hops=3 block=64" in text and "sub=4x16,4x4,4x1" in text
+    text = ta.ta_plan_describe(1, 4, 4, 128, 128, [8, 16], True, ta.TA_DTYPE_BF16, 0)
+    assert text.splitlines()[0].startswith("hops=1") and "src=v dst=out" in text
+    # not when the block exceeds a tile, hops are kept apart on request, or a hop is generic
+    assert "tc-fused" not in ta.ta_plan_describe(1, 4, 4, 512, 64, [32, 16], True, ta.TA_DTYPE_BF16, 0)
+    assert "tc-fused" not in ta.ta_plan_describe(1, 4, 4, 512, 64, [8, 8, 8], True, ta.TA_DTYPE_BF16,
+                                                 ta.TA_FLAG_NO_HOP_FUSION)
+    assert "tc-fused" not in ta.ta_plan_describe(1, 4, 4, 512, 64, [8, 8, 8], True, ta.TA_DTYPE_F32, 0)
