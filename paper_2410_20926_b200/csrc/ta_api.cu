@@ -92,8 +92,15 @@ int build_plan(int B, int H, int H_kv, int N, int D, const int *dims, int ndims,
             f.stride = 1;
             f.outer = (long long)N / block;
             tile_packing(f);
-            plan->hops[first] = f;
-            plan->nhops = first + 1;
+            // Measured on B200: at D = 128 the fused pass is faster than the passes it replaces
+            // (HBM-bound either way, fewer bytes); at D = 64 a tile carries half the bytes, the
+            // fused pass is bound by its softmax / epilogue chain instead and only pays when the
+            // problem is so small that the launches themselves dominate.
+            const long long tiles = (long long)B * H * f.tiles_inner * f.tiles_outer;
+            if (D == 128 || tiles <= 2 * 148) {
+                plan->hops[first] = f;
+                plan->nhops = first + 1;
+            }
         }
     }
     const size_t tensor_bytes = (size_t)B * H * N * D * elem_bytes(dtype);

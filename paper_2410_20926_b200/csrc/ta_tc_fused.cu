@@ -16,10 +16,17 @@
 // The rows a row attends to in hop f are not a contiguous range of the tile, so each row keeps
 // one 128-bit visibility mask per fused hop in shared memory.
 //
-// One CTA of 128 threads per SM, persistent; the loads of the next tile are issued before the
-// current one is processed (two stages of Q, K, X).  S, P (bf16, A operand of the value MMA) and
-// O live in tensor memory.  Every wait is bounded; on expiry the CTA records an error word,
-// stops issuing work, lets its copies land, frees its TMEM and returns.
+// Persistent, one CTA per SM, warp-specialised like the per-hop kernel:
+//   warp 0      TMA producer: K once per work item (the query heads of a GQA group share it),
+//               Q and the value tile X per head, into rings of shared memory
+//   warp 1      MMA issuer: polls for whichever of S(t) = Q K^T or O(t, f) = P_f X has its
+//               operands ready (two tiles are in flight, one per warpgroup)
+//   warps 4-7   softmax + epilogue of the even tiles   } per tile: for each fused hop f, P_f from
+//   warps 8-11  softmax + epilogue of the odd tiles    } S and the row's mask, then X <- O / rowsum
+//   warp 2      TMA store of finished tiles; hands the X slot back to the producer
+// Tensor memory: S x 2 (kept for all fused hops of its tile), P x 2 (bf16, A operand of the value
+// MMA), O (x 2 at D = 64).  Every wait is bounded; when one expires the CTA raises a flag that
+// ends all its roles, waits for its copies in flight, frees its TMEM and returns.
 #include <cuda_bf16.h>
 
 #include "ta_internal.h"
@@ -29,12 +36,14 @@ namespace ta {
 namespace {
 
 constexpr int kTileRows = 128;
-constexpr int kThreads = 128;
+constexpr int kThreads = 384;
+constexpr int kNK = 2, kNQ = 2;
 
 struct FusedArgs {
     int block, rows, co, causal, g, H, H_kv, xin_is_kv, nf;
+    int gi, hsplit;            // query heads per work item, items per GQA group
     int sub_n[TA_MAX_DIMS], sub_stride[TA_MAX_DIMS];
-    long long tiles_outer, total_tiles;
+    long long tiles_outer, total_items;
     float scale_log2;
 };
 
@@ -43,14 +52,33 @@ struct FusedCfg {
     static constexpr int kHalves = D / 64;
     static constexpr uint32_t kSlabBytes = kTileRows * 128;
     static constexpr uint32_t kTileBytes = kHalves * kSlabBytes;
-    static constexpr uint32_t kStageBytes = 3 * kTileBytes;                 // Q, K, X
-    static constexpr uint32_t kOffMask = 2 * kStageBytes;                   // [nf][128 rows][4 words]
+    static constexpr int kNX = D == 128 ? 2 : 4;                             // value-tile ring
+    static constexpr uint32_t kOffK = 0;
+    static constexpr uint32_t kOffQ = kOffK + kNK * kTileBytes;
+    static constexpr uint32_t kOffX = kOffQ + kNQ * kTileBytes;
+    static constexpr uint32_t kOffMask = kOffX + kNX * kTileBytes;          // [hop][128 rows][4 words]
     static constexpr uint32_t kMaskBytes = TA_MAX_DIMS * kTileRows * 16;
     static constexpr uint32_t kOffBar = kOffMask + kMaskBytes;
-    static constexpr uint32_t kSmemBytes = kOffBar + 4 * 8 + 16 + 1024;
+    static constexpr int kNumBars = 2 * kNK + 2 * kNQ + 3 * kNX + 2 + 2 + 2 + 2;
+    static constexpr uint32_t kSmemBytes = kOffBar + kNumBars * 8 + 16 + 1024;
     static constexpr uint32_t kTmemCols = 512;
-    static constexpr uint32_t kColS = 0, kColP = 128, kColO = 256;
+    // S: 2 x 128 | O: one buffer of 128 columns (D = 128) or two of 64 (D = 64) | P: 2 x 64
+    static constexpr uint32_t kColS = 0, kColO = 256, kColP = 384;
+    static constexpr int kNO = D == 64 ? 2 : 1;
 };
+
+struct FusedItem {
+    int c_outer, kv_head, q_head0;
+};
+__device__ __forceinline__ FusedItem decode_fused_item(const FusedArgs &a, long long item) {
+    FusedItem c;
+    long long rest = item;
+    const int hs = (int)(rest % a.hsplit); rest /= a.hsplit;
+    c.c_outer = (int)(rest % a.tiles_outer) * a.co; rest /= a.tiles_outer;
+    c.kv_head = (int)rest;
+    c.q_head0 = (c.kv_head / a.H_kv) * a.H + (c.kv_head % a.H_kv) * a.g + hs * a.gi;
+    return c;
+}
 
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
@@ -64,50 +92,64 @@ hop_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     using C = FusedCfg<D>;
     constexpr int kHalves = C::kHalves;
     constexpr uint32_t kSlabBytes = C::kSlabBytes, kTileBytes = C::kTileBytes;
+    constexpr int kNX = C::kNX, kNO = C::kNO;
 
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const uint32_t s0 = smem_u32(smem);
-    auto sQ = [&](int s) { return s0 + (uint32_t)s * C::kStageBytes; };
-    auto sK = [&](int s) { return s0 + (uint32_t)s * C::kStageBytes + kTileBytes; };
-    auto sX = [&](int s) { return s0 + (uint32_t)s * C::kStageBytes + 2 * kTileBytes; };
+    const uint32_t sK = s0 + C::kOffK, sQ = s0 + C::kOffQ, sX = s0 + C::kOffX;
     uint32_t *masks = (uint32_t *)(smem + C::kOffMask);
     const uint32_t bar0 = s0 + C::kOffBar;
-    auto full = [&](int s) { return bar0 + 8u * (uint32_t)s; };
-    const uint32_t bar_s = bar0 + 16, bar_o = bar0 + 24;
-    uint32_t *tmem_slot = (uint32_t *)(smem + C::kOffBar + 32);
+    auto k_full = [&](int i) { return bar0 + 8u * (uint32_t)i; };
+    auto k_free = [&](int i) { return bar0 + 8u * (uint32_t)(kNK + i); };
+    auto q_full = [&](int i) { return bar0 + 8u * (uint32_t)(2 * kNK + i); };
+    auto q_free = [&](int i) { return bar0 + 8u * (uint32_t)(2 * kNK + kNQ + i); };
+    constexpr int kB0 = 2 * kNK + 2 * kNQ;
+    auto x_full = [&](int i) { return bar0 + 8u * (uint32_t)(kB0 + i); };
+    auto x_free = [&](int i) { return bar0 + 8u * (uint32_t)(kB0 + kNX + i); };
+    auto out_full = [&](int i) { return bar0 + 8u * (uint32_t)(kB0 + 2 * kNX + i); };
+    constexpr int kB1 = kB0 + 3 * kNX;
+    auto s_full = [&](int i) { return bar0 + 8u * (uint32_t)(kB1 + i); };       // S(t) complete, per warpgroup
+    auto p_full = [&](int i) { return bar0 + 8u * (uint32_t)(kB1 + 2 + i); };   // P_f written (4 warps)
+    auto o_full = [&](int i) { return bar0 + 8u * (uint32_t)(kB1 + 4 + i); };   // O(t, f) complete
+    auto o_free = [&](int i) { return bar0 + 8u * (uint32_t)(kB1 + 6 + i); };   // O read out (4 warps)
+    uint32_t *tmem_slot = (uint32_t *)(smem + C::kOffBar + C::kNumBars * 8);
+    volatile uint32_t *abort_flag = tmem_slot + 1;
 
-    const int tid = threadIdx.x, warp = tid >> 5;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
-    // ---- one-time setup: zero the operand stages (rows a box never fills must stay finite),
-    // barriers, tensor memory, and the visibility masks of this thread's row
-    for (uint32_t i = tid; i < C::kOffBar / 16; i += kThreads) ((uint4 *)smem)[i] = make_uint4(0, 0, 0, 0);
+    // ---- one-time setup
+    for (uint32_t i = tid; i < C::kOffBar / 16; i += kThreads)
+        ((uint4 *)smem)[i] = make_uint4(0, 0, 0, 0);   // rows a box never fills must stay finite
     if (tid == 0) {
-        for (int i = 0; i < 4; ++i) mbar_init(bar0 + 8u * (uint32_t)i, 1);
+        for (int i = 0; i < kNK; ++i) { mbar_init(k_full(i), 1); mbar_init(k_free(i), 1); }
+        for (int i = 0; i < kNQ; ++i) { mbar_init(q_full(i), 1); mbar_init(q_free(i), 1); }
+        for (int i = 0; i < kNX; ++i) { mbar_init(x_full(i), 1); mbar_init(x_free(i), 1); mbar_init(out_full(i), 4); }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(s_full(i), 1); mbar_init(p_full(i), 4); mbar_init(o_full(i), 1); mbar_init(o_free(i), 4);
+        }
+        *abort_flag = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
-    const int r = tid;                                // this thread's tile row = TMEM lane
-    const bool row_valid = r < a.rows;
-    const int blk = r / a.block, rr = r % a.block;
-    if (row_valid) {
+    if (tid < kTileRows && tid < a.rows) {
+        // visibility of the tile's columns from row `tid` in each fused hop: the mode-f vector
+        // through the row -- same block, every coordinate but the f-th equal (causal: up to its own)
+        const int blk = tid / a.block, rr = tid % a.block;
         for (int f = 0; f < a.nf; ++f) {
-            // the mode-f vector through row rr: same block, every coordinate but the f-th equal
             const int st = a.sub_stride[f], n = a.sub_n[f];
             const int coord = (rr / st) % n;
             const int first = blk * a.block + rr - coord * st;
             const int last = a.causal ? coord : n - 1;
-            uint32_t w[4] = {0u, 0u, 0u, 0u};
+            uint32_t *m = masks + ((size_t)f * kTileRows + tid) * 4;
             for (int u = 0; u <= last; ++u) {
                 const int col = first + u * st;
-                w[col >> 5] |= 1u << (col & 31);
+                m[col >> 5] |= 1u << (col & 31);
             }
-            uint32_t *m = masks + ((size_t)f * kTileRows + r) * 4;
-            m[0] = w[0]; m[1] = w[1]; m[2] = w[2]; m[3] = w[3];
         }
     }
     fence_proxy_async_smem();
-    if (warp == 0) {
+    if (warp == 3) {
         __syncwarp();
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
                      "r"(C::kTmemCols)
@@ -118,168 +160,283 @@ hop_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    const uint32_t tmem_lane = tmem_base + ((uint32_t)(warp * 32) << 16);
 
-    constexpr uint32_t idesc_s = instr_desc(128, 0);
-    constexpr uint32_t idesc_o = instr_desc(D, 1);
-    // columns any row of this warp can see: the blocks its 32 rows belong to (causal: up to the row)
-    const int w_lo = ((warp * 32) / a.block) * a.block;
-    int w_hi = min(a.rows, ((warp * 32 + 31) / a.block + 1) * a.block);
-    if (a.causal) w_hi = min(w_hi, warp * 32 + 32);
-    const bool warp_valid = warp * 32 < a.rows;
-    const int nchunks = (a.rows + 31) >> 5;
-    const int kblocks = (a.rows + 15) >> 4;
+    const long long my_items = (a.total_items - blockIdx.x + gridDim.x - 1) / gridDim.x;
+    const uint32_t T = (uint32_t)(my_items * a.gi);
     const uint32_t slab_tx = (uint32_t)a.rows * 128u;
 
-    auto issue_loads = [&](long long tile, int s) {
-        long long rest = tile;
-        const int hg = (int)(rest % a.g); rest /= a.g;
-        const int c_outer = (int)(rest % a.tiles_outer) * a.co; rest /= a.tiles_outer;
-        const int kv_head = (int)rest;
-        const int q_head = (kv_head / a.H_kv) * a.H + (kv_head % a.H_kv) * a.g + hg;
-        const int x_head = a.xin_is_kv ? kv_head : q_head;
-        mbar_expect_tx(full(s), 3 * kHalves * slab_tx);
+    if (warp == 0) {
+        // =============================================================== TMA producer
+        if (lane == 0) {
+            uint32_t t = 0, it = 0;
+            uint32_t armed = 0, last_par = 0;   // bit per barrier slot: k 0-1, q 2-3, x 4-7
+            auto arm = [&](uint32_t bit, uint32_t parity) {
+                armed |= bit;
+                last_par = parity ? (last_par | bit) : (last_par & ~bit);
+            };
+            bool ok = true;
+            for (long long item = blockIdx.x; ok && item < a.total_items; item += gridDim.x, ++it) {
+                const FusedItem c = decode_fused_item(a, item);
+                const int ks = it & 1;
+                const uint32_t kpar = (it >> 1) & 1;
+                ok = mbar_wait_abortable(k_free(ks), kpar ^ 1, 0x90, abort_flag);
+                if (!ok) break;
+                mbar_expect_tx(k_full(ks), kHalves * slab_tx);
+                arm(1u << ks, kpar);
 #pragma unroll
-        for (int h = 0; h < kHalves; ++h) tma_load_5d(sQ(s) + h * kSlabBytes, &map_q, full(s), 64 * h, 0, 0, c_outer, q_head);
+                for (int h = 0; h < kHalves; ++h)
+                    tma_load_5d(sK + ks * kTileBytes + h * kSlabBytes, &map_k, k_full(ks), 64 * h, 0, 0, c.c_outer, c.kv_head);
+                for (int j = 0; j < a.gi; ++j, ++t) {
+                    const int q_head = c.q_head0 + j;
+                    const int x_head = a.xin_is_kv ? c.kv_head : q_head;
+                    const int qs = t & 1;
+                    const uint32_t qpar = (t >> 1) & 1;
+                    ok = mbar_wait_abortable(q_free(qs), qpar ^ 1, 0x91, abort_flag);
+                    if (!ok) break;
+                    mbar_expect_tx(q_full(qs), kHalves * slab_tx);
+                    arm(4u << qs, qpar);
 #pragma unroll
-        for (int h = 0; h < kHalves; ++h) tma_load_5d(sK(s) + h * kSlabBytes, &map_k, full(s), 64 * h, 0, 0, c_outer, kv_head);
+                    for (int h = 0; h < kHalves; ++h)
+                        tma_load_5d(sQ + qs * kTileBytes + h * kSlabBytes, &map_q, q_full(qs), 64 * h, 0, 0, c.c_outer, q_head);
+                    const int xs = t % kNX;
+                    const uint32_t xpar = (t / kNX) & 1;
+                    ok = mbar_wait_abortable(x_free(xs), xpar ^ 1, 0x92, abort_flag);
+                    if (!ok) break;
+                    mbar_expect_tx(x_full(xs), kHalves * slab_tx);
+                    arm(16u << xs, xpar);
 #pragma unroll
-        for (int h = 0; h < kHalves; ++h) tma_load_5d(sX(s) + h * kSlabBytes, &map_xin, full(s), 64 * h, 0, 0, c_outer, x_head);
-    };
-
-    bool ok = true;
-    bool prefetched = false;                          // thread 0: a load is in flight into the other stage
-    uint32_t it = 0, uses_o = 0;
-    if (tid == 0 && (long long)blockIdx.x < a.total_tiles) issue_loads(blockIdx.x, 0);
-    for (long long tile = blockIdx.x; tile < a.total_tiles; tile += gridDim.x, ++it) {
-        const int s = it & 1;
-        long long rest = tile;
-        const int hg = (int)(rest % a.g); rest /= a.g;
-        const int c_outer = (int)(rest % a.tiles_outer) * a.co; rest /= a.tiles_outer;
-        const int kv_head = (int)rest;
-        const int q_head = (kv_head / a.H_kv) * a.H + (kv_head % a.H_kv) * a.g + hg;
-
-        if (tid == 0) {
-            // the other stage was read out by the store of the previous tile (waited for below)
-            prefetched = tile + gridDim.x < a.total_tiles;
-            if (prefetched) issue_loads(tile + gridDim.x, s ^ 1);
-            ok = mbar_wait(full(s), (it >> 1) & 1, 0x81);
-            if (ok) {
-                tc_fence_after();
-#pragma unroll
-                for (int kb = 0; kb < D / 16; ++kb) {
-                    const uint32_t off = (kb >> 2) * kSlabBytes + (kb & 3) * 32;
-                    tc_mma_ss(tmem_base + C::kColS, smem_desc_sw128(sQ(s) + off, 16, 1024),
-                              smem_desc_sw128(sK(s) + off, 16, 1024), idesc_s, kb > 0);
+                    for (int h = 0; h < kHalves; ++h)
+                        tma_load_5d(sX + xs * kTileBytes + h * kSlabBytes, &map_xin, x_full(xs), 64 * h, 0, 0, c.c_outer, x_head);
                 }
-                tc_commit(bar_s);
+            }
+            if (!ok) {
+                // leaving early: let the copies already issued land (bounded)
+                const unsigned long long t0 = globaltimer_ns();
+                for (int slot = 0; slot < 4 + kNX; ++slot) {
+                    if (!(armed & (1u << slot))) continue;
+                    const uint32_t bar = slot < 2 ? k_full(slot) : (slot < 4 ? q_full(slot - 2) : x_full(slot - 4));
+                    while (!mbar_try_wait(bar, (last_par >> slot) & 1u) && globaltimer_ns() - t0 < 10000000ull) {
+                    }
+                }
             }
         }
-        __syncwarp();
-        if (ok) ok = mbar_wait(bar_s, it & 1, 0x82);
-        ok = __syncthreads_and(ok ? 1 : 0) != 0;
-        if (!ok) break;
-        tc_fence_after();
-
-        for (int f = 0; f < a.nf; ++f, ++uses_o) {
-            // ---- softmax of this row over its mode-f vector; P (un-normalised, bf16) -> tensor memory
-            const uint32_t *mword = masks + ((size_t)f * kTileRows + r) * 4;   // this row's visibility bits
-            float m = -INFINITY;
-            uint32_t v[32];
-#pragma unroll 1
-            for (int c = 0; c < nchunks; ++c) {
-                if (!(warp_valid && 32 * c < w_hi && 32 * c + 32 > w_lo)) continue;   // warp-uniform
-                tmem_ld32(tmem_lane + C::kColS + 32 * c, v);
-                const uint32_t bits = mword[c];
+    } else if (warp == 1) {
+        // =============================================================== MMA issuer
+        // Two tiles are in flight, one per warpgroup ("chain" b = tile parity).  A chain is busy
+        // from its S = Q K^T until the value MMA of its last fused hop has been issued.
+        if (lane == 0) {
+            constexpr uint32_t idesc_s = instr_desc(128, 0);
+            constexpr uint32_t idesc_o = instr_desc(D, 1);
+            const int kblocks = (a.rows + 15) >> 4;
+            uint32_t t1 = 0, it = 0, j = 0, tiles_done = 0;
+            bool busy[2] = {false, false};
+            uint32_t tile_of[2] = {0, 0}, hop_of[2] = {0, 0};   // chain: its tile and next fused hop
+            uint32_t p_seen[2] = {0, 0};                        // phases of p_full(b) consumed
+            uint32_t o_issued[2] = {0, 0};                      // value MMAs issued by chain b
+            int last_user[2] = {-1, -1};                        // chain that last wrote each O buffer
+            uint32_t idle = 0;
+            unsigned long long idle_since = 0;
+            while (tiles_done < T) {
+                bool progressed = false;
+                const int b1 = t1 & 1;
+                if (t1 < T && !busy[b1]) {
+                    const int ks = it & 1, qs = t1 & 1;
+                    if ((j != 0 || mbar_test_wait(k_full(ks), (it >> 1) & 1)) && mbar_test_wait(q_full(qs), (t1 >> 1) & 1)) {
+                        tc_fence_after();
+                        const uint32_t q_base = sQ + qs * kTileBytes, k_base = sK + ks * kTileBytes;
 #pragma unroll
-                for (int jj = 0; jj < 32; ++jj)
-                    if ((bits >> jj) & 1u) m = fmaxf(m, __uint_as_float(v[jj]));
-            }
-            const float m_scaled = row_valid ? m * a.scale_log2 : 0.f;
-            float sum = 0.f;
-#pragma unroll 1
-            for (int c = 0; c < nchunks; ++c) {
-                uint32_t pk[16];
-                if (warp_valid && 32 * c < w_hi && 32 * c + 32 > w_lo) {
-                    tmem_ld32(tmem_lane + C::kColS + 32 * c, v);
-                    const uint32_t bits = mword[c];
-#pragma unroll
-                    for (int jj = 0; jj < 32; jj += 2) {
-                        float p0 = fast_exp2(__uint_as_float(v[jj]) * a.scale_log2 - m_scaled);
-                        float p1 = fast_exp2(__uint_as_float(v[jj + 1]) * a.scale_log2 - m_scaled);
-                        p0 = ((bits >> jj) & 1u) ? p0 : 0.f;
-                        p1 = ((bits >> (jj + 1)) & 1u) ? p1 : 0.f;
-                        const uint32_t w = pack_bf16x2(p0, p1);
-                        pk[jj >> 1] = w;
-                        sum += __uint_as_float(w << 16) + __uint_as_float(w & 0xFFFF0000u);
+                        for (int kb = 0; kb < D / 16; ++kb) {
+                            const uint32_t off = (kb >> 2) * kSlabBytes + (kb & 3) * 32;
+                            tc_mma_ss(tmem_base + C::kColS + b1 * 128, smem_desc_sw128(q_base + off, 16, 1024),
+                                      smem_desc_sw128(k_base + off, 16, 1024), idesc_s, kb > 0);
+                        }
+                        tc_commit(s_full(b1));
+                        tc_commit(q_free(qs));
+                        if (++j == (uint32_t)a.gi) {
+                            tc_commit(k_free(ks));
+                            j = 0;
+                            ++it;
+                        }
+                        busy[b1] = true;
+                        tile_of[b1] = t1;
+                        hop_of[b1] = 0;
+                        ++t1;
+                        progressed = true;
                     }
-                } else {
-#pragma unroll
-                    for (int jj = 0; jj < 16; ++jj) pk[jj] = 0u;
                 }
-                tmem_st16(tmem_lane + C::kColP + 16 * c, pk);
+#pragma unroll
+                for (int k = 0; k < 2; ++k) {
+                    const int b = (t1 + k) & 1;                 // the older tile first
+                    if (!busy[b]) continue;
+                    const uint32_t tile = tile_of[b];
+                    const int xs = tile % kNX;
+                    const int ob = kNO == 2 ? b : 0;
+                    const int lu = last_user[ob];
+                    if (!mbar_test_wait(p_full(b), p_seen[b] & 1)) continue;
+                    if (hop_of[b] == 0 && !mbar_test_wait(x_full(xs), (tile / kNX) & 1)) continue;
+                    if (lu >= 0 && !mbar_test_wait(o_free(lu), (o_issued[lu] - 1) & 1)) continue;
+                    tc_fence_after();
+                    // O[128 x D] = P_f[128 x rows] X[rows x D]; P from tensor memory, X MN-major from shared memory
+                    const uint32_t d_tmem = tmem_base + C::kColO + (kNO == 2 ? 64 * b : 0);
+                    const uint32_t p_tmem = tmem_base + C::kColP + 64 * b;
+                    const uint32_t x_base = sX + xs * kTileBytes;
+                    for (int kb = 0; kb < kblocks; ++kb)
+                        tc_mma_ts(d_tmem, p_tmem + kb * 8, smem_desc_sw128(x_base + kb * 2048, kSlabBytes, 1024), idesc_o,
+                                  kb > 0);
+                    tc_commit(o_full(b));
+                    ++p_seen[b];
+                    ++o_issued[b];
+                    last_user[ob] = b;
+                    if (++hop_of[b] == (uint32_t)a.nf) {
+                        busy[b] = false;
+                        ++tiles_done;
+                    }
+                    progressed = true;
+                }
+                if (progressed) {
+                    idle = 0;
+                    idle_since = 0;
+                } else if (++idle < 1024) {
+                    __nanosleep(40);
+                } else {
+                    idle = 0;
+                    if (*abort_flag) break;
+                    const unsigned long long now = globaltimer_ns();
+                    if (idle_since == 0) idle_since = now;
+                    if (now - idle_since > kWaitLimitNs) {
+                        atomicCAS(&g_status_word, 0u, kErrWaitExpired | 0xA0u);
+                        *abort_flag = 1u;
+                        break;
+                    }
+                }
             }
-            tmem_st_wait();
-            const float inv = row_valid ? 1.f / sum : 1.f;
-            tc_fence_before();
-            __syncthreads();
+        }
+    } else if (warp == 2) {
+        // =============================================================== TMA store
+        if (lane == 0) {
+            uint32_t t = 0;
+            bool ok = true;
+            for (long long item = blockIdx.x; ok && item < a.total_items; item += gridDim.x) {
+                const FusedItem c = decode_fused_item(a, item);
+                for (int j = 0; j < a.gi; ++j, ++t) {
+                    const int xs = t % kNX;
+                    ok = mbar_wait_abortable(out_full(xs), (t / kNX) & 1, 0xB0, abort_flag);
+                    if (!ok) break;
+#pragma unroll
+                    for (int h = 0; h < kHalves; ++h)
+                        tma_store_5d(&map_xout, sX + xs * kTileBytes + h * kSlabBytes, 64 * h, 0, 0, c.c_outer, c.q_head0 + j);
+                    tma_store_commit_and_wait_read();
+                    mbar_arrive(x_free(xs));
+                }
+            }
+            tma_store_wait_all();
+        }
+    } else if (warp >= 4) {
+        // =============================================================== softmax + epilogue
+        const int b = (warp - 4) >> 2;                  // tile parity this warpgroup serves
+        const int wq = warp & 3;                        // TMEM lane quarter of this warp
+        const uint32_t tmem_lane = tmem_base + ((uint32_t)(wq * 32) << 16);
+        const int r = wq * 32 + lane;                   // this thread's tile row = TMEM lane
+        const bool row_valid = r < a.rows;
+        // columns any row of this warp can see: the blocks its 32 rows belong to (causal: up to the row)
+        const int w_lo = ((wq * 32) / a.block) * a.block;
+        int w_hi = min(a.rows, ((wq * 32 + 31) / a.block + 1) * a.block);
+        if (a.causal) w_hi = min(w_hi, wq * 32 + 32);
+        const bool warp_valid = wq * 32 < a.rows;
+        const int nchunks = (a.rows + 31) >> 5;
+        const uint32_t s_col = tmem_lane + C::kColS + b * 128, p_col = tmem_lane + C::kColP + b * 64;
+        const uint32_t o_col = tmem_lane + C::kColO + (kNO == 2 ? 64 * b : 0);
 
-            // ---- X <- P X
-            if (tid == 0) {
-                tc_fence_after();
-                for (int kb = 0; kb < kblocks; ++kb)
-                    tc_mma_ts(tmem_base + C::kColO, tmem_base + C::kColP + kb * 8,
-                              smem_desc_sw128(sX(s) + kb * 2048, kSlabBytes, 1024), idesc_o, kb > 0);
-                tc_commit(bar_o);
-            }
-            __syncwarp();
-            ok = mbar_wait(bar_o, uses_o & 1, 0x83);
-            ok = __syncthreads_and(ok ? 1 : 0) != 0;
+        bool ok = true;
+        uint32_t o_seen = 0;                            // phases of o_full(b) consumed
+        for (uint32_t t = b; ok && t < T; t += 2) {
+            ok = mbar_wait_abortable(s_full(b), (t >> 1) & 1, 0xC0, abort_flag);
+            ok = __all_sync(0xffffffffu, ok);           // keep the warp converged for the aligned TMEM ops
             if (!ok) break;
             tc_fence_after();
-            if (warp_valid) {
-                const uint32_t x_row = sX(s) + (uint32_t)r * 128u;
+            const int xs = t % kNX;
+            for (int f = 0; f < a.nf; ++f, ++o_seen) {
+                // ---- softmax of this row over its mode-f vector; P (un-normalised, bf16) -> tensor memory
+                const uint32_t *mword = masks + ((size_t)f * kTileRows + r) * 4;
+                float m = -INFINITY;
+                uint32_t v[32];
 #pragma unroll 1
-                for (int c = 0; c < D / 32; ++c) {
-                    tmem_ld32(tmem_lane + C::kColO + 32 * c, v);
+                for (int c = 0; c < nchunks; ++c) {
+                    if (!(warp_valid && 32 * c < w_hi && 32 * c + 32 > w_lo)) continue;   // warp-uniform
+                    tmem_ld32(s_col + 32 * c, v);
+                    const uint32_t bits = mword[c];
+#pragma unroll
+                    for (int jj = 0; jj < 32; ++jj)
+                        if ((bits >> jj) & 1u) m = fmaxf(m, __uint_as_float(v[jj]));
+                }
+                const float m_scaled = row_valid ? m * a.scale_log2 : 0.f;
+                float sum = 0.f;
+#pragma unroll 1
+                for (int c = 0; c < nchunks; ++c) {
                     uint32_t pk[16];
+                    if (warp_valid && 32 * c < w_hi && 32 * c + 32 > w_lo) {
+                        tmem_ld32(s_col + 32 * c, v);
+                        const uint32_t bits = mword[c];
 #pragma unroll
-                    for (int jj = 0; jj < 32; jj += 2)
-                        pk[jj >> 1] = pack_bf16x2(__uint_as_float(v[jj]) * inv, __uint_as_float(v[jj + 1]) * inv);
-                    if (row_valid) {
-                        const uint32_t slab = x_row + (uint32_t)(c >> 1) * kSlabBytes;
+                        for (int jj = 0; jj < 32; jj += 2) {
+                            float p0 = fast_exp2(__uint_as_float(v[jj]) * a.scale_log2 - m_scaled);
+                            float p1 = fast_exp2(__uint_as_float(v[jj + 1]) * a.scale_log2 - m_scaled);
+                            p0 = ((bits >> jj) & 1u) ? p0 : 0.f;
+                            p1 = ((bits >> (jj + 1)) & 1u) ? p1 : 0.f;
+                            const uint32_t w = pack_bf16x2(p0, p1);
+                            pk[jj >> 1] = w;
+                            sum += __uint_as_float(w << 16) + __uint_as_float(w & 0xFFFF0000u);
+                        }
+                    } else {
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            const uint32_t chunk = (uint32_t)(((c & 1) * 4 + i) ^ (r & 7));
-                            st_shared_v4(slab + chunk * 16, pk[4 * i], pk[4 * i + 1], pk[4 * i + 2], pk[4 * i + 3]);
+                        for (int jj = 0; jj < 16; ++jj) pk[jj] = 0u;
+                    }
+                    tmem_st16(p_col + 16 * c, pk);
+                }
+                tmem_st_wait();
+                const float inv = row_valid ? 1.f / sum : 1.f;
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(p_full(b));
+
+                // ---- X <- O / rowsum (bf16, in place in the value slot: the next fused hop's operand,
+                // and after the last one the tile the store warp writes out)
+                ok = mbar_wait_abortable(o_full(b), o_seen & 1, 0xC1, abort_flag);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                tc_fence_after();
+                if (warp_valid) {
+                    const uint32_t x_row = sX + xs * kTileBytes + (uint32_t)r * 128u;
+#pragma unroll 1
+                    for (int c = 0; c < D / 32; ++c) {
+                        tmem_ld32(o_col + 32 * c, v);
+                        uint32_t pk[16];
+#pragma unroll
+                        for (int jj = 0; jj < 32; jj += 2)
+                            pk[jj >> 1] = pack_bf16x2(__uint_as_float(v[jj]) * inv, __uint_as_float(v[jj + 1]) * inv);
+                        if (row_valid) {
+                            const uint32_t slab = x_row + (uint32_t)(c >> 1) * kSlabBytes;
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                const uint32_t chunk = (uint32_t)(((c & 1) * 4 + i) ^ (r & 7));
+                                st_shared_v4(slab + chunk * 16, pk[4 * i], pk[4 * i + 1], pk[4 * i + 2], pk[4 * i + 3]);
+                            }
                         }
                     }
                 }
+                fence_proxy_async_smem();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(o_free(b));
             }
-            fence_proxy_async_smem();     // the next MMA (or the store) reads X through the async proxy
-            tc_fence_before();
-            __syncthreads();
-        }
-        if (!ok) break;
-        if (tid == 0) {
-#pragma unroll
-            for (int h = 0; h < kHalves; ++h) tma_store_5d(&map_xout, sX(s) + h * kSlabBytes, 64 * h, 0, 0, c_outer, q_head);
-            tma_store_commit_and_wait_read();
-            prefetched = false;           // (re-evaluated at the top of the next iteration)
+            if (!ok) break;
+            if (lane == 0) mbar_arrive(out_full(xs));
         }
     }
-    if (tid == 0) {
-        if (!ok && prefetched) {
-            // leaving early: let the load in flight land before shared memory is released
-            const unsigned long long t0 = globaltimer_ns();
-            while (!mbar_try_wait(full((it & 1) ^ 1), ((it + 1) >> 1) & 1) && globaltimer_ns() - t0 < 10000000ull) {
-            }
-        }
-        tma_store_wait_all();
-    }
+
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) {
+    if (warp == 3) {
         __syncwarp();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(C::kTmemCols) : "memory");
     }
@@ -302,10 +459,6 @@ int launch_fused_d(const Problem &pb, const HopDesc &hd, const void *xin, int xi
         a.sub_n[f] = f < hd.nf ? hd.sub_n[f] : 1;
         a.sub_stride[f] = f < hd.nf ? hd.sub_stride[f] : 1;
     }
-    a.tiles_outer = hd.tiles_outer;
-    a.total_tiles = (long long)pb.B * pb.H * hd.tiles_outer;
-    a.scale_log2 = pb.scale * 1.4426950408889634f;
-
     static int num_sms = 0;
     if (num_sms == 0) {
         int dev = 0;
@@ -313,6 +466,15 @@ int launch_fused_d(const Problem &pb, const HopDesc &hd, const void *xin, int xi
         if (cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || num_sms <= 0)
             num_sms = 148;
     }
+    a.tiles_outer = hd.tiles_outer;
+    // a work item = the gi query heads of a GQA group on one tile position (they share the K tile)
+    const long long positions = (long long)pb.B * pb.H_kv * hd.tiles_outer;
+    a.hsplit = 1;
+    for (int d = 2; d <= a.g && positions * a.hsplit < 2ll * num_sms; ++d)
+        if (a.g % d == 0) a.hsplit = d;
+    a.gi = a.g / a.hsplit;
+    a.total_items = positions * a.hsplit;
+    a.scale_log2 = pb.scale * 1.4426950408889634f;
     constexpr size_t smem = FusedCfg<D>::kSmemBytes;
     auto kern = hop_fused_kernel<D>;
     static bool configured = false;
@@ -321,7 +483,7 @@ int launch_fused_d(const Problem &pb, const HopDesc &hd, const void *xin, int xi
             return TA_ERR_CUDA;
         configured = true;
     }
-    const unsigned grid = (unsigned)(a.total_tiles < num_sms ? a.total_tiles : num_sms);
+    const unsigned grid = (unsigned)(a.total_items < num_sms ? a.total_items : num_sms);
     kern<<<grid, kThreads, smem, pb.stream>>>(mq, mk, mxi, mxo, a);
     count_launch();
     return cudaPeekAtLastError() == cudaSuccess ? TA_OK : TA_ERR_CUDA;
