@@ -79,9 +79,10 @@ enum { TA_WS_FORWARD = 0, TA_WS_FORWARD_SAVE = 1, TA_WS_BACKWARD = 2, TA_WS_BACK
  *   out [B,H,N,D]: device, bf16, written (used as the in-place value tensor between hops).
  *   dims: host array of ndims positive ints, prod == N.  causal: 0 or 1.
  * Scale is 1/sqrt(D) in every hop (Eq. 4).
- * Hops the tensor-core kernel covers (D in {64,128}, n_i <= 128) run in place in `out` and
- * need no other memory.  Other hops (large n_i, other D) run on the generic kernel, which
- * cannot update in place: for them the library uses an internal device scratch buffer of
+ * Hops with D in {64,128} and n_i <= 128 run on the tensor-core kernel in place in `out` and
+ * need no other memory.  Hops with n_i > 128 (key-block loop with online softmax on the tensor
+ * cores, D in {64,128}) and hops with another D (generic CUDA-core kernel) cannot update in
+ * place: for them the library uses an internal device scratch buffer of
  * B*H*N*D elements that it allocates on first need and keeps (cudaMalloc: synchronous, so
  * such a first call must not happen during stream capture).  ta_forward_ex takes a caller
  * workspace instead.

@@ -28,8 +28,8 @@ int validate_shape(int B, int H, int H_kv, int N, int D, const int *dims, int nd
     return TA_OK;
 }
 
-static bool tc_eligible(int D, int n, int dtype, unsigned flags) {
-    return dtype == TA_DTYPE_BF16 && (D == 64 || D == 128) && n <= 128 && !(flags & TA_FLAG_NO_TENSOR_CORE);
+static bool tc_eligible(int D, int dtype, unsigned flags) {
+    return dtype == TA_DTYPE_BF16 && (D == 64 || D == 128) && !(flags & TA_FLAG_NO_TENSOR_CORE);
 }
 
 // Packs whole segments into a 128-row tile: ci consecutive `inner` positions, then co
@@ -52,7 +52,7 @@ int build_plan(int B, int H, int H_kv, int N, int D, const int *dims, int ndims,
                unsigned flags, int hop_begin, int hop_end, Plan *plan) {
     int rc = validate_shape(B, H, H_kv, N, D, dims, ndims, dtype);
     if (rc != TA_OK) return rc;
-    if (flags & ~(unsigned)(TA_FLAG_NO_TENSOR_CORE | TA_FLAG_NO_HOP_FUSION | TA_FLAG_SAVE_HOPS))
+    if (flags & ~(unsigned)(TA_FLAG_NO_TENSOR_CORE | TA_FLAG_NO_HOP_FUSION | TA_FLAG_SAVE_HOPS | kPlanFlagRope))
         return TA_ERR_UNSUPPORTED;
     if (hop_begin == 0 && hop_end == 0) hop_end = ndims;
     if (hop_begin < 0 || hop_end > ndims || hop_begin > hop_end) return TA_ERR_INVALID_ARG;
@@ -65,7 +65,11 @@ int build_plan(int B, int H, int H_kv, int N, int D, const int *dims, int ndims,
         h.stride = 1;
         for (int l = i + 1; l < ndims; ++l) h.stride *= dims[l];
         h.outer = (long long)N / ((long long)h.n * h.stride);
-        h.path = tc_eligible(D, h.n, dtype, flags) ? PATH_TC : PATH_SIMT;
+        h.path = PATH_SIMT;
+        if (tc_eligible(D, dtype, flags)) {
+            if (h.n <= 128) h.path = PATH_TC;
+            else if (!(flags & kPlanFlagRope)) h.path = PATH_TC_LONG;   // the long-segment kernel does not rotate
+        }
         if (h.path == PATH_TC) tile_packing(h);
     }
     // Hop fusion: the longest run of trailing dimensions i0..ndims-1 whose product is at most one
@@ -129,7 +133,7 @@ int build_plan(int B, int H, int H_kv, int N, int D, const int *dims, int ndims,
             dst = h.src;
         }
     }
-    if (plan->hops[0].path == PATH_SIMT && plan->hops[0].src == plan->hops[0].dst) {
+    if (plan->hops[0].path != PATH_TC && plan->hops[0].src == plan->hops[0].dst) {
         // only reachable with hop_begin > 0: the caller's `out` is first copied to scratch
         plan->hops[0].src = BUF_SCRATCH;
     }
@@ -197,7 +201,8 @@ static int forward_impl(const ta_params &p) {
     if (p.rope_base > 0.f && (p.D & 1)) return TA_ERR_UNSUPPORTED;
     Plan plan;
     // the positional encoding gives every hop its own rotated Q and K: nothing to share, no fusion
-    const unsigned plan_flags = p.flags | (p.rope_base > 0.f ? (unsigned)TA_FLAG_NO_HOP_FUSION : 0u);
+    if (p.flags & kPlanFlagRope) return TA_ERR_UNSUPPORTED;
+    const unsigned plan_flags = p.flags | (p.rope_base > 0.f ? (unsigned)TA_FLAG_NO_HOP_FUSION | kPlanFlagRope : 0u);
     int rc = build_plan(p.B, p.H, p.H_kv, p.N, p.D, p.dims, p.ndims, p.dtype, plan_flags, p.hop_begin,
                         p.hop_end, &plan);
     if (rc != TA_OK) return rc;
@@ -247,8 +252,9 @@ static int forward_impl(const ta_params &p) {
         const void *xin = buffer(h.src);
         const int xin_heads = h.src == BUF_V ? p.H_kv : p.H;
         void *xout = buffer(h.dst);
-        rc = h.path == PATH_TC ? launch_hop_tc(pb, h, xin, xin_heads, xout)
-                               : launch_hop_simt(pb, h, xin, xin_heads, xout);
+        rc = h.path == PATH_TC        ? launch_hop_tc(pb, h, xin, xin_heads, xout)
+             : h.path == PATH_TC_LONG ? launch_hop_tc_long(pb, h, xin, xin_heads, xout)
+                                      : launch_hop_simt(pb, h, xin, xin_heads, xout);
         if (rc != TA_OK) return rc;
     }
     return TA_OK;
@@ -382,6 +388,9 @@ int ta_plan_describe(int B, int H, int H_kv, int N, int D, const int *dims, int 
             emit("hop=%d path=tc n=%d stride=%lld outer=%lld ci=%d co=%d rows=%d tiles_per_head=%lld src=%s dst=%s\n",
                  h.hop, h.n, h.stride, h.outer, h.ci, h.co, h.rows, h.tiles_inner * h.tiles_outer,
                  buf_name(h.src), buf_name(h.dst));
+        else if (h.path == PATH_TC_LONG)
+            emit("hop=%d path=tc-long n=%d stride=%lld outer=%lld key_blocks=%d src=%s dst=%s\n", h.hop, h.n, h.stride,
+                 h.outer, (h.n + 127) / 128, buf_name(h.src), buf_name(h.dst));
         else
             emit("hop=%d path=simt n=%d stride=%lld outer=%lld src=%s dst=%s\n", h.hop, h.n, h.stride, h.outer,
                  buf_name(h.src), buf_name(h.dst));
@@ -391,11 +400,11 @@ int ta_plan_describe(int B, int H, int H_kv, int N, int D, const int *dims, int 
 
 int ta_device_status(void) {
     if (cudaDeviceSynchronize() != cudaSuccess) return TA_ERR_CUDA;
-    unsigned int w1 = 0, w2 = 0, w3 = 0;
+    unsigned int w1 = 0, w2 = 0, w3 = 0, w4 = 0;
     if (read_status_tc_forward(&w1) != TA_OK || read_status_tc_backward(&w2) != TA_OK ||
-        read_status_tc_fused(&w3) != TA_OK)
+        read_status_tc_fused(&w3) != TA_OK || read_status_tc_long(&w4) != TA_OK)
         return TA_ERR_CUDA;
-    return (w1 | w2 | w3) ? TA_ERR_TIMEOUT : TA_OK;
+    return (w1 | w2 | w3 | w4) ? TA_ERR_TIMEOUT : TA_OK;
 }
 
 unsigned long long ta_launch_count(void) { return g_launches.load(); }

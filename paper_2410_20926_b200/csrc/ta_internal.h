@@ -15,8 +15,12 @@ enum BufferId { BUF_V = 0, BUF_OUT = 1, BUF_SCRATCH = 2 };
 
 enum HopPath {
     PATH_SIMT = 0,  // generic CUDA-core kernel, any n_i / D, fp32 or bf16 storage
-    PATH_TC = 1     // tcgen05 tensor-core kernel: bf16, D in {64,128}, n_i <= 128
+    PATH_TC = 1,     // tcgen05 tensor-core kernel: bf16, D in {64,128}, n_i <= 128 (in place)
+    PATH_TC_LONG = 2 // tcgen05 kernel with a loop over key blocks and online softmax: n_i > 128
 };
+
+// build_plan flag used inside the library only: the call carries the positional encoding
+constexpr unsigned kPlanFlagRope = 1u << 30;
 
 // One hop of Algorithm 1 as a strided view X[outer][t][inner][D] of a head:
 //   token(outer, t, inner) = outer * n * stride + t * stride + inner.
@@ -75,6 +79,9 @@ int launch_hop_simt(const Problem &pb, const HopDesc &hd, const void *xin, int x
                     void *xout);
 int launch_hop_tc(const Problem &pb, const HopDesc &hd, const void *xin, int xin_heads,
                   void *xout);
+// Long segments (n_i > 128): key-block loop with online softmax, ta_tc_long.cu.  xin != xout.
+int launch_hop_tc_long(const Problem &pb, const HopDesc &hd, const void *xin, int xin_heads, void *xout);
+int read_status_tc_long(unsigned int *word);
 // Fused trailing hops (hd.nf > 1), ta_tc_fused.cu; called through launch_hop_tc.
 int launch_hop_tc_fused(const Problem &pb, const HopDesc &hd, const void *xin, int xin_heads, void *xout);
 // out[b,h] = v[b, h / (H/H_kv)] (all dims equal to 1).
@@ -99,6 +106,9 @@ void count_launch(unsigned n = 1);
 
 // TMA map of one tensor through a hop's strided view (ta_tc.cu); elem = 2 (bf16) or 4 (fp32).
 int make_hop_map(CUtensorMap *map, const void *base, int heads_total, int N, int D, const HopDesc &hd, int elem);
+// Same view with an explicit box: box_t positions along the hop's dimension, box_inner x box_outer segments.
+int make_view_map(CUtensorMap *map, const void *base, int heads_total, int N, int D, const HopDesc &hd, int elem,
+                  int box_t, int box_inner, int box_outer);
 
 // Device error words (bounded waits that expired), one per tensor-core translation unit:
 // copies the word to *word and clears it.

@@ -88,8 +88,9 @@ extern "C" int ta_forward_static(const void *q, const void *k, const void *v, vo
         const void *xin = h.src == BUF_V ? v : (h.src == BUF_OUT ? (const void *)out : (const void *)scratch);
         void *xout = h.dst == BUF_OUT ? out : scratch;
         const int xin_heads = h.src == BUF_V ? H_kv : H;
-        rc = h.path == PATH_TC ? launch_hop_tc(pb, h, xin, xin_heads, xout)
-                               : launch_hop_simt(pb, h, xin, xin_heads, xout);
+        rc = h.path == PATH_TC        ? launch_hop_tc(pb, h, xin, xin_heads, xout)
+             : h.path == PATH_TC_LONG ? launch_hop_tc_long(pb, h, xin, xin_heads, xout)
+                                      : launch_hop_simt(pb, h, xin, xin_heads, xout);
         if (rc != TA_OK) return rc;
     }
     return TA_OK;

@@ -495,6 +495,11 @@ EncodeTiledFn encode_fn() {
 // Rank-5 map of one tensor [heads][N][D] seen through hop `hd`: dims (D, t, inner, outer, head),
 // box (128 bytes of D, n, ci, co, 1), 128-byte swizzle.  elem = 2 (bf16) or 4 (fp32).
 int make_hop_map(CUtensorMap *map, const void *base, int heads_total, int N, int D, const HopDesc &hd, int elem) {
+    return make_view_map(map, base, heads_total, N, D, hd, elem, hd.n, hd.ci, hd.co);
+}
+
+int make_view_map(CUtensorMap *map, const void *base, int heads_total, int N, int D, const HopDesc &hd, int elem,
+                  int box_t, int box_inner, int box_outer) {
     EncodeTiledFn enc = encode_fn();
     if (!enc) return TA_ERR_CUDA;
     const cuuint64_t e = (cuuint64_t)elem;
@@ -502,7 +507,7 @@ int make_hop_map(CUtensorMap *map, const void *base, int heads_total, int N, int
                           (cuuint64_t)heads_total};
     cuuint64_t gstr[4] = {(cuuint64_t)hd.stride * D * e, (cuuint64_t)D * e, (cuuint64_t)hd.n * hd.stride * D * e,
                           (cuuint64_t)N * D * e};
-    cuuint32_t box[5] = {(cuuint32_t)(128 / elem), (cuuint32_t)hd.n, (cuuint32_t)hd.ci, (cuuint32_t)hd.co, 1u};
+    cuuint32_t box[5] = {(cuuint32_t)(128 / elem), (cuuint32_t)box_t, (cuuint32_t)box_inner, (cuuint32_t)box_outer, 1u};
     cuuint32_t estr[5] = {1, 1, 1, 1, 1};
     CUresult r = enc(map, elem == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 5,
                      const_cast<void *>(base), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,

@@ -71,6 +71,25 @@ def test_mixed_paths_use_scratch():
     check_case(1, 2, 1, 4 * 160, 64, [4, 160], True, "bf16", seed=106)
 
 
+# ---------------------------------------------------------------- long segments (n > 128): key-block loop
+@pytest.mark.parametrize("dims,D,causal,H,Hkv", [
+    ([256], 128, True, 4, 2),          # ordinary causal attention, two key blocks
+    ([300], 64, False, 4, 4),          # ragged last block
+    ([2, 384], 128, True, 8, 2),
+    ([130, 3], 64, True, 2, 1),        # long hop over a strided dimension
+    ([3, 129], 128, False, 2, 2),
+    ([1000], 64, True, 2, 2),          # eight key blocks: running maximum moves many times
+])
+def test_long_segments_tensor_core(dims, D, causal, H, Hkv):
+    assert "tc-long" in ta.ta_plan_describe(1, H, Hkv, math.prod(dims), D, dims, causal, ta.TA_DTYPE_BF16, 0)
+    check_case(2, H, Hkv, math.prod(dims), D, dims, causal, "bf16", seed=113)
+
+
+def test_full_attention_4096_sampled_heads():
+    """One dimension = ordinary attention (Eq. 1) at a length where the loop runs 32 key blocks."""
+    check_case(1, 8, 2, 4096, 128, [4096], True, "bf16", seed=114, heads=[(0, 0), (0, 5)])
+
+
 def test_unit_dims_and_broadcast():
     check_case(1, 4, 2, 64, 64, [1, 64, 1], True, "bf16", seed=107)
     inp = ta_inputs.make_inputs(2, 4, 2, 1, 64, "bf16", 108)

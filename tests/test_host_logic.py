@@ -105,10 +105,12 @@ def test_plan_skips_unit_dims_and_routes_generic_hops():
     _, hops = parse_plan(ta.ta_plan_describe(1, 2, 2, 256, 64, [16, 1, 16], False))
     assert [h["hop"] for h in hops] == ["0", "2"]
     head, hops = parse_plan(ta.ta_plan_describe(1, 2, 2, 256, 64, [1, 1, 1, 256], False))
-    assert [h["path"] for h in hops] == ["simt"]                       # n > 128
+    assert [h["path"] for h in hops] == ["tc-long"]                    # n > 128: key-block loop
+    head, hops = parse_plan(ta.ta_plan_describe(1, 2, 2, 256, 96, [1, 1, 1, 256], False))
+    assert [h["path"] for h in hops] == ["simt"]                       # head dim the tensor-core kernels lack
     head, hops = parse_plan(ta.ta_plan_describe(1, 2, 2, 16384, 64, [4, 4096], False))
     assert [(h["path"], h["src"], h["dst"]) for h in hops] == \
-        [("tc", "v", "scratch"), ("simt", "scratch", "out")]
+        [("tc", "v", "scratch"), ("tc-long", "scratch", "out")]        # the long hop is not in place
     assert int(head["scratch_bytes"]) == 2 * 16384 * 64 * 2
     head, hops = parse_plan(ta.ta_plan_describe(1, 2, 2, 27, 64, [3, 3, 3], True,
                                                 dtype=ta.TA_DTYPE_F32))
