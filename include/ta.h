@@ -134,7 +134,7 @@ typedef struct ta_params {
  * tiles in shared memory, between the TMA load and the MMA -- no rotated copy of q or k ever
  * exists in global memory.  D must be even (else TA_ERR_UNSUPPORTED); a negative or NaN base
  * is TA_ERR_INVALID_ARG.  The value tensor is never rotated.
- * ta_backward does not take the positional encoding.
+ * ta_backward_ex takes the same rope_base (ta_backward, the short form, does not).
  */
 int ta_forward_ex(const ta_params *p);
 
@@ -175,6 +175,9 @@ typedef struct ta_bwd_params {
     int grad_dtype;               /* TA_DTYPE_BF16, or TA_DTYPE_F32: dq/dk/dv are the fp32      */
                                   /* accumulators themselves (no final rounding, less workspace)*/
     float softmax_scale;          /* 0 -> 1/sqrt(D)                                            */
+    float rope_base;              /* 0: none; > 0: tensorized positional encoding as in        */
+                                  /* ta_forward_ex (q, k un-rotated; dq, dk are the gradients   */
+                                  /* with respect to the un-rotated q, k).  D must be even.     */
     const void *saved_hops;       /* X_1..X_{m-1} as written by ta_forward_ex(TA_FLAG_SAVE_HOPS) */
                                   /* (the part of its workspace after the scratch tensor), or    */
                                   /* NULL: recomputed                                          */

@@ -57,7 +57,7 @@ class ta_bwd_params(ctypes.Structure):
                 ("N", ctypes.c_int), ("D", ctypes.c_int),
                 ("dims", ctypes.POINTER(ctypes.c_int)), ("ndims", ctypes.c_int),
                 ("causal", ctypes.c_int), ("dtype", ctypes.c_int), ("grad_dtype", ctypes.c_int),
-                ("softmax_scale", ctypes.c_float),
+                ("softmax_scale", ctypes.c_float), ("rope_base", ctypes.c_float),
                 ("saved_hops", ctypes.c_void_p),
                 ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
                 ("stream", ctypes.c_void_p)]
@@ -196,7 +196,7 @@ def ta_backward(dout, q, k, v, out, dq, dk, dv, B, H, H_kv, N, D, dims, causal, 
 
 def ta_backward_ex(dout, q, k, v, dq, dk, dv, B, H, H_kv, N, D, dims, causal,
                    grad_dtype=TA_DTYPE_BF16, softmax_scale=0.0, saved_hops=None, workspace=None,
-                   workspace_bytes=0, stream=None, check=True) -> int:
+                   workspace_bytes=0, rope_base=0.0, stream=None, check=True) -> int:
     d, nd = _dims(dims)
     p = ta_bwd_params()
     p.struct_bytes = ctypes.sizeof(ta_bwd_params)
@@ -205,6 +205,7 @@ def ta_backward_ex(dout, q, k, v, dq, dk, dv, B, H, H_kv, N, D, dims, causal,
     p.B, p.H, p.H_kv, p.N, p.D = B, H, H_kv, N, D
     p.dims, p.ndims, p.causal = d, nd, int(bool(causal))
     p.dtype, p.grad_dtype, p.softmax_scale = TA_DTYPE_BF16, grad_dtype, softmax_scale
+    p.rope_base = rope_base
     p.saved_hops = _ptr(saved_hops)
     p.workspace, p.workspace_bytes = _ptr(workspace), workspace_bytes
     p.stream = _stream(stream)

@@ -47,6 +47,8 @@ int backward_impl(const ta_bwd_params &p) {
     if (!p.dout || !p.q || !p.k || !p.v || !p.dq || !p.dk || !p.dv) return TA_ERR_INVALID_ARG;
     if (p.dtype != TA_DTYPE_BF16) return TA_ERR_UNSUPPORTED;
     if (p.grad_dtype != TA_DTYPE_BF16 && p.grad_dtype != TA_DTYPE_F32) return TA_ERR_UNSUPPORTED;
+    if (p.rope_base < 0.f || !(p.rope_base == p.rope_base)) return TA_ERR_INVALID_ARG;
+    if (p.rope_base > 0.f && (p.D & 1)) return TA_ERR_UNSUPPORTED;
     Plan plan;
     // hop by hop: the backward needs every hop's input
     int rc = build_plan(p.B, p.H, p.H_kv, p.N, p.D, p.dims, p.ndims, p.dtype, TA_FLAG_NO_HOP_FUSION, 0, 0, &plan);
@@ -75,7 +77,7 @@ int backward_impl(const ta_bwd_params &p) {
     for (int i = 0; i < p.ndims; ++i) pb.dims[i] = p.dims[i];
     pb.ndims = p.ndims; pb.causal = p.causal ? 1 : 0; pb.dtype = p.dtype;
     pb.scale = p.softmax_scale != 0.f ? p.softmax_scale : 1.0f / sqrtf((float)p.D);
-    pb.rope_base = 0.f;
+    pb.rope_base = p.rope_base;
     pb.flags = 0; pb.hop_begin = 0; pb.hop_end = p.ndims;
     pb.stream = (cudaStream_t)p.stream;
 

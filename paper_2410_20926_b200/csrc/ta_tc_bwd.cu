@@ -21,9 +21,14 @@
 // Persistent, one CTA per SM.  Warps 0-3 compute (thread 0 issues the MMAs and the stores);
 // warp 4 issues the TMA loads: Q and G of the next head land in a second stage while the
 // current head computes, X and K as soon as the MMAs that read their slots have completed, so
-// that loads overlap the epilogue.  Every wait is bounded; when one expires the CTA raises a
+// that loads overlap the epilogue.  With the tensorized positional encoding (Section 3.2, per-hop
+// RoPE; template parameter kRope) warps 5-12 rotate the K and Q tiles in place in shared memory
+// before thread 0 sees them, exactly as in the forward kernel, and the epilogue turns dQ and dK --
+// gradients with respect to the rotated vectors -- back by the transposed rotation before they
+// leave the SM.  Every wait is bounded; when one expires the CTA raises a
 // flag that ends both roles, lets its copies land, frees its TMEM and returns.
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 
 #include "ta_internal.h"
 #include "ta_ptx.cuh"
@@ -33,12 +38,14 @@ namespace {
 
 constexpr int kTileRows = 128;
 constexpr int kThreads = 160;          // + the producer warp
+constexpr int kThreadsRope = 416;      // + two warpgroups that rotate Q and K tiles
 
 struct BwdArgs {
     int n, rows, ci, co, causal, g, H, H_kv, x_is_kv, first_hop;
     int accumulate;                    // 0: dQ / dK are stored (first hop processed), 1: reduce-added
     long long tiles_inner, tiles_outer, total_items;
     float scale_log2, scale;
+    float rope_log2_base;              // log2 of the RoPE base (rotating variant only)
 };
 
 template <int D>
@@ -53,8 +60,9 @@ struct BwdCfg {
     static constexpr uint32_t kOffXP = kOffStage + 2 * kStageBytes;  // X, then P
     static constexpr uint32_t kOffDS = kOffXP + kPBytes;             // dS, then the bf16 G_i staging
     static constexpr uint32_t kOffBar = kOffDS + kPBytes;
-    static constexpr int kNumBars = 10;
-    static constexpr uint32_t kSmemBytes = kOffBar + kNumBars * 8 + 16 + 1024;
+    static constexpr int kNumBars = 13;
+    static constexpr uint32_t kOffTheta = kOffBar + kNumBars * 8 + 16;   // D/2 RoPE frequencies (fp32)
+    static constexpr uint32_t kSmemBytes = kOffTheta + 64 * 4 + 1024;
     static constexpr uint32_t kTmemCols = 512;
     // S then G_i | dP then dQ | dK summed over the group | dV summed over the group (first hop)
     static constexpr uint32_t kColS = 0, kColDP = 128, kColDK = 256, kColDV = 384;
@@ -89,8 +97,8 @@ __device__ __forceinline__ bool wg_all(bool pred) {
 }
 __device__ __forceinline__ void wg_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
-template <int D>
-__global__ void __launch_bounds__(kThreads, 1)
+template <int D, bool kRope>
+__global__ void __launch_bounds__(kRope ? kThreadsRope : kThreads, 1)
 hop_tc_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                   const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_gin,
                   const __grid_constant__ CUtensorMap map_gout, const __grid_constant__ CUtensorMap map_dq,
@@ -111,14 +119,18 @@ hop_tc_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                    o_done = bar0 + 72;
     auto qg_full = [&](int s) { return bar0 + 16u + 8u * (uint32_t)s; };
     auto qg_free = [&](int s) { return bar0 + 32u + 8u * (uint32_t)s; };
+    const uint32_t k_rot = bar0 + 80;                                // rotated K ready (8 warps)
+    auto q_rot = [&](int s) { return bar0 + 88u + 8u * (uint32_t)s; };   // rotated Q of stage s ready
+    float *theta_tab = (float *)(smem + C::kOffTheta);
     uint32_t *tmem_slot = (uint32_t *)(smem + C::kOffBar + C::kNumBars * 8);
     volatile uint32_t *abort_flag = tmem_slot + 1;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
-    for (uint32_t i = tid; i < C::kOffBar / 16; i += kThreads) ((uint4 *)smem)[i] = make_uint4(0, 0, 0, 0);
+    for (uint32_t i = tid; i < C::kOffBar / 16; i += blockDim.x) ((uint4 *)smem)[i] = make_uint4(0, 0, 0, 0);
+    if (kRope && tid < D / 2) theta_tab[tid] = exp2f(-2.f * (float)tid / (float)D * a.rope_log2_base);
     if (tid == 0) {
-        for (int i = 0; i < C::kNumBars; ++i) mbar_init(bar0 + 8u * (uint32_t)i, 1);
+        for (int i = 0; i < C::kNumBars; ++i) mbar_init(bar0 + 8u * (uint32_t)i, i >= 10 ? 8 : 1);
         *abort_flag = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -192,7 +204,78 @@ hop_tc_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 }
             }
         }
-    } else {
+    } else if (kRope && warp >= 5) {
+        // =============================================================== RoPE on the K and Q tiles
+        // (same scheme as the forward kernel: a thread owns one 16-byte chunk of features and
+        // their partners c + D/2 at fixed positions of every segment; cos / sin in registers)
+        constexpr int kChunks = D / 16;
+        const int rt = tid - 5 * 32;                      // 0 .. 255
+        const int chunk = rt % kChunks;
+        const int tsub = rt / kChunks;
+        constexpr int kTStep = 256 / kChunks;
+        constexpr int kMaxPos = 128 / kTStep;
+        const int segs = a.rows / a.n;
+        __half2 cs[kMaxPos][8];
+#pragma unroll
+        for (int pi = 0; pi < kMaxPos; ++pi)
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const float ang = (float)(tsub + kTStep * pi) *
+                                  exp2f(-2.f * (float)(8 * chunk + e) / (float)D * a.rope_log2_base);
+                cs[pi][e] = __floats2half2_rn(__cosf(ang), __sinf(ang));
+            }
+        auto rotate_tile = [&](uint32_t tile) {
+#pragma unroll
+            for (int pi = 0; pi < kMaxPos; ++pi) {
+                const int t = tsub + kTStep * pi;
+                if (t >= a.n) break;
+#pragma unroll 2
+                for (int sg = 0; sg < segs; ++sg) {
+                    const int r = sg * a.n + t;
+                    const uint32_t row = tile + (uint32_t)r * 128u;
+                    const uint32_t addr_a = row + (((uint32_t)chunk ^ (uint32_t)(r & 7)) << 4);
+                    const uint32_t addr_b = D == 128 ? addr_a + kSlabBytes
+                                                     : row + (((uint32_t)(chunk + 4) ^ (uint32_t)(r & 7)) << 4);
+                    uint32_t ua[4], ub[4];
+                    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                                 : "=r"(ua[0]), "=r"(ua[1]), "=r"(ua[2]), "=r"(ua[3]) : "r"(addr_a) : "memory");
+                    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                                 : "=r"(ub[0]), "=r"(ub[1]), "=r"(ub[2]), "=r"(ub[3]) : "r"(addr_b) : "memory");
+#pragma unroll
+                    for (int e2 = 0; e2 < 4; ++e2) {
+                        const float a0 = __uint_as_float(ua[e2] << 16), a1 = __uint_as_float(ua[e2] & 0xFFFF0000u);
+                        const float b0 = __uint_as_float(ub[e2] << 16), b1 = __uint_as_float(ub[e2] & 0xFFFF0000u);
+                        const float2 f0 = __half22float2(cs[pi][2 * e2]), f1 = __half22float2(cs[pi][2 * e2 + 1]);
+                        ua[e2] = pack_bf16x2(a0 * f0.x - b0 * f0.y, a1 * f1.x - b1 * f1.y);
+                        ub[e2] = pack_bf16x2(b0 * f0.x + a0 * f0.y, b1 * f1.x + a1 * f1.y);
+                    }
+                    st_shared_v4(addr_a, ua[0], ua[1], ua[2], ua[3]);
+                    st_shared_v4(addr_b, ub[0], ub[1], ub[2], ub[3]);
+                }
+            }
+            fence_proxy_async_smem();
+            __syncwarp();
+        };
+        bool ok = true;
+        uint32_t t = 0, it = 0;
+        for (long long item = blockIdx.x; ok && item < a.total_items; item += gridDim.x, ++it) {
+            for (int j = 0; j < a.g; ++j, ++t) {
+                const int s = t & 1;
+                ok = mbar_wait_abortable(qg_full(s), (t >> 1) & 1, 0x68, abort_flag);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                rotate_tile(sQ(s));
+                if (lane == 0) mbar_arrive(q_rot(s));
+                if (j == 0) {
+                    ok = mbar_wait_abortable(k_full, it & 1, 0x69, abort_flag);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    rotate_tile(sK);
+                    if (lane == 0) mbar_arrive(k_rot);
+                }
+            }
+        }
+    } else if (warp < 4) {
         // =============================================================== compute warps
         const uint32_t tmem_lane = tmem_base + ((uint32_t)(warp * 32) << 16);
         constexpr uint32_t idesc_s = instr_desc(128, 0, 0);        // A, B K-major, N = 128
@@ -225,6 +308,37 @@ hop_tc_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             }
         };
 
+        // the same for a gradient with respect to ROTATED vectors (dQ, dK under the positional
+        // encoding): row r sits at position r mod n, feature c is paired with c + D/2, and the
+        // gradient of the un-rotated vector is the transposed rotation of the rotated one's
+        const float pos = (float)(r % a.n);
+        auto stage_f32_unrotated = [&](uint32_t col0, uint32_t stage) {
+            if (!warp_valid) return;
+            constexpr int kHalfChunks = D / 64;          // 32-column chunks in half a row
+            uint32_t va[32], vb[32];
+#pragma unroll 1
+            for (int c = 0; c < kHalfChunks; ++c) {
+                tmem_ld32(tmem_lane + col0 + 32 * c, va);
+                tmem_ld32(tmem_lane + col0 + 32 * (c + kHalfChunks), vb);
+                if (!row_valid) continue;
+#pragma unroll
+                for (int jj = 0; jj < 32; ++jj) {
+                    const float ang = pos * theta_tab[32 * c + jj];
+                    const float cs = __cosf(ang), sn = __sinf(ang);
+                    const float x1 = __uint_as_float(va[jj]), x2 = __uint_as_float(vb[jj]);
+                    va[jj] = __float_as_uint(x1 * cs + x2 * sn);
+                    vb[jj] = __float_as_uint(x2 * cs - x1 * sn);
+                }
+                const uint32_t row_a = stage + (uint32_t)c * kSlabBytes + (uint32_t)r * 128u;
+                const uint32_t row_b = stage + (uint32_t)(c + kHalfChunks) * kSlabBytes + (uint32_t)r * 128u;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    st_shared_v4(row_a + (uint32_t)((i ^ (r & 7)) * 16), va[4 * i], va[4 * i + 1], va[4 * i + 2], va[4 * i + 3]);
+                    st_shared_v4(row_b + (uint32_t)((i ^ (r & 7)) * 16), vb[4 * i], vb[4 * i + 1], vb[4 * i + 2], vb[4 * i + 3]);
+                }
+            }
+        };
+
         uint32_t t = 0, it = 0;
         bool ok = true;
         for (long long item = blockIdx.x; ok && item < a.total_items; item += gridDim.x, ++it) {
@@ -239,8 +353,9 @@ hop_tc_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 // ---- S = Q K^T and dP = G X^T
                 if (tid == 0) {
                     bool k0 = true;
-                    if (j == 0) k0 = mbar_wait_abortable(k_full, it & 1, 0x71, abort_flag);
+                    if (j == 0) k0 = mbar_wait_abortable(kRope ? k_rot : k_full, it & 1, 0x71, abort_flag);
                     if (k0) k0 = mbar_wait_abortable(qg_full(s), (t >> 1) & 1, 0x72, abort_flag);
+                    if (kRope && k0) k0 = mbar_wait_abortable(q_rot(s), (t >> 1) & 1, 0x76, abort_flag);
                     if (k0) {
                         tc_fence_after();
 #pragma unroll
@@ -371,7 +486,8 @@ hop_tc_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 tc_fence_after();
 
                 // ---- epilogue: dQ (fp32, over this head's Q and G tiles) and G_i (bf16, over dS)
-                stage_f32(C::kColDP, q_base);
+                if (kRope) stage_f32_unrotated(C::kColDP, q_base);
+                else stage_f32(C::kColDP, q_base);
                 if (!a.first_hop && warp_valid) {
                     uint32_t v[32];
 #pragma unroll 1
@@ -411,7 +527,8 @@ hop_tc_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     // ---- once per item: dK (and, in the first hop, dV) of the whole group
                     wg_sync();                         // the staging space has been read out
                     tc_fence_after();
-                    stage_f32(C::kColDK, q_base);
+                    if (kRope) stage_f32_unrotated(C::kColDK, q_base);
+                    else stage_f32(C::kColDK, q_base);
                     fence_proxy_async_smem();
                     tc_fence_before();
                     wg_sync();
@@ -509,6 +626,7 @@ int launch_bwd_d(const Problem &pb, const HopDesc &hd, const void *x, int x_head
     a.total_items = (long long)pb.B * pb.H_kv * hd.tiles_inner * hd.tiles_outer;
     a.scale = pb.scale;
     a.scale_log2 = pb.scale * 1.4426950408889634f;
+    a.rope_log2_base = pb.rope_base > 0.f ? log2f(pb.rope_base) : 0.f;
 
     static int num_sms = 0;
     if (num_sms == 0) {
@@ -518,15 +636,20 @@ int launch_bwd_d(const Problem &pb, const HopDesc &hd, const void *x, int x_head
             num_sms = 148;
     }
     constexpr size_t smem = BwdCfg<D>::kSmemBytes;
-    auto kern = hop_tc_bwd_kernel<D>;
     static bool configured = false;
     if (!configured) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        if (cudaFuncSetAttribute(hop_tc_bwd_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+                cudaSuccess ||
+            cudaFuncSetAttribute(hop_tc_bwd_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+                cudaSuccess)
             return TA_ERR_CUDA;
         configured = true;
     }
     const unsigned grid = (unsigned)(a.total_items < num_sms ? a.total_items : num_sms);
-    kern<<<grid, kThreads, smem, pb.stream>>>(mq, mk, mx, mgi, mgo, mdq, mdk, mdv, a);
+    if (pb.rope_base > 0.f)
+        hop_tc_bwd_kernel<D, true><<<grid, kThreadsRope, smem, pb.stream>>>(mq, mk, mx, mgi, mgo, mdq, mdk, mdv, a);
+    else
+        hop_tc_bwd_kernel<D, false><<<grid, kThreads, smem, pb.stream>>>(mq, mk, mx, mgi, mgo, mdq, mdk, mdv, a);
     count_launch();
     return cudaPeekAtLastError() == cudaSuccess ? TA_OK : TA_ERR_CUDA;
 }

@@ -25,7 +25,7 @@ pytestmark = pytest.mark.gpu
 RTOL = 2.0 ** -8
 
 
-def gpu_backward(inp, B, H, Hkv, N, D, dims, causal, grad_f32, saved=None):
+def gpu_backward(inp, B, H, Hkv, N, D, dims, causal, grad_f32, saved=None, rope_base=0.0):
     import torch
     q, k, v, do = (to_device(inp, n, "bf16") for n in ("q", "k", "v", "dout"))
     tdt = torch.float32 if grad_f32 else torch.bfloat16
@@ -35,10 +35,10 @@ def gpu_backward(inp, B, H, Hkv, N, D, dims, causal, grad_f32, saved=None):
     mode = ta.TA_WS_BACKWARD_F32_GRADS if grad_f32 else ta.TA_WS_BACKWARD
     nbytes = ta.ta_workspace_bytes(B, H, Hkv, N, D, dims, ta.TA_DTYPE_BF16, mode)
     ws = torch.empty(max(nbytes, 256), dtype=torch.uint8, device="cuda")
-    if grad_f32 or saved is not None:
+    if grad_f32 or saved is not None or rope_base:
         ta.ta_backward_ex(do, q, k, v, dq, dk, dv, B, H, Hkv, N, D, dims, causal,
                           grad_dtype=ta.TA_DTYPE_F32 if grad_f32 else ta.TA_DTYPE_BF16,
-                          saved_hops=saved, workspace=ws, workspace_bytes=nbytes)
+                          saved_hops=saved, workspace=ws, workspace_bytes=nbytes, rope_base=rope_base)
     else:
         ta.ta_backward(do, q, k, v, None, dq, dk, dv, B, H, Hkv, N, D, dims, causal, workspace=ws,
                        workspace_bytes=nbytes)
@@ -74,6 +74,27 @@ def test_backward_small(dims, D, causal, B, H, Hkv, grad_f32):
     inp = ta_inputs.make_inputs(B, H, Hkv, N, D, "bf16", 301, with_dout=True)
     got = gpu_backward(inp, B, H, Hkv, N, D, dims, causal, grad_f32)
     ref = oracle.backward(inp["dout"], inp["q"], inp["k"], inp["v"], dims, causal)
+    for name, g, r in zip(("dq", "dk", "dv"), got, ref):
+        assert_grad_close(g, r, name)
+
+
+@pytest.mark.parametrize("dims,D,causal,B,H,Hkv", [
+    ([128], 128, True, 1, 2, 1),
+    ([8, 16, 32], 128, True, 1, 4, 2),
+    ([16, 16], 64, False, 2, 4, 4),
+    ([5, 24, 7], 128, True, 1, 4, 2),
+    ([2, 4, 12], 64, False, 1, 4, 1),
+    ([4, 64], 128, True, 1, 8, 2),
+])
+@pytest.mark.parametrize("grad_f32", [False, True])
+def test_backward_with_positional_encoding(dims, D, causal, B, H, Hkv, grad_f32):
+    """dq, dk with respect to the UN-rotated q, k when every hop rotates them by its coordinate."""
+    N = math.prod(dims)
+    inp = ta_inputs.make_inputs(B, H, Hkv, N, D, "bf16", 304, with_dout=True)
+    got = gpu_backward(inp, B, H, Hkv, N, D, dims, causal, grad_f32, rope_base=10000.0)
+    ref = oracle.backward(inp["dout"], inp["q"], inp["k"], inp["v"], dims, causal, rope_base=10000.0)
+    plain = oracle.backward(inp["dout"], inp["q"], inp["k"], inp["v"], dims, causal)
+    assert np.abs(ref[0] - plain[0]).max() > 0.05          # the encoding changes the gradients visibly
     for name, g, r in zip(("dq", "dk", "dv"), got, ref):
         assert_grad_close(g, r, name)
 
