@@ -38,8 +38,8 @@ UNIT = "tokens/s"
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per token per launch of the hop kernel, from
 # the ncu capture of config 3 summarised in profiles/hop_pipe_kernel_config3_ncu_full.md
-# (mean of the three hops, 758.9 MB for 32768 tokens); traffic is proportional to the tokens.
-NCU_TRAFFIC_BYTES_PER_TOKEN_PER_LAUNCH = 758.9e6 / 32768
+# (mean of the three hops, 758.8 MB for 32768 tokens); traffic is proportional to the tokens.
+NCU_TRAFFIC_BYTES_PER_TOKEN_PER_LAUNCH = 758.8e6 / 32768
 
 
 # ------------------------------------------------------------------ roofline arithmetic
@@ -140,8 +140,8 @@ def oracle_sample(cfg, inp, min_seconds: float = 0.0):
     t_head = dt / reps
     value = cfg.B * cfg.N / (t_head * cfg.B * cfg.H)
     return {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
-            "sample": f"{reps} of {cfg.B * cfg.H} heads of the workload (all {cfg.N} tokens, "
-                      f"all hops), {dt:.1f} s, scaled to the batch"}, t_head
+            "sample": f"{reps} single-head passes over the workload's heads (all {cfg.N} tokens, all hops; "
+                      f"the batch has {cfg.B * cfg.H} heads), {dt:.1f} s, scaled to the batch"}, t_head
 
 
 # ------------------------------------------------------------------ distributed plumbing
@@ -306,7 +306,7 @@ def run_ours(args, cfg):
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": NCU_TRAFFIC_BYTES_PER_TOKEN_PER_LAUNCH * cfg.B * cfg.N,
                 "traffic_source": "ncu capture of config 3 scaled by tokens (profiles/)", "peak_source": peak_src,
-                "kernel": "hop_pipe_kernel<128>", "algorithmic_bytes_per_launch": bytes_per_launch,
+                "kernel": "hop_pipe_kernel<128, false>", "algorithmic_bytes_per_launch": bytes_per_launch,
                 "launches_per_step": n_launch, "avg_launch_ms": launch_ms,
                 "useful_tflops": step_flops(cfg) / (ms / args.steps * 1e-3) / 1e12}
     cpu, _ = oracle_sample(cfg, inp, min_seconds=args.cpu_seconds)
