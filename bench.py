@@ -1,5 +1,5 @@
 #!/usr/bin/env python
-"""Benchmark of the tensorized-attention forward on B200 (metric of the benchmark spec).
+"""Benchmark of the tensorized-attention forward on B200 (tokens per second at 128k tokens).
 
 One step = one whole forward pass (every hop of Algorithm 1) over one batch of synthetic
 Llama-8B-shaped q, k, v: causal, B=1, H=32, H_kv=8, D=128, N=131072 viewed as 32x64x64, bf16.

@@ -341,6 +341,7 @@ hop_tc_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
 
         uint32_t t = 0, it = 0;
         bool ok = true;
+        int pending_stage = -1;   // thread 0: stage whose output stores have been issued but not yet read out
         for (long long item = blockIdx.x; ok && item < a.total_items; item += gridDim.x, ++it) {
             const BwdItem c = decode_bwd_item(a, item);
             for (int j = 0; j < a.g; ++j, ++t) {
@@ -375,6 +376,13 @@ hop_tc_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                                       smem_desc_sw128(sXP + off, 16, 1024), idesc_s, kb > 0);
                         }
                         tc_commit(s_done);
+                    }
+                    if (pending_stage >= 0) {
+                        // the previous head's stores overlap this head's score MMAs; their staging
+                        // space (that stage and the dS slot) is needed again only from here on
+                        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                        mbar_arrive(qg_free(pending_stage));
+                        pending_stage = -1;
                     }
                     ok = k0;
                 }
@@ -521,7 +529,8 @@ hop_tc_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                         for (int h = 0; h < kHalves; ++h)
                             tma_store_5d(&map_gout, sdS + h * kSlabBytes, 64 * h, 0, c.c_inner, c.c_outer, q_head);
                     }
-                    tma_store_commit_and_wait_read();
+                    if (last_head) tma_store_commit_and_wait_read();   // the staging space is reused right below
+                    else asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                 }
                 if (last_head) {
                     // ---- once per item: dK (and, in the first hop, dV) of the whole group
@@ -557,7 +566,10 @@ hop_tc_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                         }
                     }
                 }
-                if (tid == 0) mbar_arrive(qg_free(s));   // this stage may take the head after next
+                if (tid == 0) {
+                    if (last_head) mbar_arrive(qg_free(s));   // read out: this stage may take the head after next
+                    else pending_stage = s;                   // handed back once the stores have been read
+                }
             }
         }
         if (tid == 0) tma_store_wait_all();
