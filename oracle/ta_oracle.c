@@ -36,6 +36,12 @@
  *     x'_{c+D/2} = x_{c+D/2} cos a + x_c sin a ,       c = 0 .. D/2-1,
  * so that a hop's scores depend on the relative position t - u along that dimension.
  * The value tensor is never rotated.
+ *
+ * Per-hop sparsity masks (the paper notes that M_i may be any sparsity mask, Section 3.1 /
+ * Eq. 3): besides the causal mask, hop i may carry a sliding window w_i > 0 along its
+ * dimension -- key position u is visible from query position t iff |t - u| < w_i (and u <= t
+ * when causal).  w_i = 0 means no window.  Every row keeps its own position, so no row is
+ * fully masked.
  */
 #include <math.h>
 #include <stdlib.h>
@@ -46,13 +52,20 @@
 
 /* Attention weights of one segment: P[t*n+u], rows sum to 1 (Eq. 1 / Eq. 4). */
 static void segment_weights(const double *Q, const double *K, long base, long stride,
-                            int n, int D, double scale, int causal, double *P)
+                            int n, int D, double scale, int causal, int window, double *P)
 {
     for (int t = 0; t < n; ++t) {
         const double *qt = Q + (base + (long)t * stride) * D;
-        int nu = causal ? t + 1 : n;          /* visible keys of row t */
+        /* visible keys of row t: [u0, nu) */
+        int nu = causal ? t + 1 : n;
+        int u0 = 0;
+        if (window > 0) {
+            if (t - window + 1 > u0) u0 = t - window + 1;
+            if (!causal && t + window < nu) nu = t + window;
+        }
         double mx = -INFINITY;
-        for (int u = 0; u < nu; ++u) {
+        for (int u = 0; u < u0; ++u) P[t * n + u] = 0.0;   /* outside the window: weight exactly 0 */
+        for (int u = u0; u < nu; ++u) {
             const double *ku = K + (base + (long)u * stride) * D;
             double s = 0.0;
             for (int c = 0; c < D; ++c) s += qt[c] * ku[c];
@@ -61,12 +74,12 @@ static void segment_weights(const double *Q, const double *K, long base, long st
             if (s > mx) mx = s;
         }
         double den = 0.0;
-        for (int u = 0; u < nu; ++u) {
+        for (int u = u0; u < nu; ++u) {
             double e = exp(P[t * n + u] - mx);
             P[t * n + u] = e;
             den += e;
         }
-        for (int u = 0; u < nu; ++u) P[t * n + u] /= den;
+        for (int u = u0; u < nu; ++u) P[t * n + u] /= den;
         for (int u = nu; u < n; ++u) P[t * n + u] = 0.0;   /* masked: weight exactly 0 */
     }
 }
@@ -108,7 +121,7 @@ static void rope_rotate(const double *x, double *y, long N, int D, long stride, 
  */
 static int forward_head_impl(const double *q, const double *k, const double *v, double *out,
                              long N, int D, const int *dims, int ndims, int causal,
-                             double scale, double rope_base, double *xs)
+                             double scale, double rope_base, const int *window, double *xs)
 {
     if (!q || !k || !v || !out || !dims || ndims < 1 || N < 1 || D < 1) return -1;
     long prod = 1;
@@ -149,7 +162,7 @@ static int forward_head_impl(const double *q, const double *k, const double *v, 
                 if (!P) continue;
                 long outer = g / s, inner = g % s;
                 long base = outer * n * s + inner;
-                segment_weights(q, k, base, s, n, D, scale, causal, P);   /* A_i */
+                segment_weights(q, k, base, s, n, D, scale, causal, window ? window[i] : 0, P);   /* A_i */
                 for (int t = 0; t < n; ++t) {               /* O_i = A_i O_i, folded back */
                     double *o = nxt + (base + (long)t * s) * D;
                     for (int c = 0; c < D; ++c) o[c] = 0.0;
@@ -176,7 +189,7 @@ int ta_oracle_forward_head(const double *q, const double *k, const double *v, do
                            long N, int D, const int *dims, int ndims, int causal,
                            double scale, double *xs)
 {
-    return forward_head_impl(q, k, v, out, N, D, dims, ndims, causal, scale, 0.0, xs);
+    return forward_head_impl(q, k, v, out, N, D, dims, ndims, causal, scale, 0.0, NULL, xs);
 }
 
 /* As above with the tensorized positional encoding (rope_base > 0, e.g. 10000). */
@@ -185,7 +198,17 @@ int ta_oracle_forward_head_rope(const double *q, const double *k, const double *
                                 double scale, double rope_base, double *xs)
 {
     if (!(rope_base > 0.0)) return -1;
-    return forward_head_impl(q, k, v, out, N, D, dims, ndims, causal, scale, rope_base, xs);
+    return forward_head_impl(q, k, v, out, N, D, dims, ndims, causal, scale, rope_base, NULL, xs);
+}
+
+/* Every option: rope_base 0 = none; window NULL or [ndims] ints, 0 = no window in that hop. */
+int ta_oracle_forward_head_ex(const double *q, const double *k, const double *v, double *out,
+                              long N, int D, const int *dims, int ndims, int causal,
+                              double scale, double rope_base, const int *window, double *xs)
+{
+    if (rope_base < 0.0) return -1;
+    if (window) for (int i = 0; i < ndims; ++i) if (window[i] < 0) return -1;
+    return forward_head_impl(q, k, v, out, N, D, dims, ndims, causal, scale, rope_base, window, xs);
 }
 
 /*
@@ -205,7 +228,7 @@ int ta_oracle_forward_head_rope(const double *q, const double *k, const double *
 static int backward_head_impl(const double *q, const double *k, const double *xs,
                               const double *dout, double *dq, double *dk, double *dv,
                               long N, int D, const int *dims, int ndims, int causal,
-                              double scale, double rope_base)
+                              double scale, double rope_base, const int *window)
 {
     if (!q || !k || !xs || !dout || !dq || !dk || !dv || !dims || ndims < 1) return -1;
     long prod = 1;
@@ -257,7 +280,7 @@ static int backward_head_impl(const double *q, const double *k, const double *xs
                 if (!P || !dS) continue;
                 long outer = sg / s, inner = sg % s;
                 long base = outer * n * s + inner;
-                segment_weights(q, k, base, s, n, D, scale, causal, P);
+                segment_weights(q, k, base, s, n, D, scale, causal, window ? window[i] : 0, P);
                 /* dP[t][u] = <G_{i+1}[t], X_i[u]>, then dS */
                 for (int t = 0; t < n; ++t) {
                     const double *gt = g + (base + (long)t * s) * D;
@@ -315,7 +338,7 @@ int ta_oracle_backward_head(const double *q, const double *k, const double *xs,
                             long N, int D, const int *dims, int ndims, int causal,
                             double scale)
 {
-    return backward_head_impl(q, k, xs, dout, dq, dk, dv, N, D, dims, ndims, causal, scale, 0.0);
+    return backward_head_impl(q, k, xs, dout, dq, dk, dv, N, D, dims, ndims, causal, scale, 0.0, NULL);
 }
 
 int ta_oracle_backward_head_rope(const double *q, const double *k, const double *xs,
@@ -325,7 +348,17 @@ int ta_oracle_backward_head_rope(const double *q, const double *k, const double 
 {
     if (!(rope_base > 0.0)) return -1;
     return backward_head_impl(q, k, xs, dout, dq, dk, dv, N, D, dims, ndims, causal, scale,
-                              rope_base);
+                              rope_base, NULL);
+}
+
+int ta_oracle_backward_head_ex(const double *q, const double *k, const double *xs,
+                               const double *dout, double *dq, double *dk, double *dv,
+                               long N, int D, const int *dims, int ndims, int causal,
+                               double scale, double rope_base, const int *window)
+{
+    if (rope_base < 0.0) return -1;
+    return backward_head_impl(q, k, xs, dout, dq, dk, dv, N, D, dims, ndims, causal, scale,
+                              rope_base, window);
 }
 
 int ta_oracle_num_threads(void)

@@ -63,6 +63,14 @@ def _lib():
         lib.ta_oracle_backward_head_rope.argtypes = [dp, dp, dp, dp, dp, dp, dp, ctypes.c_long,
                                                      ctypes.c_int, ip, ctypes.c_int, ctypes.c_int,
                                                      ctypes.c_double, ctypes.c_double]
+        lib.ta_oracle_forward_head_ex.restype = ctypes.c_int
+        lib.ta_oracle_forward_head_ex.argtypes = [dp, dp, dp, dp, ctypes.c_long, ctypes.c_int, ip,
+                                                  ctypes.c_int, ctypes.c_int, ctypes.c_double,
+                                                  ctypes.c_double, ip, dp]
+        lib.ta_oracle_backward_head_ex.restype = ctypes.c_int
+        lib.ta_oracle_backward_head_ex.argtypes = [dp, dp, dp, dp, dp, dp, dp, ctypes.c_long,
+                                                   ctypes.c_int, ip, ctypes.c_int, ctypes.c_int,
+                                                   ctypes.c_double, ctypes.c_double, ip]
         lib.ta_oracle_num_threads.restype = ctypes.c_int
         _LIB = lib
     return _LIB
@@ -97,7 +105,20 @@ def _check(q, k, v, dims):
     return B, H, Hkv, N, D, dims
 
 
-def _fwd_head(lib, qh, kh, vh, out, N, D, cdims, m, causal, scale, rope_base, xs):
+def _cwindow(window, m):
+    if window is None:
+        return None
+    w = [int(x) for x in window]
+    if len(w) != m or any(x < 0 for x in w):
+        raise ValueError("window: one non-negative int per dimension")
+    return (ctypes.c_int * m)(*w)
+
+
+def _fwd_head(lib, qh, kh, vh, out, N, D, cdims, m, causal, scale, rope_base, xs, cwin=None):
+    if cwin is not None:
+        return lib.ta_oracle_forward_head_ex(_dptr(qh), _dptr(kh), _dptr(vh), _dptr(out), N, D, cdims, m,
+                                             int(bool(causal)), scale, float(rope_base or 0.0), cwin,
+                                             _dptr(xs) if xs is not None else None)
     if rope_base:
         return lib.ta_oracle_forward_head_rope(_dptr(qh), _dptr(kh), _dptr(vh), _dptr(out), N, D,
                                                cdims, m, int(bool(causal)), scale,
@@ -107,7 +128,7 @@ def _fwd_head(lib, qh, kh, vh, out, N, D, cdims, m, causal, scale, rope_base, xs
 
 
 def forward(q, k, v, dims, causal: bool, scale: float | None = None, heads=None,
-            return_xs: bool = False, rope_base: float | None = None):
+            return_xs: bool = False, rope_base: float | None = None, window=None):
     """Algorithm 1 for every (or the listed) head, fp64.
 
     q: [B,H,N,D]; k, v: [B,H_kv,N,D] (any float dtype; converted head by head to fp64).
@@ -115,6 +136,8 @@ def forward(q, k, v, dims, causal: bool, scale: float | None = None, heads=None,
     heads: optional list of (b, h) pairs; then the result is [len(heads), N, D].
     rope_base: None / 0 for no positional encoding, else the RoPE base (Llama: 10000) of the
     tensorized positional encoding (hop i rotates q, k by the coordinate along dimension i).
+    window: None, or one int per dimension: w_i > 0 keeps, in hop i, only keys within w_i
+    positions of the query along dimension i (|t - u| < w_i); 0 = no window.
     Returns out [B,H,N,D] fp64 (and, with return_xs, the list of per-head [m+1,N,D]
     value tensors X_0=V ... X_m=out keyed like the output).
     """
@@ -122,6 +145,7 @@ def forward(q, k, v, dims, causal: bool, scale: float | None = None, heads=None,
     g = H // Hkv
     scale = 1.0 / math.sqrt(D) if scale is None else float(scale)
     cdims = (ctypes.c_int * len(dims))(*dims)
+    cwin = _cwindow(window, len(dims))
     pairs = [(b, h) for b in range(B) for h in range(H)] if heads is None else list(heads)
     out = np.empty((len(pairs), N, D), dtype=np.float64)
     xs_all = []
@@ -130,7 +154,7 @@ def forward(q, k, v, dims, causal: bool, scale: float | None = None, heads=None,
         qh, kh, vh = _f64(q[b, h]), _f64(k[b, h // g]), _f64(v[b, h // g])
         xs = np.empty((len(dims) + 1, N, D), dtype=np.float64) if return_xs else None
         rc = _fwd_head(lib, qh, kh, vh, out[idx], N, D, cdims, len(dims), causal, scale,
-                       rope_base, xs)
+                       rope_base, xs, cwin)
         if rc != 0:
             raise RuntimeError("ta_oracle_forward_head failed")
         if return_xs:
@@ -141,7 +165,7 @@ def forward(q, k, v, dims, causal: bool, scale: float | None = None, heads=None,
 
 
 def backward(dout, q, k, v, dims, causal: bool, scale: float | None = None, groups=None,
-             rope_base: float | None = None):
+             rope_base: float | None = None, window=None):
     """Gradients of sum(out * dout) w.r.t. q, k, v (fp64), GQA groups summed into dk, dv.
 
     groups: optional list of (b, kv_head) pairs; then only those KV heads and their query
@@ -151,6 +175,7 @@ def backward(dout, q, k, v, dims, causal: bool, scale: float | None = None, grou
     g = H // Hkv
     scale = 1.0 / math.sqrt(D) if scale is None else float(scale)
     cdims = (ctypes.c_int * len(dims))(*dims)
+    cwin = _cwindow(window, len(dims))
     sel = [(b, kv) for b in range(B) for kv in range(Hkv)] if groups is None else list(groups)
     dq = np.zeros((len(sel), g, N, D))
     dk = np.zeros((len(sel), N, D))
@@ -163,11 +188,16 @@ def backward(dout, q, k, v, dims, causal: bool, scale: float | None = None, grou
             qh = _f64(q[b, h])
             o = np.empty((N, D))
             xs = np.empty((len(dims) + 1, N, D))
-            rc = _fwd_head(lib, qh, kh, vh, o, N, D, cdims, len(dims), causal, scale, rope_base, xs)
+            rc = _fwd_head(lib, qh, kh, vh, o, N, D, cdims, len(dims), causal, scale, rope_base, xs, cwin)
             if rc != 0:
                 raise RuntimeError("ta_oracle_forward_head failed")
             dqh, dkh, dvh = np.empty((N, D)), np.empty((N, D)), np.empty((N, D))
-            if rope_base:
+            if cwin is not None:
+                rc = lib.ta_oracle_backward_head_ex(_dptr(qh), _dptr(kh), _dptr(xs),
+                                                    _dptr(_f64(dout[b, h])), _dptr(dqh), _dptr(dkh),
+                                                    _dptr(dvh), N, D, cdims, len(dims),
+                                                    int(bool(causal)), scale, float(rope_base or 0.0), cwin)
+            elif rope_base:
                 rc = lib.ta_oracle_backward_head_rope(_dptr(qh), _dptr(kh), _dptr(xs),
                                                       _dptr(_f64(dout[b, h])), _dptr(dqh),
                                                       _dptr(dkh), _dptr(dvh), N, D, cdims,
@@ -193,7 +223,7 @@ def backward(dout, q, k, v, dims, causal: bool, scale: float | None = None, grou
 # --------------------------------------------------------------------------------------
 
 def dense_hop_matrix(qh, kh, dims, i: int, causal: bool, scale: float | None = None,
-                     rope_base: float | None = None):
+                     rope_base: float | None = None, window=None):
     """The N x N matrix of hop i for one head (Eq. 3 written over flat token indices).
 
     Entry [j, k] is the softmax weight of key token k for query token j; it is non-zero only
@@ -209,8 +239,11 @@ def dense_hop_matrix(qh, kh, dims, i: int, causal: bool, scale: float | None = N
         cj, ck = coords[:, l][:, None], coords[:, l][None, :]
         if l != i:
             allowed &= cj == ck
-        elif causal:
-            allowed &= ck <= cj
+        else:
+            if causal:
+                allowed &= ck <= cj
+            if window is not None and window[i] > 0:
+                allowed &= np.abs(cj - ck) < window[i]
     if rope_base:
         # relative form of the rotary score: features c and c + D/2 form one complex number
         half = D // 2
@@ -233,23 +266,23 @@ def dense_hop_matrix(qh, kh, dims, i: int, causal: bool, scale: float | None = N
 
 
 def dense_effective_matrix(qh, kh, dims, causal: bool, scale: float | None = None,
-                           rope_base: float | None = None):
+                           rope_base: float | None = None, window=None):
     """A_eff = A^_{m-1} ... A^_1 A^_0, the N x N map from V to the output of one head."""
     N = np.asarray(qh).shape[0]
     a = np.eye(N)
     for i in range(len(dims)):
-        a = dense_hop_matrix(qh, kh, dims, i, causal, scale, rope_base) @ a
+        a = dense_hop_matrix(qh, kh, dims, i, causal, scale, rope_base, window) @ a
     return a
 
 
 def forward_dense(q, k, v, dims, causal: bool, scale: float | None = None,
-                  rope_base: float | None = None):
+                  rope_base: float | None = None, window=None):
     """Brute-force forward for all heads via dense_effective_matrix (tiny N only)."""
     B, H, Hkv, N, D, dims = _check(q, k, v, dims)
     g = H // Hkv
     out = np.empty((B, H, N, D))
     for b in range(B):
         for h in range(H):
-            a = dense_effective_matrix(q[b, h], k[b, h // g], dims, causal, scale, rope_base)
+            a = dense_effective_matrix(q[b, h], k[b, h // g], dims, causal, scale, rope_base, window)
             out[b, h] = a @ np.asarray(v[b, h // g], dtype=np.float64)
     return out

@@ -1,0 +1,103 @@
+"""Pins for the oracle's per-hop sliding-window masks (the paper allows any sparsity mask M_i in
+Eq. 3; here: in hop i a key is visible iff it lies within w_i positions of the query along
+dimension i, and not after it when causal).  Each check compares the C route with something
+that does not share its loops: the dense brute-force route (a boolean N x N mask built from
+coordinates), closed forms, and special cases that reduce to the unmasked operator."""
+import math
+
+import numpy as np
+import pytest
+
+import oracle
+
+
+def rnd(shape, seed):
+    return np.random.default_rng(seed).standard_normal(shape)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("dims,window", [([3, 4, 2], [2, 3, 1]), ([12], [5]), ([5, 4], [0, 2]), ([2, 9], [1, 4])])
+def test_windowed_route_matches_dense_mask_route(dims, window, causal):
+    N = math.prod(dims)
+    q, k, v = rnd((1, 4, N, 6), 31), rnd((1, 2, N, 6), 32), rnd((1, 2, N, 6), 33)
+    a = oracle.forward(q, k, v, dims, causal, window=window)
+    b = oracle.forward_dense(q, k, v, dims, causal, window=window)
+    np.testing.assert_allclose(a, b, rtol=0, atol=1e-13)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_wide_or_zero_window_is_no_window(causal):
+    dims = [3, 5, 4]
+    q, k, v = rnd((1, 2, 60, 4), 34), rnd((1, 2, 60, 4), 35), rnd((1, 2, 60, 4), 36)
+    plain = oracle.forward(q, k, v, dims, causal)
+    np.testing.assert_allclose(oracle.forward(q, k, v, dims, causal, window=[0, 0, 0]), plain, atol=0)
+    np.testing.assert_allclose(oracle.forward(q, k, v, dims, causal, window=[3, 5, 4]), plain, atol=1e-15)
+    assert np.abs(oracle.forward(q, k, v, dims, causal, window=[3, 2, 4]) - plain).max() > 1e-3
+
+
+def test_window_of_one_makes_the_hop_an_identity():
+    dims = [4, 6]
+    q, k, v = rnd((1, 2, 24, 4), 37), rnd((1, 2, 24, 4), 38), rnd((1, 2, 24, 4), 39)
+    for causal in (False, True):
+        a = oracle.forward(q, k, v, dims, causal, window=[1, 0])
+        # hop 0 sees only the query's own position: the value tensor passes through unchanged,
+        # and what is left is hop 1 alone = independent attentions over the rows of length 6
+        ref = np.concatenate([oracle.forward(q[:, :, r * 6:(r + 1) * 6], k[:, :, r * 6:(r + 1) * 6],
+                                             v[:, :, r * 6:(r + 1) * 6], [6], causal) for r in range(4)], axis=2)
+        np.testing.assert_allclose(a, ref, atol=1e-14)
+
+
+def test_zero_queries_average_the_window():
+    """q = 0: uniform weights over the visible keys -> a moving average (closed form)."""
+    n, w = 9, 3
+    v = rnd((1, 1, n, 2), 40)
+    k = rnd((1, 1, n, 2), 41)
+    q = np.zeros((1, 1, n, 2))
+    got = oracle.forward(q, k, v, [n], True, window=[w])[0, 0]
+    for t in range(n):
+        np.testing.assert_allclose(got[t], v[0, 0, max(0, t - w + 1):t + 1].mean(axis=0), atol=1e-14)
+    got = oracle.forward(q, k, v, [n], False, window=[w])[0, 0]
+    for t in range(n):
+        np.testing.assert_allclose(got[t], v[0, 0, max(0, t - w + 1):min(n, t + w)].mean(axis=0), atol=1e-14)
+
+
+def test_influence_set_is_the_window_box():
+    """Perturbing one token changes exactly the tokens within the windows along every dimension."""
+    dims, window = [3, 5], [2, 3]
+    q, k, v = rnd((1, 1, 15, 4), 42), rnd((1, 1, 15, 4), 43), rnd((1, 1, 15, 4), 44)
+    base = oracle.forward(q, k, v, dims, True, window=window)
+    src = (1, 1)
+    v2 = v.copy()
+    v2[0, 0, src[0] * 5 + src[1]] += 1.0
+    diff = np.abs(oracle.forward(q, k, v2, dims, True, window=window) - base).max(axis=-1)[0, 0].reshape(3, 5)
+    for j0 in range(3):
+        for j1 in range(5):
+            reach = 0 <= j0 - src[0] < window[0] and 0 <= j1 - src[1] < window[1]
+            assert (diff[j0, j1] > 1e-9) == reach, (j0, j1, diff[j0, j1])
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_backward_with_window_finite_differences(causal):
+    rng = np.random.default_rng(45)
+    dims, window, D, H, Hkv = [3, 2, 4], [2, 0, 3], 4, 2, 1
+    N = math.prod(dims)
+    q = rng.standard_normal((1, H, N, D))
+    k, v = rng.standard_normal((1, Hkv, N, D)), rng.standard_normal((1, Hkv, N, D))
+    dout = rng.standard_normal((1, H, N, D))
+    dq, dk, dv = oracle.backward(dout, q, k, v, dims, causal, window=window, rope_base=50.0)
+
+    def loss(q_, k_, v_):
+        return float((oracle.forward(q_, k_, v_, dims, causal, window=window, rope_base=50.0) * dout).sum())
+
+    eps = 1e-6
+    for name, arr, grad in (("q", q, dq), ("k", k, dk), ("v", v, dv)):
+        for _ in range(10):
+            idx = tuple(rng.integers(0, s) for s in arr.shape)
+            old = arr[idx]
+            arr[idx] = old + eps
+            lp = loss(q, k, v)
+            arr[idx] = old - eps
+            lm = loss(q, k, v)
+            arr[idx] = old
+            fd = (lp - lm) / (2 * eps)
+            assert abs(fd - grad[idx]) < 2e-7 * max(1.0, abs(fd)), (name, idx, fd, grad[idx])
