@@ -116,6 +116,7 @@ typedef struct ta_params {
                            /* instead of v.                                                  */
     float rope_base;       /* 0: none.  > 0 (Llama: 10000): tensorized positional encoding    */
                            /* (Section 3.2), applied inside the kernels -- see ta_forward_ex  */
+    const int *window;     /* host, ndims ints, or NULL: per-hop sliding window, see below     */
     ta_stream_t stream;
 } ta_params;
 
@@ -135,6 +136,12 @@ typedef struct ta_params {
  * exists in global memory.  D must be even (else TA_ERR_UNSUPPORTED); a negative or NaN base
  * is TA_ERR_INVALID_ARG.  The value tensor is never rotated.
  * ta_backward_ex takes the same rope_base (ta_backward, the short form, does not).
+ *
+ * Per-hop sparsity mask (Eq. 3 allows any mask M_i): window[i] = w > 0 keeps, in hop i, only
+ * the keys within w positions of the query along dimension i (|t - u| < w; with `causal` also
+ * u <= t, i.e. the last w positions up to the query's own); window[i] = 0 or window == NULL:
+ * no window.  A query always sees its own position, so no row is empty.  Negative entries
+ * are TA_ERR_INVALID_ARG.  ta_backward_ex takes the same array.
  */
 int ta_forward_ex(const ta_params *p);
 
@@ -178,6 +185,7 @@ typedef struct ta_bwd_params {
     float rope_base;              /* 0: none; > 0: tensorized positional encoding as in        */
                                   /* ta_forward_ex (q, k un-rotated; dq, dk are the gradients   */
                                   /* with respect to the un-rotated q, k).  D must be even.     */
+    const int *window;            /* host, ndims ints, or NULL: sliding windows as in ta_forward_ex */
     const void *saved_hops;       /* X_1..X_{m-1} as written by ta_forward_ex(TA_FLAG_SAVE_HOPS) */
                                   /* (the part of its workspace after the scratch tensor), or    */
                                   /* NULL: recomputed                                          */

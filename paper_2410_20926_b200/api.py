@@ -45,6 +45,7 @@ class ta_params(ctypes.Structure):
                 ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
                 ("flags", ctypes.c_uint), ("hop_begin", ctypes.c_int), ("hop_end", ctypes.c_int),
                 ("rope_base", ctypes.c_float),
+                ("window", ctypes.POINTER(ctypes.c_int)),
                 ("stream", ctypes.c_void_p)]
 
 
@@ -58,6 +59,7 @@ class ta_bwd_params(ctypes.Structure):
                 ("dims", ctypes.POINTER(ctypes.c_int)), ("ndims", ctypes.c_int),
                 ("causal", ctypes.c_int), ("dtype", ctypes.c_int), ("grad_dtype", ctypes.c_int),
                 ("softmax_scale", ctypes.c_float), ("rope_base", ctypes.c_float),
+                ("window", ctypes.POINTER(ctypes.c_int)),
                 ("saved_hops", ctypes.c_void_p),
                 ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
                 ("stream", ctypes.c_void_p)]
@@ -168,9 +170,19 @@ def ta_forward_f32(q, k, v, out, B, H, H_kv, N, D, dims, causal, stream=None, ch
                  check)
 
 
+def _window(window, nd):
+    """Per-dimension sliding windows as a C int array (None stays NULL)."""
+    if window is None:
+        return None
+    w = [int(x) for x in window]
+    if len(w) != nd:
+        raise ValueError("window needs one entry per dimension")
+    return (ctypes.c_int * nd)(*w)
+
+
 def ta_forward_ex(q, k, v, out, B, H, H_kv, N, D, dims, causal, dtype=TA_DTYPE_BF16,
                   softmax_scale=0.0, workspace=None, workspace_bytes=0, flags=0, hop_begin=0,
-                  hop_end=0, rope_base=0.0, stream=None, check=True) -> int:
+                  hop_end=0, rope_base=0.0, window=None, stream=None, check=True) -> int:
     d, nd = _dims(dims)
     p = ta_params()
     p.struct_bytes = ctypes.sizeof(ta_params)
@@ -181,6 +193,9 @@ def ta_forward_ex(q, k, v, out, B, H, H_kv, N, D, dims, causal, dtype=TA_DTYPE_B
     p.workspace, p.workspace_bytes = _ptr(workspace), workspace_bytes
     p.flags, p.hop_begin, p.hop_end = flags, hop_begin, hop_end
     p.rope_base = rope_base
+    win = _window(window, nd)          # kept alive until the call returns
+    if win is not None:
+        p.window = win
     p.stream = _stream(stream)
     return _done(load().ta_forward_ex(ctypes.byref(p)), "ta_forward_ex", check)
 
@@ -196,7 +211,7 @@ def ta_backward(dout, q, k, v, out, dq, dk, dv, B, H, H_kv, N, D, dims, causal, 
 
 def ta_backward_ex(dout, q, k, v, dq, dk, dv, B, H, H_kv, N, D, dims, causal,
                    grad_dtype=TA_DTYPE_BF16, softmax_scale=0.0, saved_hops=None, workspace=None,
-                   workspace_bytes=0, rope_base=0.0, stream=None, check=True) -> int:
+                   workspace_bytes=0, rope_base=0.0, window=None, stream=None, check=True) -> int:
     d, nd = _dims(dims)
     p = ta_bwd_params()
     p.struct_bytes = ctypes.sizeof(ta_bwd_params)
@@ -206,6 +221,9 @@ def ta_backward_ex(dout, q, k, v, dq, dk, dv, B, H, H_kv, N, D, dims, causal,
     p.dims, p.ndims, p.causal = d, nd, int(bool(causal))
     p.dtype, p.grad_dtype, p.softmax_scale = TA_DTYPE_BF16, grad_dtype, softmax_scale
     p.rope_base = rope_base
+    win = _window(window, nd)
+    if win is not None:
+        p.window = win
     p.saved_hops = _ptr(saved_hops)
     p.workspace, p.workspace_bytes = _ptr(workspace), workspace_bytes
     p.stream = _stream(stream)

@@ -91,6 +91,7 @@ int build_plan(int B, int H, int H_kv, int N, int D, const int *dims, int ndims,
             for (int j = 0; j < nf; ++j) {
                 f.sub_n[j] = plan->hops[first + j].n;
                 f.sub_stride[j] = (int)plan->hops[first + j].stride;
+                f.sub_hop[j] = plan->hops[first + j].hop;
             }
             f.n = (int)block;
             f.stride = 1;
@@ -199,6 +200,9 @@ static int forward_impl(const ta_params &p) {
     if (!p.q || !p.k || !p.v || !p.out) return TA_ERR_INVALID_ARG;
     if (p.rope_base < 0.f || !(p.rope_base == p.rope_base)) return TA_ERR_INVALID_ARG;
     if (p.rope_base > 0.f && (p.D & 1)) return TA_ERR_UNSUPPORTED;
+    if (p.window && p.ndims >= 1 && p.ndims <= TA_MAX_DIMS)
+        for (int i = 0; i < p.ndims; ++i)
+            if (p.window[i] < 0) return TA_ERR_INVALID_ARG;
     Plan plan;
     // the positional encoding gives every hop its own rotated Q and K: nothing to share, no fusion
     if (p.flags & kPlanFlagRope) return TA_ERR_UNSUPPORTED;
@@ -221,6 +225,7 @@ static int forward_impl(const ta_params &p) {
     pb.ndims = p.ndims; pb.causal = p.causal ? 1 : 0; pb.dtype = p.dtype;
     pb.scale = p.softmax_scale != 0.f ? p.softmax_scale : 1.0f / sqrtf((float)p.D);
     pb.rope_base = p.rope_base;
+    for (int i = 0; i < TA_MAX_DIMS; ++i) pb.window[i] = (p.window && i < p.ndims) ? p.window[i] : 0;
     pb.flags = p.flags; pb.hop_begin = p.hop_begin; pb.hop_end = p.hop_end;
     pb.stream = (cudaStream_t)p.stream;
 

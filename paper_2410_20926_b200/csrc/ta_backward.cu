@@ -49,6 +49,9 @@ int backward_impl(const ta_bwd_params &p) {
     if (p.grad_dtype != TA_DTYPE_BF16 && p.grad_dtype != TA_DTYPE_F32) return TA_ERR_UNSUPPORTED;
     if (p.rope_base < 0.f || !(p.rope_base == p.rope_base)) return TA_ERR_INVALID_ARG;
     if (p.rope_base > 0.f && (p.D & 1)) return TA_ERR_UNSUPPORTED;
+    if (p.window && p.ndims >= 1 && p.ndims <= TA_MAX_DIMS)
+        for (int i = 0; i < p.ndims; ++i)
+            if (p.window[i] < 0) return TA_ERR_INVALID_ARG;
     Plan plan;
     // hop by hop: the backward needs every hop's input
     int rc = build_plan(p.B, p.H, p.H_kv, p.N, p.D, p.dims, p.ndims, p.dtype, TA_FLAG_NO_HOP_FUSION, 0, 0, &plan);
@@ -78,6 +81,7 @@ int backward_impl(const ta_bwd_params &p) {
     pb.ndims = p.ndims; pb.causal = p.causal ? 1 : 0; pb.dtype = p.dtype;
     pb.scale = p.softmax_scale != 0.f ? p.softmax_scale : 1.0f / sqrtf((float)p.D);
     pb.rope_base = p.rope_base;
+    for (int i = 0; i < TA_MAX_DIMS; ++i) pb.window[i] = (p.window && i < p.ndims) ? p.window[i] : 0;
     pb.flags = 0; pb.hop_begin = 0; pb.hop_end = p.ndims;
     pb.stream = (cudaStream_t)p.stream;
 

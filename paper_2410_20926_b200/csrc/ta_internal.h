@@ -40,7 +40,7 @@ struct HopDesc {
     // 1): nf > 1 sub-hops, sub-hop f attends along a dimension of extent sub_n[f] whose
     // coordinate has stride sub_stride[f] tokens inside the block.  nf <= 1: an ordinary hop.
     int nf;
-    int sub_n[TA_MAX_DIMS], sub_stride[TA_MAX_DIMS];
+    int sub_n[TA_MAX_DIMS], sub_stride[TA_MAX_DIMS], sub_hop[TA_MAX_DIMS];   // sub_hop: index in dims
 };
 
 struct Plan {
@@ -61,6 +61,7 @@ struct Problem {
     int dtype;
     float scale;  // already resolved (1/sqrt(D) default)
     float rope_base;  // 0 = no positional encoding
+    int window[TA_MAX_DIMS];  // per dimension: 0 = none, w > 0 = keys within w positions of the query
     unsigned flags;
     int hop_begin, hop_end;
     cudaStream_t stream;

@@ -29,6 +29,7 @@ struct SimtArgs {
     long long items;              // B*H*segs_per_head*qblocks
     float scale;
     float rope_log2_base;         // 0: no positional encoding; else log2 of the RoPE base
+    int window;                   // 0, or sliding window along the hop's dimension
 };
 
 // Tensorized positional encoding (Section 3.2): rows of `x` ([rows][ld] fp32 in shared memory)
@@ -141,11 +142,14 @@ hop_simt_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__res
                 float s = 0.f;
                 for (int c = 0; c < D; ++c) s = fmaf(qr[c], kr[c], s);
                 s *= a.scale;
-                const bool valid = key < a.n && (!a.causal || key <= t);
+                const bool valid = key < a.n && (!a.causal || key <= t) &&
+                                   (a.window == 0 || (key > t - a.window && key < t + a.window));
                 s = valid ? s : -INFINITY;
-                const float m_new = fmaxf(m[r], warp_max(s));  // finite: key 0 is always visible
-                const float p = valid ? expf(s - m_new) : 0.f;
-                const float alpha = expf(m[r] - m_new);
+                // a block may hold no visible key of this row (window): keep the arithmetic finite
+                const float m_new = fmaxf(m[r], warp_max(s));
+                const float m_ref = m_new == -INFINITY ? 0.f : m_new;
+                const float p = valid ? expf(s - m_ref) : 0.f;
+                const float alpha = m[r] == -INFINITY ? 1.f : expf(m[r] - m_ref);
                 l[r] = l[r] * alpha + warp_sum(p);
                 m[r] = m_new;
 #pragma unroll
@@ -196,6 +200,7 @@ int launch_t(const Problem &pb, const HopDesc &hd, const void *xin, int xin_head
     a.items = (long long)pb.B * pb.H * a.segs_per_head * a.qblocks;
     a.scale = pb.scale;
     a.rope_log2_base = pb.rope_base > 0.f ? log2f(pb.rope_base) : 0.f;
+    a.window = pb.window[hd.hop];
     size_t smem = sizeof(float) * ((size_t)BQ * pb.D + 2 * (size_t)BK * (pb.D + 1));
     auto kern = hop_simt_kernel<T, DPL>;
     if (smem > 48 * 1024) {

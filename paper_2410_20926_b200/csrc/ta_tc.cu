@@ -67,6 +67,7 @@ struct TcArgs {
     int n, rows, ci, co, causal, g, H, H_kv, xin_is_kv;
     int gi, hsplit;            // query heads per work item, items per GQA group (gi * hsplit == g)
     long long tiles_inner, tiles_outer, total_items;
+    int window;                // 0, or w: keys within w positions of the query along the hop's dimension
     float scale_log2;
     float rope_log2_base;      // log2 of the RoPE base (rotating variant only)
 };
@@ -369,8 +370,12 @@ hop_pipe_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         const int r = wq * 32 + lane;                   // this thread's tile row = TMEM lane
         const int seg = r / a.n;
         const bool row_valid = r < a.rows;
-        const int c_lo = seg * a.n;
-        const int c_hi = a.causal ? r + 1 : c_lo + a.n; // visible key columns [c_lo, c_hi)
+        int c_lo = seg * a.n;
+        int c_hi = a.causal ? r + 1 : c_lo + a.n;       // visible key columns [c_lo, c_hi)
+        if (a.window > 0) {                             // sliding window along the hop's dimension
+            c_lo = max(c_lo, r - a.window + 1);
+            if (!a.causal) c_hi = min(c_hi, r + a.window);
+        }
         // columns any row of this warp needs (warp-uniform)
         const int w_lo = ((wq * 32) / a.n) * a.n;
         int w_hi = min(a.rows, ((wq * 32 + 31) / a.n + 1) * a.n);
@@ -545,6 +550,7 @@ int launch_d(const Problem &pb, const HopDesc &hd, const void *xin, int xin_head
         if (a.g % d == 0) a.hsplit = d;
     a.gi = a.g / a.hsplit;
     a.total_items = positions * a.hsplit;
+    a.window = pb.window[hd.hop];
     a.scale_log2 = pb.scale * 1.4426950408889634f;
     a.rope_log2_base = pb.rope_base > 0.f ? log2f(pb.rope_base) : 0.f;
 

@@ -43,6 +43,7 @@ constexpr int kThreadsRope = 416;      // + two warpgroups that rotate Q and K t
 struct BwdArgs {
     int n, rows, ci, co, causal, g, H, H_kv, x_is_kv, first_hop;
     int accumulate;                    // 0: dQ / dK are stored (first hop processed), 1: reduce-added
+    int window;                        // 0, or sliding window along the hop's dimension
     long long tiles_inner, tiles_outer, total_items;
     float scale_log2, scale;
     float rope_log2_base;              // log2 of the RoPE base (rotating variant only)
@@ -285,8 +286,12 @@ hop_tc_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         const int r = warp * 32 + lane;
         const int seg = r / a.n;
         const bool row_valid = r < a.rows;
-        const int c_lo = seg * a.n;
-        const int c_hi = a.causal ? r + 1 : c_lo + a.n;
+        int c_lo = seg * a.n;
+        int c_hi = a.causal ? r + 1 : c_lo + a.n;
+        if (a.window > 0) {
+            c_lo = max(c_lo, r - a.window + 1);
+            if (!a.causal) c_hi = min(c_hi, r + a.window);
+        }
         const int w_lo = ((warp * 32) / a.n) * a.n;
         int w_hi = min(a.rows, ((warp * 32 + 31) / a.n + 1) * a.n);
         if (a.causal) w_hi = min(w_hi, warp * 32 + 32);
@@ -634,6 +639,7 @@ int launch_bwd_d(const Problem &pb, const HopDesc &hd, const void *x, int x_head
     a.g = pb.H / pb.H_kv; a.H = pb.H; a.H_kv = pb.H_kv; a.x_is_kv = x_heads != pb.H ? 1 : 0;
     a.first_hop = first_hop ? 1 : 0;
     a.accumulate = accumulate ? 1 : 0;
+    a.window = pb.window[hd.hop];
     a.tiles_inner = hd.tiles_inner; a.tiles_outer = hd.tiles_outer;
     a.total_items = (long long)pb.B * pb.H_kv * hd.tiles_inner * hd.tiles_outer;
     a.scale = pb.scale;

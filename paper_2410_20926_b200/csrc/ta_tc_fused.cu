@@ -42,7 +42,7 @@ constexpr int kNK = 2, kNQ = 2;
 struct FusedArgs {
     int block, rows, co, causal, g, H, H_kv, xin_is_kv, nf;
     int gi, hsplit;            // query heads per work item, items per GQA group
-    int sub_n[TA_MAX_DIMS], sub_stride[TA_MAX_DIMS];
+    int sub_n[TA_MAX_DIMS], sub_stride[TA_MAX_DIMS], sub_window[TA_MAX_DIMS];
     long long tiles_outer, total_items;
     float scale_log2;
 };
@@ -142,7 +142,9 @@ hop_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             const int first = blk * a.block + rr - coord * st;
             const int last = a.causal ? coord : n - 1;
             uint32_t *m = masks + ((size_t)f * kTileRows + tid) * 4;
+            const int w = a.sub_window[f];              // sliding window along this dimension (0: none)
             for (int u = 0; u <= last; ++u) {
+                if (w > 0 && (u <= coord - w || u >= coord + w)) continue;
                 const int col = first + u * st;
                 m[col >> 5] |= 1u << (col & 31);
             }
@@ -458,6 +460,7 @@ int launch_fused_d(const Problem &pb, const HopDesc &hd, const void *xin, int xi
     for (int f = 0; f < TA_MAX_DIMS; ++f) {
         a.sub_n[f] = f < hd.nf ? hd.sub_n[f] : 1;
         a.sub_stride[f] = f < hd.nf ? hd.sub_stride[f] : 1;
+        a.sub_window[f] = f < hd.nf ? pb.window[hd.sub_hop[f]] : 0;
     }
     static int num_sms = 0;
     if (num_sms == 0) {

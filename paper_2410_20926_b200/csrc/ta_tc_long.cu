@@ -35,6 +35,7 @@ constexpr int kNKV = 2;   // key / value block ring
 
 struct LongArgs {
     int n, causal, g, H, H_kv, xin_is_kv, qblocks;
+    int window;                // 0, or w: keys within w positions of the query (blocks outside are skipped)
     long long stride, outer, total_items;
     float scale_log2;
 };
@@ -55,7 +56,8 @@ struct LongCfg {
 };
 
 struct LongItem {
-    int t0, inner, outer, q_head, kv_head, nkv;
+    int t0, inner, outer, q_head, kv_head;
+    int j0, nkv, keys_end;     // key blocks j0 .. j0+nkv-1 (128 keys each), keys [.., keys_end) in all
 };
 // item -> (query block, inner, outer, head).  Query blocks of a segment are adjacent, later
 // (longer, when causal) blocks first, so that the CTAs of one wave carry similar loads.
@@ -68,8 +70,15 @@ __device__ __forceinline__ LongItem decode_long_item(const LongArgs &a, long lon
     c.q_head = (int)rest;                                          // b * H + h
     c.kv_head = (c.q_head / a.H) * a.H_kv + (c.q_head % a.H) / a.g;
     c.t0 = qb * kTileRows;
-    const int last = a.causal ? min(c.t0 + kTileRows, a.n) : a.n;  // keys [0, last)
-    c.nkv = (last + kTileRows - 1) / kTileRows;
+    // keys any row of the tile can see: [first, keys_end)
+    int first = 0;
+    c.keys_end = a.causal ? min(c.t0 + kTileRows, a.n) : a.n;
+    if (a.window > 0) {
+        first = max(0, c.t0 - a.window + 1);
+        if (!a.causal) c.keys_end = min(a.n, c.t0 + kTileRows - 1 + a.window);
+    }
+    c.j0 = first / kTileRows;
+    c.nkv = (c.keys_end + kTileRows - 1) / kTileRows - c.j0;
     return c;
 }
 
@@ -89,7 +98,7 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32
         : "memory");
 }
 
-template <int D>
+template <int D, bool kWindow>
 __global__ void __launch_bounds__(kThreads, 1)
 hop_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                 const __grid_constant__ CUtensorMap map_xin, const __grid_constant__ CUtensorMap map_xout,
@@ -173,10 +182,10 @@ hop_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     arm(4u << st, par);
 #pragma unroll
                     for (int h = 0; h < kHalves; ++h)
-                        tma_load_5d(sKb(st) + h * kSlabBytes, &map_k, kv_full(st), 64 * h, kTileRows * j, c.inner, c.outer, c.kv_head);
+                        tma_load_5d(sKb(st) + h * kSlabBytes, &map_k, kv_full(st), 64 * h, kTileRows * (c.j0 + j), c.inner, c.outer, c.kv_head);
 #pragma unroll
                     for (int h = 0; h < kHalves; ++h)
-                        tma_load_5d(sXb(st) + h * kSlabBytes, &map_xin, kv_full(st), 64 * h, kTileRows * j, c.inner, c.outer, x_head);
+                        tma_load_5d(sXb(st) + h * kSlabBytes, &map_xin, kv_full(st), 64 * h, kTileRows * (c.j0 + j), c.inner, c.outer, x_head);
                 }
             }
             if (!ok) {
@@ -199,7 +208,6 @@ hop_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             for (long long item = blockIdx.x; ok && item < a.total_items; item += gridDim.x, ++ic) {
                 const LongItem c = decode_long_item(a, item);
                 const int qs = ic & 1;
-                const int keys_end = a.causal ? min(c.t0 + kTileRows, a.n) : a.n;
                 ok = mbar_wait_abortable(q_full(qs), (ic >> 1) & 1, 0xE0, abort_flag);
                 if (!ok) break;
                 auto issue_s = [&](int j) -> bool {
@@ -221,7 +229,7 @@ hop_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     const int st = g % kNKV;
                     if (!mbar_wait_abortable(p_full(g & 1), (g >> 1) & 1, 0xE2, abort_flag)) return false;
                     tc_fence_after();
-                    const int keys = min(kTileRows, keys_end - kTileRows * j);
+                    const int keys = min(kTileRows, c.keys_end - kTileRows * (c.j0 + j));
                     const int kblocks = (keys + 15) >> 4;
                     for (int kb = 0; kb < kblocks; ++kb)
                         tc_mma_ts(tmem_base + C::kColO, tmem_base + C::kColS + (g & 1) * 128 + kb * 8,
@@ -272,17 +280,22 @@ hop_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             const LongItem c = decode_long_item(a, item);
             const int t = c.t0 + r;                     // position of this row in the segment
             const bool row_valid = t < a.n;
-            const int keys_end = a.causal ? min(c.t0 + kTileRows, a.n) : a.n;
             float m_run = -INFINITY, l_run = 0.f;       // running maximum (scaled, log2 domain) and sum
             for (int j = 0; j < c.nkv; ++j, ++g) {
                 const uint32_t buf = g & 1;
                 const uint32_t s_col = tmem_lane + C::kColS + buf * 128;
-                const int u0 = kTileRows * j;
-                const int keys = min(kTileRows, keys_end - u0);            // key columns of this block
+                const int u0 = kTileRows * (c.j0 + j);
+                const int keys = min(kTileRows, c.keys_end - u0);          // key columns of this block
                 // columns any row of this warp can see in this block (warp-uniform)
                 const bool diag = a.causal && u0 == c.t0;
                 const int w_hi = diag ? min(keys, wq * 32 + 32) : keys;
-                const int c_hi = !row_valid ? 0 : (diag ? min(keys, r + 1) : keys);   // this row: columns [0, c_hi)
+                // this row: columns [c_lo, c_hi) of the block
+                int c_hi = !row_valid ? 0 : (diag ? min(keys, r + 1) : keys);
+                int c_lo = 0;                           // stays a compile-time 0 without a window
+                if (kWindow) {
+                    c_lo = max(0, t - a.window + 1 - u0);
+                    if (!a.causal) c_hi = min(c_hi, t + a.window - u0);
+                }
                 const int nchunks = (keys + 31) >> 5;
 
                 ok = mbar_wait_abortable(s_full(buf), (g >> 1) & 1, 0xF4, abort_flag);
@@ -298,10 +311,13 @@ hop_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     tmem_ld32(s_col + 32 * cc, v);
 #pragma unroll
                     for (int jj = 0; jj < 32; ++jj)
-                        if (32 * cc + jj < c_hi) bm = fmaxf(bm, __uint_as_float(v[jj]));
+                        if (32 * cc + jj >= c_lo && 32 * cc + jj < c_hi) bm = fmaxf(bm, __uint_as_float(v[jj]));
                 }
-                const float m_new = row_valid ? fmaxf(m_run, bm * a.scale_log2) : 0.f;
-                const float alpha = row_valid ? fast_exp2(m_run - m_new) : 1.f;     // 0 on the first block
+                // (with a window a row may see nothing in a block: the running maximum then stays -inf
+                // until its first visible key, and the reference below keeps the arithmetic finite)
+                const float m_new = fmaxf(m_run, bm * a.scale_log2);
+                const float m_ref = m_new == -INFINITY ? 0.f : m_new;
+                const float alpha = m_run == -INFINITY ? 1.f : fast_exp2(m_run - m_ref);
 
                 // ---- O <- alpha O, once the previous block's value MMA has completed
                 if (j > 0) {
@@ -330,10 +346,10 @@ hop_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 #pragma unroll
                         for (int jj = 0; jj < 32; jj += 2) {
                             const int col = 32 * cc + jj;
-                            float p0 = fast_exp2(__uint_as_float(v[jj]) * a.scale_log2 - m_new);
-                            float p1 = fast_exp2(__uint_as_float(v[jj + 1]) * a.scale_log2 - m_new);
-                            p0 = col < c_hi ? p0 : 0.f;
-                            p1 = col + 1 < c_hi ? p1 : 0.f;
+                            float p0 = fast_exp2(__uint_as_float(v[jj]) * a.scale_log2 - m_ref);
+                            float p1 = fast_exp2(__uint_as_float(v[jj + 1]) * a.scale_log2 - m_ref);
+                            p0 = (col >= c_lo && col < c_hi) ? p0 : 0.f;
+                            p1 = (col + 1 >= c_lo && col + 1 < c_hi) ? p1 : 0.f;
                             const uint32_t w = pack_bf16x2(p0, p1);
                             pk[jj >> 1] = w;
                             sum += __uint_as_float(w << 16) + __uint_as_float(w & 0xFFFF0000u);
@@ -409,6 +425,7 @@ int launch_long_d(const Problem &pb, const HopDesc &hd, const void *xin, int xin
     a.qblocks = (hd.n + kTileRows - 1) / kTileRows;
     a.stride = hd.stride; a.outer = hd.outer;
     a.total_items = (long long)pb.B * pb.H * hd.outer * hd.stride * a.qblocks;
+    a.window = pb.window[hd.hop];
     a.scale_log2 = pb.scale * 1.4426950408889634f;
 
     static int num_sms = 0;
@@ -419,15 +436,20 @@ int launch_long_d(const Problem &pb, const HopDesc &hd, const void *xin, int xin
             num_sms = 148;
     }
     constexpr size_t smem = LongCfg<D>::kSmemBytes;
-    auto kern = hop_long_kernel<D>;
     static bool configured = false;
     if (!configured) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        if (cudaFuncSetAttribute(hop_long_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+                cudaSuccess ||
+            cudaFuncSetAttribute(hop_long_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+                cudaSuccess)
             return TA_ERR_CUDA;
         configured = true;
     }
     const unsigned grid = (unsigned)(a.total_items < num_sms ? a.total_items : num_sms);
-    kern<<<grid, kThreads, smem, pb.stream>>>(mq, mk, mxi, mxo, a);
+    if (a.window > 0)
+        hop_long_kernel<D, true><<<grid, kThreads, smem, pb.stream>>>(mq, mk, mxi, mxo, a);
+    else
+        hop_long_kernel<D, false><<<grid, kThreads, smem, pb.stream>>>(mq, mk, mxi, mxo, a);
     count_launch();
     return cudaPeekAtLastError() == cudaSuccess ? TA_OK : TA_ERR_CUDA;
 }
