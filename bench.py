@@ -271,7 +271,7 @@ def run_ours(args, cfg):
     value = aggregate(cfg.B * cfg.N, world, ms, args.steps)
 
     # ---- end to end: host buffers in, host buffer out, copies inside the timed region
-    e2e_steps = max(1, min(args.steps, 5))
+    e2e_steps = max(1, min(args.steps, 10))
     for _ in range(2):
         ta.ta_forward_host(host["q"], host["k"], host["v"], host["out"], cfg.B, cfg.H, cfg.H_kv, cfg.N, cfg.D,
                            dims, cfg.causal, stream=stream)

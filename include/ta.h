@@ -203,10 +203,16 @@ size_t ta_workspace_bytes(int B, int H, int H_kv, int N, int D,
 
 /*
  * Whole forward pass from HOST buffers (bf16 or fp32 by `dtype`): copies q, k, v to device
- * staging memory owned by the library (allocated on first use, grown on demand, released by
- * ta_release), runs ta_forward_ex there and copies `out` back, all on `stream`; the host
- * buffers should be pinned for the copies to be asynchronous.  Returns after enqueueing; the
- * caller synchronises `stream` before reading out_host.
+ * staging memory owned by the library (two sets, allocated on first use, grown on demand,
+ * released by ta_release), runs ta_forward_ex there on `stream` and copies `out` back.  The
+ * uploads and the download run on two copy streams of the library, tied to `stream` by events:
+ * `stream` completes only when out_host has been written, while the upload of the NEXT call can
+ * already run during this call's kernels and download (PCIe is full duplex), so back-to-back
+ * calls cost about the longer of the two transfer directions.  The upload starts when the call
+ * is made (it is not ordered after earlier work on `stream`): q_host, k_host, v_host must hold
+ * their data by then and stay untouched, like out_host, until `stream` has completed this
+ * call.  The host buffers should be pinned for the copies to be asynchronous.  Returns after
+ * enqueueing; the caller synchronises `stream` before reading out_host.
  */
 int ta_forward_host(const void *q_host, const void *k_host, const void *v_host, void *out_host,
                     int B, int H, int H_kv, int N, int D,

@@ -179,6 +179,50 @@ struct Arena {
 static std::mutex g_arena_mutex;
 static Arena g_scratch, g_staging;
 
+// Copy engine of ta_forward_host: uploads and downloads run on two streams of their own and
+// the staging memory has two sets, so that the upload of one call overlaps the kernels and the
+// download of the previous one (PCIe is full duplex).
+struct HostPipe {
+    bool ready = false;
+    int device = -1;
+    cudaStream_t s_in = nullptr, s_out = nullptr;
+    cudaEvent_t in_done[2] = {}, k_done[2] = {}, out_done[2] = {};
+    bool used[2] = {false, false};
+    unsigned turn = 0;
+    int init() {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess) return TA_ERR_CUDA;
+        if (ready && dev == device) return TA_OK;
+        if (ready) destroy();
+        if (cudaStreamCreateWithFlags(&s_in, cudaStreamNonBlocking) != cudaSuccess ||
+            cudaStreamCreateWithFlags(&s_out, cudaStreamNonBlocking) != cudaSuccess)
+            return TA_ERR_CUDA;
+        for (int i = 0; i < 2; ++i)
+            if (cudaEventCreateWithFlags(&in_done[i], cudaEventDisableTiming) != cudaSuccess ||
+                cudaEventCreateWithFlags(&k_done[i], cudaEventDisableTiming) != cudaSuccess ||
+                cudaEventCreateWithFlags(&out_done[i], cudaEventDisableTiming) != cudaSuccess)
+                return TA_ERR_CUDA;
+        used[0] = used[1] = false;
+        turn = 0;
+        device = dev;
+        ready = true;
+        return TA_OK;
+    }
+    void destroy() {
+        if (!ready) return;
+        cudaStreamDestroy(s_in);
+        cudaStreamDestroy(s_out);
+        for (int i = 0; i < 2; ++i) {
+            cudaEventDestroy(in_done[i]);
+            cudaEventDestroy(k_done[i]);
+            cudaEventDestroy(out_done[i]);
+        }
+        ready = false;
+        device = -1;
+    }
+};
+static HostPipe g_host_pipe;
+
 static int check_arch() {
     static std::atomic<int> cached{1};  // 1 = unknown
     int c = cached.load();
@@ -320,22 +364,39 @@ int ta_forward_host(const void *qh, const void *kh, const void *vh, void *outh, 
     const size_t e = elem_bytes(dtype);
     const size_t qb = (size_t)B * H * N * D * e, kb = (size_t)B * H_kv * N * D * e;
     auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
-    char *base;
-    {
-        std::lock_guard<std::mutex> lock(g_arena_mutex);
-        rc = g_staging.reserve(2 * up(qb) + 2 * up(kb));
-        if (rc != TA_OK) return rc;
-        base = (char *)g_staging.ptr;
+    const size_t set_bytes = 2 * up(qb) + 2 * up(kb);
+    std::lock_guard<std::mutex> lock(g_arena_mutex);   // one call at a time enqueues into the pipe
+    HostPipe &hp = g_host_pipe;
+    if ((rc = hp.init()) != TA_OK) return rc;
+    if (g_staging.bytes < 2 * set_bytes || g_staging.device != hp.device) {
+        // growing the staging memory: nothing of an earlier call may still be using it
+        if (g_staging.ptr) cudaDeviceSynchronize();
+        hp.used[0] = hp.used[1] = false;
+        if ((rc = g_staging.reserve(2 * set_bytes)) != TA_OK) return rc;
     }
+    const int set = (int)(hp.turn++ & 1u);
+    char *base = (char *)g_staging.ptr + (size_t)set * set_bytes;
     char *dq = base, *dk = dq + up(qb), *dv = dk + up(kb), *dout = dv + up(kb);
     cudaStream_t s = (cudaStream_t)stream;
-    if (cudaMemcpyAsync(dq, qh, qb, cudaMemcpyHostToDevice, s) != cudaSuccess ||
-        cudaMemcpyAsync(dk, kh, kb, cudaMemcpyHostToDevice, s) != cudaSuccess ||
-        cudaMemcpyAsync(dv, vh, kb, cudaMemcpyHostToDevice, s) != cudaSuccess)
+    // upload (own stream): only waits until this staging set's previous result has been read back
+    if (hp.used[set] && cudaStreamWaitEvent(hp.s_in, hp.out_done[set], 0) != cudaSuccess) return TA_ERR_CUDA;
+    if (cudaMemcpyAsync(dq, qh, qb, cudaMemcpyHostToDevice, hp.s_in) != cudaSuccess ||
+        cudaMemcpyAsync(dk, kh, kb, cudaMemcpyHostToDevice, hp.s_in) != cudaSuccess ||
+        cudaMemcpyAsync(dv, vh, kb, cudaMemcpyHostToDevice, hp.s_in) != cudaSuccess ||
+        cudaEventRecord(hp.in_done[set], hp.s_in) != cudaSuccess)
         return TA_ERR_CUDA;
+    // kernels on the caller's stream
+    if (cudaStreamWaitEvent(s, hp.in_done[set], 0) != cudaSuccess) return TA_ERR_CUDA;
     rc = forward_simple(dq, dk, dv, dout, B, H, H_kv, N, D, dims, ndims, causal, dtype, stream);
     if (rc != TA_OK) return rc;
-    if (cudaMemcpyAsync(outh, dout, qb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return TA_ERR_CUDA;
+    if (cudaEventRecord(hp.k_done[set], s) != cudaSuccess) return TA_ERR_CUDA;
+    // download (own stream); the caller's stream completes only after it
+    if (cudaStreamWaitEvent(hp.s_out, hp.k_done[set], 0) != cudaSuccess ||
+        cudaMemcpyAsync(outh, dout, qb, cudaMemcpyDeviceToHost, hp.s_out) != cudaSuccess ||
+        cudaEventRecord(hp.out_done[set], hp.s_out) != cudaSuccess ||
+        cudaStreamWaitEvent(s, hp.out_done[set], 0) != cudaSuccess)
+        return TA_ERR_CUDA;
+    hp.used[set] = true;
     return TA_OK;
 }
 
@@ -416,9 +477,10 @@ unsigned long long ta_launch_count(void) { return g_launches.load(); }
 
 int ta_release(void) {
     std::lock_guard<std::mutex> lock(g_arena_mutex);
-    if (g_scratch.ptr || g_staging.ptr) cudaDeviceSynchronize();
+    if (g_scratch.ptr || g_staging.ptr || g_host_pipe.ready) cudaDeviceSynchronize();
     g_scratch.release();
     g_staging.release();
+    g_host_pipe.destroy();
     return TA_OK;
 }
 

@@ -157,3 +157,24 @@ def test_full_size_configs_sampled_heads(idx, heads):
     vmax = np.repeat(inp["v"].max(axis=2), g, axis=1)[:, :, None, :]
     vmin = np.repeat(inp["v"].min(axis=2), g, axis=1)[:, :, None, :]
     assert (got <= vmax + 0.05).all() and (got >= vmin - 0.05).all()
+
+
+def test_forward_host_back_to_back_calls_use_both_staging_sets():
+    """Host-buffer entry point: three calls in a row on one stream (uploads overlap the previous
+    call's kernels and download); every result must equal the device-resident run of its input."""
+    import torch
+    B, H, Hkv, D, dims = 1, 4, 2, 128, [8, 16, 32]
+    N = math.prod(dims)
+    stream = torch.cuda.current_stream()
+    outs, refs = [], []
+    for i in range(3):
+        inp = ta_inputs.make_inputs(B, H, Hkv, N, D, "bf16", 120 + i)
+        host = [torch.from_numpy(inp[n + "_bits"].view(np.int16)).view(torch.bfloat16).pin_memory() for n in "qkv"]
+        out_h = torch.empty((B, H, N, D), dtype=torch.bfloat16).pin_memory()
+        ta.ta_forward_host(host[0], host[1], host[2], out_h, B, H, Hkv, N, D, dims, True, stream=stream)
+        outs.append((host, out_h))
+        refs.append(gpu_forward(inp, B, H, Hkv, N, D, dims, True, "bf16"))
+    torch.cuda.synchronize()
+    ta.ta_device_status()
+    for (host, out_h), ref in zip(outs, refs):
+        np.testing.assert_array_equal(out_h.float().numpy(), ref)
