@@ -3,23 +3,27 @@
 // (Algorithm 1 loop body, Eq. 4; the softmax row no longer fits one tile, so it is taken
 // block by block with a running maximum and sum -- "online" softmax in fp32).
 //
-// A work item is 128 consecutive positions t0 .. t0+127 of one segment of one query head.  Its
-// Q tile stays in shared memory while the segment's keys go by in blocks of 128 (causal: up to
-// the block of the diagonal); per key block j
-//     S_j = Q K_j^T (tcgen05.mma, fp32 in TMEM, double-buffered)
-//     m <- max(m, rowmax S_j),  alpha = 2^(m_old - m),  l <- alpha l + rowsum P_j,
-//     P_j = 2^(S_j scale log2e - m)  (bf16, written back to TMEM over S_j)
-//     O <- alpha O  (in TMEM, only when some row's maximum moved)   then   O += P_j X_j
-// and finally O / l -> bf16 -> shared memory -> TMA store.  Rows of the strided view are reached
-// with the same rank-5 TMA maps as the short-segment kernel (box = 128 positions of one
-// segment); positions past n are zero-filled on load and clipped on store.  Several items read
-// the value rows another item writes, so the hop is not in place: xin != xout.
+// A work item is a pair of adjacent query tiles (2 x 128 consecutive positions) of one segment
+// of one query head.  Their Q tiles stay in shared memory while the segment's keys go by ONCE in
+// blocks of 128 (causal: up to each tile's diagonal block; with a window: only the blocks a
+// tile can see); per tile c and key block j
+//     S = Q_c K_j^T (tcgen05.mma, fp32 in TMEM)
+//     m <- max(m, rowmax S),  alpha = 2^(m_old - m),  l <- alpha l + rowsum P,
+//     P = 2^(S scale log2e - m)  (bf16, written back to TMEM over S)
+//     O_c <- alpha O_c  (in TMEM, only when some row's maximum moved)   then   O_c += P X_j
+// and finally O_c / l -> bf16 -> global memory (each thread owns one output row).  The two tiles
+// belong to two softmax warpgroups that alternate on the tensor pipe: while one computes its
+// softmax the MMAs of the other run.  Rows of the strided view are reached with the same rank-5
+// TMA maps as the short-segment kernel (box = 128 positions of one segment); positions past n
+// are zero-filled on load and skipped on store.  Several items read the value rows another item
+// writes, so the hop is not in place: xin != xout.
 //
-// Persistent, one CTA per SM: warp 0 TMA producer (Q per item, K_j / X_j into a two-stage
-// ring), warp 1 MMA issuer, warps 4-7 softmax / rescaling / epilogue (one TMEM lane = one
-// query row per thread), warp 2 TMA store.  Every wait is bounded; when one expires the CTA
-// raises a flag that ends all its roles, waits for its copies in flight, frees its TMEM and
-// returns.
+// Persistent, one CTA per SM: warp 0 TMA producer (the Q pair per item, K_j / X_j into a
+// two-stage ring shared by both tiles), warp 1 MMA issuer (polls for whichever of the two
+// tiles' next MMA has its operands ready), warps 4-7 and 8-11 softmax / rescaling / epilogue of
+// tile 0 and tile 1 (one TMEM lane = one query row per thread).  Every wait is bounded; when one
+// expires the CTA raises a flag that ends all its roles, waits for its copies in flight, frees
+// its TMEM and returns.
 #include <cuda_bf16.h>
 
 #include "ta_internal.h"
@@ -29,14 +33,14 @@ namespace ta {
 namespace {
 
 constexpr int kTileRows = 128;
-constexpr int kThreads = 256;
-constexpr int kNQ = 2;    // Q slots (one per item in flight)
+constexpr int kThreads = 384;
 constexpr int kNKV = 2;   // key / value block ring
 
 struct LongArgs {
-    int n, causal, g, H, H_kv, xin_is_kv, qblocks;
+    int n, causal, g, H, H_kv, xin_is_kv, qblocks, qpairs;
     int window;                // 0, or w: keys within w positions of the query (blocks outside are skipped)
     long long stride, outer, total_items;
+    long long row_stride, seg_outer_stride, head_stride;   // elements: between positions, outer blocks, heads
     float scale_log2;
 };
 
@@ -45,46 +49,54 @@ struct LongCfg {
     static constexpr int kHalves = D / 64;
     static constexpr uint32_t kSlabBytes = kTileRows * 128;
     static constexpr uint32_t kTileBytes = kHalves * kSlabBytes;
-    static constexpr uint32_t kOffQ = 0;
-    static constexpr uint32_t kOffKV = kOffQ + kNQ * kTileBytes;           // per stage: K then X
-    static constexpr uint32_t kOffOut = kOffKV + kNKV * 2 * kTileBytes;    // output staging
-    static constexpr uint32_t kOffBar = kOffOut + kTileBytes;
-    static constexpr int kNumBars = 2 * kNQ + 2 * kNKV + 2 + 2 + 1 + 2;
+    static constexpr uint32_t kOffQ = 0;                                   // the item's two Q tiles
+    static constexpr uint32_t kOffKV = kOffQ + 2 * kTileBytes;             // per stage: K then X
+    static constexpr uint32_t kOffBar = kOffKV + kNKV * 2 * kTileBytes;
+    static constexpr int kNumBars = 2 + 2 * kNKV + 6;
     static constexpr uint32_t kSmemBytes = kOffBar + kNumBars * 8 + 16 + 1024;
     static constexpr uint32_t kTmemCols = 512;
-    static constexpr uint32_t kColS = 0, kColO = 256;   // S: 2 x 128 (P over the first 64 of each), O: D
+    static constexpr uint32_t kColS = 0, kColO = 256;   // S_c at 128 c (P over its first 64 columns), O_c at 256 + 128 c
 };
 
 struct LongItem {
     int t0, inner, outer, q_head, kv_head;
-    int j0, nkv, keys_end;     // key blocks j0 .. j0+nkv-1 (128 keys each), keys [.., keys_end) in all
+    int ntiles;                // 1 or 2 query tiles (t0 and t0 + 128)
+    int j0[2], je[2];          // key blocks [j0, je) of each tile (128 keys each)
+    int keys_end[2];           // keys [.., keys_end) of each tile
+    int jlo, jhi;              // union of the two ranges: the blocks the item loads
 };
-// item -> (query block, inner, outer, head).  Query blocks of a segment are adjacent, later
-// (longer, when causal) blocks first, so that the CTAs of one wave carry similar loads.
+// item -> (pair of query tiles, inner, outer, head).  Pairs of a segment are adjacent, later
+// (longer, when causal) pairs first, so that the CTAs of one wave carry similar loads.
 __device__ __forceinline__ LongItem decode_long_item(const LongArgs &a, long long item) {
     LongItem c;
     long long rest = item;
-    const int qb = a.qblocks - 1 - (int)(rest % a.qblocks); rest /= a.qblocks;
+    const int pb = a.qpairs - 1 - (int)(rest % a.qpairs); rest /= a.qpairs;
     c.inner = (int)(rest % a.stride); rest /= a.stride;
     c.outer = (int)(rest % a.outer); rest /= a.outer;
     c.q_head = (int)rest;                                          // b * H + h
     c.kv_head = (c.q_head / a.H) * a.H_kv + (c.q_head % a.H) / a.g;
-    c.t0 = qb * kTileRows;
-    // keys any row of the tile can see: [first, keys_end)
-    int first = 0;
-    c.keys_end = a.causal ? min(c.t0 + kTileRows, a.n) : a.n;
-    if (a.window > 0) {
-        first = max(0, c.t0 - a.window + 1);
-        if (!a.causal) c.keys_end = min(a.n, c.t0 + kTileRows - 1 + a.window);
+    c.t0 = 2 * pb * kTileRows;
+    c.ntiles = 2 * pb + 1 < a.qblocks ? 2 : 1;
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        const int t0 = c.t0 + i * kTileRows;
+        // keys any row of the tile can see: [first, keys_end)
+        int first = 0;
+        int keys_end = a.causal ? min(t0 + kTileRows, a.n) : a.n;
+        if (a.window > 0) {
+            first = max(0, t0 - a.window + 1);
+            if (!a.causal) keys_end = min(a.n, t0 + kTileRows - 1 + a.window);
+        }
+        c.keys_end[i] = keys_end;
+        c.j0[i] = first / kTileRows;
+        c.je[i] = (keys_end + kTileRows - 1) / kTileRows;
     }
-    c.j0 = first / kTileRows;
-    c.nkv = (c.keys_end + kTileRows - 1) / kTileRows - c.j0;
+    if (c.ntiles == 1) { c.j0[1] = c.je[1] = c.je[0]; }            // an absent tile has no blocks
+    c.jlo = c.j0[0];
+    c.jhi = max(c.je[0], c.je[1]);
     return c;
 }
 
-__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
-    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
-}
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32]) {
     __syncwarp();
     asm volatile(
@@ -101,8 +113,7 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32
 template <int D, bool kWindow>
 __global__ void __launch_bounds__(kThreads, 1)
 hop_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                const __grid_constant__ CUtensorMap map_xin, const __grid_constant__ CUtensorMap map_xout,
-                const LongArgs a) {
+                const __grid_constant__ CUtensorMap map_xin, __nv_bfloat16 *__restrict__ xout, const LongArgs a) {
     using C = LongCfg<D>;
     constexpr int kHalves = C::kHalves;
     constexpr uint32_t kSlabBytes = C::kSlabBytes, kTileBytes = C::kTileBytes;
@@ -110,20 +121,17 @@ hop_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const uint32_t s0 = smem_u32(smem);
-    auto sQ = [&](int s) { return s0 + C::kOffQ + (uint32_t)s * kTileBytes; };
+    auto sQ = [&](int c) { return s0 + C::kOffQ + (uint32_t)c * kTileBytes; };
     auto sKb = [&](int s) { return s0 + C::kOffKV + (uint32_t)s * 2 * kTileBytes; };
     auto sXb = [&](int s) { return s0 + C::kOffKV + (uint32_t)s * 2 * kTileBytes + kTileBytes; };
-    const uint32_t sOut = s0 + C::kOffOut;
     const uint32_t bar0 = s0 + C::kOffBar;
-    auto q_full = [&](int i) { return bar0 + 8u * (uint32_t)i; };
-    auto q_free = [&](int i) { return bar0 + 8u * (uint32_t)(kNQ + i); };
-    auto kv_full = [&](int i) { return bar0 + 8u * (uint32_t)(2 * kNQ + i); };
-    auto kv_free = [&](int i) { return bar0 + 8u * (uint32_t)(2 * kNQ + kNKV + i); };
-    constexpr int kB1 = 2 * kNQ + 2 * kNKV;
-    auto s_full = [&](int i) { return bar0 + 8u * (uint32_t)(kB1 + i); };
-    auto p_full = [&](int i) { return bar0 + 8u * (uint32_t)(kB1 + 2 + i); };
-    const uint32_t pv_done = bar0 + 8u * (uint32_t)(kB1 + 4);
-    const uint32_t out_full = bar0 + 8u * (uint32_t)(kB1 + 5), out_free = bar0 + 8u * (uint32_t)(kB1 + 6);
+    const uint32_t q_full = bar0, q_free = bar0 + 8;
+    auto kv_full = [&](int i) { return bar0 + 8u * (uint32_t)(2 + i); };
+    auto kv_free = [&](int i) { return bar0 + 8u * (uint32_t)(2 + kNKV + i); };
+    constexpr int kB1 = 2 + 2 * kNKV;
+    auto s_full = [&](int c) { return bar0 + 8u * (uint32_t)(kB1 + c); };        // S of tile c complete
+    auto p_full = [&](int c) { return bar0 + 8u * (uint32_t)(kB1 + 2 + c); };    // P of tile c written (4 warps)
+    auto pv_done = [&](int c) { return bar0 + 8u * (uint32_t)(kB1 + 4 + c); };   // value MMA of tile c complete
     uint32_t *tmem_slot = (uint32_t *)(smem + C::kOffBar + C::kNumBars * 8);
     volatile uint32_t *abort_flag = tmem_slot + 1;
 
@@ -133,8 +141,7 @@ hop_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     if (tid == 0) {
         for (int i = 0; i < C::kNumBars; ++i) {
             const uint32_t bar = bar0 + 8u * (uint32_t)i;
-            // arrivals: one per softmax warp on p_full / out_full, a single thread or commit elsewhere
-            mbar_init(bar, (bar == p_full(0) || bar == p_full(1) || bar == out_full) ? 4 : 1);
+            mbar_init(bar, (bar == p_full(0) || bar == p_full(1)) ? 4 : 1);   // one arrival per softmax warp
         }
         *abort_flag = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -156,7 +163,7 @@ hop_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         // =============================================================== TMA producer
         if (lane == 0) {
             uint32_t ic = 0, g = 0;
-            uint32_t armed = 0, last_par = 0;        // bits: q 0-1, kv 2-3
+            uint32_t armed = 0, last_par = 0;        // bits: q 0, kv 1-2
             auto arm = [&](uint32_t bit, uint32_t parity) {
                 armed |= bit;
                 last_par = parity ? (last_par | bit) : (last_par & ~bit);
@@ -165,34 +172,34 @@ hop_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             for (long long item = blockIdx.x; ok && item < a.total_items; item += gridDim.x, ++ic) {
                 const LongItem c = decode_long_item(a, item);
                 const int x_head = a.xin_is_kv ? c.kv_head : c.q_head;
-                const int qs = ic & 1;
-                ok = mbar_wait_abortable(q_free(qs), ((ic >> 1) & 1) ^ 1, 0xD0, abort_flag);
+                ok = mbar_wait_abortable(q_free, (ic & 1) ^ 1, 0xD0, abort_flag);
                 if (!ok) break;
-                mbar_expect_tx(q_full(qs), kTileBytes);
-                arm(1u << qs, (ic >> 1) & 1);
+                mbar_expect_tx(q_full, c.ntiles * kTileBytes);
+                arm(1u, ic & 1);
+                for (int i = 0; i < c.ntiles; ++i)
 #pragma unroll
-                for (int h = 0; h < kHalves; ++h)
-                    tma_load_5d(sQ(qs) + h * kSlabBytes, &map_q, q_full(qs), 64 * h, c.t0, c.inner, c.outer, c.q_head);
-                for (int j = 0; j < c.nkv; ++j, ++g) {
+                    for (int h = 0; h < kHalves; ++h)
+                        tma_load_5d(sQ(i) + h * kSlabBytes, &map_q, q_full, 64 * h, c.t0 + kTileRows * i, c.inner, c.outer, c.q_head);
+                for (int j = c.jlo; j < c.jhi; ++j, ++g) {
                     const int st = g % kNKV;
                     const uint32_t par = (g / kNKV) & 1;
                     ok = mbar_wait_abortable(kv_free(st), par ^ 1, 0xD1, abort_flag);
                     if (!ok) break;
                     mbar_expect_tx(kv_full(st), 2 * kTileBytes);
-                    arm(4u << st, par);
+                    arm(2u << st, par);
 #pragma unroll
                     for (int h = 0; h < kHalves; ++h)
-                        tma_load_5d(sKb(st) + h * kSlabBytes, &map_k, kv_full(st), 64 * h, kTileRows * (c.j0 + j), c.inner, c.outer, c.kv_head);
+                        tma_load_5d(sKb(st) + h * kSlabBytes, &map_k, kv_full(st), 64 * h, kTileRows * j, c.inner, c.outer, c.kv_head);
 #pragma unroll
                     for (int h = 0; h < kHalves; ++h)
-                        tma_load_5d(sXb(st) + h * kSlabBytes, &map_xin, kv_full(st), 64 * h, kTileRows * (c.j0 + j), c.inner, c.outer, x_head);
+                        tma_load_5d(sXb(st) + h * kSlabBytes, &map_xin, kv_full(st), 64 * h, kTileRows * j, c.inner, c.outer, x_head);
                 }
             }
             if (!ok) {
                 const unsigned long long t0 = globaltimer_ns();
-                for (int slot = 0; slot < 4; ++slot) {
+                for (int slot = 0; slot < 1 + kNKV; ++slot) {
                     if (!(armed & (1u << slot))) continue;
-                    const uint32_t bar = slot < 2 ? q_full(slot) : kv_full(slot - 2);
+                    const uint32_t bar = slot == 0 ? q_full : kv_full(slot - 1);
                     while (!mbar_try_wait(bar, (last_par >> slot) & 1u) && globaltimer_ns() - t0 < 10000000ull) {
                     }
                 }
@@ -200,94 +207,115 @@ hop_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         }
     } else if (warp == 1) {
         // =============================================================== MMA issuer
+        // Two chains (the item's two query tiles) share the key blocks.  Chain c alternates
+        // S_c(j) = Q_c K_j^T and O_c += P_c(j) X_j; its single S buffer is free again once the
+        // value MMA that reads P from it has been issued.  A key block's stage is released when
+        // the last chain that uses the block has issued its value MMA.
         if (lane == 0) {
             constexpr uint32_t idesc_s = instr_desc(128, 0);
             constexpr uint32_t idesc_o = instr_desc(D, 1);
             uint32_t ic = 0, g0 = 0;
+            uint32_t p_seen[2] = {0, 0};              // phases of p_full(c) consumed
             bool ok = true;
             for (long long item = blockIdx.x; ok && item < a.total_items; item += gridDim.x, ++ic) {
                 const LongItem c = decode_long_item(a, item);
-                const int qs = ic & 1;
-                ok = mbar_wait_abortable(q_full(qs), (ic >> 1) & 1, 0xE0, abort_flag);
+                ok = mbar_wait_abortable(q_full, ic & 1, 0xE0, abort_flag);
                 if (!ok) break;
-                auto issue_s = [&](int j) -> bool {
-                    const uint32_t g = g0 + j;
-                    const int st = g % kNKV;
-                    if (!mbar_wait_abortable(kv_full(st), (g / kNKV) & 1, 0xE1, abort_flag)) return false;
-                    tc_fence_after();
+                int js[2] = {c.j0[0], c.j0[1]};       // next block whose S is to be issued
+                int jp[2] = {c.j0[0], c.j0[1]};       // next block whose value MMA is to be issued
+                bool q_released = false;
+                uint32_t idle = 0;
+                unsigned long long idle_since = 0;
+                while (jp[0] < c.je[0] || jp[1] < c.je[1]) {
+                    bool progressed = false;
 #pragma unroll
-                    for (int kb = 0; kb < D / 16; ++kb) {
-                        const uint32_t off = (kb >> 2) * kSlabBytes + (kb & 3) * 32;
-                        tc_mma_ss(tmem_base + C::kColS + (g & 1) * 128, smem_desc_sw128(sQ(qs) + off, 16, 1024),
-                                  smem_desc_sw128(sKb(st) + off, 16, 1024), idesc_s, kb > 0);
+                    for (int ch = 0; ch < 2; ++ch) {
+                        // ---- S_ch(js)
+                        if (js[ch] < c.je[ch] && js[ch] == jp[ch]) {
+                            const uint32_t g = g0 + (uint32_t)(js[ch] - c.jlo);
+                            const int st = g % kNKV;
+                            if (mbar_test_wait(kv_full(st), (g / kNKV) & 1)) {
+                                tc_fence_after();
+#pragma unroll
+                                for (int kb = 0; kb < D / 16; ++kb) {
+                                    const uint32_t off = (kb >> 2) * kSlabBytes + (kb & 3) * 32;
+                                    tc_mma_ss(tmem_base + C::kColS + ch * 128, smem_desc_sw128(sQ(ch) + off, 16, 1024),
+                                              smem_desc_sw128(sKb(st) + off, 16, 1024), idesc_s, kb > 0);
+                                }
+                                tc_commit(s_full(ch));
+                                ++js[ch];
+                                progressed = true;
+                            }
+                        }
+                        // ---- O_ch += P_ch(jp) X_jp
+                        if (jp[ch] < js[ch] && mbar_test_wait(p_full(ch), p_seen[ch] & 1)) {
+                            const int j = jp[ch];
+                            const uint32_t g = g0 + (uint32_t)(j - c.jlo);
+                            const int st = g % kNKV;
+                            tc_fence_after();
+                            const int keys = min(kTileRows, c.keys_end[ch] - kTileRows * j);
+                            const int kblocks = (keys + 15) >> 4;
+                            for (int kb = 0; kb < kblocks; ++kb)
+                                tc_mma_ts(tmem_base + C::kColO + ch * 128, tmem_base + C::kColS + ch * 128 + kb * 8,
+                                          smem_desc_sw128(sXb(st) + kb * 2048, kSlabBytes, 1024), idesc_o,
+                                          (kb > 0 || j > c.j0[ch]) ? 1u : 0u);
+                            tc_commit(pv_done(ch));
+                            ++p_seen[ch];
+                            ++jp[ch];
+                            // release the key block once the other chain is past it (or never uses it)
+                            const int o = ch ^ 1;
+                            if (!(j >= c.j0[o] && j < c.je[o]) || jp[o] > j) tc_commit(kv_free(st));
+                            progressed = true;
+                        }
                     }
-                    tc_commit(s_full(g & 1));
-                    return true;
-                };
-                auto issue_pv = [&](int j) -> bool {
-                    const uint32_t g = g0 + j;
-                    const int st = g % kNKV;
-                    if (!mbar_wait_abortable(p_full(g & 1), (g >> 1) & 1, 0xE2, abort_flag)) return false;
-                    tc_fence_after();
-                    const int keys = min(kTileRows, c.keys_end - kTileRows * (c.j0 + j));
-                    const int kblocks = (keys + 15) >> 4;
-                    for (int kb = 0; kb < kblocks; ++kb)
-                        tc_mma_ts(tmem_base + C::kColO, tmem_base + C::kColS + (g & 1) * 128 + kb * 8,
-                                  smem_desc_sw128(sXb(st) + kb * 2048, kSlabBytes, 1024), idesc_o, (kb > 0 || j > 0) ? 1u : 0u);
-                    tc_commit(kv_free(st));
-                    tc_commit(pv_done);
-                    return true;
-                };
-                ok = issue_s(0);
-                for (int j = 0; ok && j < c.nkv; ++j) {
-                    if (j + 1 < c.nkv) {
-                        ok = issue_s(j + 1);
-                        if (!ok) break;
+                    if (!q_released && js[0] == c.je[0] && js[1] == c.je[1]) {
+                        tc_commit(q_free);            // every S of this item has been issued
+                        q_released = true;
                     }
-                    if (j + 1 == c.nkv) tc_commit(q_free(qs));     // every S of this item has been issued
-                    ok = issue_pv(j);
+                    if (progressed) {
+                        idle = 0;
+                        idle_since = 0;
+                    } else if (++idle < 1024) {
+                        __nanosleep(20);
+                    } else {
+                        idle = 0;
+                        if (*abort_flag) { ok = false; break; }
+                        const unsigned long long now = globaltimer_ns();
+                        if (idle_since == 0) idle_since = now;
+                        if (now - idle_since > kWaitLimitNs) {
+                            atomicCAS(&g_status_word, 0u, kErrWaitExpired | 0xE5u);
+                            *abort_flag = 1u;
+                            ok = false;
+                            break;
+                        }
+                    }
                 }
-                g0 += c.nkv;
+                g0 += (uint32_t)(c.jhi - c.jlo);
             }
-        }
-    } else if (warp == 2) {
-        // =============================================================== TMA store
-        if (lane == 0) {
-            uint32_t ic = 0;
-            bool ok = true;
-            for (long long item = blockIdx.x; ok && item < a.total_items; item += gridDim.x, ++ic) {
-                const LongItem c = decode_long_item(a, item);
-                ok = mbar_wait_abortable(out_full, ic & 1, 0xF0, abort_flag);
-                if (!ok) break;
-#pragma unroll
-                for (int h = 0; h < kHalves; ++h)
-                    tma_store_5d(&map_xout, sOut + h * kSlabBytes, 64 * h, c.t0, c.inner, c.outer, c.q_head);
-                tma_store_commit_and_wait_read();
-                mbar_arrive(out_free);
-            }
-            tma_store_wait_all();
         }
     } else if (warp >= 4) {
         // =============================================================== softmax, rescaling, epilogue
+        const int ch = (warp - 4) >> 2;                 // which of the item's two query tiles
         const int wq = warp & 3;                        // TMEM lane quarter of this warp
         const uint32_t tmem_lane = tmem_base + ((uint32_t)(wq * 32) << 16);
         const int r = wq * 32 + lane;                   // this thread's query row of the tile
-        const uint32_t o_col = tmem_lane + C::kColO;
+        const uint32_t s_col = tmem_lane + C::kColS + ch * 128;
+        const uint32_t o_col = tmem_lane + C::kColO + ch * 128;
 
         bool ok = true;
-        uint32_t ic = 0, g = 0;
-        for (long long item = blockIdx.x; ok && item < a.total_items; item += gridDim.x, ++ic) {
+        uint32_t blocks_seen = 0;                       // key blocks this chain has processed (all items)
+        for (long long item = blockIdx.x; ok && item < a.total_items; item += gridDim.x) {
             const LongItem c = decode_long_item(a, item);
-            const int t = c.t0 + r;                     // position of this row in the segment
+            if (ch >= c.ntiles) continue;
+            const int t = c.t0 + kTileRows * ch + r;    // position of this row in the segment
             const bool row_valid = t < a.n;
+            const int keys_end = c.keys_end[ch];
             float m_run = -INFINITY, l_run = 0.f;       // running maximum (scaled, log2 domain) and sum
-            for (int j = 0; j < c.nkv; ++j, ++g) {
-                const uint32_t buf = g & 1;
-                const uint32_t s_col = tmem_lane + C::kColS + buf * 128;
-                const int u0 = kTileRows * (c.j0 + j);
-                const int keys = min(kTileRows, c.keys_end - u0);          // key columns of this block
+            for (int j = c.j0[ch]; j < c.je[ch]; ++j, ++blocks_seen) {
+                const int u0 = kTileRows * j;
+                const int keys = min(kTileRows, keys_end - u0);            // key columns of this block
                 // columns any row of this warp can see in this block (warp-uniform)
-                const bool diag = a.causal && u0 == c.t0;
+                const bool diag = a.causal && u0 == c.t0 + kTileRows * ch;
                 const int w_hi = diag ? min(keys, wq * 32 + 32) : keys;
                 // this row: columns [c_lo, c_hi) of the block
                 int c_hi = !row_valid ? 0 : (diag ? min(keys, r + 1) : keys);
@@ -298,20 +326,38 @@ hop_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 }
                 const int nchunks = (keys + 31) >> 5;
 
-                ok = mbar_wait_abortable(s_full(buf), (g >> 1) & 1, 0xF4, abort_flag);
+                ok = mbar_wait_abortable(s_full(ch), blocks_seen & 1, 0xF4, abort_flag);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 tc_fence_after();
 
+                // a block every row sees completely needs no per-element masks (most blocks of a long segment)
+                const bool full = !diag && !kWindow && keys == kTileRows && row_valid;
+                const bool full_w = __all_sync(0xffffffffu, full);
                 float bm = -INFINITY;
                 uint32_t v[32];
+                if (full_w) {
 #pragma unroll 1
-                for (int cc = 0; cc < nchunks; ++cc) {
-                    if (32 * cc >= w_hi) continue;      // warp-uniform
-                    tmem_ld32(s_col + 32 * cc, v);
+                    for (int cc = 0; cc < 4; ++cc) {
+                        tmem_ld32(s_col + 32 * cc, v);
+                        float b0 = fmaxf(__uint_as_float(v[0]), __uint_as_float(v[1]));
+                        float b1 = fmaxf(__uint_as_float(v[2]), __uint_as_float(v[3]));
 #pragma unroll
-                    for (int jj = 0; jj < 32; ++jj)
-                        if (32 * cc + jj >= c_lo && 32 * cc + jj < c_hi) bm = fmaxf(bm, __uint_as_float(v[jj]));
+                        for (int jj = 4; jj < 32; jj += 4) {
+                            b0 = fmaxf(b0, fmaxf(__uint_as_float(v[jj]), __uint_as_float(v[jj + 1])));
+                            b1 = fmaxf(b1, fmaxf(__uint_as_float(v[jj + 2]), __uint_as_float(v[jj + 3])));
+                        }
+                        bm = fmaxf(bm, fmaxf(b0, b1));
+                    }
+                } else {
+#pragma unroll 1
+                    for (int cc = 0; cc < nchunks; ++cc) {
+                        if (32 * cc >= w_hi) continue;      // warp-uniform
+                        tmem_ld32(s_col + 32 * cc, v);
+#pragma unroll
+                        for (int jj = 0; jj < 32; ++jj)
+                            if (32 * cc + jj >= c_lo && 32 * cc + jj < c_hi) bm = fmaxf(bm, __uint_as_float(v[jj]));
+                    }
                 }
                 // (with a window a row may see nothing in a block: the running maximum then stays -inf
                 // until its first visible key, and the reference below keeps the arithmetic finite)
@@ -320,8 +366,8 @@ hop_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 const float alpha = m_run == -INFINITY ? 1.f : fast_exp2(m_run - m_ref);
 
                 // ---- O <- alpha O, once the previous block's value MMA has completed
-                if (j > 0) {
-                    ok = mbar_wait_abortable(pv_done, (g - 1) & 1, 0xF5, abort_flag);
+                if (j > c.j0[ch]) {
+                    ok = mbar_wait_abortable(pv_done(ch), (blocks_seen - 1) & 1, 0xF5, abort_flag);
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
                     tc_fence_after();
@@ -336,68 +382,86 @@ hop_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     }
                 }
 
-                // ---- P_j (un-normalised, bf16) over the S columns already consumed
+                // ---- P (un-normalised, bf16) over the S columns already consumed
                 float sum = 0.f;
+                if (full_w) {
+                    // the row sum is taken over the fp32 weights here (the rounding of P averages out)
+                    float sum1 = 0.f;
 #pragma unroll 1
-                for (int cc = 0; cc < nchunks; ++cc) {
-                    uint32_t pk[16];
-                    if (32 * cc < w_hi) {
+                    for (int cc = 0; cc < 4; ++cc) {
+                        uint32_t pk[16];
                         tmem_ld32(s_col + 32 * cc, v);
 #pragma unroll
                         for (int jj = 0; jj < 32; jj += 2) {
-                            const int col = 32 * cc + jj;
-                            float p0 = fast_exp2(__uint_as_float(v[jj]) * a.scale_log2 - m_ref);
-                            float p1 = fast_exp2(__uint_as_float(v[jj + 1]) * a.scale_log2 - m_ref);
-                            p0 = (col >= c_lo && col < c_hi) ? p0 : 0.f;
-                            p1 = (col + 1 >= c_lo && col + 1 < c_hi) ? p1 : 0.f;
-                            const uint32_t w = pack_bf16x2(p0, p1);
-                            pk[jj >> 1] = w;
-                            sum += __uint_as_float(w << 16) + __uint_as_float(w & 0xFFFF0000u);
+                            const float p0 = fast_exp2(fmaf(__uint_as_float(v[jj]), a.scale_log2, -m_ref));
+                            const float p1 = fast_exp2(fmaf(__uint_as_float(v[jj + 1]), a.scale_log2, -m_ref));
+                            pk[jj >> 1] = pack_bf16x2(p0, p1);
+                            sum += p0;
+                            sum1 += p1;
                         }
-                    } else {
-#pragma unroll
-                        for (int jj = 0; jj < 16; ++jj) pk[jj] = 0u;
+                        tmem_st16(s_col + 16 * cc, pk);
                     }
-                    tmem_st16(s_col + 16 * cc, pk);
+                    sum += sum1;
+                } else {
+#pragma unroll 1
+                    for (int cc = 0; cc < nchunks; ++cc) {
+                        uint32_t pk[16];
+                        if (32 * cc < w_hi) {
+                            tmem_ld32(s_col + 32 * cc, v);
+#pragma unroll
+                            for (int jj = 0; jj < 32; jj += 2) {
+                                const int col = 32 * cc + jj;
+                                float p0 = fast_exp2(__uint_as_float(v[jj]) * a.scale_log2 - m_ref);
+                                float p1 = fast_exp2(__uint_as_float(v[jj + 1]) * a.scale_log2 - m_ref);
+                                p0 = (col >= c_lo && col < c_hi) ? p0 : 0.f;
+                                p1 = (col + 1 >= c_lo && col + 1 < c_hi) ? p1 : 0.f;
+                                const uint32_t w = pack_bf16x2(p0, p1);
+                                pk[jj >> 1] = w;
+                                sum += __uint_as_float(w << 16) + __uint_as_float(w & 0xFFFF0000u);
+                            }
+                        } else {
+#pragma unroll
+                            for (int jj = 0; jj < 16; ++jj) pk[jj] = 0u;
+                        }
+                        tmem_st16(s_col + 16 * cc, pk);
+                    }
                 }
                 tmem_st_wait();
                 l_run = l_run * alpha + sum;
                 m_run = m_new;
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(p_full(buf));
+                if (lane == 0) mbar_arrive(p_full(ch));
             }
             if (!ok) break;
 
-            // ---- epilogue: O / l -> bf16 -> staging (box layout) -> store warp
-            ok = mbar_wait_abortable(pv_done, (g - 1) & 1, 0xF6, abort_flag);
-            if (ok) ok = mbar_wait_abortable(out_free, (ic & 1) ^ 1, 0xF7, abort_flag);
+            // ---- epilogue: O / l -> bf16 -> this thread's output row in global memory
+            ok = mbar_wait_abortable(pv_done(ch), (blocks_seen - 1) & 1, 0xF6, abort_flag);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
             {
                 const float inv = (row_valid && l_run > 0.f) ? 1.f / l_run : 0.f;
+                __nv_bfloat16 *dst = xout + (long long)c.q_head * a.head_stride + (long long)c.outer * a.seg_outer_stride +
+                                     (long long)t * a.row_stride + (long long)c.inner * D;
                 uint32_t v[32];
-                const uint32_t row = sOut + (uint32_t)r * 128u;
 #pragma unroll 1
                 for (int cc = 0; cc < D / 32; ++cc) {
-                    tmem_ld32(o_col + 32 * cc, v);
-                    uint32_t pk[16];
+                    tmem_ld32(o_col + 32 * cc, v);      // whole warp; rows past n discard it
+                    if (row_valid) {
 #pragma unroll
-                    for (int jj = 0; jj < 32; jj += 2)
-                        pk[jj >> 1] = pack_bf16x2(__uint_as_float(v[jj]) * inv, __uint_as_float(v[jj + 1]) * inv);
-                    const uint32_t slab = row + (uint32_t)(cc >> 1) * kSlabBytes;
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const uint32_t chunk = (uint32_t)(((cc & 1) * 4 + i) ^ (r & 7));
-                        st_shared_v4(slab + chunk * 16, pk[4 * i], pk[4 * i + 1], pk[4 * i + 2], pk[4 * i + 3]);
+                        for (int i = 0; i < 4; ++i) {
+                            uint4 w;
+                            w.x = pack_bf16x2(__uint_as_float(v[8 * i]) * inv, __uint_as_float(v[8 * i + 1]) * inv);
+                            w.y = pack_bf16x2(__uint_as_float(v[8 * i + 2]) * inv, __uint_as_float(v[8 * i + 3]) * inv);
+                            w.z = pack_bf16x2(__uint_as_float(v[8 * i + 4]) * inv, __uint_as_float(v[8 * i + 5]) * inv);
+                            w.w = pack_bf16x2(__uint_as_float(v[8 * i + 6]) * inv, __uint_as_float(v[8 * i + 7]) * inv);
+                            *reinterpret_cast<uint4 *>(dst + 32 * cc + 8 * i) = w;
+                        }
                     }
                 }
             }
-            fence_proxy_async_smem();
             tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(out_full);
         }
     }
 
@@ -411,20 +475,23 @@ hop_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 
 template <int D>
 int launch_long_d(const Problem &pb, const HopDesc &hd, const void *xin, int xin_heads, void *xout) {
-    CUtensorMap mq, mk, mxi, mxo;
+    CUtensorMap mq, mk, mxi;
     int rc;
     // box: 128 positions of one segment (positions past n are zero-filled / clipped)
     if ((rc = make_view_map(&mq, pb.q, pb.B * pb.H, pb.N, D, hd, 2, kTileRows, 1, 1)) != TA_OK) return rc;
     if ((rc = make_view_map(&mk, pb.k, pb.B * pb.H_kv, pb.N, D, hd, 2, kTileRows, 1, 1)) != TA_OK) return rc;
     if ((rc = make_view_map(&mxi, xin, pb.B * xin_heads, pb.N, D, hd, 2, kTileRows, 1, 1)) != TA_OK) return rc;
-    if ((rc = make_view_map(&mxo, xout, pb.B * pb.H, pb.N, D, hd, 2, kTileRows, 1, 1)) != TA_OK) return rc;
 
     LongArgs a;
     a.n = hd.n; a.causal = pb.causal; a.g = pb.H / pb.H_kv; a.H = pb.H; a.H_kv = pb.H_kv;
     a.xin_is_kv = xin_heads != pb.H ? 1 : 0;
     a.qblocks = (hd.n + kTileRows - 1) / kTileRows;
+    a.qpairs = (a.qblocks + 1) / 2;
     a.stride = hd.stride; a.outer = hd.outer;
-    a.total_items = (long long)pb.B * pb.H * hd.outer * hd.stride * a.qblocks;
+    a.total_items = (long long)pb.B * pb.H * hd.outer * hd.stride * a.qpairs;
+    a.row_stride = hd.stride * (long long)D;
+    a.seg_outer_stride = (long long)hd.n * hd.stride * D;
+    a.head_stride = (long long)pb.N * D;
     a.window = pb.window[hd.hop];
     a.scale_log2 = pb.scale * 1.4426950408889634f;
 
@@ -447,9 +514,9 @@ int launch_long_d(const Problem &pb, const HopDesc &hd, const void *xin, int xin
     }
     const unsigned grid = (unsigned)(a.total_items < num_sms ? a.total_items : num_sms);
     if (a.window > 0)
-        hop_long_kernel<D, true><<<grid, kThreads, smem, pb.stream>>>(mq, mk, mxi, mxo, a);
+        hop_long_kernel<D, true><<<grid, kThreads, smem, pb.stream>>>(mq, mk, mxi, (__nv_bfloat16 *)xout, a);
     else
-        hop_long_kernel<D, false><<<grid, kThreads, smem, pb.stream>>>(mq, mk, mxi, mxo, a);
+        hop_long_kernel<D, false><<<grid, kThreads, smem, pb.stream>>>(mq, mk, mxi, (__nv_bfloat16 *)xout, a);
     count_launch();
     return cudaPeekAtLastError() == cudaSuccess ? TA_OK : TA_ERR_CUDA;
 }
