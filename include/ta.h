@@ -64,7 +64,8 @@ enum {
 /* flags of ta_params.flags */
 enum {
     TA_FLAG_NO_TENSOR_CORE = 1u << 0, /* run every hop on the generic CUDA-core kernel        */
-    TA_FLAG_NO_HOP_FUSION = 1u << 1,  /* one launch per hop, no cross-hop scheduling / fusion  */
+    TA_FLAG_NO_HOP_FUSION = 1u << 1,  /* one launch per hop: trailing hops that together fit one  */
+                                      /* 128-row tile are not fused into one pass               */
     TA_FLAG_SAVE_HOPS = 1u << 2       /* store hop inputs X_1..X_{m-1} in the workspace (for ta_backward) */
 };
 
@@ -226,14 +227,14 @@ int ta_forward_host(const void *q_host, const void *k_host, const void *v_host, 
  * latency-critical serving loop (cudaMalloc synchronises the device), processes whose device
  * memory is entirely managed by a pool the library cannot reach, and plug-ins that are only
  * permitted to launch kernels.  Same arguments and result as ta_forward_ex with default
- * options (dtype = TA_DTYPE_*), but the second value buffer that hops on the generic kernel
- * need (fp32 storage, n_i > 128, head dims other than 64 / 128) comes from a fixed array of
+ * options (dtype = TA_DTYPE_*), but the second value buffer that hops which cannot update in
+ * place need (fp32 storage, n_i > 128, head dims other than 64 / 128) comes from a fixed array of
  * TA_STATIC_SCRATCH_BYTES that is part of the loaded module -- every GPU that loads the
  * library holds those bytes until the process exits.  The call makes no cudaMalloc / cudaFree
  * and calls no allocating routine.
  *   - Problems whose value tensor (B*H*N*D elements) exceeds the array are rejected with
  *     TA_ERR_TOO_LARGE before anything is launched.  Problems that need no second buffer
- *     (every hop on the tensor-core kernel) have no size limit here.
+ *     (bf16, D in {64,128}, every n_i <= 128) have no size limit here.
  *   - The first call on each device looks up the array's device address (with that device
  *     current); make that first call before any stream capture begins.
  *   - All calls on a device share the one array and it keeps the previous call's contents.
@@ -248,7 +249,8 @@ int ta_forward_static(const void *q, const void *k, const void *v, void *out,
 
 /*
  * Text description of the launch plan the library would use for a problem (one line per hop:
- * kernel path, segment length, stride, tile packing, source / destination buffer).  Pure
+ * kernel path -- tc, tc-fused, tc-long or simt --, segment length, stride, tile packing,
+ * source / destination buffer).  Pure
  * host code: needs no GPU.  Writes at most `cap` bytes including the terminating NUL into
  * `buf` (host) and returns TA_OK or the TA_ERR_* the forward call would return.
  */
