@@ -29,12 +29,12 @@
 // Every wait is an mbarrier wait with a time limit; when one expires the CTA raises a flag that
 // ends all its roles, waits for its copies in flight, frees its TMEM and returns.
 #include <cuda_bf16.h>
-#include <cuda_fp16.h>
 
 #include <mutex>
 
 #include "ta_internal.h"
 #include "ta_ptx.cuh"
+#include "ta_rope.cuh"
 
 namespace ta {
 
@@ -86,10 +86,6 @@ __device__ __forceinline__ ItemCoord decode_item(const TcArgs &a, long long item
     c.kv_head = (int)rest;                                      // b * H_kv + kvh
     c.q_head0 = (c.kv_head / a.H_kv) * a.H + (c.kv_head % a.H_kv) * a.g + hs * a.gi;
     return c;
-}
-
-__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
-    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 
 // ----------------------------------------------------------------------------- the kernel
@@ -288,62 +284,8 @@ hop_pipe_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         }
     } else if (kRope && warp >= 12) {
         // =============================================================== RoPE on the K and Q tiles
-        // Row r of a tile sits at position t = r mod n of its segment, the same in every tile.
-        // A thread owns one 16-byte chunk of features (8 adjacent c < D/2, and their partners
-        // c + D/2) at the positions t = tsub, tsub + kTStep, .. (< n) of EVERY segment of the
-        // tile, so the cos / sin it needs never change: they sit in registers as fp16 pairs
-        // (absolute error 2^-12, far below bf16), computed once per launch, and a tile costs one
-        // 16-byte load and store per 8 features plus the multiply-adds.
-        constexpr int kChunks = D / 16;                   // 16-byte chunks of the first half of a row
-        const int rt = tid - 12 * 32;                     // 0 .. 255
-        const int chunk = rt % kChunks;
-        const int tsub = rt / kChunks;                    // 0 .. 31 (D = 128) or 0 .. 63 (D = 64)
-        constexpr int kTStep = 256 / kChunks;             // positions covered by one sweep of the threads
-        constexpr int kMaxPos = 128 / kTStep;             // sweeps to reach n = 128
-        const int segs = a.rows / a.n;
-        __half2 cs[kMaxPos][8];
-#pragma unroll
-        for (int pi = 0; pi < kMaxPos; ++pi)
-#pragma unroll
-            for (int e = 0; e < 8; ++e) {
-                const float ang = (float)(tsub + kTStep * pi) *
-                                  exp2f(-2.f * (float)(8 * chunk + e) / (float)D * a.rope_log2_base);
-                cs[pi][e] = __floats2half2_rn(__cosf(ang), __sinf(ang));
-            }
-
-        auto rotate_tile = [&](uint32_t tile) {
-#pragma unroll
-            for (int pi = 0; pi < kMaxPos; ++pi) {
-                const int t = tsub + kTStep * pi;
-                if (t >= a.n) break;
-#pragma unroll 2
-                for (int sg = 0; sg < segs; ++sg) {
-                    const int r = sg * a.n + t;
-                    const uint32_t row = tile + (uint32_t)r * 128u;
-                    const uint32_t addr_a = row + (((uint32_t)chunk ^ (uint32_t)(r & 7)) << 4);
-                    const uint32_t addr_b = D == 128 ? addr_a + kSlabBytes                   // partner: second slab
-                                                     : row + (((uint32_t)(chunk + 4) ^ (uint32_t)(r & 7)) << 4);
-                    uint32_t ua[4], ub[4];
-                    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
-                                 : "=r"(ua[0]), "=r"(ua[1]), "=r"(ua[2]), "=r"(ua[3]) : "r"(addr_a) : "memory");
-                    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
-                                 : "=r"(ub[0]), "=r"(ub[1]), "=r"(ub[2]), "=r"(ub[3]) : "r"(addr_b) : "memory");
-#pragma unroll
-                    for (int e2 = 0; e2 < 4; ++e2) {
-                        const float a0 = __uint_as_float(ua[e2] << 16), a1 = __uint_as_float(ua[e2] & 0xFFFF0000u);
-                        const float b0 = __uint_as_float(ub[e2] << 16), b1 = __uint_as_float(ub[e2] & 0xFFFF0000u);
-                        const float2 f0 = __half22float2(cs[pi][2 * e2]), f1 = __half22float2(cs[pi][2 * e2 + 1]);
-                        ua[e2] = pack_bf16x2(a0 * f0.x - b0 * f0.y, a1 * f1.x - b1 * f1.y);
-                        ub[e2] = pack_bf16x2(b0 * f0.x + a0 * f0.y, b1 * f1.x + a1 * f1.y);
-                    }
-                    st_shared_v4(addr_a, ua[0], ua[1], ua[2], ua[3]);
-                    st_shared_v4(addr_b, ub[0], ub[1], ub[2], ub[3]);
-                }
-            }
-            fence_proxy_async_smem();
-            __syncwarp();
-        };
-
+        RopeRotator<D> rot;
+        rot.init(tid - 12 * 32, a.n, a.rows, a.rope_log2_base);
         bool ok = true;
         uint32_t t = 0, it = 0;
         for (long long item = blockIdx.x; ok && item < a.total_items; item += gridDim.x, ++it) {
@@ -351,14 +293,14 @@ hop_pipe_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             ok = mbar_wait_abortable(k_full(ks), (it >> 1) & 1, 0x50, abort_flag);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
-            rotate_tile(sK + ks * kTileBytes);
+            rot.rotate(sK + ks * kTileBytes);
             if (lane == 0) mbar_arrive(k_rot(ks));
             for (int j = 0; j < a.gi; ++j, ++t) {
                 const int qs = t & 1;
                 ok = mbar_wait_abortable(q_full(qs), (t >> 1) & 1, 0x51, abort_flag);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
-                rotate_tile(sQ + qs * kTileBytes);
+                rot.rotate(sQ + qs * kTileBytes);
                 if (lane == 0) mbar_arrive(q_rot(qs));
             }
         }

@@ -80,10 +80,6 @@ __device__ __forceinline__ FusedItem decode_fused_item(const FusedArgs &a, long 
     return c;
 }
 
-__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
-    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
-}
-
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 hop_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,

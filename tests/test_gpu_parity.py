@@ -90,6 +90,12 @@ def test_full_attention_4096_sampled_heads():
     check_case(1, 8, 2, 4096, 128, [4096], True, "bf16", seed=114, heads=[(0, 0), (0, 5)])
 
 
+def test_full_attention_8192_llama_heads_sampled():
+    """Ordinary causal attention at 8 192 tokens with Llama head shapes (64 key blocks per segment,
+    32 pairs of query tiles): one whole head against the oracle."""
+    check_case(1, 32, 8, 8192, 128, [8192], True, "bf16", seed=115, heads=[(0, 13)])
+
+
 def test_unit_dims_and_broadcast():
     check_case(1, 4, 2, 64, 64, [1, 64, 1], True, "bf16", seed=107)
     inp = ta_inputs.make_inputs(2, 4, 2, 1, 64, "bf16", 108)

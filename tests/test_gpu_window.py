@@ -89,3 +89,14 @@ def test_backward_with_window(dims, window, D, causal):
     ref = oracle.backward(inp["dout"], inp["q"], inp["k"], inp["v"], dims, causal, window=window)
     for name, g, r in zip(("dq", "dk", "dv"), got, ref):
         assert_grad_close(g, r, name)
+
+
+def test_window_llama_shape_sampled_heads():
+    """Config 3's shape (32 768 tokens as 32x32x32, H=32, H_kv=8, D=128) with windows 8, 16, 4."""
+    c = ta_inputs.CONFIGS[3]
+    window = [8, 16, 4]
+    inp = ta_inputs.make_config_inputs(c)
+    got = gpu_forward(inp, c.B, c.H, c.H_kv, c.N, c.D, list(c.dims), True, "bf16", window=window)
+    heads = [(0, 2), (0, 29)]
+    ref = oracle.forward(inp["q"], inp["k"], inp["v"], list(c.dims), True, window=window, heads=heads)
+    assert_close(np.stack([got[b, h] for b, h in heads]), ref, "bf16")
