@@ -30,6 +30,9 @@ def main(argv=None) -> int:
     ap.add_argument("--no-fusion", action="store_true")
     ap.add_argument("--no-tensor-core", action="store_true")
     ap.add_argument("--f32-grads", action="store_true")
+    ap.add_argument("--saved-hops", action="store_true",
+                    help="backward: take the hop inputs from a forward run with TA_FLAG_SAVE_HOPS instead of "
+                         "recomputing them (the forward is not part of the timed repetitions)")
     ap.add_argument("--warmup", type=int, default=1)
     ap.add_argument("--reps", type=int, default=3)
     ap.add_argument("--seed", type=int, default=1)
@@ -64,11 +67,18 @@ def main(argv=None) -> int:
         mode = ta.TA_WS_BACKWARD_F32_GRADS if args.f32_grads else ta.TA_WS_BACKWARD
         nbytes = ta.ta_workspace_bytes(B, H, Hkv, N, D, dims, ta.TA_DTYPE_BF16, mode)
         ws = torch.empty(max(nbytes, 256), dtype=torch.uint8, device="cuda")
+        saved = None
+        if args.saved_hops:
+            nsave = ta.ta_workspace_bytes(B, H, Hkv, N, D, dims, ta.TA_DTYPE_BF16, ta.TA_WS_FORWARD_SAVE)
+            saved = torch.empty(max(nsave, 256), dtype=torch.uint8, device="cuda")
+            ta.ta_forward_ex(q, k, v, torch.empty_like(q), B, H, Hkv, N, D, dims, causal,
+                             flags=ta.TA_FLAG_SAVE_HOPS, workspace=saved, workspace_bytes=nsave,
+                             rope_base=args.rope_base)
 
         def step():
             ta.ta_backward_ex(dout, q, k, v, dq, dk, dv, B, H, Hkv, N, D, dims, causal,
                               grad_dtype=ta.TA_DTYPE_F32 if args.f32_grads else ta.TA_DTYPE_BF16,
-                              workspace=ws, workspace_bytes=nbytes, rope_base=args.rope_base)
+                              saved_hops=saved, workspace=ws, workspace_bytes=nbytes, rope_base=args.rope_base)
 
     for _ in range(args.warmup):
         step()
