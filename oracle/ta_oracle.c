@@ -41,7 +41,9 @@
  * Eq. 3): besides the causal mask, hop i may carry a sliding window w_i > 0 along its
  * dimension -- key position u is visible from query position t iff |t - u| < w_i (and u <= t
  * when causal).  w_i = 0 means no window.  Every row keeps its own position, so no row is
- * fully masked.
+ * fully masked.  Hop i may also carry an explicit n_i x n_i mask (row = query position, column
+ * = key position, non-zero = visible), applied on top of the causal flag and the window; a row
+ * left without any visible key is an error.
  */
 #include <math.h>
 #include <stdlib.h>
@@ -51,37 +53,46 @@
 #endif
 
 /* Attention weights of one segment: P[t*n+u], rows sum to 1 (Eq. 1 / Eq. 4). */
-static void segment_weights(const double *Q, const double *K, long base, long stride,
-                            int n, int D, double scale, int causal, int window, double *P)
+/* Is key position u visible from query position t in this hop? */
+static int visible(int t, int u, int causal, int window, const unsigned char *mask, int n)
+{
+    if (causal && u > t) return 0;
+    if (window > 0 && (t - u >= window || u - t >= window)) return 0;
+    if (mask && !mask[(long)t * n + u]) return 0;
+    return 1;
+}
+
+/* Attention weights of one segment: P[t*n+u], rows sum to 1 (Eq. 1 / Eq. 4); entries the mask
+ * removes have weight exactly 0.  Returns -1 if a row has no visible key. */
+static int segment_weights(const double *Q, const double *K, long base, long stride,
+                           int n, int D, double scale, int causal, int window,
+                           const unsigned char *mask, double *P)
 {
     for (int t = 0; t < n; ++t) {
         const double *qt = Q + (base + (long)t * stride) * D;
-        /* visible keys of row t: [u0, nu) */
-        int nu = causal ? t + 1 : n;
-        int u0 = 0;
-        if (window > 0) {
-            if (t - window + 1 > u0) u0 = t - window + 1;
-            if (!causal && t + window < nu) nu = t + window;
-        }
         double mx = -INFINITY;
-        for (int u = 0; u < u0; ++u) P[t * n + u] = 0.0;   /* outside the window: weight exactly 0 */
-        for (int u = u0; u < nu; ++u) {
+        int any = 0;
+        for (int u = 0; u < n; ++u) {
+            if (!visible(t, u, causal, window, mask, n)) { P[t * n + u] = 0.0; continue; }
             const double *ku = K + (base + (long)u * stride) * D;
             double s = 0.0;
             for (int c = 0; c < D; ++c) s += qt[c] * ku[c];
             s *= scale;
             P[t * n + u] = s;
             if (s > mx) mx = s;
+            any = 1;
         }
+        if (!any) return -1;
         double den = 0.0;
-        for (int u = u0; u < nu; ++u) {
+        for (int u = 0; u < n; ++u) {
+            if (!visible(t, u, causal, window, mask, n)) continue;
             double e = exp(P[t * n + u] - mx);
             P[t * n + u] = e;
             den += e;
         }
-        for (int u = u0; u < nu; ++u) P[t * n + u] /= den;
-        for (int u = nu; u < n; ++u) P[t * n + u] = 0.0;   /* masked: weight exactly 0 */
+        for (int u = 0; u < n; ++u) P[t * n + u] /= den;   /* masked entries stay 0 */
     }
+    return 0;
 }
 
 /* stride s_i and the enumeration of segments of hop i:
@@ -121,7 +132,8 @@ static void rope_rotate(const double *x, double *y, long N, int D, long stride, 
  */
 static int forward_head_impl(const double *q, const double *k, const double *v, double *out,
                              long N, int D, const int *dims, int ndims, int causal,
-                             double scale, double rope_base, const int *window, double *xs)
+                             double scale, double rope_base, const int *window,
+                             const unsigned char *const *masks, double *xs)
 {
     if (!q || !k || !v || !out || !dims || ndims < 1 || N < 1 || D < 1) return -1;
     long prod = 1;
@@ -162,7 +174,12 @@ static int forward_head_impl(const double *q, const double *k, const double *v, 
                 if (!P) continue;
                 long outer = g / s, inner = g % s;
                 long base = outer * n * s + inner;
-                segment_weights(q, k, base, s, n, D, scale, causal, window ? window[i] : 0, P);   /* A_i */
+                if (segment_weights(q, k, base, s, n, D, scale, causal, window ? window[i] : 0,
+                                    masks ? masks[i] : NULL, P) != 0) {                 /* A_i */
+                    #pragma omp atomic write
+                    fail = 1;
+                    continue;
+                }
                 for (int t = 0; t < n; ++t) {               /* O_i = A_i O_i, folded back */
                     double *o = nxt + (base + (long)t * s) * D;
                     for (int c = 0; c < D; ++c) o[c] = 0.0;
@@ -189,7 +206,7 @@ int ta_oracle_forward_head(const double *q, const double *k, const double *v, do
                            long N, int D, const int *dims, int ndims, int causal,
                            double scale, double *xs)
 {
-    return forward_head_impl(q, k, v, out, N, D, dims, ndims, causal, scale, 0.0, NULL, xs);
+    return forward_head_impl(q, k, v, out, N, D, dims, ndims, causal, scale, 0.0, NULL, NULL, xs);
 }
 
 /* As above with the tensorized positional encoding (rope_base > 0, e.g. 10000). */
@@ -198,17 +215,19 @@ int ta_oracle_forward_head_rope(const double *q, const double *k, const double *
                                 double scale, double rope_base, double *xs)
 {
     if (!(rope_base > 0.0)) return -1;
-    return forward_head_impl(q, k, v, out, N, D, dims, ndims, causal, scale, rope_base, NULL, xs);
+    return forward_head_impl(q, k, v, out, N, D, dims, ndims, causal, scale, rope_base, NULL, NULL, xs);
 }
 
-/* Every option: rope_base 0 = none; window NULL or [ndims] ints, 0 = no window in that hop. */
+/* Every option: rope_base 0 = none; window NULL or [ndims] ints, 0 = no window in that hop;
+ * masks NULL or [ndims] pointers, each NULL or an n_i x n_i byte matrix (non-zero = visible). */
 int ta_oracle_forward_head_ex(const double *q, const double *k, const double *v, double *out,
                               long N, int D, const int *dims, int ndims, int causal,
-                              double scale, double rope_base, const int *window, double *xs)
+                              double scale, double rope_base, const int *window,
+                              const unsigned char *const *masks, double *xs)
 {
     if (rope_base < 0.0) return -1;
     if (window) for (int i = 0; i < ndims; ++i) if (window[i] < 0) return -1;
-    return forward_head_impl(q, k, v, out, N, D, dims, ndims, causal, scale, rope_base, window, xs);
+    return forward_head_impl(q, k, v, out, N, D, dims, ndims, causal, scale, rope_base, window, masks, xs);
 }
 
 /*
@@ -228,7 +247,8 @@ int ta_oracle_forward_head_ex(const double *q, const double *k, const double *v,
 static int backward_head_impl(const double *q, const double *k, const double *xs,
                               const double *dout, double *dq, double *dk, double *dv,
                               long N, int D, const int *dims, int ndims, int causal,
-                              double scale, double rope_base, const int *window)
+                              double scale, double rope_base, const int *window,
+                              const unsigned char *const *masks)
 {
     if (!q || !k || !xs || !dout || !dq || !dk || !dv || !dims || ndims < 1) return -1;
     long prod = 1;
@@ -280,7 +300,12 @@ static int backward_head_impl(const double *q, const double *k, const double *xs
                 if (!P || !dS) continue;
                 long outer = sg / s, inner = sg % s;
                 long base = outer * n * s + inner;
-                segment_weights(q, k, base, s, n, D, scale, causal, window ? window[i] : 0, P);
+                if (segment_weights(q, k, base, s, n, D, scale, causal, window ? window[i] : 0,
+                                    masks ? masks[i] : NULL, P) != 0) {
+                    #pragma omp atomic write
+                    fail = 1;
+                    continue;
+                }
                 /* dP[t][u] = <G_{i+1}[t], X_i[u]>, then dS */
                 for (int t = 0; t < n; ++t) {
                     const double *gt = g + (base + (long)t * s) * D;
@@ -338,7 +363,7 @@ int ta_oracle_backward_head(const double *q, const double *k, const double *xs,
                             long N, int D, const int *dims, int ndims, int causal,
                             double scale)
 {
-    return backward_head_impl(q, k, xs, dout, dq, dk, dv, N, D, dims, ndims, causal, scale, 0.0, NULL);
+    return backward_head_impl(q, k, xs, dout, dq, dk, dv, N, D, dims, ndims, causal, scale, 0.0, NULL, NULL);
 }
 
 int ta_oracle_backward_head_rope(const double *q, const double *k, const double *xs,
@@ -348,17 +373,18 @@ int ta_oracle_backward_head_rope(const double *q, const double *k, const double 
 {
     if (!(rope_base > 0.0)) return -1;
     return backward_head_impl(q, k, xs, dout, dq, dk, dv, N, D, dims, ndims, causal, scale,
-                              rope_base, NULL);
+                              rope_base, NULL, NULL);
 }
 
 int ta_oracle_backward_head_ex(const double *q, const double *k, const double *xs,
                                const double *dout, double *dq, double *dk, double *dv,
                                long N, int D, const int *dims, int ndims, int causal,
-                               double scale, double rope_base, const int *window)
+                               double scale, double rope_base, const int *window,
+                               const unsigned char *const *masks)
 {
     if (rope_base < 0.0) return -1;
     return backward_head_impl(q, k, xs, dout, dq, dk, dv, N, D, dims, ndims, causal, scale,
-                              rope_base, window);
+                              rope_base, window, masks);
 }
 
 int ta_oracle_num_threads(void)

@@ -66,11 +66,12 @@ def _lib():
         lib.ta_oracle_forward_head_ex.restype = ctypes.c_int
         lib.ta_oracle_forward_head_ex.argtypes = [dp, dp, dp, dp, ctypes.c_long, ctypes.c_int, ip,
                                                   ctypes.c_int, ctypes.c_int, ctypes.c_double,
-                                                  ctypes.c_double, ip, dp]
+                                                  ctypes.c_double, ip, ctypes.POINTER(ctypes.c_void_p), dp]
         lib.ta_oracle_backward_head_ex.restype = ctypes.c_int
         lib.ta_oracle_backward_head_ex.argtypes = [dp, dp, dp, dp, dp, dp, dp, ctypes.c_long,
                                                    ctypes.c_int, ip, ctypes.c_int, ctypes.c_int,
-                                                   ctypes.c_double, ctypes.c_double, ip]
+                                                   ctypes.c_double, ctypes.c_double, ip,
+                                                   ctypes.POINTER(ctypes.c_void_p)]
         lib.ta_oracle_num_threads.restype = ctypes.c_int
         _LIB = lib
     return _LIB
@@ -114,10 +115,29 @@ def _cwindow(window, m):
     return (ctypes.c_int * m)(*w)
 
 
-def _fwd_head(lib, qh, kh, vh, out, N, D, cdims, m, causal, scale, rope_base, xs, cwin=None):
-    if cwin is not None:
+def _cmasks(masks, dims):
+    """Per-dimension masks as a C array of byte-matrix pointers; returns (array or None, keep-alive)."""
+    if masks is None:
+        return None, None
+    if len(masks) != len(dims):
+        raise ValueError("masks: one entry (or None) per dimension")
+    keep, ptrs = [], []
+    for mk, n in zip(masks, dims):
+        if mk is None:
+            ptrs.append(None)
+            continue
+        a = np.ascontiguousarray(np.asarray(mk) != 0, dtype=np.uint8)
+        if a.shape != (n, n):
+            raise ValueError("mask of a dimension of extent n must be n x n")
+        keep.append(a)
+        ptrs.append(a.ctypes.data)
+    return (ctypes.c_void_p * len(dims))(*ptrs), keep
+
+
+def _fwd_head(lib, qh, kh, vh, out, N, D, cdims, m, causal, scale, rope_base, xs, cwin=None, cmask=None):
+    if cwin is not None or cmask is not None:
         return lib.ta_oracle_forward_head_ex(_dptr(qh), _dptr(kh), _dptr(vh), _dptr(out), N, D, cdims, m,
-                                             int(bool(causal)), scale, float(rope_base or 0.0), cwin,
+                                             int(bool(causal)), scale, float(rope_base or 0.0), cwin, cmask,
                                              _dptr(xs) if xs is not None else None)
     if rope_base:
         return lib.ta_oracle_forward_head_rope(_dptr(qh), _dptr(kh), _dptr(vh), _dptr(out), N, D,
@@ -128,7 +148,7 @@ def _fwd_head(lib, qh, kh, vh, out, N, D, cdims, m, causal, scale, rope_base, xs
 
 
 def forward(q, k, v, dims, causal: bool, scale: float | None = None, heads=None,
-            return_xs: bool = False, rope_base: float | None = None, window=None):
+            return_xs: bool = False, rope_base: float | None = None, window=None, masks=None):
     """Algorithm 1 for every (or the listed) head, fp64.
 
     q: [B,H,N,D]; k, v: [B,H_kv,N,D] (any float dtype; converted head by head to fp64).
@@ -138,6 +158,8 @@ def forward(q, k, v, dims, causal: bool, scale: float | None = None, heads=None,
     tensorized positional encoding (hop i rotates q, k by the coordinate along dimension i).
     window: None, or one int per dimension: w_i > 0 keeps, in hop i, only keys within w_i
     positions of the query along dimension i (|t - u| < w_i); 0 = no window.
+    masks: None, or one entry per dimension: None or an n_i x n_i array (row = query position,
+    column = key position, non-zero = visible) applied on top of `causal` and `window`.
     Returns out [B,H,N,D] fp64 (and, with return_xs, the list of per-head [m+1,N,D]
     value tensors X_0=V ... X_m=out keyed like the output).
     """
@@ -146,6 +168,7 @@ def forward(q, k, v, dims, causal: bool, scale: float | None = None, heads=None,
     scale = 1.0 / math.sqrt(D) if scale is None else float(scale)
     cdims = (ctypes.c_int * len(dims))(*dims)
     cwin = _cwindow(window, len(dims))
+    cmask, _keep = _cmasks(masks, dims)
     pairs = [(b, h) for b in range(B) for h in range(H)] if heads is None else list(heads)
     out = np.empty((len(pairs), N, D), dtype=np.float64)
     xs_all = []
@@ -154,7 +177,7 @@ def forward(q, k, v, dims, causal: bool, scale: float | None = None, heads=None,
         qh, kh, vh = _f64(q[b, h]), _f64(k[b, h // g]), _f64(v[b, h // g])
         xs = np.empty((len(dims) + 1, N, D), dtype=np.float64) if return_xs else None
         rc = _fwd_head(lib, qh, kh, vh, out[idx], N, D, cdims, len(dims), causal, scale,
-                       rope_base, xs, cwin)
+                       rope_base, xs, cwin, cmask)
         if rc != 0:
             raise RuntimeError("ta_oracle_forward_head failed")
         if return_xs:
@@ -165,7 +188,7 @@ def forward(q, k, v, dims, causal: bool, scale: float | None = None, heads=None,
 
 
 def backward(dout, q, k, v, dims, causal: bool, scale: float | None = None, groups=None,
-             rope_base: float | None = None, window=None):
+             rope_base: float | None = None, window=None, masks=None):
     """Gradients of sum(out * dout) w.r.t. q, k, v (fp64), GQA groups summed into dk, dv.
 
     groups: optional list of (b, kv_head) pairs; then only those KV heads and their query
@@ -176,6 +199,7 @@ def backward(dout, q, k, v, dims, causal: bool, scale: float | None = None, grou
     scale = 1.0 / math.sqrt(D) if scale is None else float(scale)
     cdims = (ctypes.c_int * len(dims))(*dims)
     cwin = _cwindow(window, len(dims))
+    cmask, _keep = _cmasks(masks, dims)
     sel = [(b, kv) for b in range(B) for kv in range(Hkv)] if groups is None else list(groups)
     dq = np.zeros((len(sel), g, N, D))
     dk = np.zeros((len(sel), N, D))
@@ -188,15 +212,16 @@ def backward(dout, q, k, v, dims, causal: bool, scale: float | None = None, grou
             qh = _f64(q[b, h])
             o = np.empty((N, D))
             xs = np.empty((len(dims) + 1, N, D))
-            rc = _fwd_head(lib, qh, kh, vh, o, N, D, cdims, len(dims), causal, scale, rope_base, xs, cwin)
+            rc = _fwd_head(lib, qh, kh, vh, o, N, D, cdims, len(dims), causal, scale, rope_base, xs, cwin, cmask)
             if rc != 0:
                 raise RuntimeError("ta_oracle_forward_head failed")
             dqh, dkh, dvh = np.empty((N, D)), np.empty((N, D)), np.empty((N, D))
-            if cwin is not None:
+            if cwin is not None or cmask is not None:
                 rc = lib.ta_oracle_backward_head_ex(_dptr(qh), _dptr(kh), _dptr(xs),
                                                     _dptr(_f64(dout[b, h])), _dptr(dqh), _dptr(dkh),
                                                     _dptr(dvh), N, D, cdims, len(dims),
-                                                    int(bool(causal)), scale, float(rope_base or 0.0), cwin)
+                                                    int(bool(causal)), scale, float(rope_base or 0.0), cwin,
+                                                    cmask)
             elif rope_base:
                 rc = lib.ta_oracle_backward_head_rope(_dptr(qh), _dptr(kh), _dptr(xs),
                                                       _dptr(_f64(dout[b, h])), _dptr(dqh),
@@ -223,7 +248,7 @@ def backward(dout, q, k, v, dims, causal: bool, scale: float | None = None, grou
 # --------------------------------------------------------------------------------------
 
 def dense_hop_matrix(qh, kh, dims, i: int, causal: bool, scale: float | None = None,
-                     rope_base: float | None = None, window=None):
+                     rope_base: float | None = None, window=None, masks=None):
     """The N x N matrix of hop i for one head (Eq. 3 written over flat token indices).
 
     Entry [j, k] is the softmax weight of key token k for query token j; it is non-zero only
@@ -244,6 +269,8 @@ def dense_hop_matrix(qh, kh, dims, i: int, causal: bool, scale: float | None = N
                 allowed &= ck <= cj
             if window is not None and window[i] > 0:
                 allowed &= np.abs(cj - ck) < window[i]
+            if masks is not None and masks[i] is not None:
+                allowed &= np.asarray(masks[i])[cj, ck] != 0        # looked up by the two coordinates
     if rope_base:
         # relative form of the rotary score: features c and c + D/2 form one complex number
         half = D // 2
@@ -266,23 +293,23 @@ def dense_hop_matrix(qh, kh, dims, i: int, causal: bool, scale: float | None = N
 
 
 def dense_effective_matrix(qh, kh, dims, causal: bool, scale: float | None = None,
-                           rope_base: float | None = None, window=None):
+                           rope_base: float | None = None, window=None, masks=None):
     """A_eff = A^_{m-1} ... A^_1 A^_0, the N x N map from V to the output of one head."""
     N = np.asarray(qh).shape[0]
     a = np.eye(N)
     for i in range(len(dims)):
-        a = dense_hop_matrix(qh, kh, dims, i, causal, scale, rope_base, window) @ a
+        a = dense_hop_matrix(qh, kh, dims, i, causal, scale, rope_base, window, masks) @ a
     return a
 
 
 def forward_dense(q, k, v, dims, causal: bool, scale: float | None = None,
-                  rope_base: float | None = None, window=None):
+                  rope_base: float | None = None, window=None, masks=None):
     """Brute-force forward for all heads via dense_effective_matrix (tiny N only)."""
     B, H, Hkv, N, D, dims = _check(q, k, v, dims)
     g = H // Hkv
     out = np.empty((B, H, N, D))
     for b in range(B):
         for h in range(H):
-            a = dense_effective_matrix(q[b, h], k[b, h // g], dims, causal, scale, rope_base, window)
+            a = dense_effective_matrix(q[b, h], k[b, h // g], dims, causal, scale, rope_base, window, masks)
             out[b, h] = a @ np.asarray(v[b, h // g], dtype=np.float64)
     return out

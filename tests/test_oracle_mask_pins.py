@@ -101,3 +101,82 @@ def test_backward_with_window_finite_differences(causal):
             arr[idx] = old
             fd = (lp - lm) / (2 * eps)
             assert abs(fd - grad[idx]) < 2e-7 * max(1.0, abs(fd)), (name, idx, fd, grad[idx])
+
+
+# ---------------------------------------------------------------- explicit per-hop masks M_i
+def random_mask(n, rng, keep_diag=True):
+    m = rng.random((n, n)) < 0.5
+    if keep_diag:
+        m |= np.eye(n, dtype=bool)          # every row keeps its own position
+    return m
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_explicit_masks_match_dense_route(causal):
+    rng = np.random.default_rng(51)
+    dims = [3, 4, 5]
+    N = 60
+    masks = [random_mask(3, rng), None, random_mask(5, rng)]
+    q, k, v = rnd((1, 4, N, 6), 52), rnd((1, 2, N, 6), 53), rnd((1, 2, N, 6), 54)
+    a = oracle.forward(q, k, v, dims, causal, masks=masks, window=[0, 3, 0])
+    b = oracle.forward_dense(q, k, v, dims, causal, masks=masks, window=[0, 3, 0])
+    np.testing.assert_allclose(a, b, rtol=0, atol=1e-13)
+
+
+def test_mask_expresses_the_causal_flag_and_the_window():
+    """Three features that must agree: an explicit lower-triangular mask is the causal flag, and an
+    explicit band mask is the window parameter."""
+    dims = [4, 6]
+    q, k, v = rnd((1, 2, 24, 4), 55), rnd((1, 2, 24, 4), 56), rnd((1, 2, 24, 4), 57)
+    tril = [np.tril(np.ones((n, n), dtype=bool)) for n in dims]
+    np.testing.assert_allclose(oracle.forward(q, k, v, dims, False, masks=tril),
+                               oracle.forward(q, k, v, dims, True), atol=1e-15)
+    band = [np.abs(np.subtract.outer(np.arange(n), np.arange(n))) < w for n, w in zip(dims, (2, 3))]
+    np.testing.assert_allclose(oracle.forward(q, k, v, dims, True, masks=band),
+                               oracle.forward(q, k, v, dims, True, window=[2, 3]), atol=1e-15)
+    ones = [np.ones((n, n)) for n in dims]
+    np.testing.assert_allclose(oracle.forward(q, k, v, dims, True, masks=ones),
+                               oracle.forward(q, k, v, dims, True), atol=0)
+
+
+def test_zero_queries_average_the_masked_set():
+    rng = np.random.default_rng(58)
+    n = 7
+    m = random_mask(n, rng)
+    v = rnd((1, 1, n, 3), 59)
+    got = oracle.forward(np.zeros((1, 1, n, 3)), rnd((1, 1, n, 3), 60), v, [n], False, masks=[m])[0, 0]
+    for t in range(n):
+        np.testing.assert_allclose(got[t], v[0, 0, m[t]].mean(axis=0), atol=1e-14)
+
+
+def test_mask_with_an_empty_row_is_rejected():
+    m = np.ones((4, 4), dtype=bool)
+    m[2] = False
+    q = rnd((1, 1, 4, 2), 61)
+    with pytest.raises(RuntimeError):
+        oracle.forward(q, q, q, [4], False, masks=[m])
+
+
+def test_backward_with_explicit_mask_finite_differences():
+    rng = np.random.default_rng(62)
+    dims, D = [3, 4], 4
+    masks = [random_mask(3, rng), random_mask(4, rng)]
+    q, k, v = rng.standard_normal((1, 2, 12, D)), rng.standard_normal((1, 1, 12, D)), rng.standard_normal((1, 1, 12, D))
+    dout = rng.standard_normal((1, 2, 12, D))
+    dq, dk, dv = oracle.backward(dout, q, k, v, dims, False, masks=masks)
+
+    def loss(q_, k_, v_):
+        return float((oracle.forward(q_, k_, v_, dims, False, masks=masks) * dout).sum())
+
+    eps = 1e-6
+    for name, arr, grad in (("q", q, dq), ("k", k, dk), ("v", v, dv)):
+        for _ in range(10):
+            idx = tuple(rng.integers(0, s) for s in arr.shape)
+            old = arr[idx]
+            arr[idx] = old + eps
+            lp = loss(q, k, v)
+            arr[idx] = old - eps
+            lm = loss(q, k, v)
+            arr[idx] = old
+            fd = (lp - lm) / (2 * eps)
+            assert abs(fd - grad[idx]) < 2e-7 * max(1.0, abs(fd)), (name, idx, fd, grad[idx])
