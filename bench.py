@@ -306,7 +306,7 @@ def run_ours(args, cfg):
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": NCU_TRAFFIC_BYTES_PER_TOKEN_PER_LAUNCH * cfg.B * cfg.N,
                 "traffic_source": "ncu capture of config 3 scaled by tokens (profiles/)", "peak_source": peak_src,
-                "kernel": "hop_pipe_kernel<128, false>", "algorithmic_bytes_per_launch": bytes_per_launch,
+                "kernel": "hop_pipe_kernel<128, false, false>", "algorithmic_bytes_per_launch": bytes_per_launch,
                 "launches_per_step": n_launch, "avg_launch_ms": launch_ms,
                 "useful_tflops": step_flops(cfg) / (ms / args.steps * 1e-3) / 1e12}
     cpu, _ = oracle_sample(cfg, inp, min_seconds=args.cpu_seconds)

@@ -118,6 +118,7 @@ typedef struct ta_params {
     float rope_base;       /* 0: none.  > 0 (Llama: 10000): tensorized positional encoding    */
                            /* (Section 3.2), applied inside the kernels -- see ta_forward_ex  */
     const int *window;     /* host, ndims ints, or NULL: per-hop sliding window, see below     */
+    const unsigned char *const *hop_masks; /* host, ndims pointers, or NULL: explicit M_i, see below */
     ta_stream_t stream;
 } ta_params;
 
@@ -143,6 +144,12 @@ typedef struct ta_params {
  * u <= t, i.e. the last w positions up to the query's own); window[i] = 0 or window == NULL:
  * no window.  A query always sees its own position, so no row is empty.  Negative entries
  * are TA_ERR_INVALID_ARG.  ta_backward_ex takes the same array.
+ *
+ * Explicit masks: hop_masks[i] = NULL, or a host matrix of n_i x n_i bytes (row = query position
+ * along dimension i, column = key position, non-zero = visible), the same for every mode-i
+ * vector of the hop, applied on top of `causal` and window[i].  Read during the call.  Supported
+ * for n_i <= 128 (TA_ERR_UNSUPPORTED beyond); a query position left without any visible key is
+ * TA_ERR_INVALID_ARG.  Hops are not fused when a mask is given.  ta_backward_ex takes the same.
  */
 int ta_forward_ex(const ta_params *p);
 
@@ -187,6 +194,7 @@ typedef struct ta_bwd_params {
                                   /* ta_forward_ex (q, k un-rotated; dq, dk are the gradients   */
                                   /* with respect to the un-rotated q, k).  D must be even.     */
     const int *window;            /* host, ndims ints, or NULL: sliding windows as in ta_forward_ex */
+    const unsigned char *const *hop_masks; /* host, ndims pointers, or NULL: explicit masks, as in ta_forward_ex */
     const void *saved_hops;       /* X_1..X_{m-1} as written by ta_forward_ex(TA_FLAG_SAVE_HOPS) */
                                   /* (the part of its workspace after the scratch tensor), or    */
                                   /* NULL: recomputed                                          */

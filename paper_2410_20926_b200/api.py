@@ -46,6 +46,7 @@ class ta_params(ctypes.Structure):
                 ("flags", ctypes.c_uint), ("hop_begin", ctypes.c_int), ("hop_end", ctypes.c_int),
                 ("rope_base", ctypes.c_float),
                 ("window", ctypes.POINTER(ctypes.c_int)),
+                ("hop_masks", ctypes.POINTER(ctypes.c_void_p)),
                 ("stream", ctypes.c_void_p)]
 
 
@@ -60,6 +61,7 @@ class ta_bwd_params(ctypes.Structure):
                 ("causal", ctypes.c_int), ("dtype", ctypes.c_int), ("grad_dtype", ctypes.c_int),
                 ("softmax_scale", ctypes.c_float), ("rope_base", ctypes.c_float),
                 ("window", ctypes.POINTER(ctypes.c_int)),
+                ("hop_masks", ctypes.POINTER(ctypes.c_void_p)),
                 ("saved_hops", ctypes.c_void_p),
                 ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
                 ("stream", ctypes.c_void_p)]
@@ -180,9 +182,35 @@ def _window(window, nd):
     return (ctypes.c_int * nd)(*w)
 
 
+def _hop_masks(hop_masks, dims):
+    """Per-dimension explicit masks M_i as a C array of host pointers (None stays NULL).
+
+    `hop_masks` has one entry per dimension: None (no explicit mask for that hop) or an n_i x n_i
+    array whose non-zero entries mark the visible (query position, key position) pairs.  Returns
+    (pointer array, buffers to keep alive until the call returns).
+    """
+    if hop_masks is None:
+        return None, None
+    import numpy as np
+    dims = [int(x) for x in dims]
+    if len(hop_masks) != len(dims):
+        raise ValueError("hop_masks needs one entry per dimension")
+    keep, arr = [], (ctypes.c_void_p * len(dims))()
+    for i, (m, n) in enumerate(zip(hop_masks, dims)):
+        if m is None:
+            arr[i] = None
+            continue
+        m8 = np.ascontiguousarray((np.asarray(m) != 0).astype(np.uint8))
+        if m8.shape != (n, n):
+            raise ValueError(f"hop_masks[{i}] must have shape ({n}, {n})")
+        keep.append(m8)
+        arr[i] = m8.ctypes.data
+    return arr, keep
+
+
 def ta_forward_ex(q, k, v, out, B, H, H_kv, N, D, dims, causal, dtype=TA_DTYPE_BF16,
                   softmax_scale=0.0, workspace=None, workspace_bytes=0, flags=0, hop_begin=0,
-                  hop_end=0, rope_base=0.0, window=None, stream=None, check=True) -> int:
+                  hop_end=0, rope_base=0.0, window=None, hop_masks=None, stream=None, check=True) -> int:
     d, nd = _dims(dims)
     p = ta_params()
     p.struct_bytes = ctypes.sizeof(ta_params)
@@ -196,6 +224,9 @@ def ta_forward_ex(q, k, v, out, B, H, H_kv, N, D, dims, causal, dtype=TA_DTYPE_B
     win = _window(window, nd)          # kept alive until the call returns
     if win is not None:
         p.window = win
+    masks, _keep = _hop_masks(hop_masks, dims)
+    if masks is not None:
+        p.hop_masks = masks
     p.stream = _stream(stream)
     return _done(load().ta_forward_ex(ctypes.byref(p)), "ta_forward_ex", check)
 
@@ -211,7 +242,8 @@ def ta_backward(dout, q, k, v, out, dq, dk, dv, B, H, H_kv, N, D, dims, causal, 
 
 def ta_backward_ex(dout, q, k, v, dq, dk, dv, B, H, H_kv, N, D, dims, causal,
                    grad_dtype=TA_DTYPE_BF16, softmax_scale=0.0, saved_hops=None, workspace=None,
-                   workspace_bytes=0, rope_base=0.0, window=None, stream=None, check=True) -> int:
+                   workspace_bytes=0, rope_base=0.0, window=None, hop_masks=None, stream=None,
+                   check=True) -> int:
     d, nd = _dims(dims)
     p = ta_bwd_params()
     p.struct_bytes = ctypes.sizeof(ta_bwd_params)
@@ -224,6 +256,9 @@ def ta_backward_ex(dout, q, k, v, dq, dk, dv, B, H, H_kv, N, D, dims, causal,
     win = _window(window, nd)
     if win is not None:
         p.window = win
+    masks, _keep = _hop_masks(hop_masks, dims)
+    if masks is not None:
+        p.hop_masks = masks
     p.saved_hops = _ptr(saved_hops)
     p.workspace, p.workspace_bytes = _ptr(workspace), workspace_bytes
     p.stream = _stream(stream)

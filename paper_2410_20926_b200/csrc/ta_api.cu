@@ -144,6 +144,43 @@ int build_plan(int B, int H, int H_kv, int N, int D, const int *dims, int ndims,
     return TA_OK;
 }
 
+int build_hop_mask(const Problem &pb, const HopDesc &hd, HopMask *hm) {
+    const int n = hd.n;
+    if (n > 128) return TA_ERR_UNSUPPORTED;
+    const unsigned char *m = pb.masks[hd.hop];
+    const int w = pb.window[hd.hop];
+    memset(hm, 0, sizeof(*hm));
+    for (int t = 0; t < n; ++t) {
+        bool any = false;
+        for (int u = 0; u < n; ++u) {
+            if (pb.causal && u > t) continue;
+            if (w > 0 && (t - u >= w || u - t >= w)) continue;
+            if (m && !m[(size_t)t * n + u]) continue;
+            hm->bits[t][u >> 5] |= 1u << (u & 31);
+            any = true;
+        }
+        if (!any) return TA_ERR_INVALID_ARG;
+    }
+    return TA_OK;
+}
+
+int take_masks(Problem *pb, const Plan &plan, const int *window, const unsigned char *const *hop_masks, int ndims) {
+    for (int i = 0; i < TA_MAX_DIMS; ++i) {
+        pb->window[i] = (window && i < ndims) ? window[i] : 0;
+        pb->masks[i] = (hop_masks && i < ndims) ? hop_masks[i] : nullptr;
+        if (pb->window[i] < 0) return TA_ERR_INVALID_ARG;
+    }
+    // every masked hop is checked before anything is launched
+    for (int j = 0; j < plan.nhops; ++j) {
+        const HopDesc &h = plan.hops[j];
+        if (h.nf > 1 || !pb->masks[h.hop]) continue;
+        HopMask hm;
+        const int rc = build_hop_mask(*pb, h, &hm);
+        if (rc != TA_OK) return rc;
+    }
+    return TA_OK;
+}
+
 // ---------------------------------------------------------------------------------------
 // Device scratch / staging arenas owned by the library (grow-only, one per process).
 // ---------------------------------------------------------------------------------------
@@ -250,7 +287,11 @@ static int forward_impl(const ta_params &p) {
     Plan plan;
     // the positional encoding gives every hop its own rotated Q and K: nothing to share, no fusion
     if (p.flags & kPlanFlagRope) return TA_ERR_UNSUPPORTED;
-    const unsigned plan_flags = p.flags | (p.rope_base > 0.f ? (unsigned)TA_FLAG_NO_HOP_FUSION | kPlanFlagRope : 0u);
+    bool any_mask = false;
+    if (p.hop_masks && p.ndims >= 1 && p.ndims <= TA_MAX_DIMS)
+        for (int i = 0; i < p.ndims; ++i) any_mask = any_mask || p.hop_masks[i] != nullptr;
+    const unsigned plan_flags = p.flags | (p.rope_base > 0.f ? (unsigned)TA_FLAG_NO_HOP_FUSION | kPlanFlagRope : 0u) |
+                                (any_mask ? (unsigned)TA_FLAG_NO_HOP_FUSION : 0u);
     int rc = build_plan(p.B, p.H, p.H_kv, p.N, p.D, p.dims, p.ndims, p.dtype, plan_flags, p.hop_begin,
                         p.hop_end, &plan);
     if (rc != TA_OK) return rc;
@@ -269,7 +310,7 @@ static int forward_impl(const ta_params &p) {
     pb.ndims = p.ndims; pb.causal = p.causal ? 1 : 0; pb.dtype = p.dtype;
     pb.scale = p.softmax_scale != 0.f ? p.softmax_scale : 1.0f / sqrtf((float)p.D);
     pb.rope_base = p.rope_base;
-    for (int i = 0; i < TA_MAX_DIMS; ++i) pb.window[i] = (p.window && i < p.ndims) ? p.window[i] : 0;
+    if ((rc = take_masks(&pb, plan, p.window, p.hop_masks, p.ndims)) != TA_OK) return rc;
     pb.flags = p.flags; pb.hop_begin = p.hop_begin; pb.hop_end = p.hop_end;
     pb.stream = (cudaStream_t)p.stream;
 

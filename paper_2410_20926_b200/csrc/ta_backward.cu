@@ -81,7 +81,8 @@ int backward_impl(const ta_bwd_params &p) {
     pb.ndims = p.ndims; pb.causal = p.causal ? 1 : 0; pb.dtype = p.dtype;
     pb.scale = p.softmax_scale != 0.f ? p.softmax_scale : 1.0f / sqrtf((float)p.D);
     pb.rope_base = p.rope_base;
-    for (int i = 0; i < TA_MAX_DIMS; ++i) pb.window[i] = (p.window && i < p.ndims) ? p.window[i] : 0;
+    pb.causal = p.causal ? 1 : 0;
+    if ((rc = take_masks(&pb, plan, p.window, p.hop_masks, p.ndims)) != TA_OK) return rc;
     pb.flags = 0; pb.hop_begin = 0; pb.hop_end = p.ndims;
     pb.stream = (cudaStream_t)p.stream;
 

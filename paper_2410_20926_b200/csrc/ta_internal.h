@@ -62,6 +62,7 @@ struct Problem {
     float scale;  // already resolved (1/sqrt(D) default)
     float rope_base;  // 0 = no positional encoding
     int window[TA_MAX_DIMS];  // per dimension: 0 = none, w > 0 = keys within w positions of the query
+    const unsigned char *masks[TA_MAX_DIMS];  // per dimension: NULL or host n x n bytes, non-zero = visible
     unsigned flags;
     int hop_begin, hop_end;
     cudaStream_t stream;
@@ -73,6 +74,17 @@ static inline size_t elem_bytes(int dtype) { return dtype == TA_DTYPE_F32 ? 4 : 
 int validate_shape(int B, int H, int H_kv, int N, int D, const int *dims, int ndims, int dtype);
 int build_plan(int B, int H, int H_kv, int N, int D, const int *dims, int ndims, int dtype,
                unsigned flags, int hop_begin, int hop_end, Plan *plan);
+
+// Visibility of key position u from query position t along a hop's dimension (bit u of row t;
+// n <= 128): the explicit mask of the dimension combined with the causal flag and the window.
+// Passed to the kernels by value (kernel parameter space).
+struct HopMask {
+    uint32_t bits[128][4];
+};
+// Host: fills hm for hop `hd`; TA_ERR_UNSUPPORTED if n > 128, TA_ERR_INVALID_ARG if a row is empty.
+int build_hop_mask(const Problem &pb, const HopDesc &hd, HopMask *hm);
+// Host: sets pb.window / pb.masks from the caller's arrays and checks them against the plan.
+int take_masks(Problem *pb, const Plan &plan, const int *window, const unsigned char *const *hop_masks, int ndims);
 
 // Kernel launchers (each returns TA_OK or TA_ERR_CUDA).  xin has `xin_heads` heads per batch
 // (H_kv when reading v, H otherwise); xout always has H heads.

@@ -10,6 +10,8 @@
 // tolerance) and of hops the tcgen05 kernel does not cover.
 #include <cuda_bf16.h>
 
+#include <string.h>
+
 #include "ta_internal.h"
 
 namespace ta {
@@ -30,6 +32,7 @@ struct SimtArgs {
     float scale;
     float rope_log2_base;         // 0: no positional encoding; else log2 of the RoPE base
     int window;                   // 0, or sliding window along the hop's dimension
+    int masked;                   // 1: visibility comes from the HopMask parameter (n <= 128)
 };
 
 // Tensorized positional encoding (Section 3.2): rows of `x` ([rows][ld] fp32 in shared memory)
@@ -69,7 +72,7 @@ __device__ __forceinline__ float warp_sum(float x) {
 template <typename T, int DPL>  // DPL = columns per lane, D <= 32 * DPL
 __global__ void __launch_bounds__(kThreads)
 hop_simt_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__restrict__ xin,
-                T *__restrict__ xout, SimtArgs a) {
+                T *__restrict__ xout, SimtArgs a, const __grid_constant__ HopMask hop_mask) {
     extern __shared__ float smem[];
     const int D = a.D, ldk = D + 1;
     float *sQ = smem;                 // [BQ][D]
@@ -142,8 +145,9 @@ hop_simt_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__res
                 float s = 0.f;
                 for (int c = 0; c < D; ++c) s = fmaf(qr[c], kr[c], s);
                 s *= a.scale;
-                const bool valid = key < a.n && (!a.causal || key <= t) &&
-                                   (a.window == 0 || (key > t - a.window && key < t + a.window));
+                bool valid = key < a.n && (!a.causal || key <= t) &&
+                             (a.window == 0 || (key > t - a.window && key < t + a.window));
+                if (a.masked) valid = valid && ((hop_mask.bits[t][key >> 5] >> (key & 31)) & 1u);
                 s = valid ? s : -INFINITY;
                 // a block may hold no visible key of this row (window): keep the arithmetic finite
                 const float m_new = fmaxf(m[r], warp_max(s));
@@ -201,6 +205,15 @@ int launch_t(const Problem &pb, const HopDesc &hd, const void *xin, int xin_head
     a.scale = pb.scale;
     a.rope_log2_base = pb.rope_base > 0.f ? log2f(pb.rope_base) : 0.f;
     a.window = pb.window[hd.hop];
+    a.masked = 0;
+    HopMask hm;
+    if (pb.masks[hd.hop]) {
+        const int rc = build_hop_mask(pb, hd, &hm);   // explicit mask ^ causal flag ^ window
+        if (rc != TA_OK) return rc;
+        a.masked = 1;
+    } else {
+        memset(&hm, 0, sizeof(hm));
+    }
     size_t smem = sizeof(float) * ((size_t)BQ * pb.D + 2 * (size_t)BK * (pb.D + 1));
     auto kern = hop_simt_kernel<T, DPL>;
     if (smem > 48 * 1024) {
@@ -209,7 +222,7 @@ int launch_t(const Problem &pb, const HopDesc &hd, const void *xin, int xin_head
     }
     long long grid = a.items < (1ll << 20) ? a.items : (1ll << 20);
     kern<<<(unsigned)grid, kThreads, smem, pb.stream>>>((const T *)pb.q, (const T *)pb.k, (const T *)xin,
-                                                       (T *)xout, a);
+                                                       (T *)xout, a, hm);
     count_launch();
     return cudaPeekAtLastError() == cudaSuccess ? TA_OK : TA_ERR_CUDA;
 }

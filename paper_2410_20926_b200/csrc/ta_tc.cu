@@ -35,6 +35,7 @@
 #include "ta_internal.h"
 #include "ta_ptx.cuh"
 #include "ta_rope.cuh"
+#include "ta_mask.cuh"
 
 namespace ta {
 
@@ -89,11 +90,11 @@ __device__ __forceinline__ ItemCoord decode_item(const TcArgs &a, long long item
 }
 
 // ----------------------------------------------------------------------------- the kernel
-template <int D, bool kRope>
+template <int D, bool kRope, bool kMask>
 __global__ void __launch_bounds__(kRope ? kThreadsRope : kThreads, 1)
 hop_pipe_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                 const __grid_constant__ CUtensorMap map_xin, const __grid_constant__ CUtensorMap map_xout,
-                const TcArgs a) {
+                const TcArgs a, const __grid_constant__ typename MaskArg<kMask>::type hop_mask) {
     using C = PipeCfg<D>;
     constexpr int kHalves = C::kHalves;
     constexpr uint32_t kSlabBytes = C::kSlabBytes, kTileBytes = C::kTileBytes;
@@ -322,6 +323,11 @@ hop_pipe_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         const int w_lo = ((wq * 32) / a.n) * a.n;
         int w_hi = min(a.rows, ((wq * 32 + 31) / a.n + 1) * a.n);
         if (a.causal) w_hi = min(w_hi, wq * 32 + 32);
+        // explicit mask (already combined with the causal flag and the window): this row's bits
+        // over the tile's key columns
+        uint32_t mrow[4];
+        tile_row_mask(hop_mask, row_valid ? r % a.n : 0, seg * a.n, mrow);
+        if (kMask && !row_valid) mrow[0] = mrow[1] = mrow[2] = mrow[3] = 0u;
         const bool warp_valid = wq * 32 < a.rows;
         const int nchunks = (a.rows + 31) >> 5;         // 32-column chunks of P the MMA reads
         const uint32_t s_col = tmem_lane + C::kColS + b * 128, o_col = tmem_lane + C::kColO + b * 128;
@@ -346,7 +352,8 @@ hop_pipe_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 for (int jj = 0; jj < 32; ++jj) {
                     const int col = 32 * c + jj;
                     const float s = __uint_as_float(v[jj]);
-                    if (col >= c_lo && col < c_hi) m = fmaxf(m, s);
+                    const bool vis = kMask ? ((mask_chunk(mrow, c) >> jj) & 1u) != 0 : (col >= c_lo && col < c_hi);
+                    if (vis) m = fmaxf(m, s);
                 }
             }
             const float m_scaled = row_valid ? m * a.scale_log2 : 0.f;
@@ -361,8 +368,14 @@ hop_pipe_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                         const int col = 32 * c + jj;
                         float p0 = fast_exp2(__uint_as_float(v[jj]) * a.scale_log2 - m_scaled);
                         float p1 = fast_exp2(__uint_as_float(v[jj + 1]) * a.scale_log2 - m_scaled);
-                        p0 = (row_valid && col >= c_lo && col < c_hi) ? p0 : 0.f;
-                        p1 = (row_valid && col + 1 >= c_lo && col + 1 < c_hi) ? p1 : 0.f;
+                        if (kMask) {
+                            const uint32_t bits = mask_chunk(mrow, c);
+                            p0 = ((bits >> jj) & 1u) ? p0 : 0.f;
+                            p1 = ((bits >> (jj + 1)) & 1u) ? p1 : 0.f;
+                        } else {
+                            p0 = (row_valid && col >= c_lo && col < c_hi) ? p0 : 0.f;
+                            p1 = (row_valid && col + 1 >= c_lo && col + 1 < c_hi) ? p1 : 0.f;
+                        }
                         const uint32_t w = pack_bf16x2(p0, p1);
                         pk[jj >> 1] = w;
                         sum += __uint_as_float(w << 16) + __uint_as_float(w & 0xFFFF0000u);
@@ -500,17 +513,27 @@ int launch_d(const Problem &pb, const HopDesc &hd, const void *xin, int xin_head
     const unsigned grid = (unsigned)(a.total_items < num_sms ? a.total_items : num_sms);
     static bool configured = false;
     if (!configured) {
-        if (cudaFuncSetAttribute(hop_pipe_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
-                cudaSuccess ||
-            cudaFuncSetAttribute(hop_pipe_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
-                cudaSuccess)
+        const cudaFuncAttribute attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
+        if (cudaFuncSetAttribute(hop_pipe_kernel<D, false, false>, attr, (int)smem) != cudaSuccess ||
+            cudaFuncSetAttribute(hop_pipe_kernel<D, true, false>, attr, (int)smem) != cudaSuccess ||
+            cudaFuncSetAttribute(hop_pipe_kernel<D, false, true>, attr, (int)smem) != cudaSuccess ||
+            cudaFuncSetAttribute(hop_pipe_kernel<D, true, true>, attr, (int)smem) != cudaSuccess)
             return TA_ERR_CUDA;
         configured = true;
     }
-    if (pb.rope_base > 0.f)
-        hop_pipe_kernel<D, true><<<grid, kThreadsRope, smem, pb.stream>>>(mq, mk, mxi, mxo, a);
-    else
-        hop_pipe_kernel<D, false><<<grid, kThreads, smem, pb.stream>>>(mq, mk, mxi, mxo, a);
+    if (pb.masks[hd.hop]) {
+        HopMask hm;                                  // explicit mask ^ causal flag ^ window, by value
+        const int rc = build_hop_mask(pb, hd, &hm);
+        if (rc != TA_OK) return rc;
+        if (pb.rope_base > 0.f)
+            hop_pipe_kernel<D, true, true><<<grid, kThreadsRope, smem, pb.stream>>>(mq, mk, mxi, mxo, a, hm);
+        else
+            hop_pipe_kernel<D, false, true><<<grid, kThreads, smem, pb.stream>>>(mq, mk, mxi, mxo, a, hm);
+    } else if (pb.rope_base > 0.f) {
+        hop_pipe_kernel<D, true, false><<<grid, kThreadsRope, smem, pb.stream>>>(mq, mk, mxi, mxo, a, NoMask{});
+    } else {
+        hop_pipe_kernel<D, false, false><<<grid, kThreads, smem, pb.stream>>>(mq, mk, mxi, mxo, a, NoMask{});
+    }
     count_launch();
     return cudaPeekAtLastError() == cudaSuccess ? TA_OK : TA_ERR_CUDA;
 }

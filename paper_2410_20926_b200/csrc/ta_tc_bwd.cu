@@ -32,6 +32,7 @@
 #include "ta_internal.h"
 #include "ta_ptx.cuh"
 #include "ta_rope.cuh"
+#include "ta_mask.cuh"
 
 namespace ta {
 namespace {
@@ -94,13 +95,13 @@ __device__ __forceinline__ bool wg_all(bool pred) {
 }
 __device__ __forceinline__ void wg_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
-template <int D, bool kRope>
+template <int D, bool kRope, bool kMask>
 __global__ void __launch_bounds__(kRope ? kThreadsRope : kThreads, 1)
 hop_tc_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                   const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_gin,
                   const __grid_constant__ CUtensorMap map_gout, const __grid_constant__ CUtensorMap map_dq,
                   const __grid_constant__ CUtensorMap map_dk, const __grid_constant__ CUtensorMap map_dv,
-                  const BwdArgs a) {
+                  const BwdArgs a, const __grid_constant__ typename MaskArg<kMask>::type hop_mask) {
     using C = BwdCfg<D>;
     constexpr int kHalves = C::kHalves;
     constexpr uint32_t kSlabBytes = C::kSlabBytes, kTileBytes = C::kTileBytes, kStageBytes = C::kStageBytes;
@@ -245,6 +246,16 @@ hop_tc_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         int w_hi = min(a.rows, ((warp * 32 + 31) / a.n + 1) * a.n);
         if (a.causal) w_hi = min(w_hi, warp * 32 + 32);
         const bool warp_valid = warp * 32 < a.rows;
+        // explicit mask (already combined with the causal flag and the window): this row's bits
+        // over the tile's key columns
+        uint32_t mrow[4];
+        tile_row_mask(hop_mask, row_valid ? r % a.n : 0, seg * a.n, mrow);
+        if (kMask && !row_valid) mrow[0] = mrow[1] = mrow[2] = mrow[3] = 0u;
+        auto visible = [&](int cc, int jj) -> bool {
+            if (kMask) return ((mask_chunk(mrow, cc) >> jj) & 1u) != 0;
+            const int col = 32 * cc + jj;
+            return row_valid && col >= c_lo && col < c_hi;
+        };
         const int kblocks = (a.rows + 15) >> 4;
 
         // fp32 accumulator columns -> shared staging in the layout of the fp32 maps (32-column slabs)
@@ -356,8 +367,7 @@ hop_tc_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                         tmem_ld32(tmem_lane + C::kColS + 32 * cc, vs);
 #pragma unroll
                         for (int jj = 0; jj < 32; ++jj) {
-                            const int col = 32 * cc + jj;
-                            if (col >= c_lo && col < c_hi) m = fmaxf(m, __uint_as_float(vs[jj]));
+                            if (visible(cc, jj)) m = fmaxf(m, __uint_as_float(vs[jj]));
                         }
                     }
                     const float m_s = row_valid ? m * a.scale_log2 : 0.f;
@@ -369,9 +379,8 @@ hop_tc_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                         tmem_ld32(tmem_lane + C::kColDP + 32 * cc, vd);
 #pragma unroll
                         for (int jj = 0; jj < 32; ++jj) {
-                            const int col = 32 * cc + jj;
                             float p = fast_exp2(__uint_as_float(vs[jj]) * a.scale_log2 - m_s);
-                            const bool vis = row_valid && col >= c_lo && col < c_hi;
+                            const bool vis = visible(cc, jj);
                             p = vis ? p : 0.f;
                             l += p;
                             dot += vis ? p * __uint_as_float(vd[jj]) : 0.f;
@@ -391,8 +400,7 @@ hop_tc_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                                 float pv[2], dv[2];
 #pragma unroll
                                 for (int e = 0; e < 2; ++e) {
-                                    const int col = 32 * cc + jj + e;
-                                    const bool vis = row_valid && col >= c_lo && col < c_hi;
+                                    const bool vis = visible(cc, jj + e);
                                     float p = fast_exp2(__uint_as_float(vs[jj + e]) * a.scale_log2 - m_s) * inv_l;
                                     p = vis ? p : 0.f;
                                     pv[e] = p;
@@ -605,18 +613,28 @@ int launch_bwd_d(const Problem &pb, const HopDesc &hd, const void *x, int x_head
     constexpr size_t smem = BwdCfg<D>::kSmemBytes;
     static bool configured = false;
     if (!configured) {
-        if (cudaFuncSetAttribute(hop_tc_bwd_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
-                cudaSuccess ||
-            cudaFuncSetAttribute(hop_tc_bwd_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
-                cudaSuccess)
+        const cudaFuncAttribute attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
+        if (cudaFuncSetAttribute(hop_tc_bwd_kernel<D, false, false>, attr, (int)smem) != cudaSuccess ||
+            cudaFuncSetAttribute(hop_tc_bwd_kernel<D, true, false>, attr, (int)smem) != cudaSuccess ||
+            cudaFuncSetAttribute(hop_tc_bwd_kernel<D, false, true>, attr, (int)smem) != cudaSuccess ||
+            cudaFuncSetAttribute(hop_tc_bwd_kernel<D, true, true>, attr, (int)smem) != cudaSuccess)
             return TA_ERR_CUDA;
         configured = true;
     }
     const unsigned grid = (unsigned)(a.total_items < num_sms ? a.total_items : num_sms);
-    if (pb.rope_base > 0.f)
-        hop_tc_bwd_kernel<D, true><<<grid, kThreadsRope, smem, pb.stream>>>(mq, mk, mx, mgi, mgo, mdq, mdk, mdv, a);
-    else
-        hop_tc_bwd_kernel<D, false><<<grid, kThreads, smem, pb.stream>>>(mq, mk, mx, mgi, mgo, mdq, mdk, mdv, a);
+    if (pb.masks[hd.hop]) {
+        HopMask hm;                                  // explicit mask ^ causal flag ^ window, by value
+        const int rc = build_hop_mask(pb, hd, &hm);
+        if (rc != TA_OK) return rc;
+        if (pb.rope_base > 0.f)
+            hop_tc_bwd_kernel<D, true, true><<<grid, kThreadsRope, smem, pb.stream>>>(mq, mk, mx, mgi, mgo, mdq, mdk, mdv, a, hm);
+        else
+            hop_tc_bwd_kernel<D, false, true><<<grid, kThreads, smem, pb.stream>>>(mq, mk, mx, mgi, mgo, mdq, mdk, mdv, a, hm);
+    } else if (pb.rope_base > 0.f) {
+        hop_tc_bwd_kernel<D, true, false><<<grid, kThreadsRope, smem, pb.stream>>>(mq, mk, mx, mgi, mgo, mdq, mdk, mdv, a, NoMask{});
+    } else {
+        hop_tc_bwd_kernel<D, false, false><<<grid, kThreads, smem, pb.stream>>>(mq, mk, mx, mgi, mgo, mdq, mdk, mdv, a, NoMask{});
+    }
     count_launch();
     return cudaPeekAtLastError() == cudaSuccess ? TA_OK : TA_ERR_CUDA;
 }

@@ -1,0 +1,147 @@
+"""GPU parity of explicit per-hop masks M_i (Eq. 3 of the paper allows any sparsity mask in a
+hop; here hop i takes an n_i x n_i matrix of visible (query position, key position) pairs, the
+same for every segment, batch and head) against the fp64 oracle: forward on the tensor-core and
+generic kernels, with the causal flag, a window and the positional encoding on top, the backward,
+and the argument checks.  Tolerances as for the unmasked operator."""
+import math
+
+import numpy as np
+import pytest
+
+import oracle
+import paper_2410_20926_b200 as ta
+from paper_2410_20926_b200 import inputs as ta_inputs
+
+from helpers import assert_close, gpu_forward
+from test_gpu_backward import assert_grad_close, gpu_backward
+
+pytestmark = pytest.mark.gpu
+
+
+def random_masks(dims, seed, density=0.5, skip=()):
+    """One random 0/1 matrix per dimension with the diagonal set (so that no row is empty, with or
+    without the causal flag); dimensions listed in `skip` get no mask."""
+    rng = np.random.default_rng(seed)
+    out = []
+    for i, n in enumerate(dims):
+        if i in skip:
+            out.append(None)
+            continue
+        m = (rng.random((n, n)) < density).astype(np.uint8)
+        m[np.arange(n), np.arange(n)] = 1
+        out.append(m)
+    return out
+
+
+def run(B, H, Hkv, D, dims, masks, causal, dtype, seed, flags=0, expect=None, **kw):
+    N = math.prod(dims)
+    if expect is not None:
+        # masked calls are planned without hop fusion
+        assert expect in ta.ta_plan_describe(B, H, Hkv, N, D, dims, causal,
+                                             ta.TA_DTYPE_BF16 if dtype == "bf16" else ta.TA_DTYPE_F32,
+                                             flags | ta.TA_FLAG_NO_HOP_FUSION)
+    inp = ta_inputs.make_inputs(B, H, Hkv, N, D, dtype, seed)
+    got = gpu_forward(inp, B, H, Hkv, N, D, dims, causal, dtype, flags, hop_masks=masks, **kw)
+    okw = {"window": kw.get("window"), "rope_base": kw.get("rope_base") or None}
+    ref = oracle.forward(inp["q"], inp["k"], inp["v"], dims, causal, masks=masks, **okw)
+    assert_close(got, ref, dtype)
+    plain = oracle.forward(inp["q"], inp["k"], inp["v"], dims, causal, **okw)
+    assert np.abs(ref - plain).max() > 0.05          # the masks change the result visibly
+    return got
+
+
+@pytest.mark.parametrize("dims,D,causal,skip", [
+    ([4, 64], 128, True, ()),
+    ([64, 64], 128, False, (0,)),
+    ([32, 8, 32], 128, True, (1,)),
+    ([5, 24, 7], 64, False, ()),           # several segments per tile, ragged tiles
+    ([128], 128, False, ()),
+    ([3, 100], 64, True, ()),
+    ([8, 8, 8], 64, False, ()),            # would be fused without masks
+])
+def test_masks_tensor_core_kernel(dims, D, causal, skip):
+    run(2, 4, 2, D, dims, random_masks(dims, 11, skip=skip), causal, "bf16", 701, expect="tc")
+
+
+def test_masks_with_window_and_positional_encoding():
+    dims = [8, 64]
+    run(1, 4, 2, 128, dims, random_masks(dims, 12), True, "bf16", 702, window=[3, 20])
+    run(1, 4, 2, 128, dims, random_masks(dims, 13), True, "bf16", 703, rope_base=10000.0)
+    run(1, 4, 2, 64, dims, random_masks(dims, 14), False, "bf16", 704, rope_base=10000.0, window=[0, 40])
+
+
+def test_masks_generic_kernel():
+    run(2, 4, 2, 40, [3, 5, 7], random_masks([3, 5, 7], 15), True, "f32", 705)
+    run(1, 4, 2, 64, [6, 100], random_masks([6, 100], 16), False, "f32", 706)
+    run(1, 2, 1, 64, [16, 16], random_masks([16, 16], 17), True, "bf16", 707, flags=ta.TA_FLAG_NO_TENSOR_CORE)
+
+
+def test_triangular_and_band_masks_reproduce_the_flag_and_the_window():
+    """A lower-triangular matrix is the causal flag, a band matrix is the window: the masked
+    kernels must then give what the unmasked ones give (same products, same sums)."""
+    B, H, Hkv, D, dims = 1, 4, 2, 128, [16, 64]
+    N = math.prod(dims)
+    inp = ta_inputs.make_inputs(B, H, Hkv, N, D, "bf16", 708)
+    tri = [np.tril(np.ones((n, n), np.uint8)) for n in dims]
+    a = gpu_forward(inp, B, H, Hkv, N, D, dims, False, "bf16", ta.TA_FLAG_NO_HOP_FUSION, hop_masks=tri)
+    b = gpu_forward(inp, B, H, Hkv, N, D, dims, True, "bf16", ta.TA_FLAG_NO_HOP_FUSION)
+    np.testing.assert_array_equal(a, b)
+    w = [5, 9]
+    band = [(np.abs(np.subtract.outer(np.arange(n), np.arange(n))) < wi).astype(np.uint8) for n, wi in zip(dims, w)]
+    a = gpu_forward(inp, B, H, Hkv, N, D, dims, True, "bf16", ta.TA_FLAG_NO_HOP_FUSION, hop_masks=band)
+    b = gpu_forward(inp, B, H, Hkv, N, D, dims, True, "bf16", ta.TA_FLAG_NO_HOP_FUSION, window=w)
+    np.testing.assert_array_equal(a, b)
+
+
+def test_mask_argument_checks():
+    import torch
+    x = torch.zeros(1, 2, 64, 64, dtype=torch.bfloat16, device="cuda")
+    out = torch.empty_like(x)
+    empty_row = np.ones((8, 8), np.uint8)
+    empty_row[3, :] = 0
+    rc = ta.ta_forward_ex(x, x, x, out, 1, 2, 2, 64, 64, [8, 8], False, hop_masks=[None, empty_row], check=False)
+    assert rc == ta.TA_ERR_INVALID_ARG
+    # a row whose only visible keys lie after the query is empty once the causal flag is applied
+    upper = np.triu(np.ones((8, 8), np.uint8), 1)
+    upper[7, 7] = 1
+    rc = ta.ta_forward_ex(x, x, x, out, 1, 2, 2, 64, 64, [8, 8], True, hop_masks=[upper, None], check=False)
+    assert rc == ta.TA_ERR_INVALID_ARG
+    rc = ta.ta_forward_ex(x, x, x, out, 1, 2, 2, 64, 64, [8, 8], False, hop_masks=[upper, None], check=False)
+    assert rc == ta.TA_OK
+    # explicit masks are limited to segments of at most 128 positions
+    y = torch.zeros(1, 2, 256, 64, dtype=torch.bfloat16, device="cuda")
+    rc = ta.ta_forward_ex(y, y, y, torch.empty_like(y), 1, 2, 2, 256, 64, [256], True,
+                          hop_masks=[np.tril(np.ones((256, 256), np.uint8))], check=False)
+    assert rc == ta.TA_ERR_UNSUPPORTED
+    with pytest.raises(ValueError):
+        ta.ta_forward_ex(x, x, x, out, 1, 2, 2, 64, 64, [8, 8], False, hop_masks=[np.ones((4, 4))])
+
+
+@pytest.mark.parametrize("dims,D,causal,skip,rope", [
+    ([8, 16, 32], 128, True, (1,), 0.0),
+    ([16, 16], 64, False, (), 0.0),
+    ([128], 128, True, (), 0.0),
+    ([5, 24], 64, False, (), 0.0),
+    ([8, 64], 128, True, (), 10000.0),
+])
+def test_backward_with_masks(dims, D, causal, skip, rope):
+    B, H, Hkv = 1, 4, 2
+    N = math.prod(dims)
+    masks = random_masks(dims, 18, skip=skip)
+    inp = ta_inputs.make_inputs(B, H, Hkv, N, D, "bf16", 709, with_dout=True)
+    got = gpu_backward(inp, B, H, Hkv, N, D, dims, causal, True, hop_masks=masks, rope_base=rope)
+    ref = oracle.backward(inp["dout"], inp["q"], inp["k"], inp["v"], dims, causal, masks=masks,
+                          rope_base=rope or None)
+    for name, g, r in zip(("dq", "dk", "dv"), got, ref):
+        assert_grad_close(g, r, name)
+
+
+def test_masks_llama_shape_sampled_heads():
+    """32 768 tokens as 32x32x32, H=32, H_kv=8, D=128, causal, with a random mask on every hop."""
+    c = ta_inputs.CONFIGS[3]
+    masks = random_masks(list(c.dims), 19)
+    inp = ta_inputs.make_config_inputs(c)
+    got = gpu_forward(inp, c.B, c.H, c.H_kv, c.N, c.D, list(c.dims), True, "bf16", hop_masks=masks)
+    heads = [(0, 5), (0, 30)]
+    ref = oracle.forward(inp["q"], inp["k"], inp["v"], list(c.dims), True, masks=masks, heads=heads)
+    assert_close(np.stack([got[b, h] for b, h in heads]), ref, "bf16")
