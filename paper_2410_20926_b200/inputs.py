@@ -88,3 +88,25 @@ def make_inputs(B, H, H_kv, N, D, dtype: str, seed: int, with_dout: bool = False
 
 def make_config_inputs(cfg: Config) -> dict:
     return make_inputs(cfg.B, cfg.H, cfg.H_kv, cfg.N, cfg.D, cfg.dtype, cfg.seed, cfg.backward)
+
+
+def make_device_inputs(B, H, H_kv, N, D, seed: int, device="cuda"):
+    """bf16 q [B,H,N,D], k, v [B,H_kv,N,D] ~ N(0,1) drawn on the device, one batch entry at a
+    time (for tensors too large to draw on the host).  Recipe: ``torch.Generator(device)`` seeded
+    with `seed`; per batch entry ``randn`` of q, then k, then v in float32, rounded to bf16."""
+    import torch
+    gen = torch.Generator(device=device).manual_seed(seed)
+    q = torch.empty(B, H, N, D, dtype=torch.bfloat16, device=device)
+    k = torch.empty(B, H_kv, N, D, dtype=torch.bfloat16, device=device)
+    v = torch.empty(B, H_kv, N, D, dtype=torch.bfloat16, device=device)
+    for b in range(B):
+        for t, heads in ((q, H), (k, H_kv), (v, H_kv)):
+            for h0 in range(0, heads, 8):
+                h1 = min(heads, h0 + 8)
+                t[b, h0:h1] = torch.randn(h1 - h0, N, D, device=device, generator=gen).bfloat16()
+    return q, k, v
+
+
+def head_to_host(t, b: int, h: int) -> np.ndarray:
+    """One head of a device tensor as a float64 array [1,1,N,D] (exact: bf16 -> fp64)."""
+    return t[b, h].float().cpu().numpy().astype(np.float64)[None, None]
