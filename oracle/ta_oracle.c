@@ -44,6 +44,11 @@
  * fully masked.  Hop i may also carry an explicit n_i x n_i mask (row = query position, column
  * = key position, non-zero = visible), applied on top of the causal flag and the window; a row
  * left without any visible key is an error.
+ *
+ * Valid length (padding; M_i of Eq. 3 may depend on the segment): with len < N only the tokens
+ * with flat index < len exist.  A padding token is never visible as a key; a padding query has
+ * an all-zero row of weights, so its output row is 0 and nothing flows back through it (its rows
+ * of dq, dk, dv are 0 and its row of dout is ignored).  len = N means no padding.
  */
 #include <math.h>
 #include <stdlib.h>
@@ -66,14 +71,19 @@ static int visible(int t, int u, int causal, int window, const unsigned char *ma
  * removes have weight exactly 0.  Returns -1 if a row has no visible key. */
 static int segment_weights(const double *Q, const double *K, long base, long stride,
                            int n, int D, double scale, int causal, int window,
-                           const unsigned char *mask, double *P)
+                           const unsigned char *mask, long len, double *P)
 {
     for (int t = 0; t < n; ++t) {
         const double *qt = Q + (base + (long)t * stride) * D;
         double mx = -INFINITY;
         int any = 0;
+        if (base + (long)t * stride >= len) {               /* padding query: no weights at all */
+            for (int u = 0; u < n; ++u) P[t * n + u] = 0.0;
+            continue;
+        }
         for (int u = 0; u < n; ++u) {
-            if (!visible(t, u, causal, window, mask, n)) { P[t * n + u] = 0.0; continue; }
+            if (base + (long)u * stride >= len ||           /* padding key */
+                !visible(t, u, causal, window, mask, n)) { P[t * n + u] = 0.0; continue; }
             const double *ku = K + (base + (long)u * stride) * D;
             double s = 0.0;
             for (int c = 0; c < D; ++c) s += qt[c] * ku[c];
@@ -85,7 +95,7 @@ static int segment_weights(const double *Q, const double *K, long base, long str
         if (!any) return -1;
         double den = 0.0;
         for (int u = 0; u < n; ++u) {
-            if (!visible(t, u, causal, window, mask, n)) continue;
+            if (base + (long)u * stride >= len || !visible(t, u, causal, window, mask, n)) continue;
             double e = exp(P[t * n + u] - mx);
             P[t * n + u] = e;
             den += e;
@@ -133,9 +143,10 @@ static void rope_rotate(const double *x, double *y, long N, int D, long stride, 
 static int forward_head_impl(const double *q, const double *k, const double *v, double *out,
                              long N, int D, const int *dims, int ndims, int causal,
                              double scale, double rope_base, const int *window,
-                             const unsigned char *const *masks, double *xs)
+                             const unsigned char *const *masks, long len, double *xs)
 {
     if (!q || !k || !v || !out || !dims || ndims < 1 || N < 1 || D < 1) return -1;
+    if (len < 0 || len > N) return -1;
     long prod = 1;
     for (int i = 0; i < ndims; ++i) { if (dims[i] < 1) return -1; prod *= dims[i]; }
     if (prod != N) return -1;
@@ -175,7 +186,7 @@ static int forward_head_impl(const double *q, const double *k, const double *v, 
                 long outer = g / s, inner = g % s;
                 long base = outer * n * s + inner;
                 if (segment_weights(q, k, base, s, n, D, scale, causal, window ? window[i] : 0,
-                                    masks ? masks[i] : NULL, P) != 0) {                 /* A_i */
+                                    masks ? masks[i] : NULL, len, P) != 0) {            /* A_i */
                     #pragma omp atomic write
                     fail = 1;
                     continue;
@@ -206,7 +217,7 @@ int ta_oracle_forward_head(const double *q, const double *k, const double *v, do
                            long N, int D, const int *dims, int ndims, int causal,
                            double scale, double *xs)
 {
-    return forward_head_impl(q, k, v, out, N, D, dims, ndims, causal, scale, 0.0, NULL, NULL, xs);
+    return forward_head_impl(q, k, v, out, N, D, dims, ndims, causal, scale, 0.0, NULL, NULL, N, xs);
 }
 
 /* As above with the tensorized positional encoding (rope_base > 0, e.g. 10000). */
@@ -215,7 +226,7 @@ int ta_oracle_forward_head_rope(const double *q, const double *k, const double *
                                 double scale, double rope_base, double *xs)
 {
     if (!(rope_base > 0.0)) return -1;
-    return forward_head_impl(q, k, v, out, N, D, dims, ndims, causal, scale, rope_base, NULL, NULL, xs);
+    return forward_head_impl(q, k, v, out, N, D, dims, ndims, causal, scale, rope_base, NULL, NULL, N, xs);
 }
 
 /* Every option: rope_base 0 = none; window NULL or [ndims] ints, 0 = no window in that hop;
@@ -227,7 +238,18 @@ int ta_oracle_forward_head_ex(const double *q, const double *k, const double *v,
 {
     if (rope_base < 0.0) return -1;
     if (window) for (int i = 0; i < ndims; ++i) if (window[i] < 0) return -1;
-    return forward_head_impl(q, k, v, out, N, D, dims, ndims, causal, scale, rope_base, window, masks, xs);
+    return forward_head_impl(q, k, v, out, N, D, dims, ndims, causal, scale, rope_base, window, masks, N, xs);
+}
+
+/* As ta_oracle_forward_head_ex with a valid length: tokens with flat index >= len are padding. */
+int ta_oracle_forward_head_len(const double *q, const double *k, const double *v, double *out,
+                               long N, int D, const int *dims, int ndims, int causal,
+                               double scale, double rope_base, const int *window,
+                               const unsigned char *const *masks, long len, double *xs)
+{
+    if (rope_base < 0.0) return -1;
+    if (window) for (int i = 0; i < ndims; ++i) if (window[i] < 0) return -1;
+    return forward_head_impl(q, k, v, out, N, D, dims, ndims, causal, scale, rope_base, window, masks, len, xs);
 }
 
 /*
@@ -248,9 +270,10 @@ static int backward_head_impl(const double *q, const double *k, const double *xs
                               const double *dout, double *dq, double *dk, double *dv,
                               long N, int D, const int *dims, int ndims, int causal,
                               double scale, double rope_base, const int *window,
-                              const unsigned char *const *masks)
+                              const unsigned char *const *masks, long len)
 {
     if (!q || !k || !xs || !dout || !dq || !dk || !dv || !dims || ndims < 1) return -1;
+    if (len < 0 || len > N) return -1;
     long prod = 1;
     for (int i = 0; i < ndims; ++i) { if (dims[i] < 1) return -1; prod *= dims[i]; }
     if (prod != N) return -1;
@@ -301,7 +324,7 @@ static int backward_head_impl(const double *q, const double *k, const double *xs
                 long outer = sg / s, inner = sg % s;
                 long base = outer * n * s + inner;
                 if (segment_weights(q, k, base, s, n, D, scale, causal, window ? window[i] : 0,
-                                    masks ? masks[i] : NULL, P) != 0) {
+                                    masks ? masks[i] : NULL, len, P) != 0) {
                     #pragma omp atomic write
                     fail = 1;
                     continue;
@@ -315,10 +338,10 @@ static int backward_head_impl(const double *q, const double *k, const double *xs
                         double a = 0.0;
                         for (int c = 0; c < D; ++c) a += gt[c] * xu[c];
                         dS[t * n + u] = a;
-                        dot += P[t * n + u] * a;
+                        if (P[t * n + u] != 0.0) dot += P[t * n + u] * a;
                     }
-                    for (int u = 0; u < n; ++u)
-                        dS[t * n + u] = P[t * n + u] * (dS[t * n + u] - dot);
+                    for (int u = 0; u < n; ++u)        /* weight 0 (masked, padding): exactly 0 */
+                        dS[t * n + u] = P[t * n + u] != 0.0 ? P[t * n + u] * (dS[t * n + u] - dot) : 0.0;
                 }
                 /* G_i = P^T G_{i+1};  dQ += scale dS K;  dK += scale dS^T Q
                  * (segments are disjoint token sets, so no two threads touch the same row) */
@@ -330,6 +353,7 @@ static int backward_head_impl(const double *q, const double *k, const double *xs
                         const double *gt = g + (base + (long)t * s) * D;
                         const double *qt = q + (base + (long)t * s) * D;
                         double p = P[t * n + u], ds = scale * dS[t * n + u];
+                        if (p == 0.0) continue;             /* then ds = 0 too: nothing flows */
                         for (int c = 0; c < D; ++c) { go[c] += p * gt[c]; dku[c] += ds * qt[c]; }
                     }
                 }
@@ -338,6 +362,7 @@ static int backward_head_impl(const double *q, const double *k, const double *xs
                     for (int u = 0; u < n; ++u) {
                         const double *ku = k + (base + (long)u * s) * D;
                         double ds = scale * dS[t * n + u];
+                        if (P[t * n + u] == 0.0) continue;
                         for (int c = 0; c < D; ++c) dqt[c] += ds * ku[c];
                     }
                 }
@@ -363,7 +388,7 @@ int ta_oracle_backward_head(const double *q, const double *k, const double *xs,
                             long N, int D, const int *dims, int ndims, int causal,
                             double scale)
 {
-    return backward_head_impl(q, k, xs, dout, dq, dk, dv, N, D, dims, ndims, causal, scale, 0.0, NULL, NULL);
+    return backward_head_impl(q, k, xs, dout, dq, dk, dv, N, D, dims, ndims, causal, scale, 0.0, NULL, NULL, N);
 }
 
 int ta_oracle_backward_head_rope(const double *q, const double *k, const double *xs,
@@ -373,7 +398,7 @@ int ta_oracle_backward_head_rope(const double *q, const double *k, const double 
 {
     if (!(rope_base > 0.0)) return -1;
     return backward_head_impl(q, k, xs, dout, dq, dk, dv, N, D, dims, ndims, causal, scale,
-                              rope_base, NULL, NULL);
+                              rope_base, NULL, NULL, N);
 }
 
 int ta_oracle_backward_head_ex(const double *q, const double *k, const double *xs,
@@ -384,7 +409,19 @@ int ta_oracle_backward_head_ex(const double *q, const double *k, const double *x
 {
     if (rope_base < 0.0) return -1;
     return backward_head_impl(q, k, xs, dout, dq, dk, dv, N, D, dims, ndims, causal, scale,
-                              rope_base, window, masks);
+                              rope_base, window, masks, N);
+}
+
+/* As ta_oracle_backward_head_ex with a valid length (xs from ta_oracle_forward_head_len). */
+int ta_oracle_backward_head_len(const double *q, const double *k, const double *xs,
+                                const double *dout, double *dq, double *dk, double *dv,
+                                long N, int D, const int *dims, int ndims, int causal,
+                                double scale, double rope_base, const int *window,
+                                const unsigned char *const *masks, long len)
+{
+    if (rope_base < 0.0) return -1;
+    return backward_head_impl(q, k, xs, dout, dq, dk, dv, N, D, dims, ndims, causal, scale,
+                              rope_base, window, masks, len);
 }
 
 int ta_oracle_num_threads(void)

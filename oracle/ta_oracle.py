@@ -72,6 +72,16 @@ def _lib():
                                                    ctypes.c_int, ip, ctypes.c_int, ctypes.c_int,
                                                    ctypes.c_double, ctypes.c_double, ip,
                                                    ctypes.POINTER(ctypes.c_void_p)]
+        lib.ta_oracle_forward_head_len.restype = ctypes.c_int
+        lib.ta_oracle_forward_head_len.argtypes = [dp, dp, dp, dp, ctypes.c_long, ctypes.c_int, ip,
+                                                   ctypes.c_int, ctypes.c_int, ctypes.c_double,
+                                                   ctypes.c_double, ip, ctypes.POINTER(ctypes.c_void_p),
+                                                   ctypes.c_long, dp]
+        lib.ta_oracle_backward_head_len.restype = ctypes.c_int
+        lib.ta_oracle_backward_head_len.argtypes = [dp, dp, dp, dp, dp, dp, dp, ctypes.c_long,
+                                                    ctypes.c_int, ip, ctypes.c_int, ctypes.c_int,
+                                                    ctypes.c_double, ctypes.c_double, ip,
+                                                    ctypes.POINTER(ctypes.c_void_p), ctypes.c_long]
         lib.ta_oracle_num_threads.restype = ctypes.c_int
         _LIB = lib
     return _LIB
@@ -134,7 +144,21 @@ def _cmasks(masks, dims):
     return (ctypes.c_void_p * len(dims))(*ptrs), keep
 
 
-def _fwd_head(lib, qh, kh, vh, out, N, D, cdims, m, causal, scale, rope_base, xs, cwin=None, cmask=None):
+def _clens(seq_lens, B, N):
+    if seq_lens is None:
+        return None
+    lens = [int(x) for x in seq_lens]
+    if len(lens) != B or any(x < 0 or x > N for x in lens):
+        raise ValueError("seq_lens: one length in [0, N] per batch entry")
+    return lens
+
+
+def _fwd_head(lib, qh, kh, vh, out, N, D, cdims, m, causal, scale, rope_base, xs, cwin=None, cmask=None,
+              length=None):
+    if length is not None:
+        return lib.ta_oracle_forward_head_len(_dptr(qh), _dptr(kh), _dptr(vh), _dptr(out), N, D, cdims, m,
+                                              int(bool(causal)), scale, float(rope_base or 0.0), cwin, cmask,
+                                              int(length), _dptr(xs) if xs is not None else None)
     if cwin is not None or cmask is not None:
         return lib.ta_oracle_forward_head_ex(_dptr(qh), _dptr(kh), _dptr(vh), _dptr(out), N, D, cdims, m,
                                              int(bool(causal)), scale, float(rope_base or 0.0), cwin, cmask,
@@ -148,7 +172,8 @@ def _fwd_head(lib, qh, kh, vh, out, N, D, cdims, m, causal, scale, rope_base, xs
 
 
 def forward(q, k, v, dims, causal: bool, scale: float | None = None, heads=None,
-            return_xs: bool = False, rope_base: float | None = None, window=None, masks=None):
+            return_xs: bool = False, rope_base: float | None = None, window=None, masks=None,
+            seq_lens=None):
     """Algorithm 1 for every (or the listed) head, fp64.
 
     q: [B,H,N,D]; k, v: [B,H_kv,N,D] (any float dtype; converted head by head to fp64).
@@ -160,6 +185,8 @@ def forward(q, k, v, dims, causal: bool, scale: float | None = None, heads=None,
     positions of the query along dimension i (|t - u| < w_i); 0 = no window.
     masks: None, or one entry per dimension: None or an n_i x n_i array (row = query position,
     column = key position, non-zero = visible) applied on top of `causal` and `window`.
+    seq_lens: None, or one valid length per batch entry: tokens with flat index >= seq_lens[b]
+    are padding (never visible as keys; their output rows are 0).
     Returns out [B,H,N,D] fp64 (and, with return_xs, the list of per-head [m+1,N,D]
     value tensors X_0=V ... X_m=out keyed like the output).
     """
@@ -169,6 +196,7 @@ def forward(q, k, v, dims, causal: bool, scale: float | None = None, heads=None,
     cdims = (ctypes.c_int * len(dims))(*dims)
     cwin = _cwindow(window, len(dims))
     cmask, _keep = _cmasks(masks, dims)
+    lens = _clens(seq_lens, B, N)
     pairs = [(b, h) for b in range(B) for h in range(H)] if heads is None else list(heads)
     out = np.empty((len(pairs), N, D), dtype=np.float64)
     xs_all = []
@@ -177,7 +205,7 @@ def forward(q, k, v, dims, causal: bool, scale: float | None = None, heads=None,
         qh, kh, vh = _f64(q[b, h]), _f64(k[b, h // g]), _f64(v[b, h // g])
         xs = np.empty((len(dims) + 1, N, D), dtype=np.float64) if return_xs else None
         rc = _fwd_head(lib, qh, kh, vh, out[idx], N, D, cdims, len(dims), causal, scale,
-                       rope_base, xs, cwin, cmask)
+                       rope_base, xs, cwin, cmask, None if lens is None else lens[b])
         if rc != 0:
             raise RuntimeError("ta_oracle_forward_head failed")
         if return_xs:
@@ -188,8 +216,9 @@ def forward(q, k, v, dims, causal: bool, scale: float | None = None, heads=None,
 
 
 def backward(dout, q, k, v, dims, causal: bool, scale: float | None = None, groups=None,
-             rope_base: float | None = None, window=None, masks=None):
+             rope_base: float | None = None, window=None, masks=None, seq_lens=None):
     """Gradients of sum(out * dout) w.r.t. q, k, v (fp64), GQA groups summed into dk, dv.
+    With seq_lens the rows of padding tokens are 0 in all three and their rows of dout are ignored.
 
     groups: optional list of (b, kv_head) pairs; then only those KV heads and their query
     heads are computed and the result is (dq [len, g, N, D], dk [len, N, D], dv [len, N, D]).
@@ -200,6 +229,7 @@ def backward(dout, q, k, v, dims, causal: bool, scale: float | None = None, grou
     cdims = (ctypes.c_int * len(dims))(*dims)
     cwin = _cwindow(window, len(dims))
     cmask, _keep = _cmasks(masks, dims)
+    lens = _clens(seq_lens, B, N)
     sel = [(b, kv) for b in range(B) for kv in range(Hkv)] if groups is None else list(groups)
     dq = np.zeros((len(sel), g, N, D))
     dk = np.zeros((len(sel), N, D))
@@ -212,11 +242,18 @@ def backward(dout, q, k, v, dims, causal: bool, scale: float | None = None, grou
             qh = _f64(q[b, h])
             o = np.empty((N, D))
             xs = np.empty((len(dims) + 1, N, D))
-            rc = _fwd_head(lib, qh, kh, vh, o, N, D, cdims, len(dims), causal, scale, rope_base, xs, cwin, cmask)
+            rc = _fwd_head(lib, qh, kh, vh, o, N, D, cdims, len(dims), causal, scale, rope_base, xs, cwin, cmask,
+                           None if lens is None else lens[b])
             if rc != 0:
                 raise RuntimeError("ta_oracle_forward_head failed")
             dqh, dkh, dvh = np.empty((N, D)), np.empty((N, D)), np.empty((N, D))
-            if cwin is not None or cmask is not None:
+            if lens is not None:
+                rc = lib.ta_oracle_backward_head_len(_dptr(qh), _dptr(kh), _dptr(xs),
+                                                     _dptr(_f64(dout[b, h])), _dptr(dqh), _dptr(dkh),
+                                                     _dptr(dvh), N, D, cdims, len(dims),
+                                                     int(bool(causal)), scale, float(rope_base or 0.0), cwin,
+                                                     cmask, int(lens[b]))
+            elif cwin is not None or cmask is not None:
                 rc = lib.ta_oracle_backward_head_ex(_dptr(qh), _dptr(kh), _dptr(xs),
                                                     _dptr(_f64(dout[b, h])), _dptr(dqh), _dptr(dkh),
                                                     _dptr(dvh), N, D, cdims, len(dims),
@@ -248,7 +285,7 @@ def backward(dout, q, k, v, dims, causal: bool, scale: float | None = None, grou
 # --------------------------------------------------------------------------------------
 
 def dense_hop_matrix(qh, kh, dims, i: int, causal: bool, scale: float | None = None,
-                     rope_base: float | None = None, window=None, masks=None):
+                     rope_base: float | None = None, window=None, masks=None, length=None):
     """The N x N matrix of hop i for one head (Eq. 3 written over flat token indices).
 
     Entry [j, k] is the softmax weight of key token k for query token j; it is non-zero only
@@ -286,6 +323,16 @@ def dense_hop_matrix(qh, kh, dims, i: int, causal: bool, scale: float | None = N
         s = s * scale
     else:
         s = (qh @ kh.T) * scale
+    if length is not None:
+        # padding tokens (flat index >= length): no column, and an all-zero row
+        exists = np.arange(N) < int(length)
+        allowed &= exists[None, :]
+        s = np.where(allowed, s, -np.inf)
+        a = np.zeros((N, N))
+        live = s[exists]
+        e = np.exp(live - live.max(axis=1, keepdims=True))
+        a[exists] = e / e.sum(axis=1, keepdims=True)
+        return a
     s = np.where(allowed, s, -np.inf)
     s = s - s.max(axis=1, keepdims=True)
     e = np.exp(s)
@@ -293,23 +340,24 @@ def dense_hop_matrix(qh, kh, dims, i: int, causal: bool, scale: float | None = N
 
 
 def dense_effective_matrix(qh, kh, dims, causal: bool, scale: float | None = None,
-                           rope_base: float | None = None, window=None, masks=None):
+                           rope_base: float | None = None, window=None, masks=None, length=None):
     """A_eff = A^_{m-1} ... A^_1 A^_0, the N x N map from V to the output of one head."""
     N = np.asarray(qh).shape[0]
     a = np.eye(N)
     for i in range(len(dims)):
-        a = dense_hop_matrix(qh, kh, dims, i, causal, scale, rope_base, window, masks) @ a
+        a = dense_hop_matrix(qh, kh, dims, i, causal, scale, rope_base, window, masks, length) @ a
     return a
 
 
 def forward_dense(q, k, v, dims, causal: bool, scale: float | None = None,
-                  rope_base: float | None = None, window=None, masks=None):
+                  rope_base: float | None = None, window=None, masks=None, seq_lens=None):
     """Brute-force forward for all heads via dense_effective_matrix (tiny N only)."""
     B, H, Hkv, N, D, dims = _check(q, k, v, dims)
     g = H // Hkv
     out = np.empty((B, H, N, D))
     for b in range(B):
         for h in range(H):
-            a = dense_effective_matrix(q[b, h], k[b, h // g], dims, causal, scale, rope_base, window, masks)
+            a = dense_effective_matrix(q[b, h], k[b, h // g], dims, causal, scale, rope_base, window, masks,
+                                       None if seq_lens is None else seq_lens[b])
             out[b, h] = a @ np.asarray(v[b, h // g], dtype=np.float64)
     return out
