@@ -119,6 +119,7 @@ typedef struct ta_params {
                            /* (Section 3.2), applied inside the kernels -- see ta_forward_ex  */
     const int *window;     /* host, ndims ints, or NULL: per-hop sliding window, see below     */
     const unsigned char *const *hop_masks; /* host, ndims pointers, or NULL: explicit M_i, see below */
+    const int *seq_lens;   /* DEVICE, B ints, or NULL: valid length per batch entry, see below  */
     ta_stream_t stream;
 } ta_params;
 
@@ -150,6 +151,17 @@ typedef struct ta_params {
  * vector of the hop, applied on top of `causal` and window[i].  Read during the call.  Supported
  * for n_i <= 128 (TA_ERR_UNSUPPORTED beyond); a query position left without any visible key is
  * TA_ERR_INVALID_ARG.  Hops are not fused when a mask is given.  ta_backward_ex takes the same.
+ *
+ * Valid lengths (padding to prod(dims), batches of different lengths; a mask M_i that depends
+ * on the segment): with seq_lens != NULL only the tokens of batch entry b with flat index
+ * < seq_lens[b] exist.  A padding token is never visible as a key, and the row of `out` of a
+ * padding query is written as 0.  seq_lens is read on the device, in stream order (no host
+ * synchronisation); values are clamped to [0, N].  The padding rows of q, k and v must hold
+ * finite values (they are multiplied by weights that are exactly 0).  With `causal` the rows
+ * below the length equal those of the call without seq_lens (a causal hop only reads tokens of
+ * smaller flat index).  Hops are not fused, and segments longer than 128 run on the generic
+ * kernel.  ta_backward_ex takes the same array: the padding rows of dq, dk, dv are 0 and those
+ * of dout are not used (but must be finite).
  */
 int ta_forward_ex(const ta_params *p);
 
@@ -195,6 +207,7 @@ typedef struct ta_bwd_params {
                                   /* with respect to the un-rotated q, k).  D must be even.     */
     const int *window;            /* host, ndims ints, or NULL: sliding windows as in ta_forward_ex */
     const unsigned char *const *hop_masks; /* host, ndims pointers, or NULL: explicit masks, as in ta_forward_ex */
+    const int *seq_lens;          /* DEVICE, B ints, or NULL: valid lengths, as in ta_forward_ex */
     const void *saved_hops;       /* X_1..X_{m-1} as written by ta_forward_ex(TA_FLAG_SAVE_HOPS) */
                                   /* (the part of its workspace after the scratch tensor), or    */
                                   /* NULL: recomputed                                          */

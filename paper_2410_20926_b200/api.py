@@ -47,6 +47,7 @@ class ta_params(ctypes.Structure):
                 ("rope_base", ctypes.c_float),
                 ("window", ctypes.POINTER(ctypes.c_int)),
                 ("hop_masks", ctypes.POINTER(ctypes.c_void_p)),
+                ("seq_lens", ctypes.c_void_p),
                 ("stream", ctypes.c_void_p)]
 
 
@@ -62,6 +63,7 @@ class ta_bwd_params(ctypes.Structure):
                 ("softmax_scale", ctypes.c_float), ("rope_base", ctypes.c_float),
                 ("window", ctypes.POINTER(ctypes.c_int)),
                 ("hop_masks", ctypes.POINTER(ctypes.c_void_p)),
+                ("seq_lens", ctypes.c_void_p),
                 ("saved_hops", ctypes.c_void_p),
                 ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
                 ("stream", ctypes.c_void_p)]
@@ -210,7 +212,8 @@ def _hop_masks(hop_masks, dims):
 
 def ta_forward_ex(q, k, v, out, B, H, H_kv, N, D, dims, causal, dtype=TA_DTYPE_BF16,
                   softmax_scale=0.0, workspace=None, workspace_bytes=0, flags=0, hop_begin=0,
-                  hop_end=0, rope_base=0.0, window=None, hop_masks=None, stream=None, check=True) -> int:
+                  hop_end=0, rope_base=0.0, window=None, hop_masks=None, seq_lens=None, stream=None,
+                  check=True) -> int:
     d, nd = _dims(dims)
     p = ta_params()
     p.struct_bytes = ctypes.sizeof(ta_params)
@@ -227,6 +230,7 @@ def ta_forward_ex(q, k, v, out, B, H, H_kv, N, D, dims, causal, dtype=TA_DTYPE_B
     masks, _keep = _hop_masks(hop_masks, dims)
     if masks is not None:
         p.hop_masks = masks
+    p.seq_lens = _ptr(seq_lens)        # device int32 tensor [B] or None
     p.stream = _stream(stream)
     return _done(load().ta_forward_ex(ctypes.byref(p)), "ta_forward_ex", check)
 
@@ -242,8 +246,8 @@ def ta_backward(dout, q, k, v, out, dq, dk, dv, B, H, H_kv, N, D, dims, causal, 
 
 def ta_backward_ex(dout, q, k, v, dq, dk, dv, B, H, H_kv, N, D, dims, causal,
                    grad_dtype=TA_DTYPE_BF16, softmax_scale=0.0, saved_hops=None, workspace=None,
-                   workspace_bytes=0, rope_base=0.0, window=None, hop_masks=None, stream=None,
-                   check=True) -> int:
+                   workspace_bytes=0, rope_base=0.0, window=None, hop_masks=None, seq_lens=None,
+                   stream=None, check=True) -> int:
     d, nd = _dims(dims)
     p = ta_bwd_params()
     p.struct_bytes = ctypes.sizeof(ta_bwd_params)
@@ -259,6 +263,7 @@ def ta_backward_ex(dout, q, k, v, dq, dk, dv, B, H, H_kv, N, D, dims, causal,
     masks, _keep = _hop_masks(hop_masks, dims)
     if masks is not None:
         p.hop_masks = masks
+    p.seq_lens = _ptr(seq_lens)
     p.saved_hops = _ptr(saved_hops)
     p.workspace, p.workspace_bytes = _ptr(workspace), workspace_bytes
     p.stream = _stream(stream)

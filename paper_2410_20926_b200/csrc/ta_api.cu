@@ -52,7 +52,7 @@ int build_plan(int B, int H, int H_kv, int N, int D, const int *dims, int ndims,
                unsigned flags, int hop_begin, int hop_end, Plan *plan) {
     int rc = validate_shape(B, H, H_kv, N, D, dims, ndims, dtype);
     if (rc != TA_OK) return rc;
-    if (flags & ~(unsigned)(TA_FLAG_NO_TENSOR_CORE | TA_FLAG_NO_HOP_FUSION | TA_FLAG_SAVE_HOPS | kPlanFlagRope))
+    if (flags & ~(unsigned)(TA_FLAG_NO_TENSOR_CORE | TA_FLAG_NO_HOP_FUSION | TA_FLAG_SAVE_HOPS | kPlanFlagRope | kPlanFlagLens))
         return TA_ERR_UNSUPPORTED;
     if (hop_begin == 0 && hop_end == 0) hop_end = ndims;
     if (hop_begin < 0 || hop_end > ndims || hop_begin > hop_end) return TA_ERR_INVALID_ARG;
@@ -68,7 +68,8 @@ int build_plan(int B, int H, int H_kv, int N, int D, const int *dims, int ndims,
         h.path = PATH_SIMT;
         if (tc_eligible(D, dtype, flags)) {
             if (h.n <= 128) h.path = PATH_TC;
-            else if (!(flags & kPlanFlagRope)) h.path = PATH_TC_LONG;   // the long-segment kernel does not rotate
+            // the long-segment kernel neither rotates nor takes valid lengths
+            else if (!(flags & (kPlanFlagRope | kPlanFlagLens))) h.path = PATH_TC_LONG;
         }
         if (h.path == PATH_TC) tile_packing(h);
     }
@@ -286,12 +287,13 @@ static int forward_impl(const ta_params &p) {
             if (p.window[i] < 0) return TA_ERR_INVALID_ARG;
     Plan plan;
     // the positional encoding gives every hop its own rotated Q and K: nothing to share, no fusion
-    if (p.flags & kPlanFlagRope) return TA_ERR_UNSUPPORTED;
+    if (p.flags & (kPlanFlagRope | kPlanFlagLens)) return TA_ERR_UNSUPPORTED;
     bool any_mask = false;
     if (p.hop_masks && p.ndims >= 1 && p.ndims <= TA_MAX_DIMS)
         for (int i = 0; i < p.ndims; ++i) any_mask = any_mask || p.hop_masks[i] != nullptr;
     const unsigned plan_flags = p.flags | (p.rope_base > 0.f ? (unsigned)TA_FLAG_NO_HOP_FUSION | kPlanFlagRope : 0u) |
-                                (any_mask ? (unsigned)TA_FLAG_NO_HOP_FUSION : 0u);
+                                (any_mask ? (unsigned)TA_FLAG_NO_HOP_FUSION : 0u) |
+                                (p.seq_lens ? (unsigned)TA_FLAG_NO_HOP_FUSION | kPlanFlagLens : 0u);
     int rc = build_plan(p.B, p.H, p.H_kv, p.N, p.D, p.dims, p.ndims, p.dtype, plan_flags, p.hop_begin,
                         p.hop_end, &plan);
     if (rc != TA_OK) return rc;
@@ -310,6 +312,7 @@ static int forward_impl(const ta_params &p) {
     pb.ndims = p.ndims; pb.causal = p.causal ? 1 : 0; pb.dtype = p.dtype;
     pb.scale = p.softmax_scale != 0.f ? p.softmax_scale : 1.0f / sqrtf((float)p.D);
     pb.rope_base = p.rope_base;
+    pb.seq_lens = p.seq_lens;
     if ((rc = take_masks(&pb, plan, p.window, p.hop_masks, p.ndims)) != TA_OK) return rc;
     pb.flags = p.flags; pb.hop_begin = p.hop_begin; pb.hop_end = p.hop_end;
     pb.stream = (cudaStream_t)p.stream;

@@ -81,6 +81,7 @@ int backward_impl(const ta_bwd_params &p) {
     pb.ndims = p.ndims; pb.causal = p.causal ? 1 : 0; pb.dtype = p.dtype;
     pb.scale = p.softmax_scale != 0.f ? p.softmax_scale : 1.0f / sqrtf((float)p.D);
     pb.rope_base = p.rope_base;
+    pb.seq_lens = p.seq_lens;
     pb.causal = p.causal ? 1 : 0;
     if ((rc = take_masks(&pb, plan, p.window, p.hop_masks, p.ndims)) != TA_OK) return rc;
     pb.flags = 0; pb.hop_begin = 0; pb.hop_end = p.ndims;
@@ -94,6 +95,7 @@ int backward_impl(const ta_bwd_params &p) {
     const int k = plan.nhops;
 
     if (k == 0) {
+        if (p.seq_lens) return TA_ERR_UNSUPPORTED;   // no hop to apply the valid lengths in
         if (cudaMemsetAsync(dq_acc, 0, tq * 4, pb.stream) != cudaSuccess ||
             cudaMemsetAsync(dk_acc, 0, tkv * 4, pb.stream) != cudaSuccess)
             return TA_ERR_CUDA;

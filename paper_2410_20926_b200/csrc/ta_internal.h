@@ -21,6 +21,7 @@ enum HopPath {
 
 // build_plan flag used inside the library only: the call carries the positional encoding
 constexpr unsigned kPlanFlagRope = 1u << 30;
+constexpr unsigned kPlanFlagLens = 1u << 29;   // valid lengths given: the long-segment kernel does not take them
 
 // One hop of Algorithm 1 as a strided view X[outer][t][inner][D] of a head:
 //   token(outer, t, inner) = outer * n * stride + t * stride + inner.
@@ -63,6 +64,7 @@ struct Problem {
     float rope_base;  // 0 = no positional encoding
     int window[TA_MAX_DIMS];  // per dimension: 0 = none, w > 0 = keys within w positions of the query
     const unsigned char *masks[TA_MAX_DIMS];  // per dimension: NULL or host n x n bytes, non-zero = visible
+    const int *seq_lens;                      // device, B valid lengths, or NULL
     unsigned flags;
     int hop_begin, hop_end;
     cudaStream_t stream;

@@ -79,6 +79,7 @@ extern "C" int ta_forward_static(const void *q, const void *k, const void *v, vo
     pb.ndims = ndims; pb.causal = causal ? 1 : 0; pb.dtype = dtype;
     pb.scale = 1.0f / sqrtf((float)D);
     pb.rope_base = 0.f;
+    pb.seq_lens = nullptr;
     for (int i = 0; i < TA_MAX_DIMS; ++i) { pb.window[i] = 0; pb.masks[i] = nullptr; }
     pb.flags = 0; pb.hop_begin = 0; pb.hop_end = ndims;
     pb.stream = (cudaStream_t)stream;

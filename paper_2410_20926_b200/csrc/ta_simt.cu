@@ -33,6 +33,7 @@ struct SimtArgs {
     float rope_log2_base;         // 0: no positional encoding; else log2 of the RoPE base
     int window;                   // 0, or sliding window along the hop's dimension
     int masked;                   // 1: visibility comes from the HopMask parameter (n <= 128)
+    const int *lens;              // device, valid length per batch entry, or nullptr
 };
 
 // Tensorized positional encoding (Section 3.2): rows of `x` ([rows][ld] fp32 in shared memory)
@@ -96,6 +97,13 @@ hop_simt_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__res
         const T *xh_p = xin + xh * (long long)a.N * D;
         T *oh = xout + bh * (long long)a.N * D;
         const int t0 = qb * BQ;
+        // valid length: the first `exist` positions of this segment are tokens of the batch entry
+        int exist = a.n;
+        if (a.lens != nullptr) {
+            const long long len = min(max(__ldg(a.lens + b), 0), a.N);
+            const long long left = (len - base + a.stride - 1) / a.stride;
+            exist = len <= base ? 0 : (int)(left < a.n ? left : a.n);
+        }
 
         __syncthreads();   // previous item's smem no longer in use
         for (int idx = threadIdx.x; idx < BQ * D; idx += kThreads) {
@@ -117,13 +125,13 @@ hop_simt_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__res
         }
 
         const int t_last = min(a.n, t0 + BQ) - 1;
-        const int key_end = a.causal ? t_last + 1 : a.n;
+        const int key_end = min(a.causal ? t_last + 1 : a.n, exist);
         for (int k0 = 0; k0 < key_end; k0 += BK) {
             __syncthreads();
             for (int idx = threadIdx.x; idx < BK * D; idx += kThreads) {
                 int u = idx / D, c = idx % D, key = k0 + u;
                 float kvv = 0.f, xv = 0.f;
-                if (key < a.n) {
+                if (key < exist) {
                     long long off = (base + (long long)key * a.stride) * D + c;
                     kvv = to_f32<T>(kh[off]);
                     xv = to_f32<T>(xh_p[off]);
@@ -145,7 +153,7 @@ hop_simt_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__res
                 float s = 0.f;
                 for (int c = 0; c < D; ++c) s = fmaf(qr[c], kr[c], s);
                 s *= a.scale;
-                bool valid = key < a.n && (!a.causal || key <= t) &&
+                bool valid = key < exist && t < exist && (!a.causal || key <= t) &&
                              (a.window == 0 || (key > t - a.window && key < t + a.window));
                 if (a.masked) valid = valid && ((hop_mask.bits[t][key >> 5] >> (key & 31)) & 1u);
                 s = valid ? s : -INFINITY;
@@ -172,7 +180,7 @@ hop_simt_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__res
         for (int r = 0; r < kRowsPerWarp; ++r) {
             const int t = t0 + warp * kRowsPerWarp + r;
             if (t >= a.n) continue;
-            const float inv = 1.f / l[r];
+            const float inv = l[r] > 0.f ? 1.f / l[r] : 0.f;   // a padding row has seen nothing: 0
 #pragma unroll
             for (int j = 0; j < DPL; ++j) {
                 const int c = lane + 32 * j;
@@ -184,13 +192,14 @@ hop_simt_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__res
 
 template <typename T>
 __global__ void broadcast_kv_kernel(const T *__restrict__ v, T *__restrict__ out, long long per_head,
-                                    int H, int H_kv, long long total) {
+                                    int H, int H_kv, long long total, const int *lens, int D) {
     const int g = H / H_kv;
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
          i += (long long)gridDim.x * blockDim.x) {
         long long bh = i / per_head, r = i % per_head;
         long long b = bh / H, h = bh % H;
-        out[i] = v[(b * H_kv + h / g) * per_head + r];
+        const bool exists = lens == nullptr || r / D < __ldg(lens + b);
+        out[i] = exists ? v[(b * H_kv + h / g) * per_head + r] : from_f32<T>(0.f);
     }
 }
 
@@ -206,6 +215,7 @@ int launch_t(const Problem &pb, const HopDesc &hd, const void *xin, int xin_head
     a.rope_log2_base = pb.rope_base > 0.f ? log2f(pb.rope_base) : 0.f;
     a.window = pb.window[hd.hop];
     a.masked = 0;
+    a.lens = pb.seq_lens;
     HopMask hm;
     if (pb.masks[hd.hop]) {
         const int rc = build_hop_mask(pb, hd, &hm);   // explicit mask ^ causal flag ^ window
@@ -251,10 +261,10 @@ int launch_broadcast_kv(const Problem &pb) {
     const unsigned grid = (unsigned)((total + 255) / 256 < 148 * 16 ? (total + 255) / 256 : 148 * 16);
     if (pb.dtype == TA_DTYPE_F32)
         broadcast_kv_kernel<float><<<grid, 256, 0, pb.stream>>>((const float *)pb.v, (float *)pb.out, per_head,
-                                                                pb.H, pb.H_kv, total);
+                                                                pb.H, pb.H_kv, total, pb.seq_lens, pb.D);
     else
         broadcast_kv_kernel<__nv_bfloat16><<<grid, 256, 0, pb.stream>>>(
-            (const __nv_bfloat16 *)pb.v, (__nv_bfloat16 *)pb.out, per_head, pb.H, pb.H_kv, total);
+            (const __nv_bfloat16 *)pb.v, (__nv_bfloat16 *)pb.out, per_head, pb.H, pb.H_kv, total, pb.seq_lens, pb.D);
     count_launch();
     return cudaPeekAtLastError() == cudaSuccess ? TA_OK : TA_ERR_CUDA;
 }

@@ -71,6 +71,8 @@ struct TcArgs {
     int window;                // 0, or w: keys within w positions of the query along the hop's dimension
     float scale_log2;
     float rope_log2_base;      // log2 of the RoPE base (rotating variant only)
+    int stride;                // token stride of the hop's dimension
+    const int *lens;           // device, one valid length per batch entry, or nullptr (masked variant only)
 };
 
 struct ItemCoord {
@@ -335,6 +337,22 @@ hop_pipe_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         bool ok = true;
         for (uint32_t t = b; t < T; t += 2) {
             const uint32_t par = (t >> 1) & 1;
+            // valid length: only the first `exist` positions of this row's segment are tokens
+            // (flat index below the batch entry's length); a padding row sees nothing
+            uint32_t mt[4] = {mrow[0], mrow[1], mrow[2], mrow[3]};
+            if (kMask && a.lens != nullptr) {
+                const ItemCoord c = decode_item(a, (long long)blockIdx.x + (long long)(t / (uint32_t)a.gi) * gridDim.x);
+                const int len = __ldg(a.lens + c.kv_head / a.H_kv);
+                const long long first = (long long)(c.c_outer + seg / a.ci) * a.n * a.stride + (c.c_inner + seg % a.ci);
+                const long long left = ((long long)len - first + a.stride - 1) / a.stride;
+                const int exist = len <= first ? 0 : (int)(left < a.n ? left : a.n);
+                const int limit = (r % a.n) < exist ? seg * a.n + exist : 0;      // columns below it exist
+#pragma unroll
+                for (int cch = 0; cch < 4; ++cch) {
+                    const int nb = limit - 32 * cch;
+                    mt[cch] &= nb >= 32 ? 0xffffffffu : (nb <= 0 ? 0u : ((1u << nb) - 1u));
+                }
+            }
             ok = mbar_wait_abortable(s_full(b), par, 0x40, abort_flag);
             ok = __all_sync(0xffffffffu, ok);           // keep the warp converged for the aligned TMEM ops
             if (!ok) break;
@@ -352,11 +370,12 @@ hop_pipe_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 for (int jj = 0; jj < 32; ++jj) {
                     const int col = 32 * c + jj;
                     const float s = __uint_as_float(v[jj]);
-                    const bool vis = kMask ? ((mask_chunk(mrow, c) >> jj) & 1u) != 0 : (col >= c_lo && col < c_hi);
+                    const bool vis = kMask ? ((mask_chunk(mt, c) >> jj) & 1u) != 0 : (col >= c_lo && col < c_hi);
                     if (vis) m = fmaxf(m, s);
                 }
             }
-            const float m_scaled = row_valid ? m * a.scale_log2 : 0.f;
+            // (a padding row of the masked variant has seen nothing: keep the arithmetic finite)
+            const float m_scaled = (row_valid && !(kMask && m == -INFINITY)) ? m * a.scale_log2 : 0.f;
             float sum = 0.f;
 #pragma unroll 1
             for (int c = 0; c < nchunks; ++c) {
@@ -369,7 +388,7 @@ hop_pipe_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                         float p0 = fast_exp2(__uint_as_float(v[jj]) * a.scale_log2 - m_scaled);
                         float p1 = fast_exp2(__uint_as_float(v[jj + 1]) * a.scale_log2 - m_scaled);
                         if (kMask) {
-                            const uint32_t bits = mask_chunk(mrow, c);
+                            const uint32_t bits = mask_chunk(mt, c);
                             p0 = ((bits >> jj) & 1u) ? p0 : 0.f;
                             p1 = ((bits >> (jj + 1)) & 1u) ? p1 : 0.f;
                         } else {
@@ -387,7 +406,7 @@ hop_pipe_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 tmem_st16(s_col + 16 * c, pk);
             }
             tmem_st_wait();
-            const float inv = row_valid ? 1.f / sum : 1.f;
+            const float inv = row_valid ? (kMask ? (sum > 0.f ? 1.f / sum : 0.f) : 1.f / sum) : 1.f;
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(p_full(b));
@@ -508,6 +527,8 @@ int launch_d(const Problem &pb, const HopDesc &hd, const void *xin, int xin_head
     a.window = pb.window[hd.hop];
     a.scale_log2 = pb.scale * 1.4426950408889634f;
     a.rope_log2_base = pb.rope_base > 0.f ? log2f(pb.rope_base) : 0.f;
+    a.stride = (int)hd.stride;
+    a.lens = pb.seq_lens;
 
     constexpr size_t smem = PipeCfg<D>::kSmemBytes;
     const unsigned grid = (unsigned)(a.total_items < num_sms ? a.total_items : num_sms);
@@ -521,7 +542,7 @@ int launch_d(const Problem &pb, const HopDesc &hd, const void *xin, int xin_head
             return TA_ERR_CUDA;
         configured = true;
     }
-    if (pb.masks[hd.hop]) {
+    if (pb.masks[hd.hop] || pb.seq_lens) {
         HopMask hm;                                  // explicit mask ^ causal flag ^ window, by value
         const int rc = build_hop_mask(pb, hd, &hm);
         if (rc != TA_OK) return rc;

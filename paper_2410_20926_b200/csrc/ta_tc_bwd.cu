@@ -48,6 +48,8 @@ struct BwdArgs {
     long long tiles_inner, tiles_outer, total_items;
     float scale_log2, scale;
     float rope_log2_base;              // log2 of the RoPE base (rotating variant only)
+    int stride;                        // token stride of the hop's dimension
+    const int *lens;                   // device, valid length per batch entry, or nullptr (masked variant only)
 };
 
 template <int D>
@@ -251,8 +253,9 @@ hop_tc_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         uint32_t mrow[4];
         tile_row_mask(hop_mask, row_valid ? r % a.n : 0, seg * a.n, mrow);
         if (kMask && !row_valid) mrow[0] = mrow[1] = mrow[2] = mrow[3] = 0u;
+        uint32_t mt[4] = {mrow[0], mrow[1], mrow[2], mrow[3]};   // ... and below the batch entry's valid length
         auto visible = [&](int cc, int jj) -> bool {
-            if (kMask) return ((mask_chunk(mrow, cc) >> jj) & 1u) != 0;
+            if (kMask) return ((mask_chunk(mt, cc) >> jj) & 1u) != 0;
             const int col = 32 * cc + jj;
             return row_valid && col >= c_lo && col < c_hi;
         };
@@ -309,6 +312,20 @@ hop_tc_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         int pending_stage = -1;   // thread 0: stage whose output stores have been issued but not yet read out
         for (long long item = blockIdx.x; ok && item < a.total_items; item += gridDim.x, ++it) {
             const BwdItem c = decode_bwd_item(a, item);
+            if (kMask && a.lens != nullptr) {
+                // only the first `exist` positions of this row's segment are tokens; a padding row
+                // sees nothing (its P and dS rows are 0, so nothing flows through it)
+                const int len = __ldg(a.lens + c.kv_head / a.H_kv);
+                const long long first = (long long)(c.c_outer + seg / a.ci) * a.n * a.stride + (c.c_inner + seg % a.ci);
+                const long long left = ((long long)len - first + a.stride - 1) / a.stride;
+                const int exist = len <= first ? 0 : (int)(left < a.n ? left : a.n);
+                const int limit = (r % a.n) < exist ? seg * a.n + exist : 0;
+#pragma unroll
+                for (int cch = 0; cch < 4; ++cch) {
+                    const int nb = limit - 32 * cch;
+                    mt[cch] = mrow[cch] & (nb >= 32 ? 0xffffffffu : (nb <= 0 ? 0u : ((1u << nb) - 1u)));
+                }
+            }
             for (int j = 0; j < a.g; ++j, ++t) {
                 const int s = t & 1;
                 const uint32_t par = t & 1;
@@ -370,7 +387,7 @@ hop_tc_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                             if (visible(cc, jj)) m = fmaxf(m, __uint_as_float(vs[jj]));
                         }
                     }
-                    const float m_s = row_valid ? m * a.scale_log2 : 0.f;
+                    const float m_s = (row_valid && !(kMask && m == -INFINITY)) ? m * a.scale_log2 : 0.f;
                     float l = 0.f, dot = 0.f;
 #pragma unroll 1
                     for (int cc = 0; cc < 4; ++cc) {
@@ -386,7 +403,7 @@ hop_tc_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                             dot += vis ? p * __uint_as_float(vd[jj]) : 0.f;
                         }
                     }
-                    const float inv_l = row_valid ? 1.f / l : 0.f;
+                    const float inv_l = (row_valid && !(kMask && l == 0.f)) ? 1.f / l : 0.f;
                     const float delta = dot * inv_l;
                     const uint32_t rowP = sXP + (uint32_t)r * 128u, rowS = sdS + (uint32_t)r * 128u;
 #pragma unroll 1
@@ -602,6 +619,8 @@ int launch_bwd_d(const Problem &pb, const HopDesc &hd, const void *x, int x_head
     a.scale = pb.scale;
     a.scale_log2 = pb.scale * 1.4426950408889634f;
     a.rope_log2_base = pb.rope_base > 0.f ? log2f(pb.rope_base) : 0.f;
+    a.stride = (int)hd.stride;
+    a.lens = pb.seq_lens;
 
     static int num_sms = 0;
     if (num_sms == 0) {
@@ -622,7 +641,7 @@ int launch_bwd_d(const Problem &pb, const HopDesc &hd, const void *x, int x_head
         configured = true;
     }
     const unsigned grid = (unsigned)(a.total_items < num_sms ? a.total_items : num_sms);
-    if (pb.masks[hd.hop]) {
+    if (pb.masks[hd.hop] || pb.seq_lens) {
         HopMask hm;                                  // explicit mask ^ causal flag ^ window, by value
         const int rc = build_hop_mask(pb, hd, &hm);
         if (rc != TA_OK) return rc;

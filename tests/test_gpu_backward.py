@@ -26,7 +26,7 @@ RTOL = 2.0 ** -8
 
 
 def gpu_backward(inp, B, H, Hkv, N, D, dims, causal, grad_f32, saved=None, rope_base=0.0, window=None,
-                 hop_masks=None):
+                 hop_masks=None, seq_lens=None):
     import torch
     q, k, v, do = (to_device(inp, n, "bf16") for n in ("q", "k", "v", "dout"))
     tdt = torch.float32 if grad_f32 else torch.bfloat16
@@ -36,11 +36,12 @@ def gpu_backward(inp, B, H, Hkv, N, D, dims, causal, grad_f32, saved=None, rope_
     mode = ta.TA_WS_BACKWARD_F32_GRADS if grad_f32 else ta.TA_WS_BACKWARD
     nbytes = ta.ta_workspace_bytes(B, H, Hkv, N, D, dims, ta.TA_DTYPE_BF16, mode)
     ws = torch.empty(max(nbytes, 256), dtype=torch.uint8, device="cuda")
-    if grad_f32 or saved is not None or rope_base or window is not None or hop_masks is not None:
+    if grad_f32 or saved is not None or rope_base or window is not None or hop_masks is not None \
+            or seq_lens is not None:
         ta.ta_backward_ex(do, q, k, v, dq, dk, dv, B, H, Hkv, N, D, dims, causal,
                           grad_dtype=ta.TA_DTYPE_F32 if grad_f32 else ta.TA_DTYPE_BF16,
                           saved_hops=saved, workspace=ws, workspace_bytes=nbytes, rope_base=rope_base,
-                          window=window, hop_masks=hop_masks)
+                          window=window, hop_masks=hop_masks, seq_lens=seq_lens)
     else:
         ta.ta_backward(do, q, k, v, None, dq, dk, dv, B, H, Hkv, N, D, dims, causal, workspace=ws,
                        workspace_bytes=nbytes)
