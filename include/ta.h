@@ -66,7 +66,11 @@ enum {
     TA_FLAG_NO_TENSOR_CORE = 1u << 0, /* run every hop on the generic CUDA-core kernel        */
     TA_FLAG_NO_HOP_FUSION = 1u << 1,  /* one launch per hop: trailing hops that together fit one  */
                                       /* 128-row tile are not fused into one pass               */
-    TA_FLAG_SAVE_HOPS = 1u << 2       /* store hop inputs X_1..X_{m-1} in the workspace (for ta_backward) */
+    TA_FLAG_SAVE_HOPS = 1u << 2,      /* store hop inputs X_1..X_{m-1} in the workspace (for ta_backward) */
+    TA_FLAG_NO_HOP_OVERLAP = 1u << 3  /* launch every hop fully serialised.  By default a hop's kernel  */
+                                      /* may start on SMs the previous hop has left and prefetch its   */
+                                      /* first Q / K tiles (programmatic dependent launch); it waits    */
+                                      /* for that hop before touching the value tensor.  Same results.  */
 };
 
 /* modes of ta_workspace_bytes */

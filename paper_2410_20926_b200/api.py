@@ -18,7 +18,7 @@ TA_OK = 0
 TA_ERR_INVALID_ARG, TA_ERR_SHAPE, TA_ERR_UNSUPPORTED, TA_ERR_ALIGNMENT = -1, -2, -3, -4
 TA_ERR_WORKSPACE, TA_ERR_ARCH, TA_ERR_CUDA, TA_ERR_TIMEOUT, TA_ERR_TOO_LARGE = -5, -6, -7, -8, -9
 TA_DTYPE_BF16, TA_DTYPE_F32 = 0, 1
-TA_FLAG_NO_TENSOR_CORE, TA_FLAG_NO_HOP_FUSION, TA_FLAG_SAVE_HOPS = 1, 2, 4
+TA_FLAG_NO_TENSOR_CORE, TA_FLAG_NO_HOP_FUSION, TA_FLAG_SAVE_HOPS, TA_FLAG_NO_HOP_OVERLAP = 1, 2, 4, 8
 TA_WS_FORWARD, TA_WS_FORWARD_SAVE, TA_WS_BACKWARD, TA_WS_BACKWARD_F32_GRADS = 0, 1, 2, 3
 
 EXPORTS = ("ta_forward", "ta_forward_f32", "ta_forward_ex", "ta_backward", "ta_workspace_bytes",

@@ -29,6 +29,7 @@ def main(argv=None) -> int:
     ap.add_argument("--rope-base", type=float, default=0.0)
     ap.add_argument("--no-fusion", action="store_true")
     ap.add_argument("--no-tensor-core", action="store_true")
+    ap.add_argument("--no-overlap", action="store_true", help="launch every hop fully serialised")
     ap.add_argument("--f32-grads", action="store_true")
     ap.add_argument("--saved-hops", action="store_true",
                     help="backward: take the hop inputs from a forward run with TA_FLAG_SAVE_HOPS instead of "
@@ -52,7 +53,8 @@ def main(argv=None) -> int:
         return torch.randn(B, heads, N, D, device="cuda", generator=gen).bfloat16()
 
     q, k, v = draw(H), draw(Hkv), draw(Hkv)
-    flags = (ta.TA_FLAG_NO_HOP_FUSION if args.no_fusion else 0) | (ta.TA_FLAG_NO_TENSOR_CORE if args.no_tensor_core else 0)
+    flags = (ta.TA_FLAG_NO_HOP_FUSION if args.no_fusion else 0) | (ta.TA_FLAG_NO_TENSOR_CORE if args.no_tensor_core else 0) \
+        | (ta.TA_FLAG_NO_HOP_OVERLAP if args.no_overlap else 0)
     if args.op == "forward":
         out = torch.empty_like(q)
 

@@ -52,7 +52,8 @@ int build_plan(int B, int H, int H_kv, int N, int D, const int *dims, int ndims,
                unsigned flags, int hop_begin, int hop_end, Plan *plan) {
     int rc = validate_shape(B, H, H_kv, N, D, dims, ndims, dtype);
     if (rc != TA_OK) return rc;
-    if (flags & ~(unsigned)(TA_FLAG_NO_TENSOR_CORE | TA_FLAG_NO_HOP_FUSION | TA_FLAG_SAVE_HOPS | kPlanFlagRope | kPlanFlagLens))
+    if (flags & ~(unsigned)(TA_FLAG_NO_TENSOR_CORE | TA_FLAG_NO_HOP_FUSION | TA_FLAG_SAVE_HOPS | TA_FLAG_NO_HOP_OVERLAP |
+                            kPlanFlagRope | kPlanFlagLens))
         return TA_ERR_UNSUPPORTED;
     if (hop_begin == 0 && hop_end == 0) hop_end = ndims;
     if (hop_begin < 0 || hop_end > ndims || hop_begin > hop_end) return TA_ERR_INVALID_ARG;
@@ -313,6 +314,7 @@ static int forward_impl(const ta_params &p) {
     pb.scale = p.softmax_scale != 0.f ? p.softmax_scale : 1.0f / sqrtf((float)p.D);
     pb.rope_base = p.rope_base;
     pb.seq_lens = p.seq_lens;
+    pb.pdl = 0;
     if ((rc = take_masks(&pb, plan, p.window, p.hop_masks, p.ndims)) != TA_OK) return rc;
     pb.flags = p.flags; pb.hop_begin = p.hop_begin; pb.hop_end = p.hop_end;
     pb.stream = (cudaStream_t)p.stream;
@@ -345,6 +347,7 @@ static int forward_impl(const ta_params &p) {
         const void *xin = buffer(h.src);
         const int xin_heads = h.src == BUF_V ? p.H_kv : p.H;
         void *xout = buffer(h.dst);
+        pb.pdl = (j > 0 && !(p.flags & TA_FLAG_NO_HOP_OVERLAP)) ? 1 : 0;   // follows a hop kernel of this call
         rc = h.path == PATH_TC        ? launch_hop_tc(pb, h, xin, xin_heads, xout)
              : h.path == PATH_TC_LONG ? launch_hop_tc_long(pb, h, xin, xin_heads, xout)
                                       : launch_hop_simt(pb, h, xin, xin_heads, xout);

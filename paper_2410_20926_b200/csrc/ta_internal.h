@@ -65,6 +65,7 @@ struct Problem {
     int window[TA_MAX_DIMS];  // per dimension: 0 = none, w > 0 = keys within w positions of the query
     const unsigned char *masks[TA_MAX_DIMS];  // per dimension: NULL or host n x n bytes, non-zero = visible
     const int *seq_lens;                      // device, B valid lengths, or NULL
+    int pdl;   // 1: this launch follows a hop kernel of the same call in the stream and may overlap its tail
     unsigned flags;
     int hop_begin, hop_end;
     cudaStream_t stream;

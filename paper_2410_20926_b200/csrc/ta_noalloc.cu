@@ -80,6 +80,7 @@ extern "C" int ta_forward_static(const void *q, const void *k, const void *v, vo
     pb.scale = 1.0f / sqrtf((float)D);
     pb.rope_base = 0.f;
     pb.seq_lens = nullptr;
+    pb.pdl = 0;
     for (int i = 0; i < TA_MAX_DIMS; ++i) { pb.window[i] = 0; pb.masks[i] = nullptr; }
     pb.flags = 0; pb.hop_begin = 0; pb.hop_end = ndims;
     pb.stream = (cudaStream_t)stream;
@@ -90,6 +91,7 @@ extern "C" int ta_forward_static(const void *q, const void *k, const void *v, vo
         const void *xin = h.src == BUF_V ? v : (h.src == BUF_OUT ? (const void *)out : (const void *)scratch);
         void *xout = h.dst == BUF_OUT ? out : scratch;
         const int xin_heads = h.src == BUF_V ? H_kv : H;
+        pb.pdl = j > 0 ? 1 : 0;
         rc = h.path == PATH_TC        ? launch_hop_tc(pb, h, xin, xin_heads, xout)
              : h.path == PATH_TC_LONG ? launch_hop_tc_long(pb, h, xin, xin_heads, xout)
                                       : launch_hop_simt(pb, h, xin, xin_heads, xout);

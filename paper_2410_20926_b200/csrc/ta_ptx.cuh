@@ -223,4 +223,12 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 
 
 }  // namespace
+// Programmatic dependent launch: a kernel launched with the programmatic-stream-serialization
+// attribute may start while its predecessor in the stream is still draining; griddep_wait()
+// returns once the predecessor has completed and its writes are visible (at once if the launch
+// carries no such dependency).  griddep_launch_dependents() lets the successor be scheduled as
+// soon as every CTA of this grid has issued it (or exited).
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 }  // namespace ta

@@ -152,6 +152,9 @@ hop_pipe_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    // every CTA of this (persistent, fully resident) grid is running: the next hop's kernel may be
+    // scheduled on SMs as they drain; it touches nothing this hop writes before its own wait
+    if (tid == 0) griddep_launch_dependents();
 
     // tiles this CTA processes: its work items (round robin over the grid) x gi heads each
     const long long my_items = (a.total_items - blockIdx.x + gridDim.x - 1) / gridDim.x;
@@ -169,6 +172,7 @@ hop_pipe_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 last_par = parity ? (last_par | bit) : (last_par & ~bit);
             };
             bool ok = true;
+            bool prev_hop_done = false;   // Q and K are inputs of the call; the value tensor is the previous hop's output
             for (long long item = blockIdx.x; ok && item < a.total_items; item += gridDim.x, ++it) {
                 const ItemCoord c = decode_item(a, item);
                 const int ks = it & 1;
@@ -196,6 +200,10 @@ hop_pipe_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     const uint32_t xpar = (t / kNX) & 1;
                     ok = mbar_wait_abortable(x_free(xs), xpar ^ 1, 0x12, abort_flag);
                     if (!ok) break;
+                    if (!prev_hop_done) {
+                        griddep_wait();
+                        prev_hop_done = true;
+                    }
                     mbar_expect_tx(x_full(xs), kHalves * slab_tx);
                     arm(16u << xs, xpar);
 #pragma unroll
@@ -542,19 +550,37 @@ int launch_d(const Problem &pb, const HopDesc &hd, const void *xin, int xin_head
             return TA_ERR_CUDA;
         configured = true;
     }
+    // A hop that follows another hop kernel of the same call is launched with programmatic stream
+    // serialization: its CTAs may start on SMs the previous hop has left and fetch their first K and
+    // Q tiles (inputs of the call) while that hop drains; they wait for it before touching the
+    // value tensor.  The saving is a fixed few microseconds per hop boundary (3.5 % of a 0.4 ms
+    // call), so it is used for short hops only: on hops of more than 32 work items per CTA it
+    // measured within noise, and slightly negative on the 128k-token shape.
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(pb.rope_base > 0.f ? kThreadsRope : kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = pb.stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = (pb.pdl && a.total_items <= 32ll * num_sms) ? 1 : 0;
+    cudaError_t err;
     if (pb.masks[hd.hop] || pb.seq_lens) {
         HopMask hm;                                  // explicit mask ^ causal flag ^ window, by value
         const int rc = build_hop_mask(pb, hd, &hm);
         if (rc != TA_OK) return rc;
         if (pb.rope_base > 0.f)
-            hop_pipe_kernel<D, true, true><<<grid, kThreadsRope, smem, pb.stream>>>(mq, mk, mxi, mxo, a, hm);
+            err = cudaLaunchKernelEx(&cfg, hop_pipe_kernel<D, true, true>, mq, mk, mxi, mxo, a, hm);
         else
-            hop_pipe_kernel<D, false, true><<<grid, kThreads, smem, pb.stream>>>(mq, mk, mxi, mxo, a, hm);
+            err = cudaLaunchKernelEx(&cfg, hop_pipe_kernel<D, false, true>, mq, mk, mxi, mxo, a, hm);
     } else if (pb.rope_base > 0.f) {
-        hop_pipe_kernel<D, true, false><<<grid, kThreadsRope, smem, pb.stream>>>(mq, mk, mxi, mxo, a, NoMask{});
+        err = cudaLaunchKernelEx(&cfg, hop_pipe_kernel<D, true, false>, mq, mk, mxi, mxo, a, NoMask{});
     } else {
-        hop_pipe_kernel<D, false, false><<<grid, kThreads, smem, pb.stream>>>(mq, mk, mxi, mxo, a, NoMask{});
+        err = cudaLaunchKernelEx(&cfg, hop_pipe_kernel<D, false, false>, mq, mk, mxi, mxo, a, NoMask{});
     }
+    if (err != cudaSuccess) return TA_ERR_CUDA;
     count_launch();
     return cudaPeekAtLastError() == cudaSuccess ? TA_OK : TA_ERR_CUDA;
 }

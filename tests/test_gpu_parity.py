@@ -184,3 +184,23 @@ def test_forward_host_back_to_back_calls_use_both_staging_sets():
     ta.ta_device_status()
     for (host, out_h), ref in zip(outs, refs):
         np.testing.assert_array_equal(out_h.float().numpy(), ref)
+
+
+@pytest.mark.parametrize("B,H,Hkv,D,dims,causal,kw", [
+    (1, 4, 2, 128, [8, 16, 32], True, {}),
+    (2, 8, 2, 64, [16, 4, 4, 4], False, {}),
+    (1, 16, 4, 128, [32, 32, 32], True, {}),
+    (1, 4, 2, 128, [16, 8, 64], True, {"rope_base": 10000.0}),
+    (1, 4, 2, 128, [4, 300, 16], True, {}),          # short, long, short segments
+])
+def test_overlapped_hop_launches_give_identical_results(B, H, Hkv, D, dims, causal, kw):
+    """A hop's kernel may start while the previous hop drains (it prefetches Q and K, then waits
+    for that hop before it touches the value tensor).  Repeated runs must reproduce, bit for
+    bit, the run whose launches are fully serialised."""
+    N = math.prod(dims)
+    inp = ta_inputs.make_inputs(B, H, Hkv, N, D, "bf16", 130)
+    base = ta.TA_FLAG_NO_HOP_FUSION
+    ref = gpu_forward(inp, B, H, Hkv, N, D, dims, causal, "bf16", base | ta.TA_FLAG_NO_HOP_OVERLAP, **kw)
+    for _ in range(10):
+        got = gpu_forward(inp, B, H, Hkv, N, D, dims, causal, "bf16", base, **kw)
+        np.testing.assert_array_equal(got, ref)
