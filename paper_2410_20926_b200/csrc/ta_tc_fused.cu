@@ -173,6 +173,7 @@ hop_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 last_par = parity ? (last_par | bit) : (last_par & ~bit);
             };
             bool ok = true;
+            bool prev_hop_done = false;
             for (long long item = blockIdx.x; ok && item < a.total_items; item += gridDim.x, ++it) {
                 const FusedItem c = decode_fused_item(a, item);
                 const int ks = it & 1;
@@ -200,6 +201,10 @@ hop_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                     const uint32_t xpar = (t / kNX) & 1;
                     ok = mbar_wait_abortable(x_free(xs), xpar ^ 1, 0x92, abort_flag);
                     if (!ok) break;
+                    if (!prev_hop_done) {      // launched while the previous hop drains: its output is read from here on
+                        griddep_wait();
+                        prev_hop_done = true;
+                    }
                     mbar_expect_tx(x_full(xs), kHalves * slab_tx);
                     arm(16u << xs, xpar);
 #pragma unroll
@@ -483,7 +488,18 @@ int launch_fused_d(const Problem &pb, const HopDesc &hd, const void *xin, int xi
         configured = true;
     }
     const unsigned grid = (unsigned)(a.total_items < num_sms ? a.total_items : num_sms);
-    kern<<<grid, kThreads, smem, pb.stream>>>(mq, mk, mxi, mxo, a);
+    // after another hop of the same call: may start while that hop drains (see launch_hop_tc)
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = pb.stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = (pb.pdl && a.total_items <= 32ll * num_sms) ? 1 : 0;
+    if (cudaLaunchKernelEx(&cfg, kern, mq, mk, mxi, mxo, a) != cudaSuccess) return TA_ERR_CUDA;
     count_launch();
     return cudaPeekAtLastError() == cudaSuccess ? TA_OK : TA_ERR_CUDA;
 }

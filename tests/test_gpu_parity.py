@@ -192,6 +192,7 @@ def test_forward_host_back_to_back_calls_use_both_staging_sets():
     (1, 16, 4, 128, [32, 32, 32], True, {}),
     (1, 4, 2, 128, [16, 8, 64], True, {"rope_base": 10000.0}),
     (1, 4, 2, 128, [4, 300, 16], True, {}),          # short, long, short segments
+    (2, 8, 2, 128, [16, 4, 4, 4], False, {"fused": True}),   # the fused pass follows hop 0
 ])
 def test_overlapped_hop_launches_give_identical_results(B, H, Hkv, D, dims, causal, kw):
     """A hop's kernel may start while the previous hop drains (it prefetches Q and K, then waits
@@ -199,7 +200,10 @@ def test_overlapped_hop_launches_give_identical_results(B, H, Hkv, D, dims, caus
     bit, the run whose launches are fully serialised."""
     N = math.prod(dims)
     inp = ta_inputs.make_inputs(B, H, Hkv, N, D, "bf16", 130)
-    base = ta.TA_FLAG_NO_HOP_FUSION
+    kw = dict(kw)
+    base = 0 if kw.pop("fused", False) else ta.TA_FLAG_NO_HOP_FUSION
+    if base == 0:
+        assert "tc-fused" in ta.ta_plan_describe(B, H, Hkv, N, D, dims, causal, ta.TA_DTYPE_BF16, 0)
     ref = gpu_forward(inp, B, H, Hkv, N, D, dims, causal, "bf16", base | ta.TA_FLAG_NO_HOP_OVERLAP, **kw)
     for _ in range(10):
         got = gpu_forward(inp, B, H, Hkv, N, D, dims, causal, "bf16", base, **kw)
