@@ -27,6 +27,11 @@
  *     aborted.  On an error return no kernel has been launched by that call.
  *   - Hops with n_i == 1 are identities and are skipped.  ndims == 1 is ordinary attention.
  *   - Kernels are built for sm_100a only; on another device the calls return TA_ERR_ARCH.
+ *   - Host threads: the calls may be made from several threads at once, on the same or on
+ *     different streams and devices (the calling thread's current device is used).  Two calls
+ *     whose kernels can overlap on the GPU must not share memory they write; that includes the
+ *     library-owned scratch tensor used when `workspace` is NULL and a problem mixes kernels
+ *     (ta_workspace_bytes(.., TA_WS_FORWARD) != 0): give such concurrent calls a workspace each.
  */
 #ifndef TA_B200_H
 #define TA_B200_H
@@ -291,6 +296,11 @@ unsigned long long ta_launch_count(void);
 
 /* Frees device memory the library holds (staging and scratch arenas).  Synchronises. */
 int ta_release(void);
+
+/* The CUDA runtime error code (cudaError_t as int) behind the last TA_ERR_CUDA that
+ * ta_forward*, ta_backward* returned to the calling host thread; 0 if none.  A value
+ * <= -1000 is -(1000 + CUresult) of the driver's tensor-map encoder (-1000: encoder not found). */
+int ta_last_cuda_error(void);
 
 const char *ta_status_string(int status);
 int ta_version(void);

@@ -23,14 +23,18 @@ TA_WS_FORWARD, TA_WS_FORWARD_SAVE, TA_WS_BACKWARD, TA_WS_BACKWARD_F32_GRADS = 0,
 
 EXPORTS = ("ta_forward", "ta_forward_f32", "ta_forward_ex", "ta_backward", "ta_workspace_bytes",
            "ta_forward_host", "ta_plan_describe", "ta_device_status", "ta_launch_count",
-           "ta_release", "ta_status_string", "ta_version", "ta_forward_static", "ta_backward_ex")
+           "ta_release", "ta_status_string", "ta_version", "ta_forward_static", "ta_backward_ex",
+           "ta_last_cuda_error")
 TA_STATIC_SCRATCH_BYTES = 16 << 20
 
 
 class TaError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
-        super().__init__(f"{where} failed: {status} ({ta_status_string(status)})")
+        detail = ta_status_string(status)
+        if status == TA_ERR_CUDA:
+            detail += f", cudaError {ta_last_cuda_error()}"
+        super().__init__(f"{where} failed: {status} ({detail})")
 
 
 class ta_params(ctypes.Structure):
@@ -102,6 +106,8 @@ def load():
     lib.ta_release.argtypes = []
     lib.ta_status_string.argtypes = [ci]
     lib.ta_status_string.restype = ctypes.c_char_p
+    lib.ta_last_cuda_error.argtypes = []
+    lib.ta_last_cuda_error.restype = ctypes.c_int
     lib.ta_version.argtypes = []
     for name in EXPORTS:
         getattr(lib, name)          # every symbol of include/ta.h must be exported
@@ -143,6 +149,11 @@ def _done(status: int, where: str, check: bool) -> int:
 
 def ta_status_string(status: int) -> str:
     return load().ta_status_string(int(status)).decode()
+
+
+def ta_last_cuda_error() -> int:
+    """cudaError_t behind the last TA_ERR_CUDA this thread got from a forward / backward call."""
+    return int(load().ta_last_cuda_error())
 
 
 def ta_version() -> int:

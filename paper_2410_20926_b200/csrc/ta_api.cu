@@ -11,6 +11,7 @@
 namespace ta {
 
 static std::atomic<unsigned long long> g_launches{0};
+thread_local int tl_last_cuda_error = 0;
 void count_launch(unsigned n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
 int validate_shape(int B, int H, int H_kv, int N, int D, const int *dims, int ndims, int dtype) {
@@ -144,6 +145,18 @@ int build_plan(int B, int H, int H_kv, int N, int D, const int *dims, int ndims,
         if (plan->hops[j].src == BUF_SCRATCH || plan->hops[j].dst == BUF_SCRATCH) plan->need_scratch = true;
     if (plan->need_scratch) plan->scratch_bytes = tensor_bytes;
     return TA_OK;
+}
+
+int current_device_sms(int *dev) {
+    static std::atomic<int> cache[64];
+    int d = 0;
+    if (cudaGetDevice(&d) != cudaSuccess) d = 0;
+    if (dev) *dev = d;
+    int n = (d >= 0 && d < 64) ? cache[d].load(std::memory_order_relaxed) : 0;
+    if (n > 0) return n;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, d) != cudaSuccess || n <= 0) n = 148;
+    if (d >= 0 && d < 64) cache[d].store(n, std::memory_order_relaxed);
+    return n;
 }
 
 int build_hop_mask(const Problem &pb, const HopDesc &hd, HopMask *hm) {
@@ -360,11 +373,20 @@ static int forward_impl(const ta_params &p) {
 
 using namespace ta;
 
+// Result of an entry point: remembers which CUDA error stands behind a TA_ERR_CUDA.
+static int finish(int rc) {
+    if (rc == TA_ERR_CUDA && tl_last_cuda_error == 0) tl_last_cuda_error = (int)cudaPeekAtLastError();
+    return rc;
+}
+
 extern "C" {
+
+int ta_last_cuda_error(void) { return tl_last_cuda_error; }
 
 int ta_forward_ex(const ta_params *p) {
     if (!p || p->struct_bytes != sizeof(ta_params)) return TA_ERR_INVALID_ARG;
-    return forward_impl(*p);
+    tl_last_cuda_error = 0;
+    return finish(forward_impl(*p));
 }
 
 static int forward_simple(const void *q, const void *k, const void *v, void *out, int B, int H, int H_kv,
@@ -377,7 +399,8 @@ static int forward_simple(const void *q, const void *k, const void *v, void *out
     p.B = B; p.H = H; p.H_kv = H_kv; p.N = N; p.D = D;
     p.dims = dims; p.ndims = ndims; p.causal = causal; p.dtype = dtype;
     p.stream = stream;
-    return forward_impl(p);
+    tl_last_cuda_error = 0;
+    return finish(forward_impl(p));
 }
 
 int ta_forward(const void *q, const void *k, const void *v, void *out, int B, int H, int H_kv, int N, int D,
@@ -449,7 +472,8 @@ int ta_forward_host(const void *qh, const void *kh, const void *vh, void *outh, 
 
 int ta_backward_ex(const ta_bwd_params *p) {
     if (!p || p->struct_bytes != sizeof(ta_bwd_params)) return TA_ERR_INVALID_ARG;
-    return backward_impl(*p);
+    tl_last_cuda_error = 0;
+    return finish(backward_impl(*p));
 }
 
 int ta_backward(const void *dout, const void *q, const void *k, const void *v, const void *out, void *dq,
@@ -463,7 +487,8 @@ int ta_backward(const void *dout, const void *q, const void *k, const void *v, c
     p.B = B; p.H = H; p.H_kv = H_kv; p.N = N; p.D = D; p.dims = dims; p.ndims = ndims; p.causal = causal;
     p.dtype = TA_DTYPE_BF16; p.grad_dtype = TA_DTYPE_BF16;
     p.workspace = workspace; p.workspace_bytes = workspace_bytes; p.stream = stream;
-    return backward_impl(p);
+    tl_last_cuda_error = 0;
+    return finish(backward_impl(p));
 }
 
 static const char *buf_name(int id) {

@@ -6,6 +6,8 @@
 #include <stddef.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "ta.h"
 
 namespace ta {
@@ -131,5 +133,47 @@ int make_view_map(CUtensorMap *map, const void *base, int heads_total, int N, in
 int read_status_tc_forward(unsigned int *word);
 int read_status_tc_backward(unsigned int *word);
 int read_status_tc_fused(unsigned int *word);
+
+// CUDA error code seen by the last call of this host thread that returned TA_ERR_CUDA.
+extern thread_local int tl_last_cuda_error;
+inline int cuda_fail(cudaError_t e) {
+    tl_last_cuda_error = (int)e;
+    return TA_ERR_CUDA;
+}
+
+// Every kernel of the library is launched through here: the launch's own return value decides
+// (an error some earlier CUDA call left behind in this thread is neither consumed nor mistaken
+// for ours).  overlap_prev: programmatic stream serialization -- the kernel may be scheduled
+// while the previous kernel in the stream drains and must execute griddepcontrol.wait before it
+// touches anything that kernel writes.
+template <typename... KArgs, typename... Args>
+inline int launch_kernel(void (*kern)(KArgs...), unsigned grid, unsigned block, size_t smem, cudaStream_t stream,
+                         bool overlap_prev, Args &&...args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = overlap_prev ? 1 : 0;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, static_cast<Args &&>(args)...);
+    if (e != cudaSuccess) return cuda_fail(e);
+    count_launch();
+    return TA_OK;
+}
+
+// SM count of the calling thread's current device (looked up once per device); *dev gets its ordinal.
+int current_device_sms(int *dev);
+
+// "Configured once per device" marker for a launcher's kernel attributes (the maximum dynamic
+// shared memory of a function is a per-device setting).  Ordinals beyond 63 configure on every call.
+struct PerDeviceOnce {
+    std::atomic<unsigned long long> done{0};
+    bool is_done(int dev) const { return dev >= 0 && dev < 64 && ((done.load(std::memory_order_acquire) >> dev) & 1ull); }
+    void mark(int dev) { if (dev >= 0 && dev < 64) done.fetch_or(1ull << dev, std::memory_order_release); }
+};
 
 }  // namespace ta

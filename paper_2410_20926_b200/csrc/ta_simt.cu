@@ -231,10 +231,8 @@ int launch_t(const Problem &pb, const HopDesc &hd, const void *xin, int xin_head
             return TA_ERR_CUDA;
     }
     long long grid = a.items < (1ll << 20) ? a.items : (1ll << 20);
-    kern<<<(unsigned)grid, kThreads, smem, pb.stream>>>((const T *)pb.q, (const T *)pb.k, (const T *)xin,
-                                                       (T *)xout, a, hm);
-    count_launch();
-    return cudaPeekAtLastError() == cudaSuccess ? TA_OK : TA_ERR_CUDA;
+    return launch_kernel(kern, (unsigned)grid, kThreads, smem, pb.stream, false, (const T *)pb.q, (const T *)pb.k,
+                         (const T *)xin, (T *)xout, a, hm);
 }
 
 template <typename T>
@@ -260,13 +258,10 @@ int launch_broadcast_kv(const Problem &pb) {
     const long long total = per_head * pb.B * pb.H;
     const unsigned grid = (unsigned)((total + 255) / 256 < 148 * 16 ? (total + 255) / 256 : 148 * 16);
     if (pb.dtype == TA_DTYPE_F32)
-        broadcast_kv_kernel<float><<<grid, 256, 0, pb.stream>>>((const float *)pb.v, (float *)pb.out, per_head,
-                                                                pb.H, pb.H_kv, total, pb.seq_lens, pb.D);
-    else
-        broadcast_kv_kernel<__nv_bfloat16><<<grid, 256, 0, pb.stream>>>(
-            (const __nv_bfloat16 *)pb.v, (__nv_bfloat16 *)pb.out, per_head, pb.H, pb.H_kv, total, pb.seq_lens, pb.D);
-    count_launch();
-    return cudaPeekAtLastError() == cudaSuccess ? TA_OK : TA_ERR_CUDA;
+        return launch_kernel(broadcast_kv_kernel<float>, grid, 256, 0, pb.stream, false, (const float *)pb.v,
+                             (float *)pb.out, per_head, pb.H, pb.H_kv, total, pb.seq_lens, pb.D);
+    return launch_kernel(broadcast_kv_kernel<__nv_bfloat16>, grid, 256, 0, pb.stream, false, (const __nv_bfloat16 *)pb.v,
+                         (__nv_bfloat16 *)pb.out, per_head, pb.H, pb.H_kv, total, pb.seq_lens, pb.D);
 }
 
 }  // namespace ta

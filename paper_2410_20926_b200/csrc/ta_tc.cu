@@ -488,7 +488,10 @@ int make_hop_map(CUtensorMap *map, const void *base, int heads_total, int N, int
 int make_view_map(CUtensorMap *map, const void *base, int heads_total, int N, int D, const HopDesc &hd, int elem,
                   int box_t, int box_inner, int box_outer) {
     EncodeTiledFn enc = encode_fn();
-    if (!enc) return TA_ERR_CUDA;
+    if (!enc) {
+        tl_last_cuda_error = -1000;
+        return TA_ERR_CUDA;
+    }
     const cuuint64_t e = (cuuint64_t)elem;
     cuuint64_t gdim[5] = {(cuuint64_t)D, (cuuint64_t)hd.n, (cuuint64_t)hd.stride, (cuuint64_t)hd.outer,
                           (cuuint64_t)heads_total};
@@ -496,10 +499,28 @@ int make_view_map(CUtensorMap *map, const void *base, int heads_total, int N, in
                           (cuuint64_t)N * D * e};
     cuuint32_t box[5] = {(cuuint32_t)(128 / elem), (cuuint32_t)box_t, (cuuint32_t)box_inner, (cuuint32_t)box_outer, 1u};
     cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    // The encoder is a driver call and needs a context current on this host thread; a thread whose
+    // first CUDA activity is this library (its caller's streams and buffers may all come from
+    // pools filled by other threads) has none until a runtime call binds the primary context.
+    static thread_local bool context_bound = false;
+    if (!context_bound) {
+        cudaFree(nullptr);
+        context_bound = true;
+    }
     CUresult r = enc(map, elem == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 5,
                      const_cast<void *>(base), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                      CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS ? TA_OK : TA_ERR_CUDA;
+    if (r == CUDA_ERROR_INVALID_CONTEXT) {   // e.g. the thread's context was popped since: bind and retry once
+        cudaFree(nullptr);
+        r = enc(map, elem == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 5,
+                const_cast<void *>(base), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    }
+    if (r != CUDA_SUCCESS) {
+        tl_last_cuda_error = -1000 - (int)r;   // a driver (CUresult) code, not a runtime one
+        return TA_ERR_CUDA;
+    }
+    return TA_OK;
 }
 
 namespace {
@@ -513,13 +534,8 @@ int launch_d(const Problem &pb, const HopDesc &hd, const void *xin, int xin_head
     if ((rc = make_hop_map(&mxi, xin, pb.B * xin_heads, pb.N, D, hd, 2)) != TA_OK) return rc;
     if ((rc = make_hop_map(&mxo, xout, pb.B * pb.H, pb.N, D, hd, 2)) != TA_OK) return rc;
 
-    static int num_sms = 0;
-    if (num_sms == 0) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        if (cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || num_sms <= 0)
-            num_sms = 148;
-    }
+    int dev = 0;
+    const int num_sms = current_device_sms(&dev);
     TcArgs a;
     a.n = hd.n; a.rows = hd.rows; a.ci = hd.ci; a.co = hd.co; a.causal = pb.causal;
     a.g = pb.H / pb.H_kv; a.H = pb.H; a.H_kv = pb.H_kv; a.xin_is_kv = xin_heads != pb.H ? 1 : 0;
@@ -540,15 +556,15 @@ int launch_d(const Problem &pb, const HopDesc &hd, const void *xin, int xin_head
 
     constexpr size_t smem = PipeCfg<D>::kSmemBytes;
     const unsigned grid = (unsigned)(a.total_items < num_sms ? a.total_items : num_sms);
-    static bool configured = false;
-    if (!configured) {
+    static PerDeviceOnce configured;
+    if (!configured.is_done(dev)) {
         const cudaFuncAttribute attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
         if (cudaFuncSetAttribute(hop_pipe_kernel<D, false, false>, attr, (int)smem) != cudaSuccess ||
             cudaFuncSetAttribute(hop_pipe_kernel<D, true, false>, attr, (int)smem) != cudaSuccess ||
             cudaFuncSetAttribute(hop_pipe_kernel<D, false, true>, attr, (int)smem) != cudaSuccess ||
             cudaFuncSetAttribute(hop_pipe_kernel<D, true, true>, attr, (int)smem) != cudaSuccess)
             return TA_ERR_CUDA;
-        configured = true;
+        configured.mark(dev);
     }
     // A hop that follows another hop kernel of the same call is launched with programmatic stream
     // serialization: its CTAs may start on SMs the previous hop has left and fetch their first K and
@@ -556,33 +572,22 @@ int launch_d(const Problem &pb, const HopDesc &hd, const void *xin, int xin_head
     // value tensor.  The saving is a fixed few microseconds per hop boundary (3.5 % of a 0.4 ms
     // call), so it is used for short hops only: on hops of more than 32 work items per CTA it
     // measured within noise, and slightly negative on the 128k-token shape.
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(grid);
-    cfg.blockDim = dim3(pb.rope_base > 0.f ? kThreadsRope : kThreads);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = pb.stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = (pb.pdl && a.total_items <= 32ll * num_sms) ? 1 : 0;
-    cudaError_t err;
+    const bool overlap = pb.pdl && a.total_items <= 32ll * num_sms;
     if (pb.masks[hd.hop] || pb.seq_lens) {
         HopMask hm;                                  // explicit mask ^ causal flag ^ window, by value
         const int rc = build_hop_mask(pb, hd, &hm);
         if (rc != TA_OK) return rc;
         if (pb.rope_base > 0.f)
-            err = cudaLaunchKernelEx(&cfg, hop_pipe_kernel<D, true, true>, mq, mk, mxi, mxo, a, hm);
-        else
-            err = cudaLaunchKernelEx(&cfg, hop_pipe_kernel<D, false, true>, mq, mk, mxi, mxo, a, hm);
-    } else if (pb.rope_base > 0.f) {
-        err = cudaLaunchKernelEx(&cfg, hop_pipe_kernel<D, true, false>, mq, mk, mxi, mxo, a, NoMask{});
-    } else {
-        err = cudaLaunchKernelEx(&cfg, hop_pipe_kernel<D, false, false>, mq, mk, mxi, mxo, a, NoMask{});
+            return launch_kernel(hop_pipe_kernel<D, true, true>, grid, kThreadsRope, smem, pb.stream, overlap, mq, mk, mxi,
+                                 mxo, a, hm);
+        return launch_kernel(hop_pipe_kernel<D, false, true>, grid, kThreads, smem, pb.stream, overlap, mq, mk, mxi, mxo, a,
+                             hm);
     }
-    if (err != cudaSuccess) return TA_ERR_CUDA;
-    count_launch();
-    return cudaPeekAtLastError() == cudaSuccess ? TA_OK : TA_ERR_CUDA;
+    if (pb.rope_base > 0.f)
+        return launch_kernel(hop_pipe_kernel<D, true, false>, grid, kThreadsRope, smem, pb.stream, overlap, mq, mk, mxi, mxo,
+                             a, NoMask{});
+    return launch_kernel(hop_pipe_kernel<D, false, false>, grid, kThreads, smem, pb.stream, overlap, mq, mk, mxi, mxo, a,
+                         NoMask{});
 }
 
 }  // namespace

@@ -622,23 +622,18 @@ int launch_bwd_d(const Problem &pb, const HopDesc &hd, const void *x, int x_head
     a.stride = (int)hd.stride;
     a.lens = pb.seq_lens;
 
-    static int num_sms = 0;
-    if (num_sms == 0) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        if (cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || num_sms <= 0)
-            num_sms = 148;
-    }
+    int dev = 0;
+    const int num_sms = current_device_sms(&dev);
     constexpr size_t smem = BwdCfg<D>::kSmemBytes;
-    static bool configured = false;
-    if (!configured) {
+    static PerDeviceOnce configured;
+    if (!configured.is_done(dev)) {
         const cudaFuncAttribute attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
         if (cudaFuncSetAttribute(hop_tc_bwd_kernel<D, false, false>, attr, (int)smem) != cudaSuccess ||
             cudaFuncSetAttribute(hop_tc_bwd_kernel<D, true, false>, attr, (int)smem) != cudaSuccess ||
             cudaFuncSetAttribute(hop_tc_bwd_kernel<D, false, true>, attr, (int)smem) != cudaSuccess ||
             cudaFuncSetAttribute(hop_tc_bwd_kernel<D, true, true>, attr, (int)smem) != cudaSuccess)
             return TA_ERR_CUDA;
-        configured = true;
+        configured.mark(dev);
     }
     const unsigned grid = (unsigned)(a.total_items < num_sms ? a.total_items : num_sms);
     if (pb.masks[hd.hop] || pb.seq_lens) {
@@ -646,16 +641,16 @@ int launch_bwd_d(const Problem &pb, const HopDesc &hd, const void *x, int x_head
         const int rc = build_hop_mask(pb, hd, &hm);
         if (rc != TA_OK) return rc;
         if (pb.rope_base > 0.f)
-            hop_tc_bwd_kernel<D, true, true><<<grid, kThreadsRope, smem, pb.stream>>>(mq, mk, mx, mgi, mgo, mdq, mdk, mdv, a, hm);
-        else
-            hop_tc_bwd_kernel<D, false, true><<<grid, kThreads, smem, pb.stream>>>(mq, mk, mx, mgi, mgo, mdq, mdk, mdv, a, hm);
-    } else if (pb.rope_base > 0.f) {
-        hop_tc_bwd_kernel<D, true, false><<<grid, kThreadsRope, smem, pb.stream>>>(mq, mk, mx, mgi, mgo, mdq, mdk, mdv, a, NoMask{});
-    } else {
-        hop_tc_bwd_kernel<D, false, false><<<grid, kThreads, smem, pb.stream>>>(mq, mk, mx, mgi, mgo, mdq, mdk, mdv, a, NoMask{});
+            return launch_kernel(hop_tc_bwd_kernel<D, true, true>, grid, kThreadsRope, smem, pb.stream, false, mq, mk, mx,
+                                 mgi, mgo, mdq, mdk, mdv, a, hm);
+        return launch_kernel(hop_tc_bwd_kernel<D, false, true>, grid, kThreads, smem, pb.stream, false, mq, mk, mx, mgi,
+                             mgo, mdq, mdk, mdv, a, hm);
     }
-    count_launch();
-    return cudaPeekAtLastError() == cudaSuccess ? TA_OK : TA_ERR_CUDA;
+    if (pb.rope_base > 0.f)
+        return launch_kernel(hop_tc_bwd_kernel<D, true, false>, grid, kThreadsRope, smem, pb.stream, false, mq, mk, mx, mgi,
+                             mgo, mdq, mdk, mdv, a, NoMask{});
+    return launch_kernel(hop_tc_bwd_kernel<D, false, false>, grid, kThreads, smem, pb.stream, false, mq, mk, mx, mgi, mgo,
+                         mdq, mdk, mdv, a, NoMask{});
 }
 
 }  // namespace
@@ -674,9 +669,7 @@ int launch_f32_to_bf16(const float *src, void *dst, long long n, cudaStream_t st
     long long blocks = (n / 4 + 255) / 256;
     if (blocks > 148 * 32) blocks = 148 * 32;
     if (blocks < 1) blocks = 1;
-    f32_to_bf16_kernel<<<(unsigned)blocks, 256, 0, stream>>>(src, (__nv_bfloat16 *)dst, n);
-    count_launch();
-    return cudaPeekAtLastError() == cudaSuccess ? TA_OK : TA_ERR_CUDA;
+    return launch_kernel(f32_to_bf16_kernel, (unsigned)blocks, 256, 0, stream, false, src, (__nv_bfloat16 *)dst, n);
 }
 
 int launch_group_sum(const void *dout, void *dv, int dv_is_f32, int B, int H, int H_kv, long long per_head,
@@ -685,13 +678,10 @@ int launch_group_sum(const void *dout, void *dv, int dv_is_f32, int B, int H, in
     long long blocks = (total + 255) / 256;
     if (blocks > 148 * 32) blocks = 148 * 32;
     if (dv_is_f32)
-        group_sum_kernel<float><<<(unsigned)blocks, 256, 0, stream>>>((const __nv_bfloat16 *)dout, (float *)dv, per_head,
-                                                                     H, H_kv, total);
-    else
-        group_sum_kernel<__nv_bfloat16><<<(unsigned)blocks, 256, 0, stream>>>(
-            (const __nv_bfloat16 *)dout, (__nv_bfloat16 *)dv, per_head, H, H_kv, total);
-    count_launch();
-    return cudaPeekAtLastError() == cudaSuccess ? TA_OK : TA_ERR_CUDA;
+        return launch_kernel(group_sum_kernel<float>, (unsigned)blocks, 256, 0, stream, false, (const __nv_bfloat16 *)dout,
+                             (float *)dv, per_head, H, H_kv, total);
+    return launch_kernel(group_sum_kernel<__nv_bfloat16>, (unsigned)blocks, 256, 0, stream, false,
+                         (const __nv_bfloat16 *)dout, (__nv_bfloat16 *)dv, per_head, H, H_kv, total);
 }
 
 int read_status_tc_backward(unsigned int *word) {

@@ -463,13 +463,8 @@ int launch_fused_d(const Problem &pb, const HopDesc &hd, const void *xin, int xi
         a.sub_stride[f] = f < hd.nf ? hd.sub_stride[f] : 1;
         a.sub_window[f] = f < hd.nf ? pb.window[hd.sub_hop[f]] : 0;
     }
-    static int num_sms = 0;
-    if (num_sms == 0) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        if (cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || num_sms <= 0)
-            num_sms = 148;
-    }
+    int dev = 0;
+    const int num_sms = current_device_sms(&dev);
     a.tiles_outer = hd.tiles_outer;
     // a work item = the gi query heads of a GQA group on one tile position (they share the K tile)
     const long long positions = (long long)pb.B * pb.H_kv * hd.tiles_outer;
@@ -481,27 +476,16 @@ int launch_fused_d(const Problem &pb, const HopDesc &hd, const void *xin, int xi
     a.scale_log2 = pb.scale * 1.4426950408889634f;
     constexpr size_t smem = FusedCfg<D>::kSmemBytes;
     auto kern = hop_fused_kernel<D>;
-    static bool configured = false;
-    if (!configured) {
+    static PerDeviceOnce configured;
+    if (!configured.is_done(dev)) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
             return TA_ERR_CUDA;
-        configured = true;
+        configured.mark(dev);
     }
     const unsigned grid = (unsigned)(a.total_items < num_sms ? a.total_items : num_sms);
     // after another hop of the same call: may start while that hop drains (see launch_hop_tc)
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(grid);
-    cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = pb.stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = (pb.pdl && a.total_items <= 32ll * num_sms) ? 1 : 0;
-    if (cudaLaunchKernelEx(&cfg, kern, mq, mk, mxi, mxo, a) != cudaSuccess) return TA_ERR_CUDA;
-    count_launch();
-    return cudaPeekAtLastError() == cudaSuccess ? TA_OK : TA_ERR_CUDA;
+    const bool overlap = pb.pdl && a.total_items <= 32ll * num_sms;
+    return launch_kernel(kern, grid, kThreads, smem, pb.stream, overlap, mq, mk, mxi, mxo, a);
 }
 
 }  // namespace

@@ -495,30 +495,24 @@ int launch_long_d(const Problem &pb, const HopDesc &hd, const void *xin, int xin
     a.window = pb.window[hd.hop];
     a.scale_log2 = pb.scale * 1.4426950408889634f;
 
-    static int num_sms = 0;
-    if (num_sms == 0) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        if (cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || num_sms <= 0)
-            num_sms = 148;
-    }
+    int dev = 0;
+    const int num_sms = current_device_sms(&dev);
     constexpr size_t smem = LongCfg<D>::kSmemBytes;
-    static bool configured = false;
-    if (!configured) {
+    static PerDeviceOnce configured;
+    if (!configured.is_done(dev)) {
         if (cudaFuncSetAttribute(hop_long_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
                 cudaSuccess ||
             cudaFuncSetAttribute(hop_long_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
                 cudaSuccess)
             return TA_ERR_CUDA;
-        configured = true;
+        configured.mark(dev);
     }
     const unsigned grid = (unsigned)(a.total_items < num_sms ? a.total_items : num_sms);
     if (a.window > 0)
-        hop_long_kernel<D, true><<<grid, kThreads, smem, pb.stream>>>(mq, mk, mxi, (__nv_bfloat16 *)xout, a);
-    else
-        hop_long_kernel<D, false><<<grid, kThreads, smem, pb.stream>>>(mq, mk, mxi, (__nv_bfloat16 *)xout, a);
-    count_launch();
-    return cudaPeekAtLastError() == cudaSuccess ? TA_OK : TA_ERR_CUDA;
+        return launch_kernel(hop_long_kernel<D, true>, grid, kThreads, smem, pb.stream, false, mq, mk, mxi,
+                             (__nv_bfloat16 *)xout, a);
+    return launch_kernel(hop_long_kernel<D, false>, grid, kThreads, smem, pb.stream, false, mq, mk, mxi,
+                         (__nv_bfloat16 *)xout, a);
 }
 
 }  // namespace

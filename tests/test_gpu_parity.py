@@ -10,7 +10,7 @@ import oracle
 import paper_2410_20926_b200 as ta
 from paper_2410_20926_b200 import inputs as ta_inputs
 
-from helpers import assert_close, check_case, gpu_forward
+from helpers import assert_close, check_case, gpu_forward, to_device
 
 pytestmark = pytest.mark.gpu
 
@@ -208,3 +208,47 @@ def test_overlapped_hop_launches_give_identical_results(B, H, Hkv, D, dims, caus
     for _ in range(10):
         got = gpu_forward(inp, B, H, Hkv, N, D, dims, causal, "bf16", base, **kw)
         np.testing.assert_array_equal(got, ref)
+
+
+def test_concurrent_host_threads_and_streams():
+    """Four host threads, each with its own stream and problem, call the library at the same time
+    and repeatedly; every result must equal the one the same problem gives when run alone."""
+    import threading
+
+    import torch
+    cases = [(1, 4, 2, 128, [8, 16, 32], True), (2, 4, 4, 64, [16, 4, 4, 4], False),
+             (1, 2, 1, 128, [2, 300], True), (1, 8, 2, 128, [32, 32], True)]
+    work = []
+    for i, (B, H, Hkv, D, dims, causal) in enumerate(cases):
+        N = math.prod(dims)
+        inp = ta_inputs.make_inputs(B, H, Hkv, N, D, "bf16", 140 + i)
+        q, k, v = (to_device(inp, n, "bf16") for n in ("q", "k", "v"))
+        ref = torch.empty_like(q)
+        ta.ta_forward(q, k, v, ref, B, H, Hkv, N, D, dims, causal)
+        work.append((q, k, v, ref, B, H, Hkv, N, D, dims, causal))
+    torch.cuda.synchronize()
+    errors = []
+
+    def worker(w):
+        q, k, v, ref, B, H, Hkv, N, D, dims, causal = w
+        try:
+            stream = torch.cuda.Stream()
+            outs = [torch.empty_like(q) for _ in range(25)]
+            for out in outs:
+                ta.ta_forward(q, k, v, out, B, H, Hkv, N, D, dims, causal, stream=stream)
+            stream.synchronize()
+            for out in outs:
+                if not torch.equal(out, ref):
+                    errors.append(("mismatch", dims))
+                    break
+        except Exception as e:      # noqa: BLE001 - reported below
+            errors.append((repr(e), dims))
+
+    threads = [threading.Thread(target=worker, args=(w,)) for w in work]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    torch.cuda.synchronize()
+    ta.ta_device_status()
+    assert not errors, errors
