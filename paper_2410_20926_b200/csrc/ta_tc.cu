@@ -477,6 +477,21 @@ EncodeTiledFn encode_fn() {
     return fn;
 }
 
+typedef CUresult (*CtxGetCurrentFn)(CUcontext *);
+bool thread_has_context() {
+    static CtxGetCurrentFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuCtxGetCurrent", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = (CtxGetCurrentFn)p;
+    });
+    CUcontext ctx = nullptr;
+    return fn && fn(&ctx) == CUDA_SUCCESS && ctx != nullptr;
+}
+
 }  // namespace
 
 // Rank-5 map of one tensor [heads][N][D] seen through hop `hd`: dims (D, t, inner, outer, head),
@@ -502,11 +517,9 @@ int make_view_map(CUtensorMap *map, const void *base, int heads_total, int N, in
     // The encoder is a driver call and needs a context current on this host thread; a thread whose
     // first CUDA activity is this library (its caller's streams and buffers may all come from
     // pools filled by other threads) has none until a runtime call binds the primary context.
-    static thread_local bool context_bound = false;
-    if (!context_bound) {
-        cudaFree(nullptr);
-        context_bound = true;
-    }
+    // (Asked of the driver each time rather than remembered: the bind itself is not allowed
+    // inside a stream capture, and a capturing thread always has a context.)
+    if (!thread_has_context()) cudaFree(nullptr);
     CUresult r = enc(map, elem == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 5,
                      const_cast<void *>(base), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                      CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
