@@ -39,7 +39,7 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per token per launch of the hop kernel, from
 # the ncu capture of config 3 summarised in profiles/hop_pipe_kernel_config3_ncu_full.md
 # (mean of the three hops, 758.8 MB for 32768 tokens); traffic is proportional to the tokens.
-NCU_TRAFFIC_BYTES_PER_TOKEN_PER_LAUNCH = 758.8e6 / 32768
+NCU_TRAFFIC_BYTES_PER_TOKEN_PER_LAUNCH = 757.9e6 / 32768
 
 
 # ------------------------------------------------------------------ roofline arithmetic
