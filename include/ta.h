@@ -187,10 +187,12 @@ int ta_forward_ex(const ta_params *p);
  *   gradient G carried between hops, and fp32 accumulators for dq, dk, dv, which are rounded
  *   to bf16 once at the end.
  * Arithmetic: bf16 operands, fp32 accumulation; the attention weights are recomputed.
- * The sums over the query heads of a group are taken in tensor memory inside one CTA and the
- * sums over hops in launch order, so the result is bit-reproducible from run to run.
- * Supported where every hop runs on the tensor-core kernel (D in {64,128}, all n_i <= 128);
- * otherwise TA_ERR_UNSUPPORTED.
+ * The sums over the query heads of a group are taken inside one CTA and the sums over hops in
+ * launch order (no atomics), so the result is bit-reproducible from run to run.
+ * Hops with D in {64,128} and n_i <= 128 run on the tensor-core backward kernel; the others
+ * (segments longer than 128, other head dims up to 256) on generic CUDA-core kernels with fp32
+ * arithmetic, which need a second G buffer and two floats per query row in the workspace
+ * (ta_workspace_bytes accounts for them).  D > 256: TA_ERR_UNSUPPORTED.
  */
 int ta_backward(const void *dout, const void *q, const void *k, const void *v, const void *out,
                 void *dq, void *dk, void *dv,

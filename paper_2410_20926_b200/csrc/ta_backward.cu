@@ -11,8 +11,14 @@ namespace {
 size_t up256(size_t x) { return (x + 255) & ~(size_t)255; }
 
 struct BwdLayout {
-    size_t save_off, gbuf_off, dq_off, dk_off, dv_off, total;
+    size_t save_off, gbuf_off, gbuf2_off, stats_off, dq_off, dk_off, dv_off, total;
 };
+
+bool any_generic_hop(const Plan &plan) {
+    for (int j = 0; j < plan.nhops; ++j)
+        if (plan.hops[j].path != PATH_TC) return true;
+    return false;
+}
 
 // [saved hop inputs X_1..X_{k-1}] [G buffer] [dq fp32] [dk fp32] [dv fp32]; the last three only
 // when the caller wants bf16 gradients, the first only when the hop inputs are recomputed.
@@ -24,6 +30,12 @@ BwdLayout layout(const Plan &plan, int B, int H, int H_kv, int N, int D, bool ne
     if (need_save && plan.nhops > 1) off += up256((size_t)(plan.nhops - 1) * tq * 2);
     L.gbuf_off = off;
     if (plan.nhops > 1) off += up256(tq * 2);
+    // hops on the generic kernels cannot update G in place and keep two floats per query row
+    const bool generic = any_generic_hop(plan);
+    L.gbuf2_off = off;
+    if (generic && plan.nhops > 2) off += up256(tq * 2);
+    L.stats_off = off;
+    if (generic) off += up256((size_t)B * H * N * 8);
     L.dq_off = off;
     if (need_acc) off += up256(tq * 4);
     L.dk_off = off;
@@ -54,10 +66,12 @@ int backward_impl(const ta_bwd_params &p) {
             if (p.window[i] < 0) return TA_ERR_INVALID_ARG;
     Plan plan;
     // hop by hop: the backward needs every hop's input
-    int rc = build_plan(p.B, p.H, p.H_kv, p.N, p.D, p.dims, p.ndims, p.dtype, TA_FLAG_NO_HOP_FUSION, 0, 0, &plan);
+    // (with the positional encoding or valid lengths, long segments are recomputed on the generic kernel)
+    const unsigned plan_flags = (unsigned)TA_FLAG_NO_HOP_FUSION | (p.rope_base > 0.f ? kPlanFlagRope : 0u) |
+                                (p.seq_lens ? kPlanFlagLens : 0u);
+    int rc = build_plan(p.B, p.H, p.H_kv, p.N, p.D, p.dims, p.ndims, p.dtype, plan_flags, 0, 0, &plan);
     if (rc != TA_OK) return rc;
-    for (int j = 0; j < plan.nhops; ++j)
-        if (plan.hops[j].path != PATH_TC) return TA_ERR_UNSUPPORTED;   // backward exists on the tensor-core path only
+    if (p.D > 256) return TA_ERR_UNSUPPORTED;   // limit of the generic backward kernels
     auto misaligned = [](const void *x) { return (reinterpret_cast<uintptr_t>(x) & 15u) != 0; };
     if (misaligned(p.dout) || misaligned(p.q) || misaligned(p.k) || misaligned(p.v) || misaligned(p.dq) ||
         misaligned(p.dk) || misaligned(p.dv) || (p.saved_hops && misaligned(p.saved_hops)))
@@ -112,17 +126,33 @@ int backward_impl(const ta_bwd_params &p) {
         auto hop_input = [&](int j) -> const void * { return j == 0 ? p.v : (const void *)(saved + (size_t)(j - 1) * tq * 2); };
         if (!p.saved_hops) {
             for (int j = 0; j + 1 < k; ++j) {
-                rc = launch_hop_tc(pb, plan.hops[j], hop_input(j), j == 0 ? p.H_kv : p.H,
-                                   ws + L.save_off + (size_t)j * tq * 2);
+                const HopDesc &h = plan.hops[j];
+                const void *xin = hop_input(j);
+                const int xin_heads = j == 0 ? p.H_kv : p.H;
+                void *xout = ws + L.save_off + (size_t)j * tq * 2;
+                rc = h.path == PATH_TC        ? launch_hop_tc(pb, h, xin, xin_heads, xout)
+                     : h.path == PATH_TC_LONG ? launch_hop_tc_long(pb, h, xin, xin_heads, xout)
+                                              : launch_hop_simt(pb, h, xin, xin_heads, xout);
                 if (rc != TA_OK) return rc;
             }
         }
-        void *gbuf = k > 1 ? (void *)(ws + L.gbuf_off) : nullptr;
+        // G travels from hop to hop in bf16: in place through the tensor-core kernel, from one
+        // buffer to the other through the generic kernels
+        void *gbuf[2] = {k > 1 ? (void *)(ws + L.gbuf_off) : nullptr, (void *)(ws + L.gbuf2_off)};
+        void *stats = ws + L.stats_off;
+        const void *g_in = p.dout;
         for (int j = k - 1; j >= 0; --j) {
-            const void *g_in = j == k - 1 ? p.dout : (const void *)gbuf;
-            rc = launch_hop_tc_bwd(pb, plan.hops[j], hop_input(j), j == 0 ? p.H_kv : p.H, g_in, j == 0 ? nullptr : gbuf,
-                                   dq_acc, dk_acc, dv_acc, j == 0, j != k - 1);
+            const HopDesc &h = plan.hops[j];
+            void *g_out = nullptr;
+            if (j > 0) g_out = (h.path == PATH_TC && g_in != p.dout) ? const_cast<void *>(g_in)
+                                                                      : (g_in == gbuf[0] ? gbuf[1] : gbuf[0]);
+            rc = h.path == PATH_TC
+                     ? launch_hop_tc_bwd(pb, h, hop_input(j), j == 0 ? p.H_kv : p.H, g_in, g_out, dq_acc, dk_acc, dv_acc,
+                                         j == 0, j != k - 1)
+                     : launch_hop_simt_bwd(pb, h, hop_input(j), j == 0 ? p.H_kv : p.H, g_in, g_out, dq_acc, dk_acc,
+                                           dv_acc, stats, j == 0, j != k - 1);
             if (rc != TA_OK) return rc;
+            g_in = g_out;
         }
     }
     if (need_acc) {

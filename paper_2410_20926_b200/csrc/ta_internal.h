@@ -112,6 +112,12 @@ int launch_broadcast_kv(const Problem &pb);
 // true: added to.  dv_acc is always overwritten (only the first hop writes it).
 int launch_hop_tc_bwd(const Problem &pb, const HopDesc &hd, const void *x, int x_heads, const void *g_in,
                       void *g_out, float *dq_acc, float *dk_acc, float *dv_acc, bool first_hop, bool accumulate);
+// Backward of one hop on the generic CUDA-core kernels (ta_simt_bwd.cu): any n_i, D <= 256, bf16
+// storage.  Same arguments; g_out must differ from g_in (the key side reads every row of g_in),
+// stats: B*H*N float2 of scratch (per-row log-sum-exp and rowsum(A o dP)).
+int launch_hop_simt_bwd(const Problem &pb, const HopDesc &hd, const void *x, int x_heads, const void *g_in,
+                        void *g_out, float *dq_acc, float *dk_acc, float *dv_acc, void *stats, bool first_hop,
+                        bool accumulate);
 int launch_f32_to_bf16(const float *src, void *dst, long long n, cudaStream_t stream);
 int launch_group_sum(const void *dout, void *dv, int dv_is_f32, int B, int H, int H_kv, long long per_head,
                      cudaStream_t stream);

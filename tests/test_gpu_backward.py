@@ -130,9 +130,13 @@ def test_backward_with_saved_hops_matches_recompute():
 def test_backward_rejects_unsupported_and_small_workspace():
     import torch
     x = torch.zeros(1, 2, 256, 64, dtype=torch.bfloat16, device="cuda")
+    y = torch.zeros(1, 2, 4, 320, dtype=torch.bfloat16, device="cuda")
+    rc = ta.ta_backward(y, y, y, y, None, y, y, y, 1, 2, 2, 4, 320, [4], True, workspace=None,
+                        workspace_bytes=0, check=False)
+    assert rc == ta.TA_ERR_UNSUPPORTED                     # head dims above 256
     rc = ta.ta_backward(x, x, x, x, None, x, x, x, 1, 2, 2, 256, 64, [256], True, workspace=None,
                         workspace_bytes=0, check=False)
-    assert rc == ta.TA_ERR_UNSUPPORTED                     # n = 256 runs on the generic kernel
+    assert rc == ta.TA_ERR_WORKSPACE                       # the generic backward needs its statistics buffer
     rc = ta.ta_backward(x, x, x, x, None, x, x, x, 1, 2, 2, 256, 64, [16, 16], True, workspace=None,
                         workspace_bytes=0, check=False)
     assert rc == ta.TA_ERR_WORKSPACE
@@ -154,3 +158,55 @@ def test_config5_forward_backward_sampled_groups():
         assert_grad_close(got[2][b, kv], rv[idx], "dv")
     for t in got:
         assert np.isfinite(t).all()
+
+
+@pytest.mark.parametrize("dims,D,causal,B,H,Hkv,kw", [
+    ([300], 64, True, 1, 4, 2, {}),                       # one long dimension = ordinary attention
+    ([2, 200], 128, False, 1, 4, 2, {}),                  # a short hop (tensor cores) and a long one
+    ([150, 4], 64, True, 2, 2, 1, {}),                    # long hop first: its gradient feeds dV
+    ([5, 7, 6], 40, True, 1, 4, 2, {}),                   # head dim the tensor-core kernels do not take
+    ([3, 140, 2], 128, False, 1, 2, 2, {}),               # tensor-core, generic, tensor-core
+    ([260], 64, True, 1, 2, 1, {"window": [50]}),
+    ([2, 160], 64, True, 1, 4, 2, {"rope_base": 10000.0}),
+    ([12, 9], 48, False, 1, 2, 1, {"rope_base": 10000.0, "window": [5, 0]}),
+])
+def test_backward_generic_kernels(dims, D, causal, B, H, Hkv, kw):
+    """Hops the tensor-core backward does not cover (segments longer than 128, other head dims)
+    run on the generic backward kernels, alone or mixed with tensor-core hops."""
+    N = math.prod(dims)
+    inp = ta_inputs.make_inputs(B, H, Hkv, N, D, "bf16", 170, with_dout=True)
+    for grad_f32 in (True, False):
+        got = gpu_backward(inp, B, H, Hkv, N, D, dims, causal, grad_f32, **kw)
+        ref = oracle.backward(inp["dout"], inp["q"], inp["k"], inp["v"], dims, causal,
+                              rope_base=kw.get("rope_base"), window=kw.get("window"))
+        for name, g, r in zip(("dq", "dk", "dv"), got, ref):
+            assert_grad_close(g, r, name)
+
+
+def test_backward_generic_with_lengths_and_masks():
+    B, H, Hkv, D, dims = 2, 2, 1, 64, [2, 150]
+    N = math.prod(dims)
+    import torch
+    lens = [270, 140]
+    inp = ta_inputs.make_inputs(B, H, Hkv, N, D, "bf16", 171, with_dout=True)
+    got = gpu_backward(inp, B, H, Hkv, N, D, dims, False, True,
+                       seq_lens=torch.tensor(lens, dtype=torch.int32, device="cuda"))
+    ref = oracle.backward(inp["dout"], inp["q"], inp["k"], inp["v"], dims, False, seq_lens=lens)
+    for name, g, r in zip(("dq", "dk", "dv"), got, ref):
+        assert_grad_close(g, r, name)
+        for b, L in enumerate(lens):
+            assert (g[b, :, L:] == 0).all(), name
+    # explicit masks on a head dim that only the generic kernels take
+    dims, D = [6, 20], 40
+    N = math.prod(dims)
+    rng = np.random.default_rng(3)
+    masks = []
+    for n in dims:
+        m = (rng.random((n, n)) < 0.5).astype(np.uint8)
+        m[np.arange(n), np.arange(n)] = 1
+        masks.append(m)
+    inp = ta_inputs.make_inputs(1, 2, 2, N, D, "bf16", 172, with_dout=True)
+    got = gpu_backward(inp, 1, 2, 2, N, D, dims, True, True, hop_masks=masks)
+    ref = oracle.backward(inp["dout"], inp["q"], inp["k"], inp["v"], dims, True, masks=masks)
+    for name, g, r in zip(("dq", "dk", "dv"), got, ref):
+        assert_grad_close(g, r, name)

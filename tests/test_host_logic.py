@@ -148,9 +148,20 @@ def test_backward_validation_and_workspace_sizes():
     rc = ta.ta_backward(16, 16, 16, 16, None, 16, 16, 16, 1, 4, 2, 512, 128, [8, 64], True,
                         workspace=256, workspace_bytes=1024, stream=0, check=False)
     assert rc == ta.TA_ERR_WORKSPACE
-    rc = ta.ta_backward(16, 16, 16, 16, None, 16, 16, 16, 1, 4, 2, 512, 96, [8, 64], True,
+    rc = ta.ta_backward(16, 16, 16, 16, None, 16, 16, 16, 1, 4, 2, 512, 320, [8, 64], True,
                         workspace=256, workspace_bytes=1 << 30, stream=0, check=False)
-    assert rc == ta.TA_ERR_UNSUPPORTED          # head dim 96 has no tensor-core backward
+    assert rc == ta.TA_ERR_UNSUPPORTED          # head dims above 256 have no backward
+    # hops on the generic backward kernels (segments > 128, other head dims) add a second G
+    # buffer (three or more hops) and two floats per query row
+    e96 = 4 * 512 * 96
+    need96 = ta.ta_workspace_bytes(1, 4, 2, 512, 96, [8, 64], ta.TA_DTYPE_BF16, ta.TA_WS_BACKWARD_F32_GRADS)
+    assert need96 == 2 * e96 + 2 * e96 + 4 * 512 * 8
+    need3 = ta.ta_workspace_bytes(1, 4, 2, 512, 128, [2, 2, 128], ta.TA_DTYPE_BF16, ta.TA_WS_BACKWARD_F32_GRADS)
+    assert need3 == 2 * 2 * e + 2 * e
+    need3g = ta.ta_workspace_bytes(1, 4, 2, 512, 128, [2, 1, 256], ta.TA_DTYPE_BF16, ta.TA_WS_BACKWARD_F32_GRADS)
+    assert need3g == 2 * e + 2 * e + 4 * 512 * 8      # two hops: one G buffer, statistics
+    need4g = ta.ta_workspace_bytes(1, 4, 2, 1024, 128, [2, 2, 256], ta.TA_DTYPE_BF16, ta.TA_WS_BACKWARD_F32_GRADS)
+    assert need4g == 2 * 2 * (2 * e) + 2 * (2 * e) + 2 * (2 * e) + 4 * 1024 * 8
 
 
 def test_plan_fuses_trailing_dimensions_that_fit_a_tile():
