@@ -209,7 +209,8 @@ typedef struct ta_bwd_params {
     const int *dims;              /* host                                                      */
     int ndims;
     int causal;
-    int dtype;                    /* storage of q, k, v, dout: TA_DTYPE_BF16                   */
+    int dtype;                    /* storage of q, k, v, dout: TA_DTYPE_BF16, or TA_DTYPE_F32    */
+                                  /* (generic kernels, fp32 throughout; needs grad_dtype F32)   */
     int grad_dtype;               /* TA_DTYPE_BF16, or TA_DTYPE_F32: dq/dk/dv are the fp32      */
                                   /* accumulators themselves (no final rounding, less workspace)*/
     float softmax_scale;          /* 0 -> 1/sqrt(D)                                            */

@@ -256,7 +256,7 @@ def ta_backward(dout, q, k, v, out, dq, dk, dv, B, H, H_kv, N, D, dims, causal, 
 
 
 def ta_backward_ex(dout, q, k, v, dq, dk, dv, B, H, H_kv, N, D, dims, causal,
-                   grad_dtype=TA_DTYPE_BF16, softmax_scale=0.0, saved_hops=None, workspace=None,
+                   grad_dtype=TA_DTYPE_BF16, softmax_scale=0.0, saved_hops=None, workspace=None, dtype=TA_DTYPE_BF16,
                    workspace_bytes=0, rope_base=0.0, window=None, hop_masks=None, seq_lens=None,
                    stream=None, check=True) -> int:
     d, nd = _dims(dims)
@@ -266,7 +266,7 @@ def ta_backward_ex(dout, q, k, v, dq, dk, dv, B, H, H_kv, N, D, dims, causal,
     p.dq, p.dk, p.dv = _ptr(dq), _ptr(dk), _ptr(dv)
     p.B, p.H, p.H_kv, p.N, p.D = B, H, H_kv, N, D
     p.dims, p.ndims, p.causal = d, nd, int(bool(causal))
-    p.dtype, p.grad_dtype, p.softmax_scale = TA_DTYPE_BF16, grad_dtype, softmax_scale
+    p.dtype, p.grad_dtype, p.softmax_scale = dtype, grad_dtype, softmax_scale
     p.rope_base = rope_base
     win = _window(window, nd)
     if win is not None:

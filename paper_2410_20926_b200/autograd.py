@@ -3,8 +3,8 @@
 Marshalling only.  The forward is ``ta_forward_ex`` (with ``TA_FLAG_SAVE_HOPS`` when a gradient is
 needed, so the hop inputs X_1..X_{m-1} are kept instead of recomputed), the backward is
 ``ta_backward_ex`` on those saved hops; every step runs in the library's CUDA kernels and there
-is no fallback.  q: [B, H, N, D]; k, v: [B, H_kv, N, D]; contiguous bf16 CUDA tensors
-(float32 is accepted for the forward only).
+is no fallback.  q: [B, H, N, D]; k, v: [B, H_kv, N, D]; contiguous CUDA tensors, all bfloat16
+(tensor-core kernels) or all float32 (generic kernels, fp32 arithmetic throughout).
 """
 from __future__ import annotations
 
@@ -25,7 +25,7 @@ def _check(q, k, v, dims):
     if math.prod(int(x) for x in dims) != N:
         raise ValueError("prod(dims) must equal the sequence length")
     if q.dtype not in (torch.bfloat16, torch.float32) or k.dtype != q.dtype or v.dtype != q.dtype:
-        raise ValueError("q, k, v must all be bfloat16 (or all float32, forward only)")
+        raise ValueError("q, k, v must all be bfloat16 or all float32")
     return B, H, k.shape[1], N, D
 
 
@@ -39,8 +39,6 @@ def _function():
             q, k, v = q.contiguous(), k.contiguous(), v.contiguous()
             dims = [int(x) for x in dims]
             need_grad = any(ctx.needs_input_grad[:3])
-            if need_grad and q.dtype != torch.bfloat16:
-                raise ValueError("the backward takes bfloat16 tensors")
             dtype = ta.TA_DTYPE_BF16 if q.dtype == torch.bfloat16 else ta.TA_DTYPE_F32
             mode = ta.TA_WS_FORWARD_SAVE if need_grad else ta.TA_WS_FORWARD
             nbytes = ta.ta_workspace_bytes(B, H, H_kv, N, D, dims, dtype, mode)
@@ -67,13 +65,17 @@ def _function():
             B, H, H_kv, N, D, dims, causal, softmax_scale, rope_base, window, hop_masks, seq_lens = ctx.args
             dout = dout.contiguous()
             dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
-            nbytes = ta.ta_workspace_bytes(B, H, H_kv, N, D, dims, ta.TA_DTYPE_BF16, ta.TA_WS_BACKWARD)
+            f32 = q.dtype == torch.float32
+            dtype = ta.TA_DTYPE_F32 if f32 else ta.TA_DTYPE_BF16
+            nbytes = ta.ta_workspace_bytes(B, H, H_kv, N, D, dims, dtype,
+                                           ta.TA_WS_BACKWARD_F32_GRADS if f32 else ta.TA_WS_BACKWARD)
             ws = torch.empty(max(nbytes, 256), dtype=torch.uint8, device=q.device)
             real_hops = sum(1 for n in dims if n > 1)
             saved = ctx.saved_ws[ctx.saved_off:] if real_hops > 1 else None
             with torch.cuda.device(q.device):
                 ta.ta_backward_ex(dout, q, k, v, dq, dk, dv, B, H, H_kv, N, D, dims, causal,
-                                  softmax_scale=softmax_scale or 0.0, saved_hops=saved, workspace=ws,
+                                  dtype=dtype, grad_dtype=dtype, softmax_scale=softmax_scale or 0.0,
+                                  saved_hops=saved, workspace=ws,
                                   workspace_bytes=nbytes, rope_base=rope_base or 0.0, window=window,
                                   hop_masks=hop_masks, seq_lens=seq_lens)
             return dq, dk, dv, None, None, None, None, None, None, None

@@ -418,9 +418,9 @@ size_t ta_workspace_bytes(int B, int H, int H_kv, int N, int D, const int *dims,
     Plan plan;
     unsigned flags = mode == TA_WS_FORWARD_SAVE ? TA_FLAG_SAVE_HOPS : 0u;
     if (build_plan(B, H, H_kv, N, D, dims, ndims, dtype, flags, 0, 0, &plan) != TA_OK) return 0;
-    if (mode == TA_WS_BACKWARD) return backward_workspace_bytes(B, H, H_kv, N, D, dims, ndims, TA_DTYPE_BF16, false);
+    if (mode == TA_WS_BACKWARD) return backward_workspace_bytes(B, H, H_kv, N, D, dims, ndims, dtype, TA_DTYPE_BF16, false);
     if (mode == TA_WS_BACKWARD_F32_GRADS)
-        return backward_workspace_bytes(B, H, H_kv, N, D, dims, ndims, TA_DTYPE_F32, false);
+        return backward_workspace_bytes(B, H, H_kv, N, D, dims, ndims, dtype, TA_DTYPE_F32, false);
     return plan.scratch_bytes + plan.save_bytes;
 }
 

@@ -22,18 +22,18 @@ bool any_generic_hop(const Plan &plan) {
 
 // [saved hop inputs X_1..X_{k-1}] [G buffer] [dq fp32] [dk fp32] [dv fp32]; the last three only
 // when the caller wants bf16 gradients, the first only when the hop inputs are recomputed.
-BwdLayout layout(const Plan &plan, int B, int H, int H_kv, int N, int D, bool need_save, bool need_acc) {
+BwdLayout layout(const Plan &plan, int B, int H, int H_kv, int N, int D, bool need_save, bool need_acc, size_t elem) {
     const size_t tq = (size_t)B * H * N * D, tkv = (size_t)B * H_kv * N * D;
     BwdLayout L;
     size_t off = 0;
     L.save_off = off;
-    if (need_save && plan.nhops > 1) off += up256((size_t)(plan.nhops - 1) * tq * 2);
+    if (need_save && plan.nhops > 1) off += up256((size_t)(plan.nhops - 1) * tq * elem);
     L.gbuf_off = off;
-    if (plan.nhops > 1) off += up256(tq * 2);
+    if (plan.nhops > 1) off += up256(tq * elem);
     // hops on the generic kernels cannot update G in place and keep two floats per query row
     const bool generic = any_generic_hop(plan);
     L.gbuf2_off = off;
-    if (generic && plan.nhops > 2) off += up256(tq * 2);
+    if (generic && plan.nhops > 2) off += up256(tq * elem);
     L.stats_off = off;
     if (generic) off += up256((size_t)B * H * N * 8);
     L.dq_off = off;
@@ -48,17 +48,21 @@ BwdLayout layout(const Plan &plan, int B, int H, int H_kv, int N, int D, bool ne
 
 }  // namespace
 
-size_t backward_workspace_bytes(int B, int H, int H_kv, int N, int D, const int *dims, int ndims, int grad_dtype,
-                                bool have_saved_hops) {
+size_t backward_workspace_bytes(int B, int H, int H_kv, int N, int D, const int *dims, int ndims, int dtype,
+                                int grad_dtype, bool have_saved_hops) {
     Plan plan;
-    if (build_plan(B, H, H_kv, N, D, dims, ndims, TA_DTYPE_BF16, TA_FLAG_NO_HOP_FUSION, 0, 0, &plan) != TA_OK) return 0;
-    return layout(plan, B, H, H_kv, N, D, !have_saved_hops, grad_dtype != TA_DTYPE_F32).total;
+    if (dtype == TA_DTYPE_F32 && grad_dtype != TA_DTYPE_F32) return 0;   // fp32 tensors take fp32 gradients
+    if (build_plan(B, H, H_kv, N, D, dims, ndims, dtype, TA_FLAG_NO_HOP_FUSION, 0, 0, &plan) != TA_OK) return 0;
+    return layout(plan, B, H, H_kv, N, D, !have_saved_hops, grad_dtype != TA_DTYPE_F32,
+                  dtype == TA_DTYPE_F32 ? 4 : 2).total;
 }
 
 int backward_impl(const ta_bwd_params &p) {
     if (!p.dout || !p.q || !p.k || !p.v || !p.dq || !p.dk || !p.dv) return TA_ERR_INVALID_ARG;
-    if (p.dtype != TA_DTYPE_BF16) return TA_ERR_UNSUPPORTED;
+    if (p.dtype != TA_DTYPE_BF16 && p.dtype != TA_DTYPE_F32) return TA_ERR_UNSUPPORTED;
     if (p.grad_dtype != TA_DTYPE_BF16 && p.grad_dtype != TA_DTYPE_F32) return TA_ERR_UNSUPPORTED;
+    if (p.dtype == TA_DTYPE_F32 && p.grad_dtype != TA_DTYPE_F32) return TA_ERR_UNSUPPORTED;   // fp32 in, fp32 gradients
+    const size_t elem = p.dtype == TA_DTYPE_F32 ? 4 : 2;
     if (p.rope_base < 0.f || !(p.rope_base == p.rope_base)) return TA_ERR_INVALID_ARG;
     if (p.rope_base > 0.f && (p.D & 1)) return TA_ERR_UNSUPPORTED;
     if (p.window && p.ndims >= 1 && p.ndims <= TA_MAX_DIMS)
@@ -77,7 +81,7 @@ int backward_impl(const ta_bwd_params &p) {
         misaligned(p.dk) || misaligned(p.dv) || (p.saved_hops && misaligned(p.saved_hops)))
         return TA_ERR_ALIGNMENT;
     const bool need_acc = p.grad_dtype != TA_DTYPE_F32;
-    const BwdLayout L = layout(plan, p.B, p.H, p.H_kv, p.N, p.D, p.saved_hops == nullptr, need_acc);
+    const BwdLayout L = layout(plan, p.B, p.H, p.H_kv, p.N, p.D, p.saved_hops == nullptr, need_acc, elem);
     if (L.total > 0) {
         if (!p.workspace || p.workspace_bytes < L.total) return TA_ERR_WORKSPACE;
         if (reinterpret_cast<uintptr_t>(p.workspace) & 255u) return TA_ERR_ALIGNMENT;
@@ -111,6 +115,7 @@ int backward_impl(const ta_bwd_params &p) {
 
     if (k == 0) {
         if (p.seq_lens) return TA_ERR_UNSUPPORTED;   // no hop to apply the valid lengths in
+        if (p.dtype != TA_DTYPE_BF16) return TA_ERR_UNSUPPORTED;
         if (cudaMemsetAsync(dq_acc, 0, tq * 4, pb.stream) != cudaSuccess ||
             cudaMemsetAsync(dk_acc, 0, tkv * 4, pb.stream) != cudaSuccess)
             return TA_ERR_CUDA;
@@ -123,13 +128,13 @@ int backward_impl(const ta_bwd_params &p) {
         // them, and hop 0 stores dv; every row of every head is covered by exactly one tile.
         // X_j = input of hop j: X_0 = v, X_1.. = saved (or recomputed here by running hops 0..k-2)
         const char *saved = p.saved_hops ? (const char *)p.saved_hops : ws + L.save_off;
-        auto hop_input = [&](int j) -> const void * { return j == 0 ? p.v : (const void *)(saved + (size_t)(j - 1) * tq * 2); };
+        auto hop_input = [&](int j) -> const void * { return j == 0 ? p.v : (const void *)(saved + (size_t)(j - 1) * tq * elem); };
         if (!p.saved_hops) {
             for (int j = 0; j + 1 < k; ++j) {
                 const HopDesc &h = plan.hops[j];
                 const void *xin = hop_input(j);
                 const int xin_heads = j == 0 ? p.H_kv : p.H;
-                void *xout = ws + L.save_off + (size_t)j * tq * 2;
+                void *xout = ws + L.save_off + (size_t)j * tq * elem;
                 rc = h.path == PATH_TC        ? launch_hop_tc(pb, h, xin, xin_heads, xout)
                      : h.path == PATH_TC_LONG ? launch_hop_tc_long(pb, h, xin, xin_heads, xout)
                                               : launch_hop_simt(pb, h, xin, xin_heads, xout);

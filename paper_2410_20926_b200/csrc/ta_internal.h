@@ -123,8 +123,8 @@ int launch_group_sum(const void *dout, void *dv, int dv_is_f32, int B, int H, in
                      cudaStream_t stream);
 
 int backward_impl(const ta_bwd_params &p);
-size_t backward_workspace_bytes(int B, int H, int H_kv, int N, int D, const int *dims, int ndims, int grad_dtype,
-                                bool have_saved_hops);
+size_t backward_workspace_bytes(int B, int H, int H_kv, int N, int D, const int *dims, int ndims, int dtype,
+                                int grad_dtype, bool have_saved_hops);
 
 void count_launch(unsigned n = 1);
 

@@ -1,5 +1,5 @@
 // Generic CUDA-core backward of one hop of tensorized attention: any segment length n_i, any
-// head dim <= 256, bf16 storage, fp32 arithmetic.  Used by ta_backward for the hops the tcgen05
+// head dim <= 256, bf16 or fp32 storage, fp32 arithmetic.  Used by ta_backward for the hops the tcgen05
 // backward kernel does not cover (segments longer than 128, head dims other than 64 / 128).
 //
 // The paper gives no backward; this is the chain rule through X_{i+1} = A_i X_i for one hop:
@@ -58,10 +58,10 @@ __device__ __forceinline__ bool pair_visible(const SimtBwdArgs &a, const HopMask
 }
 
 // ------------------------------------------------------------------------------------ query side
-template <int DPL>
+template <typename T, int DPL>
 __global__ void __launch_bounds__(kThreads)
-hop_simt_bwd_q_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restrict__ k,
-                      const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__restrict__ g,
+hop_simt_bwd_q_kernel(const T *__restrict__ q, const T *__restrict__ k,
+                      const T *__restrict__ x, const T *__restrict__ g,
                       float *__restrict__ dq_acc, float2 *__restrict__ stats, SimtBwdArgs a,
                       const __grid_constant__ HopMask hop_mask) {
     extern __shared__ float smem[];
@@ -84,8 +84,7 @@ hop_simt_bwd_q_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *
         const long long outer = seg / a.stride, inner = seg % a.stride;
         const long long base = outer * a.n * a.stride + inner;
         const long long per_head = (long long)a.N * D;
-        const __nv_bfloat16 *qh = q + bh * per_head, *kh = k + kvh * per_head, *xp = x + xh * per_head,
-                            *gh = g + bh * per_head;
+        const T *qh = q + bh * per_head, *kh = k + kvh * per_head, *xp = x + xh * per_head, *gh = g + bh * per_head;
         const int t0 = qb * BR;
         const int exist = segment_exist(a, b, base);
 
@@ -94,8 +93,8 @@ hop_simt_bwd_q_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *
             const int r = idx / D, c = idx % D, t = t0 + r;
             const bool in = t < a.n && t < exist;
             const long long off = (base + (long long)t * a.stride) * D + c;
-            sQ[idx] = in ? __bfloat162float(qh[off]) : 0.f;
-            sG[idx] = in ? __bfloat162float(gh[off]) : 0.f;
+            sQ[idx] = in ? to_f32<T>(qh[off]) : 0.f;
+            sG[idx] = in ? to_f32<T>(gh[off]) : 0.f;
         }
         if (a.rope_log2_base != 0.f) {
             __syncthreads();
@@ -120,8 +119,8 @@ hop_simt_bwd_q_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *
                 float kv = 0.f, xv = 0.f;
                 if (key < exist) {
                     const long long off = (base + (long long)key * a.stride) * D + c;
-                    kv = __bfloat162float(kh[off]);
-                    xv = __bfloat162float(xp[off]);
+                    kv = to_f32<T>(kh[off]);
+                    xv = to_f32<T>(xp[off]);
                 }
                 sK[u * ld + c] = kv;
                 sX[u * ld + c] = xv;
@@ -245,11 +244,11 @@ hop_simt_bwd_q_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *
 }
 
 // -------------------------------------------------------------------------------------- key side
-template <int DPL>
+template <typename T, int DPL>
 __global__ void __launch_bounds__(kThreads)
-hop_simt_bwd_k_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restrict__ k,
-                      const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__restrict__ g,
-                      const float2 *__restrict__ stats, __nv_bfloat16 *__restrict__ g_out,
+hop_simt_bwd_k_kernel(const T *__restrict__ q, const T *__restrict__ k,
+                      const T *__restrict__ x, const T *__restrict__ g,
+                      const float2 *__restrict__ stats, T *__restrict__ g_out,
                       float *__restrict__ dk_acc, float *__restrict__ dv_acc, SimtBwdArgs a,
                       const __grid_constant__ HopMask hop_mask) {
     extern __shared__ float smem[];
@@ -270,7 +269,7 @@ hop_simt_bwd_k_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *
         const long long outer = seg / a.stride, inner = seg % a.stride;
         const long long base = outer * a.n * a.stride + inner;
         const long long per_head = (long long)a.N * D;
-        const __nv_bfloat16 *kh = k + kvh * per_head;
+        const T *kh = k + kvh * per_head;
         const int u0 = kb * BR;
         const int exist = segment_exist(a, b, base);
         const int q_end = min(a.n, exist);
@@ -284,7 +283,7 @@ hop_simt_bwd_k_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *
         __syncthreads();
         for (int idx = threadIdx.x; idx < BR * D; idx += kThreads) {
             const int r = idx / D, c = idx % D, key = u0 + r;
-            sK[idx] = key < exist ? __bfloat162float(kh[(base + (long long)key * a.stride) * D + c]) : 0.f;
+            sK[idx] = key < exist ? to_f32<T>(kh[(base + (long long)key * a.stride) * D + c]) : 0.f;
         }
         if (a.rope_log2_base != 0.f) {
             __syncthreads();
@@ -294,12 +293,12 @@ hop_simt_bwd_k_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *
         for (int hh = 0; hh < grp; ++hh) {
             const long long bh = (long long)b * a.H + (long long)kv * grp + hh;
             const long long xh = (a.x_heads == a.H) ? bh : kvh;
-            const __nv_bfloat16 *qh = q + bh * per_head, *gh = g + bh * per_head, *xp = x + xh * per_head;
+            const T *qh = q + bh * per_head, *gh = g + bh * per_head, *xp = x + xh * per_head;
             if (hh == 0 || a.x_heads == a.H) {
                 __syncthreads();
                 for (int idx = threadIdx.x; idx < BR * D; idx += kThreads) {
                     const int r = idx / D, c = idx % D, key = u0 + r;
-                    sX[idx] = key < exist ? __bfloat162float(xp[(base + (long long)key * a.stride) * D + c]) : 0.f;
+                    sX[idx] = key < exist ? to_f32<T>(xp[(base + (long long)key * a.stride) * D + c]) : 0.f;
                 }
             }
             float acc_g[kPerWarp][DPL];
@@ -316,8 +315,8 @@ hop_simt_bwd_k_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *
                     float qv = 0.f, gv = 0.f;
                     if (t < q_end) {
                         const long long off = (base + (long long)t * a.stride) * D + c;
-                        qv = __bfloat162float(qh[off]);
-                        gv = __bfloat162float(gh[off]);
+                        qv = to_f32<T>(qh[off]);
+                        gv = to_f32<T>(gh[off]);
                     }
                     sQ[r * ld + c] = qv;
                     sG[r * ld + c] = gv;
@@ -367,7 +366,7 @@ hop_simt_bwd_k_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *
                     const int c = lane + 32 * j;
                     if (c >= D) continue;
                     if (a.first_hop) acc_v[r][j] += acc_g[r][j];
-                    else g_out[bh * per_head + (base + (long long)key * a.stride) * D + c] = __float2bfloat16_rn(acc_g[r][j]);
+                    else g_out[bh * per_head + (base + (long long)key * a.stride) * D + c] = from_f32<T>(acc_g[r][j]);
                 }
             }
         }
@@ -409,7 +408,7 @@ hop_simt_bwd_k_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *
     }
 }
 
-template <int DPL>
+template <typename T, int DPL>
 int launch_dpl(const Problem &pb, const HopDesc &hd, const void *x, int x_heads, const void *g_in, void *g_out,
                float *dq_acc, float *dk_acc, float *dv_acc, float2 *stats, bool first_hop, bool accumulate) {
     SimtBwdArgs a;
@@ -433,24 +432,23 @@ int launch_dpl(const Problem &pb, const HopDesc &hd, const void *x, int x_heads,
         memset(&hm, 0, sizeof(hm));
     }
     const size_t smem = sizeof(float) * (2 * (size_t)BR * pb.D + 2 * (size_t)BL * (pb.D + 1));
-    auto kq = hop_simt_bwd_q_kernel<DPL>;
-    auto kk = hop_simt_bwd_k_kernel<DPL>;
+    auto kq = hop_simt_bwd_q_kernel<T, DPL>;
+    auto kk = hop_simt_bwd_k_kernel<T, DPL>;
     if (smem > 48 * 1024) {
         if (cudaFuncSetAttribute(kq, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
             cudaFuncSetAttribute(kk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
             return cuda_fail(cudaPeekAtLastError());
     }
-    const __nv_bfloat16 *q = (const __nv_bfloat16 *)pb.q, *k = (const __nv_bfloat16 *)pb.k;
+    const T *q = (const T *)pb.q, *k = (const T *)pb.k;
     a.items = (long long)pb.B * pb.H * a.segs_per_head * a.rblocks;
     long long grid = a.items < (1ll << 20) ? a.items : (1ll << 20);
-    int rc = launch_kernel(kq, (unsigned)grid, kThreads, smem, pb.stream, false, q, k, (const __nv_bfloat16 *)x,
-                           (const __nv_bfloat16 *)g_in, dq_acc, stats, a, hm);
+    int rc = launch_kernel(kq, (unsigned)grid, kThreads, smem, pb.stream, false, q, k, (const T *)x,
+                           (const T *)g_in, dq_acc, stats, a, hm);
     if (rc != TA_OK) return rc;
     a.items = (long long)pb.B * pb.H_kv * a.segs_per_head * a.rblocks;
     grid = a.items < (1ll << 20) ? a.items : (1ll << 20);
-    return launch_kernel(kk, (unsigned)grid, kThreads, smem, pb.stream, false, q, k, (const __nv_bfloat16 *)x,
-                         (const __nv_bfloat16 *)g_in, (const float2 *)stats, (__nv_bfloat16 *)g_out, dk_acc, dv_acc, a,
-                         hm);
+    return launch_kernel(kk, (unsigned)grid, kThreads, smem, pb.stream, false, q, k, (const T *)x,
+                         (const T *)g_in, (const float2 *)stats, (T *)g_out, dk_acc, dv_acc, a, hm);
 }
 
 }  // namespace
@@ -458,13 +456,18 @@ int launch_dpl(const Problem &pb, const HopDesc &hd, const void *x, int x_heads,
 int launch_hop_simt_bwd(const Problem &pb, const HopDesc &hd, const void *x, int x_heads, const void *g_in,
                         void *g_out, float *dq_acc, float *dk_acc, float *dv_acc, void *stats, bool first_hop,
                         bool accumulate) {
-    if (pb.dtype != TA_DTYPE_BF16) return TA_ERR_UNSUPPORTED;
     if (!first_hop && (g_out == nullptr || g_out == g_in)) return TA_ERR_INVALID_ARG;   // the key side reads all of g_in
     float2 *st = (float2 *)stats;
-    if (pb.D <= 32) return launch_dpl<1>(pb, hd, x, x_heads, g_in, g_out, dq_acc, dk_acc, dv_acc, st, first_hop, accumulate);
-    if (pb.D <= 64) return launch_dpl<2>(pb, hd, x, x_heads, g_in, g_out, dq_acc, dk_acc, dv_acc, st, first_hop, accumulate);
-    if (pb.D <= 128) return launch_dpl<4>(pb, hd, x, x_heads, g_in, g_out, dq_acc, dk_acc, dv_acc, st, first_hop, accumulate);
-    if (pb.D <= 256) return launch_dpl<8>(pb, hd, x, x_heads, g_in, g_out, dq_acc, dk_acc, dv_acc, st, first_hop, accumulate);
+#define TA_BWD_DISPATCH(T)                                                                                              \
+    do {                                                                                                                \
+        if (pb.D <= 32) return launch_dpl<T, 1>(pb, hd, x, x_heads, g_in, g_out, dq_acc, dk_acc, dv_acc, st, first_hop, accumulate);  \
+        if (pb.D <= 64) return launch_dpl<T, 2>(pb, hd, x, x_heads, g_in, g_out, dq_acc, dk_acc, dv_acc, st, first_hop, accumulate);  \
+        if (pb.D <= 128) return launch_dpl<T, 4>(pb, hd, x, x_heads, g_in, g_out, dq_acc, dk_acc, dv_acc, st, first_hop, accumulate); \
+        if (pb.D <= 256) return launch_dpl<T, 8>(pb, hd, x, x_heads, g_in, g_out, dq_acc, dk_acc, dv_acc, st, first_hop, accumulate); \
+    } while (0)
+    if (pb.dtype == TA_DTYPE_F32) TA_BWD_DISPATCH(float);
+    else if (pb.dtype == TA_DTYPE_BF16) TA_BWD_DISPATCH(__nv_bfloat16);
+#undef TA_BWD_DISPATCH
     return TA_ERR_UNSUPPORTED;
 }
 

@@ -55,6 +55,13 @@ def test_autograd_forward_only_and_argument_checks():
         ta.tensorized_attention(q, k, v, [16, 15])
     with pytest.raises(ValueError):
         ta.tensorized_attention(q.cpu(), k.cpu(), v.cpu(), dims)
-    q.requires_grad_(True)
-    with pytest.raises(ValueError):
-        ta.tensorized_attention(q, k, v, dims)          # the backward takes bfloat16 only
+    # fp32 tensors: gradients through the generic kernels, fp32 throughout
+    for t in (q, k, v):
+        t.requires_grad_(True)
+    out = ta.tensorized_attention(q, k, v, dims, causal=False)
+    out.sum().backward()
+    torch.cuda.synchronize()
+    ta.ta_device_status()
+    ones = np.ones((B, H, 256, D))
+    for t, r in zip((q, k, v), oracle.backward(ones, inp["q"], inp["k"], inp["v"], dims, False)):
+        assert np.abs(t.grad.cpu().numpy() - r).max() <= 1e-4 * max(1.0, np.abs(r).max())

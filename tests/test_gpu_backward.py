@@ -210,3 +210,39 @@ def test_backward_generic_with_lengths_and_masks():
     ref = oracle.backward(inp["dout"], inp["q"], inp["k"], inp["v"], dims, True, masks=masks)
     for name, g, r in zip(("dq", "dk", "dv"), got, ref):
         assert_grad_close(g, r, name)
+
+
+@pytest.mark.parametrize("dims,D,causal,B,H,Hkv,kw", [
+    ([16, 16], 64, False, 1, 2, 2, {}),                     # config 1's shape
+    ([5, 7, 6], 40, True, 2, 4, 2, {}),
+    ([200], 64, True, 1, 4, 2, {"window": [60]}),
+    ([6, 40], 128, True, 1, 4, 2, {"rope_base": 10000.0}),
+])
+def test_backward_fp32_storage(dims, D, causal, B, H, Hkv, kw):
+    """fp32 tensors and fp32 gradients (generic kernels, fp32 arithmetic throughout): the
+    gradients must match the fp64 oracle to the forward's fp32 tolerance, scaled by their size."""
+    import torch
+    N = math.prod(dims)
+    inp = ta_inputs.make_inputs(B, H, Hkv, N, D, "f32", 190, with_dout=True)
+    q, k, v, do = (to_device(inp, n, "f32") for n in ("q", "k", "v", "dout"))
+    dq = torch.full((B, H, N, D), float("nan"), dtype=torch.float32, device="cuda")
+    dk = torch.full((B, Hkv, N, D), float("nan"), dtype=torch.float32, device="cuda")
+    dv = torch.full((B, Hkv, N, D), float("nan"), dtype=torch.float32, device="cuda")
+    nbytes = ta.ta_workspace_bytes(B, H, Hkv, N, D, dims, ta.TA_DTYPE_F32, ta.TA_WS_BACKWARD_F32_GRADS)
+    assert nbytes > 0
+    ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    ta.ta_backward_ex(do, q, k, v, dq, dk, dv, B, H, Hkv, N, D, dims, causal, dtype=ta.TA_DTYPE_F32,
+                      grad_dtype=ta.TA_DTYPE_F32, workspace=ws, workspace_bytes=nbytes, **kw)
+    torch.cuda.synchronize()
+    ta.ta_device_status()
+    ref = oracle.backward(inp["dout"], inp["q"], inp["k"], inp["v"], dims, causal,
+                          rope_base=kw.get("rope_base"), window=kw.get("window"))
+    for name, g, r in zip(("dq", "dk", "dv"), (dq, dk, dv), ref):
+        g = g.cpu().numpy().astype(np.float64)
+        assert np.isfinite(g).all(), name
+        err = np.abs(g - r).max()
+        assert err <= 1e-4 * max(1.0, np.abs(r).max()), (name, err, np.abs(r).max())
+    # bf16 gradients of fp32 tensors are not offered
+    rc = ta.ta_backward_ex(do, q, k, v, dq, dk, dv, B, H, Hkv, N, D, dims, causal, dtype=ta.TA_DTYPE_F32,
+                           grad_dtype=ta.TA_DTYPE_BF16, workspace=ws, workspace_bytes=nbytes, check=False)
+    assert rc == ta.TA_ERR_UNSUPPORTED
