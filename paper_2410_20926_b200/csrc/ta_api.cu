@@ -233,12 +233,16 @@ static Arena g_scratch, g_staging;
 
 // Copy engine of ta_forward_host: uploads and downloads run on two streams of their own and
 // the staging memory has two sets, so that the upload of one call overlaps the kernels and the
-// download of the previous one (PCIe is full duplex).
+// download of the previous one (PCIe is full duplex).  Inside a call the (batch, KV head) pairs
+// are independent, so a large call is cut into up to kHostGroups groups of them that follow one
+// another through upload, kernels and download: the kernels and the download of a group run
+// under the upload of the next ones, and a single call costs little more than its upload.
+constexpr int kHostGroups = 16;
 struct HostPipe {
     bool ready = false;
     int device = -1;
     cudaStream_t s_in = nullptr, s_out = nullptr;
-    cudaEvent_t in_done[2] = {}, k_done[2] = {}, out_done[2] = {};
+    cudaEvent_t in_done[2][kHostGroups] = {}, k_done[2][kHostGroups] = {}, out_done[2] = {};
     bool used[2] = {false, false};
     unsigned turn = 0;
     int init() {
@@ -249,11 +253,13 @@ struct HostPipe {
         if (cudaStreamCreateWithFlags(&s_in, cudaStreamNonBlocking) != cudaSuccess ||
             cudaStreamCreateWithFlags(&s_out, cudaStreamNonBlocking) != cudaSuccess)
             return TA_ERR_CUDA;
-        for (int i = 0; i < 2; ++i)
-            if (cudaEventCreateWithFlags(&in_done[i], cudaEventDisableTiming) != cudaSuccess ||
-                cudaEventCreateWithFlags(&k_done[i], cudaEventDisableTiming) != cudaSuccess ||
-                cudaEventCreateWithFlags(&out_done[i], cudaEventDisableTiming) != cudaSuccess)
-                return TA_ERR_CUDA;
+        for (int i = 0; i < 2; ++i) {
+            if (cudaEventCreateWithFlags(&out_done[i], cudaEventDisableTiming) != cudaSuccess) return TA_ERR_CUDA;
+            for (int g = 0; g < kHostGroups; ++g)
+                if (cudaEventCreateWithFlags(&in_done[i][g], cudaEventDisableTiming) != cudaSuccess ||
+                    cudaEventCreateWithFlags(&k_done[i][g], cudaEventDisableTiming) != cudaSuccess)
+                    return TA_ERR_CUDA;
+        }
         used[0] = used[1] = false;
         turn = 0;
         device = dev;
@@ -265,15 +271,18 @@ struct HostPipe {
         cudaStreamDestroy(s_in);
         cudaStreamDestroy(s_out);
         for (int i = 0; i < 2; ++i) {
-            cudaEventDestroy(in_done[i]);
-            cudaEventDestroy(k_done[i]);
             cudaEventDestroy(out_done[i]);
+            for (int g = 0; g < kHostGroups; ++g) {
+                cudaEventDestroy(in_done[i][g]);
+                cudaEventDestroy(k_done[i][g]);
+            }
         }
         ready = false;
         device = -1;
     }
 };
 static HostPipe g_host_pipe;
+static std::mutex g_host_mutex;   // ta_forward_host calls, one at a time; taken before g_arena_mutex
 
 static int check_arch() {
     static std::atomic<int> cached{1};  // 1 = unknown
@@ -435,7 +444,9 @@ int ta_forward_host(const void *qh, const void *kh, const void *vh, void *outh, 
     const size_t qb = (size_t)B * H * N * D * e, kb = (size_t)B * H_kv * N * D * e;
     auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
     const size_t set_bytes = 2 * up(qb) + 2 * up(kb);
-    std::lock_guard<std::mutex> lock(g_arena_mutex);   // one call at a time enqueues into the pipe
+    // one call at a time enqueues into the pipe (a lock of its own: the forward pass below takes
+    // the arena lock when it needs the library's scratch tensor)
+    std::lock_guard<std::mutex> lock(g_host_mutex);
     HostPipe &hp = g_host_pipe;
     if ((rc = hp.init()) != TA_OK) return rc;
     if (g_staging.bytes < 2 * set_bytes || g_staging.device != hp.device) {
@@ -448,22 +459,37 @@ int ta_forward_host(const void *qh, const void *kh, const void *vh, void *outh, 
     char *base = (char *)g_staging.ptr + (size_t)set * set_bytes;
     char *dq = base, *dk = dq + up(qb), *dv = dk + up(kb), *dout = dv + up(kb);
     cudaStream_t s = (cudaStream_t)stream;
+    // groups of (batch, KV head) pairs: whole batch entries, each cut into `parts` equal runs of
+    // KV heads (with their query heads), as long as a group still carries 32 MB of queries
+    int parts = 1;
+    for (int d = 1; d <= H_kv; ++d)
+        if (H_kv % d == 0 && (long long)B * d <= kHostGroups && qb / ((size_t)B * d) >= (32u << 20)) parts = d;
+    const int groups = (long long)B * parts <= kHostGroups ? B * parts : 1;
+    const int gB = groups == 1 ? B : 1, gH = groups == 1 ? H : H / parts, gHkv = groups == 1 ? H_kv : H_kv / parts;
+    const size_t gq = qb / groups, gk = kb / groups;          // bytes of a group's q (= out) and k (= v)
     // upload (own stream): only waits until this staging set's previous result has been read back
     if (hp.used[set] && cudaStreamWaitEvent(hp.s_in, hp.out_done[set], 0) != cudaSuccess) return TA_ERR_CUDA;
-    if (cudaMemcpyAsync(dq, qh, qb, cudaMemcpyHostToDevice, hp.s_in) != cudaSuccess ||
-        cudaMemcpyAsync(dk, kh, kb, cudaMemcpyHostToDevice, hp.s_in) != cudaSuccess ||
-        cudaMemcpyAsync(dv, vh, kb, cudaMemcpyHostToDevice, hp.s_in) != cudaSuccess ||
-        cudaEventRecord(hp.in_done[set], hp.s_in) != cudaSuccess)
-        return TA_ERR_CUDA;
-    // kernels on the caller's stream
-    if (cudaStreamWaitEvent(s, hp.in_done[set], 0) != cudaSuccess) return TA_ERR_CUDA;
-    rc = forward_simple(dq, dk, dv, dout, B, H, H_kv, N, D, dims, ndims, causal, dtype, stream);
-    if (rc != TA_OK) return rc;
-    if (cudaEventRecord(hp.k_done[set], s) != cudaSuccess) return TA_ERR_CUDA;
-    // download (own stream); the caller's stream completes only after it
-    if (cudaStreamWaitEvent(hp.s_out, hp.k_done[set], 0) != cudaSuccess ||
-        cudaMemcpyAsync(outh, dout, qb, cudaMemcpyDeviceToHost, hp.s_out) != cudaSuccess ||
-        cudaEventRecord(hp.out_done[set], hp.s_out) != cudaSuccess ||
+    for (int g = 0; g < groups; ++g) {
+        if (cudaMemcpyAsync(dq + g * gq, (const char *)qh + g * gq, gq, cudaMemcpyHostToDevice, hp.s_in) != cudaSuccess ||
+            cudaMemcpyAsync(dk + g * gk, (const char *)kh + g * gk, gk, cudaMemcpyHostToDevice, hp.s_in) != cudaSuccess ||
+            cudaMemcpyAsync(dv + g * gk, (const char *)vh + g * gk, gk, cudaMemcpyHostToDevice, hp.s_in) != cudaSuccess ||
+            cudaEventRecord(hp.in_done[set][g], hp.s_in) != cudaSuccess)
+            return TA_ERR_CUDA;
+    }
+    for (int g = 0; g < groups; ++g) {
+        // kernels on the caller's stream, as soon as the group's tensors are in
+        if (cudaStreamWaitEvent(s, hp.in_done[set][g], 0) != cudaSuccess) return TA_ERR_CUDA;
+        rc = forward_simple(dq + g * gq, dk + g * gk, dv + g * gk, dout + g * gq, gB, gH, gHkv, N, D, dims, ndims, causal,
+                            dtype, stream);
+        if (rc != TA_OK) return rc;
+        if (cudaEventRecord(hp.k_done[set][g], s) != cudaSuccess) return TA_ERR_CUDA;
+        // download (own stream)
+        if (cudaStreamWaitEvent(hp.s_out, hp.k_done[set][g], 0) != cudaSuccess ||
+            cudaMemcpyAsync((char *)outh + g * gq, dout + g * gq, gq, cudaMemcpyDeviceToHost, hp.s_out) != cudaSuccess)
+            return TA_ERR_CUDA;
+    }
+    // the caller's stream completes only after the last download
+    if (cudaEventRecord(hp.out_done[set], hp.s_out) != cudaSuccess ||
         cudaStreamWaitEvent(s, hp.out_done[set], 0) != cudaSuccess)
         return TA_ERR_CUDA;
     hp.used[set] = true;
@@ -548,6 +574,7 @@ int ta_device_status(void) {
 unsigned long long ta_launch_count(void) { return g_launches.load(); }
 
 int ta_release(void) {
+    std::lock_guard<std::mutex> host_lock(g_host_mutex);
     std::lock_guard<std::mutex> lock(g_arena_mutex);
     if (g_scratch.ptr || g_staging.ptr || g_host_pipe.ready) cudaDeviceSynchronize();
     g_scratch.release();

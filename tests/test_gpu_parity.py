@@ -252,3 +252,33 @@ def test_concurrent_host_threads_and_streams():
     torch.cuda.synchronize()
     ta.ta_device_status()
     assert not errors, errors
+
+
+def test_forward_host_groups_of_heads_and_scratch():
+    """Host-buffer entry point on a call large enough to be cut into groups of (batch, KV head)
+    pairs that pipeline through upload, kernels and download, and on an fp32 problem whose hops
+    need the library's scratch tensor; results must equal the device-resident runs."""
+    import torch
+    stream = torch.cuda.current_stream()
+    # 2 x 8 KV heads x 4 query heads x 4096 tokens x 128 x 2 B = 64 MB of queries per batch entry
+    B, H, Hkv, D, dims = 2, 32, 8, 128, [64, 64]
+    N = math.prod(dims)
+    inp = ta_inputs.make_inputs(B, H, Hkv, N, D, "bf16", 145)
+    host = [torch.from_numpy(inp[n + "_bits"].view(np.int16)).view(torch.bfloat16).pin_memory() for n in "qkv"]
+    out_h = torch.empty((B, H, N, D), dtype=torch.bfloat16).pin_memory()
+    for _ in range(2):
+        out_h.fill_(float("nan"))
+        ta.ta_forward_host(host[0], host[1], host[2], out_h, B, H, Hkv, N, D, dims, True, stream=stream)
+        torch.cuda.synchronize()
+        ta.ta_device_status()
+        np.testing.assert_array_equal(out_h.float().numpy(), gpu_forward(inp, B, H, Hkv, N, D, dims, True, "bf16"))
+    B, H, Hkv, D, dims = 1, 2, 2, 64, [4, 4, 16]
+    N = math.prod(dims)
+    inp = ta_inputs.make_inputs(B, H, Hkv, N, D, "f32", 146)
+    host = [torch.from_numpy(inp[n]).pin_memory() for n in "qkv"]
+    out_h = torch.empty((B, H, N, D), dtype=torch.float32).pin_memory()
+    ta.ta_forward_host(host[0], host[1], host[2], out_h, B, H, Hkv, N, D, dims, True, dtype=ta.TA_DTYPE_F32,
+                       stream=stream)
+    torch.cuda.synchronize()
+    ta.ta_device_status()
+    np.testing.assert_array_equal(out_h.numpy(), gpu_forward(inp, B, H, Hkv, N, D, dims, True, "f32"))
