@@ -168,8 +168,7 @@ typedef struct ta_params {
  * synchronisation); values are clamped to [0, N].  The padding rows of q, k and v must hold
  * finite values (they are multiplied by weights that are exactly 0).  With `causal` the rows
  * below the length equal those of the call without seq_lens (a causal hop only reads tokens of
- * smaller flat index).  Hops are not fused, and segments longer than 128 run on the generic
- * kernel.  ta_backward_ex takes the same array: the padding rows of dq, dk, dv are 0 and those
+ * smaller flat index).  Hops are not fused.  ta_backward_ex takes the same array: the padding rows of dq, dk, dv are 0 and those
  * of dout are not used (but must be finite).
  */
 int ta_forward_ex(const ta_params *p);

@@ -54,7 +54,7 @@ int build_plan(int B, int H, int H_kv, int N, int D, const int *dims, int ndims,
     int rc = validate_shape(B, H, H_kv, N, D, dims, ndims, dtype);
     if (rc != TA_OK) return rc;
     if (flags & ~(unsigned)(TA_FLAG_NO_TENSOR_CORE | TA_FLAG_NO_HOP_FUSION | TA_FLAG_SAVE_HOPS | TA_FLAG_NO_HOP_OVERLAP |
-                            kPlanFlagRope | kPlanFlagLens))
+                            kPlanFlagRope))
         return TA_ERR_UNSUPPORTED;
     if (hop_begin == 0 && hop_end == 0) hop_end = ndims;
     if (hop_begin < 0 || hop_end > ndims || hop_begin > hop_end) return TA_ERR_INVALID_ARG;
@@ -70,8 +70,7 @@ int build_plan(int B, int H, int H_kv, int N, int D, const int *dims, int ndims,
         h.path = PATH_SIMT;
         if (tc_eligible(D, dtype, flags)) {
             if (h.n <= 128) h.path = PATH_TC;
-            // the long-segment kernel neither rotates nor takes valid lengths
-            else if (!(flags & (kPlanFlagRope | kPlanFlagLens))) h.path = PATH_TC_LONG;
+            else if (!(flags & kPlanFlagRope)) h.path = PATH_TC_LONG;   // the long-segment kernel does not rotate
         }
         if (h.path == PATH_TC) tile_packing(h);
     }
@@ -310,13 +309,13 @@ static int forward_impl(const ta_params &p) {
             if (p.window[i] < 0) return TA_ERR_INVALID_ARG;
     Plan plan;
     // the positional encoding gives every hop its own rotated Q and K: nothing to share, no fusion
-    if (p.flags & (kPlanFlagRope | kPlanFlagLens)) return TA_ERR_UNSUPPORTED;
+    if (p.flags & kPlanFlagRope) return TA_ERR_UNSUPPORTED;
     bool any_mask = false;
     if (p.hop_masks && p.ndims >= 1 && p.ndims <= TA_MAX_DIMS)
         for (int i = 0; i < p.ndims; ++i) any_mask = any_mask || p.hop_masks[i] != nullptr;
     const unsigned plan_flags = p.flags | (p.rope_base > 0.f ? (unsigned)TA_FLAG_NO_HOP_FUSION | kPlanFlagRope : 0u) |
                                 (any_mask ? (unsigned)TA_FLAG_NO_HOP_FUSION : 0u) |
-                                (p.seq_lens ? (unsigned)TA_FLAG_NO_HOP_FUSION | kPlanFlagLens : 0u);
+                                (p.seq_lens ? (unsigned)TA_FLAG_NO_HOP_FUSION : 0u);
     int rc = build_plan(p.B, p.H, p.H_kv, p.N, p.D, p.dims, p.ndims, p.dtype, plan_flags, p.hop_begin,
                         p.hop_end, &plan);
     if (rc != TA_OK) return rc;

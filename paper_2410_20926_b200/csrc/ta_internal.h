@@ -23,7 +23,6 @@ enum HopPath {
 
 // build_plan flag used inside the library only: the call carries the positional encoding
 constexpr unsigned kPlanFlagRope = 1u << 30;
-constexpr unsigned kPlanFlagLens = 1u << 29;   // valid lengths given: the long-segment kernel does not take them
 
 // One hop of Algorithm 1 as a strided view X[outer][t][inner][D] of a head:
 //   token(outer, t, inner) = outer * n * stride + t * stride + inner.

@@ -42,6 +42,8 @@ struct LongArgs {
     long long stride, outer, total_items;
     long long row_stride, seg_outer_stride, head_stride;   // elements: between positions, outer blocks, heads
     float scale_log2;
+    const int *lens;           // device, valid length per batch entry, or nullptr (kWindow variant only)
+    int N;
 };
 
 template <int D>
@@ -64,6 +66,7 @@ struct LongItem {
     int j0[2], je[2];          // key blocks [j0, je) of each tile (128 keys each)
     int keys_end[2];           // keys [.., keys_end) of each tile
     int jlo, jhi;              // union of the two ranges: the blocks the item loads
+    int exist;                 // positions of the segment that are tokens (n without valid lengths)
 };
 // item -> (pair of query tiles, inner, outer, head).  Pairs of a segment are adjacent, later
 // (longer, when causal) pairs first, so that the CTAs of one wave carry similar loads.
@@ -77,6 +80,13 @@ __device__ __forceinline__ LongItem decode_long_item(const LongArgs &a, long lon
     c.kv_head = (c.q_head / a.H) * a.H_kv + (c.q_head % a.H) / a.g;
     c.t0 = 2 * pb * kTileRows;
     c.ntiles = 2 * pb + 1 < a.qblocks ? 2 : 1;
+    c.exist = a.n;
+    if (a.lens != nullptr) {
+        const long long len = min(max(__ldg(a.lens + c.q_head / a.H), 0), a.N);
+        const long long first_token = (long long)c.outer * a.n * a.stride + c.inner;
+        const long long left = (len - first_token + a.stride - 1) / a.stride;
+        c.exist = len <= first_token ? 0 : (int)(left < a.n ? left : a.n);
+    }
 #pragma unroll
     for (int i = 0; i < 2; ++i) {
         const int t0 = c.t0 + i * kTileRows;
@@ -87,8 +97,11 @@ __device__ __forceinline__ LongItem decode_long_item(const LongArgs &a, long lon
             first = max(0, t0 - a.window + 1);
             if (!a.causal) keys_end = min(a.n, t0 + kTileRows - 1 + a.window);
         }
-        c.keys_end[i] = keys_end;
         c.j0[i] = first / kTileRows;
+        // padding keys are not visited, except that every tile keeps one block (its rows then see
+        // nothing in it and come out as zeros), so that no role ever meets an empty chain
+        keys_end = max(min(keys_end, c.exist), c.j0[i] * kTileRows + 1);
+        c.keys_end[i] = keys_end;
         c.je[i] = (keys_end + kTileRows - 1) / kTileRows;
     }
     if (c.ntiles == 1) { c.j0[1] = c.je[1] = c.je[0]; }            // an absent tile has no blocks
@@ -321,8 +334,11 @@ hop_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 int c_hi = !row_valid ? 0 : (diag ? min(keys, r + 1) : keys);
                 int c_lo = 0;                           // stays a compile-time 0 without a window
                 if (kWindow) {
-                    c_lo = max(0, t - a.window + 1 - u0);
-                    if (!a.causal) c_hi = min(c_hi, t + a.window - u0);
+                    if (a.window > 0) {
+                        c_lo = max(0, t - a.window + 1 - u0);
+                        if (!a.causal) c_hi = min(c_hi, t + a.window - u0);
+                    }
+                    c_hi = t < c.exist ? min(c_hi, c.exist - u0) : 0;     // valid length: padding keys, padding rows
                 }
                 const int nchunks = (keys + 31) >> 5;
 
@@ -494,6 +510,8 @@ int launch_long_d(const Problem &pb, const HopDesc &hd, const void *xin, int xin
     a.head_stride = (long long)pb.N * D;
     a.window = pb.window[hd.hop];
     a.scale_log2 = pb.scale * 1.4426950408889634f;
+    a.lens = pb.seq_lens;
+    a.N = pb.N;
 
     int dev = 0;
     const int num_sms = current_device_sms(&dev);
@@ -508,7 +526,7 @@ int launch_long_d(const Problem &pb, const HopDesc &hd, const void *xin, int xin
         configured.mark(dev);
     }
     const unsigned grid = (unsigned)(a.total_items < num_sms ? a.total_items : num_sms);
-    if (a.window > 0)
+    if (a.window > 0 || a.lens != nullptr)
         return launch_kernel(hop_long_kernel<D, true>, grid, kThreads, smem, pb.stream, false, mq, mk, mxi,
                              (__nv_bfloat16 *)xout, a);
     return launch_kernel(hop_long_kernel<D, false>, grid, kThreads, smem, pb.stream, false, mq, mk, mxi,

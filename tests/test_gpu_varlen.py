@@ -77,9 +77,24 @@ def test_lengths_generic_kernel_and_long_segments():
     run(2, 4, 2, 40, [3, 5, 7], [100, 13], False, "f32", 806)
     run(2, 4, 2, 64, [6, 100], [599, 250], True, "f32", 807)
     run(1, 2, 1, 64, [16, 16], [77], False, "bf16", 808, flags=ta.TA_FLAG_NO_TENSOR_CORE)
-    # segments longer than 128 with lengths run on the generic kernel
-    B, H, Hkv, D, dims = 2, 2, 1, 64, [2, 300]
-    run(B, H, Hkv, D, dims, [450, 299], False, "bf16", 809)
+
+
+@pytest.mark.parametrize("dims,D,causal,lens", [
+    ([2, 300], 64, False, [450, 299]),            # second row of the tensor cut short / missing
+    ([700], 128, True, [257, 700]),               # ordinary attention, batch entries of different lengths
+    ([700], 64, False, [1, 0]),                   # one token; an empty batch entry
+    ([3, 260], 128, False, [400, 780]),
+    ([1024], 128, True, [1000, 130]),
+])
+def test_lengths_long_segments_tensor_core(dims, D, causal, lens):
+    B, H, Hkv = 2, 4, 2
+    assert "tc-long" in ta.ta_plan_describe(B, H, Hkv, math.prod(dims), D, dims, causal, ta.TA_DTYPE_BF16, 0)
+    run(B, H, Hkv, D, dims, lens, causal, "bf16", 809)
+
+
+def test_lengths_long_segments_with_window_and_generic_kernel():
+    run(2, 4, 2, 64, [600], [599, 123], True, "bf16", 813, window=[100])
+    run(1, 2, 1, 64, [2, 300], [450], False, "bf16", 814, flags=ta.TA_FLAG_NO_TENSOR_CORE)
 
 
 def test_full_length_is_no_padding_and_causal_rows_do_not_depend_on_the_length():
