@@ -53,8 +53,7 @@ int build_plan(int B, int H, int H_kv, int N, int D, const int *dims, int ndims,
                unsigned flags, int hop_begin, int hop_end, Plan *plan) {
     int rc = validate_shape(B, H, H_kv, N, D, dims, ndims, dtype);
     if (rc != TA_OK) return rc;
-    if (flags & ~(unsigned)(TA_FLAG_NO_TENSOR_CORE | TA_FLAG_NO_HOP_FUSION | TA_FLAG_SAVE_HOPS | TA_FLAG_NO_HOP_OVERLAP |
-                            kPlanFlagRope))
+    if (flags & ~(unsigned)(TA_FLAG_NO_TENSOR_CORE | TA_FLAG_NO_HOP_FUSION | TA_FLAG_SAVE_HOPS | TA_FLAG_NO_HOP_OVERLAP))
         return TA_ERR_UNSUPPORTED;
     if (hop_begin == 0 && hop_end == 0) hop_end = ndims;
     if (hop_begin < 0 || hop_end > ndims || hop_begin > hop_end) return TA_ERR_INVALID_ARG;
@@ -70,7 +69,7 @@ int build_plan(int B, int H, int H_kv, int N, int D, const int *dims, int ndims,
         h.path = PATH_SIMT;
         if (tc_eligible(D, dtype, flags)) {
             if (h.n <= 128) h.path = PATH_TC;
-            else if (!(flags & kPlanFlagRope)) h.path = PATH_TC_LONG;   // the long-segment kernel does not rotate
+            else h.path = PATH_TC_LONG;
         }
         if (h.path == PATH_TC) tile_packing(h);
     }
@@ -228,7 +227,7 @@ struct Arena {
     }
 };
 static std::mutex g_arena_mutex;
-static Arena g_scratch, g_staging;
+static Arena g_scratch, g_staging, g_rotated;
 
 // Copy engine of ta_forward_host: uploads and downloads run on two streams of their own and
 // the staging memory has two sets, so that the upload of one call overlaps the kernels and the
@@ -280,6 +279,16 @@ struct HostPipe {
         device = -1;
     }
 };
+// Rotated copies of Q and K for a long-segment hop with the positional encoding (ta_tc_long.cu):
+// library-owned, grown on demand, shared by all calls.
+int rotated_arena(size_t bytes, void **ptr) {
+    std::lock_guard<std::mutex> lock(g_arena_mutex);
+    const int rc = g_rotated.reserve(bytes);
+    if (rc != TA_OK) return rc;
+    *ptr = g_rotated.ptr;
+    return TA_OK;
+}
+
 static HostPipe g_host_pipe;
 static std::mutex g_host_mutex;   // ta_forward_host calls, one at a time; taken before g_arena_mutex
 
@@ -309,11 +318,10 @@ static int forward_impl(const ta_params &p) {
             if (p.window[i] < 0) return TA_ERR_INVALID_ARG;
     Plan plan;
     // the positional encoding gives every hop its own rotated Q and K: nothing to share, no fusion
-    if (p.flags & kPlanFlagRope) return TA_ERR_UNSUPPORTED;
     bool any_mask = false;
     if (p.hop_masks && p.ndims >= 1 && p.ndims <= TA_MAX_DIMS)
         for (int i = 0; i < p.ndims; ++i) any_mask = any_mask || p.hop_masks[i] != nullptr;
-    const unsigned plan_flags = p.flags | (p.rope_base > 0.f ? (unsigned)TA_FLAG_NO_HOP_FUSION | kPlanFlagRope : 0u) |
+    const unsigned plan_flags = p.flags | (p.rope_base > 0.f ? (unsigned)TA_FLAG_NO_HOP_FUSION : 0u) |
                                 (any_mask ? (unsigned)TA_FLAG_NO_HOP_FUSION : 0u) |
                                 (p.seq_lens ? (unsigned)TA_FLAG_NO_HOP_FUSION : 0u);
     int rc = build_plan(p.B, p.H, p.H_kv, p.N, p.D, p.dims, p.ndims, p.dtype, plan_flags, p.hop_begin,
@@ -575,9 +583,10 @@ unsigned long long ta_launch_count(void) { return g_launches.load(); }
 int ta_release(void) {
     std::lock_guard<std::mutex> host_lock(g_host_mutex);
     std::lock_guard<std::mutex> lock(g_arena_mutex);
-    if (g_scratch.ptr || g_staging.ptr || g_host_pipe.ready) cudaDeviceSynchronize();
+    if (g_scratch.ptr || g_staging.ptr || g_rotated.ptr || g_host_pipe.ready) cudaDeviceSynchronize();
     g_scratch.release();
     g_staging.release();
+    g_rotated.release();
     g_host_pipe.destroy();
     return TA_OK;
 }

@@ -70,8 +70,7 @@ int backward_impl(const ta_bwd_params &p) {
             if (p.window[i] < 0) return TA_ERR_INVALID_ARG;
     Plan plan;
     // hop by hop: the backward needs every hop's input
-    // (with the positional encoding, long segments are recomputed on the generic kernel)
-    const unsigned plan_flags = (unsigned)TA_FLAG_NO_HOP_FUSION | (p.rope_base > 0.f ? kPlanFlagRope : 0u);
+    const unsigned plan_flags = (unsigned)TA_FLAG_NO_HOP_FUSION;
     int rc = build_plan(p.B, p.H, p.H_kv, p.N, p.D, p.dims, p.ndims, p.dtype, plan_flags, 0, 0, &plan);
     if (rc != TA_OK) return rc;
     if (p.D > 256) return TA_ERR_UNSUPPORTED;   // limit of the generic backward kernels

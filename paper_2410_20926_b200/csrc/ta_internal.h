@@ -22,7 +22,6 @@ enum HopPath {
 };
 
 // build_plan flag used inside the library only: the call carries the positional encoding
-constexpr unsigned kPlanFlagRope = 1u << 30;
 
 // One hop of Algorithm 1 as a strided view X[outer][t][inner][D] of a head:
 //   token(outer, t, inner) = outer * n * stride + t * stride + inner.
@@ -99,6 +98,8 @@ int launch_hop_tc(const Problem &pb, const HopDesc &hd, const void *xin, int xin
 // Long segments (n_i > 128): key-block loop with online softmax, ta_tc_long.cu.  xin != xout.
 int launch_hop_tc_long(const Problem &pb, const HopDesc &hd, const void *xin, int xin_heads, void *xout);
 int read_status_tc_long(unsigned int *word);
+// Library-owned buffer of at least `bytes` (grown on demand) for that kernel's rotated Q / K copies.
+int rotated_arena(size_t bytes, void **ptr);
 // Fused trailing hops (hd.nf > 1), ta_tc_fused.cu; called through launch_hop_tc.
 int launch_hop_tc_fused(const Problem &pb, const HopDesc &hd, const void *xin, int xin_heads, void *xout);
 // out[b,h] = v[b, h / (H/H_kv)] (all dims equal to 1).

@@ -535,11 +535,61 @@ int launch_long_d(const Problem &pb, const HopDesc &hd, const void *xin, int xin
 
 }  // namespace
 
+// Tensorized positional encoding (Section 3.2) for a long-segment hop: dst = src with every row
+// rotated by its coordinate along the hop's dimension (feature c paired with c + D/2, angle
+// position * base^(-2c/D)).  A long hop re-reads each K block once per pair of query tiles, so
+// rotating inside the pipeline would repeat the work n / 256 times; one elementwise pass over Q
+// and K costs two reads and writes of them against a hop whose time grows with n.  The angle is
+// reduced modulo 2 pi in double precision (positions reach 10^5, where an fp32 product is off by
+// milliradians).
+namespace {
+__global__ void rope_copy_kernel(const __nv_bfloat16 *__restrict__ src, __nv_bfloat16 *__restrict__ dst,
+                                 long long pairs, int N, int D, long long stride, int n, double log2_base) {
+    const int half = D >> 1;
+    for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < pairs;
+         idx += (long long)gridDim.x * blockDim.x) {
+        const int c = (int)(idx % half);
+        const long long row = idx / half;                       // head * N + token
+        const long long token = row % N;
+        const int pos = (int)((token / stride) % n);
+        const double theta = exp2(-2.0 * (double)c / (double)D * log2_base);
+        const double angle = fmod((double)pos * theta, 6.283185307179586476925);
+        float sn, cs;
+        sincosf((float)angle, &sn, &cs);
+        const long long o = row * D + c;
+        const float x1 = __bfloat162float(src[o]), x2 = __bfloat162float(src[o + half]);
+        dst[o] = __float2bfloat16_rn(x1 * cs - x2 * sn);
+        dst[o + half] = __float2bfloat16_rn(x2 * cs + x1 * sn);
+    }
+}
+}  // namespace
+
 int launch_hop_tc_long(const Problem &pb, const HopDesc &hd, const void *xin, int xin_heads, void *xout) {
     if (xin == xout) return TA_ERR_INVALID_ARG;
-    if (pb.D == 128) return launch_long_d<128>(pb, hd, xin, xin_heads, xout);
-    if (pb.D == 64) return launch_long_d<64>(pb, hd, xin, xin_heads, xout);
-    return TA_ERR_UNSUPPORTED;
+    if (pb.D != 128 && pb.D != 64) return TA_ERR_UNSUPPORTED;
+    Problem hop = pb;
+    if (pb.rope_base > 0.f) {
+        const size_t tq = (size_t)pb.B * pb.H * pb.N * pb.D, tkv = (size_t)pb.B * pb.H_kv * pb.N * pb.D;
+        const size_t q_bytes = (tq * 2 + 255) & ~(size_t)255;
+        void *buf = nullptr;
+        int rc = rotated_arena(q_bytes + tkv * 2, &buf);
+        if (rc != TA_OK) return rc;
+        __nv_bfloat16 *rq = (__nv_bfloat16 *)buf, *rk = (__nv_bfloat16 *)((char *)buf + q_bytes);
+        const double log2_base = log2((double)pb.rope_base);
+        const long long pq = (long long)(tq / 2), pk = (long long)(tkv / 2);
+        auto blocks = [](long long pairs) { return (unsigned)(pairs / 256 + 1 < 148 * 32 ? pairs / 256 + 1 : 148 * 32); };
+        rc = launch_kernel(rope_copy_kernel, blocks(pq), 256, 0, pb.stream, false, (const __nv_bfloat16 *)pb.q, rq, pq, pb.N,
+                           pb.D, (long long)hd.stride, hd.n, log2_base);
+        if (rc != TA_OK) return rc;
+        rc = launch_kernel(rope_copy_kernel, blocks(pk), 256, 0, pb.stream, false, (const __nv_bfloat16 *)pb.k, rk, pk, pb.N,
+                           pb.D, (long long)hd.stride, hd.n, log2_base);
+        if (rc != TA_OK) return rc;
+        hop.q = rq;
+        hop.k = rk;
+        hop.rope_base = 0.f;
+    }
+    if (pb.D == 128) return launch_long_d<128>(hop, hd, xin, xin_heads, xout);
+    return launch_long_d<64>(hop, hd, xin, xin_heads, xout);
 }
 
 int read_status_tc_long(unsigned int *word) {

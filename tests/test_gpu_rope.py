@@ -48,7 +48,7 @@ def test_rope_generic_f32(dims, D, causal):
 
 def test_rope_generic_bf16_and_mixed_paths():
     run(1, 4, 2, 64, [6, 20], True, "bf16", seed=404, flags=ta.TA_FLAG_NO_TENSOR_CORE)
-    run(1, 2, 1, 64, [4, 160], True, "bf16", seed=405)      # hop 1 (n = 160) on the generic kernel
+    run(1, 2, 1, 64, [4, 160], True, "bf16", seed=405)      # hop 1 (n = 160): long-segment kernel on rotated copies
 
 
 def test_rope_rejects_odd_head_dim_and_negative_base():
@@ -67,3 +67,22 @@ def test_rope_llama_shape_sampled_heads():
     """Config 3 (32 768 tokens as 32x32x32, H=32, H_kv=8, D=128) with the positional encoding."""
     c = ta_inputs.CONFIGS[3]
     run(c.B, c.H, c.H_kv, c.D, list(c.dims), True, "bf16", seed=c.seed, heads=[(0, 5), (0, 30)])
+
+
+@pytest.mark.parametrize("dims,D,causal", [
+    ([2048], 128, True),            # ordinary attention with RoPE, positions up to 2047
+    ([4, 1000], 64, False),
+    ([3, 300, 2], 128, True),       # short, long, short: only the long hop works on rotated copies
+])
+def test_rope_long_segments_tensor_core(dims, D, causal):
+    """Segments longer than 128 with the positional encoding: Q and K are rotated once per hop into
+    library-owned copies and the long-segment tensor-core kernel runs on those."""
+    B, H, Hkv = 1, 4, 2
+    N = math.prod(dims)
+    assert "tc-long" in ta.ta_plan_describe(B, H, Hkv, N, D, dims, causal, ta.TA_DTYPE_BF16, 0)
+    inp = ta_inputs.make_inputs(B, H, Hkv, N, D, "bf16", 410)
+    got = gpu_forward(inp, B, H, Hkv, N, D, dims, causal, "bf16", rope_base=10000.0)
+    ref = oracle.forward(inp["q"], inp["k"], inp["v"], dims, causal, rope_base=10000.0)
+    assert_close(got, ref, "bf16")
+    plain = oracle.forward(inp["q"], inp["k"], inp["v"], dims, causal)
+    assert np.abs(ref - plain).max() > 0.05

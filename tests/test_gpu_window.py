@@ -66,7 +66,7 @@ def test_window_generic_kernel_and_with_positional_encoding():
     run(2, 4, 2, 40, [3, 5, 7], [2, 3, 4], True, "f32", 604)
     run(1, 4, 2, 64, [200], [37], False, "f32", 605)
     run(1, 4, 2, 128, [8, 64], [3, 20], True, "bf16", 606, rope_base=10000.0)
-    run(1, 2, 1, 64, [300], [64], True, "bf16", 607, rope_base=10000.0)    # long + rope: generic kernel
+    run(1, 2, 1, 64, [300], [64], True, "bf16", 607, rope_base=10000.0)    # long + rope: rotated copies, long-segment kernel
 
 
 def test_window_rejects_negative_entries():
