@@ -147,6 +147,8 @@ typedef struct ta_params {
  * tiles in shared memory, between the TMA load and the MMA -- no rotated copy of q or k ever
  * exists in global memory.  D must be even (else TA_ERR_UNSUPPORTED); a negative or NaN base
  * is TA_ERR_INVALID_ARG.  The value tensor is never rotated.
+ * (Hops with n_i > 128 instead run on rotated copies of q and k, written once per hop into a
+ * buffer owned by the library and shared by all calls: two such calls must not overlap on the GPU.)
  * ta_backward_ex takes the same rope_base (ta_backward, the short form, does not).
  *
  * Per-hop sparsity mask (Eq. 3 allows any mask M_i): window[i] = w > 0 keeps, in hop i, only
