@@ -190,10 +190,13 @@ int ta_forward_ex(const ta_params *p);
  * Arithmetic: bf16 operands, fp32 accumulation; the attention weights are recomputed.
  * The sums over the query heads of a group are taken inside one CTA and the sums over hops in
  * launch order (no atomics), so the result is bit-reproducible from run to run.
- * Hops with D in {64,128} and n_i <= 128 run on the tensor-core backward kernel; the others
- * (segments longer than 128, other head dims up to 256) on generic CUDA-core kernels with fp32
- * arithmetic, which need a second G buffer and two floats per query row in the workspace
- * (ta_workspace_bytes accounts for them).  D > 256: TA_ERR_UNSUPPORTED.
+ * Hops with D in {64,128} run on tensor-core backward kernels: one for n_i <= 128, and for longer
+ * segments a block-by-block one (its dQ is summed by reduce-adds whose order is not fixed, so it
+ * is reproducible only up to fp32 summation order).  Other head dims up to 256, and long segments
+ * that carry a window, a mask, valid lengths or the positional encoding, run on generic CUDA-core
+ * kernels with fp32 arithmetic.  Hops with n_i > 128 or on the generic kernels need a second G
+ * buffer and two floats per query row in the workspace (ta_workspace_bytes accounts for them).
+ * D > 256: TA_ERR_UNSUPPORTED.
  */
 int ta_backward(const void *dout, const void *q, const void *k, const void *v, const void *out,
                 void *dq, void *dk, void *dv,

@@ -6,7 +6,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(os.path.dirname(HERE))
 LIB = os.path.join(os.path.dirname(HERE), "libta_b200.so")
-SOURCES = ["ta_api.cu", "ta_simt.cu", "ta_tc.cu", "ta_tc_fused.cu", "ta_tc_long.cu", "ta_tc_bwd.cu", "ta_simt_bwd.cu", "ta_backward.cu", "ta_noalloc.cu"]
+SOURCES = ["ta_api.cu", "ta_simt.cu", "ta_tc.cu", "ta_tc_fused.cu", "ta_tc_long.cu", "ta_tc_bwd.cu", "ta_tc_bwd_long.cu", "ta_simt_bwd.cu", "ta_backward.cu", "ta_noalloc.cu"]
 
 
 def _stale() -> bool:

@@ -571,11 +571,12 @@ int ta_plan_describe(int B, int H, int H_kv, int N, int D, const int *dims, int 
 
 int ta_device_status(void) {
     if (cudaDeviceSynchronize() != cudaSuccess) return TA_ERR_CUDA;
-    unsigned int w1 = 0, w2 = 0, w3 = 0, w4 = 0;
+    unsigned int w1 = 0, w2 = 0, w3 = 0, w4 = 0, w5 = 0;
     if (read_status_tc_forward(&w1) != TA_OK || read_status_tc_backward(&w2) != TA_OK ||
-        read_status_tc_fused(&w3) != TA_OK || read_status_tc_long(&w4) != TA_OK)
+        read_status_tc_fused(&w3) != TA_OK || read_status_tc_long(&w4) != TA_OK ||
+        read_status_tc_backward_long(&w5) != TA_OK)
         return TA_ERR_CUDA;
-    return (w1 | w2 | w3 | w4) ? TA_ERR_TIMEOUT : TA_OK;
+    return (w1 | w2 | w3 | w4 | w5) ? TA_ERR_TIMEOUT : TA_OK;
 }
 
 unsigned long long ta_launch_count(void) { return g_launches.load(); }

@@ -149,11 +149,15 @@ int backward_impl(const ta_bwd_params &p) {
             void *g_out = nullptr;
             if (j > 0) g_out = (h.path == PATH_TC && g_in != p.dout) ? const_cast<void *>(g_in)
                                                                       : (g_in == gbuf[0] ? gbuf[1] : gbuf[0]);
-            rc = h.path == PATH_TC
-                     ? launch_hop_tc_bwd(pb, h, hop_input(j), j == 0 ? p.H_kv : p.H, g_in, g_out, dq_acc, dk_acc, dv_acc,
-                                         j == 0, j != k - 1)
-                     : launch_hop_simt_bwd(pb, h, hop_input(j), j == 0 ? p.H_kv : p.H, g_in, g_out, dq_acc, dk_acc,
-                                           dv_acc, stats, j == 0, j != k - 1);
+            const int x_heads = j == 0 ? p.H_kv : p.H;
+            if (h.path == PATH_TC)
+                rc = launch_hop_tc_bwd(pb, h, hop_input(j), x_heads, g_in, g_out, dq_acc, dk_acc, dv_acc, j == 0, j != k - 1);
+            else if (tc_bwd_long_eligible(pb, h))
+                rc = launch_hop_tc_bwd_long(pb, h, hop_input(j), x_heads, g_in, g_out, dq_acc, dk_acc, dv_acc, stats, j == 0,
+                                            j != k - 1);
+            else
+                rc = launch_hop_simt_bwd(pb, h, hop_input(j), x_heads, g_in, g_out, dq_acc, dk_acc, dv_acc, stats, j == 0,
+                                         j != k - 1);
             if (rc != TA_OK) return rc;
             g_in = g_out;
         }

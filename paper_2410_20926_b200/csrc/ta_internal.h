@@ -98,6 +98,10 @@ int launch_hop_tc(const Problem &pb, const HopDesc &hd, const void *xin, int xin
 // Long segments (n_i > 128): key-block loop with online softmax, ta_tc_long.cu.  xin != xout.
 int launch_hop_tc_long(const Problem &pb, const HopDesc &hd, const void *xin, int xin_heads, void *xout);
 int read_status_tc_long(unsigned int *word);
+// Statistics pass of the long-segment backward: stats[q_head * N + token] = (log2-sum-exp of the
+// row's scaled scores, <g_t, out_t>), B*H*N float2; g laid out like q.
+int launch_hop_tc_long_stats(const Problem &pb, const HopDesc &hd, const void *xin, int xin_heads, const void *g,
+                             void *stats);
 // Library-owned buffer of at least `bytes` (grown on demand) for that kernel's rotated Q / K copies.
 int rotated_arena(size_t bytes, void **ptr);
 // Fused trailing hops (hd.nf > 1), ta_tc_fused.cu; called through launch_hop_tc.
@@ -118,6 +122,13 @@ int launch_hop_tc_bwd(const Problem &pb, const HopDesc &hd, const void *x, int x
 int launch_hop_simt_bwd(const Problem &pb, const HopDesc &hd, const void *x, int x_heads, const void *g_in,
                         void *g_out, float *dq_acc, float *dk_acc, float *dv_acc, void *stats, bool first_hop,
                         bool accumulate);
+// Backward of a long-segment hop on tensor cores (ta_tc_bwd_long.cu) where tc_bwd_long_eligible:
+// bf16, D in {64,128}, no window / mask / valid lengths / positional encoding.  Same arguments as
+// launch_hop_simt_bwd (g_out != g_in; stats: B*H*N float2 of scratch).
+bool tc_bwd_long_eligible(const Problem &pb, const HopDesc &hd);
+int launch_hop_tc_bwd_long(const Problem &pb, const HopDesc &hd, const void *x, int x_heads, const void *g_in,
+                           void *g_out, float *dq_acc, float *dk_acc, float *dv_acc, void *stats, bool first_hop,
+                           bool accumulate);
 int launch_f32_to_bf16(const float *src, void *dst, long long n, cudaStream_t stream);
 int launch_group_sum(const void *dout, void *dv, int dv_is_f32, int B, int H, int H_kv, long long per_head,
                      cudaStream_t stream);
@@ -139,6 +150,7 @@ int make_view_map(CUtensorMap *map, const void *base, int heads_total, int N, in
 int read_status_tc_forward(unsigned int *word);
 int read_status_tc_backward(unsigned int *word);
 int read_status_tc_fused(unsigned int *word);
+int read_status_tc_backward_long(unsigned int *word);
 
 // CUDA error code seen by the last call of this host thread that returned TA_ERR_CUDA.
 extern thread_local int tl_last_cuda_error;

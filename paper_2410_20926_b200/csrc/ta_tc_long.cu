@@ -44,6 +44,11 @@ struct LongArgs {
     float scale_log2;
     const int *lens;           // device, valid length per batch entry, or nullptr (kWindow variant only)
     int N;
+    // statistics pass of the backward: instead of the output rows, write per query row
+    // (log2-sum-exp of the scaled scores, <G_t, O_t>) -- stats[q_head * N + token]; g = gradient
+    // with respect to the hop's output, laid out like q
+    float2 *stats;
+    const __nv_bfloat16 *stats_g;
 };
 
 template <int D>
@@ -456,7 +461,32 @@ hop_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
-            {
+            if (a.stats != nullptr) {
+                const float inv = (row_valid && l_run > 0.f) ? 1.f / l_run : 0.f;
+                const long long row_off = (long long)c.q_head * a.head_stride + (long long)c.outer * a.seg_outer_stride +
+                                          (long long)t * a.row_stride + (long long)c.inner * D;
+                const __nv_bfloat16 *grow = a.stats_g + row_off;
+                float dot = 0.f;
+                uint32_t v[32];
+#pragma unroll 1
+                for (int cc = 0; cc < D / 32; ++cc) {
+                    tmem_ld32(o_col + 32 * cc, v);
+                    if (row_valid) {
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const uint4 w = __ldg(reinterpret_cast<const uint4 *>(grow + 32 * cc + 8 * i));
+                            const uint32_t ws[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                dot = fmaf(__uint_as_float(ws[e] << 16), __uint_as_float(v[8 * i + 2 * e]), dot);
+                                dot = fmaf(__uint_as_float(ws[e] & 0xFFFF0000u), __uint_as_float(v[8 * i + 2 * e + 1]), dot);
+                            }
+                        }
+                    }
+                }
+                if (row_valid)
+                    a.stats[row_off / D] = make_float2(l_run > 0.f ? m_run + log2f(l_run) : INFINITY, dot * inv);
+            } else {
                 const float inv = (row_valid && l_run > 0.f) ? 1.f / l_run : 0.f;
                 __nv_bfloat16 *dst = xout + (long long)c.q_head * a.head_stride + (long long)c.outer * a.seg_outer_stride +
                                      (long long)t * a.row_stride + (long long)c.inner * D;
@@ -490,7 +520,8 @@ hop_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 }
 
 template <int D>
-int launch_long_d(const Problem &pb, const HopDesc &hd, const void *xin, int xin_heads, void *xout) {
+int launch_long_d(const Problem &pb, const HopDesc &hd, const void *xin, int xin_heads, void *xout, void *stats = nullptr,
+                  const void *stats_g = nullptr) {
     CUtensorMap mq, mk, mxi;
     int rc;
     // box: 128 positions of one segment (positions past n are zero-filled / clipped)
@@ -512,6 +543,8 @@ int launch_long_d(const Problem &pb, const HopDesc &hd, const void *xin, int xin
     a.scale_log2 = pb.scale * 1.4426950408889634f;
     a.lens = pb.seq_lens;
     a.N = pb.N;
+    a.stats = (float2 *)stats;
+    a.stats_g = (const __nv_bfloat16 *)stats_g;
 
     int dev = 0;
     const int num_sms = current_device_sms(&dev);
@@ -590,6 +623,16 @@ int launch_hop_tc_long(const Problem &pb, const HopDesc &hd, const void *xin, in
     }
     if (pb.D == 128) return launch_long_d<128>(hop, hd, xin, xin_heads, xout);
     return launch_long_d<64>(hop, hd, xin, xin_heads, xout);
+}
+
+// The backward's statistics pass over a long-segment hop (no positional encoding): same pipeline,
+// per query row (log2-sum-exp of the scaled scores, <G_t, O_t>) instead of the output.
+int launch_hop_tc_long_stats(const Problem &pb, const HopDesc &hd, const void *xin, int xin_heads, const void *g,
+                             void *stats) {
+    if (pb.rope_base > 0.f || !stats || !g) return TA_ERR_INVALID_ARG;
+    if (pb.D == 128) return launch_long_d<128>(pb, hd, xin, xin_heads, nullptr, stats, g);
+    if (pb.D == 64) return launch_long_d<64>(pb, hd, xin, xin_heads, nullptr, stats, g);
+    return TA_ERR_UNSUPPORTED;
 }
 
 int read_status_tc_long(unsigned int *word) {

@@ -246,3 +246,22 @@ def test_backward_fp32_storage(dims, D, causal, B, H, Hkv, kw):
     rc = ta.ta_backward_ex(do, q, k, v, dq, dk, dv, B, H, Hkv, N, D, dims, causal, dtype=ta.TA_DTYPE_F32,
                            grad_dtype=ta.TA_DTYPE_BF16, workspace=ws, workspace_bytes=nbytes, check=False)
     assert rc == ta.TA_ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("dims,D,causal,B,H,Hkv", [
+    ([1024], 128, True, 1, 4, 2),                 # ordinary attention, 8 key blocks
+    ([700], 64, False, 2, 2, 1),                  # ragged last block, every query tile meets every block
+    ([2, 384], 128, True, 1, 4, 4),               # short hop (in place) then long hop
+    ([260, 3], 64, True, 1, 4, 2),                # long hop first: its gradient is dV, summed over the group
+    ([3, 300, 2], 128, False, 1, 2, 1),           # tensor-core short, long, short
+])
+def test_backward_long_segments_tensor_core(dims, D, causal, B, H, Hkv):
+    """Segments longer than 128 (no window, mask, lengths or positional encoding) run their backward
+    on the long-segment tensor-core kernel: statistics pass, then key block by key block."""
+    N = math.prod(dims)
+    inp = ta_inputs.make_inputs(B, H, Hkv, N, D, "bf16", 175, with_dout=True)
+    ref = oracle.backward(inp["dout"], inp["q"], inp["k"], inp["v"], dims, causal)
+    for grad_f32 in (True, False):
+        got = gpu_backward(inp, B, H, Hkv, N, D, dims, causal, grad_f32)
+        for name, g, r in zip(("dq", "dk", "dv"), got, ref):
+            assert_grad_close(g, r, name)
