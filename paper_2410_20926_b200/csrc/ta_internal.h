@@ -123,7 +123,7 @@ int launch_hop_simt_bwd(const Problem &pb, const HopDesc &hd, const void *x, int
                         void *g_out, float *dq_acc, float *dk_acc, float *dv_acc, void *stats, bool first_hop,
                         bool accumulate);
 // Backward of a long-segment hop on tensor cores (ta_tc_bwd_long.cu) where tc_bwd_long_eligible:
-// bf16, D in {64,128}, no window / mask / valid lengths / positional encoding.  Same arguments as
+// bf16, D in {64,128}, no explicit mask, no positional encoding.  Same arguments as
 // launch_hop_simt_bwd (g_out != g_in; stats: B*H*N float2 of scratch).
 bool tc_bwd_long_eligible(const Problem &pb, const HopDesc &hd);
 int launch_hop_tc_bwd_long(const Problem &pb, const HopDesc &hd, const void *x, int x_heads, const void *g_in,

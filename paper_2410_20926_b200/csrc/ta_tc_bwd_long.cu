@@ -1,6 +1,6 @@
 // Tensor-core backward kernel for one hop with segments longer than a tile (n_i > 128) on sm_100a:
-// bf16 storage, head dim 64 or 128, causal or not, no window / positional encoding / valid lengths
-// (those run on the generic kernels).  The chain rule through X_{i+1} = A_i X_i (the paper gives
+// bf16 storage, head dim 64 or 128, causal flag, sliding window and valid lengths as in the forward
+// (explicit masks and the positional encoding run on the generic kernels).  The chain rule through X_{i+1} = A_i X_i (the paper gives
 // no backward), block by block as in the long-segment forward:
 //
 //     P_ij  = exp2(S_ij * scale * log2 e - lse_i)          S_ij = Q_i K_j^T,  lse_i from the statistics pass
@@ -36,6 +36,8 @@ struct LongBwdArgs {
     long long stride, outer, total_items;
     float scale_log2, scale;
     const float2 *stats;               // [B*H][N]: (lse in the log2 domain, delta)
+    int window;                        // 0, or sliding window along the hop's dimension
+    const int *lens;                   // device, valid length per batch entry, or nullptr
 };
 
 template <int D>
@@ -59,7 +61,8 @@ struct LongBwdCfg {
 
 struct LongBwdItem {
     int jb, inner, outer, kv_head, q_head0;
-    int i_lo, steps_per_head;          // query tiles [i_lo, nblocks) see this key block
+    int i_lo, steps_per_head;          // query tiles [i_lo, i_lo + steps_per_head) can see this key block
+    int exist;                         // positions of the segment that are tokens (n without valid lengths)
 };
 __device__ __forceinline__ LongBwdItem decode_item(const LongBwdArgs &a, long long item) {
     LongBwdItem c;
@@ -72,7 +75,20 @@ __device__ __forceinline__ LongBwdItem decode_item(const LongBwdArgs &a, long lo
     c.kv_head = (int)rest;
     c.q_head0 = (c.kv_head / a.H_kv) * a.H + (c.kv_head % a.H_kv) * a.g;
     c.i_lo = a.causal ? c.jb : 0;
-    c.steps_per_head = a.nblocks - c.i_lo;
+    int i_hi = a.nblocks - 1;
+    if (a.window > 0) {                // tiles with a row within the window of one of the block's keys
+        const int u0 = kTileRows * c.jb, u1 = min(a.n, u0 + kTileRows) - 1;
+        if (!a.causal) c.i_lo = max(0, u0 - a.window + 1) / kTileRows;
+        i_hi = min(i_hi, (u1 + a.window - 1) / kTileRows);
+    }
+    c.steps_per_head = i_hi - c.i_lo + 1;
+    c.exist = a.n;
+    if (a.lens != nullptr) {
+        const long long len = min(max(__ldg(a.lens + c.kv_head / a.H_kv), 0), a.N);
+        const long long first_token = (long long)c.outer * a.n * a.stride + c.inner;
+        const long long left = (len - first_token + a.stride - 1) / a.stride;
+        c.exist = len <= first_token ? 0 : (int)(left < a.n ? left : a.n);
+    }
     return c;
 }
 
@@ -219,7 +235,8 @@ hop_tc_bwd_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
         for (long long item = blockIdx.x; ok && item < a.total_items; item += gridDim.x, ++it) {
             const LongBwdItem c = decode_item(a, item);
             const int steps = a.g * c.steps_per_head;
-            const int keys = min(kTileRows, a.n - kTileRows * c.jb);          // key positions of the block
+            // key positions of the block that are tokens (none: every weight is 0 and the item writes zeros)
+            const int keys = max(0, min(kTileRows, min(a.n, c.exist) - kTileRows * c.jb));
             for (int v = 0; v < steps; ++v, ++t) {
                 const int s = t & 1;
                 const uint32_t par = t & 1;
@@ -273,12 +290,18 @@ hop_tc_bwd_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                 // ---- P and dS of this thread's query row from its statistics; P -> X slot, dS -> its slot
                 {
                     const int tq = kTileRows * qi + r;                       // position of the row in the segment
-                    const bool row_in = tq < a.n;
+                    const bool row_in = tq < min(a.n, c.exist);
                     float2 st = make_float2(INFINITY, 0.f);
                     if (row_in)
                         st = __ldg(a.stats + (long long)q_head * a.N + ((long long)c.outer * a.n + tq) * a.stride + c.inner);
-                    // key columns this row sees in the block: [0, c_hi)
-                    const int c_hi = !row_in ? 0 : ((a.causal && qi == c.jb) ? min(keys, r + 1) : keys);
+                    // key columns this row sees in the block: [c_lo, c_hi)
+                    int c_hi = !row_in ? 0 : ((a.causal && qi == c.jb) ? min(keys, r + 1) : keys);
+                    int c_lo = 0;
+                    if (a.window > 0) {
+                        const int u0 = kTileRows * c.jb;
+                        c_lo = max(0, tq - a.window + 1 - u0);
+                        if (!a.causal) c_hi = min(c_hi, tq + a.window - u0);
+                    }
                     const uint32_t rowP = sXP + (uint32_t)r * 128u, rowS = sdS + (uint32_t)r * 128u;
                     uint32_t vs[32], vd[32];
 #pragma unroll 1
@@ -291,7 +314,7 @@ hop_tc_bwd_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                             float pv[2], dv[2];
 #pragma unroll
                             for (int e = 0; e < 2; ++e) {
-                                const bool vis = 32 * cc + jj + e < c_hi;
+                                const bool vis = 32 * cc + jj + e >= c_lo && 32 * cc + jj + e < c_hi;
                                 float p = fast_exp2(__uint_as_float(vs[jj + e]) * a.scale_log2 - st.x);
                                 p = vis ? p : 0.f;
                                 pv[e] = p;
@@ -461,6 +484,8 @@ int launch_d(const Problem &pb, const HopDesc &hd, const void *x, int x_heads, c
     a.scale = pb.scale;
     a.scale_log2 = pb.scale * 1.4426950408889634f;
     a.stats = (const float2 *)stats;
+    a.window = pb.window[hd.hop];
+    a.lens = pb.seq_lens;
 
     int dev = 0;
     const int num_sms = current_device_sms(&dev);
@@ -482,7 +507,7 @@ int launch_d(const Problem &pb, const HopDesc &hd, const void *x, int x_heads, c
 // Conditions under which this kernel takes a long-segment hop (else the generic backward does).
 bool tc_bwd_long_eligible(const Problem &pb, const HopDesc &hd) {
     return hd.path == PATH_TC_LONG && pb.dtype == TA_DTYPE_BF16 && (pb.D == 64 || pb.D == 128) && pb.rope_base == 0.f &&
-           pb.window[hd.hop] == 0 && pb.masks[hd.hop] == nullptr && pb.seq_lens == nullptr;
+           pb.masks[hd.hop] == nullptr;
 }
 
 int launch_hop_tc_bwd_long(const Problem &pb, const HopDesc &hd, const void *x, int x_heads, const void *g_in,

@@ -265,3 +265,27 @@ def test_backward_long_segments_tensor_core(dims, D, causal, B, H, Hkv):
         got = gpu_backward(inp, B, H, Hkv, N, D, dims, causal, grad_f32)
         for name, g, r in zip(("dq", "dk", "dv"), got, ref):
             assert_grad_close(g, r, name)
+
+
+@pytest.mark.parametrize("dims,D,causal,kw", [
+    ([700], 64, False, {"window": [90]}),                  # two-sided window: tiles outside it are skipped
+    ([1024], 128, True, {"window": [130]}),
+    ([2, 384], 128, True, {"window": [0, 200]}),
+    ([700], 64, False, {"lens": [333, 700]}),              # batch entries of different lengths
+    ([3, 300], 128, True, {"lens": [450, 1]}),
+    ([600], 64, True, {"lens": [600, 129], "window": [64]}),
+])
+def test_backward_long_segments_windows_and_lengths(dims, D, causal, kw):
+    import torch
+    B, H, Hkv = 2, 4, 2
+    N = math.prod(dims)
+    lens, window = kw.get("lens"), kw.get("window")
+    inp = ta_inputs.make_inputs(B, H, Hkv, N, D, "bf16", 176, with_dout=True)
+    got = gpu_backward(inp, B, H, Hkv, N, D, dims, causal, True, window=window,
+                       seq_lens=None if lens is None else torch.tensor(lens, dtype=torch.int32, device="cuda"))
+    ref = oracle.backward(inp["dout"], inp["q"], inp["k"], inp["v"], dims, causal, window=window, seq_lens=lens)
+    for name, g, r in zip(("dq", "dk", "dv"), got, ref):
+        assert_grad_close(g, r, name)
+        if lens is not None:
+            for b, L in enumerate(lens):
+                assert (g[b, :, L:] == 0).all(), name
