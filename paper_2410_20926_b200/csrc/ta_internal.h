@@ -98,6 +98,11 @@ int launch_hop_tc(const Problem &pb, const HopDesc &hd, const void *xin, int xin
 // Long segments (n_i > 128): key-block loop with online softmax, ta_tc_long.cu.  xin != xout.
 int launch_hop_tc_long(const Problem &pb, const HopDesc &hd, const void *xin, int xin_heads, void *xout);
 int read_status_tc_long(unsigned int *word);
+// Positional encoding on long-segment hops: rotated bf16 copies of q and k in the library-owned
+// buffer (plus extra_bytes of scratch behind them), and dst (=|+=) R^T src for fp32 gradients.
+int rope_rotated_copies(const Problem &pb, const HopDesc &hd, const void **rq, const void **rk, size_t extra_bytes,
+                        void **extra);
+int rope_unrotate_add(const Problem &pb, const HopDesc &hd, const float *src, float *dst, int heads, bool accumulate);
 // Statistics pass of the long-segment backward: stats[q_head * N + token] = (log2-sum-exp of the
 // row's scaled scores, <g_t, out_t>), B*H*N float2; g laid out like q.
 int launch_hop_tc_long_stats(const Problem &pb, const HopDesc &hd, const void *xin, int xin_heads, const void *g,
@@ -123,7 +128,7 @@ int launch_hop_simt_bwd(const Problem &pb, const HopDesc &hd, const void *x, int
                         void *g_out, float *dq_acc, float *dk_acc, float *dv_acc, void *stats, bool first_hop,
                         bool accumulate);
 // Backward of a long-segment hop on tensor cores (ta_tc_bwd_long.cu) where tc_bwd_long_eligible:
-// bf16, D in {64,128}, no explicit mask, no positional encoding.  Same arguments as
+// bf16, D in {64,128}, no explicit mask.  Same arguments as
 // launch_hop_simt_bwd (g_out != g_in; stats: B*H*N float2 of scratch).
 bool tc_bwd_long_eligible(const Problem &pb, const HopDesc &hd);
 int launch_hop_tc_bwd_long(const Problem &pb, const HopDesc &hd, const void *x, int x_heads, const void *g_in,

@@ -1,6 +1,7 @@
 // Tensor-core backward kernel for one hop with segments longer than a tile (n_i > 128) on sm_100a:
 // bf16 storage, head dim 64 or 128, causal flag, sliding window and valid lengths as in the forward
-// (explicit masks and the positional encoding run on the generic kernels).  The chain rule through X_{i+1} = A_i X_i (the paper gives
+// (explicit masks run on the generic kernels; with the positional encoding the hop runs on rotated
+// copies of q and k and its dQ, dK are turned back afterwards).  The chain rule through X_{i+1} = A_i X_i (the paper gives
 // no backward), block by block as in the long-segment forward:
 //
 //     P_ij  = exp2(S_ij * scale * log2 e - lse_i)          S_ij = Q_i K_j^T,  lse_i from the statistics pass
@@ -506,7 +507,7 @@ int launch_d(const Problem &pb, const HopDesc &hd, const void *x, int x_heads, c
 
 // Conditions under which this kernel takes a long-segment hop (else the generic backward does).
 bool tc_bwd_long_eligible(const Problem &pb, const HopDesc &hd) {
-    return hd.path == PATH_TC_LONG && pb.dtype == TA_DTYPE_BF16 && (pb.D == 64 || pb.D == 128) && pb.rope_base == 0.f &&
+    return hd.path == PATH_TC_LONG && pb.dtype == TA_DTYPE_BF16 && (pb.D == 64 || pb.D == 128) &&
            pb.masks[hd.hop] == nullptr;
 }
 
@@ -515,6 +516,23 @@ int launch_hop_tc_bwd_long(const Problem &pb, const HopDesc &hd, const void *x, 
                            bool accumulate) {
     if (!tc_bwd_long_eligible(pb, hd)) return TA_ERR_UNSUPPORTED;
     if (!first_hop && (g_out == nullptr || g_out == g_in)) return TA_ERR_INVALID_ARG;   // other items read g_in
+    if (pb.rope_base > 0.f) {
+        // Positional encoding: the hop runs on rotated copies of q and k (as in the forward); its dQ
+        // and dK are gradients with respect to the rotated vectors, so they go to scratch of their own
+        // and are turned back (R^T) while they are stored in / added to the accumulators.
+        const size_t tq = (size_t)pb.B * pb.H * pb.N * pb.D, tkv = (size_t)pb.B * pb.H_kv * pb.N * pb.D;
+        Problem hop = pb;
+        void *extra = nullptr;
+        int rc = rope_rotated_copies(pb, hd, &hop.q, &hop.k, (tq + tkv) * sizeof(float), &extra);
+        if (rc != TA_OK) return rc;
+        hop.rope_base = 0.f;
+        float *dq_rot = (float *)extra, *dk_rot = dq_rot + tq;
+        rc = pb.D == 128 ? launch_d<128>(hop, hd, x, x_heads, g_in, g_out, dq_rot, dk_rot, dv_acc, stats, first_hop, false)
+                         : launch_d<64>(hop, hd, x, x_heads, g_in, g_out, dq_rot, dk_rot, dv_acc, stats, first_hop, false);
+        if (rc != TA_OK) return rc;
+        if ((rc = rope_unrotate_add(pb, hd, dq_rot, dq_acc, pb.H, accumulate)) != TA_OK) return rc;
+        return rope_unrotate_add(pb, hd, dk_rot, dk_acc, pb.H_kv, accumulate);
+    }
     if (pb.D == 128)
         return launch_d<128>(pb, hd, x, x_heads, g_in, g_out, dq_acc, dk_acc, dv_acc, stats, first_hop, accumulate);
     return launch_d<64>(pb, hd, x, x_heads, g_in, g_out, dq_acc, dk_acc, dv_acc, stats, first_hop, accumulate);

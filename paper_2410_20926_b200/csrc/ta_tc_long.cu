@@ -597,28 +597,69 @@ __global__ void rope_copy_kernel(const __nv_bfloat16 *__restrict__ src, __nv_bfl
 }
 }  // namespace
 
+// dst (fp32) = or += the transposed rotation of src (fp32): gradients with respect to rotated
+// vectors turned back to gradients with respect to the un-rotated ones.
+namespace {
+__global__ void rope_unrotate_add_kernel(const float *__restrict__ src, float *__restrict__ dst, long long pairs, int N,
+                                         int D, long long stride, int n, double log2_base, int accumulate) {
+    const int half = D >> 1;
+    for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < pairs;
+         idx += (long long)gridDim.x * blockDim.x) {
+        const int c = (int)(idx % half);
+        const long long row = idx / half;
+        const long long token = row % N;
+        const int pos = (int)((token / stride) % n);
+        const double theta = exp2(-2.0 * (double)c / (double)D * log2_base);
+        const double angle = fmod((double)pos * theta, 6.283185307179586476925);
+        float sn, cs;
+        sincosf((float)angle, &sn, &cs);
+        const long long o = row * D + c;
+        const float x1 = src[o], x2 = src[o + half];
+        const float y1 = x1 * cs + x2 * sn, y2 = x2 * cs - x1 * sn;
+        dst[o] = accumulate ? dst[o] + y1 : y1;
+        dst[o + half] = accumulate ? dst[o + half] + y2 : y2;
+    }
+}
+unsigned rope_blocks(long long pairs) { return (unsigned)(pairs / 256 + 1 < 148 * 32 ? pairs / 256 + 1 : 148 * 32); }
+}  // namespace
+
+// Rotated bf16 copies of q and k for hop `hd` in the library-owned buffer, followed by
+// `extra_bytes` of scratch (*extra).
+int rope_rotated_copies(const Problem &pb, const HopDesc &hd, const void **rq_out, const void **rk_out,
+                        size_t extra_bytes, void **extra) {
+    const size_t tq = (size_t)pb.B * pb.H * pb.N * pb.D, tkv = (size_t)pb.B * pb.H_kv * pb.N * pb.D;
+    const size_t q_bytes = (tq * 2 + 255) & ~(size_t)255, k_bytes = (tkv * 2 + 255) & ~(size_t)255;
+    void *buf = nullptr;
+    int rc = rotated_arena(q_bytes + k_bytes + extra_bytes, &buf);
+    if (rc != TA_OK) return rc;
+    __nv_bfloat16 *rq = (__nv_bfloat16 *)buf, *rk = (__nv_bfloat16 *)((char *)buf + q_bytes);
+    const double log2_base = log2((double)pb.rope_base);
+    const long long pq = (long long)(tq / 2), pk = (long long)(tkv / 2);
+    rc = launch_kernel(rope_copy_kernel, rope_blocks(pq), 256, 0, pb.stream, false, (const __nv_bfloat16 *)pb.q, rq, pq,
+                       pb.N, pb.D, (long long)hd.stride, hd.n, log2_base);
+    if (rc != TA_OK) return rc;
+    rc = launch_kernel(rope_copy_kernel, rope_blocks(pk), 256, 0, pb.stream, false, (const __nv_bfloat16 *)pb.k, rk, pk,
+                       pb.N, pb.D, (long long)hd.stride, hd.n, log2_base);
+    if (rc != TA_OK) return rc;
+    *rq_out = rq;
+    *rk_out = rk;
+    if (extra) *extra = (char *)buf + q_bytes + k_bytes;
+    return TA_OK;
+}
+
+int rope_unrotate_add(const Problem &pb, const HopDesc &hd, const float *src, float *dst, int heads, bool accumulate) {
+    const long long pairs = (long long)pb.B * heads * pb.N * pb.D / 2;
+    return launch_kernel(rope_unrotate_add_kernel, rope_blocks(pairs), 256, 0, pb.stream, false, src, dst, pairs, pb.N,
+                         pb.D, (long long)hd.stride, hd.n, log2((double)pb.rope_base), accumulate ? 1 : 0);
+}
+
 int launch_hop_tc_long(const Problem &pb, const HopDesc &hd, const void *xin, int xin_heads, void *xout) {
     if (xin == xout) return TA_ERR_INVALID_ARG;
     if (pb.D != 128 && pb.D != 64) return TA_ERR_UNSUPPORTED;
     Problem hop = pb;
     if (pb.rope_base > 0.f) {
-        const size_t tq = (size_t)pb.B * pb.H * pb.N * pb.D, tkv = (size_t)pb.B * pb.H_kv * pb.N * pb.D;
-        const size_t q_bytes = (tq * 2 + 255) & ~(size_t)255;
-        void *buf = nullptr;
-        int rc = rotated_arena(q_bytes + tkv * 2, &buf);
+        const int rc = rope_rotated_copies(pb, hd, &hop.q, &hop.k, 0, nullptr);
         if (rc != TA_OK) return rc;
-        __nv_bfloat16 *rq = (__nv_bfloat16 *)buf, *rk = (__nv_bfloat16 *)((char *)buf + q_bytes);
-        const double log2_base = log2((double)pb.rope_base);
-        const long long pq = (long long)(tq / 2), pk = (long long)(tkv / 2);
-        auto blocks = [](long long pairs) { return (unsigned)(pairs / 256 + 1 < 148 * 32 ? pairs / 256 + 1 : 148 * 32); };
-        rc = launch_kernel(rope_copy_kernel, blocks(pq), 256, 0, pb.stream, false, (const __nv_bfloat16 *)pb.q, rq, pq, pb.N,
-                           pb.D, (long long)hd.stride, hd.n, log2_base);
-        if (rc != TA_OK) return rc;
-        rc = launch_kernel(rope_copy_kernel, blocks(pk), 256, 0, pb.stream, false, (const __nv_bfloat16 *)pb.k, rk, pk, pb.N,
-                           pb.D, (long long)hd.stride, hd.n, log2_base);
-        if (rc != TA_OK) return rc;
-        hop.q = rq;
-        hop.k = rk;
         hop.rope_base = 0.f;
     }
     if (pb.D == 128) return launch_long_d<128>(hop, hd, xin, xin_heads, xout);

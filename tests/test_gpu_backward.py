@@ -274,6 +274,9 @@ def test_backward_long_segments_tensor_core(dims, D, causal, B, H, Hkv):
     ([700], 64, False, {"lens": [333, 700]}),              # batch entries of different lengths
     ([3, 300], 128, True, {"lens": [450, 1]}),
     ([600], 64, True, {"lens": [600, 129], "window": [64]}),
+    ([1024], 128, True, {"rope_base": 10000.0}),           # ordinary attention with RoPE
+    ([3, 300], 64, False, {"rope_base": 10000.0, "window": [0, 100]}),
+    ([260, 2], 128, True, {"rope_base": 10000.0, "lens": [500, 77]}),
 ])
 def test_backward_long_segments_windows_and_lengths(dims, D, causal, kw):
     import torch
@@ -281,9 +284,11 @@ def test_backward_long_segments_windows_and_lengths(dims, D, causal, kw):
     N = math.prod(dims)
     lens, window = kw.get("lens"), kw.get("window")
     inp = ta_inputs.make_inputs(B, H, Hkv, N, D, "bf16", 176, with_dout=True)
-    got = gpu_backward(inp, B, H, Hkv, N, D, dims, causal, True, window=window,
+    rope = kw.get("rope_base", 0.0)
+    got = gpu_backward(inp, B, H, Hkv, N, D, dims, causal, True, window=window, rope_base=rope,
                        seq_lens=None if lens is None else torch.tensor(lens, dtype=torch.int32, device="cuda"))
-    ref = oracle.backward(inp["dout"], inp["q"], inp["k"], inp["v"], dims, causal, window=window, seq_lens=lens)
+    ref = oracle.backward(inp["dout"], inp["q"], inp["k"], inp["v"], dims, causal, window=window, seq_lens=lens,
+                          rope_base=rope or None)
     for name, g, r in zip(("dq", "dk", "dv"), got, ref):
         assert_grad_close(g, r, name)
         if lens is not None:
