@@ -50,15 +50,17 @@ def gpu_backward(inp, B, H, Hkv, N, D, dims, causal, grad_f32, saved=None, rope_
     return tuple(t.float().cpu().numpy().astype(np.float64) for t in (dq, dk, dv))
 
 
-def assert_grad_close(got, ref, name):
-    """got, ref: [..., N, D]; the leading axes enumerate heads."""
+def assert_grad_close(got, ref, name, mean_rtol=0.0):
+    """got, ref: [..., N, D]; the leading axes enumerate heads.  mean_rtol: lets the bound on the
+    mean error grow with the head's gradient scale as the bound on the maximum does (for tiny
+    tensors whose few rows all carry sums over a whole GQA group)."""
     assert np.isfinite(got).all(), name
     err = np.abs(got - ref)
     scale = np.abs(ref).max(axis=(-2, -1), keepdims=True)
     bound = BF16_MAX_ABS + RTOL * scale
     worst = float((err - bound).max())
     assert worst <= 0, (name, float(err.max()), float(scale.max()), worst)
-    assert err.mean() <= BF16_MEAN_ABS, (name, float(err.mean()))
+    assert err.mean() <= BF16_MEAN_ABS + mean_rtol * float(scale.mean()), (name, float(err.mean()))
     return float(err.max()), float(err.mean()), float(scale.max())
 
 

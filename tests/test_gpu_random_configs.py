@@ -1,0 +1,79 @@
+"""Seeded random configurations: tensor shapes, head dims, GQA ratios and every combination of the
+options (causal flag, windows, explicit masks, valid lengths, positional encoding, fusion on/off),
+forward and backward, against the fp64 oracle.  Catches interactions the targeted tests do not
+enumerate.  Tolerances as everywhere else, except that the bound on the mean error of a gradient
+grows with the size of the gradient the way the bound on its maximum does: some of these tensors
+have a handful of rows, each a sum over a whole GQA group."""
+import math
+
+import numpy as np
+import pytest
+
+import oracle
+import paper_2410_20926_b200 as ta
+from paper_2410_20926_b200 import inputs as ta_inputs
+
+from helpers import assert_close, gpu_forward
+from test_gpu_backward import assert_grad_close, gpu_backward
+
+pytestmark = pytest.mark.gpu
+
+
+def random_config(seed):
+    rng = np.random.default_rng(1000 + seed)
+    D = int(rng.choice([64, 128, 128, 64, 40]))
+    ndims = int(rng.integers(1, 5))
+    while True:
+        dims = [int(rng.choice([1, 2, 3, 4, 5, 8, 12, 16, 24, 32, 64, 100, 128, 150, 260])) for _ in range(ndims)]
+        N = math.prod(dims)
+        if 2 <= N <= 6000:
+            break
+    Hkv = int(rng.choice([1, 2]))
+    H = Hkv * int(rng.choice([1, 2, 4]))
+    B = int(rng.choice([1, 2]))
+    causal = bool(rng.integers(0, 2))
+    kw, okw = {}, {}
+    if rng.random() < 0.4:
+        w = [int(rng.integers(1, n + 1)) if (n > 1 and rng.random() < 0.7) else 0 for n in dims]
+        kw["window"], okw["window"] = w, w
+    if rng.random() < 0.3:
+        masks = []
+        for n in dims:
+            if n > 128 or n == 1 or rng.random() < 0.3:
+                masks.append(None)
+                continue
+            m = (rng.random((n, n)) < 0.6).astype(np.uint8)
+            m[np.arange(n), np.arange(n)] = 1
+            masks.append(m)
+        if any(m is not None for m in masks):
+            kw["hop_masks"], okw["masks"] = masks, masks
+    if rng.random() < 0.35:
+        lens = [int(rng.integers(0, N + 1)) for _ in range(B)]
+        kw["lens"], okw["seq_lens"] = lens, lens
+    if rng.random() < 0.35 and D % 2 == 0:
+        kw["rope_base"], okw["rope_base"] = 10000.0, 10000.0
+    flags = ta.TA_FLAG_NO_HOP_FUSION if rng.random() < 0.5 else 0
+    return B, H, Hkv, D, dims, causal, kw, okw, flags
+
+
+@pytest.mark.parametrize("seed", range(48))
+def test_random_configuration(seed):
+    import torch
+    B, H, Hkv, D, dims, causal, kw, okw, flags = random_config(seed)
+    N = math.prod(dims)
+    gkw = dict(kw)
+    lens = gkw.pop("lens", None)
+    if lens is not None:
+        gkw["seq_lens"] = torch.tensor(lens, dtype=torch.int32, device="cuda")
+    inp = ta_inputs.make_inputs(B, H, Hkv, N, D, "bf16", 2000 + seed, with_dout=True)
+    got = gpu_forward(inp, B, H, Hkv, N, D, dims, causal, "bf16", flags, **gkw)
+    ref = oracle.forward(inp["q"], inp["k"], inp["v"], dims, causal, **okw)
+    assert_close(got, ref, "bf16")
+    if all(n == 1 for n in dims) and lens is not None:
+        return                                   # no hop to apply the lengths in: the backward declines
+    bkw = {k: v for k, v in gkw.items()}
+    grads = gpu_backward(inp, B, H, Hkv, N, D, dims, causal, bool(seed % 2), **bkw)
+    refs = oracle.backward(inp["dout"], inp["q"], inp["k"], inp["v"], dims, causal, **okw)
+    for name, g, r in zip(("dq", "dk", "dv"), grads, refs):
+        # mean bound: a tenth of the bound on the maximum, as for the forward (2e-3 vs 2e-2)
+        assert_grad_close(g, r, name, mean_rtol=2.0 ** -8 / 10)
