@@ -6,7 +6,7 @@ import oracle
 import paper_2410_20926_b200 as ta
 from paper_2410_20926_b200 import inputs as ta_inputs
 
-# Tolerances stated for this build: bf16 storage / fp32 accumulate, and the fp32 path.
+# Tolerances: bf16 storage with fp32 accumulation, and the fp32 path.
 BF16_MAX_ABS, BF16_MEAN_ABS = 2e-2, 2e-3
 F32_MAX_ABS = 1e-4
 
