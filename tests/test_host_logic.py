@@ -177,3 +177,11 @@ def test_plan_fuses_trailing_dimensions_that_fit_a_tile():
     assert "tc-fused" not in ta.ta_plan_describe(1, 4, 4, 512, 64, [8, 8, 8], True, ta.TA_DTYPE_BF16,
                                                  ta.TA_FLAG_NO_HOP_FUSION)
     assert "tc-fused" not in ta.ta_plan_describe(1, 4, 4, 512, 64, [8, 8, 8], True, ta.TA_DTYPE_F32, 0)
+
+
+def test_autograd_binding_refuses_cpu_tensors_and_bad_shapes():
+    """The torch.autograd binding has no CPU path: it must say so before any library call."""
+    import torch
+    q = torch.zeros(1, 2, 16, 64, dtype=torch.bfloat16)
+    with pytest.raises(ValueError, match="CUDA"):
+        ta.tensorized_attention(q, q, q, [4, 4])
