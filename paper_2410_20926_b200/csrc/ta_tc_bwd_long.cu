@@ -67,10 +67,12 @@ struct LongBwdItem {
 };
 __device__ __forceinline__ LongBwdItem decode_item(const LongBwdArgs &a, long long item) {
     LongBwdItem c;
-    long long rest = item;
-    // the key blocks of a segment are adjacent items (when causal their loads differ: block 0 meets
-    // every query tile, the last block one), so a wave of CTAs carries a mix of long and short items
-    c.jb = (int)(rest % a.nblocks); rest /= a.nblocks;
+    // Items are numbered with the key block slowest: when causal, block 0 meets every query tile and
+    // the last block one, so the numbering runs from the longest items to the shortest (see
+    // item_of_round for how they are dealt to the CTAs).
+    const long long per_block = a.total_items / a.nblocks;
+    c.jb = (int)(item / per_block);
+    long long rest = item % per_block;
     c.inner = (int)(rest % a.stride); rest /= a.stride;
     c.outer = (int)(rest % a.outer); rest /= a.outer;
     c.kv_head = (int)rest;
@@ -91,6 +93,15 @@ __device__ __forceinline__ LongBwdItem decode_item(const LongBwdArgs &a, long lo
         c.exist = len <= first_token ? 0 : (int)(left < a.n ? left : a.n);
     }
     return c;
+}
+
+// The item a CTA takes in its k-th round: the rounds run forth and back over the CTAs, so that the
+// CTA that got the longest item of one round gets the shortest of the next (items are numbered
+// longest first).  -1: none in this round.
+__device__ __forceinline__ long long item_of_round(const LongBwdArgs &a, long long k) {
+    const long long g = gridDim.x, b = blockIdx.x;
+    const long long item = k * g + ((k & 1) ? g - 1 - b : b);
+    return item < a.total_items ? item : -1;
 }
 
 __device__ __forceinline__ bool wg_all(bool pred) {
@@ -161,7 +172,9 @@ hop_tc_bwd_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                 armed |= bit;
                 last_par = parity ? (last_par | bit) : (last_par & ~bit);
             };
-            for (long long item = blockIdx.x; ok && item < a.total_items; item += gridDim.x, ++it) {
+            for (long long round = 0; ok && round * gridDim.x < a.total_items; ++round) {
+                const long long item = item_of_round(a, round);
+                if (item < 0) continue;
                 const LongBwdItem c = decode_item(a, item);
                 const int steps = a.g * c.steps_per_head;
                 for (int v = 0; v < steps; ++v, ++t) {
@@ -197,6 +210,7 @@ hop_tc_bwd_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                     for (int h = 0; h < kHalves; ++h)
                         tma_load_5d(sXP + h * kSlabBytes, &map_x, x_full, 64 * h, kTileRows * c.jb, c.inner, c.outer, x_head);
                 }
+                ++it;
             }
             if (!ok) {
                 const unsigned long long t0 = globaltimer_ns();
@@ -233,7 +247,9 @@ hop_tc_bwd_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
         uint32_t t = 0, it = 0;
         bool ok = true;
         int pending_stage = -1;   // thread 0: stage whose output stores have been issued but not yet read out
-        for (long long item = blockIdx.x; ok && item < a.total_items; item += gridDim.x, ++it) {
+        for (long long round = 0; ok && round * gridDim.x < a.total_items; ++round, ++it) {
+            const long long item = item_of_round(a, round);
+            if (item < 0) { --it; continue; }
             const LongBwdItem c = decode_item(a, item);
             const int steps = a.g * c.steps_per_head;
             // key positions of the block that are tokens (none: every weight is 0 and the item writes zeros)
