@@ -44,6 +44,7 @@ struct LongArgs {
     float scale_log2;
     const int *lens;           // device, valid length per batch entry, or nullptr (kWindow variant only)
     int N;
+    int pair_major;            // item numbering, see decode_long_item
     // statistics pass of the backward: instead of the output rows, write per query row
     // (log2-sum-exp of the scaled scores, <G_t, O_t>) -- stats[q_head * N + token]; g = gradient
     // with respect to the hop's output, laid out like q
@@ -77,8 +78,21 @@ struct LongItem {
 // (longer, when causal) pairs first, so that the CTAs of one wave carry similar loads.
 __device__ __forceinline__ LongItem decode_long_item(const LongArgs &a, long long item) {
     LongItem c;
-    long long rest = item;
-    const int pb = a.qpairs - 1 - (int)(rest % a.qpairs); rest /= a.qpairs;
+    // Later (longer, when causal) pairs of query tiles first.  While the K and V of every head
+    // together fit the L2, the pair is the slowest index: the numbering then runs from the longest
+    // items to the shortest over the whole launch (see long_item_of_round), which evens out the
+    // CTAs' loads.  Beyond that the pairs of a segment stay adjacent, so that a wave of CTAs works
+    // on few heads and finds their K / V blocks in L2.
+    int pb;
+    long long rest;
+    if (a.pair_major) {
+        const long long per_pair = a.total_items / a.qpairs;
+        pb = a.qpairs - 1 - (int)(item / per_pair);
+        rest = item % per_pair;
+    } else {
+        pb = a.qpairs - 1 - (int)(item % a.qpairs);
+        rest = item / a.qpairs;
+    }
     c.inner = (int)(rest % a.stride); rest /= a.stride;
     c.outer = (int)(rest % a.outer); rest /= a.outer;
     c.q_head = (int)rest;                                          // b * H + h
@@ -113,6 +127,14 @@ __device__ __forceinline__ LongItem decode_long_item(const LongArgs &a, long lon
     c.jlo = c.j0[0];
     c.jhi = max(c.je[0], c.je[1]);
     return c;
+}
+
+// The item a CTA takes in its k-th round: the rounds run forth and back over the CTAs, so that the
+// CTA that got the longest item of one round gets the shortest of the next.  -1: none in this round.
+__device__ __forceinline__ long long long_item_of_round(const LongArgs &a, long long k) {
+    const long long g = gridDim.x, b = blockIdx.x;
+    const long long item = k * g + ((k & 1) ? g - 1 - b : b);
+    return item < a.total_items ? item : -1;
 }
 
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32]) {
@@ -187,7 +209,9 @@ hop_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 last_par = parity ? (last_par | bit) : (last_par & ~bit);
             };
             bool ok = true;
-            for (long long item = blockIdx.x; ok && item < a.total_items; item += gridDim.x, ++ic) {
+            for (long long round = 0; ok && round * gridDim.x < a.total_items; ++round, ++ic) {
+                const long long item = long_item_of_round(a, round);
+                if (item < 0) { --ic; continue; }
                 const LongItem c = decode_long_item(a, item);
                 const int x_head = a.xin_is_kv ? c.kv_head : c.q_head;
                 ok = mbar_wait_abortable(q_free, (ic & 1) ^ 1, 0xD0, abort_flag);
@@ -235,7 +259,9 @@ hop_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             uint32_t ic = 0, g0 = 0;
             uint32_t p_seen[2] = {0, 0};              // phases of p_full(c) consumed
             bool ok = true;
-            for (long long item = blockIdx.x; ok && item < a.total_items; item += gridDim.x, ++ic) {
+            for (long long round = 0; ok && round * gridDim.x < a.total_items; ++round, ++ic) {
+                const long long item = long_item_of_round(a, round);
+                if (item < 0) { --ic; continue; }
                 const LongItem c = decode_long_item(a, item);
                 ok = mbar_wait_abortable(q_full, ic & 1, 0xE0, abort_flag);
                 if (!ok) break;
@@ -322,7 +348,9 @@ hop_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 
         bool ok = true;
         uint32_t blocks_seen = 0;                       // key blocks this chain has processed (all items)
-        for (long long item = blockIdx.x; ok && item < a.total_items; item += gridDim.x) {
+        for (long long round = 0; ok && round * gridDim.x < a.total_items; ++round) {
+            const long long item = long_item_of_round(a, round);
+            if (item < 0) continue;
             const LongItem c = decode_long_item(a, item);
             if (ch >= c.ntiles) continue;
             const int t = c.t0 + kTileRows * ch + r;    // position of this row in the segment
@@ -543,6 +571,8 @@ int launch_long_d(const Problem &pb, const HopDesc &hd, const void *xin, int xin
     a.scale_log2 = pb.scale * 1.4426950408889634f;
     a.lens = pb.seq_lens;
     a.N = pb.N;
+    // K and V of all heads (bf16) against the 126 MB L2
+    a.pair_major = 2ull * pb.B * pb.H_kv * pb.N * D * 2 <= (96ull << 20) ? 1 : 0;
     a.stats = (float2 *)stats;
     a.stats_g = (const __nv_bfloat16 *)stats_g;
 
