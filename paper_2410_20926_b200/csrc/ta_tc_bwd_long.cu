@@ -39,6 +39,7 @@ struct LongBwdArgs {
     const float2 *stats;               // [B*H][N]: (lse in the log2 domain, delta)
     int window;                        // 0, or sliding window along the hop's dimension
     const int *lens;                   // device, valid length per batch entry, or nullptr
+    int gi, hsplit;                    // query heads per item, items per (key block, KV head): gi * hsplit == g
 };
 
 template <int D>
@@ -73,10 +74,11 @@ __device__ __forceinline__ LongBwdItem decode_item(const LongBwdArgs &a, long lo
     const long long per_block = a.total_items / a.nblocks;
     c.jb = (int)(item / per_block);
     long long rest = item % per_block;
+    const int hs = (int)(rest % a.hsplit); rest /= a.hsplit;       // which of the group's head chunks
     c.inner = (int)(rest % a.stride); rest /= a.stride;
     c.outer = (int)(rest % a.outer); rest /= a.outer;
     c.kv_head = (int)rest;
-    c.q_head0 = (c.kv_head / a.H_kv) * a.H + (c.kv_head % a.H_kv) * a.g;
+    c.q_head0 = (c.kv_head / a.H_kv) * a.H + (c.kv_head % a.H_kv) * a.g + hs * a.gi;
     c.i_lo = a.causal ? c.jb : 0;
     int i_hi = a.nblocks - 1;
     if (a.window > 0) {                // tiles with a row within the window of one of the block's keys
@@ -176,7 +178,7 @@ hop_tc_bwd_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                 const long long item = item_of_round(a, round);
                 if (item < 0) continue;
                 const LongBwdItem c = decode_item(a, item);
-                const int steps = a.g * c.steps_per_head;
+                const int steps = a.gi * c.steps_per_head;
                 for (int v = 0; v < steps; ++v, ++t) {
                     const int q_head = c.q_head0 + v / c.steps_per_head;
                     const int qi = c.i_lo + v % c.steps_per_head;
@@ -251,7 +253,7 @@ hop_tc_bwd_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             const long long item = item_of_round(a, round);
             if (item < 0) { --it; continue; }
             const LongBwdItem c = decode_item(a, item);
-            const int steps = a.g * c.steps_per_head;
+            const int steps = a.gi * c.steps_per_head;
             // key positions of the block that are tokens (none: every weight is 0 and the item writes zeros)
             const int keys = max(0, min(kTileRows, min(a.n, c.exist) - kTileRows * c.jb));
             for (int v = 0; v < steps; ++v, ++t) {
@@ -444,8 +446,12 @@ hop_tc_bwd_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                         wg_sync();
                         if (tid == 0) {
 #pragma unroll
-                            for (int sl = 0; sl < D / 32; ++sl)
-                                tma_store_5d(&map_dv, q_base + sl * kSlabBytes, 32 * sl, kTileRows * c.jb, c.inner, c.outer, c.kv_head);
+                            for (int sl = 0; sl < D / 32; ++sl) {
+                                if (a.hsplit > 1)      // several items share the block: summed in global memory
+                                    tma_reduce_add_5d(&map_dv, q_base + sl * kSlabBytes, 32 * sl, kTileRows * c.jb, c.inner, c.outer, c.kv_head);
+                                else
+                                    tma_store_5d(&map_dv, q_base + sl * kSlabBytes, 32 * sl, kTileRows * c.jb, c.inner, c.outer, c.kv_head);
+                            }
                             tma_store_commit_and_wait_read();
                         }
                     }
@@ -493,19 +499,34 @@ int launch_d(const Problem &pb, const HopDesc &hd, const void *x, int x_heads, c
     a.n = hd.n; a.causal = pb.causal; a.g = pb.H / pb.H_kv; a.H = pb.H; a.H_kv = pb.H_kv;
     a.x_is_kv = x_heads != pb.H ? 1 : 0;
     a.first_hop = first_hop ? 1 : 0;
-    a.accumulate_dk = accumulate ? 1 : 0;
+    a.accumulate_dk = accumulate ? 1 : 0;      // (forced below when the heads of a group are split over items)
     a.N = pb.N;
     a.nblocks = (hd.n + kTileRows - 1) / kTileRows;
     a.stride = hd.stride; a.outer = hd.outer;
-    a.total_items = (long long)pb.B * pb.H_kv * hd.outer * hd.stride * a.nblocks;
+    int dev = 0;
+    const int num_sms = current_device_sms(&dev);
+    // the query heads of a group are split over several items when there are too few items to fill
+    // the GPU; their dK (and dV) are then summed in global memory by reduce-adds into cleared buffers
+    const long long blocks_total = (long long)pb.B * pb.H_kv * hd.outer * hd.stride * a.nblocks;
+    a.hsplit = 1;
+    for (int d = 2; d <= a.g && blocks_total * a.hsplit < 4ll * num_sms; ++d)
+        if (a.g % d == 0) a.hsplit = d;
+    a.gi = a.g / a.hsplit;
+    a.total_items = blocks_total * a.hsplit;
+    const size_t tkv = (size_t)pb.B * pb.H_kv * pb.N * pb.D;
+    if (a.hsplit > 1) {
+        if (!accumulate && cudaMemsetAsync(dk_acc, 0, tkv * sizeof(float), pb.stream) != cudaSuccess)
+            return cuda_fail(cudaPeekAtLastError());
+        if (first_hop && cudaMemsetAsync(dv_acc, 0, tkv * sizeof(float), pb.stream) != cudaSuccess)
+            return cuda_fail(cudaPeekAtLastError());
+    }
     a.scale = pb.scale;
     a.scale_log2 = pb.scale * 1.4426950408889634f;
     a.stats = (const float2 *)stats;
     a.window = pb.window[hd.hop];
     a.lens = pb.seq_lens;
 
-    int dev = 0;
-    const int num_sms = current_device_sms(&dev);
+    if (a.hsplit > 1) a.accumulate_dk = 1;
     constexpr size_t smem = LongBwdCfg<D>::kSmemBytes;
     static PerDeviceOnce configured;
     if (!configured.is_done(dev)) {
