@@ -191,8 +191,9 @@ int ta_forward_ex(const ta_params *p);
  * The sums over the query heads of a group are taken inside one CTA and the sums over hops in
  * launch order (no atomics), so the result is bit-reproducible from run to run.
  * Hops with D in {64,128} run on tensor-core backward kernels: one for n_i <= 128, and for longer
- * segments a block-by-block one (its dQ is summed by reduce-adds whose order is not fixed, so it
- * is reproducible only up to fp32 summation order).  Other head dims up to 256 run on generic
+ * segments a block-by-block one (its dQ -- and, on small problems where a group's heads are split
+ * over CTAs, dK and dV -- are summed by reduce-adds whose order is not fixed, so they are
+ * reproducible only up to fp32 summation order).  Other head dims up to 256 run on generic
  * CUDA-core kernels with fp32 arithmetic.  Hops with n_i > 128 or on the generic kernels need a second G
  * buffer and two floats per query row in the workspace (ta_workspace_bytes accounts for them).
  * D > 256: TA_ERR_UNSUPPORTED.
