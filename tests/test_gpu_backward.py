@@ -257,6 +257,7 @@ def test_backward_fp32_storage(dims, D, causal, B, H, Hkv, kw):
     ([260, 3], 64, True, 1, 4, 2),                # long hop first: its gradient is dV, summed over the group
     ([3, 300, 2], 128, False, 1, 2, 1),           # tensor-core short, long, short
     ([16, 300], 64, True, 4, 8, 4),               # enough key blocks that a group's heads stay in one item
+    ([4096], 64, True, 1, 2, 1),                  # 32 key blocks: the statistics carry over many blocks
 ])
 def test_backward_long_segments_tensor_core(dims, D, causal, B, H, Hkv):
     """Segments longer than 128 (no window, mask, lengths or positional encoding) run their backward
