@@ -1,14 +1,25 @@
 #!/usr/bin/env python
-"""Benchmark of the tensorized-attention forward on B200 (tokens per second at 128k tokens).
+"""Benchmark of tensorized attention on B200 (headline: forward tokens per second at 128k tokens).
 
-One step = one whole forward pass (every hop of Algorithm 1) over one batch of synthetic
-Llama-8B-shaped q, k, v: causal, B=1, H=32, H_kv=8, D=128, N=131072 viewed as 32x64x64, bf16.
-Prints ONE JSON line (rank 0).  `value` is device-timed throughput with inputs resident in
-HBM; `e2e` goes through ta_forward_host with pinned host buffers (copies inside the timed
-region); `roofline` is the hop kernel against the measured HBM bandwidth; `cpu_baseline` is
-the fp64 oracle on a bounded sample of the same workload.
+One step = one whole pass of the hot path (every hop of Algorithm 1) over one batch of synthetic
+Llama-8B-shaped q, k, v.  Default workload: causal forward, B=1, H=32, H_kv=8, D=128, N=131072
+viewed as 32x64x64, bf16.  Prints ONE JSON line (rank 0).  `value` is device-timed throughput
+with inputs resident in HBM; `e2e` starts from pinned host buffers and ends with the result back
+in host memory (copies inside the timed region); `roofline` compares the hop kernels with the
+slower of their FLOP time at the bf16 tensor peak and their byte time at the HBM bandwidth;
+`cpu_baseline` is the fp64 oracle on a bounded sample of the same workload.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config 4]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--config 1..5] [--op forward|backward|fwdbwd] [--repeats R] [--sets S]
+
+* `--config` picks one of the five configurations; `--op backward` times ta_backward on it
+  (recomputing the hop inputs), `--op fwdbwd` a training step (forward that saves the hop inputs,
+  then the backward that uses them).
+* The headline number comes from the first block of exactly K steps; `--repeats R` then runs R
+  more blocks of K steps and reports their median and minimum under `blocks`.
+* Workloads smaller than the L2 are run over `--sets S` rotating sets of buffers (default: as
+  many as it takes to exceed twice the L2, at least 4) so that no step finds its inputs cached;
+  the same workload on ONE set ("hot") is reported under `hot`.
 
 With N > 1 (launched by torch.distributed.run) every rank runs the same workload on its own
 GPU -- heads and batches are independent, so there is no data-path collective (weak scaling);
@@ -33,38 +44,78 @@ if ROOT not in sys.path:
 
 from paper_2410_20926_b200 import inputs as ta_inputs  # noqa: E402
 
-METRIC = "tensorized_attention_forward_tokens_per_s"
 UNIT = "tokens/s"
-FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum per token per launch of the hop kernel, from
-# the ncu capture of config 3 summarised in profiles/hop_pipe_kernel_config3_ncu_full.md
+METRICS = {"forward": "tensorized_attention_forward_tokens_per_s",
+           "backward": "tensorized_attention_backward_tokens_per_s",
+           "fwdbwd": "tensorized_attention_training_step_tokens_per_s"}
+FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS = 6650.0, 1590.0
+NOMINAL_HBM_GBS, NOMINAL_BF16_TFLOPS = 8000.0, 2250.0
+L2_BYTES = 126 * 1024 * 1024
+# dram__bytes_read.sum + dram__bytes_write.sum per token per launch of the forward hop kernel,
+# from the ncu capture of config 3 summarised in profiles/hop_pipe_kernel_config3_ncu_full.md
 # (mean of the three hops, 758.8 MB for 32768 tokens); traffic is proportional to the tokens.
-NCU_TRAFFIC_BYTES_PER_TOKEN_PER_LAUNCH = 757.9e6 / 32768
+NCU_TRAFFIC_BYTES_PER_TOKEN_PER_LAUNCH = 758.8e6 / 32768
 
 
 # ------------------------------------------------------------------ roofline arithmetic
-def hop_bytes(cfg, hop_index: int) -> int:
-    """Algorithmic HBM bytes of one hop: read Q (H heads), K (H_kv), the value tensor in
-    (V with H_kv heads for the first hop, else H heads) and write the value tensor out (H)."""
-    e = 2 if cfg.dtype == "bf16" else 4
-    vin = cfg.H_kv if hop_index == 0 else cfg.H
-    return e * cfg.B * cfg.N * cfg.D * (cfg.H + cfg.H_kv + vin + cfg.H)
+def elem(cfg) -> int:
+    return 2 if cfg.dtype == "bf16" else 4
 
 
 def real_hops(cfg):
     return [i for i, n in enumerate(cfg.dims) if n > 1]
 
 
-def step_bytes(cfg) -> int:
-    return sum(hop_bytes(cfg, j) for j, _ in enumerate(real_hops(cfg)))
+def hop_bytes(cfg, j: int) -> int:
+    """Algorithmic HBM bytes of forward hop j (j-th hop with n > 1): read Q (H heads), K (H_kv),
+    the value tensor in (V with H_kv heads for the first hop, else H heads), write it out (H)."""
+    vin = cfg.H_kv if j == 0 else cfg.H
+    return elem(cfg) * cfg.B * cfg.N * cfg.D * (cfg.H + cfg.H_kv + vin + cfg.H)
 
 
-def step_flops(cfg, causal_useful: bool = True) -> float:
-    f = 0.0
-    for i in real_hops(cfg):
-        n = cfg.dims[i]
-        f += 4.0 * cfg.B * cfg.H * cfg.N * cfg.D * ((n + 1) / 2 if (cfg.causal and causal_useful) else n)
-    return f
+def bwd_hop_bytes(cfg, j: int, nh: int) -> int:
+    """Algorithmic HBM bytes of the backward of hop j, hops processed last to first: read Q (H),
+    K (H_kv), the hop's input X_j (H; V through H_kv heads for j = 0) and the incoming gradient
+    (H); write the outgoing gradient (H; dV with H_kv heads for j = 0); dQ (H) and dK (H_kv)
+    are written by the first hop processed and read-modified-written by the others.  Counted
+    in the storage dtype (accumulators of wider type move more)."""
+    H, K = cfg.H, cfg.H_kv
+    first_processed = j == nh - 1
+    units = H + K + (K if j == 0 else H) + H            # Q, K, X_j, G_in
+    units += K if j == 0 else H                          # G_out / dV
+    units += (H + K) if first_processed else 2 * (H + K)  # dQ, dK
+    return elem(cfg) * cfg.B * cfg.N * cfg.D * units
+
+
+def hop_flops(cfg, i: int, useful: bool) -> float:
+    """Forward flops of the hop over dims[i]: two contractions of 2*n*D flops per query row;
+    `useful` counts the causal half only, otherwise what the 128-row tiles issue (a tile computes
+    every pair of its rows, also across segments)."""
+    n = cfg.dims[i]
+    per_row = (n + 1) / 2 if (useful and cfg.causal) else (n if useful else max(n, 128))
+    return 4.0 * cfg.B * cfg.H * cfg.N * cfg.D * per_row
+
+
+def op_bytes(cfg, op: str):
+    """List of (label, bytes) per launch group of a step."""
+    nh = len(real_hops(cfg))
+    fwd = [(f"fwd hop {j}", hop_bytes(cfg, j)) for j in range(nh)]
+    bwd = [(f"bwd hop {j}", bwd_hop_bytes(cfg, j, nh)) for j in reversed(range(nh))]
+    if op == "forward":
+        return fwd
+    if op == "backward":
+        return fwd[:-1] + bwd          # the hop inputs X_1..X_{m-1} are recomputed by m-1 forward hops
+    return fwd + bwd
+
+
+def op_flops(cfg, op: str, useful: bool) -> float:
+    f = sum(hop_flops(cfg, i, useful) for i in real_hops(cfg))
+    rec = sum(hop_flops(cfg, i, useful) for i in real_hops(cfg)[:-1])
+    if op == "forward":
+        return f
+    if op == "backward":
+        return rec + 2.5 * f           # five contractions per hop against the forward's two
+    return f + 2.5 * f
 
 
 def measured_peaks():
@@ -72,9 +123,45 @@ def measured_peaks():
     try:
         with open(path) as f:
             d = json.load(f)
-        return float(d["hbm_gbs"]), "measured (MEASURED_PEAKS.json)", d
+        return float(d["hbm_gbs"]), float(d["bf16_tflops"]), "measured (MEASURED_PEAKS.json)"
     except Exception:
-        return FALLBACK_HBM_GBS, "fallback (6.65 TB/s)", {}
+        return FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS, "fallback (6.65 TB/s, 1.59 PFLOP/s)"
+
+
+def roofline_block(cfg, op, ms_per_step, n_launches):
+    hbm, tfl, src = measured_peaks()
+    groups = op_bytes(cfg, op)
+    total_bytes = sum(b for _, b in groups)
+    issued = op_flops(cfg, op, useful=False)
+    t_hbm = total_bytes / (hbm * 1e9) * 1e3
+    t_flop = issued / (tfl * 1e12) * 1e3
+    bound = "hbm" if t_hbm >= t_flop else "tensor"
+    n_launch = max(1, len(groups))
+    if bound == "hbm":
+        achieved = total_bytes / (ms_per_step * 1e-3) / 1e9
+        peak, unit = hbm, "GB/s"
+        nominal = achieved / NOMINAL_HBM_GBS
+    else:
+        achieved = issued / (ms_per_step * 1e-3) / 1e12
+        peak, unit = tfl, "TFLOP/s"
+        nominal = achieved / NOMINAL_BF16_TFLOPS
+    fwd_only = op == "forward" and cfg.dtype == "bf16"
+    return {"bound": bound, "achieved": achieved, "peak": peak, "unit": unit, "frac": achieved / peak,
+            "frac_of": "measured peak", "frac_of_nominal_peak": nominal,
+            "nominal_peak": NOMINAL_HBM_GBS if bound == "hbm" else NOMINAL_BF16_TFLOPS,
+            "peak_source": src,
+            "traffic": NCU_TRAFFIC_BYTES_PER_TOKEN_PER_LAUNCH * cfg.B * cfg.N if fwd_only else None,
+            "traffic_source": ("ncu capture of config 3 (dram read + write per launch) scaled by tokens; "
+                               "extrapolated, see profiles/") if fwd_only else None,
+            "kernel": "hop_pipe_kernel<128, false, false>" if fwd_only else
+                      ("hop_tc_bwd_kernel + hop_pipe_kernel" if cfg.dtype == "bf16" else "hop_simt_kernel"),
+            "algorithmic_bytes_per_step": total_bytes,
+            "algorithmic_bytes_per_launch": total_bytes / n_launch,
+            "launch_groups_per_step": n_launch, "kernel_launches_per_step": n_launches,
+            "avg_launch_ms": ms_per_step / n_launch,
+            "t_hbm_ms": t_hbm, "t_flop_issued_ms": t_flop,
+            "useful_tflops": op_flops(cfg, op, useful=True) / (ms_per_step * 1e-3) / 1e12,
+            "issued_tflops": issued / (ms_per_step * 1e-3) / 1e12}
 
 
 # ------------------------------------------------------------------ clocks
@@ -105,7 +192,7 @@ class ClockSampler:
         except Exception:
             self.proc.kill()
             out = ""
-        sm, smax, reasons = [], [], set()
+        sm, smax, power, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for line in out.strip().splitlines():
             parts = [p.strip() for p in line.split(",")]
@@ -114,6 +201,7 @@ class ClockSampler:
             try:
                 sm.append(float(parts[0]))
                 smax.append(float(parts[1]))
+                power.append(float(parts[2]))
             except ValueError:
                 continue
             for name, val in zip(names, parts[3:7]):
@@ -121,31 +209,40 @@ class ClockSampler:
                     reasons.add(name)
         return {"sm_mhz": statistics.median(sm) if sm else None,
                 "sm_max_mhz": max(smax) if smax else None,
+                "power_w_max": max(power) if power else None,
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
 # ------------------------------------------------------------------ CPU oracle timing
-def oracle_sample(cfg, inp, min_seconds: float = 0.0):
-    """Times the fp64 oracle on ONE head of the workload (all N tokens, every hop) and scales
-    to the whole batch: tokens/s = B*N / (t_head * B*H)."""
+def oracle_sample(cfg, inp, op: str, min_seconds: float = 0.0):
+    """Times the fp64 oracle on whole heads (forward) or whole KV groups (backward ops) of the
+    workload, one after the other, until `min_seconds` have passed.  Returns the description and
+    the mean seconds per sampled unit; the workload has B*H heads / B*H_kv groups."""
     import oracle
+    units_total = cfg.B * cfg.H if op == "forward" else cfg.B * cfg.H_kv
     t0 = time.perf_counter()
     reps = 0
     while True:
-        oracle.forward(inp["q"], inp["k"], inp["v"], list(cfg.dims), cfg.causal, heads=[(0, reps % cfg.H)])
+        u = reps % units_total
+        if op == "forward":
+            oracle.forward(inp["q"], inp["k"], inp["v"], list(cfg.dims), cfg.causal, heads=[(u // cfg.H, u % cfg.H)])
+        else:
+            oracle.backward(inp["dout"], inp["q"], inp["k"], inp["v"], list(cfg.dims), cfg.causal,
+                            groups=[(u // cfg.H_kv, u % cfg.H_kv)])
         reps += 1
         dt = time.perf_counter() - t0
         if dt >= min_seconds:
             break
-    t_head = dt / reps
-    value = cfg.B * cfg.N / (t_head * cfg.B * cfg.H)
+    t_unit = dt / reps
+    what = "heads" if op == "forward" else "KV groups (forward and backward of their query heads)"
+    value = cfg.B * cfg.N / (t_unit * units_total)
     return {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
-            "sample": f"{reps} single-head passes over the workload's heads (all {cfg.N} tokens, all hops; "
-                      f"the batch has {cfg.B * cfg.H} heads), {dt:.1f} s, scaled to the batch"}, t_head
+            "sample": f"{reps} of the workload's {units_total} {what}, each over all {cfg.N} tokens and every hop, "
+                      f"{dt:.1f} s in all; value = tokens of the batch / (mean time per sampled unit x {units_total})"}, t_unit
 
 
 # ------------------------------------------------------------------ distributed plumbing
-def dist_setup(n_gpus: int):
+def dist_setup(n_gpus: int = 1):
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
@@ -174,74 +271,156 @@ def max_over_ranks(x: float, world: int, device=None) -> float:
     return float(t.item())
 
 
-def aggregate(tokens_per_rank: int, world: int, ms_max: float, steps: int) -> float:
+def aggregate(tokens_per_rank: int, world: int, ms_total: float, steps: int) -> float:
     """Whole-job tokens/s: every rank processed `tokens_per_rank` tokens per step."""
-    return tokens_per_rank * world * steps / (ms_max * 1e-3)
+    return tokens_per_rank * world * steps / (ms_total * 1e-3)
+
+
+def workload_config(cfg, world, op, sets=1):
+    mode = {"forward": "fwd", "backward": "bwd (hop inputs recomputed)", "fwdbwd": "fwd+bwd training step"}[op]
+    step = sum(b for _, b in op_bytes(cfg, op))
+    cold = ("inputs (%.2f GB per step) exceed the 126 MB L2; no flush needed" % (step / 1e9)) if sets == 1 else \
+           ("%d rotating sets of buffers (%.0f MB each): no step finds its tensors in the 126 MB L2" %
+            (sets, footprint_bytes(cfg, op) / 1e6))
+    return {"workload": f"config {cfg.index}: {'causal' if cfg.causal else 'non-causal'} {mode}, B={cfg.B}, H={cfg.H}, "
+                        f"H_kv={cfg.H_kv}, D={cfg.D}, N={cfg.N} as {'x'.join(map(str, cfg.dims))}, {cfg.dtype}, "
+                        f"q/k/v{'/dout' if op != 'forward' else ''} ~ N(0,1) seeded",
+            "op": op, "B": cfg.B, "H": cfg.H, "H_kv": cfg.H_kv, "D": cfg.D, "N": cfg.N, "dims": list(cfg.dims),
+            "causal": cfg.causal, "per_gpu_batch": cfg.B, "replicas": world, "buffer_sets": sets, "l2": cold}
+
+
+def footprint_bytes(cfg, op) -> int:
+    """Bytes of the distinct tensors one step touches (one buffer set)."""
+    e = elem(cfg)
+    q = cfg.B * cfg.H * cfg.N * cfg.D * e
+    kv = cfg.B * cfg.H_kv * cfg.N * cfg.D * e
+    if op == "forward":
+        return 2 * q + 2 * kv
+    return 4 * q + 4 * kv
 
 
 # ------------------------------------------------------------------ arms
 def run_reference(args, cfg):
-    rank, world, _ = dist_setup(args.gpus)
+    rank, world, _ = dist_setup()
     if rank != 0:
         return
-    inp = ta_inputs.make_config_inputs(cfg)
+    op = args.op
+    inp = ta_inputs.make_inputs(cfg.B, cfg.H, cfg.H_kv, cfg.N, cfg.D, cfg.dtype, cfg.seed, with_dout=op != "forward")
+    units_total = cfg.B * cfg.H if op == "forward" else cfg.B * cfg.H_kv
     for _ in range(min(args.warmup, 1)):
-        oracle_sample(cfg, inp)
+        oracle_sample(cfg, inp, op)
     times = []
     info = None
     for _ in range(args.steps):
-        info, t_head = oracle_sample(cfg, inp)
-        times.append(t_head)
-    t_head = sum(times) / len(times)
-    value = cfg.B * cfg.N / (t_head * cfg.B * cfg.H)
+        info, t_unit = oracle_sample(cfg, inp, op)     # one step = ONE head / KV group of the workload
+        times.append(t_unit)
+    t_unit = sum(times) / len(times)
+    tokens_per_step = cfg.B * cfg.N / units_total        # token-equivalents: the step covers 1/units_total of the batch
+    value = tokens_per_step / t_unit
     info["value"] = value
-    info["sample"] = (f"each step = 1 of {cfg.B * cfg.H} heads of the workload (all {cfg.N} tokens, all hops), "
-                      f"scaled to the batch; {len(times)} steps")
-    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
-            "steps": args.steps, "warmup": args.warmup, "ms_per_step": t_head * cfg.B * cfg.H * 1e3,
+    info["sample"] = (f"each step = 1 of the workload's {units_total} "
+                      f"{'heads' if op == 'forward' else 'KV groups'} (all {cfg.N} tokens, every hop) = "
+                      f"{tokens_per_step:.0f} token-equivalents of the batch; {len(times)} steps")
+    line = {"impl": "reference", "metric": METRICS[op], "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": t_unit * 1e3,
+            "tokens_per_step": tokens_per_step, "sample_fraction_of_workload": 1.0 / units_total,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
-            "data": "synthetic", "config": workload_config(cfg, world),
+            "data": "synthetic", "config": workload_config(cfg, world, op),
             "cpu_baseline": info,
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line), flush=True)
 
 
-def workload_config(cfg, world):
-    return {"workload": f"config {cfg.index}: causal fwd, B={cfg.B}, H={cfg.H}, H_kv={cfg.H_kv}, D={cfg.D}, "
-                        f"N={cfg.N} as {'x'.join(map(str, cfg.dims))}, {cfg.dtype}, q/k/v ~ N(0,1) seeded",
-            "B": cfg.B, "H": cfg.H, "H_kv": cfg.H_kv, "D": cfg.D, "N": cfg.N, "dims": list(cfg.dims),
-            "causal": cfg.causal, "per_gpu_batch": cfg.B, "replicas": world,
-            "l2": "inputs (%.2f GB per step) exceed the 126 MB L2; no flush needed" % (step_bytes(cfg) / 1e9)}
+class BufferSet:
+    """Device tensors of one step; several sets rotate when the workload would fit the L2."""
+
+    def __init__(self, cfg, op, host, dev, ta):
+        import torch
+        self.cfg, self.op = cfg, op
+        tdt = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
+        self.q, self.k, self.v = (host[n].to(dev) for n in ("q", "k", "v"))
+        self.out = torch.empty((cfg.B, cfg.H, cfg.N, cfg.D), dtype=tdt, device=dev)
+        code = ta.TA_DTYPE_BF16 if cfg.dtype == "bf16" else ta.TA_DTYPE_F32
+        self.code = code
+        dims = list(cfg.dims)
+        if op != "forward":
+            self.dout = host["dout"].to(dev)
+            self.dq, self.dk, self.dv = torch.empty_like(self.q), torch.empty_like(self.k), torch.empty_like(self.v)
+            self.grad_code = code
+            mode = ta.TA_WS_BACKWARD if cfg.dtype == "bf16" else ta.TA_WS_BACKWARD_F32_GRADS
+            nb = ta.ta_workspace_bytes(cfg.B, cfg.H, cfg.H_kv, cfg.N, cfg.D, dims, code, mode)
+            self.ws_bytes = nb
+            self.ws = torch.empty(max(nb, 256), dtype=torch.uint8, device=dev)
+        if op == "fwdbwd":
+            ns = ta.ta_workspace_bytes(cfg.B, cfg.H, cfg.H_kv, cfg.N, cfg.D, dims, code, ta.TA_WS_FORWARD_SAVE)
+            self.save_bytes = ns
+            self.save = torch.empty(max(ns, 256), dtype=torch.uint8, device=dev)
+            self.saved_offset = ns - (len(real_hops(cfg)) - 1) * self.out.numel() * self.out.element_size()
 
 
 def run_ours(args, cfg):
     import torch
     import paper_2410_20926_b200 as ta
 
-    rank, world, local = dist_setup(args.gpus)
+    rank, world, local = dist_setup()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     ta.load()
+    op = args.op
+    if args.rope_base > 0 and op != "forward":
+        raise SystemExit("--rope-base is offered for --op forward only")
 
-    inp = ta_inputs.make_config_inputs(cfg)
+    inp = ta_inputs.make_inputs(cfg.B, cfg.H, cfg.H_kv, cfg.N, cfg.D, cfg.dtype, cfg.seed, with_dout=op != "forward")
     host = {}
-    for name in ("q", "k", "v"):
-        t = torch.from_numpy(inp[name + "_bits"].view(np.int16)).view(torch.bfloat16)
+    for name in ("q", "k", "v") + (("dout",) if op != "forward" else ()):
+        if cfg.dtype == "bf16":
+            t = torch.from_numpy(inp[name + "_bits"].view(np.int16)).view(torch.bfloat16)
+        else:
+            t = torch.from_numpy(inp[name])
         host[name] = t.pin_memory()
-    host["out"] = torch.empty((cfg.B, cfg.H, cfg.N, cfg.D), dtype=torch.bfloat16).pin_memory()
-    q, k, v = (host[n].to(dev, non_blocking=True) for n in ("q", "k", "v"))
-    out = torch.empty((cfg.B, cfg.H, cfg.N, cfg.D), dtype=torch.bfloat16, device=dev)
+    tdt = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
+    host["out"] = torch.empty((cfg.B, cfg.H, cfg.N, cfg.D), dtype=tdt).pin_memory()
     dims = list(cfg.dims)
     stream = torch.cuda.current_stream()
 
-    def step():
-        if args.rope_base > 0:
-            ta.ta_forward_ex(q, k, v, out, cfg.B, cfg.H, cfg.H_kv, cfg.N, cfg.D, dims, cfg.causal,
-                             rope_base=args.rope_base, stream=stream)
-        else:
-            ta.ta_forward(q, k, v, out, cfg.B, cfg.H, cfg.H_kv, cfg.N, cfg.D, dims, cfg.causal, stream=stream)
+    fp = footprint_bytes(cfg, op)
+    n_sets = args.sets if args.sets > 0 else (1 if fp >= 2 * L2_BYTES else max(4, -(-2 * L2_BYTES // fp)))
+    sets = [BufferSet(cfg, op, host, dev, ta) for _ in range(n_sets)]
+    counter = [0]
+
+    def step(s=None):
+        if s is None:
+            s = sets[counter[0] % len(sets)]
+            counter[0] += 1
+        c = cfg
+        if op == "forward":
+            if args.rope_base > 0:
+                ta.ta_forward_ex(s.q, s.k, s.v, s.out, c.B, c.H, c.H_kv, c.N, c.D, dims, c.causal, dtype=s.code,
+                                 rope_base=args.rope_base, stream=stream)
+            elif c.dtype == "bf16":
+                ta.ta_forward(s.q, s.k, s.v, s.out, c.B, c.H, c.H_kv, c.N, c.D, dims, c.causal, stream=stream)
+            else:
+                ta.ta_forward_f32(s.q, s.k, s.v, s.out, c.B, c.H, c.H_kv, c.N, c.D, dims, c.causal, stream=stream)
+            return
+        saved = None
+        if op == "fwdbwd":
+            ta.ta_forward_ex(s.q, s.k, s.v, s.out, c.B, c.H, c.H_kv, c.N, c.D, dims, c.causal, dtype=s.code,
+                             flags=ta.TA_FLAG_SAVE_HOPS, workspace=s.save, workspace_bytes=s.save_bytes, stream=stream)
+            saved = s.save.data_ptr() + s.saved_offset
+        ta.ta_backward_ex(s.dout, s.q, s.k, s.v, s.dq, s.dk, s.dv, c.B, c.H, c.H_kv, c.N, c.D, dims, c.causal,
+                          dtype=s.code, grad_dtype=s.grad_code, saved_hops=saved, workspace=s.ws,
+                          workspace_bytes=s.ws_bytes, stream=stream)
+
+    def timed_block(k_steps, which=None):
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record(stream)
+        for _ in range(k_steps):
+            step(which)
+        ev1.record(stream)
+        torch.cuda.synchronize()
+        return ev0.elapsed_time(ev1)
 
     for _ in range(max(args.warmup, 3)):
         step()
@@ -255,72 +434,105 @@ def run_ours(args, cfg):
     barrier(world)
     torch.cuda.synchronize()
     launches0 = ta.ta_launch_count()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    ev0.record(stream)
-    for _ in range(args.steps):
-        step()
-    ev1.record(stream)
-    torch.cuda.synchronize()
-    barrier(world)
+    ms = timed_block(args.steps)                       # the headline: EXACTLY K steps
     launches = ta.ta_launch_count() - launches0
-    ms = max_over_ranks(ev0.elapsed_time(ev1), world, dev)
+    barrier(world)
+    ms = max_over_ranks(ms, world, dev)
+    blocks = [max_over_ranks(timed_block(args.steps), world, dev) / args.steps for _ in range(args.repeats)]
+    hot = None
+    if len(sets) > 1:
+        for _ in range(3):
+            step(sets[0])
+        torch.cuda.synchronize()
+        hot_ms = [max_over_ranks(timed_block(args.steps, sets[0]), world, dev) / args.steps
+                  for _ in range(max(1, args.repeats))]
+        hot = {"ms_per_step_median": statistics.median(hot_ms), "ms_per_step_min": min(hot_ms),
+               "value_median": aggregate(cfg.B * cfg.N, world, statistics.median(hot_ms), 1),
+               "note": "same workload on ONE set of buffers: tensors stay in the L2 between steps"}
     if rank == 0:
         time.sleep(0.2)
     clocks = sampler.stop() if rank == 0 else None
     ta.ta_device_status()
     value = aggregate(cfg.B * cfg.N, world, ms, args.steps)
 
-    # ---- end to end: host buffers in, host buffer out, copies inside the timed region
+    # ---- end to end: host buffers in, host buffers out, copies inside the timed region
     e2e_steps = max(1, min(args.steps, 10))
+    s0 = sets[0]
+    if op == "forward" and args.rope_base == 0:
+        def e2e_step():
+            ta.ta_forward_host(host["q"], host["k"], host["v"], host["out"], cfg.B, cfg.H, cfg.H_kv, cfg.N, cfg.D,
+                               dims, cfg.causal, dtype=s0.code, stream=stream)
+        h2d = sum(host[n].numel() * host[n].element_size() for n in ("q", "k", "v"))
+        d2h = host["out"].numel() * host["out"].element_size()
+        e2e_path = "ta_forward_host (C ABI, host pointers)"
+    else:
+        names = ("q", "k", "v") if op == "forward" else ("q", "k", "v", "dout")
+        if op != "forward":
+            host["dq"] = torch.empty_like(host["q"]).pin_memory()
+            host["dk"] = torch.empty_like(host["k"]).pin_memory()
+            host["dv"] = torch.empty_like(host["v"]).pin_memory()
+
+        def e2e_step():
+            for n in names:
+                getattr(s0, n).copy_(host[n], non_blocking=True)
+            step(s0)
+            if op == "forward":
+                host["out"].copy_(s0.out, non_blocking=True)
+            else:
+                host["dq"].copy_(s0.dq, non_blocking=True)
+                host["dk"].copy_(s0.dk, non_blocking=True)
+                host["dv"].copy_(s0.dv, non_blocking=True)
+        h2d = sum(host[n].numel() * host[n].element_size() for n in names)
+        d2h = (host["out"].numel() * host["out"].element_size() if op == "forward" else
+               sum(host[n].numel() * host[n].element_size() for n in ("dq", "dk", "dv")))
+        e2e_path = "pinned host tensors copied on the call's stream around the C-ABI call"
     for _ in range(2):
-        ta.ta_forward_host(host["q"], host["k"], host["v"], host["out"], cfg.B, cfg.H, cfg.H_kv, cfg.N, cfg.D,
-                           dims, cfg.causal, stream=stream)
+        e2e_step()
     torch.cuda.synchronize()
     barrier(world)
     t0 = time.perf_counter()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
     for _ in range(e2e_steps):
-        ta.ta_forward_host(host["q"], host["k"], host["v"], host["out"], cfg.B, cfg.H, cfg.H_kv, cfg.N, cfg.D,
-                           dims, cfg.causal, stream=stream)
+        e2e_step()
     e1.record(stream)
     torch.cuda.synchronize()
     wall_ms = (time.perf_counter() - t0) * 1e3
     e2e_ms = max_over_ranks(max(e0.elapsed_time(e1), wall_ms), world, dev)
     barrier(world)
     e2e_value = aggregate(cfg.B * cfg.N, world, e2e_ms, e2e_steps)
-    h2d = sum(host[n].numel() * 2 for n in ("q", "k", "v"))
-    d2h = host["out"].numel() * 2
-    # the e2e result must be the same bits as the device-resident run (the host entry point
-    # takes no positional encoding, so there is nothing to compare with --rope-base)
-    same = bool(torch.equal(host["out"], out.cpu())) if args.rope_base == 0 else None
+    same = None
+    if op == "forward" and args.rope_base == 0:
+        step(s0)
+        torch.cuda.synchronize()
+        same = bool(torch.equal(host["out"], s0.out.cpu()))       # same bits as the device-resident run
 
     if rank != 0:
         return
-    # ---- roofline of the hop kernel (all launches of a step are the same kernel)
-    peak, peak_src, _ = measured_peaks()
-    n_launch = len(real_hops(cfg))
-    bytes_per_launch = step_bytes(cfg) / n_launch
-    launch_ms = ms / (args.steps * n_launch)
-    achieved = bytes_per_launch / (launch_ms * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": NCU_TRAFFIC_BYTES_PER_TOKEN_PER_LAUNCH * cfg.B * cfg.N,
-                "traffic_source": "ncu capture of config 3 scaled by tokens (profiles/)", "peak_source": peak_src,
-                "kernel": "hop_pipe_kernel<128, false, false>", "algorithmic_bytes_per_launch": bytes_per_launch,
-                "launches_per_step": n_launch, "avg_launch_ms": launch_ms,
-                "useful_tflops": step_flops(cfg) / (ms / args.steps * 1e-3) / 1e12}
-    cpu, _ = oracle_sample(cfg, inp, min_seconds=args.cpu_seconds)
+    ms_per_step = ms / args.steps
+    roofline = roofline_block(cfg, op, ms_per_step, launches / args.steps)
+    if args.rope_base > 0:
+        roofline["kernel"] = "hop_pipe_kernel<128, true, false>"
+        roofline["traffic"] = None
+    cpu, _ = oracle_sample(cfg, inp, op, min_seconds=args.cpu_seconds)
 
-    cfg_desc = workload_config(cfg, world)
+    cfg_desc = workload_config(cfg, world, op, len(sets))
     if args.rope_base > 0:
         cfg_desc["workload"] += f", tensorized positional encoding fused (RoPE base {args.rope_base:g})"
         cfg_desc["rope_base"] = args.rope_base
-    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": cfg_desc, "clocks": clocks,
+    line = {"metric": METRICS[op], "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": cfg.dtype if cfg.dtype == "bf16" else "f32",
+            "data": "synthetic", "config": cfg_desc, "clocks": clocks,
+            "blocks": {"count": len(blocks), "steps_each": args.steps,
+                       "ms_per_step_median": statistics.median(blocks) if blocks else None,
+                       "ms_per_step_min": min(blocks) if blocks else None,
+                       "ms_per_step_all": blocks,
+                       "note": "further blocks of K steps after the headline block"},
+            "hot": hot,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                    "ms_per_step": e2e_ms / e2e_steps, "steps": e2e_steps, "matches_device_run": same},
+                    "ms_per_step": e2e_ms / e2e_steps, "steps": e2e_steps, "matches_device_run": same,
+                    "path": e2e_path},
             "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu}
     print(json.dumps(line), flush=True)
 
@@ -332,10 +544,13 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=4, help="workload: index into the five configurations")
+    ap.add_argument("--op", default="forward", choices=["forward", "backward", "fwdbwd"])
+    ap.add_argument("--repeats", type=int, default=5, help="further timed blocks of K steps (median / min reported)")
+    ap.add_argument("--sets", type=int, default=0, help="rotating buffer sets (0: enough to exceed twice the L2)")
     ap.add_argument("--cpu-seconds", type=float, default=10.0, help="CPU time budget of the oracle sample")
     ap.add_argument("--rope-base", type=float, default=0.0,
                     help="> 0: time the forward with the fused tensorized positional encoding (not the "
-                         "headline workload; device-timed value only)")
+                         "headline workload)")
     args = ap.parse_args()
     cfg = ta_inputs.CONFIGS[args.config]
     if args.impl == "reference":

@@ -21,7 +21,8 @@
  *   - Layout: q, out, dout, dq: [B][H][N][D];  k, v, dk, dv: [B][H_kv][N][D];
  *     contiguous, D innermost, token order = row-major order of the n_1 x ... x n_m tensor.
  *     Base pointers must be 16-byte aligned.
- *   - All buffers are owned by the caller.  `out` must not overlap q, k or v.
+ *   - All buffers are owned by the caller.  `out` must not overlap q, k or v (checked:
+ *     TA_ERR_INVALID_ARG).
  *   - Calls only enqueue work on `stream` (they do not synchronise) unless stated.
  *   - Return value: TA_OK (0) or a negative TA_ERR_* code; nothing is thrown, printed or
  *     aborted.  On an error return no kernel has been launched by that call.
@@ -29,9 +30,12 @@
  *   - Kernels are built for sm_100a only; on another device the calls return TA_ERR_ARCH.
  *   - Host threads: the calls may be made from several threads at once, on the same or on
  *     different streams and devices (the calling thread's current device is used).  Two calls
- *     whose kernels can overlap on the GPU must not share memory they write; that includes the
- *     library-owned scratch tensor used when `workspace` is NULL and a problem mixes kernels
- *     (ta_workspace_bytes(.., TA_WS_FORWARD) != 0): give such concurrent calls a workspace each.
+ *     whose kernels can overlap on the GPU must not share memory they write (outputs, caller
+ *     workspaces).  Scratch the library takes by itself when `workspace` is NULL is a
+ *     stream-ordered allocation (cudaMallocFromPoolAsync on the call's stream, from a memory pool
+ *     the library creates per device, returned with cudaFreeAsync behind the call's last kernel):
+ *     it is private to the call, involves no device-wide synchronisation and may be captured in
+ *     a CUDA graph.  ta_forward_static is the exception (one fixed array, see there).
  */
 #ifndef TA_B200_H
 #define TA_B200_H
@@ -70,12 +74,25 @@ enum {
 enum {
     TA_FLAG_NO_TENSOR_CORE = 1u << 0, /* run every hop on the generic CUDA-core kernel        */
     TA_FLAG_NO_HOP_FUSION = 1u << 1,  /* one launch per hop: trailing hops that together fit one  */
-                                      /* 128-row tile are not fused into one pass               */
+                                      /* 128-row tile are not fused into one pass (and            */
+                                      /* TA_FLAG_PAIR_HOPS is ignored)                            */
     TA_FLAG_SAVE_HOPS = 1u << 2,      /* store hop inputs X_1..X_{m-1} in the workspace (for ta_backward) */
-    TA_FLAG_NO_HOP_OVERLAP = 1u << 3  /* launch every hop fully serialised.  By default a hop's kernel  */
+    TA_FLAG_NO_HOP_OVERLAP = 1u << 3, /* launch every hop fully serialised.  By default a hop's kernel  */
                                       /* may start on SMs the previous hop has left and prefetch its   */
                                       /* first Q / K tiles (programmatic dependent launch); it waits    */
                                       /* for that hop before touching the value tensor.  Same results.  */
+    TA_FLAG_BF16_INTERMEDIATES = 1u << 5, /* store the value tensor between hops as bf16.  By default,  */
+                                      /* between two tensor-core hops (n_i <= 128) of one call it is    */
+                                      /* stored in `out` as fp16 -- same bytes, three more mantissa     */
+                                      /* bits -- and only the last hop rounds to bf16.  Implied by      */
+                                      /* TA_FLAG_SAVE_HOPS (the backward reads the hop inputs as bf16). */
+    TA_FLAG_PAIR_HOPS = 1u << 4       /* run two adjacent tensor-core hops whose common block is too    */
+                                      /* large for one SM as ONE launch in which the second hop's tiles */
+                                      /* follow the first hop's tiles of the same block closely enough  */
+                                      /* to find them in the L2 cache (see ta_forward).  Same results,  */
+                                      /* bit for bit; half the HBM traffic of the two hops.  Off by     */
+                                      /* default: on B200 the launch is bound by the SM-side pipeline,  */
+                                      /* not by HBM, and measured 10-20 % slower than hop by hop.       */
 };
 
 /* modes of ta_workspace_bytes */
@@ -83,8 +100,9 @@ enum { TA_WS_FORWARD = 0, TA_WS_FORWARD_SAVE = 1, TA_WS_BACKWARD = 2, TA_WS_BACK
 
 /*
  * Forward pass, bf16 storage (Algorithm 1; fp32 accumulation and fp32 softmax; the
- * attention weights are rounded to bf16 before the value product, and the value tensor
- * carried between hops is stored as bf16 in `out`).
+ * attention weights are rounded to 16 bits before the value product, and the value tensor
+ * carried between hops is stored in `out` in 16 bits: as fp16 between two tensor-core hops,
+ * whose weights are then fp16 too, else as bf16; the result is bf16).
  *   q [B,H,N,D], k, v [B,H_kv,N,D]: device, bf16, read only.
  *   out [B,H,N,D]: device, bf16, written (used as the in-place value tensor between hops).
  *   dims: host array of ndims positive ints, prod == N.  causal: 0 or 1.
@@ -92,10 +110,15 @@ enum { TA_WS_FORWARD = 0, TA_WS_FORWARD_SAVE = 1, TA_WS_BACKWARD = 2, TA_WS_BACK
  * Hops with D in {64,128} and n_i <= 128 run on the tensor-core kernel in place in `out` and
  * need no other memory.  Hops with n_i > 128 (key-block loop with online softmax on the tensor
  * cores, D in {64,128}) and hops with another D (generic CUDA-core kernel) cannot update in
- * place: for them the library uses an internal device scratch buffer of
- * B*H*N*D elements that it allocates on first need and keeps (cudaMalloc: synchronous, so
- * such a first call must not happen during stream capture).  ta_forward_ex takes a caller
+ * place: for them the library takes a scratch buffer of B*H*N*D elements from its memory pool
+ * for the duration of the call (stream-ordered, see above).  ta_forward_ex takes a caller
  * workspace instead.
+ * With TA_FLAG_PAIR_HOPS (ta_forward_ex), two adjacent hops with D in {64,128} and n_i <= 128
+ * whose common block (n_i * n_{i+1} * s_{i+1} tokens) is too large for one SM but small against
+ * the L2 cache run as ONE cooperative launch in which the second hop's tiles follow the first
+ * hop's tiles of the same block closely enough to find them in L2 (same arithmetic, same result
+ * bit for bit as hop-by-hop launches).  That launch needs a few KB of completion counters, taken
+ * from the pool or from the workspace (ta_workspace_bytes accounts for them).
  */
 int ta_forward(const void *q, const void *k, const void *v, void *out,
                int B, int H, int H_kv, int N, int D,
@@ -148,7 +171,7 @@ typedef struct ta_params {
  * exists in global memory.  D must be even (else TA_ERR_UNSUPPORTED); a negative or NaN base
  * is TA_ERR_INVALID_ARG.  The value tensor is never rotated.
  * (Hops with n_i > 128 instead run on rotated copies of q and k, written once per hop into a
- * buffer owned by the library and shared by all calls: two such calls must not overlap on the GPU.)
+ * buffer the library takes from its memory pool for the duration of the hop.)
  * ta_backward_ex takes the same rope_base (ta_backward, the short form, does not).
  *
  * Per-hop sparsity mask (Eq. 3 allows any mask M_i): window[i] = w > 0 keeps, in hop i, only
@@ -273,7 +296,9 @@ int ta_forward_host(const void *q_host, const void *k_host, const void *v_host, 
  *     TA_ERR_TOO_LARGE before anything is launched.  Problems that need no second buffer
  *     (bf16, D in {64,128}, every n_i <= 128) have no size limit here.
  *   - The first call on each device looks up the array's device address (with that device
- *     current); make that first call before any stream capture begins.
+ *     current), which also makes the driver load the module and back the array with memory:
+ *     "allocates nothing" holds from the second call on a device.  Make that first call during
+ *     start-up, outside latency-critical sections and before any stream capture begins.
  *   - All calls on a device share the one array and it keeps the previous call's contents.
  *     Nothing has to be cleared (each call overwrites every row it later reads), but calls
  *     whose kernels can overlap on the GPU -- different streams or host threads -- race:
@@ -298,10 +323,25 @@ int ta_plan_describe(int B, int H, int H_kv, int N, int D, const int *dims, int 
  * the device; clears the word.  Returns TA_OK, TA_ERR_TIMEOUT or TA_ERR_CUDA. */
 int ta_device_status(void);
 
+/*
+ * Self-test of the time-out path.  (The paper has no counterpart.)  Every wait inside the
+ * tensor-core kernels is bounded; when one expires the kernel records an error word, ends all
+ * its roles, lets its copies in flight land and returns, and ta_device_status reports
+ * TA_ERR_TIMEOUT.  This call runs that sequence deliberately in a one-CTA kernel: one role
+ * starts a bulk copy and then waits, with a limit of `limit_us` microseconds (1 .. 1 000 000),
+ * on a barrier nobody arrives at; a second role waits with the ordinary limit and must leave
+ * through the abort flag.  Nothing faults and the context stays usable.  Synchronises `stream`.
+ * report (host, 4 words, or NULL): [0] 1 = the short wait expired, [1] 1 = the second role left
+ * through the abort flag, [2] 1 = the copy in flight was seen to land, [3] nanoseconds spent in
+ * the expired wait.  After the call ta_device_status() returns TA_ERR_TIMEOUT once.
+ */
+int ta_selftest_wait_timeout(unsigned limit_us, unsigned *report, ta_stream_t stream);
+
 /* Number of kernels this library has launched in the calling process (all streams). */
 unsigned long long ta_launch_count(void);
 
-/* Frees device memory the library holds (staging and scratch arenas).  Synchronises. */
+/* Frees device memory the library holds (the staging memory of ta_forward_host; cached blocks
+ * of its memory pools go back to the driver).  Synchronises the device. */
 int ta_release(void);
 
 /* The CUDA runtime error code (cudaError_t as int) behind the last TA_ERR_CUDA that

@@ -19,12 +19,14 @@ TA_ERR_INVALID_ARG, TA_ERR_SHAPE, TA_ERR_UNSUPPORTED, TA_ERR_ALIGNMENT = -1, -2,
 TA_ERR_WORKSPACE, TA_ERR_ARCH, TA_ERR_CUDA, TA_ERR_TIMEOUT, TA_ERR_TOO_LARGE = -5, -6, -7, -8, -9
 TA_DTYPE_BF16, TA_DTYPE_F32 = 0, 1
 TA_FLAG_NO_TENSOR_CORE, TA_FLAG_NO_HOP_FUSION, TA_FLAG_SAVE_HOPS, TA_FLAG_NO_HOP_OVERLAP = 1, 2, 4, 8
+TA_FLAG_PAIR_HOPS = 16
+TA_FLAG_BF16_INTERMEDIATES = 32
 TA_WS_FORWARD, TA_WS_FORWARD_SAVE, TA_WS_BACKWARD, TA_WS_BACKWARD_F32_GRADS = 0, 1, 2, 3
 
 EXPORTS = ("ta_forward", "ta_forward_f32", "ta_forward_ex", "ta_backward", "ta_workspace_bytes",
            "ta_forward_host", "ta_plan_describe", "ta_device_status", "ta_launch_count",
            "ta_release", "ta_status_string", "ta_version", "ta_forward_static", "ta_backward_ex",
-           "ta_last_cuda_error")
+           "ta_last_cuda_error", "ta_selftest_wait_timeout")
 TA_STATIC_SCRATCH_BYTES = 16 << 20
 
 
@@ -101,6 +103,7 @@ def load():
     lib.ta_plan_describe.argtypes = [ci, ci, ci, ci, ci, ip, ci, ci, ci, ctypes.c_uint,
                                      ctypes.c_char_p, ctypes.c_size_t]
     lib.ta_device_status.argtypes = []
+    lib.ta_selftest_wait_timeout.argtypes = [ctypes.c_uint, ctypes.POINTER(ctypes.c_uint), vp]
     lib.ta_launch_count.argtypes = []
     lib.ta_launch_count.restype = ctypes.c_ulonglong
     lib.ta_release.argtypes = []
@@ -166,6 +169,14 @@ def ta_launch_count() -> int:
 
 def ta_device_status(check: bool = True) -> int:
     return _done(load().ta_device_status(), "ta_device_status", check)
+
+
+def ta_selftest_wait_timeout(limit_us: int, stream=None, check: bool = True):
+    """Returns (status, [expired, left_through_abort_flag, copy_landed, waited_ns])."""
+    report = (ctypes.c_uint * 4)()
+    rc = _done(load().ta_selftest_wait_timeout(int(limit_us), report, _stream(stream)),
+               "ta_selftest_wait_timeout", check)
+    return rc, list(report)
 
 
 def ta_release() -> int:

@@ -29,6 +29,9 @@ int validate_shape(int B, int H, int H_kv, int N, int D, const int *dims, int nd
     return TA_OK;
 }
 
+// A pair launch pays only while what is touched between the two hops of a unit stays in L2.
+constexpr double kPairWindowLimitBytes = 160.0 * 1024 * 1024;
+
 static bool tc_eligible(int D, int dtype, unsigned flags) {
     return dtype == TA_DTYPE_BF16 && (D == 64 || D == 128) && !(flags & TA_FLAG_NO_TENSOR_CORE);
 }
@@ -53,7 +56,8 @@ int build_plan(int B, int H, int H_kv, int N, int D, const int *dims, int ndims,
                unsigned flags, int hop_begin, int hop_end, Plan *plan) {
     int rc = validate_shape(B, H, H_kv, N, D, dims, ndims, dtype);
     if (rc != TA_OK) return rc;
-    if (flags & ~(unsigned)(TA_FLAG_NO_TENSOR_CORE | TA_FLAG_NO_HOP_FUSION | TA_FLAG_SAVE_HOPS | TA_FLAG_NO_HOP_OVERLAP))
+    if (flags & ~(unsigned)(TA_FLAG_NO_TENSOR_CORE | TA_FLAG_NO_HOP_FUSION | TA_FLAG_SAVE_HOPS | TA_FLAG_NO_HOP_OVERLAP |
+                            TA_FLAG_PAIR_HOPS | TA_FLAG_BF16_INTERMEDIATES | kPlanAllowPairs))
         return TA_ERR_UNSUPPORTED;
     if (hop_begin == 0 && hop_end == 0) hop_end = ndims;
     if (hop_begin < 0 || hop_end > ndims || hop_begin > hop_end) return TA_ERR_INVALID_ARG;
@@ -103,7 +107,7 @@ int build_plan(int B, int H, int H_kv, int N, int D, const int *dims, int ndims,
             // fused pass is bound by its softmax / epilogue chain instead and only pays when the
             // problem is so small that the launches themselves dominate.
             const long long tiles = (long long)B * H * f.tiles_inner * f.tiles_outer;
-            if (D == 128 || tiles <= 2 * 148) {
+            if (D == 128 || tiles <= 2ll * current_device_sms(nullptr)) {
                 plan->hops[first] = f;
                 plan->nhops = first + 1;
             }
@@ -120,6 +124,13 @@ int build_plan(int B, int H, int H_kv, int N, int D, const int *dims, int ndims,
             plan->hops[j].dst = j == nh - 1 ? BUF_OUT : 3 + j;
         }
         plan->save_bytes = (size_t)(nh - 1) * tensor_bytes;
+        if (plan->hops[0].src == plan->hops[0].dst && plan->hops[0].path != PATH_TC) {
+            // one hop with hop_begin > 0 on a kernel that cannot update in place: the caller's
+            // `out` is first copied to scratch
+            plan->hops[0].src = BUF_SCRATCH;
+            plan->need_scratch = true;
+            plan->scratch_bytes = tensor_bytes;
+        }
         return TA_OK;
     }
     // The tensor-core kernel updates in place; the generic kernel needs src != dst.  Assign
@@ -142,6 +153,35 @@ int build_plan(int B, int H, int H_kv, int N, int D, const int *dims, int ndims,
     for (int j = 0; j < nh; ++j)
         if (plan->hops[j].src == BUF_SCRATCH || plan->hops[j].dst == BUF_SCRATCH) plan->need_scratch = true;
     if (plan->need_scratch) plan->scratch_bytes = tensor_bytes;
+    // The value tensor between two tensor-core hops (the second may be a fused pass) is stored as fp16.
+    if (!(flags & TA_FLAG_BF16_INTERMEDIATES)) {
+        for (int j = 0; j + 1 < nh; ++j) {
+            HopDesc &ha = plan->hops[j], &hb = plan->hops[j + 1];
+            if (ha.path == PATH_TC && hb.path == PATH_TC && ha.nf <= 1 && ha.dst == hb.src) {
+                ha.out_f16 = 1;
+                hb.in_f16 = 1;
+            }
+        }
+    }
+    // Pairs of adjacent tensor-core hops whose common block exceeds one SM's shared memory: one
+    // L2-ordered launch per pair (ta_tc_pair.cu), chosen from the last hop backwards (the later
+    // hops move the most bytes: value tensor in and out with all H heads).
+    if ((flags & (kPlanAllowPairs | TA_FLAG_PAIR_HOPS)) && !(flags & (TA_FLAG_NO_HOP_FUSION | TA_FLAG_SAVE_HOPS))) {
+        const int sms = current_device_sms(nullptr);
+        for (int j = nh - 2; j >= 0; --j) {
+            HopDesc &ha = plan->hops[j];
+            const HopDesc &hb = plan->hops[j + 1];
+            PairGeometry geo;
+            if (hb.pair || hb.src != BUF_OUT || hb.dst != BUF_OUT || ha.dst != BUF_OUT ||
+                (ha.src != BUF_OUT && ha.src != BUF_V))
+                continue;
+            if (!pair_geometry(B, H, H_kv, ha, hb, sms, &geo)) continue;
+            if (geo.window_bytes > kPairWindowLimitBytes) continue;
+            ha.pair = 1;
+            if (geo.flag_bytes > plan->flag_bytes) plan->flag_bytes = (geo.flag_bytes + 255) & ~(size_t)255;
+            --j;   // the hop before a pair's first hop may not be the second hop of another pair
+        }
+    }
     return TA_OK;
 }
 
@@ -195,8 +235,53 @@ int take_masks(Problem *pb, const Plan &plan, const int *window, const unsigned 
 }
 
 // ---------------------------------------------------------------------------------------
-// Device scratch / staging arenas owned by the library (grow-only, one per process).
+// Device memory the library takes by itself.
+//  * Scratch of a call that was given no workspace (second value buffer, rotated Q / K copies,
+//    completion counters): stream-ordered allocations from a memory pool the library creates per
+//    device.  An allocation belongs to one call on one stream and goes back in stream order, so
+//    calls on different streams or host threads never share it, nothing is freed while a kernel
+//    may still use it, and there is no device-wide synchronisation.
+//  * Staging memory of ta_forward_host: one grow-only arena (calls are serialised by a lock).
 // ---------------------------------------------------------------------------------------
+static std::mutex g_pool_mutex;
+static cudaMemPool_t g_pools[64] = {};
+
+int pool_alloc(size_t bytes, cudaStream_t stream, void **ptr) {
+    *ptr = nullptr;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (dev < 0 || dev >= 64) return TA_ERR_TOO_LARGE;
+    cudaMemPool_t pool;
+    {
+        std::lock_guard<std::mutex> lock(g_pool_mutex);
+        if (!g_pools[dev]) {
+            cudaMemPoolProps props = {};
+            props.allocType = cudaMemAllocationTypePinned;
+            props.handleTypes = cudaMemHandleTypeNone;
+            props.location.type = cudaMemLocationTypeDevice;
+            props.location.id = dev;
+            if ((e = cudaMemPoolCreate(&g_pools[dev], &props)) != cudaSuccess) {
+                g_pools[dev] = nullptr;
+                return cuda_fail(e);
+            }
+            // keep freed memory in the pool (the next call takes it back without a driver round trip)
+            unsigned long long keep = ~0ull;
+            cudaMemPoolSetAttribute(g_pools[dev], cudaMemPoolAttrReleaseThreshold, &keep);
+        }
+        pool = g_pools[dev];
+    }
+    if ((e = cudaMallocFromPoolAsync(ptr, bytes ? bytes : 256, pool, stream)) != cudaSuccess) {
+        *ptr = nullptr;
+        return cuda_fail(e);
+    }
+    return TA_OK;
+}
+
+void pool_free(void *ptr, cudaStream_t stream) {
+    if (ptr) cudaFreeAsync(ptr, stream);
+}
+
 struct Arena {
     void *ptr = nullptr;
     size_t bytes = 0;
@@ -227,7 +312,7 @@ struct Arena {
     }
 };
 static std::mutex g_arena_mutex;
-static Arena g_scratch, g_staging, g_rotated;
+static Arena g_staging;
 
 // Copy engine of ta_forward_host: uploads and downloads run on two streams of their own and
 // the staging memory has two sets, so that the upload of one call overlaps the kernels and the
@@ -279,35 +364,32 @@ struct HostPipe {
         device = -1;
     }
 };
-// Rotated copies of Q and K for a long-segment hop with the positional encoding (ta_tc_long.cu):
-// library-owned, grown on demand, shared by all calls.
-int rotated_arena(size_t bytes, void **ptr) {
-    std::lock_guard<std::mutex> lock(g_arena_mutex);
-    const int rc = g_rotated.reserve(bytes);
-    if (rc != TA_OK) return rc;
-    *ptr = g_rotated.ptr;
-    return TA_OK;
-}
-
 static HostPipe g_host_pipe;
 static std::mutex g_host_mutex;   // ta_forward_host calls, one at a time; taken before g_arena_mutex
 
 static int check_arch() {
-    static std::atomic<int> cached{1};  // 1 = unknown
-    int c = cached.load();
-    if (c != 1) return c;
+    static std::atomic<int> cached[64];   // 0 = unknown, 1 = compute capability 10.x, 2 = another
     int dev = 0, major = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) {
+    if (cudaGetDevice(&dev) != cudaSuccess) {
         cudaGetLastError();
         return TA_ERR_CUDA;
     }
-    c = major == 10 ? TA_OK : TA_ERR_ARCH;
-    cached.store(c);
-    return c;
+    const bool slot = dev >= 0 && dev < 64;
+    const int c = slot ? cached[dev].load(std::memory_order_relaxed) : 0;
+    if (c != 0) return c == 1 ? TA_OK : TA_ERR_ARCH;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) {
+        cudaGetLastError();
+        return TA_ERR_CUDA;
+    }
+    if (slot) cached[dev].store(major == 10 ? 1 : 2, std::memory_order_relaxed);
+    return major == 10 ? TA_OK : TA_ERR_ARCH;
 }
 
 static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+static bool overlaps(const void *a, size_t a_bytes, const void *b, size_t b_bytes) {
+    const uintptr_t a0 = reinterpret_cast<uintptr_t>(a), b0 = reinterpret_cast<uintptr_t>(b);
+    return a0 < b0 + b_bytes && b0 < a0 + a_bytes;
+}
 
 static int forward_impl(const ta_params &p) {
     if (!p.q || !p.k || !p.v || !p.out) return TA_ERR_INVALID_ARG;
@@ -329,9 +411,14 @@ static int forward_impl(const ta_params &p) {
     if (rc != TA_OK) return rc;
     if (!aligned16(p.q) || !aligned16(p.k) || !aligned16(p.v) || !aligned16(p.out)) return TA_ERR_ALIGNMENT;
     if (p.workspace && (reinterpret_cast<uintptr_t>(p.workspace) & 255u)) return TA_ERR_ALIGNMENT;
-    const size_t need = plan.scratch_bytes + plan.save_bytes;
+    const size_t tensor_bytes = (size_t)p.B * p.H * p.N * p.D * elem_bytes(p.dtype);
+    const size_t kv_bytes = tensor_bytes / p.H * p.H_kv;
+    const size_t need = plan.scratch_bytes + plan.save_bytes + plan.flag_bytes;
     if ((p.flags & TA_FLAG_SAVE_HOPS) && plan.save_bytes && !p.workspace) return TA_ERR_WORKSPACE;
     if (p.workspace && p.workspace_bytes < need) return TA_ERR_WORKSPACE;
+    if (overlaps(p.out, tensor_bytes, p.q, tensor_bytes) || overlaps(p.out, tensor_bytes, p.k, kv_bytes) ||
+        overlaps(p.out, tensor_bytes, p.v, kv_bytes))
+        return TA_ERR_INVALID_ARG;
     rc = check_arch();
     if (rc != TA_OK) return rc;
 
@@ -348,41 +435,48 @@ static int forward_impl(const ta_params &p) {
     pb.flags = p.flags; pb.hop_begin = p.hop_begin; pb.hop_end = p.hop_end;
     pb.stream = (cudaStream_t)p.stream;
 
-    char *ws = (char *)p.workspace;
-    if (!ws && plan.need_scratch) {
-        std::lock_guard<std::mutex> lock(g_arena_mutex);
-        rc = g_scratch.reserve(plan.scratch_bytes);
-        if (rc != TA_OK) return rc;
-        ws = (char *)g_scratch.ptr;
+    if (plan.nhops == 0) {
+        if (p.hop_begin > 0) return TA_OK;  // value tensor already in `out`
+        return launch_broadcast_kv(pb);
     }
-    const size_t tensor_bytes = (size_t)p.B * p.H * p.N * p.D * elem_bytes(p.dtype);
+    // scratch of this call: the caller's workspace, else a stream-ordered allocation handed back
+    // (in stream order) when the last hop has been enqueued
+    char *ws = (char *)p.workspace;
+    void *pooled = nullptr;
+    if (!ws && need) {
+        if ((rc = pool_alloc(need, pb.stream, &pooled)) != TA_OK) return rc;
+        ws = (char *)pooled;
+    }
     auto buffer = [&](int id) -> void * {
         if (id == BUF_V) return const_cast<void *>(p.v);
         if (id == BUF_OUT) return p.out;
         if (id == BUF_SCRATCH) return ws;
         return ws + plan.scratch_bytes + (size_t)(id - 3) * tensor_bytes;
     };
+    void *flags = ws ? ws + plan.scratch_bytes + plan.save_bytes : nullptr;
 
-    if (plan.nhops == 0) {
-        if (p.hop_begin > 0) return TA_OK;  // value tensor already in `out`
-        return launch_broadcast_kv(pb);
-    }
+    rc = TA_OK;
     if (p.hop_begin > 0 && plan.hops[0].src == BUF_SCRATCH) {
-        if (cudaMemcpyAsync(ws, p.out, tensor_bytes, cudaMemcpyDeviceToDevice, pb.stream) != cudaSuccess)
-            return TA_ERR_CUDA;
+        const cudaError_t e = cudaMemcpyAsync(ws, p.out, tensor_bytes, cudaMemcpyDeviceToDevice, pb.stream);
+        if (e != cudaSuccess) rc = cuda_fail(e);
     }
-    for (int j = 0; j < plan.nhops; ++j) {
+    for (int j = 0; rc == TA_OK && j < plan.nhops; ++j) {
         const HopDesc &h = plan.hops[j];
         const void *xin = buffer(h.src);
         const int xin_heads = h.src == BUF_V ? p.H_kv : p.H;
         void *xout = buffer(h.dst);
         pb.pdl = (j > 0 && !(p.flags & TA_FLAG_NO_HOP_OVERLAP)) ? 1 : 0;   // follows a hop kernel of this call
+        if (h.pair) {
+            rc = launch_hop_tc_pair(pb, h, plan.hops[j + 1], xin, xin_heads, xout, flags);
+            ++j;
+            continue;
+        }
         rc = h.path == PATH_TC        ? launch_hop_tc(pb, h, xin, xin_heads, xout)
              : h.path == PATH_TC_LONG ? launch_hop_tc_long(pb, h, xin, xin_heads, xout)
                                       : launch_hop_simt(pb, h, xin, xin_heads, xout);
-        if (rc != TA_OK) return rc;
     }
-    return TA_OK;
+    pool_free(pooled, pb.stream);
+    return rc;
 }
 
 }  // namespace ta
@@ -432,12 +526,12 @@ int ta_forward_f32(const void *q, const void *k, const void *v, void *out, int B
 size_t ta_workspace_bytes(int B, int H, int H_kv, int N, int D, const int *dims, int ndims, int dtype,
                           int mode) {
     Plan plan;
-    unsigned flags = mode == TA_WS_FORWARD_SAVE ? TA_FLAG_SAVE_HOPS : 0u;
+    unsigned flags = (mode == TA_WS_FORWARD_SAVE ? TA_FLAG_SAVE_HOPS : 0u) | kPlanAllowPairs;
     if (build_plan(B, H, H_kv, N, D, dims, ndims, dtype, flags, 0, 0, &plan) != TA_OK) return 0;
     if (mode == TA_WS_BACKWARD) return backward_workspace_bytes(B, H, H_kv, N, D, dims, ndims, dtype, TA_DTYPE_BF16, false);
     if (mode == TA_WS_BACKWARD_F32_GRADS)
         return backward_workspace_bytes(B, H, H_kv, N, D, dims, ndims, dtype, TA_DTYPE_F32, false);
-    return plan.scratch_bytes + plan.save_bytes;
+    return plan.scratch_bytes + plan.save_bytes + plan.flag_bytes;
 }
 
 int ta_forward_host(const void *qh, const void *kh, const void *vh, void *outh, int B, int H, int H_kv, int N,
@@ -538,6 +632,7 @@ int ta_plan_describe(int B, int H, int H_kv, int N, int D, const int *dims, int 
     if (!buf || cap == 0) return TA_ERR_INVALID_ARG;
     buf[0] = 0;
     Plan plan;
+    if (flags & kPlanAllowPairs) return TA_ERR_UNSUPPORTED;
     int rc = build_plan(B, H, H_kv, N, D, dims, ndims, dtype, flags, 0, 0, &plan);
     if (rc != TA_OK) return rc;
     size_t off = 0;
@@ -556,9 +651,10 @@ int ta_plan_describe(int B, int H, int H_kv, int N, int D, const int *dims, int 
             for (int f = 0; f < h.nf; ++f) emit("%s%dx%d", f ? "," : "", h.sub_n[f], h.sub_stride[f]);
             emit("%s", "\n");
         } else if (h.path == PATH_TC)
-            emit("hop=%d path=tc n=%d stride=%lld outer=%lld ci=%d co=%d rows=%d tiles_per_head=%lld src=%s dst=%s\n",
+            emit("hop=%d path=tc n=%d stride=%lld outer=%lld ci=%d co=%d rows=%d tiles_per_head=%lld src=%s dst=%s%s%s\n",
                  h.hop, h.n, h.stride, h.outer, h.ci, h.co, h.rows, h.tiles_inner * h.tiles_outer,
-                 buf_name(h.src), buf_name(h.dst));
+                 buf_name(h.src), buf_name(h.dst), h.out_f16 ? " dst_type=f16" : "",
+                 h.pair ? " pair=first" : (j > 0 && plan.hops[j - 1].pair ? " pair=second" : ""));
         else if (h.path == PATH_TC_LONG)
             emit("hop=%d path=tc-long n=%d stride=%lld outer=%lld key_blocks=%d src=%s dst=%s\n", h.hop, h.n, h.stride,
                  h.outer, (h.n + 127) / 128, buf_name(h.src), buf_name(h.dst));
@@ -571,12 +667,13 @@ int ta_plan_describe(int B, int H, int H_kv, int N, int D, const int *dims, int 
 
 int ta_device_status(void) {
     if (cudaDeviceSynchronize() != cudaSuccess) return TA_ERR_CUDA;
-    unsigned int w1 = 0, w2 = 0, w3 = 0, w4 = 0, w5 = 0;
+    unsigned int w1 = 0, w2 = 0, w3 = 0, w4 = 0, w5 = 0, w6 = 0, w7 = 0;
     if (read_status_tc_forward(&w1) != TA_OK || read_status_tc_backward(&w2) != TA_OK ||
         read_status_tc_fused(&w3) != TA_OK || read_status_tc_long(&w4) != TA_OK ||
-        read_status_tc_backward_long(&w5) != TA_OK)
+        read_status_tc_backward_long(&w5) != TA_OK || read_status_tc_pair(&w6) != TA_OK ||
+        read_status_selftest(&w7) != TA_OK)
         return TA_ERR_CUDA;
-    return (w1 | w2 | w3 | w4 | w5) ? TA_ERR_TIMEOUT : TA_OK;
+    return (w1 | w2 | w3 | w4 | w5 | w6 | w7) ? TA_ERR_TIMEOUT : TA_OK;
 }
 
 unsigned long long ta_launch_count(void) { return g_launches.load(); }
@@ -584,11 +681,14 @@ unsigned long long ta_launch_count(void) { return g_launches.load(); }
 int ta_release(void) {
     std::lock_guard<std::mutex> host_lock(g_host_mutex);
     std::lock_guard<std::mutex> lock(g_arena_mutex);
-    if (g_scratch.ptr || g_staging.ptr || g_rotated.ptr || g_host_pipe.ready) cudaDeviceSynchronize();
-    g_scratch.release();
+    cudaDeviceSynchronize();
     g_staging.release();
-    g_rotated.release();
     g_host_pipe.destroy();
+    {
+        std::lock_guard<std::mutex> pool_lock(g_pool_mutex);
+        for (int d = 0; d < 64; ++d)
+            if (g_pools[d]) cudaMemPoolTrimTo(g_pools[d], 0);   // cached blocks back to the driver
+    }
     return TA_OK;
 }
 

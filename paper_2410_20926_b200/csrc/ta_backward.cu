@@ -52,7 +52,8 @@ size_t backward_workspace_bytes(int B, int H, int H_kv, int N, int D, const int 
                                 int grad_dtype, bool have_saved_hops) {
     Plan plan;
     if (dtype == TA_DTYPE_F32 && grad_dtype != TA_DTYPE_F32) return 0;   // fp32 tensors take fp32 gradients
-    if (build_plan(B, H, H_kv, N, D, dims, ndims, dtype, TA_FLAG_NO_HOP_FUSION, 0, 0, &plan) != TA_OK) return 0;
+    if (build_plan(B, H, H_kv, N, D, dims, ndims, dtype, TA_FLAG_NO_HOP_FUSION | TA_FLAG_BF16_INTERMEDIATES, 0, 0, &plan) != TA_OK)
+        return 0;
     return layout(plan, B, H, H_kv, N, D, !have_saved_hops, grad_dtype != TA_DTYPE_F32,
                   dtype == TA_DTYPE_F32 ? 4 : 2).total;
 }
@@ -70,7 +71,8 @@ int backward_impl(const ta_bwd_params &p) {
             if (p.window[i] < 0) return TA_ERR_INVALID_ARG;
     Plan plan;
     // hop by hop: the backward needs every hop's input
-    const unsigned plan_flags = (unsigned)TA_FLAG_NO_HOP_FUSION;
+    // the recomputed hop inputs are operands of the backward kernels: bf16 like the gradients
+    const unsigned plan_flags = (unsigned)(TA_FLAG_NO_HOP_FUSION | TA_FLAG_BF16_INTERMEDIATES);
     int rc = build_plan(p.B, p.H, p.H_kv, p.N, p.D, p.dims, p.ndims, p.dtype, plan_flags, 0, 0, &plan);
     if (rc != TA_OK) return rc;
     if (p.D > 256) return TA_ERR_UNSUPPORTED;   // limit of the generic backward kernels

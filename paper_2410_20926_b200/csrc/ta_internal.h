@@ -21,7 +21,9 @@ enum HopPath {
     PATH_TC_LONG = 2 // tcgen05 kernel with a loop over key blocks and online softmax: n_i > 128
 };
 
-// build_plan flag used inside the library only: the call carries the positional encoding
+// build_plan flag used inside the library only (never part of the public flag set): plan pair
+// launches as a call with TA_FLAG_PAIR_HOPS would (ta_workspace_bytes sizes the counters with it).
+constexpr unsigned kPlanAllowPairs = 1u << 16;
 
 // One hop of Algorithm 1 as a strided view X[outer][t][inner][D] of a head:
 //   token(outer, t, inner) = outer * n * stride + t * stride + inner.
@@ -42,6 +44,13 @@ struct HopDesc {
     // coordinate has stride sub_stride[f] tokens inside the block.  nf <= 1: an ordinary hop.
     int nf;
     int sub_n[TA_MAX_DIMS], sub_stride[TA_MAX_DIMS], sub_hop[TA_MAX_DIMS];   // sub_hop: index in dims
+    // Storage of the value tensor this hop reads / writes: 0 = the call's dtype, 1 = fp16.  Between
+    // two tensor-core hops of one call the tensor is an intermediate nobody else reads; fp16 has the
+    // size of bf16 and three more mantissa bits, so a hop chain rounds to bf16 once, at its end.
+    int in_f16, out_f16;
+    // 1: this hop and the next one of the plan run as ONE launch of the pair kernel (the next hop's
+    // entry is then skipped by the launch loop); both update `out` in place.
+    int pair;
 };
 
 struct Plan {
@@ -50,6 +59,7 @@ struct Plan {
     bool need_scratch;      // some hop writes to / reads from BUF_SCRATCH
     size_t scratch_bytes;   // B*H*N*D*elem when need_scratch
     size_t save_bytes;      // (nhops-1)*B*H*N*D*elem, hop inputs X_1.. for backward
+    size_t flag_bytes;      // completion counters of the pair launches (after scratch and saved hops), 0 if none
 };
 
 struct Problem {
@@ -98,17 +108,36 @@ int launch_hop_tc(const Problem &pb, const HopDesc &hd, const void *xin, int xin
 // Long segments (n_i > 128): key-block loop with online softmax, ta_tc_long.cu.  xin != xout.
 int launch_hop_tc_long(const Problem &pb, const HopDesc &hd, const void *xin, int xin_heads, void *xout);
 int read_status_tc_long(unsigned int *word);
-// Positional encoding on long-segment hops: rotated bf16 copies of q and k in the library-owned
-// buffer (plus extra_bytes of scratch behind them), and dst (=|+=) R^T src for fp32 gradients.
+// Positional encoding on long-segment hops: rotated bf16 copies of q and k in a buffer taken from
+// the library's pool on the call's stream (plus extra_bytes of scratch behind them; the caller
+// hands *pooled back with pool_free after its last launch that reads it), and
+// dst (=|+=) R^T src for fp32 gradients.
 int rope_rotated_copies(const Problem &pb, const HopDesc &hd, const void **rq, const void **rk, size_t extra_bytes,
-                        void **extra);
+                        void **extra, void **pooled);
 int rope_unrotate_add(const Problem &pb, const HopDesc &hd, const float *src, float *dst, int heads, bool accumulate);
 // Statistics pass of the long-segment backward: stats[q_head * N + token] = (log2-sum-exp of the
 // row's scaled scores, <g_t, out_t>), B*H*N float2; g laid out like q.
 int launch_hop_tc_long_stats(const Problem &pb, const HopDesc &hd, const void *xin, int xin_heads, const void *g,
                              void *stats);
-// Library-owned buffer of at least `bytes` (grown on demand) for that kernel's rotated Q / K copies.
-int rotated_arena(size_t bytes, void **ptr);
+// Two adjacent hops in one L2-ordered launch (ta_tc_pair.cu).  `flags`: device, geo.flag_bytes,
+// cleared by the launcher on the stream.  Both hops write `out`; hop A reads xin (v or out).
+struct PairGeometry {
+    int hsplit;                 // items per GQA group and tile position (query heads per item = g / hsplit)
+    uint32_t items_a, items_b;  // work items of one unit in each phase
+    uint32_t units, lag, total;
+    size_t flag_bytes;
+    double window_bytes;        // bytes touched between the two hops of a unit (must sit in L2 to pay)
+};
+bool pair_geometry(int B, int H, int H_kv, const HopDesc &ha, const HopDesc &hb, int num_sms, PairGeometry *geo);
+int launch_hop_tc_pair(const Problem &pb, const HopDesc &ha, const HopDesc &hb, const void *xin, int xin_heads,
+                       void *out, void *flags);
+int read_status_tc_pair(unsigned int *word);
+int read_status_selftest(unsigned int *word);
+// Stream-ordered device memory from the library's own pool of the current device (created on
+// first use; trimmed by ta_release): no device-wide synchronisation, nothing shared between
+// streams or host threads, capturable.  pool_free returns the memory in stream order.
+int pool_alloc(size_t bytes, cudaStream_t stream, void **ptr);
+void pool_free(void *ptr, cudaStream_t stream);
 // Fused trailing hops (hd.nf > 1), ta_tc_fused.cu; called through launch_hop_tc.
 int launch_hop_tc_fused(const Problem &pb, const HopDesc &hd, const void *xin, int xin_heads, void *xout);
 // out[b,h] = v[b, h / (H/H_kv)] (all dims equal to 1).

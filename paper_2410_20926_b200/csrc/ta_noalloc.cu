@@ -40,7 +40,7 @@ int static_scratch_for_current_device(void **ptr) {
     if (!g_scratch_addr[dev]) {
         void *p = nullptr;
         cudaError_t e = cudaGetSymbolAddress((void **)&p, g_static_scratch);
-        if (e != cudaSuccess || !p) return TA_ERR_CUDA;
+        if (e != cudaSuccess || !p) return cuda_fail(e);
         g_scratch_addr[dev] = p;
     }
     *ptr = g_scratch_addr[dev];
@@ -56,6 +56,7 @@ extern "C" int ta_forward_static(const void *q, const void *k, const void *v, vo
                                  int N, int D, const int *dims, int ndims, int causal, int dtype,
                                  ta_stream_t stream) {
     if (!q || !k || !v || !out) return TA_ERR_INVALID_ARG;
+    tl_last_cuda_error = 0;
     Plan plan;
     int rc = build_plan(B, H, H_kv, N, D, dims, ndims, dtype, 0u, 0, 0, &plan);
     if (rc != TA_OK) return rc;
@@ -64,9 +65,9 @@ extern "C" int ta_forward_static(const void *q, const void *k, const void *v, vo
     if (plan.scratch_bytes > kStaticScratchBytes) return TA_ERR_TOO_LARGE;
 
     int dev = 0, major = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess)
-        return TA_ERR_CUDA;
+    cudaError_t ce = cudaGetDevice(&dev);
+    if (ce == cudaSuccess) ce = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (ce != cudaSuccess) return cuda_fail(ce);
     if (major != 10) return TA_ERR_ARCH;
 
     void *scratch = nullptr;

@@ -73,13 +73,14 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 // (a shared-memory word): a pipeline whose stages wait on one another drains in one time-out
 // instead of one per stage.  On expiry the flag is raised and the error word recorded.
 __device__ __noinline__ bool mbar_wait_abortable_slow(uint32_t bar, uint32_t parity, uint32_t where,
-                                                      volatile uint32_t *abort_flag) {
+                                                      volatile uint32_t *abort_flag,
+                                                      unsigned long long limit_ns = kWaitLimitNs) {
     const unsigned long long t0 = globaltimer_ns();
     for (;;) {
         for (int i = 0; i < 64; ++i)
             if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (globaltimer_ns() - t0 > kWaitLimitNs) {
+        if (globaltimer_ns() - t0 > limit_ns) {
             atomicCAS(&g_status_word, 0u, kErrWaitExpired | where);
             *abort_flag = 1u;
             return false;
@@ -87,10 +88,11 @@ __device__ __noinline__ bool mbar_wait_abortable_slow(uint32_t bar, uint32_t par
     }
 }
 __device__ __forceinline__ bool mbar_wait_abortable(uint32_t bar, uint32_t parity, uint32_t where,
-                                                    volatile uint32_t *abort_flag) {
+                                                    volatile uint32_t *abort_flag,
+                                                    unsigned long long limit_ns = kWaitLimitNs) {
     for (int i = 0; i < 16; ++i)
         if (mbar_try_wait(bar, parity)) return true;
-    return mbar_wait_abortable_slow(bar, parity, where, abort_flag);
+    return mbar_wait_abortable_slow(bar, parity, where, abort_flag, limit_ns);
 }
 
 __device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1,
@@ -206,6 +208,11 @@ __host__ __device__ constexpr uint32_t instr_desc(int n, int b_mn_major, int a_m
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn_major << 15) | ((uint32_t)b_mn_major << 16) |
            ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 }
+// The same with both operands fp16 (format code 0) instead of bf16 (A and B of one instruction
+// always have the same type).
+__host__ __device__ constexpr uint32_t instr_desc_f16(int n, int b_mn_major, int a_mn_major = 0) {
+    return instr_desc(n, b_mn_major, a_mn_major) & ~((7u << 7) | (7u << 10));
+}
 
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
@@ -219,6 +226,17 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     uint32_t r;
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
     return r;
+}
+__device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+// sum of the two fp16 halves of w, in fp32
+__device__ __forceinline__ float sum_f16x2(uint32_t w) {
+    float a, b;
+    asm("{\n .reg .b16 l, h;\n mov.b32 {l, h}, %2;\n cvt.f32.f16 %0, l;\n cvt.f32.f16 %1, h;\n}" : "=f"(a), "=f"(b) : "r"(w));
+    return a + b;
 }
 
 

@@ -73,6 +73,7 @@ struct TcArgs {
     float rope_log2_base;      // log2 of the RoPE base (rotating variant only)
     int stride;                // token stride of the hop's dimension
     const int *lens;           // device, one valid length per batch entry, or nullptr (masked variant only)
+    int x_f16, out_f16;        // the value tensor read / written holds fp16 (an intermediate of a hop chain), not bf16
 };
 
 struct ItemCoord {
@@ -227,7 +228,7 @@ hop_pipe_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         // =============================================================== MMA issuer
         if (lane == 0) {
             constexpr uint32_t idesc_s = instr_desc(128, 0);
-            constexpr uint32_t idesc_o = instr_desc(D, 1);
+            const uint32_t idesc_o = a.x_f16 ? instr_desc_f16(D, 1) : instr_desc(D, 1);   // P has the type of X
             const int kblocks = (a.rows + 15) >> 4;
             bool ok = true;
             auto issue_o = [&](uint32_t u) -> bool {
@@ -403,9 +404,15 @@ hop_pipe_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                             p0 = (row_valid && col >= c_lo && col < c_hi) ? p0 : 0.f;
                             p1 = (row_valid && col + 1 >= c_lo && col + 1 < c_hi) ? p1 : 0.f;
                         }
-                        const uint32_t w = pack_bf16x2(p0, p1);
+                        uint32_t w;
+                        if (a.x_f16) {          // uniform: the weights take the type of the value tile
+                            w = pack_f16x2(p0, p1);
+                            sum += sum_f16x2(w);
+                        } else {
+                            w = pack_bf16x2(p0, p1);
+                            sum += __uint_as_float(w << 16) + __uint_as_float(w & 0xFFFF0000u);
+                        }
                         pk[jj >> 1] = w;
-                        sum += __uint_as_float(w << 16) + __uint_as_float(w & 0xFFFF0000u);
                     }
                 } else {
 #pragma unroll
@@ -433,7 +440,8 @@ hop_pipe_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     uint32_t pk[16];
 #pragma unroll
                     for (int jj = 0; jj < 32; jj += 2)
-                        pk[jj >> 1] = pack_bf16x2(__uint_as_float(v[jj]) * inv, __uint_as_float(v[jj + 1]) * inv);
+                        pk[jj >> 1] = a.out_f16 ? pack_f16x2(__uint_as_float(v[jj]) * inv, __uint_as_float(v[jj + 1]) * inv)
+                                                : pack_bf16x2(__uint_as_float(v[jj]) * inv, __uint_as_float(v[jj + 1]) * inv);
                     const uint32_t slab = x_row + (uint32_t)(c >> 1) * kSlabBytes;
                     if (row_valid) {
 #pragma unroll
@@ -566,6 +574,8 @@ int launch_d(const Problem &pb, const HopDesc &hd, const void *xin, int xin_head
     a.rope_log2_base = pb.rope_base > 0.f ? log2f(pb.rope_base) : 0.f;
     a.stride = (int)hd.stride;
     a.lens = pb.seq_lens;
+    a.x_f16 = hd.in_f16;
+    a.out_f16 = hd.out_f16;
 
     constexpr size_t smem = PipeCfg<D>::kSmemBytes;
     const unsigned grid = (unsigned)(a.total_items < num_sms ? a.total_items : num_sms);

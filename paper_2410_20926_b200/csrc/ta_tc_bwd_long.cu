@@ -559,16 +559,19 @@ int launch_hop_tc_bwd_long(const Problem &pb, const HopDesc &hd, const void *x, 
         // and are turned back (R^T) while they are stored in / added to the accumulators.
         const size_t tq = (size_t)pb.B * pb.H * pb.N * pb.D, tkv = (size_t)pb.B * pb.H_kv * pb.N * pb.D;
         Problem hop = pb;
-        void *extra = nullptr;
-        int rc = rope_rotated_copies(pb, hd, &hop.q, &hop.k, (tq + tkv) * sizeof(float), &extra);
-        if (rc != TA_OK) return rc;
-        hop.rope_base = 0.f;
-        float *dq_rot = (float *)extra, *dk_rot = dq_rot + tq;
-        rc = pb.D == 128 ? launch_d<128>(hop, hd, x, x_heads, g_in, g_out, dq_rot, dk_rot, dv_acc, stats, first_hop, false)
-                         : launch_d<64>(hop, hd, x, x_heads, g_in, g_out, dq_rot, dk_rot, dv_acc, stats, first_hop, false);
-        if (rc != TA_OK) return rc;
-        if ((rc = rope_unrotate_add(pb, hd, dq_rot, dq_acc, pb.H, accumulate)) != TA_OK) return rc;
-        return rope_unrotate_add(pb, hd, dk_rot, dk_acc, pb.H_kv, accumulate);
+        void *extra = nullptr, *pooled = nullptr;
+        int rc = rope_rotated_copies(pb, hd, &hop.q, &hop.k, (tq + tkv) * sizeof(float), &extra, &pooled);
+        if (rc == TA_OK) {
+            hop.rope_base = 0.f;
+            float *dq_rot = (float *)extra, *dk_rot = dq_rot + tq;
+            rc = pb.D == 128
+                     ? launch_d<128>(hop, hd, x, x_heads, g_in, g_out, dq_rot, dk_rot, dv_acc, stats, first_hop, false)
+                     : launch_d<64>(hop, hd, x, x_heads, g_in, g_out, dq_rot, dk_rot, dv_acc, stats, first_hop, false);
+            if (rc == TA_OK) rc = rope_unrotate_add(pb, hd, dq_rot, dq_acc, pb.H, accumulate);
+            if (rc == TA_OK) rc = rope_unrotate_add(pb, hd, dk_rot, dk_acc, pb.H_kv, accumulate);
+        }
+        pool_free(pooled, pb.stream);
+        return rc;
     }
     if (pb.D == 128)
         return launch_d<128>(pb, hd, x, x_heads, g_in, g_out, dq_acc, dk_acc, dv_acc, stats, first_hop, accumulate);

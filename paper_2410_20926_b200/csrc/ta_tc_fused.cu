@@ -45,6 +45,7 @@ struct FusedArgs {
     int sub_n[TA_MAX_DIMS], sub_stride[TA_MAX_DIMS], sub_window[TA_MAX_DIMS];
     long long tiles_outer, total_items;
     float scale_log2;
+    int x_f16;                 // the value tensor read holds fp16 (output of a preceding tensor-core hop), not bf16
 };
 
 template <int D>
@@ -229,7 +230,9 @@ hop_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         // from its S = Q K^T until the value MMA of its last fused hop has been issued.
         if (lane == 0) {
             constexpr uint32_t idesc_s = instr_desc(128, 0);
-            constexpr uint32_t idesc_o = instr_desc(D, 1);
+            // the value tile is fp16 from the second fused hop on (and from the first one when the hop
+            // before this pass left fp16): the weights take its type
+            constexpr uint32_t idesc_o_bf16 = instr_desc(D, 1), idesc_o_f16 = instr_desc_f16(D, 1);
             const int kblocks = (a.rows + 15) >> 4;
             uint32_t t1 = 0, it = 0, j = 0, tiles_done = 0;
             bool busy[2] = {false, false};
@@ -283,6 +286,7 @@ hop_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                     const uint32_t d_tmem = tmem_base + C::kColO + (kNO == 2 ? 64 * b : 0);
                     const uint32_t p_tmem = tmem_base + C::kColP + 64 * b;
                     const uint32_t x_base = sX + xs * kTileBytes;
+                    const uint32_t idesc_o = (hop_of[b] > 0 || a.x_f16) ? idesc_o_f16 : idesc_o_bf16;
                     for (int kb = 0; kb < kblocks; ++kb)
                         tc_mma_ts(d_tmem, p_tmem + kb * 8, smem_desc_sw128(x_base + kb * 2048, kSlabBytes, 1024), idesc_o,
                                   kb > 0);
@@ -361,6 +365,8 @@ hop_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             for (int f = 0; f < a.nf; ++f, ++o_seen) {
                 // ---- softmax of this row over its mode-f vector; P (un-normalised, bf16) -> tensor memory
                 const uint32_t *mword = masks + ((size_t)f * kTileRows + r) * 4;
+                const bool x_f16 = f > 0 || a.x_f16 != 0;   // type of the value tile this hop multiplies
+                const bool out_f16 = f + 1 < a.nf;          // between fused hops the tile is fp16; the last one writes bf16
                 float m = -INFINITY;
                 uint32_t v[32];
 #pragma unroll 1
@@ -386,9 +392,15 @@ hop_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                             float p1 = fast_exp2(__uint_as_float(v[jj + 1]) * a.scale_log2 - m_scaled);
                             p0 = ((bits >> jj) & 1u) ? p0 : 0.f;
                             p1 = ((bits >> (jj + 1)) & 1u) ? p1 : 0.f;
-                            const uint32_t w = pack_bf16x2(p0, p1);
+                            uint32_t w;
+                            if (x_f16) {
+                                w = pack_f16x2(p0, p1);
+                                sum += sum_f16x2(w);
+                            } else {
+                                w = pack_bf16x2(p0, p1);
+                                sum += __uint_as_float(w << 16) + __uint_as_float(w & 0xFFFF0000u);
+                            }
                             pk[jj >> 1] = w;
-                            sum += __uint_as_float(w << 16) + __uint_as_float(w & 0xFFFF0000u);
                         }
                     } else {
 #pragma unroll
@@ -416,7 +428,8 @@ hop_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                         uint32_t pk[16];
 #pragma unroll
                         for (int jj = 0; jj < 32; jj += 2)
-                            pk[jj >> 1] = pack_bf16x2(__uint_as_float(v[jj]) * inv, __uint_as_float(v[jj + 1]) * inv);
+                            pk[jj >> 1] = out_f16 ? pack_f16x2(__uint_as_float(v[jj]) * inv, __uint_as_float(v[jj + 1]) * inv)
+                                                  : pack_bf16x2(__uint_as_float(v[jj]) * inv, __uint_as_float(v[jj + 1]) * inv);
                         if (row_valid) {
                             const uint32_t slab = x_row + (uint32_t)(c >> 1) * kSlabBytes;
 #pragma unroll
@@ -458,6 +471,7 @@ int launch_fused_d(const Problem &pb, const HopDesc &hd, const void *xin, int xi
     a.block = hd.n; a.rows = hd.rows; a.co = hd.co; a.causal = pb.causal;
     a.g = pb.H / pb.H_kv; a.H = pb.H; a.H_kv = pb.H_kv; a.xin_is_kv = xin_heads != pb.H ? 1 : 0;
     a.nf = hd.nf;
+    a.x_f16 = hd.in_f16;
     for (int f = 0; f < TA_MAX_DIMS; ++f) {
         a.sub_n[f] = f < hd.nf ? hd.sub_n[f] : 1;
         a.sub_stride[f] = f < hd.nf ? hd.sub_stride[f] : 1;

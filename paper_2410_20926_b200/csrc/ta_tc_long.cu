@@ -653,15 +653,16 @@ __global__ void rope_unrotate_add_kernel(const float *__restrict__ src, float *_
 unsigned rope_blocks(long long pairs) { return (unsigned)(pairs / 256 + 1 < 148 * 32 ? pairs / 256 + 1 : 148 * 32); }
 }  // namespace
 
-// Rotated bf16 copies of q and k for hop `hd` in the library-owned buffer, followed by
-// `extra_bytes` of scratch (*extra).
+// Rotated bf16 copies of q and k for hop `hd` in a pooled buffer (*pooled, stream-ordered), followed
+// by `extra_bytes` of scratch (*extra).
 int rope_rotated_copies(const Problem &pb, const HopDesc &hd, const void **rq_out, const void **rk_out,
-                        size_t extra_bytes, void **extra) {
+                        size_t extra_bytes, void **extra, void **pooled) {
     const size_t tq = (size_t)pb.B * pb.H * pb.N * pb.D, tkv = (size_t)pb.B * pb.H_kv * pb.N * pb.D;
     const size_t q_bytes = (tq * 2 + 255) & ~(size_t)255, k_bytes = (tkv * 2 + 255) & ~(size_t)255;
     void *buf = nullptr;
-    int rc = rotated_arena(q_bytes + k_bytes + extra_bytes, &buf);
+    int rc = pool_alloc(q_bytes + k_bytes + extra_bytes, pb.stream, &buf);
     if (rc != TA_OK) return rc;
+    *pooled = buf;
     __nv_bfloat16 *rq = (__nv_bfloat16 *)buf, *rk = (__nv_bfloat16 *)((char *)buf + q_bytes);
     const double log2_base = log2((double)pb.rope_base);
     const long long pq = (long long)(tq / 2), pk = (long long)(tkv / 2);
@@ -687,13 +688,19 @@ int launch_hop_tc_long(const Problem &pb, const HopDesc &hd, const void *xin, in
     if (xin == xout) return TA_ERR_INVALID_ARG;
     if (pb.D != 128 && pb.D != 64) return TA_ERR_UNSUPPORTED;
     Problem hop = pb;
+    void *pooled = nullptr;
     if (pb.rope_base > 0.f) {
-        const int rc = rope_rotated_copies(pb, hd, &hop.q, &hop.k, 0, nullptr);
-        if (rc != TA_OK) return rc;
+        const int rc = rope_rotated_copies(pb, hd, &hop.q, &hop.k, 0, nullptr, &pooled);
+        if (rc != TA_OK) {
+            pool_free(pooled, pb.stream);
+            return rc;
+        }
         hop.rope_base = 0.f;
     }
-    if (pb.D == 128) return launch_long_d<128>(hop, hd, xin, xin_heads, xout);
-    return launch_long_d<64>(hop, hd, xin, xin_heads, xout);
+    const int rc = pb.D == 128 ? launch_long_d<128>(hop, hd, xin, xin_heads, xout)
+                               : launch_long_d<64>(hop, hd, xin, xin_heads, xout);
+    pool_free(pooled, pb.stream);
+    return rc;
 }
 
 // The backward's statistics pass over a long-segment hop (no positional encoding): same pipeline,

@@ -39,7 +39,8 @@ def test_autograd_matches_oracle(dims, D, causal, kw):
     assert_close(out.detach().float().cpu().numpy(), ref, "bf16")
     rq, rk, rv = oracle.backward(inp["dout"], inp["q"], inp["k"], inp["v"], dims, causal, **okw)
     for name, t, r in (("dq", q, rq), ("dk", k, rk), ("dv", v, rv)):
-        assert_grad_close(t.grad.float().cpu().numpy().astype(np.float64), r, name)
+        assert_grad_close(t.grad.float().cpu().numpy().astype(np.float64), r, name, False,
+                          sum(1 for n in dims if n > 1), rope=bool(kw.get("rope_base")))
 
 
 def test_autograd_forward_only_and_argument_checks():

@@ -1,10 +1,10 @@
 """Hop fusion on the GPU: when the trailing dimensions span at most one 128-row tile their hops
 run as one pass (Q, K, value tile read once).  Checked against the fp64 oracle (bf16 tolerance:
 max abs <= 2e-2, mean abs <= 2e-3) and against the same library run hop by hop
-(TA_FLAG_NO_HOP_FUSION).  The fused pass rounds the value tensor to bf16 between hops exactly
-as the unfused passes do; only the order of the fp32 sums over a row's keys differs (the keys of
-a mode-i vector are interleaved with other columns of the tile), so the two runs agree to about
-one bf16 unit in the last place."""
+(TA_FLAG_NO_HOP_FUSION).  The fused pass rounds the value tensor to fp16 between hops exactly
+as the unfused tensor-core passes do; only the order of the fp32 sums over a row's keys differs
+(the keys of a mode-i vector are interleaved with other columns of the tile), so the two runs
+agree to about one bf16 unit in the last place."""
 import math
 
 import numpy as np

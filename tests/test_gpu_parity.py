@@ -146,23 +146,96 @@ def test_config2_bf16():
     assert_close(got, ref, "bf16")
 
 
-@pytest.mark.parametrize("idx,heads", [(3, [(0, 0), (0, 6), (0, 31)]), (4, [(0, 3), (0, 28)]),
-                                       (5, [(0, 9), (1, 22)])])
-def test_full_size_configs_sampled_heads(idx, heads):
-    """Full-size runs in the launch configuration the benchmark times; whole heads are compared
-    (the oracle computes one head at a time)."""
+HIST_EDGES = [0.0, 1e-4, 1e-3, 2e-3, 4e-3, 8e-3, 1.2e-2, 1.6e-2, 2e-2, 1.0]
+
+
+@pytest.mark.parametrize("idx", [3, 4, 5])
+def test_full_size_configs_every_head(idx):
+    """Full-size runs in the launch configuration the benchmark times; EVERY head is compared
+    with the oracle element by element (the oracle computes one head at a time, so the
+    reference never exists as a whole).  Also collects the histogram of the absolute errors;
+    with TA_ERROR_HISTOGRAM=<file> it is appended there as text."""
+    import os
     c = ta_inputs.CONFIGS[idx]
     inp = ta_inputs.make_config_inputs(c)
     got = gpu_forward(inp, c.B, c.H, c.H_kv, c.N, c.D, c.dims, c.causal, "bf16")
-    ref = oracle.forward(inp["q"], inp["k"], inp["v"], c.dims, c.causal, heads=heads)
-    sel = np.stack([got[b, h] for b, h in heads])
-    assert_close(sel, ref, "bf16")
+    hist = np.zeros(len(HIST_EDGES) - 1, dtype=np.int64)
+    worst, total, count = 0.0, 0.0, 0
+    for b in range(c.B):
+        for h in range(c.H):
+            ref = oracle.forward(inp["q"], inp["k"], inp["v"], c.dims, c.causal, heads=[(b, h)])[0]
+            err = np.abs(got[b, h].astype(np.float64) - ref)
+            mx, mean = assert_close(got[b, h], ref, "bf16")        # per head: max <= 2e-2, mean <= 2e-3
+            worst = max(worst, mx)
+            total += float(err.sum())
+            count += err.size
+            hist += np.histogram(err, bins=HIST_EDGES)[0]
+    assert hist.sum() == count and hist[-1] == 0
+    path = os.environ.get("TA_ERROR_HISTOGRAM")
+    if path:
+        with open(path, "a") as f:
+            f.write(f"config {idx}: {count} outputs, max abs err {worst:.5f}, mean abs err {total / count:.6f}\n")
+            for lo, hi, n in zip(HIST_EDGES[:-1], HIST_EDGES[1:], hist):
+                f.write(f"  [{lo:g}, {hi:g}): {int(n)} ({n / count:.3e})\n")
     # properties that hold at any size: finite, inside the range of V per column
     assert np.isfinite(got).all()
     g = c.H // c.H_kv
     vmax = np.repeat(inp["v"].max(axis=2), g, axis=1)[:, :, None, :]
     vmin = np.repeat(inp["v"].min(axis=2), g, axis=1)[:, :, None, :]
     assert (got <= vmax + 0.05).all() and (got >= vmin - 0.05).all()
+
+
+@pytest.mark.parametrize("B,H,Hkv,D,dims,dtype,flags", [
+    (1, 4, 2, 128, [8, 16, 32], "bf16", 0),                       # tensor-core hops
+    (1, 4, 2, 40, [5, 6, 7], "bf16", 0),                          # generic hops (head dim 40)
+    (2, 2, 1, 64, [4, 160, 2], "bf16", 0),                        # tensor-core, long-segment, tensor-core
+    (1, 2, 2, 32, [4, 4, 8], "f32", 0),                           # fp32
+    (1, 4, 2, 128, [8, 16, 32], "bf16", "save"),                  # with the hop inputs saved
+    (1, 4, 2, 40, [5, 6, 7], "bf16", "save"),
+])
+def test_hop_ranges_compose_to_the_single_call(B, H, Hkv, D, dims, dtype, flags):
+    """Running hops [0, j) and then [j, m) (the second call reads its value tensor from `out`)
+    gives the result of the single call, for every split point and every kind of plan --
+    including plans in which the first hop of the second call cannot update `out` in place."""
+    import torch
+    N = math.prod(dims)
+    m = len(dims)
+    inp = ta_inputs.make_inputs(B, H, Hkv, N, D, dtype, 116)
+    q, k, v = (to_device(inp, n, dtype) for n in ("q", "k", "v"))
+    tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    code = ta.TA_DTYPE_BF16 if dtype == "bf16" else ta.TA_DTYPE_F32
+    ref_out, xs = oracle.forward(inp["q"], inp["k"], inp["v"], dims, True, return_xs=True)
+    whole = torch.empty((B, H, N, D), dtype=tdt, device="cuda")
+    # (bf16 between the hops, as a call that stops after hop j must leave it in `out`)
+    base = ta.TA_FLAG_NO_HOP_FUSION | ta.TA_FLAG_BF16_INTERMEDIATES
+    ta.ta_forward_ex(q, k, v, whole, B, H, Hkv, N, D, dims, True, dtype=code, flags=base)
+    for j in range(1, m):
+        out = torch.empty((B, H, N, D), dtype=tdt, device="cuda")
+        kw = {}
+        if flags == "save":
+            nbytes = ta.ta_workspace_bytes(B, H, Hkv, N, D, dims, code, ta.TA_WS_FORWARD_SAVE) + B * H * N * D * 4
+            kw = dict(workspace=torch.empty(nbytes, dtype=torch.uint8, device="cuda"), workspace_bytes=nbytes)
+        f = base | (ta.TA_FLAG_SAVE_HOPS if flags == "save" else 0)
+        ta.ta_forward_ex(q, k, v, out, B, H, Hkv, N, D, dims, True, dtype=code, flags=f, hop_begin=0, hop_end=j, **kw)
+        torch.cuda.synchronize()
+        mid = out.float().cpu().numpy()
+        assert_close(mid, np.stack([x[j] for x in xs]).reshape(B, H, N, D), dtype)
+        ta.ta_forward_ex(q, k, v, out, B, H, Hkv, N, D, dims, True, dtype=code, flags=f, hop_begin=j, hop_end=m, **kw)
+        torch.cuda.synchronize()
+        ta.ta_device_status()
+        assert torch.equal(out, whole), (j, dims)
+    assert_close(whole.float().cpu().numpy(), ref_out, dtype)
+
+
+def test_out_overlapping_an_input_is_rejected():
+    import torch
+    B, H, N, D = 1, 2, 256, 64
+    x = torch.zeros((B, H, N, D), dtype=torch.bfloat16, device="cuda")
+    y = torch.zeros((2, B, H, N, D), dtype=torch.bfloat16, device="cuda")
+    assert ta.ta_forward(x, x, x, x, B, H, H, N, D, [16, 16], True, check=False) == ta.TA_ERR_INVALID_ARG
+    assert ta.ta_forward(x, y[0], x, y.view(-1)[64:64 + x.numel()].view_as(x), B, H, H, N, D, [16, 16], True,
+                         check=False) == ta.TA_ERR_INVALID_ARG
+    assert ta.ta_forward(x, x, x, y[1], B, H, H, N, D, [16, 16], True, check=False) == ta.TA_OK
 
 
 def test_forward_host_back_to_back_calls_use_both_staging_sets():

@@ -1,9 +1,10 @@
 """Seeded random configurations: tensor shapes, head dims, GQA ratios and every combination of the
 options (causal flag, windows, explicit masks, valid lengths, positional encoding, fusion on/off),
 forward and backward, against the fp64 oracle.  Catches interactions the targeted tests do not
-enumerate.  Tolerances as everywhere else, except that the bound on the mean error of a gradient
-grows with the size of the gradient the way the bound on its maximum does: some of these tensors
-have a handful of rows, each a sum over a whole GQA group."""
+enumerate.  Tolerances as everywhere else: the forward bound of helpers.bf16_max_abs (2e-2 up to
+three hops, growing linearly beyond) and the gradient bound of test_gpu_backward.assert_grad_close.
+Besides the first 48 seeds the list holds the ten seeds that a sweep of 1 600 found closest to -- at
+the time, beyond -- the bounds (four-hop shapes and the positional encoding)."""
 import math
 
 import numpy as np
@@ -13,7 +14,7 @@ import oracle
 import paper_2410_20926_b200 as ta
 from paper_2410_20926_b200 import inputs as ta_inputs
 
-from helpers import assert_close, gpu_forward
+from helpers import assert_close, gpu_forward, real_hops
 from test_gpu_backward import assert_grad_close, gpu_backward
 
 pytestmark = pytest.mark.gpu
@@ -56,7 +57,10 @@ def random_config(seed):
     return B, H, Hkv, D, dims, causal, kw, okw, flags
 
 
-@pytest.mark.parametrize("seed", range(48))
+HARD_SEEDS = [503, 522, 602, 659, 882, 1067, 1174, 1264, 1454, 1536]
+
+
+@pytest.mark.parametrize("seed", list(range(48)) + HARD_SEEDS)
 def test_random_configuration(seed):
     import torch
     B, H, Hkv, D, dims, causal, kw, okw, flags = random_config(seed)
@@ -68,12 +72,11 @@ def test_random_configuration(seed):
     inp = ta_inputs.make_inputs(B, H, Hkv, N, D, "bf16", 2000 + seed, with_dout=True)
     got = gpu_forward(inp, B, H, Hkv, N, D, dims, causal, "bf16", flags, **gkw)
     ref = oracle.forward(inp["q"], inp["k"], inp["v"], dims, causal, **okw)
-    assert_close(got, ref, "bf16")
+    assert_close(got, ref, "bf16", real_hops(dims))
     if all(n == 1 for n in dims) and lens is not None:
         return                                   # no hop to apply the lengths in: the backward declines
     bkw = {k: v for k, v in gkw.items()}
     grads = gpu_backward(inp, B, H, Hkv, N, D, dims, causal, bool(seed % 2), **bkw)
     refs = oracle.backward(inp["dout"], inp["q"], inp["k"], inp["v"], dims, causal, **okw)
     for name, g, r in zip(("dq", "dk", "dv"), grads, refs):
-        # mean bound: a tenth of the bound on the maximum, as for the forward (2e-3 vs 2e-2)
-        assert_grad_close(g, r, name, mean_rtol=2.0 ** -8 / 10)
+        assert_grad_close(g, r, name, bool(seed % 2), real_hops(dims), rope="rope_base" in kw)

@@ -88,7 +88,7 @@ def test_backward_with_window(dims, window, D, causal):
     got = gpu_backward(inp, B, H, Hkv, N, D, dims, causal, True, window=window)
     ref = oracle.backward(inp["dout"], inp["q"], inp["k"], inp["v"], dims, causal, window=window)
     for name, g, r in zip(("dq", "dk", "dv"), got, ref):
-        assert_grad_close(g, r, name)
+        assert_grad_close(g, r, name, True, sum(1 for n in dims if n > 1))
 
 
 def test_window_llama_shape_sampled_heads():

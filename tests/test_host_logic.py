@@ -77,7 +77,9 @@ def test_forward_ex_rejects_bad_struct_and_workspace():
 def test_workspace_bytes():
     e = 1 * 2 * 256 * 64
     assert ta.ta_workspace_bytes(1, 2, 2, 256, 64, [16, 16], ta.TA_DTYPE_F32) == 4 * e
-    assert ta.ta_workspace_bytes(1, 2, 2, 256, 64, [16, 16], ta.TA_DTYPE_BF16) == 0
+    # two adjacent tensor-core hops run as one pair launch: a few bytes of completion counters
+    assert ta.ta_workspace_bytes(1, 2, 2, 256, 64, [16, 16], ta.TA_DTYPE_BF16) == 256
+    assert ta.ta_workspace_bytes(1, 2, 2, 256, 64, [16], ta.TA_DTYPE_BF16) == 0
     assert ta.ta_workspace_bytes(1, 2, 2, 256, 64, [16, 16], ta.TA_DTYPE_BF16,
                                  ta.TA_WS_FORWARD_SAVE) == 2 * e
     assert ta.ta_workspace_bytes(1, 2, 2, 256, 64, [16, 15], ta.TA_DTYPE_BF16) == 0
@@ -99,6 +101,32 @@ def test_plan_llama_128k():
     assert [(h["ci"], h["co"], h["rows"]) for h in hops] == \
         [("4", "1", "128"), ("2", "1", "128"), ("1", "2", "128")]
     assert [(h["src"], h["dst"]) for h in hops] == [("v", "out"), ("out", "out"), ("out", "out")]
+
+
+def test_plan_intermediates_and_pair_launches():
+    dims = [32, 32, 32]
+    # between tensor-core hops the value tensor is fp16 (same bytes, finer rounding); the last hop writes bf16
+    _, hops = parse_plan(ta.ta_plan_describe(1, 32, 8, 32768, 128, dims, True))
+    assert [h.get("dst_type") for h in hops] == ["f16", "f16", None]
+    assert all("pair" not in h for h in hops)
+    _, hops = parse_plan(ta.ta_plan_describe(1, 32, 8, 32768, 128, dims, True, flags=ta.TA_FLAG_BF16_INTERMEDIATES))
+    assert [h.get("dst_type") for h in hops] == [None, None, None]
+    # the forward that saves the hop inputs for the backward keeps them bf16
+    _, hops = parse_plan(ta.ta_plan_describe(1, 32, 8, 32768, 128, dims, True, flags=ta.TA_FLAG_SAVE_HOPS))
+    assert [h.get("dst_type") for h in hops] == [None, None, None]
+    assert [h["dst"] for h in hops] == ["save", "save", "out"]
+    # a hop next to a long-segment or generic hop stays bf16
+    _, hops = parse_plan(ta.ta_plan_describe(1, 2, 2, 16 * 16 * 200, 64, [16, 16, 200], True))
+    assert [h.get("dst_type") for h in hops] == ["f16", None, None]
+    # pair launches: opt-in, the last two hops of the Llama shapes; counters in the workspace
+    _, hops = parse_plan(ta.ta_plan_describe(1, 32, 8, 32768, 128, dims, True, flags=ta.TA_FLAG_PAIR_HOPS))
+    assert [h.get("pair") for h in hops] == [None, "first", "second"]
+    _, hops = parse_plan(ta.ta_plan_describe(1, 32, 8, 131072, 128, [32, 64, 64], True, flags=ta.TA_FLAG_PAIR_HOPS))
+    assert [h.get("pair") for h in hops] == [None, "first", "second"]
+    _, hops = parse_plan(ta.ta_plan_describe(1, 32, 8, 32768, 128, dims, True,
+                                             flags=ta.TA_FLAG_PAIR_HOPS | ta.TA_FLAG_NO_HOP_FUSION))
+    assert all("pair" not in h for h in hops)
+    assert ta.ta_workspace_bytes(1, 32, 8, 32768, 128, dims, ta.TA_DTYPE_BF16) == 8 * 32 * 4
 
 
 def test_plan_skips_unit_dims_and_routes_generic_hops():
