@@ -369,8 +369,8 @@ def run_ours(args, cfg):
     dev = torch.device("cuda", local)
     ta.load()
     op = args.op
-    if args.rope_base > 0 and op != "forward":
-        raise SystemExit("--rope-base is offered for --op forward only")
+    if (args.rope_base > 0 or args.pair_hops) and op != "forward":
+        raise SystemExit("--rope-base and --pair-hops are offered for --op forward only")
 
     inp = ta_inputs.make_inputs(cfg.B, cfg.H, cfg.H_kv, cfg.N, cfg.D, cfg.dtype, cfg.seed, with_dout=op != "forward")
     host = {}
@@ -396,9 +396,10 @@ def run_ours(args, cfg):
             counter[0] += 1
         c = cfg
         if op == "forward":
-            if args.rope_base > 0:
+            if args.rope_base > 0 or args.pair_hops:
                 ta.ta_forward_ex(s.q, s.k, s.v, s.out, c.B, c.H, c.H_kv, c.N, c.D, dims, c.causal, dtype=s.code,
-                                 rope_base=args.rope_base, stream=stream)
+                                 rope_base=args.rope_base, flags=ta.TA_FLAG_PAIR_HOPS if args.pair_hops else 0,
+                                 stream=stream)
             elif c.dtype == "bf16":
                 ta.ta_forward(s.q, s.k, s.v, s.out, c.B, c.H, c.H_kv, c.N, c.D, dims, c.causal, stream=stream)
             else:
@@ -458,7 +459,7 @@ def run_ours(args, cfg):
     # ---- end to end: host buffers in, host buffers out, copies inside the timed region
     e2e_steps = max(1, min(args.steps, 10))
     s0 = sets[0]
-    if op == "forward" and args.rope_base == 0:
+    if op == "forward" and args.rope_base == 0 and not args.pair_hops:
         def e2e_step():
             ta.ta_forward_host(host["q"], host["k"], host["v"], host["out"], cfg.B, cfg.H, cfg.H_kv, cfg.N, cfg.D,
                                dims, cfg.causal, dtype=s0.code, stream=stream)
@@ -502,7 +503,7 @@ def run_ours(args, cfg):
     barrier(world)
     e2e_value = aggregate(cfg.B * cfg.N, world, e2e_ms, e2e_steps)
     same = None
-    if op == "forward" and args.rope_base == 0:
+    if op == "forward" and args.rope_base == 0 and not args.pair_hops:
         step(s0)
         torch.cuda.synchronize()
         same = bool(torch.equal(host["out"], s0.out.cpu()))       # same bits as the device-resident run
@@ -514,12 +515,18 @@ def run_ours(args, cfg):
     if args.rope_base > 0:
         roofline["kernel"] = "hop_pipe_kernel<128, true, false>"
         roofline["traffic"] = None
+    if args.pair_hops:
+        roofline["kernel"] = "hop_pipe_kernel<128, false, false> + hop_pair_kernel<128>"
+        roofline["traffic"] = None
     cpu, _ = oracle_sample(cfg, inp, op, min_seconds=args.cpu_seconds)
 
     cfg_desc = workload_config(cfg, world, op, len(sets))
     if args.rope_base > 0:
         cfg_desc["workload"] += f", tensorized positional encoding fused (RoPE base {args.rope_base:g})"
         cfg_desc["rope_base"] = args.rope_base
+    if args.pair_hops:
+        cfg_desc["workload"] += ", adjacent hops paired into one L2-ordered launch (TA_FLAG_PAIR_HOPS)"
+        cfg_desc["pair_hops"] = True
     line = {"metric": METRICS[op], "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": cfg.dtype if cfg.dtype == "bf16" else "f32",
@@ -548,6 +555,8 @@ def main():
     ap.add_argument("--repeats", type=int, default=5, help="further timed blocks of K steps (median / min reported)")
     ap.add_argument("--sets", type=int, default=0, help="rotating buffer sets (0: enough to exceed twice the L2)")
     ap.add_argument("--cpu-seconds", type=float, default=10.0, help="CPU time budget of the oracle sample")
+    ap.add_argument("--pair-hops", action="store_true",
+                    help="forward with TA_FLAG_PAIR_HOPS (two adjacent hops in one L2-ordered launch; not the default path)")
     ap.add_argument("--rope-base", type=float, default=0.0,
                     help="> 0: time the forward with the fused tensorized positional encoding (not the "
                          "headline workload)")

@@ -91,8 +91,10 @@ enum {
                                       /* follow the first hop's tiles of the same block closely enough  */
                                       /* to find them in the L2 cache (see ta_forward).  Same results,  */
                                       /* bit for bit; half the HBM traffic of the two hops.  Off by     */
-                                      /* default: on B200 the launch is bound by the SM-side pipeline,  */
-                                      /* not by HBM, and measured 10-20 % slower than hop by hop.       */
+                                      /* default: on B200 the distance that keeps the CTAs from waiting */
+                                      /* on one another is longer than what the L2 retains; measured    */
+                                      /* 5-10 % slower than hop by hop.  (TA_PAIR_LAG_UNITS=<n> in the   */
+                                      /* environment sets that distance, in blocks, for measurements.)  */
 };
 
 /* modes of ta_workspace_bytes */
@@ -182,9 +184,15 @@ typedef struct ta_params {
  *
  * Explicit masks: hop_masks[i] = NULL, or a host matrix of n_i x n_i bytes (row = query position
  * along dimension i, column = key position, non-zero = visible), the same for every mode-i
- * vector of the hop, applied on top of `causal` and window[i].  Read during the call.  Supported
- * for n_i <= 128 (TA_ERR_UNSUPPORTED beyond); a query position left without any visible key is
- * TA_ERR_INVALID_ARG.  Hops are not fused when a mask is given.  ta_backward_ex takes the same.
+ * vector of the hop, applied on top of `causal` and window[i].  Read during the call.  Any
+ * pattern can be given this way (block-sparse layouts, a few always-visible leading keys plus a
+ * local band, ...).  A query position left without any visible key is TA_ERR_INVALID_ARG.  Up to
+ * n_i = 128 the mask travels as a kernel parameter; for longer dimensions the library packs it to
+ * a bit matrix (n_i * n_i / 8 bytes) in pooled device memory, copied in stream order from pageable
+ * memory (such a call cannot be captured in a CUDA graph), the tensor-core kernel skips the key
+ * blocks before the first and after the last one a block of 128 queries sees and tests one bit
+ * per score in between, and the backward of such a hop runs on the generic kernels.  Hops are not
+ * fused when a mask is given.  ta_backward_ex takes the same.
  *
  * Valid lengths (padding to prod(dims), batches of different lengths; a mask M_i that depends
  * on the segment): with seq_lens != NULL only the tokens of batch entry b with flat index

@@ -5,6 +5,7 @@
 #include <cstdio>
 #include <cstring>
 #include <mutex>
+#include <vector>
 
 #include "ta_internal.h"
 
@@ -217,8 +218,66 @@ int build_hop_mask(const Problem &pb, const HopDesc &hd, HopMask *hm) {
     return TA_OK;
 }
 
+int upload_long_masks(Problem *pb, const Plan &plan, void **pooled) {
+    *pooled = nullptr;
+    size_t total_words = 0;
+    for (int j = 0; j < plan.nhops; ++j) {
+        const HopDesc &h = plan.hops[j];
+        if (h.nf > 1 || !pb->masks[h.hop] || h.n <= 128) continue;
+        const size_t words = (size_t)((h.n + 127) / 128) * 4, qblocks = (size_t)(h.n + 127) / 128;
+        total_words += (size_t)h.n * words + 2 * qblocks;
+        total_words = (total_words + 3) & ~(size_t)3;
+    }
+    if (total_words == 0) return TA_OK;
+    std::vector<uint32_t> host(total_words, 0u);
+    struct Placed { int hop; size_t off; int words; };
+    std::vector<Placed> placed;
+    size_t off = 0;
+    for (int j = 0; j < plan.nhops; ++j) {
+        const HopDesc &h = plan.hops[j];
+        if (h.nf > 1 || !pb->masks[h.hop] || h.n <= 128) continue;
+        const int n = h.n, words = ((n + 127) / 128) * 4, qblocks = (n + 127) / 128;
+        const unsigned char *m = pb->masks[h.hop];
+        const int w = pb->window[h.hop];
+        uint32_t *bits = host.data() + off;
+        int *ranges = (int *)(bits + (size_t)n * words);
+        for (int qb = 0; qb < qblocks; ++qb) { ranges[2 * qb] = qblocks; ranges[2 * qb + 1] = 0; }
+        for (int t = 0; t < n; ++t) {
+            bool any = false;
+            for (int u = 0; u < n; ++u) {
+                if (pb->causal && u > t) break;
+                if (w > 0 && (t - u >= w || u - t >= w)) continue;
+                if (!m[(size_t)t * n + u]) continue;
+                bits[(size_t)t * words + (u >> 5)] |= 1u << (u & 31);
+                any = true;
+                int &lo = ranges[2 * (t / 128)], &hi = ranges[2 * (t / 128) + 1];
+                if (u / 128 < lo) lo = u / 128;
+                if (u / 128 + 1 > hi) hi = u / 128 + 1;
+            }
+            if (!any) return TA_ERR_INVALID_ARG;
+        }
+        placed.push_back({h.hop, off, words});
+        off += (size_t)n * words + 2 * (size_t)qblocks;
+        off = (off + 3) & ~(size_t)3;
+    }
+    void *dev = nullptr;
+    int rc = pool_alloc(total_words * sizeof(uint32_t), pb->stream, &dev);
+    if (rc != TA_OK) return rc;
+    *pooled = dev;
+    // (pageable source: the runtime stages it before the call returns, so `host` may go away)
+    const cudaError_t e = cudaMemcpyAsync(dev, host.data(), total_words * sizeof(uint32_t), cudaMemcpyHostToDevice, pb->stream);
+    if (e != cudaSuccess) return cuda_fail(e);
+    for (const Placed &pl : placed) {
+        pb->dmask[pl.hop] = (const uint32_t *)dev + pl.off;
+        pb->dmask_words[pl.hop] = pl.words;
+    }
+    return TA_OK;
+}
+
 int take_masks(Problem *pb, const Plan &plan, const int *window, const unsigned char *const *hop_masks, int ndims) {
     for (int i = 0; i < TA_MAX_DIMS; ++i) {
+        pb->dmask[i] = nullptr;
+        pb->dmask_words[i] = 0;
         pb->window[i] = (window && i < ndims) ? window[i] : 0;
         pb->masks[i] = (hop_masks && i < ndims) ? hop_masks[i] : nullptr;
         if (pb->window[i] < 0) return TA_ERR_INVALID_ARG;
@@ -226,7 +285,7 @@ int take_masks(Problem *pb, const Plan &plan, const int *window, const unsigned 
     // every masked hop is checked before anything is launched
     for (int j = 0; j < plan.nhops; ++j) {
         const HopDesc &h = plan.hops[j];
-        if (h.nf > 1 || !pb->masks[h.hop]) continue;
+        if (h.nf > 1 || !pb->masks[h.hop] || h.n > 128) continue;   // longer dimensions: upload_long_masks
         HopMask hm;
         const int rc = build_hop_mask(*pb, h, &hm);
         if (rc != TA_OK) return rc;
@@ -454,9 +513,10 @@ static int forward_impl(const ta_params &p) {
         return ws + plan.scratch_bytes + (size_t)(id - 3) * tensor_bytes;
     };
     void *flags = ws ? ws + plan.scratch_bytes + plan.save_bytes : nullptr;
+    void *pooled_masks = nullptr;
+    rc = upload_long_masks(&pb, plan, &pooled_masks);
 
-    rc = TA_OK;
-    if (p.hop_begin > 0 && plan.hops[0].src == BUF_SCRATCH) {
+    if (rc == TA_OK && p.hop_begin > 0 && plan.hops[0].src == BUF_SCRATCH) {
         const cudaError_t e = cudaMemcpyAsync(ws, p.out, tensor_bytes, cudaMemcpyDeviceToDevice, pb.stream);
         if (e != cudaSuccess) rc = cuda_fail(e);
     }
@@ -475,6 +535,7 @@ static int forward_impl(const ta_params &p) {
              : h.path == PATH_TC_LONG ? launch_hop_tc_long(pb, h, xin, xin_heads, xout)
                                       : launch_hop_simt(pb, h, xin, xin_heads, xout);
     }
+    pool_free(pooled_masks, pb.stream);
     pool_free(pooled, pb.stream);
     return rc;
 }

@@ -105,6 +105,8 @@ int backward_impl(const ta_bwd_params &p) {
     if ((rc = take_masks(&pb, plan, p.window, p.hop_masks, p.ndims)) != TA_OK) return rc;
     pb.flags = 0; pb.hop_begin = 0; pb.hop_end = p.ndims;
     pb.stream = (cudaStream_t)p.stream;
+    PooledGuard long_masks{nullptr, pb.stream};      // bit matrices of masked dimensions longer than 128
+    if ((rc = upload_long_masks(&pb, plan, &long_masks.ptr)) != TA_OK) return rc;
 
     const size_t tq = (size_t)p.B * p.H * p.N * p.D, tkv = (size_t)p.B * p.H_kv * p.N * p.D;
     char *ws = (char *)p.workspace;
@@ -115,13 +117,12 @@ int backward_impl(const ta_bwd_params &p) {
 
     if (k == 0) {
         if (p.seq_lens) return TA_ERR_UNSUPPORTED;   // no hop to apply the valid lengths in
-        if (p.dtype != TA_DTYPE_BF16) return TA_ERR_UNSUPPORTED;
         if (cudaMemsetAsync(dq_acc, 0, tq * 4, pb.stream) != cudaSuccess ||
             cudaMemsetAsync(dk_acc, 0, tkv * 4, pb.stream) != cudaSuccess)
             return TA_ERR_CUDA;
         // every dimension is 1: out = v broadcast over the group, so dv = sum of dout, dq = dk = 0
-        rc = launch_group_sum(p.dout, need_acc ? (void *)p.dv : (void *)dv_acc, need_acc ? 0 : 1, p.B, p.H, p.H_kv,
-                              (long long)p.N * p.D, pb.stream);
+        rc = launch_group_sum(p.dout, p.dtype == TA_DTYPE_F32 ? 1 : 0, need_acc ? (void *)p.dv : (void *)dv_acc,
+                              need_acc ? 0 : 1, p.B, p.H, p.H_kv, (long long)p.N * p.D, pb.stream);
         if (rc != TA_OK) return rc;
     } else {
         // No clearing: the first hop processed (the last hop) stores dq / dk, later ones add to

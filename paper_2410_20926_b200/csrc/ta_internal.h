@@ -75,6 +75,13 @@ struct Problem {
     int window[TA_MAX_DIMS];  // per dimension: 0 = none, w > 0 = keys within w positions of the query
     const unsigned char *masks[TA_MAX_DIMS];  // per dimension: NULL or host n x n bytes, non-zero = visible
     const int *seq_lens;                      // device, B valid lengths, or NULL
+    // Explicit masks of dimensions longer than 128 (too large for a kernel parameter): device
+    // bit matrix, row t = query position, bit u of the row = key position u visible (causal flag and
+    // window already folded in), dmask_words 32-bit words per row (a multiple of 4); behind the
+    // rows, per 128-position query block, the first and one-past-the-last key block (of 128) that
+    // any of its rows sees: 2 ints per block.  NULL for the other dimensions.
+    const uint32_t *dmask[TA_MAX_DIMS];
+    int dmask_words[TA_MAX_DIMS];
     int pdl;   // 1: this launch follows a hop kernel of the same call in the stream and may overlap its tail
     unsigned flags;
     int hop_begin, hop_end;
@@ -98,6 +105,10 @@ struct HopMask {
 int build_hop_mask(const Problem &pb, const HopDesc &hd, HopMask *hm);
 // Host: sets pb.window / pb.masks from the caller's arrays and checks them against the plan.
 int take_masks(Problem *pb, const Plan &plan, const int *window, const unsigned char *const *hop_masks, int ndims);
+// Masked hops with n > 128: builds their bit matrices on the host, copies them into one pooled
+// device buffer (*pooled; pool_free it after the last launch) in stream order and sets pb.dmask.
+// TA_ERR_INVALID_ARG if a query position is left without any visible key.
+int upload_long_masks(Problem *pb, const Plan &plan, void **pooled);
 
 // Kernel launchers (each returns TA_OK or TA_ERR_CUDA).  xin has `xin_heads` heads per batch
 // (H_kv when reading v, H otherwise); xout always has H heads.
@@ -138,6 +149,12 @@ int read_status_selftest(unsigned int *word);
 // streams or host threads, capturable.  pool_free returns the memory in stream order.
 int pool_alloc(size_t bytes, cudaStream_t stream, void **ptr);
 void pool_free(void *ptr, cudaStream_t stream);
+// hands a pooled buffer back (in stream order) on every way out of a scope
+struct PooledGuard {
+    void *ptr;
+    cudaStream_t stream;
+    ~PooledGuard() { pool_free(ptr, stream); }
+};
 // Fused trailing hops (hd.nf > 1), ta_tc_fused.cu; called through launch_hop_tc.
 int launch_hop_tc_fused(const Problem &pb, const HopDesc &hd, const void *xin, int xin_heads, void *xout);
 // out[b,h] = v[b, h / (H/H_kv)] (all dims equal to 1).
@@ -164,8 +181,8 @@ int launch_hop_tc_bwd_long(const Problem &pb, const HopDesc &hd, const void *x, 
                            void *g_out, float *dq_acc, float *dk_acc, float *dv_acc, void *stats, bool first_hop,
                            bool accumulate);
 int launch_f32_to_bf16(const float *src, void *dst, long long n, cudaStream_t stream);
-int launch_group_sum(const void *dout, void *dv, int dv_is_f32, int B, int H, int H_kv, long long per_head,
-                     cudaStream_t stream);
+int launch_group_sum(const void *dout, int dout_is_f32, void *dv, int dv_is_f32, int B, int H, int H_kv,
+                     long long per_head, cudaStream_t stream);
 
 int backward_impl(const ta_bwd_params &p);
 size_t backward_workspace_bytes(int B, int H, int H_kv, int N, int D, const int *dims, int ndims, int dtype,

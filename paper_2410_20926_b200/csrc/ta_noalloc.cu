@@ -82,7 +82,7 @@ extern "C" int ta_forward_static(const void *q, const void *k, const void *v, vo
     pb.rope_base = 0.f;
     pb.seq_lens = nullptr;
     pb.pdl = 0;
-    for (int i = 0; i < TA_MAX_DIMS; ++i) { pb.window[i] = 0; pb.masks[i] = nullptr; }
+    for (int i = 0; i < TA_MAX_DIMS; ++i) { pb.window[i] = 0; pb.masks[i] = nullptr; pb.dmask[i] = nullptr; pb.dmask_words[i] = 0; }
     pb.flags = 0; pb.hop_begin = 0; pb.hop_end = ndims;
     pb.stream = (cudaStream_t)stream;
 

@@ -33,7 +33,9 @@ struct SimtArgs {
     float scale;
     float rope_log2_base;         // 0: no positional encoding; else log2 of the RoPE base
     int window;                   // 0, or sliding window along the hop's dimension
-    int masked;                   // 1: visibility comes from the HopMask parameter (n <= 128)
+    int masked;                   // 1: visibility comes from the HopMask parameter (n <= 128), 2: from dmask
+    const uint32_t *dmask;        // device bit matrix of a masked dimension longer than 128
+    int dmask_words;
     const int *lens;              // device, valid length per batch entry, or nullptr
 };
 
@@ -122,7 +124,8 @@ hop_simt_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__res
                 s *= a.scale;
                 bool valid = key < exist && t < exist && (!a.causal || key <= t) &&
                              (a.window == 0 || (key > t - a.window && key < t + a.window));
-                if (a.masked) valid = valid && ((hop_mask.bits[t][key >> 5] >> (key & 31)) & 1u);
+                if (a.masked == 1) valid = valid && ((hop_mask.bits[t][key >> 5] >> (key & 31)) & 1u);
+                if (a.masked == 2) valid = valid && ((__ldg(a.dmask + (size_t)t * a.dmask_words + (key >> 5)) >> (key & 31)) & 1u);
                 s = valid ? s : -INFINITY;
                 // a block may hold no visible key of this row (window): keep the arithmetic finite
                 const float m_new = fmaxf(m[r], warp_max(s));
@@ -182,14 +185,20 @@ int launch_t(const Problem &pb, const HopDesc &hd, const void *xin, int xin_head
     a.rope_log2_base = pb.rope_base > 0.f ? log2f(pb.rope_base) : 0.f;
     a.window = pb.window[hd.hop];
     a.masked = 0;
+    a.dmask = nullptr;
+    a.dmask_words = 0;
     a.lens = pb.seq_lens;
     HopMask hm;
-    if (pb.masks[hd.hop]) {
+    memset(&hm, 0, sizeof(hm));
+    if (pb.masks[hd.hop] && hd.n > 128) {
+        if (!pb.dmask[hd.hop]) return TA_ERR_INVALID_ARG;
+        a.masked = 2;                                  // bit matrix in device memory
+        a.dmask = pb.dmask[hd.hop];
+        a.dmask_words = pb.dmask_words[hd.hop];
+    } else if (pb.masks[hd.hop]) {
         const int rc = build_hop_mask(pb, hd, &hm);   // explicit mask ^ causal flag ^ window
         if (rc != TA_OK) return rc;
         a.masked = 1;
-    } else {
-        memset(&hm, 0, sizeof(hm));
     }
     size_t smem = sizeof(float) * ((size_t)BQ * pb.D + 2 * (size_t)BK * (pb.D + 1));
     auto kern = hop_simt_kernel<T, DPL>;
@@ -216,6 +225,7 @@ int launch_d(const Problem &pb, const HopDesc &hd, const void *xin, int xin_head
 }  // namespace
 
 int launch_hop_simt(const Problem &pb, const HopDesc &hd, const void *xin, int xin_heads, void *xout) {
+    if (xin == xout) return TA_ERR_INVALID_ARG;   // CTAs read rows other CTAs write: never in place
     if (pb.dtype == TA_DTYPE_F32) return launch_d<float>(pb, hd, xin, xin_heads, xout);
     return launch_d<__nv_bfloat16>(pb, hd, xin, xin_heads, xout);
 }

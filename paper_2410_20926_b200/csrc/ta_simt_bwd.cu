@@ -14,7 +14,8 @@
 //       query heads of the GQA group and their query blocks, A = exp(s - lse), and accumulates
 //       G_in (per query head; summed over the group into dV for the first hop) and dK (summed
 //       over the group) without atomics, so the result is reproducible.
-// Masks as in the forward: causal flag, window, explicit mask (n <= 128), valid lengths.
+// Masks as in the forward: causal flag, window, explicit mask (a kernel parameter up to n = 128, a bit
+// matrix in device memory beyond), valid lengths.
 #include <cuda_bf16.h>
 
 #include <string.h>
@@ -38,7 +39,9 @@ struct SimtBwdArgs {
     long long items;
     float scale;
     float rope_log2_base;         // 0: no positional encoding
-    int window, masked;
+    int window, masked;           // masked: 1 = HopMask parameter (n <= 128), 2 = device bit matrix dmask
+    const uint32_t *dmask;
+    int dmask_words;
     const int *lens;
     int first_hop, accumulate;
 };
@@ -53,7 +56,8 @@ __device__ __forceinline__ int segment_exist(const SimtBwdArgs &a, int b, long l
 __device__ __forceinline__ bool pair_visible(const SimtBwdArgs &a, const HopMask &hm, int t, int key, int exist) {
     bool v = key < exist && t < exist && (!a.causal || key <= t) &&
              (a.window == 0 || (key > t - a.window && key < t + a.window));
-    if (a.masked) v = v && ((hm.bits[t][key >> 5] >> (key & 31)) & 1u);
+    if (a.masked == 1) v = v && ((hm.bits[t][key >> 5] >> (key & 31)) & 1u);
+    if (a.masked == 2 && v) v = ((__ldg(a.dmask + (size_t)t * a.dmask_words + (key >> 5)) >> (key & 31)) & 1u) != 0;
     return v;
 }
 
@@ -423,13 +427,19 @@ int launch_dpl(const Problem &pb, const HopDesc &hd, const void *x, int x_heads,
     a.lens = pb.seq_lens;
     a.first_hop = first_hop ? 1 : 0;
     a.accumulate = accumulate ? 1 : 0;
+    a.dmask = nullptr;
+    a.dmask_words = 0;
     HopMask hm;
-    if (pb.masks[hd.hop]) {
+    memset(&hm, 0, sizeof(hm));
+    if (pb.masks[hd.hop] && hd.n > 128) {
+        if (!pb.dmask[hd.hop]) return TA_ERR_INVALID_ARG;
+        a.masked = 2;
+        a.dmask = pb.dmask[hd.hop];
+        a.dmask_words = pb.dmask_words[hd.hop];
+    } else if (pb.masks[hd.hop]) {
         const int rc = build_hop_mask(pb, hd, &hm);
         if (rc != TA_OK) return rc;
         a.masked = 1;
-    } else {
-        memset(&hm, 0, sizeof(hm));
     }
     const size_t smem = sizeof(float) * (2 * (size_t)BR * pb.D + 2 * (size_t)BL * (pb.D + 1));
     auto kq = hop_simt_bwd_q_kernel<T, DPL>;

@@ -579,16 +579,20 @@ __global__ void f32_to_bf16_kernel(const float *__restrict__ src, __nv_bfloat16 
 }
 
 // dv[b, kvh] = sum over the group's query heads of dout[b, h]  (no real hop: out = broadcast v)
-template <typename TO>
-__global__ void group_sum_kernel(const __nv_bfloat16 *__restrict__ dout, TO *__restrict__ dv, long long per_head,
-                                 int H, int H_kv, long long total_kv) {
+template <typename TI, typename TO>
+__global__ void group_sum_kernel(const TI *__restrict__ dout, TO *__restrict__ dv, long long per_head, int H, int H_kv,
+                                 long long total_kv) {
     const int g = H / H_kv;
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total_kv;
          i += (long long)gridDim.x * blockDim.x) {
         const long long bkv = i / per_head, rr = i % per_head;
         const long long b = bkv / H_kv, kvh = bkv % H_kv;
         float s = 0.f;
-        for (int j = 0; j < g; ++j) s += __bfloat162float(dout[((b * H + kvh * g + j) * per_head) + rr]);
+        for (int j = 0; j < g; ++j) {
+            const TI x = dout[((b * H + kvh * g + j) * per_head) + rr];
+            if constexpr (sizeof(TI) == 4) s += x;
+            else s += __bfloat162float(x);
+        }
         if constexpr (sizeof(TO) == 4) dv[i] = s;
         else dv[i] = __float2bfloat16_rn(s);
     }
@@ -672,15 +676,21 @@ int launch_f32_to_bf16(const float *src, void *dst, long long n, cudaStream_t st
     return launch_kernel(f32_to_bf16_kernel, (unsigned)blocks, 256, 0, stream, false, src, (__nv_bfloat16 *)dst, n);
 }
 
-int launch_group_sum(const void *dout, void *dv, int dv_is_f32, int B, int H, int H_kv, long long per_head,
-                     cudaStream_t stream) {
+int launch_group_sum(const void *dout, int dout_is_f32, void *dv, int dv_is_f32, int B, int H, int H_kv,
+                     long long per_head, cudaStream_t stream) {
     const long long total = (long long)B * H_kv * per_head;
     long long blocks = (total + 255) / 256;
     if (blocks > 148 * 32) blocks = 148 * 32;
+    const unsigned grid = (unsigned)blocks;
+    if (dout_is_f32) {
+        if (!dv_is_f32) return TA_ERR_UNSUPPORTED;     // fp32 tensors take fp32 gradients
+        return launch_kernel(group_sum_kernel<float, float>, grid, 256, 0, stream, false, (const float *)dout, (float *)dv,
+                             per_head, H, H_kv, total);
+    }
     if (dv_is_f32)
-        return launch_kernel(group_sum_kernel<float>, (unsigned)blocks, 256, 0, stream, false, (const __nv_bfloat16 *)dout,
-                             (float *)dv, per_head, H, H_kv, total);
-    return launch_kernel(group_sum_kernel<__nv_bfloat16>, (unsigned)blocks, 256, 0, stream, false,
+        return launch_kernel(group_sum_kernel<__nv_bfloat16, float>, grid, 256, 0, stream, false,
+                             (const __nv_bfloat16 *)dout, (float *)dv, per_head, H, H_kv, total);
+    return launch_kernel(group_sum_kernel<__nv_bfloat16, __nv_bfloat16>, grid, 256, 0, stream, false,
                          (const __nv_bfloat16 *)dout, (__nv_bfloat16 *)dv, per_head, H, H_kv, total);
 }
 

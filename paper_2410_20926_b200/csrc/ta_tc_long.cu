@@ -50,6 +50,10 @@ struct LongArgs {
     // with respect to the hop's output, laid out like q
     float2 *stats;
     const __nv_bfloat16 *stats_g;
+    // explicit mask of the dimension (kWindow variant only): bit matrix [n][mask_words] with the causal
+    // flag and the window folded in, then per query block of 128 the range of key blocks it sees
+    const uint32_t *mask_bits;
+    int mask_words;
 };
 
 template <int D>
@@ -106,6 +110,17 @@ __device__ __forceinline__ LongItem decode_long_item(const LongArgs &a, long lon
         const long long left = (len - first_token + a.stride - 1) / a.stride;
         c.exist = len <= first_token ? 0 : (int)(left < a.n ? left : a.n);
     }
+    int mask_lo = 0, mask_hi = 0;
+    if (a.mask_bits != nullptr) {
+        // (one range for the pair: the two tiles walk the same key blocks, as they do without a mask)
+        const int *range = reinterpret_cast<const int *>(a.mask_bits + (size_t)a.n * a.mask_words) + 2 * (c.t0 / kTileRows);
+        mask_lo = __ldg(range);
+        mask_hi = __ldg(range + 1);
+        if (c.ntiles == 2) {
+            mask_lo = min(mask_lo, __ldg(range + 2));
+            mask_hi = max(mask_hi, __ldg(range + 3));
+        }
+    }
 #pragma unroll
     for (int i = 0; i < 2; ++i) {
         const int t0 = c.t0 + i * kTileRows;
@@ -117,6 +132,11 @@ __device__ __forceinline__ LongItem decode_long_item(const LongArgs &a, long lon
             if (!a.causal) keys_end = min(a.n, t0 + kTileRows - 1 + a.window);
         }
         c.j0[i] = first / kTileRows;
+        if (a.mask_bits != nullptr) {
+            // key blocks before the first / after the last one the mask lets the item's query blocks see
+            c.j0[i] = max(c.j0[i], mask_lo);
+            keys_end = min(keys_end, mask_hi * kTileRows);
+        }
         // padding keys are not visited, except that every tile keeps one block (its rows then see
         // nothing in it and come out as zeros), so that no role ever meets an empty chain
         keys_end = max(min(keys_end, c.exist), c.j0[i] * kTileRows + 1);
@@ -124,6 +144,9 @@ __device__ __forceinline__ LongItem decode_long_item(const LongArgs &a, long lon
         c.je[i] = (keys_end + kTileRows - 1) / kTileRows;
     }
     if (c.ntiles == 1) { c.j0[1] = c.je[1] = c.je[0]; }            // an absent tile has no blocks
+    // no key block between the two tiles' ranges may be left to neither of them (the producer loads
+    // the whole union): the second tile then walks such blocks too, seeing nothing in them
+    if (c.ntiles == 2 && c.j0[1] > c.je[0]) c.j0[1] = c.je[0];
     c.jlo = c.j0[0];
     c.jhi = max(c.je[0], c.je[1]);
     return c;
@@ -373,6 +396,11 @@ hop_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     }
                     c_hi = t < c.exist ? min(c_hi, c.exist - u0) : 0;     // valid length: padding keys, padding rows
                 }
+                // explicit mask: this row's 128 bits over the block's keys (all ones without a mask)
+                uint4 mrow = make_uint4(~0u, ~0u, ~0u, ~0u);
+                if (kWindow && a.mask_bits != nullptr && row_valid)
+                    mrow = __ldg(reinterpret_cast<const uint4 *>(a.mask_bits + (size_t)t * a.mask_words + 4 * j));
+                auto mask_word = [&](int cc) { return cc == 0 ? mrow.x : (cc == 1 ? mrow.y : (cc == 2 ? mrow.z : mrow.w)); };
                 const int nchunks = (keys + 31) >> 5;
 
                 ok = mbar_wait_abortable(s_full(ch), blocks_seen & 1, 0xF4, abort_flag);
@@ -403,9 +431,11 @@ hop_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     for (int cc = 0; cc < nchunks; ++cc) {
                         if (32 * cc >= w_hi) continue;      // warp-uniform
                         tmem_ld32(s_col + 32 * cc, v);
+                        const uint32_t mw = kWindow ? mask_word(cc) : ~0u;
 #pragma unroll
                         for (int jj = 0; jj < 32; ++jj)
-                            if (32 * cc + jj >= c_lo && 32 * cc + jj < c_hi) bm = fmaxf(bm, __uint_as_float(v[jj]));
+                            if (32 * cc + jj >= c_lo && 32 * cc + jj < c_hi && ((mw >> jj) & 1u))
+                                bm = fmaxf(bm, __uint_as_float(v[jj]));
                     }
                 }
                 // (with a window a row may see nothing in a block: the running maximum then stays -inf
@@ -457,13 +487,14 @@ hop_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                         uint32_t pk[16];
                         if (32 * cc < w_hi) {
                             tmem_ld32(s_col + 32 * cc, v);
+                            const uint32_t mw = kWindow ? mask_word(cc) : ~0u;
 #pragma unroll
                             for (int jj = 0; jj < 32; jj += 2) {
                                 const int col = 32 * cc + jj;
                                 float p0 = fast_exp2(__uint_as_float(v[jj]) * a.scale_log2 - m_ref);
                                 float p1 = fast_exp2(__uint_as_float(v[jj + 1]) * a.scale_log2 - m_ref);
-                                p0 = (col >= c_lo && col < c_hi) ? p0 : 0.f;
-                                p1 = (col + 1 >= c_lo && col + 1 < c_hi) ? p1 : 0.f;
+                                p0 = (col >= c_lo && col < c_hi && ((mw >> jj) & 1u)) ? p0 : 0.f;
+                                p1 = (col + 1 >= c_lo && col + 1 < c_hi && ((mw >> (jj + 1)) & 1u)) ? p1 : 0.f;
                                 const uint32_t w = pack_bf16x2(p0, p1);
                                 pk[jj >> 1] = w;
                                 sum += __uint_as_float(w << 16) + __uint_as_float(w & 0xFFFF0000u);
@@ -575,6 +606,9 @@ int launch_long_d(const Problem &pb, const HopDesc &hd, const void *xin, int xin
     a.pair_major = 2ull * pb.B * pb.H_kv * pb.N * D * 2 <= (96ull << 20) ? 1 : 0;
     a.stats = (float2 *)stats;
     a.stats_g = (const __nv_bfloat16 *)stats_g;
+    a.mask_bits = pb.masks[hd.hop] ? pb.dmask[hd.hop] : nullptr;
+    a.mask_words = pb.dmask_words[hd.hop];
+    if (pb.masks[hd.hop] && !a.mask_bits) return TA_ERR_INVALID_ARG;
 
     int dev = 0;
     const int num_sms = current_device_sms(&dev);
@@ -589,7 +623,7 @@ int launch_long_d(const Problem &pb, const HopDesc &hd, const void *xin, int xin
         configured.mark(dev);
     }
     const unsigned grid = (unsigned)(a.total_items < num_sms ? a.total_items : num_sms);
-    if (a.window > 0 || a.lens != nullptr)
+    if (a.window > 0 || a.lens != nullptr || a.mask_bits != nullptr)
         return launch_kernel(hop_long_kernel<D, true>, grid, kThreads, smem, pb.stream, false, mq, mk, mxi,
                              (__nv_bfloat16 *)xout, a);
     return launch_kernel(hop_long_kernel<D, false>, grid, kThreads, smem, pb.stream, false, mq, mk, mxi,

@@ -18,12 +18,15 @@
 // value tensor out once for the two hops.
 //
 // Correctness does not depend on the cache: a B item waits on a counter in global memory that the
-// A items of its unit (and head chunk) increment after their TMA stores have completed.  A items
-// never wait on other CTAs, and every B item only waits for items earlier in the sequence, which
-// are dealt round robin to a grid launched cooperatively (all CTAs resident), so the waits end;
-// they are bounded all the same.  The per-tile pipeline (TMA producer, MMA issuer, two softmax /
+// A items of its unit (and head chunk) increment after their TMA stores have completed.  The CTAs
+// claim the items of the sequence in order from a grid-wide counter (whichever CTA is ready takes
+// the next one), so a B item only ever waits for items that were claimed earlier, by CTAs that are
+// running, and A items wait for nobody: every wait ends, whatever the number of CTAs resident.
+// The waits are bounded all the same.  The per-tile pipeline (TMA producer, MMA issuer, two softmax /
 // epilogue warpgroups, store warp; S, P and O in tensor memory) is the one of the one-hop kernel.
 #include <cuda_bf16.h>
+
+#include <cstdlib>
 
 #include "ta_internal.h"
 #include "ta_ptx.cuh"
@@ -47,8 +50,8 @@ struct PairCfg {
     static constexpr uint32_t kOffQ = kOffK + kNK * kTileBytes;
     static constexpr uint32_t kOffX = kOffQ + kNQ * kTileBytes;
     static constexpr uint32_t kOffBar = kOffX + kNX * kTileBytes;
-    static constexpr int kNumBars = 2 * kNK + 2 * kNQ + 3 * kNX + 6;
-    static constexpr uint32_t kSmemBytes = kOffBar + kNumBars * 8 + 16 + 1024 /*alignment slack*/;
+    static constexpr int kNumBars = 2 * kNK + 2 * kNQ + 3 * kNX + 6 + 16 /*item ring*/;
+    static constexpr uint32_t kSmemBytes = kOffBar + kNumBars * 8 + 16 + 16 * 4 + 1024 /*alignment slack*/;
     static constexpr uint32_t kTmemCols = 512;                 // S x 2 (P over S), O x 2
     static constexpr uint32_t kColS = 0, kColO = 256;
 };
@@ -71,6 +74,7 @@ struct PairArgs {
     uint32_t flag_target;   // hop-A tiles per (unit, head chunk) = ph[0].tiles_inner * gi
     float scale_log2;
     unsigned int *flags;    // [units * hsplit] completion counters, zero when the kernel starts
+    unsigned int *next_pos; // next unclaimed position of the sequence, zero when the kernel starts
 };
 
 struct PairItem {
@@ -177,6 +181,9 @@ __device__ __forceinline__ RowConst row_const(const PhaseArgs &p, int causal, in
 }
 
 // ----------------------------------------------------------------------------- the kernel
+constexpr int kRing = 16;                    // item ring: far more than the items a CTA has in flight
+constexpr uint32_t kNoItem = 0xFFFFFFFFu;
+
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 hop_pair_kernel(const __grid_constant__ CUtensorMap map_qa, const __grid_constant__ CUtensorMap map_ka,
@@ -205,8 +212,10 @@ hop_pair_kernel(const __grid_constant__ CUtensorMap map_qa, const __grid_constan
     auto s_full = [&](int i) { return bar0 + 8u * (uint32_t)(kB1 + i); };
     auto o_full = [&](int i) { return bar0 + 8u * (uint32_t)(kB1 + 2 + i); };
     auto p_full = [&](int i) { return bar0 + 8u * (uint32_t)(kB1 + 4 + i); };
+    auto item_full = [&](int i) { return bar0 + 8u * (uint32_t)(kB1 + 6 + i); };
     uint32_t *tmem_slot = (uint32_t *)(smem + C::kOffBar + C::kNumBars * 8);
     volatile uint32_t *abort_flag = tmem_slot + 1;
+    volatile uint32_t *item_pos = tmem_slot + 2;      // [kRing] sequence positions claimed by this CTA
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
@@ -218,6 +227,7 @@ hop_pair_kernel(const __grid_constant__ CUtensorMap map_qa, const __grid_constan
         for (int i = 0; i < kNQ; ++i) { mbar_init(q_full(i), 1); mbar_init(q_free(i), 1); }
         for (int i = 0; i < kNX; ++i) { mbar_init(x_full(i), 1); mbar_init(x_free(i), 1); mbar_init(out_full(i), 4); }
         for (int i = 0; i < 2; ++i) { mbar_init(s_full(i), 1); mbar_init(o_full(i), 1); mbar_init(p_full(i), 4); }
+        for (int i = 0; i < kRing; ++i) mbar_init(item_full(i), 1);
         *abort_flag = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -235,12 +245,15 @@ hop_pair_kernel(const __grid_constant__ CUtensorMap map_qa, const __grid_constan
     const uint32_t tmem_base = *tmem_slot;
     if (tid == 0) griddep_launch_dependents();
 
-    // items of this CTA: sequence positions blockIdx.x, + gridDim.x, ...; gi tiles (heads) each
-    const uint32_t my_items = a.total > blockIdx.x ? (a.total - blockIdx.x + gridDim.x - 1) / gridDim.x : 0u;
-    const uint32_t T = my_items * (uint32_t)a.gi;
+    // The CTA's it-th item: the position the K/Q producer claimed for it from the grid-wide counter
+    // (kNoItem when the sequence is exhausted or the CTA is shutting down).
+    auto item_of = [&](uint32_t it, uint32_t where) -> uint32_t {
+        if (!mbar_wait_abortable(item_full(it % kRing), (it / kRing) & 1, where, abort_flag)) return kNoItem;
+        return item_pos[it % kRing];
+    };
 
     if (warp == 0) {
-        // =============================================================== TMA producer: K and Q tiles
+        // =============================================================== claims items; TMA producer of K and Q
         // (inputs of the call: never wait for another CTA, so they run ahead of the value tiles)
         if (lane == 0) {
             uint32_t t = 0;
@@ -250,8 +263,14 @@ hop_pair_kernel(const __grid_constant__ CUtensorMap map_qa, const __grid_constan
                 last_par = parity ? (last_par | bit) : (last_par & ~bit);
             };
             bool ok = true;
-            for (uint32_t it = 0; ok && it < my_items; ++it) {
-                const PairItem c = decode_pos(a, blockIdx.x + it * gridDim.x);
+            for (uint32_t it = 0; ok; ++it) {
+                // Items are claimed in sequence order by whichever CTA is ready for one: a B item
+                // only ever waits for items claimed before it, by CTAs that are running.
+                const uint32_t pos = atomicAdd(a.next_pos, 1u);
+                item_pos[it % kRing] = pos < a.total ? pos : kNoItem;
+                mbar_arrive(item_full(it % kRing));
+                if (pos >= a.total) break;
+                const PairItem c = decode_pos(a, pos);
                 const uint32_t slab_tx = (uint32_t)a.ph[c.phase].rows * 128u;
                 const CUtensorMap *mk = c.phase ? &map_kb : &map_ka;
                 const CUtensorMap *mq = c.phase ? &map_qb : &map_qa;
@@ -295,8 +314,10 @@ hop_pair_kernel(const __grid_constant__ CUtensorMap map_qa, const __grid_constan
             uint32_t armed = 0, last_par = 0;
             bool ok = true;
             bool prev_hop_done = false;   // the value tensor may be the previous kernel's output
-            for (uint32_t it = 0; ok && it < my_items; ++it) {
-                const PairItem c = decode_pos(a, blockIdx.x + it * gridDim.x);
+            for (uint32_t it = 0; ok; ++it) {
+                const uint32_t pos = item_of(it, 0x14);
+                if (pos == kNoItem) break;
+                const PairItem c = decode_pos(a, pos);
                 const PhaseArgs &ph = a.ph[c.phase];
                 const uint32_t slab_tx = (uint32_t)ph.rows * 128u;
                 const CUtensorMap *mx = c.phase ? &map_xb : &map_xin_a;
@@ -336,7 +357,7 @@ hop_pair_kernel(const __grid_constant__ CUtensorMap map_qa, const __grid_constan
     } else if (warp == 1) {
         // =============================================================== MMA issuer
         // S(t) = Q K^T one tile ahead of O(t-1) = P X.  K and Q come from a producer of their own
-        // that runs two tiles ahead, so the wait for Q(t) is short and does not hold back O(t-1).
+        // that runs ahead of the value tiles, so the wait for Q(t) is short and does not hold back O(t-1).
         if (lane == 0) {
             constexpr uint32_t idesc_s = instr_desc(128, 0);
             bool ok = true;
@@ -355,39 +376,38 @@ hop_pair_kernel(const __grid_constant__ CUtensorMap map_qa, const __grid_constan
                 tc_commit(o_full(u & 1));
                 return true;
             };
-            uint32_t it = 0, j = 0;
+            uint32_t t = 0;
             int kblocks = 0, kblocks_prev = 0;      // key blocks of 16 rows of tile t / tile t-1
             int f16 = 0, f16_prev = 0;              // type of their value tile
-            for (uint32_t t = 0; ok && t < T; ++t) {
-                const int ks = it & 1, qs = t % kNQ;
-                kblocks_prev = kblocks;
-                f16_prev = f16;
-                if (j == 0) {
-                    const PhaseArgs &ph = a.ph[phase_of(a, blockIdx.x + it * gridDim.x)];
+            for (uint32_t it = 0; ok; ++it) {
+                const uint32_t pos = item_of(it, 0x26);
+                if (pos == kNoItem) break;
+                const PhaseArgs &ph = a.ph[phase_of(a, pos)];
+                const int ks = it & 1;
+                for (int j = 0; ok && j < a.gi; ++j, ++t) {
+                    const int qs = t % kNQ;
+                    kblocks_prev = kblocks;
+                    f16_prev = f16;
                     kblocks = (ph.rows + 15) >> 4;
                     f16 = ph.x_f16;
-                    ok = mbar_wait_abortable(k_full(ks), (it >> 1) & 1, 0x23, abort_flag);
-                }
-                if (ok) ok = mbar_wait_abortable(q_full(qs), (t / kNQ) & 1, 0x24, abort_flag);
-                if (!ok) break;
-                tc_fence_after();
-                const uint32_t q_base = sQ + qs * kTileBytes, k_base = sK + ks * kTileBytes;
+                    if (j == 0) ok = mbar_wait_abortable(k_full(ks), (it >> 1) & 1, 0x23, abort_flag);
+                    if (ok) ok = mbar_wait_abortable(q_full(qs), (t / kNQ) & 1, 0x24, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t q_base = sQ + qs * kTileBytes, k_base = sK + ks * kTileBytes;
 #pragma unroll
-                for (int kb = 0; kb < D / 16; ++kb) {
-                    const uint32_t off = (kb >> 2) * kSlabBytes + (kb & 3) * 32;
-                    tc_mma_ss(tmem_base + C::kColS + (t & 1) * 128, smem_desc_sw128(q_base + off, 16, 1024),
-                              smem_desc_sw128(k_base + off, 16, 1024), idesc_s, kb > 0);
+                    for (int kb = 0; kb < D / 16; ++kb) {
+                        const uint32_t off = (kb >> 2) * kSlabBytes + (kb & 3) * 32;
+                        tc_mma_ss(tmem_base + C::kColS + (t & 1) * 128, smem_desc_sw128(q_base + off, 16, 1024),
+                                  smem_desc_sw128(k_base + off, 16, 1024), idesc_s, kb > 0);
+                    }
+                    tc_commit(s_full(t & 1));
+                    tc_commit(q_free(qs));
+                    if (j == a.gi - 1) tc_commit(k_free(ks));
+                    if (t > 0) ok = issue_o(t - 1, kblocks_prev, f16_prev);
                 }
-                tc_commit(s_full(t & 1));
-                tc_commit(q_free(qs));
-                if (++j == (uint32_t)a.gi) {
-                    tc_commit(k_free(ks));
-                    j = 0;
-                    ++it;
-                }
-                if (t > 0) ok = issue_o(t - 1, kblocks_prev, f16_prev);
             }
-            if (ok && T > 0) issue_o(T - 1, kblocks, f16);
+            if (ok && t > 0) issue_o(t - 1, kblocks, f16);
         }
     } else if (warp == 2 || warp == 12) {
         // =============================================================== TMA store
@@ -399,8 +419,10 @@ hop_pair_kernel(const __grid_constant__ CUtensorMap map_qa, const __grid_constan
             const uint32_t mine = warp == 2 ? 0u : 1u;
             uint32_t t = 0;
             bool ok = true;
-            for (uint32_t it = 0; ok && it < my_items; ++it) {
-                const PairItem c = decode_pos(a, blockIdx.x + it * gridDim.x);
+            for (uint32_t it = 0; ok; ++it) {
+                const uint32_t pos = item_of(it, 0x31);
+                if (pos == kNoItem) break;
+                const PairItem c = decode_pos(a, pos);
                 const CUtensorMap *mo = c.phase ? &map_xb : &map_xout_a;
                 for (int j = 0; j < a.gi; ++j, ++t) {
                     if ((t & 1u) != mine) continue;
@@ -432,97 +454,104 @@ hop_pair_kernel(const __grid_constant__ CUtensorMap map_qa, const __grid_constan
         const uint32_t s_col = tmem_lane + C::kColS + b * 128, o_col = tmem_lane + C::kColO + b * 128;
 
         bool ok = true;
-        for (uint32_t t = b; t < T; t += 2) {
-            const uint32_t par = (t >> 1) & 1;
-            const int phase = phase_of(a, blockIdx.x + (t / (uint32_t)a.gi) * gridDim.x);
+        uint32_t t = 0;
+        for (uint32_t it = 0; ok; ++it) {
+            uint32_t pos = item_of(it, 0x43);
+            pos = __shfl_sync(0xffffffffu, pos, 0);     // one answer per warp (the aligned TMEM ops need it converged)
+            if (pos == kNoItem) break;
+            const int phase = phase_of(a, pos);
             const int c_lo = phase ? rc1.c_lo : rc0.c_lo, c_hi = phase ? rc1.c_hi : rc0.c_hi;
             const int w_lo = phase ? rc1.w_lo : rc0.w_lo, w_hi = phase ? rc1.w_hi : rc0.w_hi;
             const int nchunks = phase ? rc1.nchunks : rc0.nchunks;
             const bool row_valid = (phase ? rc1.row_valid : rc0.row_valid) != 0;
             const bool warp_valid = (phase ? rc1.warp_valid : rc0.warp_valid) != 0;
             const bool x_f16 = a.ph[phase].x_f16 != 0, out_f16 = a.ph[phase].out_f16 != 0;
-            ok = mbar_wait_abortable(s_full(b), par, 0x40, abort_flag);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            tc_fence_after();
+            for (int j = 0; ok && j < a.gi; ++j, ++t) {
+                if ((t & 1u) != (uint32_t)b) continue;
+                const uint32_t par = (t >> 1) & 1;
+                ok = mbar_wait_abortable(s_full(b), par, 0x40, abort_flag);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                tc_fence_after();
 
-            float m = -INFINITY;
-            uint32_t v[32];
+                float m = -INFINITY;
+                uint32_t v[32];
 #pragma unroll 1
-            for (int c = 0; c < nchunks; ++c) {
-                if (!(warp_valid && 32 * c < w_hi && 32 * c + 32 > w_lo)) continue;   // warp-uniform
-                tmem_ld32(s_col + 32 * c, v);
-#pragma unroll
-                for (int jj = 0; jj < 32; ++jj) {
-                    const int col = 32 * c + jj;
-                    if (col >= c_lo && col < c_hi) m = fmaxf(m, __uint_as_float(v[jj]));
-                }
-            }
-            const float m_scaled = row_valid ? m * a.scale_log2 : 0.f;
-            float sum = 0.f;
-#pragma unroll 1
-            for (int c = 0; c < nchunks; ++c) {
-                uint32_t pk[16];
-                if (warp_valid && 32 * c < w_hi && 32 * c + 32 > w_lo) {
+                for (int c = 0; c < nchunks; ++c) {
+                    if (!(warp_valid && 32 * c < w_hi && 32 * c + 32 > w_lo)) continue;   // warp-uniform
                     tmem_ld32(s_col + 32 * c, v);
 #pragma unroll
-                    for (int jj = 0; jj < 32; jj += 2) {
+                    for (int jj = 0; jj < 32; ++jj) {
                         const int col = 32 * c + jj;
-                        float p0 = fast_exp2(__uint_as_float(v[jj]) * a.scale_log2 - m_scaled);
-                        float p1 = fast_exp2(__uint_as_float(v[jj + 1]) * a.scale_log2 - m_scaled);
-                        p0 = (row_valid && col >= c_lo && col < c_hi) ? p0 : 0.f;
-                        p1 = (row_valid && col + 1 >= c_lo && col + 1 < c_hi) ? p1 : 0.f;
-                        uint32_t w;
-                        if (x_f16) {            // uniform: the weights take the type of the value tile
-                            w = pack_f16x2(p0, p1);
-                            sum += sum_f16x2(w);
-                        } else {
-                            w = pack_bf16x2(p0, p1);
-                            sum += __uint_as_float(w << 16) + __uint_as_float(w & 0xFFFF0000u);
-                        }
-                        pk[jj >> 1] = w;
+                        if (col >= c_lo && col < c_hi) m = fmaxf(m, __uint_as_float(v[jj]));
                     }
-                } else {
-#pragma unroll
-                    for (int jj = 0; jj < 16; ++jj) pk[jj] = 0u;
                 }
-                tmem_st16(s_col + 16 * c, pk);
-            }
-            tmem_st_wait();
-            const float inv = row_valid ? 1.f / sum : 1.f;
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(p_full(b));
-
-            const int xs = t % kNX;
-            ok = mbar_wait_abortable(o_full(b), par, 0x42, abort_flag);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            tc_fence_after();
-            if (warp_valid) {
-                const uint32_t x_row = sX + xs * kTileBytes + (uint32_t)r * 128u;
+                const float m_scaled = row_valid ? m * a.scale_log2 : 0.f;
+                float sum = 0.f;
 #pragma unroll 1
-                for (int c = 0; c < D / 32; ++c) {
-                    tmem_ld32(o_col + 32 * c, v);
+                for (int c = 0; c < nchunks; ++c) {
                     uint32_t pk[16];
+                    if (warp_valid && 32 * c < w_hi && 32 * c + 32 > w_lo) {
+                        tmem_ld32(s_col + 32 * c, v);
 #pragma unroll
-                    for (int jj = 0; jj < 32; jj += 2)
-                        pk[jj >> 1] = out_f16 ? pack_f16x2(__uint_as_float(v[jj]) * inv, __uint_as_float(v[jj + 1]) * inv)
-                                              : pack_bf16x2(__uint_as_float(v[jj]) * inv, __uint_as_float(v[jj + 1]) * inv);
-                    const uint32_t slab = x_row + (uint32_t)(c >> 1) * kSlabBytes;
-                    if (row_valid) {
+                        for (int jj = 0; jj < 32; jj += 2) {
+                            const int col = 32 * c + jj;
+                            float p0 = fast_exp2(__uint_as_float(v[jj]) * a.scale_log2 - m_scaled);
+                            float p1 = fast_exp2(__uint_as_float(v[jj + 1]) * a.scale_log2 - m_scaled);
+                            p0 = (row_valid && col >= c_lo && col < c_hi) ? p0 : 0.f;
+                            p1 = (row_valid && col + 1 >= c_lo && col + 1 < c_hi) ? p1 : 0.f;
+                            uint32_t w;
+                            if (x_f16) {            // uniform: the weights take the type of the value tile
+                                w = pack_f16x2(p0, p1);
+                                sum += sum_f16x2(w);
+                            } else {
+                                w = pack_bf16x2(p0, p1);
+                                sum += __uint_as_float(w << 16) + __uint_as_float(w & 0xFFFF0000u);
+                            }
+                            pk[jj >> 1] = w;
+                        }
+                    } else {
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            const uint32_t chunk = (uint32_t)(((c & 1) * 4 + i) ^ (r & 7));
-                            st_shared_v4(slab + chunk * 16, pk[4 * i], pk[4 * i + 1], pk[4 * i + 2], pk[4 * i + 3]);
+                        for (int jj = 0; jj < 16; ++jj) pk[jj] = 0u;
+                    }
+                    tmem_st16(s_col + 16 * c, pk);
+                }
+                tmem_st_wait();
+                const float inv = row_valid ? 1.f / sum : 1.f;
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(p_full(b));
+
+                const int xs = t % kNX;
+                ok = mbar_wait_abortable(o_full(b), par, 0x42, abort_flag);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                tc_fence_after();
+                if (warp_valid) {
+                    const uint32_t x_row = sX + xs * kTileBytes + (uint32_t)r * 128u;
+#pragma unroll 1
+                    for (int c = 0; c < D / 32; ++c) {
+                        tmem_ld32(o_col + 32 * c, v);
+                        uint32_t pk[16];
+#pragma unroll
+                        for (int jj = 0; jj < 32; jj += 2)
+                            pk[jj >> 1] = out_f16 ? pack_f16x2(__uint_as_float(v[jj]) * inv, __uint_as_float(v[jj + 1]) * inv)
+                                                  : pack_bf16x2(__uint_as_float(v[jj]) * inv, __uint_as_float(v[jj + 1]) * inv);
+                        const uint32_t slab = x_row + (uint32_t)(c >> 1) * kSlabBytes;
+                        if (row_valid) {
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                const uint32_t chunk = (uint32_t)(((c & 1) * 4 + i) ^ (r & 7));
+                                st_shared_v4(slab + chunk * 16, pk[4 * i], pk[4 * i + 1], pk[4 * i + 2], pk[4 * i + 3]);
+                            }
                         }
                     }
                 }
+                fence_proxy_async_smem();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(out_full(xs));
             }
-            fence_proxy_async_smem();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(out_full(xs));
         }
     }
 
@@ -574,6 +603,7 @@ int launch_pair_d(const Problem &pb, const HopDesc &ha, const HopDesc &hb, const
     a.flag_target = (uint32_t)ha.tiles_inner * (uint32_t)a.gi;
     a.scale_log2 = pb.scale * 1.4426950408889634f;
     a.flags = flags;
+    a.next_pos = flags + (size_t)geo.units * geo.hsplit;
 
     constexpr size_t smem = PairCfg<D>::kSmemBytes;
     auto kern = hop_pair_kernel<D>;
@@ -583,25 +613,12 @@ int launch_pair_d(const Problem &pb, const HopDesc &ha, const HopDesc &hb, const
             return TA_ERR_CUDA;
         configured.mark(dev);
     }
-    // B items spin on counters other CTAs increment: every CTA must be resident, which a
-    // cooperative launch guarantees (the grid never exceeds one CTA per SM).
+    // Completion counters and the claim counter start at zero.  No CTA ever waits for an item that
+    // is not already claimed by a running CTA, so the grid needs no co-residency guarantee.
     const unsigned grid = (unsigned)(a.total < (uint32_t)num_sms ? a.total : (uint32_t)num_sms);
-    cudaError_t e = cudaMemsetAsync(flags, 0, geo.flag_bytes, pb.stream);
+    const cudaError_t e = cudaMemsetAsync(flags, 0, geo.flag_bytes, pb.stream);
     if (e != cudaSuccess) return cuda_fail(e);
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(grid);
-    cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = pb.stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeCooperative;
-    attr[0].val.cooperative = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    e = cudaLaunchKernelEx(&cfg, kern, mqa, mka, mxia, mxoa, mqb, mkb, mxb, a);
-    if (e != cudaSuccess) return cuda_fail(e);
-    count_launch();
-    return TA_OK;
+    return launch_kernel(kern, grid, kThreads, smem, pb.stream, false, mqa, mka, mxia, mxoa, mqb, mkb, mxb, a);
 }
 
 }  // namespace
@@ -627,16 +644,22 @@ bool pair_geometry(int B, int H, int H_kv, const HopDesc &ha, const HopDesc &hb,
     geo->items_b = (uint32_t)ib;
     geo->units = (uint32_t)units;
     geo->total = (uint32_t)total;
-    // B(u) follows A(u) by about four rounds of the grid: a tile's store is complete in global
-    // memory (and its counter incremented) three to four tile times after its loads were issued,
-    // and the value-tile producer of a B item asks for the counter about three tiles before the
-    // item is computed.  Shorter distances stall the B items on their counters (measured: half the
-    // distance costs 10-25 %), longer ones push the window out of the L2.
-    long long lag = (4ll * num_sms + (ia + ib) - 1) / (ia + ib);
+    // B(u) follows A(u) by about one and a half times as many items as there are CTAs.  The CTAs
+    // hold that many consecutive items in flight (one being computed, the next ones prefetched), and
+    // an A item's counter is incremented only when its last store has completed, so a B item that
+    // follows its A items more closely finds them unfinished and stalls its CTA (measured at 32k
+    // tokens: a third of this distance doubles the time).  A longer distance pushes the rows out of
+    // the L2 before the B items read them.
+    long long lag = (3ll * num_sms / 2 + (ia + ib) - 1) / (ia + ib);
+    // Tuning knob for measurements: TA_PAIR_LAG_UNITS=<n> in the environment overrides the distance.
+    if (const char *env = getenv("TA_PAIR_LAG_UNITS")) {
+        const long long v = atoll(env);
+        if (v >= 1) lag = v;
+    }
     if (lag < 1) lag = 1;
     if (lag > units) lag = units;
     geo->lag = (uint32_t)lag;
-    geo->flag_bytes = (size_t)units * geo->hsplit * sizeof(unsigned int);
+    geo->flag_bytes = ((size_t)units * geo->hsplit + 1) * sizeof(unsigned int);   // counters + the claim counter
     // bytes touched between A(u) and B(u): Q, K, value in and out of `lag` units
     const double unit_bytes = (double)ha.n * ha.stride * 128.0 /*D<=128 bf16 upper bound*/ * 2.0 * (3.0 * g + 1.0);
     geo->window_bytes = unit_bytes * (double)lag;

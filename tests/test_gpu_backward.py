@@ -132,6 +132,21 @@ def test_backward_all_unit_dims():
     np.testing.assert_allclose(dv, ref, atol=1e-6)
 
 
+def test_backward_all_unit_dims_fp32_storage():
+    """The forward takes fp32 tensors whose dimensions are all 1 (out = v broadcast); so does the backward."""
+    import torch
+    B, H, Hkv, D = 2, 4, 2, 32
+    inp = ta_inputs.make_inputs(B, H, Hkv, 1, D, "f32", 305, with_dout=True)
+    q, k, v, do = (to_device(inp, n, "f32") for n in ("q", "k", "v", "dout"))
+    dq, dk, dv = (torch.full_like(t, float("nan")) for t in (q, k, v))
+    ta.ta_backward_ex(do, q, k, v, dq, dk, dv, B, H, Hkv, 1, D, [1, 1], True, dtype=ta.TA_DTYPE_F32,
+                      grad_dtype=ta.TA_DTYPE_F32, workspace=None, workspace_bytes=0)
+    torch.cuda.synchronize()
+    assert (dq == 0).all() and (dk == 0).all()
+    ref = inp["dout"].reshape(B, Hkv, H // Hkv, 1, D).sum(axis=2)
+    np.testing.assert_allclose(dv.cpu().numpy(), ref, atol=1e-6)
+
+
 def test_backward_with_saved_hops_matches_recompute():
     import torch
     B, H, Hkv, D, dims = 1, 4, 2, 128, [8, 8, 16]

@@ -108,11 +108,16 @@ def test_mask_argument_checks():
     assert rc == ta.TA_ERR_INVALID_ARG
     rc = ta.ta_forward_ex(x, x, x, out, 1, 2, 2, 64, 64, [8, 8], False, hop_masks=[upper, None], check=False)
     assert rc == ta.TA_OK
-    # explicit masks are limited to segments of at most 128 positions
+    # longer dimensions take masks too; an empty row is caught on the host there as well
     y = torch.zeros(1, 2, 256, 64, dtype=torch.bfloat16, device="cuda")
-    rc = ta.ta_forward_ex(y, y, y, torch.empty_like(y), 1, 2, 2, 256, 64, [256], True,
+    o = torch.empty((1, 2, 256, 64), dtype=torch.bfloat16, device="cuda")
+    rc = ta.ta_forward_ex(y, y, y, o, 1, 2, 2, 256, 64, [256], True,
                           hop_masks=[np.tril(np.ones((256, 256), np.uint8))], check=False)
-    assert rc == ta.TA_ERR_UNSUPPORTED
+    assert rc == ta.TA_OK
+    bad = np.ones((256, 256), np.uint8)
+    bad[200, :] = 0
+    rc = ta.ta_forward_ex(y, y, y, o, 1, 2, 2, 256, 64, [256], True, hop_masks=[bad], check=False)
+    assert rc == ta.TA_ERR_INVALID_ARG
     with pytest.raises(ValueError):
         ta.ta_forward_ex(x, x, x, out, 1, 2, 2, 64, 64, [8, 8], False, hop_masks=[np.ones((4, 4))])
 
@@ -134,6 +139,81 @@ def test_backward_with_masks(dims, D, causal, skip, rope):
                           rope_base=rope or None)
     for name, g, r in zip(("dq", "dk", "dv"), got, ref):
         assert_grad_close(g, r, name, True, sum(1 for n in dims if n > 1), rope=bool(rope))
+
+
+def block_sparse_mask(n, bs, rng, density=0.4):
+    nb = (n + bs - 1) // bs
+    blocks = rng.random((nb, nb)) < density
+    blocks |= np.eye(nb, dtype=bool)
+    return np.kron(blocks, np.ones((bs, bs), dtype=np.uint8))[:n, :n].astype(np.uint8)
+
+
+def lambda_mask(n, sinks, local):
+    t, u = np.arange(n)[:, None], np.arange(n)[None, :]
+    return ((u < sinks) | ((u <= t) & (u > t - local))).astype(np.uint8)
+
+
+@pytest.mark.parametrize("dims,D,causal,kind", [
+    ([200], 64, True, "random"),              # one ragged second key block
+    ([200], 128, False, "lambda"),
+    ([1024], 128, True, "lambda"),            # sink keys + local band: the middle key blocks are empty
+    ([1024], 64, False, "block"),             # block-sparse layout of 64 x 64 blocks
+    ([1024], 128, True, "band"),              # banded: leading key blocks of a query block are skipped
+    ([3, 200], 128, True, "random"),          # short (kernel-parameter mask) and long (bit matrix) hop
+    ([260, 2], 64, False, "block"),           # long hop over a strided dimension
+])
+def test_masks_on_long_segments(dims, D, causal, kind):
+    """Explicit masks on dimensions longer than 128: bit matrix in device memory, tensor-core forward."""
+    B, H, Hkv = 2, 4, 2
+    N = math.prod(dims)
+    rng = np.random.default_rng(19)
+    masks = []
+    for n in dims:
+        if kind == "random":
+            m = (rng.random((n, n)) < 0.5).astype(np.uint8)
+            m[np.arange(n), np.arange(n)] = 1
+        elif kind == "lambda":
+            m = lambda_mask(n, 4, 48)
+        elif kind == "block":
+            m = block_sparse_mask(n, 64 if n > 128 else 1, rng)
+        else:
+            t, u = np.arange(n)[:, None], np.arange(n)[None, :]
+            m = (np.abs(t - u) < 150).astype(np.uint8)
+        masks.append(m)
+    assert "tc-long" in ta.ta_plan_describe(B, H, Hkv, N, D, dims, causal, ta.TA_DTYPE_BF16, 0)
+    inp = ta_inputs.make_inputs(B, H, Hkv, N, D, "bf16", 711)
+    got = gpu_forward(inp, B, H, Hkv, N, D, dims, causal, "bf16", hop_masks=masks)
+    ref = oracle.forward(inp["q"], inp["k"], inp["v"], dims, causal, masks=masks)
+    assert_close(got, ref, "bf16")
+    assert np.abs(ref - oracle.forward(inp["q"], inp["k"], inp["v"], dims, causal)).max() > 0.05
+    # the generic kernel reads the same bit matrix
+    got = gpu_forward(inp, B, H, Hkv, N, D, dims, causal, "bf16", ta.TA_FLAG_NO_TENSOR_CORE, hop_masks=masks)
+    assert_close(got, ref, "bf16")
+
+
+@pytest.mark.parametrize("dims,D,causal,kind", [
+    ([200], 64, True, "random"),
+    ([1024], 128, True, "lambda"),
+    ([3, 200], 128, False, "random"),
+])
+def test_backward_with_masks_on_long_segments(dims, D, causal, kind):
+    B, H, Hkv = 1, 4, 2
+    N = math.prod(dims)
+    rng = np.random.default_rng(20)
+    masks = []
+    for n in dims:
+        if kind == "lambda":
+            m = lambda_mask(n, 4, 48)
+        else:
+            m = (rng.random((n, n)) < 0.5).astype(np.uint8)
+            m[np.arange(n), np.arange(n)] = 1
+        masks.append(m)
+    inp = ta_inputs.make_inputs(B, H, Hkv, N, D, "bf16", 712, with_dout=True)
+    ref = oracle.backward(inp["dout"], inp["q"], inp["k"], inp["v"], dims, causal, masks=masks)
+    for grad_f32 in (True, False):
+        got = gpu_backward(inp, B, H, Hkv, N, D, dims, causal, grad_f32, hop_masks=masks)
+        for name, g, r in zip(("dq", "dk", "dv"), got, ref):
+            assert_grad_close(g, r, name, grad_f32, sum(1 for n in dims if n > 1))
 
 
 def test_masks_llama_shape_sampled_heads():

@@ -284,13 +284,15 @@ def test_overlapped_hop_launches_give_identical_results(B, H, Hkv, D, dims, caus
 
 
 def test_concurrent_host_threads_and_streams():
-    """Four host threads, each with its own stream and problem, call the library at the same time
+    """Six host threads, each with its own stream and problem, call the library at the same time
     and repeatedly; every result must equal the one the same problem gives when run alone."""
     import threading
 
     import torch
+    # (three of them need a scratch tensor of the same size, which each call takes for itself)
     cases = [(1, 4, 2, 128, [8, 16, 32], True), (2, 4, 4, 64, [16, 4, 4, 4], False),
-             (1, 2, 1, 128, [2, 300], True), (1, 8, 2, 128, [32, 32], True)]
+             (1, 2, 1, 128, [2, 300], True), (1, 8, 2, 128, [32, 32], True),
+             (1, 2, 1, 128, [300, 2], True), (1, 2, 2, 128, [2, 300], False)]
     work = []
     for i, (B, H, Hkv, D, dims, causal) in enumerate(cases):
         N = math.prod(dims)

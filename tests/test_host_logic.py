@@ -126,7 +126,7 @@ def test_plan_intermediates_and_pair_launches():
     _, hops = parse_plan(ta.ta_plan_describe(1, 32, 8, 32768, 128, dims, True,
                                              flags=ta.TA_FLAG_PAIR_HOPS | ta.TA_FLAG_NO_HOP_FUSION))
     assert all("pair" not in h for h in hops)
-    assert ta.ta_workspace_bytes(1, 32, 8, 32768, 128, dims, ta.TA_DTYPE_BF16) == 8 * 32 * 4
+    assert ta.ta_workspace_bytes(1, 32, 8, 32768, 128, dims, ta.TA_DTYPE_BF16) == 8 * 32 * 4 + 256
 
 
 def test_plan_skips_unit_dims_and_routes_generic_hops():

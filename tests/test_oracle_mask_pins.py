@@ -149,6 +149,57 @@ def test_zero_queries_average_the_masked_set():
         np.testing.assert_allclose(got[t], v[0, 0, m[t]].mean(axis=0), atol=1e-14)
 
 
+def block_sparse_mask(n, bs, rng, density=0.4):
+    """A block-sparse layout: visibility decided per bs x bs block, diagonal blocks kept."""
+    nb = (n + bs - 1) // bs
+    blocks = rng.random((nb, nb)) < density
+    blocks |= np.eye(nb, dtype=bool)
+    return np.kron(blocks, np.ones((bs, bs), dtype=bool))[:n, :n]
+
+
+def lambda_mask(n, sinks, local):
+    """The "Lambda" shape: the first `sinks` keys are always visible, plus the last `local` ones."""
+    t, u = np.arange(n)[:, None], np.arange(n)[None, :]
+    return (u < sinks) | ((u <= t) & (u > t - local))
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_block_sparse_and_lambda_masks_match_dense_route(causal):
+    """Structured masks of the kinds the paper names (block-sparse, global + local): the C route
+    against the dense route, which builds its N x N boolean mask from coordinates."""
+    rng = np.random.default_rng(70)
+    dims = [6, 10]
+    N = 60
+    masks = [block_sparse_mask(6, 2, rng), lambda_mask(10, 2, 3)]
+    q, k, v = rnd((1, 2, N, 5), 71), rnd((1, 1, N, 5), 72), rnd((1, 1, N, 5), 73)
+    a = oracle.forward(q, k, v, dims, causal, masks=masks)
+    b = oracle.forward_dense(q, k, v, dims, causal, masks=masks)
+    np.testing.assert_allclose(a, b, rtol=0, atol=1e-13)
+    assert np.abs(a - oracle.forward(q, k, v, dims, causal)).max() > 1e-2
+
+
+def test_lambda_mask_with_zero_queries_is_a_closed_form():
+    """q = 0 under the Lambda mask: row t is the mean of the sink keys and its local band."""
+    n, sinks, local = 12, 2, 3
+    v = rnd((1, 1, n, 3), 74)
+    got = oracle.forward(np.zeros((1, 1, n, 3)), rnd((1, 1, n, 3), 75), v, [n], True,
+                         masks=[lambda_mask(n, sinks, local)])[0, 0]
+    for t in range(n):
+        keys = sorted(set(range(min(sinks, t + 1))) | set(range(max(0, t - local + 1), t + 1)))
+        np.testing.assert_allclose(got[t], v[0, 0, keys].mean(axis=0), atol=1e-14)
+
+
+def test_block_diagonal_mask_splits_the_dimension():
+    """A block-diagonal mask over one dimension = independent attentions over its blocks."""
+    n, bs = 12, 4
+    q, k, v = rnd((1, 2, n, 4), 76), rnd((1, 2, n, 4), 77), rnd((1, 2, n, 4), 78)
+    m = np.kron(np.eye(n // bs, dtype=bool), np.ones((bs, bs), dtype=bool))
+    got = oracle.forward(q, k, v, [n], False, masks=[m])
+    ref = np.concatenate([oracle.forward(q[:, :, i:i + bs], k[:, :, i:i + bs], v[:, :, i:i + bs], [bs], False)
+                          for i in range(0, n, bs)], axis=2)
+    np.testing.assert_allclose(got, ref, atol=1e-14)
+
+
 def test_mask_with_an_empty_row_is_rejected():
     m = np.ones((4, 4), dtype=bool)
     m[2] = False
