@@ -375,7 +375,56 @@ hop_tc_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 tc_fence_after();
 
                 // ---- softmax and its derivative for this thread's row; P -> X slot, dS -> its slot
-                {
+                const int cc_lo = w_lo >> 5, cc_hi = (max(w_hi, w_lo + 1) - 1) >> 5;
+                if (warp_valid && cc_lo == cc_hi) {
+                    // Every key this warp's rows can see lies in ONE 32-column chunk (segments of at
+                    // most 32 positions aligned to the chunks: the usual case): the scores and dP are
+                    // read from tensor memory once and the weights stay in registers between the passes.
+                    const int cc = cc_lo;
+                    uint32_t vs[32], vd[32];
+                    tmem_ld32(tmem_lane + C::kColS + 32 * cc, vs);
+                    tmem_ld32(tmem_lane + C::kColDP + 32 * cc, vd);
+                    float m = -INFINITY;
+#pragma unroll
+                    for (int jj = 0; jj < 32; ++jj)
+                        if (visible(cc, jj)) m = fmaxf(m, __uint_as_float(vs[jj]));
+                    const float m_s = (row_valid && !(kMask && m == -INFINITY)) ? m * a.scale_log2 : 0.f;
+                    float l = 0.f, dot = 0.f;
+#pragma unroll
+                    for (int jj = 0; jj < 32; ++jj) {
+                        float p = fast_exp2(__uint_as_float(vs[jj]) * a.scale_log2 - m_s);
+                        p = visible(cc, jj) ? p : 0.f;
+                        vs[jj] = __float_as_uint(p);                   // un-normalised weight
+                        l += p;
+                        dot += p * __uint_as_float(vd[jj]);            // p is 0 where the key is invisible
+                    }
+                    const float inv_l = (row_valid && !(kMask && l == 0.f)) ? 1.f / l : 0.f;
+                    const float delta = dot * inv_l;
+                    const uint32_t rowP = sXP + (uint32_t)r * 128u, rowS = sdS + (uint32_t)r * 128u;
+#pragma unroll 1
+                    for (int c4 = 0; c4 < 4; ++c4) {
+                        uint32_t pp[16], ps[16];
+                        if (c4 == cc) {
+#pragma unroll
+                            for (int jj = 0; jj < 32; jj += 2) {
+                                const float p0 = __uint_as_float(vs[jj]) * inv_l, p1 = __uint_as_float(vs[jj + 1]) * inv_l;
+                                pp[jj >> 1] = pack_bf16x2(p0, p1);
+                                ps[jj >> 1] = pack_bf16x2(p0 * (__uint_as_float(vd[jj]) - delta) * a.scale,
+                                                          p1 * (__uint_as_float(vd[jj + 1]) - delta) * a.scale);
+                            }
+                        } else {
+#pragma unroll
+                            for (int jj = 0; jj < 16; ++jj) { pp[jj] = 0u; ps[jj] = 0u; }
+                        }
+                        const uint32_t slab = (uint32_t)(c4 >> 1) * kSlabBytes;
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const uint32_t chunk = (uint32_t)(((c4 & 1) * 4 + i) ^ (r & 7)) * 16;
+                            st_shared_v4(rowP + slab + chunk, pp[4 * i], pp[4 * i + 1], pp[4 * i + 2], pp[4 * i + 3]);
+                            st_shared_v4(rowS + slab + chunk, ps[4 * i], ps[4 * i + 1], ps[4 * i + 2], ps[4 * i + 3]);
+                        }
+                    }
+                } else {
                     uint32_t vs[32], vd[32];
                     float m = -INFINITY;
 #pragma unroll 1
