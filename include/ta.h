@@ -84,7 +84,10 @@ enum {
     TA_FLAG_BF16_INTERMEDIATES = 1u << 5, /* store the value tensor between hops as bf16.  By default,  */
                                       /* between two tensor-core hops (n_i <= 128) of one call it is    */
                                       /* stored in `out` as fp16 -- same bytes, three more mantissa     */
-                                      /* bits -- and only the last hop rounds to bf16.  Implied by      */
+                                      /* bits -- and only the last hop rounds to bf16.  Every value of  */
+                                      /* that tensor is a convex combination of entries of v, so fp16   */
+                                      /* is safe while |v| <= 65504 (and entries below 6e-8 flush to 0); */
+                                      /* set this flag for inputs outside that range.  Implied by       */
                                       /* TA_FLAG_SAVE_HOPS (the backward reads the hop inputs as bf16). */
     TA_FLAG_PAIR_HOPS = 1u << 4       /* run two adjacent tensor-core hops whose common block is too    */
                                       /* large for one SM as ONE launch in which the second hop's tiles */
