@@ -157,6 +157,8 @@ typedef struct ta_params {
     const int *window;     /* host, ndims ints, or NULL: per-hop sliding window, see below     */
     const unsigned char *const *hop_masks; /* host, ndims pointers, or NULL: explicit M_i, see below */
     const int *seq_lens;   /* DEVICE, B ints, or NULL: valid length per batch entry, see below  */
+    int masks_per_head;    /* 0: hop_masks[i] is one n_i x n_i matrix for every head;            */
+                           /* 1: H matrices, one per query head ([H][n_i][n_i] bytes)            */
     ta_stream_t stream;
 } ta_params;
 
@@ -194,8 +196,11 @@ typedef struct ta_params {
  * a bit matrix (n_i * n_i / 8 bytes) in pooled device memory, copied in stream order from pageable
  * memory (such a call cannot be captured in a CUDA graph), the tensor-core kernel skips the key
  * blocks before the first and after the last one a block of 128 queries sees and tests one bit
- * per score in between, and the backward of such a hop runs on the generic kernels.  Hops are not
- * fused when a mask is given.  ta_backward_ex takes the same.
+ * per score in between, and the backward of such a hop runs on the generic kernels.  With
+ * masks_per_head = 1 every non-NULL hop_masks[i] holds H matrices, one per query head (heads of a
+ * GQA group may then see different keys; their dK, dV contributions are summed as always); such
+ * masks travel as bit matrices in device memory whatever n_i is.  Hops are not fused when a mask
+ * is given.  ta_backward_ex takes the same.
  *
  * Valid lengths (padding to prod(dims), batches of different lengths; a mask M_i that depends
  * on the segment): with seq_lens != NULL only the tokens of batch entry b with flat index
@@ -258,6 +263,7 @@ typedef struct ta_bwd_params {
     const int *window;            /* host, ndims ints, or NULL: sliding windows as in ta_forward_ex */
     const unsigned char *const *hop_masks; /* host, ndims pointers, or NULL: explicit masks, as in ta_forward_ex */
     const int *seq_lens;          /* DEVICE, B ints, or NULL: valid lengths, as in ta_forward_ex */
+    int masks_per_head;           /* as in ta_forward_ex                                        */
     const void *saved_hops;       /* X_1..X_{m-1} as written by ta_forward_ex(TA_FLAG_SAVE_HOPS) */
                                   /* (the part of its workspace after the scratch tensor), or    */
                                   /* NULL: recomputed                                          */

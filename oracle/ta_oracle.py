@@ -125,8 +125,9 @@ def _cwindow(window, m):
     return (ctypes.c_int * m)(*w)
 
 
-def _cmasks(masks, dims):
-    """Per-dimension masks as a C array of byte-matrix pointers; returns (array or None, keep-alive)."""
+def _cmasks(masks, dims, head=None, heads=None):
+    """Per-dimension masks as a C array of byte-matrix pointers; returns (array or None, keep-alive).
+    An entry may be n x n (every head) or H x n x n (one matrix per query head: `head` picks it)."""
     if masks is None:
         return None, None
     if len(masks) != len(dims):
@@ -136,12 +137,21 @@ def _cmasks(masks, dims):
         if mk is None:
             ptrs.append(None)
             continue
-        a = np.ascontiguousarray(np.asarray(mk) != 0, dtype=np.uint8)
+        a = np.asarray(mk) != 0
+        if a.ndim == 3:
+            if heads is not None and a.shape[0] != heads:
+                raise ValueError("a per-head mask needs one n x n matrix per query head")
+            a = a[0 if head is None else head]
+        a = np.ascontiguousarray(a, dtype=np.uint8)
         if a.shape != (n, n):
             raise ValueError("mask of a dimension of extent n must be n x n")
         keep.append(a)
         ptrs.append(a.ctypes.data)
     return (ctypes.c_void_p * len(dims))(*ptrs), keep
+
+
+def _per_head(masks) -> bool:
+    return masks is not None and any(mk is not None and np.asarray(mk).ndim == 3 for mk in masks)
 
 
 def _clens(seq_lens, B, N):
@@ -184,7 +194,8 @@ def forward(q, k, v, dims, causal: bool, scale: float | None = None, heads=None,
     window: None, or one int per dimension: w_i > 0 keeps, in hop i, only keys within w_i
     positions of the query along dimension i (|t - u| < w_i); 0 = no window.
     masks: None, or one entry per dimension: None or an n_i x n_i array (row = query position,
-    column = key position, non-zero = visible) applied on top of `causal` and `window`.
+    column = key position, non-zero = visible) applied on top of `causal` and `window`; an
+    H x n_i x n_i array gives every query head a matrix of its own.
     seq_lens: None, or one valid length per batch entry: tokens with flat index >= seq_lens[b]
     are padding (never visible as keys; their output rows are 0).
     Returns out [B,H,N,D] fp64 (and, with return_xs, the list of per-head [m+1,N,D]
@@ -195,7 +206,8 @@ def forward(q, k, v, dims, causal: bool, scale: float | None = None, heads=None,
     scale = 1.0 / math.sqrt(D) if scale is None else float(scale)
     cdims = (ctypes.c_int * len(dims))(*dims)
     cwin = _cwindow(window, len(dims))
-    cmask, _keep = _cmasks(masks, dims)
+    cmask, _keep = _cmasks(masks, dims, heads=H)
+    per_head = _per_head(masks)
     lens = _clens(seq_lens, B, N)
     pairs = [(b, h) for b in range(B) for h in range(H)] if heads is None else list(heads)
     out = np.empty((len(pairs), N, D), dtype=np.float64)
@@ -204,6 +216,8 @@ def forward(q, k, v, dims, causal: bool, scale: float | None = None, heads=None,
     for idx, (b, h) in enumerate(pairs):
         qh, kh, vh = _f64(q[b, h]), _f64(k[b, h // g]), _f64(v[b, h // g])
         xs = np.empty((len(dims) + 1, N, D), dtype=np.float64) if return_xs else None
+        if per_head:
+            cmask, _keep = _cmasks(masks, dims, head=h, heads=H)
         rc = _fwd_head(lib, qh, kh, vh, out[idx], N, D, cdims, len(dims), causal, scale,
                        rope_base, xs, cwin, cmask, None if lens is None else lens[b])
         if rc != 0:
@@ -228,7 +242,8 @@ def backward(dout, q, k, v, dims, causal: bool, scale: float | None = None, grou
     scale = 1.0 / math.sqrt(D) if scale is None else float(scale)
     cdims = (ctypes.c_int * len(dims))(*dims)
     cwin = _cwindow(window, len(dims))
-    cmask, _keep = _cmasks(masks, dims)
+    cmask, _keep = _cmasks(masks, dims, heads=H)
+    per_head = _per_head(masks)
     lens = _clens(seq_lens, B, N)
     sel = [(b, kv) for b in range(B) for kv in range(Hkv)] if groups is None else list(groups)
     dq = np.zeros((len(sel), g, N, D))
@@ -240,6 +255,8 @@ def backward(dout, q, k, v, dims, causal: bool, scale: float | None = None, grou
         for j in range(g):
             h = kv * g + j
             qh = _f64(q[b, h])
+            if per_head:
+                cmask, _keep = _cmasks(masks, dims, head=h, heads=H)
             o = np.empty((N, D))
             xs = np.empty((len(dims) + 1, N, D))
             rc = _fwd_head(lib, qh, kh, vh, o, N, D, cdims, len(dims), causal, scale, rope_base, xs, cwin, cmask,
@@ -357,7 +374,9 @@ def forward_dense(q, k, v, dims, causal: bool, scale: float | None = None,
     out = np.empty((B, H, N, D))
     for b in range(B):
         for h in range(H):
-            a = dense_effective_matrix(q[b, h], k[b, h // g], dims, causal, scale, rope_base, window, masks,
+            masks_h = masks if masks is None else [mk if mk is None or np.asarray(mk).ndim == 2 else np.asarray(mk)[h]
+                                                   for mk in masks]          # a head's own matrix, if per head
+            a = dense_effective_matrix(q[b, h], k[b, h // g], dims, causal, scale, rope_base, window, masks_h,
                                        None if seq_lens is None else seq_lens[b])
             out[b, h] = a @ np.asarray(v[b, h // g], dtype=np.float64)
     return out

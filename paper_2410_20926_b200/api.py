@@ -54,6 +54,7 @@ class ta_params(ctypes.Structure):
                 ("window", ctypes.POINTER(ctypes.c_int)),
                 ("hop_masks", ctypes.POINTER(ctypes.c_void_p)),
                 ("seq_lens", ctypes.c_void_p),
+                ("masks_per_head", ctypes.c_int),
                 ("stream", ctypes.c_void_p)]
 
 
@@ -70,6 +71,7 @@ class ta_bwd_params(ctypes.Structure):
                 ("window", ctypes.POINTER(ctypes.c_int)),
                 ("hop_masks", ctypes.POINTER(ctypes.c_void_p)),
                 ("seq_lens", ctypes.c_void_p),
+                ("masks_per_head", ctypes.c_int),
                 ("saved_hops", ctypes.c_void_p),
                 ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
                 ("stream", ctypes.c_void_p)]
@@ -206,30 +208,36 @@ def _window(window, nd):
     return (ctypes.c_int * nd)(*w)
 
 
-def _hop_masks(hop_masks, dims):
+def _hop_masks(hop_masks, dims, H=None):
     """Per-dimension explicit masks M_i as a C array of host pointers (None stays NULL).
 
     `hop_masks` has one entry per dimension: None (no explicit mask for that hop) or an n_i x n_i
-    array whose non-zero entries mark the visible (query position, key position) pairs.  Returns
-    (pointer array, buffers to keep alive until the call returns).
+    array whose non-zero entries mark the visible (query position, key position) pairs -- or, for
+    every masked dimension alike, an H x n_i x n_i array with one matrix per query head.  Returns
+    (pointer array, buffers to keep alive until the call returns, masks_per_head flag).
     """
     if hop_masks is None:
-        return None, None
+        return None, None, 0
     import numpy as np
     dims = [int(x) for x in dims]
     if len(hop_masks) != len(dims):
         raise ValueError("hop_masks needs one entry per dimension")
     keep, arr = [], (ctypes.c_void_p * len(dims))()
+    ranks = {np.asarray(m).ndim for m in hop_masks if m is not None}
+    if len(ranks) > 1:
+        raise ValueError("hop_masks: either every mask is n x n or every mask is H x n x n")
+    per_head = int(ranks == {3})
     for i, (m, n) in enumerate(zip(hop_masks, dims)):
         if m is None:
             arr[i] = None
             continue
         m8 = np.ascontiguousarray((np.asarray(m) != 0).astype(np.uint8))
-        if m8.shape != (n, n):
-            raise ValueError(f"hop_masks[{i}] must have shape ({n}, {n})")
+        want = (H, n, n) if per_head else (n, n)
+        if m8.shape != want:
+            raise ValueError(f"hop_masks[{i}] must have shape {want}")
         keep.append(m8)
         arr[i] = m8.ctypes.data
-    return arr, keep
+    return arr, keep, per_head
 
 
 def ta_forward_ex(q, k, v, out, B, H, H_kv, N, D, dims, causal, dtype=TA_DTYPE_BF16,
@@ -249,7 +257,7 @@ def ta_forward_ex(q, k, v, out, B, H, H_kv, N, D, dims, causal, dtype=TA_DTYPE_B
     win = _window(window, nd)          # kept alive until the call returns
     if win is not None:
         p.window = win
-    masks, _keep = _hop_masks(hop_masks, dims)
+    masks, _keep, p.masks_per_head = _hop_masks(hop_masks, dims, H)
     if masks is not None:
         p.hop_masks = masks
     p.seq_lens = _ptr(seq_lens)        # device int32 tensor [B] or None
@@ -282,7 +290,7 @@ def ta_backward_ex(dout, q, k, v, dq, dk, dv, B, H, H_kv, N, D, dims, causal,
     win = _window(window, nd)
     if win is not None:
         p.window = win
-    masks, _keep = _hop_masks(hop_masks, dims)
+    masks, _keep, p.masks_per_head = _hop_masks(hop_masks, dims, H)
     if masks is not None:
         p.hop_masks = masks
     p.seq_lens = _ptr(seq_lens)

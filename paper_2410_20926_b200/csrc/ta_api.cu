@@ -220,12 +220,14 @@ int build_hop_mask(const Problem &pb, const HopDesc &hd, HopMask *hm) {
 
 int upload_long_masks(Problem *pb, const Plan &plan, void **pooled) {
     *pooled = nullptr;
+    const int mh = pb->masks_per_head ? pb->H : 1;              // matrices per masked dimension
+    auto on_device = [&](const HopDesc &h) { return h.nf <= 1 && pb->masks[h.hop] && (h.n > 128 || pb->masks_per_head); };
     size_t total_words = 0;
     for (int j = 0; j < plan.nhops; ++j) {
         const HopDesc &h = plan.hops[j];
-        if (h.nf > 1 || !pb->masks[h.hop] || h.n <= 128) continue;
+        if (!on_device(h)) continue;
         const size_t words = (size_t)((h.n + 127) / 128) * 4, qblocks = (size_t)(h.n + 127) / 128;
-        total_words += (size_t)h.n * words + 2 * qblocks;
+        total_words += (size_t)mh * ((size_t)h.n * words + 2 * qblocks);
         total_words = (total_words + 3) & ~(size_t)3;
     }
     if (total_words == 0) return TA_OK;
@@ -235,29 +237,33 @@ int upload_long_masks(Problem *pb, const Plan &plan, void **pooled) {
     size_t off = 0;
     for (int j = 0; j < plan.nhops; ++j) {
         const HopDesc &h = plan.hops[j];
-        if (h.nf > 1 || !pb->masks[h.hop] || h.n <= 128) continue;
+        if (!on_device(h)) continue;
         const int n = h.n, words = ((n + 127) / 128) * 4, qblocks = (n + 127) / 128;
-        const unsigned char *m = pb->masks[h.hop];
         const int w = pb->window[h.hop];
-        uint32_t *bits = host.data() + off;
-        int *ranges = (int *)(bits + (size_t)n * words);
-        for (int qb = 0; qb < qblocks; ++qb) { ranges[2 * qb] = qblocks; ranges[2 * qb + 1] = 0; }
-        for (int t = 0; t < n; ++t) {
-            bool any = false;
-            for (int u = 0; u < n; ++u) {
-                if (pb->causal && u > t) break;
-                if (w > 0 && (t - u >= w || u - t >= w)) continue;
-                if (!m[(size_t)t * n + u]) continue;
-                bits[(size_t)t * words + (u >> 5)] |= 1u << (u & 31);
-                any = true;
-                int &lo = ranges[2 * (t / 128)], &hi = ranges[2 * (t / 128) + 1];
-                if (u / 128 < lo) lo = u / 128;
-                if (u / 128 + 1 > hi) hi = u / 128 + 1;
+        uint32_t *bits0 = host.data() + off;
+        int *ranges0 = (int *)(bits0 + (size_t)mh * n * words);
+        for (int hh = 0; hh < mh; ++hh) {
+            const unsigned char *m = pb->masks[h.hop] + (size_t)hh * n * n;
+            uint32_t *bits = bits0 + (size_t)hh * n * words;
+            int *ranges = ranges0 + (size_t)hh * 2 * qblocks;
+            for (int qb = 0; qb < qblocks; ++qb) { ranges[2 * qb] = qblocks; ranges[2 * qb + 1] = 0; }
+            for (int t = 0; t < n; ++t) {
+                bool any = false;
+                for (int u = 0; u < n; ++u) {
+                    if (pb->causal && u > t) break;
+                    if (w > 0 && (t - u >= w || u - t >= w)) continue;
+                    if (!m[(size_t)t * n + u]) continue;
+                    bits[(size_t)t * words + (u >> 5)] |= 1u << (u & 31);
+                    any = true;
+                    int &lo = ranges[2 * (t / 128)], &hi = ranges[2 * (t / 128) + 1];
+                    if (u / 128 < lo) lo = u / 128;
+                    if (u / 128 + 1 > hi) hi = u / 128 + 1;
+                }
+                if (!any) return TA_ERR_INVALID_ARG;
             }
-            if (!any) return TA_ERR_INVALID_ARG;
         }
         placed.push_back({h.hop, off, words});
-        off += (size_t)n * words + 2 * (size_t)qblocks;
+        off += (size_t)mh * ((size_t)n * words + 2 * (size_t)qblocks);
         off = (off + 3) & ~(size_t)3;
     }
     void *dev = nullptr;
@@ -285,7 +291,7 @@ int take_masks(Problem *pb, const Plan &plan, const int *window, const unsigned 
     // every masked hop is checked before anything is launched
     for (int j = 0; j < plan.nhops; ++j) {
         const HopDesc &h = plan.hops[j];
-        if (h.nf > 1 || !pb->masks[h.hop] || h.n > 128) continue;   // longer dimensions: upload_long_masks
+        if (h.nf > 1 || !pb->masks[h.hop] || h.n > 128 || pb->masks_per_head) continue;   // those: upload_long_masks
         HopMask hm;
         const int rc = build_hop_mask(*pb, h, &hm);
         if (rc != TA_OK) return rc;
@@ -489,6 +495,7 @@ static int forward_impl(const ta_params &p) {
     pb.scale = p.softmax_scale != 0.f ? p.softmax_scale : 1.0f / sqrtf((float)p.D);
     pb.rope_base = p.rope_base;
     pb.seq_lens = p.seq_lens;
+    pb.masks_per_head = (any_mask && p.masks_per_head) ? 1 : 0;
     pb.pdl = 0;
     if ((rc = take_masks(&pb, plan, p.window, p.hop_masks, p.ndims)) != TA_OK) return rc;
     pb.flags = p.flags; pb.hop_begin = p.hop_begin; pb.hop_end = p.hop_end;

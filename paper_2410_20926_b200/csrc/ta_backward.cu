@@ -100,6 +100,7 @@ int backward_impl(const ta_bwd_params &p) {
     pb.scale = p.softmax_scale != 0.f ? p.softmax_scale : 1.0f / sqrtf((float)p.D);
     pb.rope_base = p.rope_base;
     pb.seq_lens = p.seq_lens;
+    pb.masks_per_head = (p.hop_masks && p.masks_per_head) ? 1 : 0;
     pb.pdl = 0;
     pb.causal = p.causal ? 1 : 0;
     if ((rc = take_masks(&pb, plan, p.window, p.hop_masks, p.ndims)) != TA_OK) return rc;

@@ -82,6 +82,9 @@ struct Problem {
     // any of its rows sees: 2 ints per block.  NULL for the other dimensions.
     const uint32_t *dmask[TA_MAX_DIMS];
     int dmask_words[TA_MAX_DIMS];
+    // 1: every given mask holds one matrix per query head ([H][n][n] bytes on the host; the device
+    // copy then holds H bit matrices, followed by H tables of key-block ranges), whatever n is
+    int masks_per_head;
     int pdl;   // 1: this launch follows a hop kernel of the same call in the stream and may overlap its tail
     unsigned flags;
     int hop_begin, hop_end;
@@ -105,9 +108,10 @@ struct HopMask {
 int build_hop_mask(const Problem &pb, const HopDesc &hd, HopMask *hm);
 // Host: sets pb.window / pb.masks from the caller's arrays and checks them against the plan.
 int take_masks(Problem *pb, const Plan &plan, const int *window, const unsigned char *const *hop_masks, int ndims);
-// Masked hops with n > 128: builds their bit matrices on the host, copies them into one pooled
-// device buffer (*pooled; pool_free it after the last launch) in stream order and sets pb.dmask.
-// TA_ERR_INVALID_ARG if a query position is left without any visible key.
+// Masked hops with n > 128, and every masked hop when the masks differ per head: builds their bit
+// matrices on the host, copies them into one pooled device buffer (*pooled; pool_free it after
+// the last launch) in stream order and sets pb.dmask.  TA_ERR_INVALID_ARG if a query position
+// is left without any visible key.
 int upload_long_masks(Problem *pb, const Plan &plan, void **pooled);
 
 // Kernel launchers (each returns TA_OK or TA_ERR_CUDA).  xin has `xin_heads` heads per batch

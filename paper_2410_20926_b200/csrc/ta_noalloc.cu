@@ -81,6 +81,7 @@ extern "C" int ta_forward_static(const void *q, const void *k, const void *v, vo
     pb.scale = 1.0f / sqrtf((float)D);
     pb.rope_base = 0.f;
     pb.seq_lens = nullptr;
+    pb.masks_per_head = 0;
     pb.pdl = 0;
     for (int i = 0; i < TA_MAX_DIMS; ++i) { pb.window[i] = 0; pb.masks[i] = nullptr; pb.dmask[i] = nullptr; pb.dmask_words[i] = 0; }
     pb.flags = 0; pb.hop_begin = 0; pb.hop_end = ndims;

@@ -34,8 +34,9 @@ struct SimtArgs {
     float rope_log2_base;         // 0: no positional encoding; else log2 of the RoPE base
     int window;                   // 0, or sliding window along the hop's dimension
     int masked;                   // 1: visibility comes from the HopMask parameter (n <= 128), 2: from dmask
-    const uint32_t *dmask;        // device bit matrix of a masked dimension longer than 128
+    const uint32_t *dmask;        // device bit matrix (longer dimensions, per-head masks)
     int dmask_words;
+    int dmask_heads;              // bit matrices behind dmask: 1 (every head alike) or H
     const int *lens;              // device, valid length per batch entry, or nullptr
 };
 
@@ -125,7 +126,9 @@ hop_simt_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__res
                 bool valid = key < exist && t < exist && (!a.causal || key <= t) &&
                              (a.window == 0 || (key > t - a.window && key < t + a.window));
                 if (a.masked == 1) valid = valid && ((hop_mask.bits[t][key >> 5] >> (key & 31)) & 1u);
-                if (a.masked == 2) valid = valid && ((__ldg(a.dmask + (size_t)t * a.dmask_words + (key >> 5)) >> (key & 31)) & 1u);
+                if (a.masked == 2 && valid)
+                    valid = ((__ldg(a.dmask + ((size_t)(a.dmask_heads > 1 ? h : 0) * a.n + t) * a.dmask_words + (key >> 5)) >>
+                              (key & 31)) & 1u) != 0;
                 s = valid ? s : -INFINITY;
                 // a block may hold no visible key of this row (window): keep the arithmetic finite
                 const float m_new = fmaxf(m[r], warp_max(s));
@@ -190,11 +193,13 @@ int launch_t(const Problem &pb, const HopDesc &hd, const void *xin, int xin_head
     a.lens = pb.seq_lens;
     HopMask hm;
     memset(&hm, 0, sizeof(hm));
-    if (pb.masks[hd.hop] && hd.n > 128) {
+    a.dmask_heads = 1;
+    if (pb.masks[hd.hop] && (hd.n > 128 || pb.masks_per_head)) {
         if (!pb.dmask[hd.hop]) return TA_ERR_INVALID_ARG;
         a.masked = 2;                                  // bit matrix in device memory
         a.dmask = pb.dmask[hd.hop];
         a.dmask_words = pb.dmask_words[hd.hop];
+        a.dmask_heads = pb.masks_per_head ? pb.H : 1;
     } else if (pb.masks[hd.hop]) {
         const int rc = build_hop_mask(pb, hd, &hm);   // explicit mask ^ causal flag ^ window
         if (rc != TA_OK) return rc;

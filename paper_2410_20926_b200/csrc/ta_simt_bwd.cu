@@ -41,7 +41,7 @@ struct SimtBwdArgs {
     float rope_log2_base;         // 0: no positional encoding
     int window, masked;           // masked: 1 = HopMask parameter (n <= 128), 2 = device bit matrix dmask
     const uint32_t *dmask;
-    int dmask_words;
+    int dmask_words, dmask_heads; // bit matrices behind dmask: 1 (every head alike) or H
     const int *lens;
     int first_hop, accumulate;
 };
@@ -53,11 +53,12 @@ __device__ __forceinline__ int segment_exist(const SimtBwdArgs &a, int b, long l
     return len <= base ? 0 : (int)(left < a.n ? left : a.n);
 }
 
-__device__ __forceinline__ bool pair_visible(const SimtBwdArgs &a, const HopMask &hm, int t, int key, int exist) {
+__device__ __forceinline__ bool pair_visible(const SimtBwdArgs &a, const HopMask &hm, int t, int key, int exist, int h) {
     bool v = key < exist && t < exist && (!a.causal || key <= t) &&
              (a.window == 0 || (key > t - a.window && key < t + a.window));
     if (a.masked == 1) v = v && ((hm.bits[t][key >> 5] >> (key & 31)) & 1u);
-    if (a.masked == 2 && v) v = ((__ldg(a.dmask + (size_t)t * a.dmask_words + (key >> 5)) >> (key & 31)) & 1u) != 0;
+    if (a.masked == 2 && v)
+        v = ((__ldg(a.dmask + ((size_t)(a.dmask_heads > 1 ? h : 0) * a.n + t) * a.dmask_words + (key >> 5)) >> (key & 31)) & 1u) != 0;
     return v;
 }
 
@@ -148,7 +149,7 @@ hop_simt_bwd_q_kernel(const T *__restrict__ q, const T *__restrict__ k,
                 float s = 0.f;
                 for (int c = 0; c < D; ++c) s = fmaf(qr[c], kr[c], s);
                 s *= a.scale;
-                const bool valid = pair_visible(a, hop_mask, t, key, exist);
+                const bool valid = pair_visible(a, hop_mask, t, key, exist, h);
                 s = valid ? s : -INFINITY;
                 const float m_new = fmaxf(m[r], warp_max(s));
                 const float m_ref = m_new == -INFINITY ? 0.f : m_new;
@@ -201,7 +202,7 @@ hop_simt_bwd_q_kernel(const T *__restrict__ q, const T *__restrict__ k,
                     s = fmaf(qr[c], kr[c], s);
                     dp = fmaf(gr[c], xr[c], dp);
                 }
-                const bool valid = pair_visible(a, hop_mask, t, key, exist);
+                const bool valid = pair_visible(a, hop_mask, t, key, exist, h);
                 const float p = valid ? expf(s * a.scale - lse[r]) : 0.f;
                 const float ds = valid ? p * (dp - delta[r]) * a.scale : 0.f;
                 for (int u = 0; u < BL; ++u) {
@@ -343,7 +344,7 @@ hop_simt_bwd_k_kernel(const T *__restrict__ q, const T *__restrict__ k,
                         s = fmaf(qr[c], kr[c], s);
                         dp = fmaf(gr[c], xr[c], dp);
                     }
-                    const bool valid = t < q_end && pair_visible(a, hop_mask, t, key, exist);
+                    const bool valid = t < q_end && pair_visible(a, hop_mask, t, key, exist, kv * grp + hh);
                     const float p = valid ? expf(s * a.scale - st.x) : 0.f;
                     const float ds = valid ? p * (dp - st.y) * a.scale : 0.f;
                     for (int tt = 0; tt < BL; ++tt) {
@@ -431,11 +432,13 @@ int launch_dpl(const Problem &pb, const HopDesc &hd, const void *x, int x_heads,
     a.dmask_words = 0;
     HopMask hm;
     memset(&hm, 0, sizeof(hm));
-    if (pb.masks[hd.hop] && hd.n > 128) {
+    a.dmask_heads = 1;
+    if (pb.masks[hd.hop] && (hd.n > 128 || pb.masks_per_head)) {
         if (!pb.dmask[hd.hop]) return TA_ERR_INVALID_ARG;
         a.masked = 2;
         a.dmask = pb.dmask[hd.hop];
         a.dmask_words = pb.dmask_words[hd.hop];
+        a.dmask_heads = pb.masks_per_head ? pb.H : 1;
     } else if (pb.masks[hd.hop]) {
         const int rc = build_hop_mask(pb, hd, &hm);
         if (rc != TA_OK) return rc;

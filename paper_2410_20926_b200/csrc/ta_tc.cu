@@ -30,6 +30,7 @@
 // ends all its roles, waits for its copies in flight, frees its TMEM and returns.
 #include <cuda_bf16.h>
 
+#include <cstring>
 #include <mutex>
 
 #include "ta_internal.h"
@@ -74,6 +75,8 @@ struct TcArgs {
     int stride;                // token stride of the hop's dimension
     const int *lens;           // device, one valid length per batch entry, or nullptr (masked variant only)
     int x_f16, out_f16;        // the value tensor read / written holds fp16 (an intermediate of a hop chain), not bf16
+    const uint32_t *dmask;     // masked variant, masks that differ per head: [H][n][4] words in device memory
+                               // (causal flag and window folded in); nullptr: the mask is the kernel parameter
 };
 
 struct ItemCoord {
@@ -349,6 +352,13 @@ hop_pipe_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             // valid length: only the first `exist` positions of this row's segment are tokens
             // (flat index below the batch entry's length); a padding row sees nothing
             uint32_t mt[4] = {mrow[0], mrow[1], mrow[2], mrow[3]};
+            if (kMask && a.dmask != nullptr) {
+                // this tile's query head has a mask of its own
+                const ItemCoord c = decode_item(a, (long long)blockIdx.x + (long long)(t / (uint32_t)a.gi) * gridDim.x);
+                const int head = (c.q_head0 + (int)(t % (uint32_t)a.gi)) % a.H;
+                tile_row_mask(a.dmask + (size_t)head * a.n * 4, row_valid ? r % a.n : 0, seg * a.n, mt);
+                if (!row_valid) mt[0] = mt[1] = mt[2] = mt[3] = 0u;
+            }
             if (kMask && a.lens != nullptr) {
                 const ItemCoord c = decode_item(a, (long long)blockIdx.x + (long long)(t / (uint32_t)a.gi) * gridDim.x);
                 const int len = __ldg(a.lens + c.kv_head / a.H_kv);
@@ -576,6 +586,8 @@ int launch_d(const Problem &pb, const HopDesc &hd, const void *xin, int xin_head
     a.lens = pb.seq_lens;
     a.x_f16 = hd.in_f16;
     a.out_f16 = hd.out_f16;
+    a.dmask = (pb.masks[hd.hop] && pb.masks_per_head) ? pb.dmask[hd.hop] : nullptr;
+    if (pb.masks[hd.hop] && pb.masks_per_head && !a.dmask) return TA_ERR_INVALID_ARG;
 
     constexpr size_t smem = PipeCfg<D>::kSmemBytes;
     const unsigned grid = (unsigned)(a.total_items < num_sms ? a.total_items : num_sms);
@@ -598,8 +610,14 @@ int launch_d(const Problem &pb, const HopDesc &hd, const void *xin, int xin_head
     const bool overlap = pb.pdl && a.total_items <= 32ll * num_sms;
     if (pb.masks[hd.hop] || pb.seq_lens) {
         HopMask hm;                                  // explicit mask ^ causal flag ^ window, by value
-        const int rc = build_hop_mask(pb, hd, &hm);
-        if (rc != TA_OK) return rc;
+        if (a.dmask) {
+            // per-head masks live in device memory; the parameter only says "everything visible"
+            // (the kernel replaces it per tile)
+            memset(&hm, 0, sizeof(hm));
+        } else {
+            const int rc = build_hop_mask(pb, hd, &hm);
+            if (rc != TA_OK) return rc;
+        }
         if (pb.rope_base > 0.f)
             return launch_kernel(hop_pipe_kernel<D, true, true>, grid, kThreadsRope, smem, pb.stream, overlap, mq, mk, mxi,
                                  mxo, a, hm);

@@ -29,6 +29,8 @@
 // flag that ends both roles, lets its copies land, frees its TMEM and returns.
 #include <cuda_bf16.h>
 
+#include <cstring>
+
 #include "ta_internal.h"
 #include "ta_ptx.cuh"
 #include "ta_rope.cuh"
@@ -50,6 +52,8 @@ struct BwdArgs {
     float rope_log2_base;              // log2 of the RoPE base (rotating variant only)
     int stride;                        // token stride of the hop's dimension
     const int *lens;                   // device, valid length per batch entry, or nullptr (masked variant only)
+    const uint32_t *dmask;             // masked variant, masks that differ per head: [H][n][4] words in device
+                                       // memory (causal flag and window folded in); nullptr: the kernel parameter
 };
 
 template <int D>
@@ -312,6 +316,7 @@ hop_tc_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         int pending_stage = -1;   // thread 0: stage whose output stores have been issued but not yet read out
         for (long long item = blockIdx.x; ok && item < a.total_items; item += gridDim.x, ++it) {
             const BwdItem c = decode_bwd_item(a, item);
+            uint32_t lim[4] = {~0u, ~0u, ~0u, ~0u};        // columns below the batch entry's valid length
             if (kMask && a.lens != nullptr) {
                 // only the first `exist` positions of this row's segment are tokens; a padding row
                 // sees nothing (its P and dS rows are 0, so nothing flows through it)
@@ -323,10 +328,17 @@ hop_tc_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
 #pragma unroll
                 for (int cch = 0; cch < 4; ++cch) {
                     const int nb = limit - 32 * cch;
-                    mt[cch] = mrow[cch] & (nb >= 32 ? 0xffffffffu : (nb <= 0 ? 0u : ((1u << nb) - 1u)));
+                    lim[cch] = nb >= 32 ? 0xffffffffu : (nb <= 0 ? 0u : ((1u << nb) - 1u));
+                    mt[cch] = mrow[cch] & lim[cch];
                 }
             }
             for (int j = 0; j < a.g; ++j, ++t) {
+                if (kMask && a.dmask != nullptr) {
+                    // this query head has a mask of its own
+                    tile_row_mask(a.dmask + (size_t)((c.q_head0 + j) % a.H) * a.n * 4, row_valid ? r % a.n : 0, seg * a.n, mt);
+#pragma unroll
+                    for (int cch = 0; cch < 4; ++cch) mt[cch] = row_valid ? (mt[cch] & lim[cch]) : 0u;
+                }
                 const int s = t & 1;
                 const uint32_t par = t & 1;
                 const int q_head = c.q_head0 + j;
@@ -674,6 +686,8 @@ int launch_bwd_d(const Problem &pb, const HopDesc &hd, const void *x, int x_head
     a.rope_log2_base = pb.rope_base > 0.f ? log2f(pb.rope_base) : 0.f;
     a.stride = (int)hd.stride;
     a.lens = pb.seq_lens;
+    a.dmask = (pb.masks[hd.hop] && pb.masks_per_head) ? pb.dmask[hd.hop] : nullptr;
+    if (pb.masks[hd.hop] && pb.masks_per_head && !a.dmask) return TA_ERR_INVALID_ARG;
 
     int dev = 0;
     const int num_sms = current_device_sms(&dev);
@@ -691,8 +705,12 @@ int launch_bwd_d(const Problem &pb, const HopDesc &hd, const void *x, int x_head
     const unsigned grid = (unsigned)(a.total_items < num_sms ? a.total_items : num_sms);
     if (pb.masks[hd.hop] || pb.seq_lens) {
         HopMask hm;                                  // explicit mask ^ causal flag ^ window, by value
-        const int rc = build_hop_mask(pb, hd, &hm);
-        if (rc != TA_OK) return rc;
+        if (a.dmask) {
+            memset(&hm, 0, sizeof(hm));              // per-head masks: read from device memory per head
+        } else {
+            const int rc = build_hop_mask(pb, hd, &hm);
+            if (rc != TA_OK) return rc;
+        }
         if (pb.rope_base > 0.f)
             return launch_kernel(hop_tc_bwd_kernel<D, true, true>, grid, kThreadsRope, smem, pb.stream, false, mq, mk, mx,
                                  mgi, mgo, mdq, mdk, mdv, a, hm);

@@ -54,6 +54,7 @@ struct LongArgs {
     // flag and the window folded in, then per query block of 128 the range of key blocks it sees
     const uint32_t *mask_bits;
     int mask_words;
+    int mask_heads;            // bit matrices (and range tables) behind mask_bits: 1 or H
 };
 
 template <int D>
@@ -113,7 +114,9 @@ __device__ __forceinline__ LongItem decode_long_item(const LongArgs &a, long lon
     int mask_lo = 0, mask_hi = 0;
     if (a.mask_bits != nullptr) {
         // (one range for the pair: the two tiles walk the same key blocks, as they do without a mask)
-        const int *range = reinterpret_cast<const int *>(a.mask_bits + (size_t)a.n * a.mask_words) + 2 * (c.t0 / kTileRows);
+        const int mhead = a.mask_heads > 1 ? c.q_head % a.H : 0;
+        const int *range = reinterpret_cast<const int *>(a.mask_bits + (size_t)a.mask_heads * a.n * a.mask_words) +
+                           2 * ((size_t)mhead * a.qblocks + c.t0 / kTileRows);
         mask_lo = __ldg(range);
         mask_hi = __ldg(range + 1);
         if (c.ntiles == 2) {
@@ -399,7 +402,8 @@ hop_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 // explicit mask: this row's 128 bits over the block's keys (all ones without a mask)
                 uint4 mrow = make_uint4(~0u, ~0u, ~0u, ~0u);
                 if (kWindow && a.mask_bits != nullptr && row_valid)
-                    mrow = __ldg(reinterpret_cast<const uint4 *>(a.mask_bits + (size_t)t * a.mask_words + 4 * j));
+                    mrow = __ldg(reinterpret_cast<const uint4 *>(
+                        a.mask_bits + ((size_t)(a.mask_heads > 1 ? c.q_head % a.H : 0) * a.n + t) * a.mask_words + 4 * j));
                 auto mask_word = [&](int cc) { return cc == 0 ? mrow.x : (cc == 1 ? mrow.y : (cc == 2 ? mrow.z : mrow.w)); };
                 const int nchunks = (keys + 31) >> 5;
 
@@ -608,6 +612,7 @@ int launch_long_d(const Problem &pb, const HopDesc &hd, const void *xin, int xin
     a.stats_g = (const __nv_bfloat16 *)stats_g;
     a.mask_bits = pb.masks[hd.hop] ? pb.dmask[hd.hop] : nullptr;
     a.mask_words = pb.dmask_words[hd.hop];
+    a.mask_heads = pb.masks_per_head ? pb.H : 1;
     if (pb.masks[hd.hop] && !a.mask_bits) return TA_ERR_INVALID_ARG;
 
     int dev = 0;

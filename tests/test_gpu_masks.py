@@ -216,6 +216,54 @@ def test_backward_with_masks_on_long_segments(dims, D, causal, kind):
             assert_grad_close(g, r, name, grad_f32, sum(1 for n in dims if n > 1))
 
 
+@pytest.mark.parametrize("dims,D,causal,flags", [
+    ([8, 16, 32], 128, True, 0),                         # tensor-core hops, four segments per tile
+    ([5, 24], 64, False, 0),
+    ([3, 200], 128, True, 0),                            # short hop and long hop
+    ([6, 20], 40, True, 0),                              # generic kernels (head dim 40)
+    ([4, 64], 128, True, ta.TA_FLAG_NO_TENSOR_CORE),
+])
+def test_masks_that_differ_per_head(dims, D, causal, flags):
+    """masks_per_head: every query head has its own n_i x n_i matrix per hop (heads of one GQA group
+    see different keys); forward and backward against the oracle, which takes H x n x n arrays."""
+    B, H, Hkv = 2, 4, 2
+    N = math.prod(dims)
+    rng = np.random.default_rng(21)
+    masks = []
+    for n in dims:
+        m = (rng.random((H, n, n)) < 0.5).astype(np.uint8)
+        m[:, np.arange(n), np.arange(n)] = 1
+        masks.append(m)
+    inp = ta_inputs.make_inputs(B, H, Hkv, N, D, "bf16", 713, with_dout=True)
+    got = gpu_forward(inp, B, H, Hkv, N, D, dims, causal, "bf16", flags, hop_masks=masks)
+    ref = oracle.forward(inp["q"], inp["k"], inp["v"], dims, causal, masks=masks)
+    assert_close(got, ref, "bf16")
+    shared = oracle.forward(inp["q"], inp["k"], inp["v"], dims, causal, masks=[m[0] for m in masks])
+    assert np.abs(ref[:, 1:] - shared[:, 1:]).max() > 0.05        # the other heads' masks matter
+    if flags:
+        return
+    refs = oracle.backward(inp["dout"], inp["q"], inp["k"], inp["v"], dims, causal, masks=masks)
+    for grad_f32 in (True, False):
+        grads = gpu_backward(inp, B, H, Hkv, N, D, dims, causal, grad_f32, hop_masks=masks)
+        for name, g, r in zip(("dq", "dk", "dv"), grads, refs):
+            assert_grad_close(g, r, name, grad_f32, sum(1 for n in dims if n > 1))
+
+
+def test_per_head_masks_with_equal_matrices_reproduce_the_shared_mask():
+    B, H, Hkv, D, dims = 1, 4, 2, 128, [4, 64]
+    N = math.prod(dims)
+    masks = random_masks(dims, 22)
+    inp = ta_inputs.make_inputs(B, H, Hkv, N, D, "bf16", 714)
+    a = gpu_forward(inp, B, H, Hkv, N, D, dims, True, "bf16", hop_masks=masks)
+    b = gpu_forward(inp, B, H, Hkv, N, D, dims, True, "bf16", hop_masks=[np.stack([m] * H) for m in masks])
+    np.testing.assert_array_equal(a, b)
+    with pytest.raises(ValueError):       # either every mask is per head or none
+        import torch
+        x = torch.zeros(1, 4, 256, 64, dtype=torch.bfloat16, device="cuda")
+        ta.ta_forward_ex(x, x[:, :2], x[:, :2], torch.empty_like(x), 1, 4, 2, 256, 64, [4, 64], True,
+                         hop_masks=[np.ones((4, 4)), np.ones((4, 64, 64))])
+
+
 def test_masks_llama_shape_sampled_heads():
     """32 768 tokens as 32x32x32, H=32, H_kv=8, D=128, causal, with a random mask on every hop."""
     c = ta_inputs.CONFIGS[3]

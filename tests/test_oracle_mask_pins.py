@@ -200,6 +200,40 @@ def test_block_diagonal_mask_splits_the_dimension():
     np.testing.assert_allclose(got, ref, atol=1e-14)
 
 
+@pytest.mark.parametrize("causal", [False, True])
+def test_per_head_masks(causal):
+    """An H x n x n entry gives every query head its own matrix: the C route against the dense
+    route, against one-head runs with that head's matrix, and -- all heads alike -- against the
+    shared-matrix form; gradients of a GQA group sum heads that saw different masks."""
+    rng = np.random.default_rng(80)
+    dims, H, Hkv = [4, 6], 4, 2
+    N = 24
+    m0 = np.stack([random_mask(4, rng) for _ in range(H)])
+    m1 = np.stack([random_mask(6, rng) for _ in range(H)])
+    q, k, v = rnd((1, H, N, 5), 81), rnd((1, Hkv, N, 5), 82), rnd((1, Hkv, N, 5), 83)
+    a = oracle.forward(q, k, v, dims, causal, masks=[m0, m1])
+    np.testing.assert_allclose(a, oracle.forward_dense(q, k, v, dims, causal, masks=[m0, m1]), rtol=0, atol=1e-13)
+    for h in range(H):
+        one = oracle.forward(q[:, h:h + 1], k[:, h // 2:h // 2 + 1], v[:, h // 2:h // 2 + 1], dims, causal,
+                             masks=[m0[h], m1[h]])
+        np.testing.assert_allclose(a[:, h], one[:, 0], atol=1e-15)
+    same = oracle.forward(q, k, v, dims, causal, masks=[np.stack([m0[1]] * H), None])
+    np.testing.assert_allclose(same, oracle.forward(q, k, v, dims, causal, masks=[m0[1], None]), atol=0)
+    assert np.abs(a[:, 0] - oracle.forward(q, k, v, dims, causal, masks=[m0[1], m1[1]])[:, 0]).max() > 1e-3
+    # backward: a group's dk, dv are the sums of one-head gradients taken with each head's own masks
+    dout = rnd((1, H, N, 5), 84)
+    dq, dk, dv = oracle.backward(dout, q, k, v, dims, causal, masks=[m0, m1])
+    for kv in range(Hkv):
+        sk, sv = 0.0, 0.0
+        for h in (2 * kv, 2 * kv + 1):
+            gq, gk, gv = oracle.backward(dout[:, h:h + 1], q[:, h:h + 1], k[:, kv:kv + 1], v[:, kv:kv + 1], dims, causal,
+                                         masks=[m0[h], m1[h]])
+            np.testing.assert_allclose(dq[:, h], gq[:, 0], atol=1e-14)
+            sk, sv = sk + gk[:, 0], sv + gv[:, 0]
+        np.testing.assert_allclose(dk[:, kv], sk, atol=1e-13)
+        np.testing.assert_allclose(dv[:, kv], sv, atol=1e-13)
+
+
 def test_mask_with_an_empty_row_is_rejected():
     m = np.ones((4, 4), dtype=bool)
     m[2] = False
