@@ -53,8 +53,8 @@ NOMINAL_HBM_GBS, NOMINAL_BF16_TFLOPS = 8000.0, 2250.0
 L2_BYTES = 126 * 1024 * 1024
 # dram__bytes_read.sum + dram__bytes_write.sum per token per launch of the forward hop kernel,
 # from the ncu capture of config 3 summarised in profiles/hop_pipe_kernel_config3_ncu_full.md
-# (mean of the three hops, 758.8 MB for 32768 tokens); traffic is proportional to the tokens.
-NCU_TRAFFIC_BYTES_PER_TOKEN_PER_LAUNCH = 758.8e6 / 32768
+# (mean of the three hops, 758.3 MB for 32768 tokens); traffic is proportional to the tokens.
+NCU_TRAFFIC_BYTES_PER_TOKEN_PER_LAUNCH = 758.3e6 / 32768
 
 
 # ------------------------------------------------------------------ roofline arithmetic
