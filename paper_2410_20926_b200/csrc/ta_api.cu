@@ -724,8 +724,8 @@ int ta_plan_describe(int B, int H, int H_kv, int N, int D, const int *dims, int 
                  buf_name(h.src), buf_name(h.dst), h.out_f16 ? " dst_type=f16" : "",
                  h.pair ? " pair=first" : (j > 0 && plan.hops[j - 1].pair ? " pair=second" : ""));
         else if (h.path == PATH_TC_LONG)
-            emit("hop=%d path=tc-long n=%d stride=%lld outer=%lld key_blocks=%d src=%s dst=%s\n", h.hop, h.n, h.stride,
-                 h.outer, (h.n + 127) / 128, buf_name(h.src), buf_name(h.dst));
+            emit("hop=%d path=tc-long n=%d stride=%lld outer=%lld key_blocks=%d tiles_per_item=%d src=%s dst=%s\n", h.hop,
+                 h.n, h.stride, h.outer, (h.n + 127) / 128, long_tiles_per_item(h.n), buf_name(h.src), buf_name(h.dst));
         else
             emit("hop=%d path=simt n=%d stride=%lld outer=%lld src=%s dst=%s\n", h.hop, h.n, h.stride, h.outer,
                  buf_name(h.src), buf_name(h.dst));

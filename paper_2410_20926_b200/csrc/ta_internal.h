@@ -123,6 +123,8 @@ int launch_hop_tc(const Problem &pb, const HopDesc &hd, const void *xin, int xin
 // Long segments (n_i > 128): key-block loop with online softmax, ta_tc_long.cu.  xin != xout.
 int launch_hop_tc_long(const Problem &pb, const HopDesc &hd, const void *xin, int xin_heads, void *xout);
 int read_status_tc_long(unsigned int *word);
+// Query tiles per work item of that kernel for segments of n positions: 1 (two CTAs per SM) or 2.
+int long_tiles_per_item(int n);
 // Positional encoding on long-segment hops: rotated bf16 copies of q and k in a buffer taken from
 // the library's pool on the call's stream (plus extra_bytes of scratch behind them; the caller
 // hands *pooled back with pool_free after its last launch that reads it), and

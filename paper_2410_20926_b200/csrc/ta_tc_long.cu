@@ -24,7 +24,14 @@
 // tile 0 and tile 1 (one TMEM lane = one query row per thread).  Every wait is bounded; when one
 // expires the CTA raises a flag that ends all its roles, waits for its copies in flight, frees
 // its TMEM and returns.
+//
+// Segments of a few tiles (n_i <= kSoloMaxN) take the kSolo instantiation instead: a work item is
+// ONE query tile, a CTA has one chain (warps 4-7), single Q, K and X slots (96 KB at D = 128) and
+// 256 TMEM columns, and TWO CTAs share an SM.  Such hops move about as many bytes per flop as the
+// short-segment hops: what they need is loads in flight while a chain computes, and with a second
+// CTA on the SM one CTA's loads run under the other's softmax and MMAs.
 #include <cuda_bf16.h>
+#include <stdlib.h>
 
 #include "ta_internal.h"
 #include "ta_ptx.cuh"
@@ -45,6 +52,7 @@ struct LongArgs {
     const int *lens;           // device, valid length per batch entry, or nullptr (kWindow variant only)
     int N;
     int pair_major;            // item numbering, see decode_long_item
+    int tiles_per_item;        // 2: an item is a pair of query tiles; 1: a single tile (kSolo); qpairs counts items per segment
     // statistics pass of the backward: instead of the output rows, write per query row
     // (log2-sum-exp of the scaled scores, <G_t, O_t>) -- stats[q_head * N + token]; g = gradient
     // with respect to the hop's output, laid out like q
@@ -57,18 +65,25 @@ struct LongArgs {
     int mask_heads;            // bit matrices (and range tables) behind mask_bits: 1 or H
 };
 
-template <int D>
+constexpr int kSoloThreads = 256;
+constexpr int kSoloMaxN = 1024;   // segments up to this length run one query tile per item, two CTAs per SM
+
+template <int D, bool kSolo = false>
 struct LongCfg {
     static constexpr int kHalves = D / 64;
+    static constexpr int kChains = kSolo ? 1 : 2;
     static constexpr uint32_t kSlabBytes = kTileRows * 128;
     static constexpr uint32_t kTileBytes = kHalves * kSlabBytes;
-    static constexpr uint32_t kOffQ = 0;                                   // the item's two Q tiles
-    static constexpr uint32_t kOffKV = kOffQ + 2 * kTileBytes;             // per stage: K then X
-    static constexpr uint32_t kOffBar = kOffKV + kNKV * 2 * kTileBytes;
-    static constexpr int kNumBars = 2 + 2 * kNKV + 6;
+    static constexpr uint32_t kOffQ = 0;                                   // the item's Q tiles
+    // two chains: kNKV stages of (K block, X block); one chain: one K slot and one X slot (barrier
+    // pair 0 is then K's, pair 1 X's)
+    static constexpr uint32_t kOffKV = kOffQ + kChains * kTileBytes;
+    static constexpr uint32_t kOffBar = kOffKV + (kSolo ? 1 : kNKV) * 2 * kTileBytes;
+    static constexpr int kNumBars = 2 + 2 * kNKV + 6 + 1;
     static constexpr uint32_t kSmemBytes = kOffBar + kNumBars * 8 + 16 + 1024;
-    static constexpr uint32_t kTmemCols = 512;
-    static constexpr uint32_t kColS = 0, kColO = 256;   // S_c at 128 c (P over its first 64 columns), O_c at 256 + 128 c
+    static constexpr uint32_t kTmemCols = kSolo ? 256 : 512;
+    // S_c at 128 c (P over its first 64 columns), then the O_c, 128 columns apart
+    static constexpr uint32_t kColS = 0, kColO = 128 * kChains;
 };
 
 struct LongItem {
@@ -102,8 +117,8 @@ __device__ __forceinline__ LongItem decode_long_item(const LongArgs &a, long lon
     c.outer = (int)(rest % a.outer); rest /= a.outer;
     c.q_head = (int)rest;                                          // b * H + h
     c.kv_head = (c.q_head / a.H) * a.H_kv + (c.q_head % a.H) / a.g;
-    c.t0 = 2 * pb * kTileRows;
-    c.ntiles = 2 * pb + 1 < a.qblocks ? 2 : 1;
+    c.t0 = a.tiles_per_item * pb * kTileRows;
+    c.ntiles = min(a.tiles_per_item, a.qblocks - a.tiles_per_item * pb);
     c.exist = a.n;
     if (a.lens != nullptr) {
         const long long len = min(max(__ldg(a.lens + c.q_head / a.H), 0), a.N);
@@ -176,11 +191,12 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32
         : "memory");
 }
 
-template <int D, bool kWindow>
-__global__ void __launch_bounds__(kThreads, 1)
+template <int D, bool kWindow, bool kSolo>
+__global__ void __launch_bounds__(kSolo ? kSoloThreads : kThreads, kSolo ? 2 : 1)
 hop_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                const __grid_constant__ CUtensorMap map_xin, __nv_bfloat16 *__restrict__ xout, const LongArgs a) {
-    using C = LongCfg<D>;
+                const __grid_constant__ CUtensorMap map_xin, const __grid_constant__ CUtensorMap map_out,
+                __nv_bfloat16 *__restrict__ xout, const LongArgs a) {
+    using C = LongCfg<D, kSolo>;
     constexpr int kHalves = C::kHalves;
     constexpr uint32_t kSlabBytes = C::kSlabBytes, kTileBytes = C::kTileBytes;
 
@@ -198,16 +214,17 @@ hop_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     auto s_full = [&](int c) { return bar0 + 8u * (uint32_t)(kB1 + c); };        // S of tile c complete
     auto p_full = [&](int c) { return bar0 + 8u * (uint32_t)(kB1 + 2 + c); };    // P of tile c written (4 warps)
     auto pv_done = [&](int c) { return bar0 + 8u * (uint32_t)(kB1 + 4 + c); };   // value MMA of tile c complete
+    const uint32_t out_full = bar0 + 8u * (uint32_t)(kB1 + 6);                   // kSolo: output tile staged (4 warps)
     uint32_t *tmem_slot = (uint32_t *)(smem + C::kOffBar + C::kNumBars * 8);
     volatile uint32_t *abort_flag = tmem_slot + 1;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
-    for (uint32_t i = tid; i < C::kOffBar / 16; i += kThreads) ((uint4 *)smem)[i] = make_uint4(0, 0, 0, 0);
+    for (uint32_t i = tid; i < C::kOffBar / 16; i += blockDim.x) ((uint4 *)smem)[i] = make_uint4(0, 0, 0, 0);
     if (tid == 0) {
         for (int i = 0; i < C::kNumBars; ++i) {
             const uint32_t bar = bar0 + 8u * (uint32_t)i;
-            mbar_init(bar, (bar == p_full(0) || bar == p_full(1)) ? 4 : 1);   // one arrival per softmax warp
+            mbar_init(bar, (bar == p_full(0) || bar == p_full(1) || bar == out_full) ? 4 : 1);   // one arrival per softmax warp
         }
         *abort_flag = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -248,6 +265,26 @@ hop_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 #pragma unroll
                     for (int h = 0; h < kHalves; ++h)
                         tma_load_5d(sQ(i) + h * kSlabBytes, &map_q, q_full, 64 * h, c.t0 + kTileRows * i, c.inner, c.outer, c.q_head);
+                if constexpr (kSolo) {
+                    // one K slot (barrier pair 0) and one X slot (pair 1), block after block
+                    for (int j = c.jlo; j < c.jhi; ++j, ++g) {
+                        const uint32_t par = g & 1;
+                        ok = mbar_wait_abortable(kv_free(0), par ^ 1, 0xD1, abort_flag);
+                        if (!ok) break;
+                        mbar_expect_tx(kv_full(0), kTileBytes);
+                        arm(2u, par);
+#pragma unroll
+                        for (int h = 0; h < kHalves; ++h)
+                            tma_load_5d(sKb(0) + h * kSlabBytes, &map_k, kv_full(0), 64 * h, kTileRows * j, c.inner, c.outer, c.kv_head);
+                        ok = mbar_wait_abortable(kv_free(1), par ^ 1, 0xD2, abort_flag);
+                        if (!ok) break;
+                        mbar_expect_tx(kv_full(1), kTileBytes);
+                        arm(4u, par);
+#pragma unroll
+                        for (int h = 0; h < kHalves; ++h)
+                            tma_load_5d(sXb(0) + h * kSlabBytes, &map_xin, kv_full(1), 64 * h, kTileRows * j, c.inner, c.outer, x_head);
+                    }
+                } else
                 for (int j = c.jlo; j < c.jhi; ++j, ++g) {
                     const int st = g % kNKV;
                     const uint32_t par = (g / kNKV) & 1;
@@ -291,6 +328,40 @@ hop_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 const LongItem c = decode_long_item(a, item);
                 ok = mbar_wait_abortable(q_full, ic & 1, 0xE0, abort_flag);
                 if (!ok) break;
+                if constexpr (kSolo) {
+                    // one chain, in order: S(j), then O += P(j) X_j once the softmax warps have written P
+                    for (int j = c.j0[0]; ok && j < c.je[0]; ++j, ++g0) {
+                        const uint32_t par = g0 & 1;
+                        ok = mbar_wait_abortable(kv_full(0), par, 0xE1, abort_flag);
+                        if (!ok) break;
+                        tc_fence_after();
+#pragma unroll
+                        for (int kb = 0; kb < D / 16; ++kb) {
+                            const uint32_t off = (kb >> 2) * kSlabBytes + (kb & 3) * 32;
+                            tc_mma_ss(tmem_base + C::kColS, smem_desc_sw128(sQ(0) + off, 16, 1024),
+                                      smem_desc_sw128(sKb(0) + off, 16, 1024), idesc_s, kb > 0);
+                        }
+                        tc_commit(s_full(0));
+                        tc_commit(kv_free(0));
+                        if (j == c.je[0] - 1) tc_commit(q_free);
+                        ok = mbar_wait_abortable(p_full(0), p_seen[0] & 1, 0xE2, abort_flag);
+                        if (!ok) break;
+                        ++p_seen[0];
+                        ok = mbar_wait_abortable(kv_full(1), par, 0xE3, abort_flag);
+                        if (!ok) break;
+                        tc_fence_after();
+                        const int keys = min(kTileRows, c.keys_end[0] - kTileRows * j);
+                        const int kblocks = (keys + 15) >> 4;
+                        for (int kb = 0; kb < kblocks; ++kb)
+                            tc_mma_ts(tmem_base + C::kColO, tmem_base + C::kColS + kb * 8,
+                                      smem_desc_sw128(sXb(0) + kb * 2048, kSlabBytes, 1024), idesc_o,
+                                      (kb > 0 || j > c.j0[0]) ? 1u : 0u);
+                        tc_commit(pv_done(0));
+                        // (the X slot of a tile's last block takes the output tile next: the store thread frees it)
+                        if (j < c.je[0] - 1) tc_commit(kv_free(1));
+                    }
+                    continue;
+                }
                 int js[2] = {c.j0[0], c.j0[1]};       // next block whose S is to be issued
                 int jp[2] = {c.j0[0], c.j0[1]};       // next block whose value MMA is to be issued
                 bool q_released = false;
@@ -363,9 +434,33 @@ hop_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 g0 += (uint32_t)(c.jhi - c.jlo);
             }
         }
+    } else if (kSolo && warp == 2) {
+        // =============================================================== TMA store of finished tiles (kSolo)
+        // The softmax warps stage the output tile in the X slot of the tile's last key block; the
+        // slot goes back to the producer once the store has read it.
+        if (lane == 0) {
+            uint32_t ic = 0;
+            bool ok = true;
+            for (long long round = 0; ok && round * gridDim.x < a.total_items; ++round) {
+                const long long item = long_item_of_round(a, round);
+                if (item < 0) continue;
+                const LongItem c = decode_long_item(a, item);
+                ok = mbar_wait_abortable(out_full, ic & 1, 0xC0, abort_flag);
+                if (!ok) break;
+                ++ic;
+                if (a.stats == nullptr) {
+#pragma unroll
+                    for (int h = 0; h < kHalves; ++h)
+                        tma_store_5d(&map_out, sXb(0) + h * kSlabBytes, 64 * h, c.t0, c.inner, c.outer, c.q_head);
+                    tma_store_commit_and_wait_read();
+                }
+                mbar_arrive(kv_free(1));
+            }
+            tma_store_wait_all();
+        }
     } else if (warp >= 4) {
         // =============================================================== softmax, rescaling, epilogue
-        const int ch = (warp - 4) >> 2;                 // which of the item's two query tiles
+        const int ch = kSolo ? 0 : (warp - 4) >> 2;     // which of the item's query tiles
         const int wq = warp & 3;                        // TMEM lane quarter of this warp
         const uint32_t tmem_lane = tmem_base + ((uint32_t)(wq * 32) << 16);
         const int r = wq * 32 + lane;                   // this thread's query row of the tile
@@ -412,15 +507,22 @@ hop_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 if (!ok) break;
                 tc_fence_after();
 
-                // a block every row sees completely needs no per-element masks (most blocks of a long segment)
-                const bool full = !diag && !kWindow && keys == kTileRows && row_valid;
-                const bool full_w = __all_sync(0xffffffffu, full);
+                // 32-column chunks every row of this warp sees completely need no per-element masks (all
+                // of a block below the diagonal; in the diagonal block the chunks left of the warp's own)
+                uint32_t my_full = 0;
+                if (!kWindow) {
+#pragma unroll
+                    for (int cc = 0; cc < 4; ++cc)
+                        if (32 * cc + 32 <= c_hi) my_full |= 1u << cc;
+                }
+                const uint32_t full_bits = kWindow ? 0u : __reduce_and_sync(0xffffffffu, my_full);
                 float bm = -INFINITY;
                 uint32_t v[32];
-                if (full_w) {
 #pragma unroll 1
-                    for (int cc = 0; cc < 4; ++cc) {
-                        tmem_ld32(s_col + 32 * cc, v);
+                for (int cc = 0; cc < nchunks; ++cc) {
+                    if (32 * cc >= w_hi) continue;          // warp-uniform
+                    tmem_ld32(s_col + 32 * cc, v);
+                    if ((full_bits >> cc) & 1u) {
                         float b0 = fmaxf(__uint_as_float(v[0]), __uint_as_float(v[1]));
                         float b1 = fmaxf(__uint_as_float(v[2]), __uint_as_float(v[3]));
 #pragma unroll
@@ -429,12 +531,7 @@ hop_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                             b1 = fmaxf(b1, fmaxf(__uint_as_float(v[jj + 2]), __uint_as_float(v[jj + 3])));
                         }
                         bm = fmaxf(bm, fmaxf(b0, b1));
-                    }
-                } else {
-#pragma unroll 1
-                    for (int cc = 0; cc < nchunks; ++cc) {
-                        if (32 * cc >= w_hi) continue;      // warp-uniform
-                        tmem_ld32(s_col + 32 * cc, v);
+                    } else {
                         const uint32_t mw = kWindow ? mask_word(cc) : ~0u;
 #pragma unroll
                         for (int jj = 0; jj < 32; ++jj)
@@ -466,13 +563,16 @@ hop_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 }
 
                 // ---- P (un-normalised, bf16) over the S columns already consumed
-                float sum = 0.f;
-                if (full_w) {
-                    // the row sum is taken over the fp32 weights here (the rounding of P averages out)
-                    float sum1 = 0.f;
+                // (over a chunk without masks the row sum is taken over the fp32 weights: the rounding of
+                // P averages out; elsewhere over the rounded weights)
+                float sum = 0.f, sum1 = 0.f;
 #pragma unroll 1
-                    for (int cc = 0; cc < 4; ++cc) {
-                        uint32_t pk[16];
+                for (int cc = 0; cc < nchunks; ++cc) {
+                    uint32_t pk[16];
+                    if (32 * cc >= w_hi) {
+#pragma unroll
+                        for (int jj = 0; jj < 16; ++jj) pk[jj] = 0u;
+                    } else if ((full_bits >> cc) & 1u) {
                         tmem_ld32(s_col + 32 * cc, v);
 #pragma unroll
                         for (int jj = 0; jj < 32; jj += 2) {
@@ -482,34 +582,24 @@ hop_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                             sum += p0;
                             sum1 += p1;
                         }
-                        tmem_st16(s_col + 16 * cc, pk);
-                    }
-                    sum += sum1;
-                } else {
-#pragma unroll 1
-                    for (int cc = 0; cc < nchunks; ++cc) {
-                        uint32_t pk[16];
-                        if (32 * cc < w_hi) {
-                            tmem_ld32(s_col + 32 * cc, v);
-                            const uint32_t mw = kWindow ? mask_word(cc) : ~0u;
+                    } else {
+                        tmem_ld32(s_col + 32 * cc, v);
+                        const uint32_t mw = kWindow ? mask_word(cc) : ~0u;
 #pragma unroll
-                            for (int jj = 0; jj < 32; jj += 2) {
-                                const int col = 32 * cc + jj;
-                                float p0 = fast_exp2(__uint_as_float(v[jj]) * a.scale_log2 - m_ref);
-                                float p1 = fast_exp2(__uint_as_float(v[jj + 1]) * a.scale_log2 - m_ref);
-                                p0 = (col >= c_lo && col < c_hi && ((mw >> jj) & 1u)) ? p0 : 0.f;
-                                p1 = (col + 1 >= c_lo && col + 1 < c_hi && ((mw >> (jj + 1)) & 1u)) ? p1 : 0.f;
-                                const uint32_t w = pack_bf16x2(p0, p1);
-                                pk[jj >> 1] = w;
-                                sum += __uint_as_float(w << 16) + __uint_as_float(w & 0xFFFF0000u);
-                            }
-                        } else {
-#pragma unroll
-                            for (int jj = 0; jj < 16; ++jj) pk[jj] = 0u;
+                        for (int jj = 0; jj < 32; jj += 2) {
+                            const int col = 32 * cc + jj;
+                            float p0 = fast_exp2(__uint_as_float(v[jj]) * a.scale_log2 - m_ref);
+                            float p1 = fast_exp2(__uint_as_float(v[jj + 1]) * a.scale_log2 - m_ref);
+                            p0 = (col >= c_lo && col < c_hi && ((mw >> jj) & 1u)) ? p0 : 0.f;
+                            p1 = (col + 1 >= c_lo && col + 1 < c_hi && ((mw >> (jj + 1)) & 1u)) ? p1 : 0.f;
+                            const uint32_t w = pack_bf16x2(p0, p1);
+                            pk[jj >> 1] = w;
+                            sum += __uint_as_float(w << 16) + __uint_as_float(w & 0xFFFF0000u);
                         }
-                        tmem_st16(s_col + 16 * cc, pk);
                     }
+                    tmem_st16(s_col + 16 * cc, pk);
                 }
+                sum += sum1;
                 tmem_st_wait();
                 l_run = l_run * alpha + sum;
                 m_run = m_new;
@@ -549,6 +639,26 @@ hop_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 }
                 if (row_valid)
                     a.stats[row_off / D] = make_float2(l_run > 0.f ? m_run + log2f(l_run) : INFINITY, dot * inv);
+            } else if constexpr (kSolo) {
+                // O / l -> bf16 -> the X slot (swizzled box layout) -> store thread
+                const float inv = (row_valid && l_run > 0.f) ? 1.f / l_run : 0.f;
+                const uint32_t x_row = sXb(0) + (uint32_t)r * 128u;
+                uint32_t v[32];
+#pragma unroll 1
+                for (int cc = 0; cc < D / 32; ++cc) {
+                    tmem_ld32(o_col + 32 * cc, v);
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int jj = 0; jj < 32; jj += 2)
+                        pk[jj >> 1] = pack_bf16x2(__uint_as_float(v[jj]) * inv, __uint_as_float(v[jj + 1]) * inv);
+                    const uint32_t slab = x_row + (uint32_t)(cc >> 1) * kSlabBytes;
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const uint32_t chunk = (uint32_t)(((cc & 1) * 4 + i) ^ (r & 7));
+                        st_shared_v4(slab + chunk * 16, pk[4 * i], pk[4 * i + 1], pk[4 * i + 2], pk[4 * i + 3]);
+                    }
+                }
+                fence_proxy_async_smem();
             } else {
                 const float inv = (row_valid && l_run > 0.f) ? 1.f / l_run : 0.f;
                 __nv_bfloat16 *dst = xout + (long long)c.q_head * a.head_stride + (long long)c.outer * a.seg_outer_stride +
@@ -571,6 +681,10 @@ hop_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 }
             }
             tc_fence_before();
+            if constexpr (kSolo) {
+                __syncwarp();
+                if (lane == 0) mbar_arrive(out_full);
+            }
         }
     }
 
@@ -582,6 +696,15 @@ hop_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     }
 }
 
+// Longest segment that runs one query tile per item (env TA_LONG_SOLO_MAX_N overrides, for measurements)
+int solo_max_n() {
+    static const int v = [] {
+        const char *e = getenv("TA_LONG_SOLO_MAX_N");
+        return e ? atoi(e) : kSoloMaxN;
+    }();
+    return v;
+}
+
 template <int D>
 int launch_long_d(const Problem &pb, const HopDesc &hd, const void *xin, int xin_heads, void *xout, void *stats = nullptr,
                   const void *stats_g = nullptr) {
@@ -591,12 +714,17 @@ int launch_long_d(const Problem &pb, const HopDesc &hd, const void *xin, int xin
     if ((rc = make_view_map(&mq, pb.q, pb.B * pb.H, pb.N, D, hd, 2, kTileRows, 1, 1)) != TA_OK) return rc;
     if ((rc = make_view_map(&mk, pb.k, pb.B * pb.H_kv, pb.N, D, hd, 2, kTileRows, 1, 1)) != TA_OK) return rc;
     if ((rc = make_view_map(&mxi, xin, pb.B * xin_heads, pb.N, D, hd, 2, kTileRows, 1, 1)) != TA_OK) return rc;
+    // (the statistics pass writes no output rows: its map is never used)
+    CUtensorMap mo = mq;
+    if (xout && (rc = make_view_map(&mo, xout, pb.B * pb.H, pb.N, D, hd, 2, kTileRows, 1, 1)) != TA_OK) return rc;
 
     LongArgs a;
     a.n = hd.n; a.causal = pb.causal; a.g = pb.H / pb.H_kv; a.H = pb.H; a.H_kv = pb.H_kv;
     a.xin_is_kv = xin_heads != pb.H ? 1 : 0;
+    a.tiles_per_item = long_tiles_per_item(hd.n);
+    const bool solo = a.tiles_per_item == 1;
     a.qblocks = (hd.n + kTileRows - 1) / kTileRows;
-    a.qpairs = (a.qblocks + 1) / 2;
+    a.qpairs = (a.qblocks + a.tiles_per_item - 1) / a.tiles_per_item;
     a.stride = hd.stride; a.outer = hd.outer;
     a.total_items = (long long)pb.B * pb.H * hd.outer * hd.stride * a.qpairs;
     a.row_stride = hd.stride * (long long)D;
@@ -617,21 +745,35 @@ int launch_long_d(const Problem &pb, const HopDesc &hd, const void *xin, int xin
 
     int dev = 0;
     const int num_sms = current_device_sms(&dev);
-    constexpr size_t smem = LongCfg<D>::kSmemBytes;
+    constexpr size_t smem = LongCfg<D>::kSmemBytes, smem_solo = LongCfg<D, true>::kSmemBytes;
     static PerDeviceOnce configured;
     if (!configured.is_done(dev)) {
-        if (cudaFuncSetAttribute(hop_long_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
-                cudaSuccess ||
-            cudaFuncSetAttribute(hop_long_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
-                cudaSuccess)
+        const auto dyn = cudaFuncAttributeMaxDynamicSharedMemorySize;
+        const auto carve = cudaFuncAttributePreferredSharedMemoryCarveout;
+        if (cudaFuncSetAttribute(hop_long_kernel<D, false, false>, dyn, (int)smem) != cudaSuccess ||
+            cudaFuncSetAttribute(hop_long_kernel<D, true, false>, dyn, (int)smem) != cudaSuccess ||
+            cudaFuncSetAttribute(hop_long_kernel<D, false, true>, dyn, (int)smem_solo) != cudaSuccess ||
+            cudaFuncSetAttribute(hop_long_kernel<D, true, true>, dyn, (int)smem_solo) != cudaSuccess ||
+            cudaFuncSetAttribute(hop_long_kernel<D, false, true>, carve, 100) != cudaSuccess ||
+            cudaFuncSetAttribute(hop_long_kernel<D, true, true>, carve, 100) != cudaSuccess)
             return TA_ERR_CUDA;
         configured.mark(dev);
     }
-    const unsigned grid = (unsigned)(a.total_items < num_sms ? a.total_items : num_sms);
-    if (a.window > 0 || a.lens != nullptr || a.mask_bits != nullptr)
-        return launch_kernel(hop_long_kernel<D, true>, grid, kThreads, smem, pb.stream, false, mq, mk, mxi,
+    const bool windowed = a.window > 0 || a.lens != nullptr || a.mask_bits != nullptr;
+    if (solo) {
+        // two CTAs per SM
+        const unsigned grid = (unsigned)(a.total_items < 2LL * num_sms ? a.total_items : 2LL * num_sms);
+        if (windowed)
+            return launch_kernel(hop_long_kernel<D, true, true>, grid, kSoloThreads, smem_solo, pb.stream, false, mq, mk,
+                                 mxi, mo, (__nv_bfloat16 *)xout, a);
+        return launch_kernel(hop_long_kernel<D, false, true>, grid, kSoloThreads, smem_solo, pb.stream, false, mq, mk, mxi, mo,
                              (__nv_bfloat16 *)xout, a);
-    return launch_kernel(hop_long_kernel<D, false>, grid, kThreads, smem, pb.stream, false, mq, mk, mxi,
+    }
+    const unsigned grid = (unsigned)(a.total_items < num_sms ? a.total_items : num_sms);
+    if (windowed)
+        return launch_kernel(hop_long_kernel<D, true, false>, grid, kThreads, smem, pb.stream, false, mq, mk, mxi, mo,
+                             (__nv_bfloat16 *)xout, a);
+    return launch_kernel(hop_long_kernel<D, false, false>, grid, kThreads, smem, pb.stream, false, mq, mk, mxi, mo,
                          (__nv_bfloat16 *)xout, a);
 }
 
@@ -722,6 +864,8 @@ int rope_unrotate_add(const Problem &pb, const HopDesc &hd, const float *src, fl
     return launch_kernel(rope_unrotate_add_kernel, rope_blocks(pairs), 256, 0, pb.stream, false, src, dst, pairs, pb.N,
                          pb.D, (long long)hd.stride, hd.n, log2((double)pb.rope_base), accumulate ? 1 : 0);
 }
+
+int long_tiles_per_item(int n) { return n <= solo_max_n() ? 1 : 2; }
 
 int launch_hop_tc_long(const Problem &pb, const HopDesc &hd, const void *xin, int xin_heads, void *xout) {
     if (xin == xout) return TA_ERR_INVALID_ARG;

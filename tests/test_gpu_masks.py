@@ -161,6 +161,8 @@ def lambda_mask(n, sinks, local):
     ([1024], 128, True, "band"),              # banded: leading key blocks of a query block are skipped
     ([3, 200], 128, True, "random"),          # short (kernel-parameter mask) and long (bit matrix) hop
     ([260, 2], 64, False, "block"),           # long hop over a strided dimension
+    ([1280], 64, True, "block"),              # pairs of query tiles (n > 1 024)
+    ([1100], 64, False, "lambda"),
 ])
 def test_masks_on_long_segments(dims, D, causal, kind):
     """Explicit masks on dimensions longer than 128: bit matrix in device memory, tensor-core forward."""

@@ -79,9 +79,16 @@ def test_mixed_paths_use_scratch():
     ([130, 3], 64, True, 2, 1),        # long hop over a strided dimension
     ([3, 129], 128, False, 2, 2),
     ([1000], 64, True, 2, 2),          # eight key blocks: running maximum moves many times
+    ([181, 2], 128, True, 4, 1),       # two ragged query tiles per segment, strided, one item per tile
+    ([2, 513], 64, False, 2, 2),       # five tiles, one position in the last
+    ([1300], 64, True, 2, 1),          # past the one-tile-per-item range: pairs of query tiles, ragged
+    ([1100, 2], 128, False, 2, 2),     # the same, strided and not causal
 ])
 def test_long_segments_tensor_core(dims, D, causal, H, Hkv):
-    assert "tc-long" in ta.ta_plan_describe(1, H, Hkv, math.prod(dims), D, dims, causal, ta.TA_DTYPE_BF16, 0)
+    plan = ta.ta_plan_describe(1, H, Hkv, math.prod(dims), D, dims, causal, ta.TA_DTYPE_BF16, 0)
+    assert "tc-long" in plan
+    # segments of up to 1 024 positions: one query tile per work item (two CTAs per SM); longer: pairs
+    assert ("tiles_per_item=1" if max(dims) <= 1024 else "tiles_per_item=2") in plan
     check_case(2, H, Hkv, math.prod(dims), D, dims, causal, "bf16", seed=113)
 
 

@@ -85,6 +85,8 @@ def test_lengths_generic_kernel_and_long_segments():
     ([700], 64, False, [1, 0]),                   # one token; an empty batch entry
     ([3, 260], 128, False, [400, 780]),
     ([1024], 128, True, [1000, 130]),
+    ([1400], 64, True, [1399, 200]),              # pairs of query tiles (n > 1 024)
+    ([1150], 128, False, [640, 1150]),
 ])
 def test_lengths_long_segments_tensor_core(dims, D, causal, lens):
     B, H, Hkv = 2, 4, 2

@@ -57,6 +57,8 @@ def test_window_fused_hops(dims, window, D, causal):
     ([2, 384], [0, 130], 128, True),
     ([300], [5], 64, True),             # rows that see nothing in the first block they visit
     ([130, 3], [129, 2], 64, False),
+    ([1300], [150], 64, True),          # pairs of query tiles (n > 1 024): blocks before the window skipped
+    ([1200], [300], 128, False),
 ])
 def test_window_long_segments(dims, window, D, causal):
     run(2, 4, 2, D, dims, window, causal, "bf16", 603, expect="tc-long")
