@@ -516,8 +516,25 @@ hop_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                         if (32 * cc + 32 <= c_hi) my_full |= 1u << cc;
                 }
                 const uint32_t full_bits = kWindow ? 0u : __reduce_and_sync(0xffffffffu, my_full);
+                // (with two chains per CTA a block every row sees completely -- most blocks of a long
+                // segment -- has loops of its own: measured 11 % faster there, and 9 % slower with one)
+                const bool full_w = !kSolo && full_bits == 0xFu;
                 float bm = -INFINITY;
                 uint32_t v[32];
+                if (full_w) {
+#pragma unroll 1
+                    for (int cc = 0; cc < 4; ++cc) {
+                        tmem_ld32(s_col + 32 * cc, v);
+                        float b0 = fmaxf(__uint_as_float(v[0]), __uint_as_float(v[1]));
+                        float b1 = fmaxf(__uint_as_float(v[2]), __uint_as_float(v[3]));
+#pragma unroll
+                        for (int jj = 4; jj < 32; jj += 4) {
+                            b0 = fmaxf(b0, fmaxf(__uint_as_float(v[jj]), __uint_as_float(v[jj + 1])));
+                            b1 = fmaxf(b1, fmaxf(__uint_as_float(v[jj + 2]), __uint_as_float(v[jj + 3])));
+                        }
+                        bm = fmaxf(bm, fmaxf(b0, b1));
+                    }
+                } else
 #pragma unroll 1
                 for (int cc = 0; cc < nchunks; ++cc) {
                     if (32 * cc >= w_hi) continue;          // warp-uniform
@@ -566,6 +583,22 @@ hop_long_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 // (over a chunk without masks the row sum is taken over the fp32 weights: the rounding of
                 // P averages out; elsewhere over the rounded weights)
                 float sum = 0.f, sum1 = 0.f;
+                if (full_w) {
+#pragma unroll 1
+                    for (int cc = 0; cc < 4; ++cc) {
+                        uint32_t pk[16];
+                        tmem_ld32(s_col + 32 * cc, v);
+#pragma unroll
+                        for (int jj = 0; jj < 32; jj += 2) {
+                            const float p0 = fast_exp2(fmaf(__uint_as_float(v[jj]), a.scale_log2, -m_ref));
+                            const float p1 = fast_exp2(fmaf(__uint_as_float(v[jj + 1]), a.scale_log2, -m_ref));
+                            pk[jj >> 1] = pack_bf16x2(p0, p1);
+                            sum += p0;
+                            sum1 += p1;
+                        }
+                        tmem_st16(s_col + 16 * cc, pk);
+                    }
+                } else
 #pragma unroll 1
                 for (int cc = 0; cc < nchunks; ++cc) {
                     uint32_t pk[16];
