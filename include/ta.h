@@ -72,7 +72,8 @@ enum {
 
 /* flags of ta_params.flags */
 enum {
-    TA_FLAG_NO_TENSOR_CORE = 1u << 0, /* run every hop on the generic CUDA-core kernel        */
+    TA_FLAG_NO_TENSOR_CORE = 1u << 0, /* run every hop on the generic CUDA-core kernel (and a  */
+                                      /* head dim other than 64 / 128 on the tensors as they are) */
     TA_FLAG_NO_HOP_FUSION = 1u << 1,  /* one launch per hop: trailing hops that together fit one  */
                                       /* 128-row tile are not fused into one pass (and            */
                                       /* TA_FLAG_PAIR_HOPS is ignored)                            */
@@ -114,10 +115,18 @@ enum { TA_WS_FORWARD = 0, TA_WS_FORWARD_SAVE = 1, TA_WS_BACKWARD = 2, TA_WS_BACK
  * Scale is 1/sqrt(D) in every hop (Eq. 4).
  * Hops with D in {64,128} and n_i <= 128 run on the tensor-core kernel in place in `out` and
  * need no other memory.  Hops with n_i > 128 (key-block loop with online softmax on the tensor
- * cores, D in {64,128}) and hops with another D (generic CUDA-core kernel) cannot update in
- * place: for them the library takes a scratch buffer of B*H*N*D elements from its memory pool
- * for the duration of the call (stream-ordered, see above).  ta_forward_ex takes a caller
- * workspace instead.
+ * cores, D in {64,128}) cannot update in place: for them the library takes a scratch buffer of
+ * B*H*N*D elements from its memory pool for the duration of the call (stream-ordered, see
+ * above).  ta_forward_ex takes a caller workspace instead.
+ * Other head dims below 128 (100, 96, 80, 40, odd ones ...): the same tensor-core kernels run on
+ * zero-padded copies of q, k, v with 64 or 128 columns, and the result is copied back without the
+ * padding (zero columns add nothing to Q K^T and give zero output columns; the scale stays
+ * 1/sqrt(D); the positional encoding keeps its pairs c, c + D/2 and its frequencies).  The copies
+ * -- about 2.3 x (2 H + 2 H_kv) / H times the value tensor -- and the padded problem's scratch
+ * come from the memory pool whether or not the caller passed a workspace; hop inputs saved with
+ * TA_FLAG_SAVE_HOPS arrive in the caller's workspace in the caller's layout; the backward does the
+ * same with dout and the gradients and recomputes the hop inputs.  With TA_FLAG_NO_TENSOR_CORE,
+ * for D > 128 and for fp32 tensors the generic CUDA-core kernels run on the tensors as they are.
  * With TA_FLAG_PAIR_HOPS (ta_forward_ex), two adjacent hops with D in {64,128} and n_i <= 128
  * whose common block (n_i * n_{i+1} * s_{i+1} tokens) is too large for one SM but small against
  * the L2 cache run as ONE cooperative launch in which the second hop's tiles follow the first
@@ -304,7 +313,9 @@ int ta_forward_host(const void *q_host, const void *k_host, const void *v_host, 
  * latency-critical serving loop (cudaMalloc synchronises the device), processes whose device
  * memory is entirely managed by a pool the library cannot reach, and plug-ins that are only
  * permitted to launch kernels.  Same arguments and result as ta_forward_ex with default
- * options (dtype = TA_DTYPE_*), but the second value buffer that hops which cannot update in
+ * options (dtype = TA_DTYPE_*; for bf16 head dims other than 64 and 128, which ta_forward_ex
+ * pads in buffers from its pool, the result of TA_FLAG_NO_TENSOR_CORE: the generic kernels on the
+ * tensors as they are), but the second value buffer that hops which cannot update in
  * place need (fp32 storage, n_i > 128, head dims other than 64 / 128) comes from a fixed array of
  * TA_STATIC_SCRATCH_BYTES that is part of the loaded module -- every GPU that loads the
  * library holds those bytes until the process exits.  The call makes no cudaMalloc / cudaFree

@@ -12,7 +12,7 @@ ROOT = os.path.dirname(os.path.dirname(HERE))
 LIB = os.path.join(os.path.dirname(HERE), "libta_b200.so")
 OBJ_DIR = os.path.join(HERE, "_build")
 SOURCES = ["ta_api.cu", "ta_simt.cu", "ta_tc.cu", "ta_tc_fused.cu", "ta_tc_pair.cu", "ta_tc_long.cu", "ta_tc_bwd.cu",
-           "ta_tc_bwd_long.cu", "ta_simt_bwd.cu", "ta_backward.cu", "ta_noalloc.cu", "ta_selftest.cu"]
+           "ta_tc_bwd_long.cu", "ta_simt_bwd.cu", "ta_backward.cu", "ta_noalloc.cu", "ta_selftest.cu", "ta_pad.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", HERE]
 

@@ -456,8 +456,77 @@ static bool overlaps(const void *a, size_t a_bytes, const void *b, size_t b_byte
     return a0 < b0 + b_bytes && b0 < a0 + a_bytes;
 }
 
+static int forward_impl(const ta_params &p);
+
+// A bf16 problem whose head dim has no tensor-core kernel, run on zero-padded copies (ta_pad.cu).
+// Everything lives in one stream-ordered allocation: [q'][k'][v'][out'][workspace of the padded call].
+// With TA_FLAG_SAVE_HOPS the saved hop inputs are copied back, unpadded, into the caller's workspace.
+static int forward_padded(const ta_params &p) {
+    const int DP = padded_dim(p.D);
+    Plan plan_u, plan_p;
+    int rc = build_plan(p.B, p.H, p.H_kv, p.N, p.D, p.dims, p.ndims, p.dtype, p.flags, p.hop_begin, p.hop_end, &plan_u);
+    if (rc != TA_OK) return rc;
+    if (!aligned16(p.q) || !aligned16(p.k) || !aligned16(p.v) || !aligned16(p.out)) return TA_ERR_ALIGNMENT;
+    if (p.workspace && (reinterpret_cast<uintptr_t>(p.workspace) & 255u)) return TA_ERR_ALIGNMENT;
+    const size_t tq = (size_t)p.B * p.H * p.N, tkv = (size_t)p.B * p.H_kv * p.N;     // rows
+    const size_t tensor_u = tq * p.D * 2, kv_u = tkv * p.D * 2;
+    if ((p.flags & TA_FLAG_SAVE_HOPS) && plan_u.save_bytes && !p.workspace) return TA_ERR_WORKSPACE;
+    if (p.workspace && p.workspace_bytes < plan_u.scratch_bytes + plan_u.save_bytes + plan_u.flag_bytes)
+        return TA_ERR_WORKSPACE;
+    if (overlaps(p.out, tensor_u, p.q, tensor_u) || overlaps(p.out, tensor_u, p.k, kv_u) ||
+        overlaps(p.out, tensor_u, p.v, kv_u))
+        return TA_ERR_INVALID_ARG;
+    // (the plan the padded call will build: same flags as forward_impl derives)
+    bool any_mask = false;
+    if (p.hop_masks)
+        for (int i = 0; i < p.ndims; ++i) any_mask = any_mask || p.hop_masks[i] != nullptr;
+    const unsigned fusion_off = (p.rope_base > 0.f || p.seq_lens || any_mask) ? (unsigned)TA_FLAG_NO_HOP_FUSION : 0u;
+    rc = build_plan(p.B, p.H, p.H_kv, p.N, DP, p.dims, p.ndims, p.dtype, p.flags | fusion_off, p.hop_begin, p.hop_end,
+                    &plan_p);
+    if (rc != TA_OK) return rc;
+    auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
+    const size_t q_bytes = up(tq * DP * 2), kv_bytes = up(tkv * DP * 2);
+    const size_t ws_bytes = plan_p.scratch_bytes + plan_p.save_bytes + plan_p.flag_bytes;
+    cudaStream_t stream = (cudaStream_t)p.stream;
+    void *pooled = nullptr;
+    if ((rc = pool_alloc(2 * q_bytes + 2 * kv_bytes + ws_bytes, stream, &pooled)) != TA_OK) return rc;
+    PooledGuard guard{pooled, stream};
+    char *qp = (char *)pooled, *kp = qp + q_bytes, *vp = kp + kv_bytes, *outp = vp + kv_bytes, *wsp = outp + q_bytes;
+    if ((rc = launch_pad_rows(p.q, qp, (long long)tq, p.D, DP, 2, stream)) != TA_OK) return rc;
+    if ((rc = launch_pad_rows(p.k, kp, (long long)tkv, p.D, DP, 2, stream)) != TA_OK) return rc;
+    if ((rc = launch_pad_rows(p.v, vp, (long long)tkv, p.D, DP, 2, stream)) != TA_OK) return rc;
+    // a call that starts after the first hop reads its value tensor from `out`
+    if (p.hop_begin > 0 && (rc = launch_pad_rows(p.out, outp, (long long)tq, p.D, DP, 2, stream)) != TA_OK) return rc;
+    ta_params p2 = p;
+    p2.q = qp; p2.k = kp; p2.v = vp; p2.out = outp;
+    p2.D = DP;
+    p2.softmax_scale = p.softmax_scale != 0.f ? p.softmax_scale : 1.0f / sqrtf((float)p.D);
+    if (p.rope_base > 0.f) p2.rope_base = padded_rope_base(p.rope_base, p.D, DP);
+    p2.workspace = ws_bytes ? wsp : nullptr;
+    p2.workspace_bytes = ws_bytes;
+    if ((rc = forward_impl(p2)) != TA_OK) return rc;
+    if ((rc = launch_unpad_rows(outp, p.out, (long long)tq, p.D, DP, 2, stream)) != TA_OK) return rc;
+    if (p.flags & TA_FLAG_SAVE_HOPS) {
+        const size_t slots = plan_p.save_bytes / (tq * DP * 2);
+        for (size_t i = 0; i < slots; ++i) {
+            rc = launch_unpad_rows(wsp + plan_p.scratch_bytes + i * tq * DP * 2,
+                                   (char *)p.workspace + plan_u.scratch_bytes + i * tensor_u, (long long)tq, p.D, DP, 2,
+                                   stream);
+            if (rc != TA_OK) return rc;
+        }
+    }
+    return TA_OK;
+}
+
 static int forward_impl(const ta_params &p) {
     if (!p.q || !p.k || !p.v || !p.out) return TA_ERR_INVALID_ARG;
+    if (pad_eligible(p.D, p.dtype, p.flags) && p.ndims >= 1 && p.ndims <= TA_MAX_DIMS &&
+        !(p.rope_base > 0.f && ((p.D & 1) || padded_rope_base(p.rope_base, p.D, padded_dim(p.D)) == 0.f))) {
+        bool hops = false;
+        const int he = (p.hop_begin == 0 && p.hop_end == 0) ? p.ndims : p.hop_end;
+        for (int i = p.hop_begin; i >= 0 && i < he && i < p.ndims; ++i) hops = hops || p.dims[i] > 1;
+        if (hops) return forward_padded(p);
+    }
     if (p.rope_base < 0.f || !(p.rope_base == p.rope_base)) return TA_ERR_INVALID_ARG;
     if (p.rope_base > 0.f && (p.D & 1)) return TA_ERR_UNSUPPORTED;
     if (p.window && p.ndims >= 1 && p.ndims <= TA_MAX_DIMS)
@@ -701,7 +770,11 @@ int ta_plan_describe(int B, int H, int H_kv, int N, int D, const int *dims, int 
     buf[0] = 0;
     Plan plan;
     if (flags & kPlanAllowPairs) return TA_ERR_UNSUPPORTED;
-    int rc = build_plan(B, H, H_kv, N, D, dims, ndims, dtype, flags, 0, 0, &plan);
+    // (a head dim without a tensor-core kernel: the plan of the zero-padded problem that will run)
+    int rc = validate_shape(B, H, H_kv, N, D, dims, ndims, dtype);
+    if (rc != TA_OK) return rc;
+    const int D_run = pad_eligible(D, dtype, flags) ? padded_dim(D) : D;
+    rc = build_plan(B, H, H_kv, N, D_run, dims, ndims, dtype, flags, 0, 0, &plan);
     if (rc != TA_OK) return rc;
     size_t off = 0;
     auto emit = [&](const char *fmt, auto... a) {
@@ -709,8 +782,10 @@ int ta_plan_describe(int B, int H, int H_kv, int N, int D, const int *dims, int 
         int w = snprintf(buf + off, cap - off, fmt, a...);
         if (w > 0) off += (size_t)w;
     };
-    emit("hops=%d causal=%d dtype=%s scratch_bytes=%zu save_bytes=%zu\n", plan.nhops, causal ? 1 : 0,
+    emit("hops=%d causal=%d dtype=%s scratch_bytes=%zu save_bytes=%zu", plan.nhops, causal ? 1 : 0,
          dtype == TA_DTYPE_F32 ? "f32" : "bf16", plan.scratch_bytes, plan.save_bytes);
+    if (D_run != D) emit(" padded_head_dim=%d", D_run);
+    emit("%s", "\n");
     for (int j = 0; j < plan.nhops; ++j) {
         const HopDesc &h = plan.hops[j];
         if (h.path == PATH_TC && h.nf > 1) {

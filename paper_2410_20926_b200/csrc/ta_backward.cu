@@ -58,8 +58,62 @@ size_t backward_workspace_bytes(int B, int H, int H_kv, int N, int D, const int 
                   dtype == TA_DTYPE_F32 ? 4 : 2).total;
 }
 
+int backward_impl(const ta_bwd_params &p);
+
+namespace {
+// A bf16 problem whose head dim has no tensor-core kernel: the backward of the zero-padded problem
+// (ta_pad.cu), whose gradients in the padding columns are dropped.  One stream-ordered allocation holds
+// [dout'][q'][k'][v'][dq'][dk'][dv'][workspace]; the hop inputs are recomputed there (saved ones are in
+// the caller's layout and are not used).
+int backward_padded(const ta_bwd_params &p) {
+    const int DP = padded_dim(p.D);
+    if (p.grad_dtype != TA_DTYPE_BF16 && p.grad_dtype != TA_DTYPE_F32) return TA_ERR_UNSUPPORTED;
+    int rc = validate_shape(p.B, p.H, p.H_kv, p.N, p.D, p.dims, p.ndims, p.dtype);
+    if (rc != TA_OK) return rc;
+    auto misaligned = [](const void *x) { return (reinterpret_cast<uintptr_t>(x) & 15u) != 0; };
+    if (misaligned(p.dout) || misaligned(p.q) || misaligned(p.k) || misaligned(p.v) || misaligned(p.dq) ||
+        misaligned(p.dk) || misaligned(p.dv))
+        return TA_ERR_ALIGNMENT;
+    const size_t gelem = p.grad_dtype == TA_DTYPE_F32 ? 4 : 2;
+    const size_t tq = (size_t)p.B * p.H * p.N, tkv = (size_t)p.B * p.H_kv * p.N;     // rows
+    const size_t q_bytes = up256(tq * DP * 2), kv_bytes = up256(tkv * DP * 2);
+    const size_t gq_bytes = up256(tq * DP * gelem), gkv_bytes = up256(tkv * DP * gelem);
+    const size_t ws_bytes = backward_workspace_bytes(p.B, p.H, p.H_kv, p.N, DP, p.dims, p.ndims, p.dtype, p.grad_dtype, false);
+    cudaStream_t stream = (cudaStream_t)p.stream;
+    PooledGuard guard{nullptr, stream};
+    if ((rc = pool_alloc(2 * q_bytes + 2 * kv_bytes + gq_bytes + 2 * gkv_bytes + up256(ws_bytes), stream, &guard.ptr)) != TA_OK)
+        return rc;
+    char *gp = (char *)guard.ptr, *qp = gp + q_bytes, *kp = qp + q_bytes, *vp = kp + kv_bytes, *dqp = vp + kv_bytes,
+         *dkp = dqp + gq_bytes, *dvp = dkp + gkv_bytes, *wsp = dvp + gkv_bytes;
+    if ((rc = launch_pad_rows(p.dout, gp, (long long)tq, p.D, DP, 2, stream)) != TA_OK) return rc;
+    if ((rc = launch_pad_rows(p.q, qp, (long long)tq, p.D, DP, 2, stream)) != TA_OK) return rc;
+    if ((rc = launch_pad_rows(p.k, kp, (long long)tkv, p.D, DP, 2, stream)) != TA_OK) return rc;
+    if ((rc = launch_pad_rows(p.v, vp, (long long)tkv, p.D, DP, 2, stream)) != TA_OK) return rc;
+    ta_bwd_params p2 = p;
+    p2.dout = gp; p2.q = qp; p2.k = kp; p2.v = vp;
+    p2.dq = dqp; p2.dk = dkp; p2.dv = dvp;
+    p2.D = DP;
+    p2.softmax_scale = p.softmax_scale != 0.f ? p.softmax_scale : 1.0f / sqrtf((float)p.D);
+    if (p.rope_base > 0.f) p2.rope_base = padded_rope_base(p.rope_base, p.D, DP);
+    p2.saved_hops = nullptr;
+    p2.workspace = ws_bytes ? wsp : nullptr;
+    p2.workspace_bytes = ws_bytes;
+    if ((rc = backward_impl(p2)) != TA_OK) return rc;
+    if ((rc = launch_unpad_rows(dqp, p.dq, (long long)tq, p.D, DP, (int)gelem, stream)) != TA_OK) return rc;
+    if ((rc = launch_unpad_rows(dkp, p.dk, (long long)tkv, p.D, DP, (int)gelem, stream)) != TA_OK) return rc;
+    return launch_unpad_rows(dvp, p.dv, (long long)tkv, p.D, DP, (int)gelem, stream);
+}
+}  // namespace
+
 int backward_impl(const ta_bwd_params &p) {
     if (!p.dout || !p.q || !p.k || !p.v || !p.dq || !p.dk || !p.dv) return TA_ERR_INVALID_ARG;
+    if (pad_eligible(p.D, p.dtype, 0) && p.ndims >= 1 && p.ndims <= TA_MAX_DIMS && !(p.rope_base < 0.f) &&
+        p.rope_base == p.rope_base &&
+        !(p.rope_base > 0.f && ((p.D & 1) || padded_rope_base(p.rope_base, p.D, padded_dim(p.D)) == 0.f))) {
+        bool hops = false;
+        for (int i = 0; i < p.ndims; ++i) hops = hops || p.dims[i] > 1;
+        if (hops) return backward_padded(p);
+    }
     if (p.dtype != TA_DTYPE_BF16 && p.dtype != TA_DTYPE_F32) return TA_ERR_UNSUPPORTED;
     if (p.grad_dtype != TA_DTYPE_BF16 && p.grad_dtype != TA_DTYPE_F32) return TA_ERR_UNSUPPORTED;
     if (p.dtype == TA_DTYPE_F32 && p.grad_dtype != TA_DTYPE_F32) return TA_ERR_UNSUPPORTED;   // fp32 in, fp32 gradients

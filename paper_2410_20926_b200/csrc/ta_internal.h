@@ -187,6 +187,15 @@ int launch_hop_tc_bwd_long(const Problem &pb, const HopDesc &hd, const void *x, 
                            void *g_out, float *dq_acc, float *dk_acc, float *dv_acc, void *stats, bool first_hop,
                            bool accumulate);
 int launch_f32_to_bf16(const float *src, void *dst, long long n, cudaStream_t stream);
+// Head dims without a tensor-core kernel (ta_pad.cu): bf16 problems with D < 128, D != 64 run on
+// zero-padded copies of D' = padded_dim(D) columns (first half of the features at column 0, second
+// half at D' / 2), unless TA_FLAG_NO_TENSOR_CORE asks for the generic kernels.  elem: bytes per element.
+bool pad_eligible(int D, int dtype, unsigned flags);
+int padded_dim(int D);
+int launch_pad_rows(const void *src, void *dst, long long rows, int D, int DP, int elem, cudaStream_t stream);
+int launch_unpad_rows(const void *src, void *dst, long long rows, int D, int DP, int elem, cudaStream_t stream);
+// base' with base'^(-2c / D') = base^(-2c / D); 0 when it leaves the float range
+float padded_rope_base(float base, int D, int DP);
 int launch_group_sum(const void *dout, int dout_is_f32, void *dv, int dv_is_f32, int B, int H, int H_kv,
                      long long per_head, cudaStream_t stream);
 

@@ -134,8 +134,15 @@ def test_plan_skips_unit_dims_and_routes_generic_hops():
     assert [h["hop"] for h in hops] == ["0", "2"]
     head, hops = parse_plan(ta.ta_plan_describe(1, 2, 2, 256, 64, [1, 1, 1, 256], False))
     assert [h["path"] for h in hops] == ["tc-long"]                    # n > 128: key-block loop
+    # a bf16 head dim the tensor-core kernels lack runs on zero-padded copies, unless told otherwise
     head, hops = parse_plan(ta.ta_plan_describe(1, 2, 2, 256, 96, [1, 1, 1, 256], False))
-    assert [h["path"] for h in hops] == ["simt"]                       # head dim the tensor-core kernels lack
+    assert [h["path"] for h in hops] == ["tc-long"] and head["padded_head_dim"] == "128"
+    head, hops = parse_plan(ta.ta_plan_describe(1, 2, 2, 256, 40, [16, 16], False))
+    assert [h["path"] for h in hops] == ["tc", "tc"] and head["padded_head_dim"] == "64"
+    head, hops = parse_plan(ta.ta_plan_describe(1, 2, 2, 256, 96, [1, 1, 1, 256], False, flags=ta.TA_FLAG_NO_TENSOR_CORE))
+    assert [h["path"] for h in hops] == ["simt"] and "padded_head_dim" not in head
+    head, hops = parse_plan(ta.ta_plan_describe(1, 2, 2, 256, 96, [1, 1, 1, 256], False, dtype=ta.TA_DTYPE_F32))
+    assert [h["path"] for h in hops] == ["simt"] and "padded_head_dim" not in head
     head, hops = parse_plan(ta.ta_plan_describe(1, 2, 2, 16384, 64, [4, 4096], False))
     assert [(h["path"], h["src"], h["dst"]) for h in hops] == \
         [("tc", "v", "scratch"), ("tc-long", "scratch", "out")]        # the long hop is not in place
