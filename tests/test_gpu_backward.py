@@ -124,6 +124,22 @@ def test_backward_with_positional_encoding(dims, D, causal, B, H, Hkv, grad_f32)
         assert_grad_close(g, r, name, grad_f32, hops_of(dims), rope=True)
 
 
+@pytest.mark.parametrize("n,growth", [(600, 1.0), (1300, 0.4)])
+def test_backward_long_segments_running_maximum_jumps(n, growth):
+    """Keys that grow from key block to key block: the statistics pass of the long-segment backward
+    (log-sum-exp per row) is taken over row maxima that move at almost every block."""
+    from paper_2410_20926_b200.inputs import bf16_bits, bf16_to_f32
+    B, H, Hkv, D = 1, 2, 1, 64
+    inp = ta_inputs.make_inputs(B, H, Hkv, n, D, "bf16", 310, with_dout=True)
+    factor = (1.0 + growth * (np.arange(n) // 128)).astype(np.float32)
+    bits = bf16_bits(inp["k"] * factor[None, None, :, None])
+    inp["k"], inp["k_bits"] = bf16_to_f32(bits), bits
+    got = gpu_backward(inp, B, H, Hkv, n, D, [n], False, True)
+    ref = oracle.backward(inp["dout"], inp["q"], inp["k"], inp["v"], [n], False)
+    for name, g, r in zip(("dq", "dk", "dv"), got, ref):
+        assert_grad_close(g, r, name, True, 1)
+
+
 def test_backward_all_unit_dims():
     inp = ta_inputs.make_inputs(2, 4, 2, 1, 64, "bf16", 302, with_dout=True)
     dq, dk, dv = gpu_backward(inp, 2, 4, 2, 1, 64, [1, 1], True, True)

@@ -92,6 +92,26 @@ def test_long_segments_tensor_core(dims, D, causal, H, Hkv):
     check_case(2, H, Hkv, math.prod(dims), D, dims, causal, "bf16", seed=113)
 
 
+@pytest.mark.parametrize("n,growth", [(1000, 3.0), (1300, 3.0), (1024, 0.4), (640, -0.12)])
+def test_long_segments_running_maximum_jumps(n, growth):
+    """Keys whose size changes from key block to key block: with growth 3 the row maxima jump by many
+    units (log2 domain) at most blocks, with 0.4 by a few, with a negative growth they never rise after
+    the first block.  The kernel rescales the accumulated output whenever a row's maximum moved; all
+    three regimes must give the oracle's rows (one query tile per item up to 1 024 positions, pairs of
+    tiles beyond)."""
+    from paper_2410_20926_b200.inputs import bf16_bits, bf16_to_f32
+    B, H, Hkv, D = 1, 2, 1, 64
+    inp = ta_inputs.make_inputs(B, H, Hkv, n, D, "bf16", 117)
+    factor = (1.0 + growth * (np.arange(n) // 128)).astype(np.float32)
+    bits = bf16_bits(inp["k"] * factor[None, None, :, None])
+    inp["k"], inp["k_bits"] = bf16_to_f32(bits), bits
+    got = gpu_forward(inp, B, H, Hkv, n, D, [n], False, "bf16")
+    ref = oracle.forward(inp["q"], inp["k"], inp["v"], [n], False)
+    assert_close(got, ref, "bf16", 1)
+    got = gpu_forward(inp, B, H, Hkv, n, D, [n], True, "bf16")
+    assert_close(got, oracle.forward(inp["q"], inp["k"], inp["v"], [n], True), "bf16", 1)
+
+
 def test_full_attention_4096_sampled_heads():
     """One dimension = ordinary attention (Eq. 1) at a length where the loop runs 32 key blocks."""
     check_case(1, 8, 2, 4096, 128, [4096], True, "bf16", seed=114, heads=[(0, 0), (0, 5)])
